@@ -1,0 +1,183 @@
+/*
+ * lacache.h -- C ABI of the B200 (sm_100a) first-layer cached attention path.
+ *
+ * The path is the first-layer bidirectional attention of a block-wise
+ * (semi-autoregressive) diffusion-LLM denoising step with the paper's
+ * RoPECache (Sec. 3.3.2, Eq. 1) and FACache (Sec. 3.3.3, Eq. 2-6,
+ * Algorithm 1).  Within one block only the tokens of the current block C
+ * change; all other tokens U (prompt, earlier blocks, masked suffix) are fixed
+ * (Sec. 3.3.1).  `lacache_build` is the cache-filling side of Algorithm 1
+ * (GenStep = True): it rotates and stores Q/K/V for every token and stores, for
+ * every fixed query, the online-softmax state (m, l, O~) over the fixed keys.
+ * `lacache_step` is the reuse pass (GenStep = False): only the block's fresh
+ * Q/K/V are rotated, fixed queries attend to the block's keys only and merge
+ * the result into their cached state, block queries attend to all keys, and
+ * the normalised output O = diag(l)^-1 O~ is written for all positions.
+ *
+ * General conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller unless the
+ *     name says `host`.  Tensors are contiguous, 16-byte aligned, token-major
+ *     and packed over the batch: q [T, Hq, d], k/v [T, Hkv, d], out
+ *     [T, Hq, d], lse [T, Hq]; T = sum_b (prompt_lens[b] + gen_len).  Block
+ *     tensors are sequence-major: row b * block_len + r is token r of
+ *     sequence b's current block.
+ *   - Q/K/V element type is `dtype` (bf16 or fp32).  `out` is always fp32,
+ *     `lse` fp32 in natural-log units (L = m + log l, Algorithm 1).
+ *   - Query head h reads KV head h / (Hq / Hkv).  Positions are 0-based
+ *     inside each sequence.  RoPE pairs feature c with c + d/2 and uses
+ *     frequency theta^(-2c/d); V is not rotated.
+ *   - Calls validate on the host, enqueue work on `cuda_stream` (a
+ *     cudaStream_t passed as void*, NULL = default stream) and return without
+ *     synchronising.  They never throw, abort or print.  The context owns all
+ *     caches and scratch; caller tensors are neither retained nor freed.
+ *   - There is no CPU fallback: without a CUDA device every call that would
+ *     compute returns LACACHE_ERR_CUDA.
+ *   - A context is not thread-safe; use one per host thread / stream.
+ */
+#ifndef LACACHE_H_
+#define LACACHE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lacache_ctx lacache_ctx;
+
+typedef enum {
+  LACACHE_OK = 0,
+  LACACHE_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, index out of range */
+  LACACHE_ERR_SHAPE = 2,       /* inconsistent sizes in the config */
+  LACACHE_ERR_STATE = 3,       /* step before build, etc. */
+  LACACHE_ERR_UNSUPPORTED = 4, /* head_dim / dtype / mode not implemented */
+  LACACHE_ERR_OOM = 5,
+  LACACHE_ERR_CUDA = 6,        /* a CUDA runtime call failed; see lacache_last_error */
+  LACACHE_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out */
+} lacache_status;
+
+enum { LACACHE_DTYPE_BF16 = 0, LACACHE_DTYPE_FP32 = 1 };
+/* which kernel family runs the attention: AUTO picks tcgen05 for bf16 with
+ * head_dim 128 and the fp32 CUDA-core kernels otherwise */
+enum { LACACHE_ENGINE_AUTO = 0, LACACHE_ENGINE_SIMT = 1, LACACHE_ENGINE_TCGEN05 = 2 };
+
+typedef struct {
+  int dtype;          /* LACACHE_DTYPE_*: element type of q/k/v inputs */
+  int engine;         /* LACACHE_ENGINE_* */
+  int n_q_heads;      /* Hq */
+  int n_kv_heads;     /* Hkv, divides Hq */
+  int head_dim;       /* d: 64 or 128 */
+  float rope_theta;
+  float softmax_scale;        /* <= 0 means 1/sqrt(head_dim) */
+  int batch;                  /* B >= 1 */
+  const int32_t* prompt_lens; /* HOST pointer, B entries, each >= 0; copied */
+  int gen_len;                /* G > 0, the same for every sequence */
+  int block_len;              /* L_b > 0, divides G */
+  int sc_tiles_per_chunk;     /* key tiles (64 keys) per block-query work item; 0 = auto */
+} lacache_config;
+
+/* Library version, e.g. 100 = 1.0.0.  No paper counterpart. */
+int lacache_version(void);
+
+/*
+ * Create a context: validates the config, derives the integer metadata
+ * (Sec. 3.3.1 index sets U and C per block; per-token sequence id and
+ * position), builds the RoPE cos/sin table in double precision (Eq. 1) and
+ * allocates every cache: rotated Q/K/V (RoPECache), (m, l, O~) (FACache;
+ * RowMaxcache / RowSumcache / Ocache of Algorithm 1) and scratch.  This is the
+ * only call that allocates device memory (the *_host calls allocate staging
+ * on first use).  Uses the current CUDA device.  On failure *out is NULL.
+ */
+lacache_status lacache_create(const lacache_config* cfg, lacache_ctx** out);
+
+/* Frees everything the context owns.  Synchronises the device first. */
+lacache_status lacache_destroy(lacache_ctx* ctx);
+
+/*
+ * Algorithm 1 with GenStep = True, cache side (Sec. 3.3.2-3.3.3).  Rotates
+ * q_pre/k_pre at each token's position and stores them with v_pre in the
+ * rotated cache for all T tokens, then for every fixed query i in U stores
+ * (m_i, l_i, O~_i) over the fixed keys j in U of the same sequence
+ * (Eq. 2-6).  Rows of the current block are rotated too (so the cache is
+ * complete) but get no state.  block_idx in [0, gen_len / block_len).
+ * q_pre [T,Hq,d], k_pre / v_pre [T,Hkv,d] of `dtype`.
+ */
+lacache_status lacache_build(lacache_ctx* ctx, int block_idx, const void* q_pre,
+                             const void* k_pre, const void* v_pre, void* cuda_stream);
+
+/*
+ * Algorithm 1 with GenStep = False (Sec. 3.3.3, last paragraph).  Rotates the
+ * block's fresh q_blk [B*L_b,Hq,d], k_blk / v_blk [B*L_b,Hkv,d] into the
+ * block's cache slots; fixed queries start from the cached state, visit only
+ * the block's keys and are normalised; block queries visit all keys.  Writes
+ * out [T,Hq,d] fp32 for ALL T rows and, if lse != NULL, lse [T,Hq].  The
+ * (m, l, O~) cache is read-only here.  Requires a preceding lacache_build for
+ * the same block, else LACACHE_ERR_STATE.
+ */
+lacache_status lacache_step(lacache_ctx* ctx, const void* q_blk, const void* k_blk,
+                            const void* v_blk, float* out, float* lse, void* cuda_stream);
+
+/*
+ * Plain attention for all rows over all keys (the definition in Sec. 3.3.3 /
+ * App. B.2 with the caches ignored): the vanilla full forward the method
+ * replaces.  Reads pre-RoPE q/k/v [T,...], writes out/lse.  Uses context
+ * scratch only; the caches are neither read nor written.
+ */
+lacache_status lacache_full_recompute(lacache_ctx* ctx, const void* q_pre, const void* k_pre,
+                                      const void* v_pre, float* out, float* lse,
+                                      void* cuda_stream);
+
+/*
+ * Same operations with HOST buffers: inputs are copied host->device and
+ * results device->host on `cuda_stream` inside the call (asynchronously when
+ * the host memory is pinned).  Staging is allocated on first use.  The caller
+ * synchronises the stream before reading out_host.  No paper counterpart.
+ */
+lacache_status lacache_build_host(lacache_ctx* ctx, int block_idx, const void* q_pre_host,
+                                  const void* k_pre_host, const void* v_pre_host,
+                                  void* cuda_stream);
+lacache_status lacache_step_host(lacache_ctx* ctx, const void* q_blk_host, const void* k_blk_host,
+                                 const void* v_blk_host, float* out_host, float* lse_host,
+                                 void* cuda_stream);
+
+/*
+ * Test hooks.  All outputs are device pointers, token-major fp32.
+ *   export_state: the cached triple in natural-log units, m [T,Hq], l [T,Hq],
+ *     o_acc [T,Hq,d].  The triple is not unique (any reference m gives the same
+ *     merged result); compare o_acc / l and m + log l.  Rows of the current
+ *     block are unspecified.
+ *   export_rope_cache: rotated q [T,Hq,d], rotated k [T,Hkv,d], v [T,Hkv,d] as
+ *     stored (the split bf16 planes summed).
+ *   export_index_meta (HOST outputs, any may be NULL): per token sequence id,
+ *     0-based position, is-current-block flag [T]; kv head of each q head [Hq].
+ */
+lacache_status lacache_export_state(lacache_ctx* ctx, float* m, float* l, float* o_acc,
+                                    void* cuda_stream);
+lacache_status lacache_export_rope_cache(lacache_ctx* ctx, float* q_rot, float* k_rot, float* v,
+                                         void* cuda_stream);
+lacache_status lacache_export_index_meta(lacache_ctx* ctx, int32_t* seq_of_tok_host,
+                                         int32_t* pos_of_tok_host, int32_t* is_block_host,
+                                         int32_t* kv_head_of_q_head_host);
+
+/* Total packed tokens T, and the number of kernels launched by the last
+ * build / step / full_recompute call.  No paper counterpart. */
+int lacache_total_tokens(const lacache_ctx* ctx);
+int lacache_last_launch_count(const lacache_ctx* ctx);
+/* which engine the context runs (LACACHE_ENGINE_SIMT or _TCGEN05) */
+int lacache_engine(const lacache_ctx* ctx);
+
+/*
+ * Synchronises the device and reads the device status word that bounded waits
+ * and self-checks write.  Returns LACACHE_OK, LACACHE_ERR_TIMEOUT, or
+ * LACACHE_ERR_CUDA; details in lacache_last_error.
+ */
+lacache_status lacache_poll_status(lacache_ctx* ctx);
+
+/* Human-readable text for the last error of this context ("" if none).  With
+ * ctx == NULL, the text of the last failed lacache_create on this thread. */
+const char* lacache_last_error(const lacache_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LACACHE_H_ */

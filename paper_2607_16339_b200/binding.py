@@ -1,0 +1,180 @@
+"""Thin ctypes binding over the C ABI of ``include/lacache.h``.
+
+Argument marshalling only: every step of the path runs inside the CUDA
+library.  Function names mirror the C entry points.  Tensors are torch tensors
+(device memory for the plain calls, host memory for the ``*_host`` calls);
+only their ``data_ptr()`` crosses the boundary.  There is no fallback: if
+``liblacache.so`` is missing or cannot be loaded, ``load()`` raises.
+"""
+import ctypes
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "liblacache.so")
+
+OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_STATE, ERR_UNSUPPORTED, ERR_OOM, ERR_CUDA, ERR_TIMEOUT = range(8)
+DTYPE_BF16, DTYPE_FP32 = 0, 1
+ENGINE_AUTO, ENGINE_SIMT, ENGINE_TCGEN05 = 0, 1, 2
+
+EXPORTS = [
+    "lacache_version", "lacache_create", "lacache_destroy", "lacache_build", "lacache_step",
+    "lacache_full_recompute", "lacache_build_host", "lacache_step_host", "lacache_export_state",
+    "lacache_export_rope_cache", "lacache_export_index_meta", "lacache_total_tokens",
+    "lacache_last_launch_count", "lacache_engine", "lacache_poll_status", "lacache_last_error",
+]
+
+
+class LacacheConfig(ctypes.Structure):
+    _fields_ = [
+        ("dtype", ctypes.c_int), ("engine", ctypes.c_int),
+        ("n_q_heads", ctypes.c_int), ("n_kv_heads", ctypes.c_int), ("head_dim", ctypes.c_int),
+        ("rope_theta", ctypes.c_float), ("softmax_scale", ctypes.c_float),
+        ("batch", ctypes.c_int), ("prompt_lens", ctypes.POINTER(ctypes.c_int32)),
+        ("gen_len", ctypes.c_int), ("block_len", ctypes.c_int),
+        ("sc_tiles_per_chunk", ctypes.c_int),
+    ]
+
+
+class LacacheError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__("lacache status %d: %s" % (status, message))
+        self.status = status
+
+
+_lib = None
+
+
+def load():
+    """Loads the CUDA library; raises if it is not built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("%s not found: build it with `python -m paper_2607_16339_b200.build` "
+                           "(there is no CPU fallback)" % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ip = ctypes.c_void_p, ctypes.c_int
+    lib.lacache_version.restype = ip
+    lib.lacache_create.argtypes = [ctypes.POINTER(LacacheConfig), ctypes.POINTER(vp)]
+    lib.lacache_destroy.argtypes = [vp]
+    lib.lacache_build.argtypes = [vp, ip, vp, vp, vp, vp]
+    lib.lacache_step.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.lacache_full_recompute.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.lacache_build_host.argtypes = [vp, ip, vp, vp, vp, vp]
+    lib.lacache_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.lacache_export_state.argtypes = [vp, vp, vp, vp, vp]
+    lib.lacache_export_rope_cache.argtypes = [vp, vp, vp, vp, vp]
+    lib.lacache_export_index_meta.argtypes = [vp, vp, vp, vp, vp]
+    lib.lacache_total_tokens.argtypes = [vp]
+    lib.lacache_last_launch_count.argtypes = [vp]
+    lib.lacache_engine.argtypes = [vp]
+    lib.lacache_poll_status.argtypes = [vp]
+    lib.lacache_last_error.argtypes = [vp]
+    lib.lacache_last_error.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name != "lacache_last_error":
+            getattr(lib, name).restype = ip
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+class Context:
+    """Owns one ``lacache_ctx``.  Methods mirror the C calls one to one."""
+
+    def __init__(self, dtype, n_q_heads, n_kv_heads, head_dim, rope_theta, prompt_lens, gen_len,
+                 block_len, softmax_scale=0.0, engine=ENGINE_AUTO, sc_tiles_per_chunk=0):
+        self._lib = load()
+        self._h = ctypes.c_void_p()
+        pl = (ctypes.c_int32 * len(prompt_lens))(*[int(p) for p in prompt_lens])
+        cfg = LacacheConfig(int(dtype), int(engine), int(n_q_heads), int(n_kv_heads), int(head_dim),
+                            float(rope_theta), float(softmax_scale), len(prompt_lens), pl,
+                            int(gen_len), int(block_len), int(sc_tiles_per_chunk))
+        st = self._lib.lacache_create(ctypes.byref(cfg), ctypes.byref(self._h))
+        if st != OK:
+            self._h = ctypes.c_void_p()
+            raise LacacheError(st, (self._lib.lacache_last_error(None) or b"").decode())
+        self.n_q_heads, self.n_kv_heads, self.head_dim = n_q_heads, n_kv_heads, head_dim
+        self.batch, self.block_len = len(prompt_lens), block_len
+
+    @classmethod
+    def from_workload(cls, wl, **kw):
+        return cls(DTYPE_BF16 if wl.dtype == "bf16" else DTYPE_FP32, wl.n_q_heads, wl.n_kv_heads,
+                   wl.head_dim, wl.rope_theta, wl.prompt_lens, wl.gen_len, wl.block_len, **kw)
+
+    def _check(self, st):
+        if st != OK:
+            raise LacacheError(st, (self._lib.lacache_last_error(self._h) or b"").decode())
+
+    def destroy(self):
+        if self._h:
+            self._lib.lacache_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    @property
+    def total_tokens(self):
+        return self._lib.lacache_total_tokens(self._h)
+
+    @property
+    def engine(self):
+        return self._lib.lacache_engine(self._h)
+
+    @property
+    def last_launch_count(self):
+        return self._lib.lacache_last_launch_count(self._h)
+
+    def build(self, block_idx, q_pre, k_pre, v_pre, stream=None):
+        self._check(self._lib.lacache_build(self._h, int(block_idx), _ptr(q_pre), _ptr(k_pre),
+                                            _ptr(v_pre), _stream(stream)))
+
+    def step(self, q_blk, k_blk, v_blk, out, lse=None, stream=None):
+        self._check(self._lib.lacache_step(self._h, _ptr(q_blk), _ptr(k_blk), _ptr(v_blk), _ptr(out),
+                                           _ptr(lse), _stream(stream)))
+
+    def full_recompute(self, q_pre, k_pre, v_pre, out, lse=None, stream=None):
+        self._check(self._lib.lacache_full_recompute(self._h, _ptr(q_pre), _ptr(k_pre), _ptr(v_pre),
+                                                     _ptr(out), _ptr(lse), _stream(stream)))
+
+    def build_host(self, block_idx, q_pre, k_pre, v_pre, stream=None):
+        self._check(self._lib.lacache_build_host(self._h, int(block_idx), _ptr(q_pre), _ptr(k_pre),
+                                                 _ptr(v_pre), _stream(stream)))
+
+    def step_host(self, q_blk, k_blk, v_blk, out, lse=None, stream=None):
+        self._check(self._lib.lacache_step_host(self._h, _ptr(q_blk), _ptr(k_blk), _ptr(v_blk),
+                                                _ptr(out), _ptr(lse), _stream(stream)))
+
+    def export_state(self, m, l, o_acc, stream=None):
+        self._check(self._lib.lacache_export_state(self._h, _ptr(m), _ptr(l), _ptr(o_acc), _stream(stream)))
+
+    def export_rope_cache(self, q_rot, k_rot, v, stream=None):
+        self._check(self._lib.lacache_export_rope_cache(self._h, _ptr(q_rot), _ptr(k_rot), _ptr(v),
+                                                        _stream(stream)))
+
+    def export_index_meta(self):
+        import numpy as np
+        T = self.total_tokens
+        seq = np.empty(T, np.int32); pos = np.empty(T, np.int32); isb = np.empty(T, np.int32)
+        kvh = np.empty(self.n_q_heads, np.int32)
+        p = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+        self._check(self._lib.lacache_export_index_meta(self._h, p(seq), p(pos), p(isb), p(kvh)))
+        return seq, pos, isb, kvh
+
+    def poll_status(self):
+        st = self._lib.lacache_poll_status(self._h)
+        return st, (self._lib.lacache_last_error(self._h) or b"").decode()

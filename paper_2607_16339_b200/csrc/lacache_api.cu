@@ -1,0 +1,532 @@
+// Host side of the C ABI: context, validation, the planner that derives the
+// integer metadata and the work lists, and the launch sequences.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "lacache_internal.h"
+
+using namespace lacache;
+
+struct lacache_ctx {
+  lacache_config cfg;
+  Geometry g;
+  int engine;
+  std::vector<int32_t> prompt_lens, cu, seq_of_tok, pos_of_tok;
+  std::vector<int32_t> blk_start_all;  // [n_blk][B]
+  // work lists (offsets into d_items)
+  struct ListRef { int off, n; };
+  std::vector<ListRef> build_list, step_list;  // per block
+  ListRef full_list;
+  int max_chunks = 1;
+
+  // device memory
+  std::vector<void*> allocs;
+  int32_t* d_cu = nullptr;
+  int32_t* d_blk_start_all = nullptr;
+  int32_t* d_pos = nullptr;
+  float* d_cos = nullptr;
+  float* d_sin = nullptr;
+  WorkItem* d_items = nullptr;
+  RotBuffers rot{}, rot_scratch{};
+  StateBuffers st{};
+  float *part_m = nullptr, *part_l = nullptr, *part_o = nullptr;
+  int* counters = nullptr;
+  int32_t* d_status = nullptr;
+  TcMaps* maps = nullptr;
+  TcMaps* maps_scratch = nullptr;
+  // staging for the *_host entry points
+  void *hs_q = nullptr, *hs_k = nullptr, *hs_v = nullptr;       // full arrays
+  void *hs_qb = nullptr, *hs_kb = nullptr, *hs_vb = nullptr;    // block arrays
+  float *hs_out = nullptr, *hs_lse = nullptr;
+
+  int built_block = -1;
+  int last_launches = 0;
+  int device = 0;
+  char err[512];
+};
+
+namespace {
+
+thread_local char g_create_err[512] = "";
+
+lacache_status fail(lacache_ctx* c, lacache_status st, const char* fmt, ...) {
+  char* dst = c ? c->err : g_create_err;
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(dst, 512, fmt, ap);
+  va_end(ap);
+  return st;
+}
+
+#define CU_TRY(c, expr)                                                              \
+  do {                                                                               \
+    cudaError_t e_ = (expr);                                                         \
+    if (e_ != cudaSuccess)                                                           \
+      return fail(c, e_ == cudaErrorMemoryAllocation ? LACACHE_ERR_OOM : LACACHE_ERR_CUDA, \
+                  "%s: %s", #expr, cudaGetErrorString(e_));                          \
+  } while (0)
+
+size_t elem_size(int dtype) { return dtype == LACACHE_DTYPE_BF16 ? 2 : 4; }
+
+bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+template <class T>
+cudaError_t dev_alloc(lacache_ctx* c, T** p, size_t n_elems, bool zero = false) {
+  void* q = nullptr;
+  size_t bytes = std::max<size_t>(n_elems * sizeof(T), 256);
+  cudaError_t e = cudaMalloc(&q, bytes);
+  if (e != cudaSuccess) return e;
+  c->allocs.push_back(q);
+  if (zero) {
+    e = cudaMemset(q, 0, bytes);
+    if (e != cudaSuccess) return e;
+  }
+  *p = reinterpret_cast<T*>(q);
+  return cudaSuccess;
+}
+
+// Tiles of `rows_per_item` query rows over [lo, hi) of one sequence.
+void add_row_tiles(std::vector<WorkItem>& v, int seq, int lo, int hi, int rows_per_item,
+                   int kind = ITEM_ROWS) {
+  for (int r = lo; r < hi; r += rows_per_item) {
+    WorkItem w{};
+    w.kind = kind;
+    w.seq = seq;
+    w.row0 = r;
+    w.nrows = std::min(rows_per_item, hi - r);
+    v.push_back(w);
+  }
+}
+
+lacache_status alloc_rot(lacache_ctx* c, RotBuffers* r) {
+  const Geometry& g = c->g;
+  size_t nq = (size_t)g.Hq * g.Tp * g.d, nk = (size_t)g.Hkv * g.Tp * g.d;
+  if (c->engine == LACACHE_ENGINE_TCGEN05) {
+    uint16_t *a, *b, *cc, *d, *e;
+    CU_TRY(c, dev_alloc(c, &a, nq, true));
+    CU_TRY(c, dev_alloc(c, &b, nq, true));
+    CU_TRY(c, dev_alloc(c, &cc, nk, true));
+    CU_TRY(c, dev_alloc(c, &d, nk, true));
+    CU_TRY(c, dev_alloc(c, &e, nk, true));
+    *r = RotBuffers{a, b, cc, d, e};
+  } else {
+    float *a, *b, *cc;
+    CU_TRY(c, dev_alloc(c, &a, nq, true));
+    CU_TRY(c, dev_alloc(c, &b, nk, true));
+    CU_TRY(c, dev_alloc(c, &cc, nk, true));
+    *r = RotBuffers{a, nullptr, b, nullptr, cc};
+  }
+  return LACACHE_OK;
+}
+
+lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
+  c->cfg = *cfg;
+  c->cfg.prompt_lens = nullptr;
+  c->err[0] = 0;
+  if (cfg->batch < 1 || !cfg->prompt_lens) return fail(c, LACACHE_ERR_INVALID_ARG, "batch < 1 or prompt_lens NULL");
+  if (cfg->dtype != LACACHE_DTYPE_BF16 && cfg->dtype != LACACHE_DTYPE_FP32)
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "dtype %d", cfg->dtype);
+  if (cfg->head_dim != 64 && cfg->head_dim != 128)
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "head_dim %d (64 or 128)", cfg->head_dim);
+  if (cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads % cfg->n_kv_heads)
+    return fail(c, LACACHE_ERR_SHAPE, "n_q_heads %d not a multiple of n_kv_heads %d", cfg->n_q_heads,
+                cfg->n_kv_heads);
+  if (cfg->gen_len < 1 || cfg->block_len < 1 || cfg->gen_len % cfg->block_len)
+    return fail(c, LACACHE_ERR_SHAPE, "gen_len %d not a positive multiple of block_len %d", cfg->gen_len,
+                cfg->block_len);
+  if (!(cfg->rope_theta > 0.f)) return fail(c, LACACHE_ERR_INVALID_ARG, "rope_theta must be > 0");
+  for (int b = 0; b < cfg->batch; ++b)
+    if (cfg->prompt_lens[b] < 0) return fail(c, LACACHE_ERR_SHAPE, "prompt_lens[%d] < 0", b);
+
+  bool tc_ok = cfg->dtype == LACACHE_DTYPE_BF16 && cfg->head_dim == 128 && cfg->block_len <= TC_ROWS;
+  if (cfg->engine == LACACHE_ENGINE_AUTO) c->engine = tc_ok ? LACACHE_ENGINE_TCGEN05 : LACACHE_ENGINE_SIMT;
+  else if (cfg->engine == LACACHE_ENGINE_SIMT) c->engine = LACACHE_ENGINE_SIMT;
+  else if (cfg->engine == LACACHE_ENGINE_TCGEN05) {
+    if (!tc_ok) return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs bf16, head_dim 128, block_len <= 128");
+    c->engine = LACACHE_ENGINE_TCGEN05;
+  } else return fail(c, LACACHE_ERR_INVALID_ARG, "engine %d", cfg->engine);
+
+  // ---- integer metadata (index sets of Sec. 3.3.1) ----
+  Geometry& g = c->g;
+  g.B = cfg->batch;
+  c->prompt_lens.assign(cfg->prompt_lens, cfg->prompt_lens + g.B);
+  c->cu.assign(g.B + 1, 0);
+  g.maxN = 0;
+  long long tot = 0;
+  for (int b = 0; b < g.B; ++b) {
+    int n = c->prompt_lens[b] + cfg->gen_len;
+    tot += n;
+    if (tot > (1ll << 30)) return fail(c, LACACHE_ERR_SHAPE, "too many tokens");
+    c->cu[b + 1] = (int32_t)tot;
+    g.maxN = std::max(g.maxN, n);
+  }
+  g.T = (int)tot;
+  g.Tp = (g.T + 127) / 128 * 128 + 128;
+  g.Hq = cfg->n_q_heads; g.Hkv = cfg->n_kv_heads; g.d = cfg->head_dim; g.group = g.Hq / g.Hkv;
+  g.gen_len = cfg->gen_len; g.block_len = cfg->block_len; g.n_blk = cfg->gen_len / cfg->block_len;
+  double scale = cfg->softmax_scale > 0.f ? (double)cfg->softmax_scale : 1.0 / sqrt((double)g.d);
+  g.scale_log2 = (float)(scale * 1.4426950408889634074);
+  c->seq_of_tok.resize(g.T);
+  c->pos_of_tok.resize(g.T);
+  for (int b = 0; b < g.B; ++b)
+    for (int t = c->cu[b]; t < c->cu[b + 1]; ++t) { c->seq_of_tok[t] = b; c->pos_of_tok[t] = t - c->cu[b]; }
+  c->blk_start_all.resize((size_t)g.n_blk * g.B);
+  for (int k = 0; k < g.n_blk; ++k)
+    for (int b = 0; b < g.B; ++b) c->blk_start_all[(size_t)k * g.B + b] = c->cu[b] + c->prompt_lens[b] + k * g.block_len;
+
+  // ---- work lists ----
+  const bool tc = c->engine == LACACHE_ENGINE_TCGEN05;
+  const int R = tc ? TC_ROWS : SIMT_ROWS;
+  std::vector<WorkItem> items;
+  int tpc = cfg->sc_tiles_per_chunk;
+  if (tpc <= 0) {
+    long long tiles = 0;
+    for (int b = 0; b < g.B; ++b) tiles += (c->cu[b + 1] - c->cu[b] + TC_KEYS - 1) / TC_KEYS;
+    tpc = (int)std::min<long long>(8, std::max<long long>(2, (tiles * g.Hq + 74) / 148));
+  }
+  c->max_chunks = 1;
+  for (int k = 0; k < g.n_blk; ++k) {
+    int off = (int)items.size();
+    // step list: block-query items first (the long ones), then fixed rows
+    for (int b = 0; b < g.B; ++b) {
+      int bs = c->blk_start_all[(size_t)k * g.B + b];
+      if (tc) {
+        int n = c->cu[b + 1] - c->cu[b];
+        int nkt = (n + TC_KEYS - 1) / TC_KEYS;
+        int chunks = (nkt + tpc - 1) / tpc;
+        c->max_chunks = std::max(c->max_chunks, chunks);
+        for (int ch = 0; ch < chunks; ++ch) {
+          WorkItem w{};
+          w.kind = ITEM_BLOCK_CHUNK; w.seq = b; w.row0 = bs; w.nrows = g.block_len;
+          w.chunk = ch; w.kt0 = ch * tpc; w.kt1 = std::min(nkt, (ch + 1) * tpc);
+          w.pad = chunks;
+          items.push_back(w);
+        }
+      } else {
+        add_row_tiles(items, b, bs, bs + g.block_len, R, ITEM_BLOCK_CHUNK);
+      }
+    }
+    int rows_off = (int)items.size();
+    for (int b = 0; b < g.B; ++b) {
+      int bs = c->blk_start_all[(size_t)k * g.B + b];
+      add_row_tiles(items, b, c->cu[b], bs, R);
+      add_row_tiles(items, b, bs + g.block_len, c->cu[b + 1], R);
+    }
+    c->step_list.push_back({off, (int)items.size() - off});
+    c->build_list.push_back({rows_off, (int)items.size() - rows_off});
+  }
+  {
+    int off = (int)items.size();
+    for (int b = 0; b < g.B; ++b) add_row_tiles(items, b, c->cu[b], c->cu[b + 1], R);
+    c->full_list = {off, (int)items.size() - off};
+  }
+
+  // ---- device ----
+  CU_TRY(c, cudaGetDevice(&c->device));
+  cudaDeviceProp prop;
+  CU_TRY(c, cudaGetDeviceProperties(&prop, c->device));
+  if (tc && prop.major != 10)
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs an sm_100 device, found sm_%d%d", prop.major, prop.minor);
+  CU_TRY(c, simt_prepare());
+  if (tc) CU_TRY(c, tc_prepare());
+
+  CU_TRY(c, dev_alloc(c, &c->d_cu, g.B + 1));
+  CU_TRY(c, cudaMemcpy(c->d_cu, c->cu.data(), sizeof(int32_t) * (g.B + 1), cudaMemcpyHostToDevice));
+  CU_TRY(c, dev_alloc(c, &c->d_blk_start_all, c->blk_start_all.size()));
+  CU_TRY(c, cudaMemcpy(c->d_blk_start_all, c->blk_start_all.data(), sizeof(int32_t) * c->blk_start_all.size(), cudaMemcpyHostToDevice));
+  CU_TRY(c, dev_alloc(c, &c->d_pos, g.T));
+  CU_TRY(c, cudaMemcpy(c->d_pos, c->pos_of_tok.data(), sizeof(int32_t) * g.T, cudaMemcpyHostToDevice));
+  CU_TRY(c, dev_alloc(c, &c->d_items, items.size()));
+  CU_TRY(c, cudaMemcpy(c->d_items, items.data(), sizeof(WorkItem) * items.size(), cudaMemcpyHostToDevice));
+  {
+    // cos/sin of p * theta^(-2c/d), evaluated in double, stored as fp32 (Eq. 1)
+    int half = g.d / 2;
+    std::vector<float> cs((size_t)g.maxN * half), sn((size_t)g.maxN * half);
+    for (int cidx = 0; cidx < half; ++cidx) {
+      double f = pow((double)cfg->rope_theta, -2.0 * (double)cidx / (double)g.d);
+      for (int p = 0; p < g.maxN; ++p) {
+        double ang = (double)p * f;
+        cs[(size_t)p * half + cidx] = (float)cos(ang);
+        sn[(size_t)p * half + cidx] = (float)sin(ang);
+      }
+    }
+    CU_TRY(c, dev_alloc(c, &c->d_cos, cs.size()));
+    CU_TRY(c, dev_alloc(c, &c->d_sin, sn.size()));
+    CU_TRY(c, cudaMemcpy(c->d_cos, cs.data(), sizeof(float) * cs.size(), cudaMemcpyHostToDevice));
+    CU_TRY(c, cudaMemcpy(c->d_sin, sn.data(), sizeof(float) * sn.size(), cudaMemcpyHostToDevice));
+  }
+  lacache_status st = alloc_rot(c, &c->rot);
+  if (st != LACACHE_OK) return st;
+  st = alloc_rot(c, &c->rot_scratch);
+  if (st != LACACHE_OK) return st;
+  CU_TRY(c, dev_alloc(c, &c->st.m, (size_t)g.Hq * g.Tp, true));
+  CU_TRY(c, dev_alloc(c, &c->st.l, (size_t)g.Hq * g.Tp, true));
+  CU_TRY(c, dev_alloc(c, &c->st.o, (size_t)g.Hq * g.Tp * g.d, true));
+  size_t nparts = (size_t)g.B * g.Hq * c->max_chunks * g.block_len;
+  CU_TRY(c, dev_alloc(c, &c->part_m, nparts));
+  CU_TRY(c, dev_alloc(c, &c->part_l, nparts));
+  CU_TRY(c, dev_alloc(c, &c->part_o, nparts * g.d));
+  CU_TRY(c, dev_alloc(c, &c->counters, (size_t)g.B * g.Hq, true));
+  CU_TRY(c, dev_alloc(c, &c->d_status, 4, true));
+  if (tc) {
+    c->maps = tc_make_maps(g, c->rot, c->err, sizeof(c->err));
+    if (!c->maps) return LACACHE_ERR_CUDA;
+    c->maps_scratch = tc_make_maps(g, c->rot_scratch, c->err, sizeof(c->err));
+    if (!c->maps_scratch) return LACACHE_ERR_CUDA;
+  }
+  CU_TRY(c, cudaDeviceSynchronize());
+  return LACACHE_OK;
+}
+
+void destroy_impl(lacache_ctx* c) {
+  cudaDeviceSynchronize();
+  for (void* p : c->allocs) cudaFree(p);
+  if (c->maps) tc_free_maps(c->maps);
+  if (c->maps_scratch) tc_free_maps(c->maps_scratch);
+  delete c;
+}
+
+AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk, const RotBuffers& rot,
+                   float* out, float* lse) {
+  AttnArgs a{};
+  a.mode = mode;
+  a.items = c->d_items + list.off;
+  a.n_items = list.n;
+  a.cu = c->d_cu;
+  a.blk_start = blk >= 0 ? c->d_blk_start_all + (size_t)blk * c->g.B : nullptr;
+  a.rot = rot;
+  a.st = c->st;
+  a.out = out;
+  a.lse = lse;
+  a.part_m = c->part_m; a.part_l = c->part_l; a.part_o = c->part_o;
+  a.counters = c->counters;
+  a.max_chunks = c->max_chunks;
+  a.status = c->d_status;
+  return a;
+}
+
+lacache_status run_attention(lacache_ctx* c, const AttnArgs& a, bool scratch, cudaStream_t s) {
+  if (c->engine == LACACHE_ENGINE_TCGEN05)
+    CU_TRY(c, tc_attention(c->g, a, scratch ? c->maps_scratch : c->maps, s));
+  else
+    CU_TRY(c, simt_attention(c->g, a, s));
+  c->last_launches++;
+  return LACACHE_OK;
+}
+
+lacache_status rope_all(lacache_ctx* c, const void* q, const void* k, const void* v, const RotBuffers& dst,
+                        cudaStream_t s) {
+  RopeArgs r{};
+  r.q = q; r.k = k; r.v = v;
+  r.n_src_rows = c->g.T;
+  r.blk_start = nullptr; r.block_len = c->g.block_len;
+  r.pos_of_tok = c->d_pos; r.cos_tab = c->d_cos; r.sin_tab = c->d_sin;
+  r.dst = dst;
+  r.in_dtype = c->cfg.dtype;
+  CU_TRY(c, rope_write(c->g, r, c->engine, s));
+  c->last_launches++;
+  return LACACHE_OK;
+}
+
+lacache_status ensure_staging(lacache_ctx* c) {
+  if (c->hs_out) return LACACHE_OK;
+  const Geometry& g = c->g;
+  size_t es = elem_size(c->cfg.dtype);
+  size_t nq = (size_t)g.T * g.Hq * g.d, nk = (size_t)g.T * g.Hkv * g.d;
+  size_t bq = (size_t)g.B * g.block_len * g.Hq * g.d, bk = (size_t)g.B * g.block_len * g.Hkv * g.d;
+  uint8_t *a, *b, *cc, *d, *e, *f;
+  CU_TRY(c, dev_alloc(c, &a, nq * es));
+  CU_TRY(c, dev_alloc(c, &b, nk * es));
+  CU_TRY(c, dev_alloc(c, &cc, nk * es));
+  CU_TRY(c, dev_alloc(c, &d, bq * es));
+  CU_TRY(c, dev_alloc(c, &e, bk * es));
+  CU_TRY(c, dev_alloc(c, &f, bk * es));
+  c->hs_q = a; c->hs_k = b; c->hs_v = cc; c->hs_qb = d; c->hs_kb = e; c->hs_vb = f;
+  CU_TRY(c, dev_alloc(c, &c->hs_lse, (size_t)g.T * g.Hq));
+  CU_TRY(c, dev_alloc(c, &c->hs_out, nq));
+  return LACACHE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lacache_version(void) { return 100; }
+
+lacache_status lacache_create(const lacache_config* cfg, lacache_ctx** out) {
+  if (out) *out = nullptr;
+  g_create_err[0] = 0;
+  if (!cfg || !out) return fail(nullptr, LACACHE_ERR_INVALID_ARG, "cfg or out is NULL");
+  lacache_ctx* c = new (std::nothrow) lacache_ctx();
+  if (!c) return fail(nullptr, LACACHE_ERR_OOM, "host allocation failed");
+  lacache_status st = create_impl(cfg, c);
+  if (st != LACACHE_OK) {
+    snprintf(g_create_err, sizeof(g_create_err), "%s", c->err);
+    cudaGetLastError();
+    destroy_impl(c);
+    return st;
+  }
+  *out = c;
+  return LACACHE_OK;
+}
+
+lacache_status lacache_destroy(lacache_ctx* ctx) {
+  if (!ctx) return LACACHE_ERR_INVALID_ARG;
+  destroy_impl(ctx);
+  return LACACHE_OK;
+}
+
+lacache_status lacache_build(lacache_ctx* c, int block_idx, const void* q, const void* k, const void* v,
+                             void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if (!q || !k || !v) return fail(c, LACACHE_ERR_INVALID_ARG, "NULL input pointer");
+  if (misaligned(q) || misaligned(k) || misaligned(v)) return fail(c, LACACHE_ERR_INVALID_ARG, "input pointer not 16-byte aligned");
+  if (block_idx < 0 || block_idx >= c->g.n_blk)
+    return fail(c, LACACHE_ERR_INVALID_ARG, "block_idx %d outside [0, %d)", block_idx, c->g.n_blk);
+  cudaStream_t s = (cudaStream_t)stream;
+  c->last_launches = 0;
+  c->built_block = -1;
+  lacache_status st = rope_all(c, q, k, v, c->rot, s);
+  if (st != LACACHE_OK) return st;
+  AttnArgs a = attn_args(c, MODE_BUILD, c->build_list[block_idx], block_idx, c->rot, nullptr, nullptr);
+  st = run_attention(c, a, false, s);
+  if (st != LACACHE_OK) return st;
+  c->built_block = block_idx;
+  return LACACHE_OK;
+}
+
+lacache_status lacache_step(lacache_ctx* c, const void* q, const void* k, const void* v, float* out,
+                            float* lse, void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if (c->built_block < 0) return fail(c, LACACHE_ERR_STATE, "lacache_step before a successful lacache_build");
+  if (!q || !k || !v || !out) return fail(c, LACACHE_ERR_INVALID_ARG, "NULL pointer");
+  if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(out) || (lse && misaligned(lse)))
+    return fail(c, LACACHE_ERR_INVALID_ARG, "pointer not 16-byte aligned");
+  cudaStream_t s = (cudaStream_t)stream;
+  const int blk = c->built_block;
+  c->last_launches = 0;
+  RopeArgs r{};
+  r.q = q; r.k = k; r.v = v;
+  r.n_src_rows = c->g.B * c->g.block_len;
+  r.blk_start = c->d_blk_start_all + (size_t)blk * c->g.B;
+  r.block_len = c->g.block_len;
+  r.pos_of_tok = c->d_pos; r.cos_tab = c->d_cos; r.sin_tab = c->d_sin;
+  r.dst = c->rot;
+  r.in_dtype = c->cfg.dtype;
+  CU_TRY(c, rope_write(c->g, r, c->engine, s));
+  c->last_launches++;
+  AttnArgs a = attn_args(c, MODE_STEP, c->step_list[blk], blk, c->rot, out, lse);
+  return run_attention(c, a, false, s);
+}
+
+lacache_status lacache_full_recompute(lacache_ctx* c, const void* q, const void* k, const void* v, float* out,
+                                      float* lse, void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if (!q || !k || !v || !out) return fail(c, LACACHE_ERR_INVALID_ARG, "NULL pointer");
+  if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(out) || (lse && misaligned(lse)))
+    return fail(c, LACACHE_ERR_INVALID_ARG, "pointer not 16-byte aligned");
+  cudaStream_t s = (cudaStream_t)stream;
+  c->last_launches = 0;
+  lacache_status st = rope_all(c, q, k, v, c->rot_scratch, s);
+  if (st != LACACHE_OK) return st;
+  AttnArgs a = attn_args(c, MODE_FULL, c->full_list, -1, c->rot_scratch, out, lse);
+  return run_attention(c, a, true, s);
+}
+
+lacache_status lacache_build_host(lacache_ctx* c, int block_idx, const void* q, const void* k, const void* v,
+                                  void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if (!q || !k || !v) return fail(c, LACACHE_ERR_INVALID_ARG, "NULL input pointer");
+  lacache_status st = ensure_staging(c);
+  if (st != LACACHE_OK) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  const Geometry& g = c->g;
+  size_t es = elem_size(c->cfg.dtype);
+  CU_TRY(c, cudaMemcpyAsync(c->hs_q, q, (size_t)g.T * g.Hq * g.d * es, cudaMemcpyHostToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(c->hs_k, k, (size_t)g.T * g.Hkv * g.d * es, cudaMemcpyHostToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(c->hs_v, v, (size_t)g.T * g.Hkv * g.d * es, cudaMemcpyHostToDevice, s));
+  return lacache_build(c, block_idx, c->hs_q, c->hs_k, c->hs_v, stream);
+}
+
+lacache_status lacache_step_host(lacache_ctx* c, const void* q, const void* k, const void* v, float* out,
+                                 float* lse, void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if (!q || !k || !v || !out) return fail(c, LACACHE_ERR_INVALID_ARG, "NULL pointer");
+  lacache_status st = ensure_staging(c);
+  if (st != LACACHE_OK) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  const Geometry& g = c->g;
+  size_t es = elem_size(c->cfg.dtype);
+  size_t rows = (size_t)g.B * g.block_len;
+  CU_TRY(c, cudaMemcpyAsync(c->hs_qb, q, rows * g.Hq * g.d * es, cudaMemcpyHostToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(c->hs_kb, k, rows * g.Hkv * g.d * es, cudaMemcpyHostToDevice, s));
+  CU_TRY(c, cudaMemcpyAsync(c->hs_vb, v, rows * g.Hkv * g.d * es, cudaMemcpyHostToDevice, s));
+  st = lacache_step(c, c->hs_qb, c->hs_kb, c->hs_vb, c->hs_out, lse ? c->hs_lse : nullptr, stream);
+  if (st != LACACHE_OK) return st;
+  CU_TRY(c, cudaMemcpyAsync(out, c->hs_out, sizeof(float) * g.T * g.Hq * g.d, cudaMemcpyDeviceToHost, s));
+  if (lse) CU_TRY(c, cudaMemcpyAsync(lse, c->hs_lse, sizeof(float) * g.T * g.Hq, cudaMemcpyDeviceToHost, s));
+  return LACACHE_OK;
+}
+
+lacache_status lacache_export_state(lacache_ctx* c, float* m, float* l, float* o, void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if (c->built_block < 0) return fail(c, LACACHE_ERR_STATE, "no state: lacache_build has not run");
+  ExportArgs e{};
+  e.rot = c->rot; e.st = c->st; e.m = m; e.l = l; e.o = o;
+  CU_TRY(c, export_buffers(c->g, e, c->engine, (cudaStream_t)stream));
+  return LACACHE_OK;
+}
+
+lacache_status lacache_export_rope_cache(lacache_ctx* c, float* q, float* k, float* v, void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  ExportArgs e{};
+  e.rot = c->rot; e.st = c->st; e.q_rot = q; e.k_rot = k; e.v = v;
+  CU_TRY(c, export_buffers(c->g, e, c->engine, (cudaStream_t)stream));
+  return LACACHE_OK;
+}
+
+lacache_status lacache_export_index_meta(lacache_ctx* c, int32_t* seq, int32_t* pos, int32_t* isb, int32_t* kvh) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  const Geometry& g = c->g;
+  if (seq) memcpy(seq, c->seq_of_tok.data(), sizeof(int32_t) * g.T);
+  if (pos) memcpy(pos, c->pos_of_tok.data(), sizeof(int32_t) * g.T);
+  if (isb) {
+    memset(isb, 0, sizeof(int32_t) * g.T);
+    if (c->built_block >= 0)
+      for (int b = 0; b < g.B; ++b) {
+        int bs = c->blk_start_all[(size_t)c->built_block * g.B + b];
+        for (int r = 0; r < g.block_len; ++r) isb[bs + r] = 1;
+      }
+  }
+  if (kvh)
+    for (int h = 0; h < g.Hq; ++h) kvh[h] = h / g.group;
+  return LACACHE_OK;
+}
+
+int lacache_total_tokens(const lacache_ctx* c) { return c ? c->g.T : -1; }
+int lacache_last_launch_count(const lacache_ctx* c) { return c ? c->last_launches : -1; }
+int lacache_engine(const lacache_ctx* c) { return c ? c->engine : -1; }
+
+lacache_status lacache_poll_status(lacache_ctx* c) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  CU_TRY(c, cudaDeviceSynchronize());
+  int32_t w[4];
+  CU_TRY(c, cudaMemcpy(w, c->d_status, sizeof(w), cudaMemcpyDeviceToHost));
+  if (w[0] != 0) {
+    fail(c, (lacache_status)w[0], "device status: code %d at location %d (aux %d, %d)", w[0], w[1], w[2], w[3]);
+    cudaMemset(c->d_status, 0, sizeof(w));
+    return (lacache_status)w[0];
+  }
+  return LACACHE_OK;
+}
+
+const char* lacache_last_error(const lacache_ctx* c) { return c ? c->err : g_create_err; }
+
+}  // extern "C"

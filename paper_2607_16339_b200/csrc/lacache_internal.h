@@ -1,0 +1,119 @@
+// Internal declarations shared by the host side (lacache_api.cu) and the two
+// kernel families (lacache_simt.cu: CUDA-core fp32; lacache_tc.cu: tcgen05).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/lacache.h"
+
+namespace lacache {
+
+// Work item kinds.  A launch walks a list of items; blockIdx.y is the q head.
+enum ItemKind : int32_t {
+  ITEM_ROWS = 0,   // a tile of query rows [row0, row0 + nrows) of one sequence
+  ITEM_BLOCK_CHUNK = 1,  // the block's query rows x one chunk of key tiles
+};
+struct WorkItem {
+  int32_t kind;   // ItemKind
+  int32_t seq;    // sequence index
+  int32_t row0;   // first packed token index of the query rows
+  int32_t nrows;  // number of valid query rows (<= tile rows)
+  int32_t chunk;  // ITEM_BLOCK_CHUNK: chunk index; else 0
+  int32_t kt0;    // ITEM_BLOCK_CHUNK: first key tile of the chunk
+  int32_t kt1;    // ITEM_BLOCK_CHUNK: one past the last key tile
+  int32_t pad;
+};
+
+// What a launch computes for ITEM_ROWS items.
+enum Mode : int32_t {
+  MODE_BUILD = 0,   // fixed queries x fixed keys -> cached state
+  MODE_STEP = 1,    // ITEM_ROWS: fixed queries x block keys merged into the
+                    // cached state; ITEM_BLOCK_CHUNK: block queries x all keys
+  MODE_FULL = 2,    // every query x every key, no cache
+};
+
+// Device status word layout (int32 x 4): [0] code, [1] location, [2], [3] aux
+enum StatusLoc : int32_t {
+  LOC_NONE = 0,
+  LOC_SMEM_ALIGN = 1,
+  LOC_WAIT_Q = 2,
+  LOC_WAIT_K = 3,
+  LOC_WAIT_V = 4,
+  LOC_WAIT_S = 5,
+  LOC_WAIT_O = 6,
+};
+
+struct Geometry {
+  int B, T, Tp, maxN;
+  int Hq, Hkv, d, group;
+  int gen_len, block_len, n_blk;
+  float scale_log2;  // softmax_scale * log2(e)
+};
+
+// Rotated cache / scratch set.  SIMT engine: fp32 planes (q, k, v).
+// tcgen05 engine: bf16 hi/lo planes for q and k, fp16 plane for v.
+// All planes are head-major: [H][Tp][d].
+struct RotBuffers {
+  void* q_hi; void* q_lo;   // SIMT: q_hi = fp32 q, q_lo unused
+  void* k_hi; void* k_lo;
+  void* v;
+};
+
+struct StateBuffers {       // head-major: m,l [Hq][Tp]; o [Hq][Tp][d]
+  float* m; float* l; float* o;   // m in log2 units (reference exponent)
+};
+
+struct RopeArgs {
+  const void* q; const void* k; const void* v;  // source rows, token-major
+  int n_src_rows;
+  // destination token of source row r: dst_map == nullptr ? r
+  //   : blk_start[r / block_len] + r % block_len
+  const int32_t* blk_start; int block_len;
+  const int32_t* pos_of_tok;
+  const float* cos_tab; const float* sin_tab;  // [maxN][d/2]
+  RotBuffers dst;
+  int in_dtype;
+};
+
+struct AttnArgs {
+  int mode;
+  const WorkItem* items; int n_items;
+  const int32_t* cu;         // [B+1]
+  const int32_t* blk_start;  // [B] absolute token index of the block's first row
+  RotBuffers rot;
+  StateBuffers st;
+  float* out; float* lse;    // token-major [T,Hq,d], [T,Hq]
+  // split-key partial states of block queries and their arrival counters
+  float* part_m; float* part_l; float* part_o; int* counters; int max_chunks;
+  int32_t* status;
+};
+
+struct ExportArgs {
+  RotBuffers rot; StateBuffers st;
+  float* m; float* l; float* o;          // token-major outputs (may be null)
+  float* q_rot; float* k_rot; float* v;  // token-major outputs (may be null)
+};
+
+// ---- launchers implemented by the kernel files -----------------------------
+// Each returns the cudaError_t of the launch (cudaGetLastError()).
+// engine: LACACHE_ENGINE_SIMT or LACACHE_ENGINE_TCGEN05 (selects the storage
+// format of the rotated planes).
+cudaError_t rope_write(const Geometry& g, const RopeArgs& a, int engine, cudaStream_t s);
+cudaError_t export_buffers(const Geometry& g, const ExportArgs& a, int engine, cudaStream_t s);
+
+cudaError_t simt_attention(const Geometry& g, const AttnArgs& a, cudaStream_t s);
+cudaError_t simt_prepare();  // function attributes
+
+struct TcMaps;  // opaque set of TMA descriptors, defined in lacache_tc.cu
+cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* maps, cudaStream_t s);
+cudaError_t tc_prepare();
+// builds TMA descriptors for a rotated buffer set; returns nullptr and fills
+// err on failure
+TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, char* err, int errlen);
+void tc_free_maps(TcMaps* m);
+
+constexpr int SIMT_ROWS = 32;    // query rows per SIMT work item
+constexpr int TC_ROWS = 128;     // query rows per tcgen05 work item
+constexpr int TC_KEYS = 64;      // keys per tcgen05 key tile
+
+}  // namespace lacache

@@ -1,0 +1,199 @@
+// RoPE-on-write (Eq. 1, Sec. 3.3.2) and the export kernels.
+//
+// rope_write rotates q and k at each token's position, copies v, and stores
+// the result head-major in the engine's storage format:
+//   SIMT engine    : fp32 planes.
+//   tcgen05 engine : rotated q,k as two bf16 planes hi = bf16(x),
+//                    lo = bf16(x - hi) (so hi + lo carries 16 significand
+//                    bits into the tensor-core score product); v as fp16.
+// The same kernel serves the build (all T tokens) and the step (only the
+// block's L_b tokens per sequence, scattered to their cache slots).
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "lacache_internal.h"
+
+namespace lacache {
+namespace {
+
+__device__ __forceinline__ void load8(const void* base, size_t elem_off, int in_dtype, float (&x)[8]) {
+  if (in_dtype == LACACHE_DTYPE_BF16) {
+    uint4 u = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(base) + elem_off);
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 f = __bfloat1622float2(p[i]);
+      x[2 * i] = f.x;
+      x[2 * i + 1] = f.y;
+    }
+  } else {
+    const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(base) + elem_off);
+    float4 a = p[0], b = p[1];
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
+    x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+  }
+}
+
+__device__ __forceinline__ void store8_f32(void* plane, size_t off, const float (&y)[8]) {
+  float4* p = reinterpret_cast<float4*>(reinterpret_cast<float*>(plane) + off);
+  p[0] = make_float4(y[0], y[1], y[2], y[3]);
+  p[1] = make_float4(y[4], y[5], y[6], y[7]);
+}
+
+__device__ __forceinline__ void store8_split(void* hi_plane, void* lo_plane, size_t off,
+                                             const float (&y)[8]) {
+  uint4 uh, ul;
+  __nv_bfloat162* ph = reinterpret_cast<__nv_bfloat162*>(&uh);
+  __nv_bfloat162* pl = reinterpret_cast<__nv_bfloat162*>(&ul);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat16 h0 = __float2bfloat16_rn(y[2 * i]);
+    __nv_bfloat16 h1 = __float2bfloat16_rn(y[2 * i + 1]);
+    __nv_bfloat16 l0 = __float2bfloat16_rn(y[2 * i] - __bfloat162float(h0));
+    __nv_bfloat16 l1 = __float2bfloat16_rn(y[2 * i + 1] - __bfloat162float(h1));
+    ph[i] = __halves2bfloat162(h0, h1);
+    pl[i] = __halves2bfloat162(l0, l1);
+  }
+  *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(hi_plane) + off) = uh;
+  *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(lo_plane) + off) = ul;
+}
+
+__device__ __forceinline__ void store8_f16(void* plane, size_t off, const float (&y)[8]) {
+  uint4 u;
+  __half2* p = reinterpret_cast<__half2*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    // saturate to the finite fp16 range
+    float a = fminf(fmaxf(y[2 * i], -65504.f), 65504.f);
+    float b = fminf(fmaxf(y[2 * i + 1], -65504.f), 65504.f);
+    p[i] = __floats2half2_rn(a, b);
+  }
+  *reinterpret_cast<uint4*>(reinterpret_cast<__half*>(plane) + off) = u;
+}
+
+// One thread: 8 features c0..c0+7 of the first half and their partners at
+// c0 + d/2 of one (source row, head slot).  Head slots: [0,Hq) q heads,
+// [Hq,Hq+Hkv) k heads, [Hq+Hkv,Hq+2Hkv) v heads.
+template <bool TC>
+__global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a) {
+  const int chunks = g.d / 16;
+  const int slots = g.Hq + 2 * g.Hkv;
+  const long long total = (long long)a.n_src_rows * slots * chunks;
+  long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  int chunk = (int)(idx % chunks);
+  long long t = idx / chunks;
+  int slot = (int)(t % slots);
+  int r = (int)(t / slots);
+  int tok = a.blk_start ? a.blk_start[r / a.block_len] + r % a.block_len : r;
+  const int half = g.d / 2;
+  const int c0 = chunk * 8;
+
+  const void* src;
+  int H, h;
+  int which;  // 0 q, 1 k, 2 v
+  if (slot < g.Hq) { src = a.q; H = g.Hq; h = slot; which = 0; }
+  else if (slot < g.Hq + g.Hkv) { src = a.k; H = g.Hkv; h = slot - g.Hq; which = 1; }
+  else { src = a.v; H = g.Hkv; h = slot - g.Hq - g.Hkv; which = 2; }
+
+  float x1[8], x2[8], y1[8], y2[8];
+  size_t soff = ((size_t)r * H + h) * g.d;
+  load8(src, soff + c0, a.in_dtype, x1);
+  load8(src, soff + c0 + half, a.in_dtype, x2);
+  if (which < 2) {
+    int pos = a.pos_of_tok[tok];
+    const float4* cp = reinterpret_cast<const float4*>(a.cos_tab + (size_t)pos * half + c0);
+    const float4* sp = reinterpret_cast<const float4*>(a.sin_tab + (size_t)pos * half + c0);
+    float4 ca = cp[0], cb = cp[1], sa = sp[0], sb = sp[1];
+    float cs[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+    float sn[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      // separate roundings on purpose (no fma contraction surprises)
+      y1[i] = __fsub_rn(__fmul_rn(x1[i], cs[i]), __fmul_rn(x2[i], sn[i]));
+      y2[i] = __fadd_rn(__fmul_rn(x2[i], cs[i]), __fmul_rn(x1[i], sn[i]));
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { y1[i] = x1[i]; y2[i] = x2[i]; }
+  }
+  size_t doff = ((size_t)h * g.Tp + tok) * g.d;
+  if (TC) {
+    if (which == 0) {
+      store8_split(a.dst.q_hi, a.dst.q_lo, doff + c0, y1);
+      store8_split(a.dst.q_hi, a.dst.q_lo, doff + c0 + half, y2);
+    } else if (which == 1) {
+      store8_split(a.dst.k_hi, a.dst.k_lo, doff + c0, y1);
+      store8_split(a.dst.k_hi, a.dst.k_lo, doff + c0 + half, y2);
+    } else {
+      store8_f16(a.dst.v, doff + c0, y1);
+      store8_f16(a.dst.v, doff + c0 + half, y2);
+    }
+  } else {
+    void* plane = which == 0 ? a.dst.q_hi : (which == 1 ? a.dst.k_hi : a.dst.v);
+    store8_f32(plane, doff + c0, y1);
+    store8_f32(plane, doff + c0 + half, y2);
+  }
+}
+
+// Export kernels: head-major storage -> token-major fp32.
+template <bool TC>
+__device__ __forceinline__ float read_rot(const void* hi, const void* lo, size_t off) {
+  if (TC) {
+    return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(hi)[off]) +
+           __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(lo)[off]);
+  }
+  return reinterpret_cast<const float*>(hi)[off];
+}
+
+template <bool TC>
+__global__ void __launch_bounds__(256) export_kernel(Geometry g, ExportArgs a) {
+  long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  long long nq = (long long)g.T * g.Hq * g.d;
+  if (idx >= nq) return;
+  int c = (int)(idx % g.d);
+  long long t = idx / g.d;
+  int h = (int)(t % g.Hq);
+  int tok = (int)(t / g.Hq);
+  size_t src = ((size_t)h * g.Tp + tok) * g.d + c;
+  const float LN2 = 0.69314718055994530942f;
+  if (a.o) a.o[idx] = a.st.o[src];
+  if (c == 0) {
+    if (a.m) a.m[(size_t)tok * g.Hq + h] = a.st.m[(size_t)h * g.Tp + tok] * LN2;
+    if (a.l) a.l[(size_t)tok * g.Hq + h] = a.st.l[(size_t)h * g.Tp + tok];
+  }
+  if (a.q_rot) a.q_rot[idx] = read_rot<TC>(a.rot.q_hi, a.rot.q_lo, src);
+  if (h < g.Hkv) {
+    size_t dst = ((size_t)tok * g.Hkv + h) * g.d + c;
+    if (a.k_rot) a.k_rot[dst] = read_rot<TC>(a.rot.k_hi, a.rot.k_lo, src);
+    if (a.v) {
+      a.v[dst] = TC ? __half2float(reinterpret_cast<const __half*>(a.rot.v)[src])
+                    : reinterpret_cast<const float*>(a.rot.v)[src];
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t rope_write(const Geometry& g, const RopeArgs& a, int engine, cudaStream_t s) {
+  long long total = (long long)a.n_src_rows * (g.Hq + 2 * g.Hkv) * (g.d / 16);
+  if (total == 0) return cudaSuccess;
+  unsigned blocks = (unsigned)((total + 255) / 256);
+  if (engine == LACACHE_ENGINE_TCGEN05)
+    rope_write_kernel<true><<<blocks, 256, 0, s>>>(g, a);
+  else
+    rope_write_kernel<false><<<blocks, 256, 0, s>>>(g, a);
+  return cudaGetLastError();
+}
+
+cudaError_t export_buffers(const Geometry& g, const ExportArgs& a, int engine, cudaStream_t s) {
+  long long total = (long long)g.T * g.Hq * g.d;
+  unsigned blocks = (unsigned)((total + 255) / 256);
+  if (engine == LACACHE_ENGINE_TCGEN05)
+    export_kernel<true><<<blocks, 256, 0, s>>>(g, a);
+  else
+    export_kernel<false><<<blocks, 256, 0, s>>>(g, a);
+  return cudaGetLastError();
+}
+
+}  // namespace lacache
