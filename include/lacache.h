@@ -159,6 +159,15 @@ lacache_status lacache_export_index_meta(lacache_ctx* ctx, int32_t* seq_of_tok_h
                                          int32_t* pos_of_tok_host, int32_t* is_block_host,
                                          int32_t* kv_head_of_q_head_host);
 
+/*
+ * Profiling hook: when both are non-NULL cudaEvent_t handles, every later
+ * build / step / full_recompute records `ev_start` right before and `ev_stop`
+ * right after its attention kernel launch, on the call's stream, so a caller
+ * can time that kernel alone.  Pass NULLs to switch it off.  The caller owns
+ * the events.  No paper counterpart.
+ */
+lacache_status lacache_set_timing_events(lacache_ctx* ctx, void* ev_start, void* ev_stop);
+
 /* Total packed tokens T, and the number of kernels launched by the last
  * build / step / full_recompute call.  No paper counterpart. */
 int lacache_total_tokens(const lacache_ctx* ctx);

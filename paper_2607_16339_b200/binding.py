@@ -20,7 +20,7 @@ EXPORTS = [
     "lacache_version", "lacache_create", "lacache_destroy", "lacache_build", "lacache_step",
     "lacache_full_recompute", "lacache_build_host", "lacache_step_host", "lacache_export_state",
     "lacache_export_rope_cache", "lacache_export_index_meta", "lacache_total_tokens",
-    "lacache_last_launch_count", "lacache_engine", "lacache_poll_status", "lacache_last_error",
+    "lacache_last_launch_count", "lacache_engine", "lacache_set_timing_events", "lacache_poll_status", "lacache_last_error",
 ]
 
 
@@ -65,6 +65,7 @@ def load():
     lib.lacache_export_state.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_export_rope_cache.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_export_index_meta.argtypes = [vp, vp, vp, vp, vp]
+    lib.lacache_set_timing_events.argtypes = [vp, vp, vp]
     lib.lacache_total_tokens.argtypes = [vp]
     lib.lacache_last_launch_count.argtypes = [vp]
     lib.lacache_engine.argtypes = [vp]
@@ -174,6 +175,11 @@ class Context:
         p = lambda a: a.ctypes.data_as(ctypes.c_void_p)
         self._check(self._lib.lacache_export_index_meta(self._h, p(seq), p(pos), p(isb), p(kvh)))
         return seq, pos, isb, kvh
+
+    def set_timing_events(self, ev_start, ev_stop):
+        """torch.cuda.Event pair (already recorded once) or (None, None)."""
+        h = lambda e: None if e is None else ctypes.c_void_p(e.cuda_event)
+        self._check(self._lib.lacache_set_timing_events(self._h, h(ev_start), h(ev_stop)))
 
     def poll_status(self):
         st = self._lib.lacache_poll_status(self._h)

@@ -46,6 +46,7 @@ struct lacache_ctx {
   void *hs_qb = nullptr, *hs_kb = nullptr, *hs_vb = nullptr;    // block arrays
   float *hs_out = nullptr, *hs_lse = nullptr;
 
+  cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
   int built_block = -1;
   int last_launches = 0;
   int device = 0;
@@ -313,10 +314,12 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
 }
 
 lacache_status run_attention(lacache_ctx* c, const AttnArgs& a, bool scratch, cudaStream_t s) {
+  if (c->ev_start) CU_TRY(c, cudaEventRecord(c->ev_start, s));
   if (c->engine == LACACHE_ENGINE_TCGEN05)
     CU_TRY(c, tc_attention(c->g, a, scratch ? c->maps_scratch : c->maps, s));
   else
     CU_TRY(c, simt_attention(c->g, a, s));
+  if (c->ev_stop) CU_TRY(c, cudaEventRecord(c->ev_stop, s));
   c->last_launches++;
   return LACACHE_OK;
 }
@@ -507,6 +510,14 @@ lacache_status lacache_export_index_meta(lacache_ctx* c, int32_t* seq, int32_t* 
   }
   if (kvh)
     for (int h = 0; h < g.Hq; ++h) kvh[h] = h / g.group;
+  return LACACHE_OK;
+}
+
+lacache_status lacache_set_timing_events(lacache_ctx* c, void* ev_start, void* ev_stop) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if ((ev_start == nullptr) != (ev_stop == nullptr)) return fail(c, LACACHE_ERR_INVALID_ARG, "pass both events or neither");
+  c->ev_start = (cudaEvent_t)ev_start;
+  c->ev_stop = (cudaEvent_t)ev_stop;
   return LACACHE_OK;
 }
 
