@@ -3,6 +3,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -22,9 +23,13 @@ struct lacache_ctx {
   std::vector<int32_t> blk_start_all;  // [n_blk][B]
   // work lists (offsets into d_items)
   struct ListRef { int off, n; };
-  std::vector<ListRef> build_list, step_list;  // per block
+  std::vector<ListRef> build_list, step_list;  // per block (step_list: SIMT all items; tcgen05 block-chunk items)
+  std::vector<ListRef> merge_list;             // per block: fixed-row items of a step (tcgen05)
+  int num_sms = 148;
+  int stream_ctas_override = 0;
   ListRef full_list;
   int max_chunks = 1;
+  std::vector<WorkItem> items_host;
 
   // device memory
   std::vector<void*> allocs;
@@ -94,14 +99,18 @@ cudaError_t dev_alloc(lacache_ctx* c, T** p, size_t n_elems, bool zero = false) 
 }
 
 // Tiles of `rows_per_item` query rows over [lo, hi) of one sequence.
-void add_row_tiles(std::vector<WorkItem>& v, int seq, int lo, int hi, int rows_per_item,
-                   int kind = ITEM_ROWS) {
+void add_row_tiles(std::vector<WorkItem>& v, int seq, int lo, int hi, int rows_per_item, int seq_start,
+                   int seq_end, int blk_start, int kind = ITEM_ROWS) {
   for (int r = lo; r < hi; r += rows_per_item) {
     WorkItem w{};
     w.kind = kind;
     w.seq = seq;
     w.row0 = r;
     w.nrows = std::min(rows_per_item, hi - r);
+    w.pad = 1;
+    w.seq_start = seq_start;
+    w.seq_end = seq_end;
+    w.blk_start = blk_start;
     v.push_back(w);
   }
 }
@@ -146,11 +155,11 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   for (int b = 0; b < cfg->batch; ++b)
     if (cfg->prompt_lens[b] < 0) return fail(c, LACACHE_ERR_SHAPE, "prompt_lens[%d] < 0", b);
 
-  bool tc_ok = cfg->dtype == LACACHE_DTYPE_BF16 && cfg->head_dim == 128 && cfg->block_len <= TC_ROWS;
+  bool tc_ok = cfg->dtype == LACACHE_DTYPE_BF16 && cfg->head_dim == 128 && cfg->block_len <= TC_KEYS;
   if (cfg->engine == LACACHE_ENGINE_AUTO) c->engine = tc_ok ? LACACHE_ENGINE_TCGEN05 : LACACHE_ENGINE_SIMT;
   else if (cfg->engine == LACACHE_ENGINE_SIMT) c->engine = LACACHE_ENGINE_SIMT;
   else if (cfg->engine == LACACHE_ENGINE_TCGEN05) {
-    if (!tc_ok) return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs bf16, head_dim 128, block_len <= 128");
+    if (!tc_ok) return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs bf16, head_dim 128, block_len <= 64");
     c->engine = LACACHE_ENGINE_TCGEN05;
   } else return fail(c, LACACHE_ERR_INVALID_ARG, "engine %d", cfg->engine);
 
@@ -195,7 +204,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   c->max_chunks = 1;
   for (int k = 0; k < g.n_blk; ++k) {
     int off = (int)items.size();
-    // step list: block-query items first (the long ones), then fixed rows
+    // block-query items
     for (int b = 0; b < g.B; ++b) {
       int bs = c->blk_start_all[(size_t)k * g.B + b];
       if (tc) {
@@ -208,31 +217,41 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
           w.kind = ITEM_BLOCK_CHUNK; w.seq = b; w.row0 = bs; w.nrows = g.block_len;
           w.chunk = ch; w.kt0 = ch * tpc; w.kt1 = std::min(nkt, (ch + 1) * tpc);
           w.pad = chunks;
+          w.seq_start = c->cu[b]; w.seq_end = c->cu[b + 1]; w.blk_start = bs;
           items.push_back(w);
         }
       } else {
-        add_row_tiles(items, b, bs, bs + g.block_len, R, ITEM_BLOCK_CHUNK);
+        add_row_tiles(items, b, bs, bs + g.block_len, R, c->cu[b], c->cu[b + 1], bs, ITEM_BLOCK_CHUNK);
       }
     }
     int rows_off = (int)items.size();
     for (int b = 0; b < g.B; ++b) {
       int bs = c->blk_start_all[(size_t)k * g.B + b];
-      add_row_tiles(items, b, c->cu[b], bs, R);
-      add_row_tiles(items, b, bs + g.block_len, c->cu[b + 1], R);
+      add_row_tiles(items, b, c->cu[b], bs, R, c->cu[b], c->cu[b + 1], bs);
+      add_row_tiles(items, b, bs + g.block_len, c->cu[b + 1], R, c->cu[b], c->cu[b + 1], bs);
     }
-    c->step_list.push_back({off, (int)items.size() - off});
+    if (tc) {
+      c->step_list.push_back({off, rows_off - off});
+      c->merge_list.push_back({rows_off, (int)items.size() - rows_off});
+    } else {
+      c->step_list.push_back({off, (int)items.size() - off});
+      c->merge_list.push_back({0, 0});
+    }
     c->build_list.push_back({rows_off, (int)items.size() - rows_off});
   }
   {
     int off = (int)items.size();
-    for (int b = 0; b < g.B; ++b) add_row_tiles(items, b, c->cu[b], c->cu[b + 1], R);
+    for (int b = 0; b < g.B; ++b) add_row_tiles(items, b, c->cu[b], c->cu[b + 1], R, c->cu[b], c->cu[b + 1], 0);
     c->full_list = {off, (int)items.size() - off};
   }
+  c->items_host = items;
 
   // ---- device ----
   CU_TRY(c, cudaGetDevice(&c->device));
   cudaDeviceProp prop;
   CU_TRY(c, cudaGetDeviceProperties(&prop, c->device));
+  c->num_sms = prop.multiProcessorCount;
+  if (const char* e = getenv("LACACHE_STREAM_CTAS")) c->stream_ctas_override = atoi(e);
   if (tc && prop.major != 10)
     return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs an sm_100 device, found sm_%d%d", prop.major, prop.minor);
   CU_TRY(c, simt_prepare());
@@ -277,9 +296,9 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   CU_TRY(c, dev_alloc(c, &c->counters, (size_t)g.B * g.Hq, true));
   CU_TRY(c, dev_alloc(c, &c->d_status, 4, true));
   if (tc) {
-    c->maps = tc_make_maps(g, c->rot, c->err, sizeof(c->err));
+    c->maps = tc_make_maps(g, c->rot, c->st.o, c->err, sizeof(c->err));
     if (!c->maps) return LACACHE_ERR_CUDA;
-    c->maps_scratch = tc_make_maps(g, c->rot_scratch, c->err, sizeof(c->err));
+    c->maps_scratch = tc_make_maps(g, c->rot_scratch, c->st.o, c->err, sizeof(c->err));
     if (!c->maps_scratch) return LACACHE_ERR_CUDA;
   }
   CU_TRY(c, cudaDeviceSynchronize());
@@ -310,10 +329,42 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
   a.counters = c->counters;
   a.max_chunks = c->max_chunks;
   a.status = c->d_status;
+  if (c->engine == LACACHE_ENGINE_TCGEN05) {
+    // persistent grid: one CTA per SM, split between the two roles by a cost
+    // estimate (units x per-unit cost, in arbitrary time units)
+    const int Hq = c->g.Hq;
+    long long units_stream = (long long)list.n * Hq;
+    if (mode == MODE_STEP) {
+      lacache_ctx::ListRef ml = c->merge_list[blk];
+      a.items_merge = c->d_items + ml.off;
+      a.n_items_merge = ml.n;
+      long long units_merge = (long long)ml.n * Hq;
+      double cost_stream = 0.0;
+      for (int i = 0; i < list.n; ++i) {
+        const WorkItem& w = c->items_host[list.off + i];
+        cost_stream += Hq * (1.5 + 1.0 * (w.kt1 - w.kt0));
+      }
+      double cost_merge = 2.5 * (double)units_merge;
+      int total = (int)std::min<long long>(c->num_sms, units_stream + units_merge);
+      int ns = (int)lround(total * cost_stream / std::max(1e-9, cost_stream + cost_merge));
+      if (c->stream_ctas_override > 0) ns = c->stream_ctas_override;
+      if (units_merge == 0) ns = total;
+      else ns = std::max(1, std::min(ns, total - 1));
+      ns = (int)std::min<long long>(ns, units_stream);
+      a.n_ctas_stream = ns;
+      a.n_ctas = ns + (int)std::min<long long>(units_merge, std::max(0, c->num_sms - ns));
+    } else {
+      a.n_ctas_stream = (int)std::min<long long>(c->num_sms, units_stream);
+      a.n_ctas = a.n_ctas_stream;
+    }
+  }
   return a;
 }
 
 lacache_status run_attention(lacache_ctx* c, const AttnArgs& a, bool scratch, cudaStream_t s) {
+  if (c->engine == LACACHE_ENGINE_TCGEN05 && a.out) {
+    if (!tc_set_out(scratch ? c->maps_scratch : c->maps, c->g, a.out, c->err, sizeof(c->err))) return LACACHE_ERR_CUDA;
+  }
   if (c->ev_start) CU_TRY(c, cudaEventRecord(c->ev_start, s));
   if (c->engine == LACACHE_ENGINE_TCGEN05)
     CU_TRY(c, tc_attention(c->g, a, scratch ? c->maps_scratch : c->maps, s));

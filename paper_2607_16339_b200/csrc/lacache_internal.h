@@ -21,7 +21,11 @@ struct WorkItem {
   int32_t chunk;  // ITEM_BLOCK_CHUNK: chunk index; else 0
   int32_t kt0;    // ITEM_BLOCK_CHUNK: first key tile of the chunk
   int32_t kt1;    // ITEM_BLOCK_CHUNK: one past the last key tile
-  int32_t pad;
+  int32_t pad;    // ITEM_BLOCK_CHUNK: number of chunks of this (sequence, block)
+  int32_t seq_start;  // first packed token of the sequence
+  int32_t seq_end;    // one past its last token
+  int32_t blk_start;  // first packed token of the sequence's current block
+  int32_t pad2;
 };
 
 // What a launch computes for ITEM_ROWS items.
@@ -77,7 +81,10 @@ struct RopeArgs {
 
 struct AttnArgs {
   int mode;
-  const WorkItem* items; int n_items;
+  const WorkItem* items; int n_items;   // SIMT: all items; tcgen05: stream-role items
+  // tcgen05 only: items of the merge role (fixed rows of a step), CTA split
+  const WorkItem* items_merge; int n_items_merge;
+  int n_ctas_stream; int n_ctas;
   const int32_t* cu;         // [B+1]
   const int32_t* blk_start;  // [B] absolute token index of the block's first row
   RotBuffers rot;
@@ -109,7 +116,9 @@ cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* map
 cudaError_t tc_prepare();
 // builds TMA descriptors for a rotated buffer set; returns nullptr and fills
 // err on failure
-TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, char* err, int errlen);
+TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, char* err, int errlen);
+// (re)encodes the descriptor of the caller's output buffer when it changed
+bool tc_set_out(TcMaps* m, const Geometry& g, float* out, char* err, int errlen);
 void tc_free_maps(TcMaps* m);
 
 constexpr int SIMT_ROWS = 32;    // query rows per SIMT work item

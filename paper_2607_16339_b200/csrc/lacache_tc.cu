@@ -1,28 +1,35 @@
-// tcgen05 attention kernels for sm_100a (bf16 inputs, head_dim 128).
+// tcgen05 attention kernel for sm_100a (bf16 inputs, head_dim 128).
 //
-// One CTA owns a tile of 128 query rows of one (sequence, q head) and streams
-// key tiles of 64 keys through the online-softmax recurrence of Eq. 2-6:
-//   S  = Q' K'^T      tcgen05.mma kind::f16 (bf16 operands from shared memory,
-//                     fp32 accumulator in TMEM).  Rotated Q' and K' are stored
-//                     as hi + lo bf16 planes and the product is formed as
-//                     hi.hi + hi.lo + lo.hi so the scores carry ~16 significand
-//                     bits of each operand.
-//   P~ = exp2(S c - m) computed by 128 threads, one TMEM lane (= query row)
-//                     each, with an INTEGER reference exponent m (so every
-//                     rescale factor is an exact power of two), rounded to
-//                     fp16 and written back to TMEM.
-//   O~ += P~ V        tcgen05.mma with A = P~ read from TMEM and B = V (fp16,
-//                     MN-major) from shared memory.
-// Q, K and V tiles are staged by TMA (128-byte swizzle) and tracked by
-// mbarriers; every wait is bounded and reports through the status word.
+// One persistent CTA per SM, warp-specialised:
+//   warp 0 (one lane)  producer: TMA loads of Q, K, V tiles into shared memory
+//   warp 1 (one lane)  issues tcgen05.mma and commits completion to mbarriers
+//   warps 2..9         256 "row" threads: TMEM lane r = query row r of the
+//                      tile, two threads per row (each owns half of the
+//                      columns / features)
 //
-// The same kernel runs all modes (what the key range is, where the state
-// starts and where the result goes):
-//   build : rows in U, keys in U                    -> cached (m, l, O~)
-//   step  : rows in U start from the cache, keys = the block        -> out
-//           rows in C, keys = one chunk of all keys -> partial state; the
-//           last chunk to arrive merges the partials                -> out
-//   full  : all rows, all keys                                      -> out
+// Arithmetic (Eq. 2-6 with base-2 exponentials):
+//   S  = Q' K'^T   kind::f16 MMA on bf16 operands from shared memory, fp32
+//                  accumulator in TMEM.  Rotated Q', K' are stored as
+//                  hi + lo bf16 planes; S = hi.hi + hi.lo + lo.hi.
+//   P~ = 2^(S c - m), m an INTEGER reference exponent (every rescale factor is
+//                  an exact power of two), rounded to fp16, written to TMEM.
+//   O~ = P~ V      MMA with A = P~ from TMEM, B = V (fp16, MN-major) from
+//                  shared memory.  The normaliser sums the rounded P~.
+//
+// Two roles, chosen per CTA:
+//   stream role  a tile of 128 (or 64) query rows streams key tiles of 64
+//                keys through a 2-stage K/V ring; used for the cache build
+//                (rows in U x keys in U -> cached state), the full recompute,
+//                and the block queries of a step (one chunk of key tiles per
+//                work unit; the last chunk to finish merges the partials).
+//   merge role   the reuse pass for fixed queries: per tile of 128 rows, the
+//                scores against the block's keys, then
+//                out = (alpha O~_cache + P~ V) / (alpha l_cache + sum P~).
+//                O~_cache rows come in and out rows go out as bulk async
+//                copies through a padded staging buffer, so all cache traffic
+//                is coalesced and asynchronous.
+// Every mbarrier wait is bounded; a wait that runs out sets the status word
+// and the CTA unwinds (TMEM is always freed).
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <stdio.h>
@@ -32,46 +39,62 @@
 namespace lacache {
 
 struct TcMaps {
-  alignas(64) CUtensorMap q_hi;
+  alignas(64) CUtensorMap q_hi;    // box 128 rows
   alignas(64) CUtensorMap q_lo;
-  alignas(64) CUtensorMap k_hi;
+  alignas(64) CUtensorMap q64_hi;  // box 64 rows (block queries)
+  alignas(64) CUtensorMap q64_lo;
+  alignas(64) CUtensorMap k_hi;    // box 64 rows
   alignas(64) CUtensorMap k_lo;
   alignas(64) CUtensorMap v;
+  alignas(64) CUtensorMap st_o;    // cached O~ [Hq][Tp][128] fp32, box 32 cols x 128 rows
+  alignas(64) CUtensorMap out;     // caller's out [T][Hq][128] fp32, box 32 cols x 1 head x 128 rows
+  const void* out_ptr;             // the buffer `out` was encoded for
 };
 
 namespace {
 
 constexpr int D = 128;
-constexpr int BM = TC_ROWS;   // 128 query rows
-constexpr int BN = TC_KEYS;   // 64 keys
-constexpr int THREADS = 128;
+constexpr int BM = TC_ROWS;   // 128 query rows (TMEM lanes)
+constexpr int BN = TC_KEYS;   // 64 keys per tile
+constexpr int ROW_WARPS = 8;
+constexpr int ROW_THREADS = ROW_WARPS * 32;
+constexpr int THREADS = 64 + ROW_THREADS;
 
-// shared memory map (bytes, from a 1024-aligned base)
-constexpr uint32_t SM_QHI = 0;                    // 2 boxes [128 rows][64 cols] bf16
-constexpr uint32_t SM_QLO = SM_QHI + 32768;
-constexpr uint32_t SM_KHI = SM_QLO + 32768;       // 2 boxes [64 rows][64 cols] bf16
-constexpr uint32_t SM_KLO = SM_KHI + 16384;
-constexpr uint32_t SM_V = SM_KLO + 16384;         // 2 boxes [64 keys][64 cols] fp16
-constexpr uint32_t SM_BAR = SM_V + 16384;         // mbarriers + small words
-constexpr uint32_t SM_TOTAL = SM_BAR + 128;
-constexpr uint32_t Q_BOX_BYTES = 128 * 128;       // 128 rows x 128 B
-constexpr uint32_t K_BOX_BYTES = 64 * 128;
+// ---- shared memory map (bytes from a 1024-aligned base) ----
+constexpr uint32_t SM_Q = 0;                      // hi plane, then lo plane at +32 KB
+constexpr uint32_t SM_Q_LO = 32768;
+constexpr uint32_t SM_KV = 65536;                 // 2 stages of {K hi, K lo, V}
+constexpr uint32_t KV_STAGE = 49152;
+constexpr uint32_t KV_KLO = 16384;
+constexpr uint32_t KV_V = 32768;
+constexpr uint32_t K_BOX = 64 * 128;              // one [64 rows][64 cols] 16-bit box
+constexpr uint32_t SM_IO = SM_KV + 2 * KV_STAGE;  // staging: 128 rows x (512 + 16) bytes
+constexpr uint32_t IO_ROW = 528;
+constexpr uint32_t IO_BOX = 128 * 128;             // merge role: one swizzled box of 32 fp32 columns x 128 rows
+constexpr uint32_t SM_BAR = SM_IO + BM * IO_ROW;
+constexpr uint32_t SM_TOTAL = SM_BAR + 256;
+static_assert(SM_TOTAL <= 232448, "exceeds the 227 KB per-CTA limit");
 
-// TMEM columns (fp32 words per lane)
-constexpr uint32_t TM_S = 0;      // 64 columns: scores
-constexpr uint32_t TM_P = 64;     // 32 columns: 64 fp16 probabilities, packed
-constexpr uint32_t TM_O = 128;    // 128 columns: P.V of the current tile
-constexpr uint32_t TM_COLS = 256;
+// ---- TMEM columns ----
+constexpr uint32_t TM_S = 0;      // 2 x 64: scores
+constexpr uint32_t TM_P = 128;    // 2 x 32: fp16 probabilities, two per column
+constexpr uint32_t TM_O = 256;    // 2 x 128: P.V of one tile
+constexpr uint32_t TM_COLS = 512;
 
-// barrier slots
-enum { BAR_Q = 0, BAR_K, BAR_V, BAR_S, BAR_O, BAR_SYNC, BAR_DONE, N_BARS };
+enum {
+  BAR_Q_FULL = 0, BAR_Q_FREE,
+  BAR_KV_FULL, BAR_KV_FULL1, BAR_KV_FREE, BAR_KV_FREE1,
+  BAR_S_FULL, BAR_S_FULL1, BAR_P_FULL, BAR_P_FULL1,
+  BAR_O_FULL, BAR_O_FULL1, BAR_O_FREE, BAR_O_FREE1,
+  BAR_IO_FULL, BAR_IO_FREE, BAR_EPI, BAR_DONE, N_BARS
+};
 
-constexpr long long WAIT_CYCLES = 3000000000ll;  // ~1.5 s at 2 GHz
+enum { EPI_STATE = 0, EPI_OUT = 1, EPI_PARTIAL = 2 };
+
+constexpr long long WAIT_CYCLES = 4000000000ll;  // ~2 s
 
 // ---- PTX wrappers ----------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
@@ -92,19 +115,47 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
-                                            int c1, int c2) {
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {  // non-blocking
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(map),
+               "r"(src), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+// untiled bulk copies: both addresses 16-byte aligned, size a multiple of 16
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                        uint32_t accumulate) {
   asm volatile(
@@ -114,7 +165,6 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem]
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
                                        uint32_t accumulate) {
   asm volatile(
@@ -152,108 +202,681 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// shared-memory matrix descriptor, 128-byte swizzle, sm_100 version field
+// p rounded to 11 significant bits (what fp16 keeps) with plain fp32 arithmetic
+// (Veltkamp split), so the fp16 conversion that follows is exact and the
+// normaliser can sum the very values the MMA multiplies without converting back.
+__device__ __forceinline__ float round_to_half_bits(float p) {
+  float c = __fmul_rn(p, 8193.0f);
+  return __fsub_rn(c, __fsub_rn(c, p));
+}
+__device__ __forceinline__ WorkItem load_item(const WorkItem* p) {
+  const int4* q = reinterpret_cast<const int4*>(p);
+  int4 a = __ldg(q), b = __ldg(q + 1), c = __ldg(q + 2);
+  WorkItem w;
+  w.kind = a.x; w.seq = a.y; w.row0 = a.z; w.nrows = a.w;
+  w.chunk = b.x; w.kt0 = b.y; w.kt1 = b.z; w.pad = b.w;
+  w.seq_start = c.x; w.seq_end = c.y; w.blk_start = c.z; w.pad2 = c.w;
+  return w;
+}
+
+// shared-memory matrix descriptor: 128-byte swizzle, sm_100 descriptor version
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
          ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
 }
-// instruction descriptor for kind::f16: fp32 accumulate, M x N
-constexpr uint32_t idesc_f16(uint32_t ab_format, uint32_t b_mn_major, uint32_t M, uint32_t N) {
-  return (1u << 4) | (ab_format << 7) | (ab_format << 10) | (b_mn_major << 16) | ((N >> 3) << 17) |
-         ((M >> 4) << 24);
+// kind::f16 instruction descriptor: fp32 accumulate; A/B format 0 = fp16, 1 = bf16
+__host__ __device__ constexpr uint32_t idesc_f16(uint32_t ab_format, uint32_t b_mn_major, uint32_t M, uint32_t N) {
+  return (1u << 4) | (ab_format << 7) | (ab_format << 10) | (b_mn_major << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
-constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
-constexpr uint32_t IDESC_PV = idesc_f16(0u /*f16*/, 1u, BM, D);
 
-struct Shared {
-  uint32_t base;       // shared-space address of the 1024-aligned region
+#ifdef LACACHE_DEBUG_CLOCKS
+__device__ long long g_dbg_clocks[256 * 64];
+#define DBG_CLK(k) do { if ((k) < 64) g_dbg_clocks[(size_t)blockIdx.x * 64 + (k)] = clock64(); } while (0)
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define DBG_GT(k) do { g_dbg_clocks[(size_t)blockIdx.x * 64 + (k)] = gtime(); } while (0)
+#else
+#define DBG_CLK(k) do { } while (0)
+#define DBG_GT(k) do { } while (0)
+#endif
+
+struct Cta {
+  uint32_t base;            // shared-space address of the region
+  uint8_t* gen;             // generic pointer to the same region
+  uint32_t tmem;            // TMEM base address
   volatile int* abort_flag;
+  volatile uint32_t* flag;  // scratch word for CTA-wide decisions
   int32_t* status;
+  __device__ __forceinline__ uint32_t bar(int slot) const { return base + SM_BAR + 8u * slot; }
 };
 
-// Bounded wait: false if the barrier did not complete in time or another
-// thread of the CTA already gave up.
-__device__ __forceinline__ bool wait_bar(const Shared& sh, int slot, uint32_t parity, int loc) {
-  uint32_t bar = sh.base + SM_BAR + 8u * slot;
-  if (mbar_try(bar, parity)) return true;
+// Bounded wait on phase `parity`; false if it ran out or the CTA is unwinding.
+__device__ __noinline__ bool wait_slow(const Cta& c, uint32_t bar, uint32_t parity, int loc) {
   long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
-    for (int i = 0; i < 64; ++i)
+    for (int i = 0; i < 32; ++i)
       if (mbar_try(bar, parity)) return true;
-    if (*sh.abort_flag) return false;
+    if (*c.abort_flag) return false;
     if (clock64() - t0 > WAIT_CYCLES) {
-      *sh.abort_flag = 1;
-      if (atomicCAS(sh.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
-        sh.status[1] = loc;
-        sh.status[2] = blockIdx.x;
-        sh.status[3] = threadIdx.x;
+      *c.abort_flag = 1;
+      if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
+        c.status[1] = loc;
+        c.status[2] = blockIdx.x;
+        c.status[3] = threadIdx.x;
       }
       return false;
     }
   }
 }
+__device__ __forceinline__ bool wait_bar(const Cta& c, int slot, uint32_t parity, int loc) {
+  uint32_t b = c.bar(slot);
+  if (mbar_try(b, parity)) return true;
+  return wait_slow(c, b, parity, loc);
+}
 
-__global__ void __launch_bounds__(THREADS, 2)
+// One unit of work of the stream role, decoded identically by every warp role.
+struct Unit {
+  int row0, nrows, h, kh, seq;
+  int key_base, t0, t1;   // key tiles [t0, t1): tile t holds keys key_base + 64 t ...
+  int k0, k1, x0, x1;     // valid keys [k0, k1) minus [x0, x1)
+  int epi, chunk, nchunks;
+  int q_rows;             // rows of the Q box: 128 or 64
+};
+
+__device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs& a, const WorkItem& it, int u) {
+  Unit un;
+  un.h = u / a.n_items;
+  un.kh = un.h / g.group;
+  un.seq = it.seq;
+  un.row0 = it.row0;
+  un.nrows = it.nrows;
+  un.key_base = it.seq_start;
+  un.k0 = it.seq_start;
+  un.k1 = it.seq_end;
+  un.x0 = un.x1 = 0;
+  un.t0 = 0;
+  un.t1 = (it.seq_end - it.seq_start + BN - 1) / BN;
+  un.chunk = 0;
+  un.nchunks = 1;
+  un.q_rows = BM;
+  if (a.mode == MODE_BUILD) {
+    un.x0 = it.blk_start;
+    un.x1 = it.blk_start + g.block_len;
+    un.epi = EPI_STATE;
+  } else if (a.mode == MODE_STEP) {
+    un.t0 = it.kt0;
+    un.t1 = it.kt1;
+    un.chunk = it.chunk;
+    un.nchunks = it.pad;
+    un.epi = it.pad > 1 ? EPI_PARTIAL : EPI_OUT;
+    un.q_rows = 64;
+  } else {
+    un.epi = EPI_OUT;
+  }
+  return un;
+}
+__device__ __forceinline__ bool tile_skipped(const Unit& un, int t) {
+  int lo = un.key_base + t * BN, hi = min(lo + BN, un.k1);
+  return un.x1 > un.x0 && lo >= un.x0 && hi <= un.x1;
+}
+__device__ __forceinline__ int next_tile(const Unit& un, int t) {
+  while (t < un.t1 && tile_skipped(un, t)) ++t;
+  return t;
+}
+
+__device__ __forceinline__ void issue_s_mma(const Cta& c, uint32_t kv_base, uint32_t s_tmem, uint32_t q_box,
+                                            uint32_t idesc) {
+  uint32_t acc = 0;
+#pragma unroll
+  for (int term = 0; term < 3; ++term) {  // hi.hi, hi.lo, lo.hi
+    const uint32_t qa = c.base + SM_Q + (term == 2 ? SM_Q_LO : 0u);
+    const uint32_t ka = kv_base + (term == 1 ? KV_KLO : 0u);
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+      uint32_t qoff = (ks >> 2) * q_box + (ks & 3) * 32;
+      uint32_t koff = (ks >> 2) * K_BOX + (ks & 3) * 32;
+      mma_ss(s_tmem, smem_desc(qa + qoff, 16, 1024), smem_desc(ka + koff, 16, 1024), idesc, acc);
+      acc = 1;
+    }
+  }
+}
+__device__ __forceinline__ void issue_pv_mma(uint32_t kv_base, uint32_t p_tmem, uint32_t o_tmem, int ksteps) {
+  constexpr uint32_t idesc = idesc_f16(0u /*fp16*/, 1u, BM, D);
+  for (int ks = 0; ks < ksteps; ++ks) {
+    // B = V tile, MN-major: 64 features contiguous (128 B), the next 64 features
+    // 8 KB further (LBO), groups of 8 keys 1 KB apart (SBO); 16 keys = 2 KB.
+    mma_ts(o_tmem, p_tmem + 8 * ks, smem_desc(kv_base + KV_V + ks * 2048, K_BOX, 1024), idesc, ks > 0 ? 1u : 0u);
+  }
+}
+__device__ __forceinline__ void load_kv_tile(const TcMaps& maps, uint32_t kv_base, uint32_t bar, int krow, int kh) {
+  mbar_expect_tx(bar, 6 * K_BOX);
+  tma_load_3d(kv_base, &maps.k_hi, bar, 0, krow, kh);
+  tma_load_3d(kv_base + K_BOX, &maps.k_hi, bar, 64, krow, kh);
+  tma_load_3d(kv_base + KV_KLO, &maps.k_lo, bar, 0, krow, kh);
+  tma_load_3d(kv_base + KV_KLO + K_BOX, &maps.k_lo, bar, 64, krow, kh);
+  tma_load_3d(kv_base + KV_V, &maps.v, bar, 0, krow, kh);
+  tma_load_3d(kv_base + KV_V + K_BOX, &maps.v, bar, 64, krow, kh);
+}
+__device__ __forceinline__ void load_q_tile(const Cta& c, const TcMaps& maps, int q_rows, int row0, int h) {
+  const uint32_t bar = c.bar(BAR_Q_FULL);
+  const uint32_t box = (uint32_t)q_rows * 128u;
+  const CUtensorMap* mh = q_rows == 64 ? &maps.q64_hi : &maps.q_hi;
+  const CUtensorMap* ml = q_rows == 64 ? &maps.q64_lo : &maps.q_lo;
+  mbar_expect_tx(bar, 4 * box);
+  tma_load_3d(c.base + SM_Q, mh, bar, 0, row0, h);
+  tma_load_3d(c.base + SM_Q + box, mh, bar, 64, row0, h);
+  tma_load_3d(c.base + SM_Q + SM_Q_LO, ml, bar, 0, row0, h);
+  tma_load_3d(c.base + SM_Q + SM_Q_LO + box, ml, bar, 64, row0, h);
+}
+
+// ===========================================================================
+// stream role
+// ===========================================================================
+__device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a,
+                                int first, int stride, int n_units, WorkItem it) {
+  int uu = 0, jj = 0;
+  for (int u = first; u < n_units; u += stride, ++uu) {
+    WorkItem nxt = it;
+    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
+    const Unit un = decode_stream(g, a, it, u);
+    if (uu >= 1 && !wait_bar(c, BAR_Q_FREE, (uu - 1) & 1, LOC_WAIT_Q)) return;
+    load_q_tile(c, maps, un.q_rows, un.row0, un.h);
+    for (int t = next_tile(un, un.t0); t < un.t1; t = next_tile(un, t + 1), ++jj) {
+      const int b = jj & 1, k = jj >> 1;
+      if (k >= 1 && !wait_bar(c, BAR_KV_FREE + b, (k - 1) & 1, LOC_WAIT_K)) return;
+      load_kv_tile(maps, c.base + SM_KV + b * KV_STAGE, c.bar(BAR_KV_FULL + b), un.key_base + t * BN, un.kh);
+    }
+    it = nxt;
+  }
+}
+
+// The MMA thread issues whichever product is ready: P~V of the oldest pending
+// tile as soon as its probabilities are in TMEM, else the scores of the next
+// tile as soon as its keys have landed (at most two score tiles in flight).
+__device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units,
+                           WorkItem it) {
+  constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
+  int uu = 0, js = 0, jp = 0;  // global counters of score tiles / PV tiles issued
+  for (int u = first; u < n_units; u += stride, ++uu) {
+    WorkItem nxt = it;
+    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
+    const Unit un = decode_stream(g, a, it, u);
+    const uint32_t q_box = (uint32_t)un.q_rows * 128u;
+    if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
+    int ts = next_tile(un, un.t0), tp = ts;
+    bool q_released = false;
+    long long t_idle = 0;
+    while (tp < un.t1) {
+      bool did = false;
+      if (js > jp) {  // scores of tile jp issued: its P~V may be ready
+        const int b = jp & 1, k = jp >> 1;
+        if (mbar_test(c.bar(BAR_P_FULL + b), k & 1) && (k < 1 || mbar_test(c.bar(BAR_O_FREE + b), (k - 1) & 1))) {
+          tc_fence_after();
+          issue_pv_mma(c.base + SM_KV + b * KV_STAGE, c.tmem + TM_P + 32 * b, c.tmem + TM_O + 128 * b, BN / 16);
+          tc_commit(c.bar(BAR_O_FULL + b));
+          tc_commit(c.bar(BAR_KV_FREE + b));
+          tp = next_tile(un, tp + 1);
+          ++jp;
+          did = true;
+        }
+      }
+      if (!did && ts < un.t1 && js - jp < 2) {
+        const int b = js & 1;
+        if (mbar_test(c.bar(BAR_KV_FULL + b), (js >> 1) & 1)) {
+          tc_fence_after();
+          issue_s_mma(c, c.base + SM_KV + b * KV_STAGE, c.tmem + TM_S + 64 * b, q_box, IDESC_S);
+          tc_commit(c.bar(BAR_S_FULL + b));
+          ts = next_tile(un, ts + 1);
+          ++js;
+          if (ts >= un.t1) {  // every score MMA of this unit has been issued
+            tc_commit(c.bar(BAR_Q_FREE));
+            q_released = true;
+          }
+          did = true;
+        }
+      }
+      if (did) {
+        t_idle = 0;
+      } else {  // nothing ready: bounded idle
+        if (t_idle == 0) t_idle = clock64();
+        if (*c.abort_flag) return;
+        if (clock64() - t_idle > WAIT_CYCLES) {
+          *c.abort_flag = 1;
+          if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
+            c.status[1] = LOC_WAIT_S; c.status[2] = blockIdx.x; c.status[3] = threadIdx.x;
+          }
+          return;
+        }
+      }
+    }
+    if (!q_released) tc_commit(c.bar(BAR_Q_FREE));  // a unit without key tiles
+    it = nxt;
+  }
+}
+
+// CTA-wide rendezvous of the row threads (bounded)
+__device__ __forceinline__ bool epi_sync(const Cta& c, uint32_t& phase) {
+  mbar_arrive(c.bar(BAR_EPI));
+  bool ok = wait_bar(c, BAR_EPI, phase & 1, LOC_WAIT_O);
+  ++phase;
+  return ok;
+}
+
+// Writes this thread's 64 features (times mul) into its staging half-row and
+// sends them to global memory as one 256-byte bulk copy.
+__device__ __forceinline__ void stage_and_store(const Cta& c, int r, int half, const float (&o)[64], float mul,
+                                                float* gdst, bool valid) {
+  bulk_wait_read();  // an earlier copy out of this half-row must have been read
+  const uint32_t off = SM_IO + r * IO_ROW + half * 256;
+  float4* s4 = reinterpret_cast<float4*>(c.gen + off);
+#pragma unroll
+  for (int i = 0; i < 16; ++i)
+    s4[i] = make_float4(o[4 * i] * mul, o[4 * i + 1] * mul, o[4 * i + 2] * mul, o[4 * i + 3] * mul);
+  fence_async_smem();
+  if (valid) {
+    bulk_store(gdst, c.base + off, 256);
+    bulk_commit();
+  }
+}
+
+__device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units,
+                            WorkItem it) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int quad = warp & 3;
+  const int half = (warp - 2) >> 2;         // 0: columns/features of the first half, 1: the rest
+  const int r = quad * 32 + lane;           // row of the tile = TMEM lane
+  const uint32_t tlane = c.tmem + ((uint32_t)(quad * 32) << 16);
+  const float LN2 = 0.69314718055994530942f;
+  volatile float* xch = reinterpret_cast<volatile float*>(c.gen + SM_IO + r * IO_ROW + 512);  // row padding
+  uint32_t epi_phase = 0, epi_unit = 0;
+  int jj = 0;
+  for (int u = first; u < n_units; u += stride) {
+    WorkItem nxt = it;
+    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
+    const Unit un = decode_stream(g, a, it, u);
+    it = nxt;
+    const int row = un.row0 + r;
+    const bool row_valid = r < un.nrows;
+    float m_run = -INFINITY, l_part = 0.f;
+    float o_acc[64];
+#pragma unroll
+    for (int i = 0; i < 64; ++i) o_acc[i] = 0.f;
+
+    for (int t = next_tile(un, un.t0); t < un.t1; t = next_tile(un, t + 1), ++jj) {
+      const int b = jj & 1, par = (jj >> 1) & 1;
+      const int tile_lo = un.key_base + t * BN;
+      const int v_lo = max(un.k0 - tile_lo, 0), v_hi = min(un.k1 - tile_lo, BN);
+      const int e_lo = un.x0 - tile_lo, e_hi = un.x1 - tile_lo;
+      const bool all_valid = v_lo == 0 && v_hi == BN && (un.x1 <= un.x0 || e_hi <= 0 || e_lo >= BN);
+      auto col_valid = [&](int j) { return j >= v_lo && j < v_hi && !(j >= e_lo && j < e_hi); };
+      if (!wait_bar(c, BAR_S_FULL + b, par, LOC_WAIT_S)) return;
+      tc_fence_after();
+      // row maximum over all 64 columns (both threads of the pair compute it);
+      // the thread's own 32 columns are read last and kept
+      float mx = -INFINITY;
+      uint32_t rr[32];
+      {
+        const int oc = 32 * (1 - half);
+        tmem_ld32(tlane + TM_S + 64 * b + oc, rr);
+        tmem_ld_wait();
+        if (all_valid) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(rr[j]));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (col_valid(oc + j)) mx = fmaxf(mx, __uint_as_float(rr[j]));
+        }
+      }
+      const int mc = 32 * half;
+      tmem_ld32(tlane + TM_S + 64 * b + mc, rr);
+      tmem_ld_wait();
+      if (all_valid) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(rr[j]));
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (col_valid(mc + j)) mx = fmaxf(mx, __uint_as_float(rr[j]));
+      }
+      const float m_new = fmaxf(m_run, ceilf(mx * g.scale_log2));
+      const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+      const float alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - m_new);
+      // probabilities of this thread's 32 columns
+      float psum = 0.f;
+      uint32_t pk[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        float p0 = ex2(fmaf(__uint_as_float(rr[2 * j]), g.scale_log2, -m_ref));
+        float p1 = ex2(fmaf(__uint_as_float(rr[2 * j + 1]), g.scale_log2, -m_ref));
+        if (!all_valid) {
+          if (!col_valid(mc + 2 * j)) p0 = 0.f;
+          if (!col_valid(mc + 2 * j + 1)) p1 = 0.f;
+        }
+        p0 = round_to_half_bits(p0);
+        p1 = round_to_half_bits(p1);
+        psum += p0 + p1;  // the normaliser sums exactly what the MMA multiplies
+        __half2 hp = __floats2half2_rn(p0, p1);
+        pk[j] = *reinterpret_cast<uint32_t*>(&hp);
+      }
+      tmem_st16(tlane + TM_P + 32 * b + 16 * half, pk);
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(c.bar(BAR_P_FULL + b));
+      l_part = l_part * alpha + psum;
+      m_run = m_new;
+      // O~ = alpha O~ + P~ V for this thread's 64 features
+      if (!wait_bar(c, BAR_O_FULL + b, par, LOC_WAIT_O)) return;
+      tc_fence_after();
+#pragma unroll
+      for (int q2 = 0; q2 < 2; ++q2) {
+        tmem_ld32(tlane + TM_O + 128 * b + 64 * half + 32 * q2, rr);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) o_acc[32 * q2 + j] = fmaf(o_acc[32 * q2 + j], alpha, __uint_as_float(rr[j]));
+      }
+      tc_fence_before();
+      mbar_arrive(c.bar(BAR_O_FREE + b));
+    }
+
+    // ---- epilogue: combine the pair's normaliser, then store ----
+    // (slots alternate between consecutive units so a fast thread of the next
+    // unit cannot overwrite a value its partner has not read yet)
+    const int xs = 2 * (int)(epi_unit & 1u);
+    ++epi_unit;
+    xch[xs + half] = l_part;
+    if (!epi_sync(c, epi_phase)) return;
+    const float l_run = xch[xs] + xch[xs + 1];
+    if (un.epi == EPI_STATE) {
+      size_t srow = (size_t)un.h * g.Tp + row;
+      if (row_valid && half == 0) { a.st.m[srow] = m_run; a.st.l[srow] = l_run; }
+      stage_and_store(c, r, half, o_acc, 1.f, a.st.o + srow * D + 64 * half, row_valid);
+    } else if (un.epi == EPI_OUT) {
+      size_t orow = (size_t)row * g.Hq + un.h;
+      if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_run + log2f(l_run)) * LN2;
+      stage_and_store(c, r, half, o_acc, 1.f / l_run, a.out + orow * D + 64 * half, row_valid);
+    } else {
+      // partial state of this key chunk; the last chunk of the (sequence, head)
+      // to arrive merges all of them
+      const size_t p0 = (((size_t)un.seq * g.Hq + un.h) * a.max_chunks) * g.block_len + r;
+      if (row_valid) {
+        const size_t pr = p0 + (size_t)un.chunk * g.block_len;
+        if (half == 0) { a.part_m[pr] = m_run; a.part_l[pr] = l_run; }
+        float4* dst = reinterpret_cast<float4*>(a.part_o + pr * D + 64 * half);
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          dst[i] = make_float4(o_acc[4 * i], o_acc[4 * i + 1], o_acc[4 * i + 2], o_acc[4 * i + 3]);
+      }
+      __threadfence();
+      if (!epi_sync(c, epi_phase)) return;
+      if (threadIdx.x == 64) {
+        int* cnt = &a.counters[un.seq * g.Hq + un.h];
+        int old = atomicAdd(cnt, 1);
+        int last = (old == un.nchunks - 1) ? 1 : 0;
+        if (last) *cnt = 0;
+        *c.flag = (uint32_t)last;
+        __threadfence();
+      }
+      if (!epi_sync(c, epi_phase)) return;
+      // the flag is rewritten only after every row thread has passed two more
+      // rendezvous of a later unit, so reading it here is race-free
+      const bool last = *c.flag != 0;
+      if (last) {
+        __threadfence();
+        float M = -INFINITY, L = 0.f;
+        if (row_valid) {
+          for (int ch = 0; ch < un.nchunks; ++ch) M = fmaxf(M, __ldcg(a.part_m + p0 + (size_t)ch * g.block_len));
+#pragma unroll
+          for (int i = 0; i < 64; ++i) o_acc[i] = 0.f;
+          for (int ch = 0; ch < un.nchunks; ++ch) {
+            const size_t pr = p0 + (size_t)ch * g.block_len;
+            const float mcv = __ldcg(a.part_m + pr);
+            if (mcv == -INFINITY) continue;
+            const float w = ex2(mcv - M);
+            L = fmaf(__ldcg(a.part_l + pr), w, L);
+            const float4* src = reinterpret_cast<const float4*>(a.part_o + pr * D + 64 * half);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              float4 v = __ldcg(src + i);
+              o_acc[4 * i] = fmaf(v.x, w, o_acc[4 * i]);
+              o_acc[4 * i + 1] = fmaf(v.y, w, o_acc[4 * i + 1]);
+              o_acc[4 * i + 2] = fmaf(v.z, w, o_acc[4 * i + 2]);
+              o_acc[4 * i + 3] = fmaf(v.w, w, o_acc[4 * i + 3]);
+            }
+          }
+        }
+        size_t orow = (size_t)row * g.Hq + un.h;
+        if (row_valid && half == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
+        stage_and_store(c, r, half, o_acc, row_valid ? 1.f / L : 0.f, a.out + orow * D + 64 * half, row_valid);
+      }
+    }
+  }
+}
+
+// ===========================================================================
+// merge role: fixed queries x block keys, merged into the cached state
+// ===========================================================================
+__device__ void merge_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a, int first,
+                               int stride, int n_units, WorkItem it) {
+  int uu = 0;
+  for (int u = first; u < n_units; u += stride, ++uu) {
+    WorkItem nxt = it;
+    if (u + stride < n_units) nxt = load_item(a.items_merge + (u + stride) % a.n_items_merge);
+    const int h = u / a.n_items_merge;
+    const int b = uu & 1, k = uu >> 1;
+    if (uu >= 1 && !wait_bar(c, BAR_Q_FREE, (uu - 1) & 1, LOC_WAIT_Q)) return;
+    load_q_tile(c, maps, BM, it.row0, h);
+    if (k >= 1 && !wait_bar(c, BAR_KV_FREE + b, (k - 1) & 1, LOC_WAIT_K)) return;
+    load_kv_tile(maps, c.base + SM_KV + b * KV_STAGE, c.bar(BAR_KV_FULL + b), it.blk_start, h / g.group);
+    // cached O~ tile: four boxes of 32 features x 128 rows (rows past nrows are
+    // read but never used)
+    if (uu >= 1 && !wait_bar(c, BAR_IO_FREE, (uu - 1) & 1, LOC_WAIT_V)) return;
+    mbar_expect_tx(c.bar(BAR_IO_FULL), 4 * IO_BOX);
+#pragma unroll
+    for (int cb = 0; cb < 4; ++cb)
+      tma_load_3d(c.base + SM_IO + cb * IO_BOX, &maps.st_o, c.bar(BAR_IO_FULL), 32 * cb, it.row0, h);
+    it = nxt;
+  }
+}
+
+__device__ void merge_mma(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units) {
+  const int n_s = (g.block_len + 15) & ~15;  // score columns (keys), a multiple of 16
+  const uint32_t idesc_s = idesc_f16(1u, 0u, BM, (uint32_t)n_s);
+  int uu = 0;
+  if (first < n_units) {
+    if (!wait_bar(c, BAR_Q_FULL, 0, LOC_WAIT_Q)) return;
+    if (!wait_bar(c, BAR_KV_FULL, 0, LOC_WAIT_K)) return;
+    tc_fence_after();
+    issue_s_mma(c, c.base + SM_KV, c.tmem + TM_S, BM * 128u, idesc_s);
+    tc_commit(c.bar(BAR_S_FULL));
+    tc_commit(c.bar(BAR_Q_FREE));
+  }
+  for (int u = first; u < n_units; u += stride, ++uu) {
+    const int b = uu & 1, k = uu >> 1;
+    if (!wait_bar(c, BAR_P_FULL + b, k & 1, LOC_WAIT_S)) return;
+    if (k >= 1 && !wait_bar(c, BAR_O_FREE + b, (k - 1) & 1, LOC_WAIT_O)) return;
+    tc_fence_after();
+    issue_pv_mma(c.base + SM_KV + b * KV_STAGE, c.tmem + TM_P + 32 * b, c.tmem + TM_O + 128 * b, n_s / 16);
+    tc_commit(c.bar(BAR_O_FULL + b));
+    tc_commit(c.bar(BAR_KV_FREE + b));
+    if (u + stride < n_units) {  // scores of the next unit as soon as its tiles land
+      const int bn = (uu + 1) & 1;
+      if (!wait_bar(c, BAR_Q_FULL, (uu + 1) & 1, LOC_WAIT_Q)) return;
+      if (!wait_bar(c, BAR_KV_FULL + bn, ((uu + 1) >> 1) & 1, LOC_WAIT_K)) return;
+      tc_fence_after();
+      issue_s_mma(c, c.base + SM_KV + bn * KV_STAGE, c.tmem + TM_S + 64 * bn, BM * 128u, idesc_s);
+      tc_commit(c.bar(BAR_S_FULL + bn));
+      tc_commit(c.bar(BAR_Q_FREE));
+    }
+  }
+}
+
+__device__ void merge_rows(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a, int first,
+                           int stride, int n_units, WorkItem it) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int quad = warp & 3;
+  const int half = (warp - 2) >> 2;
+  const int r = quad * 32 + lane;
+  const uint32_t tlane = c.tmem + ((uint32_t)(quad * 32) << 16);
+  const float LN2 = 0.69314718055994530942f;
+  const int n_s = (g.block_len + 15) & ~15;
+  const int L = g.block_len;
+  // staging layout (as TMA writes and reads it): box cb = features [32 cb, 32 cb + 32),
+  // row r at +128 r, its 16-byte chunk j at ((j ^ (r & 7)) << 4)
+  uint8_t* const sbox = c.gen + SM_IO + (2 * half) * IO_BOX + r * 128;
+  const int sw = r & 7;
+  uint32_t epi_phase = 0;
+  int uu = 0;
+  for (int u = first; u < n_units; u += stride, ++uu) {
+    WorkItem nxt = it;
+    if (u + stride < n_units) nxt = load_item(a.items_merge + (u + stride) % a.n_items_merge);
+    const int h = u / a.n_items_merge;
+    const int b = uu & 1, par = (uu >> 1) & 1;
+    const int row = it.row0 + r;
+    const bool row_valid = r < it.nrows;
+    const size_t srow = (size_t)h * g.Tp + row;
+    float m_c = -INFINITY, l_c = 0.f;
+    if (row_valid) { m_c = __ldg(a.st.m + srow); l_c = __ldg(a.st.l + srow); }
+
+    if (!wait_bar(c, BAR_S_FULL + b, par, LOC_WAIT_S)) return;
+    tc_fence_after();
+    // scores against the block's keys: columns [0, block_len) are valid
+    float mx = -INFINITY;
+    uint32_t s0[32], s1[32];
+    tmem_ld32(tlane + TM_S + 64 * b, s0);
+    if (n_s > 32) tmem_ld32(tlane + TM_S + 64 * b + 32, s1);
+    tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j < L) mx = fmaxf(mx, __uint_as_float(s0[j]));
+    if (n_s > 32) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (32 + j < L) mx = fmaxf(mx, __uint_as_float(s1[j]));
+    }
+    const float m_new = fmaxf(m_c, ceilf(mx * g.scale_log2));
+    const float alpha = (m_c == -INFINITY) ? 0.f : ex2(m_c - m_new);
+    float psum = 0.f;
+    {
+      uint32_t pk[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        float p0 = (2 * j < L) ? round_to_half_bits(ex2(fmaf(__uint_as_float(s0[2 * j]), g.scale_log2, -m_new))) : 0.f;
+        float p1 = (2 * j + 1 < L) ? round_to_half_bits(ex2(fmaf(__uint_as_float(s0[2 * j + 1]), g.scale_log2, -m_new))) : 0.f;
+        psum += p0 + p1;
+        __half2 hp = __floats2half2_rn(p0, p1);
+        pk[j] = *reinterpret_cast<uint32_t*>(&hp);
+      }
+      if (half == 0) tmem_st16(tlane + TM_P + 32 * b, pk);
+      if (n_s > 32) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          float p0 = (32 + 2 * j < L) ? round_to_half_bits(ex2(fmaf(__uint_as_float(s1[2 * j]), g.scale_log2, -m_new))) : 0.f;
+          float p1 = (33 + 2 * j < L) ? round_to_half_bits(ex2(fmaf(__uint_as_float(s1[2 * j + 1]), g.scale_log2, -m_new))) : 0.f;
+          psum += p0 + p1;
+          __half2 hp = __floats2half2_rn(p0, p1);
+          pk[j] = *reinterpret_cast<uint32_t*>(&hp);
+        }
+        if (half == 1) tmem_st16(tlane + TM_P + 32 * b + 16, pk);
+      }
+    }
+    tmem_st_wait();
+    tc_fence_before();
+    mbar_arrive(c.bar(BAR_P_FULL + b));
+    const float l_new = fmaf(l_c, alpha, psum);
+    const float inv = 1.f / l_new;
+    const float a_inv = alpha * inv;
+
+    if (!wait_bar(c, BAR_O_FULL + b, par, LOC_WAIT_O)) return;
+    if (!wait_bar(c, BAR_IO_FULL, uu & 1, LOC_WAIT_V)) return;
+    tc_fence_after();
+    // out = (alpha O~_cache + P~V) / l, in place in the staging tile
+#pragma unroll
+    for (int q2 = 0; q2 < 2; ++q2) {
+      uint32_t rr[32];
+      tmem_ld32(tlane + TM_O + 128 * b + 64 * half + 32 * q2, rr);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float4* p4 = reinterpret_cast<float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
+        float4 oc = *p4;
+        oc.x = fmaf(oc.x, a_inv, __uint_as_float(rr[4 * i]) * inv);
+        oc.y = fmaf(oc.y, a_inv, __uint_as_float(rr[4 * i + 1]) * inv);
+        oc.z = fmaf(oc.z, a_inv, __uint_as_float(rr[4 * i + 2]) * inv);
+        oc.w = fmaf(oc.w, a_inv, __uint_as_float(rr[4 * i + 3]) * inv);
+        *p4 = oc;
+      }
+    }
+    tc_fence_before();
+    mbar_arrive(c.bar(BAR_O_FREE + b));
+    const size_t orow = (size_t)row * g.Hq + h;
+    if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_new + log2f(l_new)) * LN2;
+    const bool full_tile = it.nrows == BM;
+    if (!full_tile && row_valid) {
+      // a tile clipped by the block or the sequence end: rows go out one by one
+      float4* dst = reinterpret_cast<float4*>(a.out + orow * D + 64 * half);
+#pragma unroll
+      for (int q2 = 0; q2 < 2; ++q2)
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          dst[8 * q2 + i] = *reinterpret_cast<const float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
+    }
+    fence_async_smem();
+    if (!epi_sync(c, epi_phase)) return;  // the whole tile is in the staging buffer
+    if (threadIdx.x == 64) {
+      if (full_tile) {
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) tma_store_3d(&maps.out, c.base + SM_IO + cb * IO_BOX, 32 * cb, h, it.row0);
+        bulk_commit();
+        bulk_wait_read();               // the copies have read the staging tile
+      }
+      mbar_arrive(c.bar(BAR_IO_FREE));  // the producer may load the next tile
+    }
+    it = nxt;
+  }
+}
+
+// ===========================================================================
+__global__ void __launch_bounds__(THREADS, 1)
 tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const AttnArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
-  Shared sh;
-  sh.base = smem_u32(smem_raw);
-  uint32_t* words = reinterpret_cast<uint32_t*>(smem_raw + SM_BAR + 8 * N_BARS);  // [0] tmem base, [1] abort, [2] last flag
-  sh.abort_flag = reinterpret_cast<volatile int*>(words + 1);
-  sh.status = a.status;
-  if ((sh.base & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
+  Cta c;
+  c.base = smem_u32(smem_raw);
+  c.gen = smem_raw;
+  uint32_t* words = reinterpret_cast<uint32_t*>(smem_raw + SM_BAR + 8 * N_BARS);  // [0] tmem, [1] abort, [2] flag
+  c.abort_flag = reinterpret_cast<volatile int*>(words + 1);
+  c.flag = reinterpret_cast<volatile uint32_t*>(words + 2);
+  c.status = a.status;
+  // role and unit range of this CTA; the first work item is fetched before the
+  // set-up below so its latency overlaps it
+  const bool stream = (int)blockIdx.x < a.n_ctas_stream;
+  int first, stride, n_units;
+  if (stream) {
+    first = blockIdx.x; stride = a.n_ctas_stream; n_units = a.n_items * g.Hq;
+  } else {
+    first = blockIdx.x - a.n_ctas_stream; stride = gridDim.x - a.n_ctas_stream; n_units = a.n_items_merge * g.Hq;
+  }
+  WorkItem it0{};
+  if (first < n_units) it0 = stream ? load_item(a.items + first % a.n_items)
+                                    : load_item(a.items_merge + first % a.n_items_merge);
+  if ((c.base & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = LOC_SMEM_ALIGN;
     return;
   }
-  auto bar = [&](int slot) { return sh.base + SM_BAR + 8u * slot; };
-
-  // ---- work item ----
-  const WorkItem it = a.items[blockIdx.x];
-  const int h = blockIdx.y;
-  const int kh = h / g.group;
-  const int seq_start = a.cu[it.seq], seq_end = a.cu[it.seq + 1];
-  const int bs = a.blk_start ? a.blk_start[it.seq] : 0;
-  const int be = bs + g.block_len;
-  int key_base, t0, t1, k0, k1, x0 = 0, x1 = 0;
-  bool from_state = false;
-  const bool chunked = (a.mode == MODE_STEP && it.kind == ITEM_BLOCK_CHUNK);
-  if (a.mode == MODE_BUILD) {
-    key_base = seq_start; k0 = seq_start; k1 = seq_end; x0 = bs; x1 = be;
-    t0 = 0; t1 = (seq_end - seq_start + BN - 1) / BN;
-  } else if (a.mode == MODE_STEP && !chunked) {
-    key_base = bs; k0 = bs; k1 = be; from_state = true;
-    t0 = 0; t1 = (g.block_len + BN - 1) / BN;
-  } else {
-    key_base = seq_start; k0 = seq_start; k1 = seq_end;
-    t0 = 0; t1 = (seq_end - seq_start + BN - 1) / BN;
-    if (chunked) { t0 = it.kt0; t1 = it.kt1; }
-  }
-  // a key tile that lies entirely inside the excluded range is skipped
-  auto tile_skipped = [&](int t) {
-    int lo = key_base + t * BN, hi = min(lo + BN, k1);
-    return x1 > x0 && lo >= x0 && hi <= x1;
-  };
-  auto next_tile = [&](int t) {
-    while (t < t1 && tile_skipped(t)) ++t;
-    return t;
-  };
-
-  // ---- setup: barriers, TMEM ----
   if (tid == 0) {
-    mbar_init(bar(BAR_Q), 1);
-    mbar_init(bar(BAR_K), 1);
-    mbar_init(bar(BAR_V), 1);
-    mbar_init(bar(BAR_S), 1);
-    mbar_init(bar(BAR_O), 1);
-    mbar_init(bar(BAR_SYNC), THREADS);
-    mbar_init(bar(BAR_DONE), THREADS);
+    for (int i = 0; i < N_BARS; ++i) {
+      uint32_t count = 1;
+      if (i == BAR_P_FULL || i == BAR_P_FULL1 || i == BAR_O_FREE || i == BAR_O_FREE1 || i == BAR_EPI)
+        count = ROW_THREADS;
+      if (i == BAR_DONE) count = THREADS;
+      mbar_init(c.bar(i), count);
+    }
     words[1] = 0;
     words[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    fence_async_smem();
   }
   __syncwarp();
   if (warp == 0) {
@@ -265,269 +888,46 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = words[0];
-  const uint32_t tlane = tmem + ((uint32_t)(warp * 32) << 16);  // this warp's 32 lanes
+  c.tmem = words[0];
 
-  uint32_t ph_q = 0, ph_k = 0, ph_v = 0, ph_s = 0, ph_o = 0, ph_sync = 0;
-  bool ok = true;
-
-  int t = next_tile(t0);
-  if (tid == 0) {
-    mbar_expect_tx(bar(BAR_Q), 4 * Q_BOX_BYTES);
-    tma_load_3d(sh.base + SM_QHI, &maps.q_hi, bar(BAR_Q), 0, it.row0, h);
-    tma_load_3d(sh.base + SM_QHI + Q_BOX_BYTES, &maps.q_hi, bar(BAR_Q), 64, it.row0, h);
-    tma_load_3d(sh.base + SM_QLO, &maps.q_lo, bar(BAR_Q), 0, it.row0, h);
-    tma_load_3d(sh.base + SM_QLO + Q_BOX_BYTES, &maps.q_lo, bar(BAR_Q), 64, it.row0, h);
-    if (t < t1) {
-      int krow = key_base + t * BN;
-      mbar_expect_tx(bar(BAR_K), 4 * K_BOX_BYTES);
-      tma_load_3d(sh.base + SM_KHI, &maps.k_hi, bar(BAR_K), 0, krow, kh);
-      tma_load_3d(sh.base + SM_KHI + K_BOX_BYTES, &maps.k_hi, bar(BAR_K), 64, krow, kh);
-      tma_load_3d(sh.base + SM_KLO, &maps.k_lo, bar(BAR_K), 0, krow, kh);
-      tma_load_3d(sh.base + SM_KLO + K_BOX_BYTES, &maps.k_lo, bar(BAR_K), 64, krow, kh);
-      mbar_expect_tx(bar(BAR_V), 2 * K_BOX_BYTES);
-      tma_load_3d(sh.base + SM_V, &maps.v, bar(BAR_V), 0, krow, kh);
-      tma_load_3d(sh.base + SM_V + K_BOX_BYTES, &maps.v, bar(BAR_V), 64, krow, kh);
+  if (warp == 0) {
+    if (stream) {
+      if (tid == 0) stream_producer(c, maps, g, a, first, stride, n_units, it0);
+    } else {
+      if (tid == 0) merge_producer(c, maps, g, a, first, stride, n_units, it0);
     }
+  } else if (warp == 1) {
+    if (tid == 32) {
+      if (stream) stream_mma(c, g, a, first, stride, n_units, it0);
+      else merge_mma(c, g, a, first, stride, n_units);
+    }
+  } else {
+    if (stream) stream_rows(c, g, a, first, stride, n_units, it0);
+    else merge_rows(c, maps, g, a, first, stride, n_units, it0);
+    bulk_wait_read();
   }
   __syncwarp();
 
-  // ---- per-row state: thread tid owns query row it.row0 + tid ----
-  const int row = it.row0 + tid;
-  const bool row_valid = tid < it.nrows;
-  float m_run = -INFINITY, l_run = 0.f;
-  float o_acc[D];
-#pragma unroll
-  for (int c = 0; c < D; ++c) o_acc[c] = 0.f;
-  if (from_state && row_valid) {
-    size_t srow = (size_t)h * g.Tp + row;
-    m_run = a.st.m[srow];
-    l_run = a.st.l[srow];
-    const float4* src = reinterpret_cast<const float4*>(a.st.o + srow * D);
-#pragma unroll
-    for (int c = 0; c < D / 4; ++c) {
-      float4 v = src[c];
-      o_acc[4 * c] = v.x; o_acc[4 * c + 1] = v.y; o_acc[4 * c + 2] = v.z; o_acc[4 * c + 3] = v.w;
-    }
-  }
-
-  if (tid == 0) ok = wait_bar(sh, BAR_Q, ph_q, LOC_WAIT_Q);  // always: no copy may outlive the CTA
-  ph_q ^= 1;
-
-  while (ok && t < t1) {
-    const int tn = next_tile(t + 1);
-    const int tile_lo = key_base + t * BN;
-    // ---- S = Q' K'^T ----
-    if (tid == 0) {
-      ok = wait_bar(sh, BAR_K, ph_k, LOC_WAIT_K);
-      if (ok) {
-        tc_fence_after();
-        uint32_t acc = 0;
-#pragma unroll
-        for (int term = 0; term < 3; ++term) {
-          // hi.hi, hi.lo, lo.hi
-          const uint32_t qa = sh.base + (term == 2 ? SM_QLO : SM_QHI);
-          const uint32_t ka = sh.base + (term == 1 ? SM_KLO : SM_KHI);
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            uint32_t qoff = (ks >> 2) * Q_BOX_BYTES + (ks & 3) * 32;
-            uint32_t koff = (ks >> 2) * K_BOX_BYTES + (ks & 3) * 32;
-            mma_ss(tmem + TM_S, smem_desc(qa + qoff, 16, 1024), smem_desc(ka + koff, 16, 1024), IDESC_S, acc);
-            acc = 1;
-          }
-        }
-        tc_commit(bar(BAR_S));
-      }
-    }
-    __syncwarp();
-    ph_k ^= 1;
-    if (!wait_bar(sh, BAR_S, ph_s, LOC_WAIT_S)) { ok = false; break; }
-    ph_s ^= 1;
-    tc_fence_after();
-    if (tid == 0 && tn < t1) {  // the K buffers are free: prefetch the next tile's keys
-      int krow = key_base + tn * BN;
-      mbar_expect_tx(bar(BAR_K), 4 * K_BOX_BYTES);
-      tma_load_3d(sh.base + SM_KHI, &maps.k_hi, bar(BAR_K), 0, krow, kh);
-      tma_load_3d(sh.base + SM_KHI + K_BOX_BYTES, &maps.k_hi, bar(BAR_K), 64, krow, kh);
-      tma_load_3d(sh.base + SM_KLO, &maps.k_lo, bar(BAR_K), 0, krow, kh);
-      tma_load_3d(sh.base + SM_KLO + K_BOX_BYTES, &maps.k_lo, bar(BAR_K), 64, krow, kh);
-    }
-    __syncwarp();
-
-    // ---- online softmax on this thread's row ----
-    // column j of the tile is key tile_lo + j; valid keys: [k0,k1) minus [x0,x1)
-    const int v_lo = max(k0 - tile_lo, 0), v_hi = min(k1 - tile_lo, BN);
-    const int e_lo = x0 - tile_lo, e_hi = x1 - tile_lo;
-    auto col_valid = [&](int j) { return j >= v_lo && j < v_hi && !(j >= e_lo && j < e_hi); };
-    float mx = -INFINITY;
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      uint32_t r[32];
-      tmem_ld32(tlane + TM_S + 32 * half, r);
-      tmem_ld_wait();
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (col_valid(32 * half + j)) mx = fmaxf(mx, __uint_as_float(r[j]));
-    }
-    // integer reference exponent (log2 units) so rescales are exact powers of two
-    const float m_new = fmaxf(m_run, ceilf(mx * g.scale_log2));
-    const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-    const float alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - m_new);
-    float psum = 0.f;
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      uint32_t r[32];
-      tmem_ld32(tlane + TM_S + 32 * half, r);
-      tmem_ld_wait();
-      uint32_t pk[16];
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        int c = 32 * half + 2 * j;
-        float p0 = col_valid(c) ? ex2(fmaf(__uint_as_float(r[2 * j]), g.scale_log2, -m_ref)) : 0.f;
-        float p1 = col_valid(c + 1) ? ex2(fmaf(__uint_as_float(r[2 * j + 1]), g.scale_log2, -m_ref)) : 0.f;
-        __half2 hp = __floats2half2_rn(p0, p1);
-        float2 back = __half22float2(hp);
-        psum += back.x + back.y;  // the normaliser sums exactly what the MMA multiplies
-        pk[j] = *reinterpret_cast<uint32_t*>(&hp);
-      }
-      tmem_st16(tlane + TM_P + 16 * half, pk);
-    }
-    tmem_st_wait();
-    l_run = l_run * alpha + psum;
-    m_run = m_new;
-    // every thread's P~ is in TMEM before the MMA reads it
-    tc_fence_before();
-    mbar_arrive(bar(BAR_SYNC));
-    if (tid == 0) {
-      ok = wait_bar(sh, BAR_SYNC, ph_sync, LOC_WAIT_S);
-      if (ok) ok = wait_bar(sh, BAR_V, ph_v, LOC_WAIT_V);
-      if (ok) {
-        tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < BN / 16; ++ks) {
-          // B = V tile, MN-major: 64 features contiguous, next 64 at +8 KB (LBO),
-          // groups of 8 keys 1 KB apart (SBO); 16 keys per MMA = 2 KB
-          mma_ts(tmem + TM_O, tmem + TM_P + 8 * ks, smem_desc(sh.base + SM_V + ks * 2048, K_BOX_BYTES, 1024),
-                 IDESC_PV, ks > 0 ? 1u : 0u);
-        }
-        tc_commit(bar(BAR_O));
-      }
-    }
-    __syncwarp();
-    ph_sync ^= 1;
-    ph_v ^= 1;
-    if (!wait_bar(sh, BAR_O, ph_o, LOC_WAIT_O)) { ok = false; break; }
-    ph_o ^= 1;
-    tc_fence_after();
-    if (tid == 0 && tn < t1) {  // the V buffer is free
-      int krow = key_base + tn * BN;
-      mbar_expect_tx(bar(BAR_V), 2 * K_BOX_BYTES);
-      tma_load_3d(sh.base + SM_V, &maps.v, bar(BAR_V), 0, krow, kh);
-      tma_load_3d(sh.base + SM_V + K_BOX_BYTES, &maps.v, bar(BAR_V), 64, krow, kh);
-    }
-    __syncwarp();
-    // ---- O~ = alpha O~ + P~ V ----
-#pragma unroll
-    for (int q4 = 0; q4 < 4; ++q4) {
-      uint32_t r[32];
-      tmem_ld32(tlane + TM_O + 32 * q4, r);
-      tmem_ld_wait();
-#pragma unroll
-      for (int j = 0; j < 32; ++j) o_acc[32 * q4 + j] = fmaf(o_acc[32 * q4 + j], alpha, __uint_as_float(r[j]));
-    }
-    tc_fence_before();
-    t = tn;
-  }
-
-  // ---- epilogue ----
-  const float LN2 = 0.69314718055994530942f;
-  if (ok && row_valid) {
-    if (a.mode == MODE_BUILD) {
-      size_t srow = (size_t)h * g.Tp + row;
-      a.st.m[srow] = m_run;
-      a.st.l[srow] = l_run;
-      float4* dst = reinterpret_cast<float4*>(a.st.o + srow * D);
-#pragma unroll
-      for (int c = 0; c < D / 4; ++c)
-        dst[c] = make_float4(o_acc[4 * c], o_acc[4 * c + 1], o_acc[4 * c + 2], o_acc[4 * c + 3]);
-    } else if (!chunked || it.pad == 1) {
-      const float inv = 1.f / l_run;
-      size_t orow = (size_t)row * g.Hq + h;
-      float4* dst = reinterpret_cast<float4*>(a.out + orow * D);
-#pragma unroll
-      for (int c = 0; c < D / 4; ++c)
-        dst[c] = make_float4(o_acc[4 * c] * inv, o_acc[4 * c + 1] * inv, o_acc[4 * c + 2] * inv, o_acc[4 * c + 3] * inv);
-      if (a.lse) a.lse[orow] = (m_run + log2f(l_run)) * LN2;
-    } else {
-      size_t prow = (((size_t)it.seq * g.Hq + h) * a.max_chunks + it.chunk) * g.block_len + tid;
-      a.part_m[prow] = m_run;
-      a.part_l[prow] = l_run;
-      float4* dst = reinterpret_cast<float4*>(a.part_o + prow * D);
-#pragma unroll
-      for (int c = 0; c < D / 4; ++c)
-        dst[c] = make_float4(o_acc[4 * c], o_acc[4 * c + 1], o_acc[4 * c + 2], o_acc[4 * c + 3]);
-    }
-  }
-  if (chunked && it.pad > 1) {
-    // the last chunk of this (sequence, head) to arrive merges all partials
-    __threadfence();
-    mbar_arrive(bar(BAR_SYNC));
-    bool synced = wait_bar(sh, BAR_SYNC, ph_sync, LOC_WAIT_O);
-    ph_sync ^= 1;
-    if (synced && tid == 0) {
-      int old = atomicAdd(&a.counters[it.seq * g.Hq + h], 1);
-      int last = (old == it.pad - 1) ? 1 : 0;
-      if (last) a.counters[it.seq * g.Hq + h] = 0;
-      words[2] = last;
-      __threadfence();
-    }
-    mbar_arrive(bar(BAR_SYNC));
-    synced = synced && wait_bar(sh, BAR_SYNC, ph_sync, LOC_WAIT_O);
-    ph_sync ^= 1;
-    if (synced && ok && words[2] && row_valid) {
-      __threadfence();
-      size_t p0 = (((size_t)it.seq * g.Hq + h) * a.max_chunks) * g.block_len + tid;
-      float M = -INFINITY;
-      for (int c = 0; c < it.pad; ++c) M = fmaxf(M, __ldcg(a.part_m + p0 + (size_t)c * g.block_len));
-      float L = 0.f;
-#pragma unroll
-      for (int c = 0; c < D; ++c) o_acc[c] = 0.f;
-      for (int ch = 0; ch < it.pad; ++ch) {
-        size_t pr = p0 + (size_t)ch * g.block_len;
-        float mc = __ldcg(a.part_m + pr);
-        if (mc == -INFINITY) continue;
-        float w = ex2(mc - M);
-        L = fmaf(__ldcg(a.part_l + pr), w, L);
-        const float4* src = reinterpret_cast<const float4*>(a.part_o + pr * D);
-#pragma unroll
-        for (int c = 0; c < D / 4; ++c) {
-          float4 v = __ldcg(src + c);
-          o_acc[4 * c] = fmaf(v.x, w, o_acc[4 * c]);
-          o_acc[4 * c + 1] = fmaf(v.y, w, o_acc[4 * c + 1]);
-          o_acc[4 * c + 2] = fmaf(v.z, w, o_acc[4 * c + 2]);
-          o_acc[4 * c + 3] = fmaf(v.w, w, o_acc[4 * c + 3]);
-        }
-      }
-      const float inv = 1.f / L;
-      size_t orow = (size_t)row * g.Hq + h;
-      float4* dst = reinterpret_cast<float4*>(a.out + orow * D);
-#pragma unroll
-      for (int c = 0; c < D / 4; ++c)
-        dst[c] = make_float4(o_acc[4 * c] * inv, o_acc[4 * c + 1] * inv, o_acc[4 * c + 2] * inv, o_acc[4 * c + 3] * inv);
-      if (a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
-    }
-  }
-
-  // ---- teardown: free TMEM once every thread is past its last TMEM access ----
+  // teardown: free TMEM once every thread is past its last TMEM access
   tc_fence_before();
-  mbar_arrive(bar(BAR_DONE));
+  mbar_arrive(c.bar(BAR_DONE));
   if (warp == 0) {
-    wait_bar(sh, BAR_DONE, 0, LOC_WAIT_O);
+    wait_bar(c, BAR_DONE, 0, LOC_WAIT_O);
     __syncwarp();
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TM_COLS) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.tmem), "r"(TM_COLS) : "memory");
   }
 }
+
+#ifdef LACACHE_DEBUG_CLOCKS
+}  // namespace
+}  // namespace lacache
+extern "C" int lacache_debug_read_clocks(long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, lacache::g_dbg_clocks, sizeof(long long) * n);
+}
+namespace lacache {
+namespace {
+#endif
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -543,6 +943,20 @@ EncodeTiledFn get_encode() {
     return nullptr;
   fn = reinterpret_cast<EncodeTiledFn>(p);
   return fn;
+}
+
+bool make_f32_map(CUtensorMap* m, void* base, cuuint64_t d1, cuuint64_t d2, cuuint32_t b1, cuuint32_t b2, char* err,
+                  int errlen) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) { snprintf(err, errlen, "cuTensorMapEncodeTiled entry point not found"); return false; }
+  cuuint64_t dims[3] = {(cuuint64_t)D, d1, d2};
+  cuuint64_t strides[2] = {(cuuint64_t)D * 4, d1 * D * 4};
+  cuuint32_t box[3] = {32, b1, b2};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { snprintf(err, errlen, "cuTensorMapEncodeTiled (fp32) failed with CUresult %d", (int)r); return false; }
+  return true;
 }
 
 bool make_plane_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, bool fp16, char* err, int errlen) {
@@ -565,13 +979,25 @@ cudaError_t tc_prepare() {
   return cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
 }
 
-TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, char* err, int errlen) {
+bool tc_set_out(TcMaps* m, const Geometry& g, float* out, char* err, int errlen) {
+  if (m->out_ptr == out) return true;
+  if (!make_f32_map(&m->out, out, (cuuint64_t)g.Hq, (cuuint64_t)g.T, 1, BM, err, errlen)) return false;
+  m->out_ptr = out;
+  return true;
+}
+
+TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, char* err, int errlen) {
   TcMaps* m = new TcMaps();
+  m->out_ptr = nullptr;
+  m->out = CUtensorMap{};
   bool ok = make_plane_map(&m->q_hi, rot.q_hi, g.Hq, g.Tp, BM, false, err, errlen) &&
             make_plane_map(&m->q_lo, rot.q_lo, g.Hq, g.Tp, BM, false, err, errlen) &&
+            make_plane_map(&m->q64_hi, rot.q_hi, g.Hq, g.Tp, 64, false, err, errlen) &&
+            make_plane_map(&m->q64_lo, rot.q_lo, g.Hq, g.Tp, 64, false, err, errlen) &&
             make_plane_map(&m->k_hi, rot.k_hi, g.Hkv, g.Tp, BN, false, err, errlen) &&
             make_plane_map(&m->k_lo, rot.k_lo, g.Hkv, g.Tp, BN, false, err, errlen) &&
-            make_plane_map(&m->v, rot.v, g.Hkv, g.Tp, BN, true, err, errlen);
+            make_plane_map(&m->v, rot.v, g.Hkv, g.Tp, BN, true, err, errlen) &&
+            make_f32_map(&m->st_o, state_o, (cuuint64_t)g.Tp, (cuuint64_t)g.Hq, BM, 1, err, errlen);
   if (!ok) { delete m; return nullptr; }
   return m;
 }
@@ -579,9 +1005,8 @@ TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, char* err, int er
 void tc_free_maps(TcMaps* m) { delete m; }
 
 cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* maps, cudaStream_t s) {
-  if (a.n_items == 0) return cudaSuccess;
-  dim3 grid(a.n_items, g.Hq);
-  tc_attn_kernel<<<grid, THREADS, SM_TOTAL, s>>>(*maps, g, a);
+  if (a.n_ctas <= 0) return cudaSuccess;
+  tc_attn_kernel<<<a.n_ctas, THREADS, SM_TOTAL, s>>>(*maps, g, a);
   return cudaGetLastError();
 }
 
