@@ -155,7 +155,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   for (int b = 0; b < cfg->batch; ++b)
     if (cfg->prompt_lens[b] < 0) return fail(c, LACACHE_ERR_SHAPE, "prompt_lens[%d] < 0", b);
 
-  bool tc_ok = cfg->dtype == LACACHE_DTYPE_BF16 && cfg->head_dim == 128 && cfg->block_len <= TC_KEYS;
+  bool tc_ok = cfg->dtype == LACACHE_DTYPE_BF16 && cfg->head_dim == 128 && cfg->block_len <= TC_MAX_BLOCK;
   if (cfg->engine == LACACHE_ENGINE_AUTO) c->engine = tc_ok ? LACACHE_ENGINE_TCGEN05 : LACACHE_ENGINE_SIMT;
   else if (cfg->engine == LACACHE_ENGINE_SIMT) c->engine = LACACHE_ENGINE_SIMT;
   else if (cfg->engine == LACACHE_ENGINE_TCGEN05) {
@@ -195,12 +195,11 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   const bool tc = c->engine == LACACHE_ENGINE_TCGEN05;
   const int R = tc ? TC_ROWS : SIMT_ROWS;
   std::vector<WorkItem> items;
+  // block-query units: chunks of `tpc` key tiles, balanced over the sequence,
+  // at most 16 chunks (the partial-state merge reads them all)
   int tpc = cfg->sc_tiles_per_chunk;
-  if (tpc <= 0) {
-    long long tiles = 0;
-    for (int b = 0; b < g.B; ++b) tiles += (c->cu[b + 1] - c->cu[b] + TC_KEYS - 1) / TC_KEYS;
-    tpc = (int)std::min<long long>(8, std::max<long long>(2, (tiles * g.Hq + 74) / 148));
-  }
+  if (const char* e = getenv("LACACHE_SC_TILES")) tpc = atoi(e);
+  if (tpc <= 0) tpc = 2;
   c->max_chunks = 1;
   for (int k = 0; k < g.n_blk; ++k) {
     int off = (int)items.size();
@@ -210,12 +209,14 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
       if (tc) {
         int n = c->cu[b + 1] - c->cu[b];
         int nkt = (n + TC_KEYS - 1) / TC_KEYS;
-        int chunks = (nkt + tpc - 1) / tpc;
+        int chunks = std::min(16, (nkt + tpc - 1) / tpc);
+        int tpc_b = (nkt + chunks - 1) / chunks;       // balanced
+        chunks = (nkt + tpc_b - 1) / tpc_b;
         c->max_chunks = std::max(c->max_chunks, chunks);
         for (int ch = 0; ch < chunks; ++ch) {
           WorkItem w{};
           w.kind = ITEM_BLOCK_CHUNK; w.seq = b; w.row0 = bs; w.nrows = g.block_len;
-          w.chunk = ch; w.kt0 = ch * tpc; w.kt1 = std::min(nkt, (ch + 1) * tpc);
+          w.chunk = ch; w.kt0 = ch * tpc_b; w.kt1 = std::min(nkt, (ch + 1) * tpc_b);
           w.pad = chunks;
           w.seq_start = c->cu[b]; w.seq_end = c->cu[b + 1]; w.blk_start = bs;
           items.push_back(w);

@@ -17,8 +17,9 @@
 //                  shared memory.  The normaliser sums the rounded P~.
 //
 // Two roles, chosen per CTA:
-//   stream role  a tile of 128 (or 64) query rows streams key tiles of 64
-//                keys through a 2-stage K/V ring; used for the cache build
+//   stream role  a tile of 128 (or 64) query rows streams key tiles of 128
+//                keys; O~ accumulates in TMEM and is rescaled in place only
+//                when a row maximum outgrows the reference exponent; used for the cache build
 //                (rows in U x keys in U -> cached state), the full recompute,
 //                and the block queries of a step (one chunk of key tiles per
 //                work unit; the last chunk to finish merges the partials).
@@ -43,9 +44,12 @@ struct TcMaps {
   alignas(64) CUtensorMap q_lo;
   alignas(64) CUtensorMap q64_hi;  // box 64 rows (block queries)
   alignas(64) CUtensorMap q64_lo;
-  alignas(64) CUtensorMap k_hi;    // box 64 rows
+  alignas(64) CUtensorMap k_hi;    // box 128 rows (stream role)
   alignas(64) CUtensorMap k_lo;
   alignas(64) CUtensorMap v;
+  alignas(64) CUtensorMap k64_hi;  // box 64 rows (the block's keys, merge role)
+  alignas(64) CUtensorMap k64_lo;
+  alignas(64) CUtensorMap v64;
   alignas(64) CUtensorMap st_o;    // cached O~ [Hq][Tp][128] fp32, box 32 cols x 128 rows
   alignas(64) CUtensorMap out;     // caller's out [T][Hq][128] fp32, box 32 cols x 1 head x 128 rows
   const void* out_ptr;             // the buffer `out` was encoded for
@@ -55,38 +59,61 @@ namespace {
 
 constexpr int D = 128;
 constexpr int BM = TC_ROWS;   // 128 query rows (TMEM lanes)
-constexpr int BN = TC_KEYS;   // 64 keys per tile
+constexpr int BN = TC_KEYS;   // 128 keys per tile (stream role)
+constexpr float RESCALE_SLACK = 3.f;
 constexpr int ROW_WARPS = 8;
 constexpr int ROW_THREADS = ROW_WARPS * 32;
 constexpr int THREADS = 64 + ROW_THREADS;
 
 // ---- shared memory map (bytes from a 1024-aligned base) ----
-constexpr uint32_t SM_Q = 0;                      // hi plane, then lo plane at +32 KB
+constexpr uint32_t SM_Q = 0;                      // Q hi plane, then lo plane at +32 KB
 constexpr uint32_t SM_Q_LO = 32768;
-constexpr uint32_t SM_KV = 65536;                 // 2 stages of {K hi, K lo, V}
+// stream role: one tile of 128 keys: K hi (2 boxes of 16 KB), K lo, then V
+constexpr uint32_t SM_K = 65536;
+constexpr uint32_t SK_LO = 32768;
+constexpr uint32_t SM_V = SM_K + 65536;
+constexpr uint32_t KS_BOX = 128 * 128;            // one [128 rows][64 cols] 16-bit box
+// merge role: the same 96 KB hold 2 stages of the block's keys: {K hi, K lo, V} of 64 rows
+constexpr uint32_t SM_KV = SM_K;
 constexpr uint32_t KV_STAGE = 49152;
 constexpr uint32_t KV_KLO = 16384;
 constexpr uint32_t KV_V = 32768;
 constexpr uint32_t K_BOX = 64 * 128;              // one [64 rows][64 cols] 16-bit box
-constexpr uint32_t SM_IO = SM_KV + 2 * KV_STAGE;  // staging: 128 rows x (512 + 16) bytes
+constexpr uint32_t SM_IO = SM_V + 32768;          // staging: 128 rows x (512 + 16) bytes
 constexpr uint32_t IO_ROW = 528;
-constexpr uint32_t IO_BOX = 128 * 128;             // merge role: one swizzled box of 32 fp32 columns x 128 rows
+constexpr uint32_t IO_BOX = 128 * 128;            // merge role: one swizzled box of 32 fp32 columns x 128 rows
+// stream role, block-query units only (64-row Q tile, at most 64 staging rows): a second
+// key stage in the unused halves of the Q and staging regions
+constexpr uint32_t SM_K1_HI = SM_Q + 32768;
+constexpr uint32_t SM_K1_LO = SM_IO + 64 * IO_ROW;
+static_assert(SM_K1_LO % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 constexpr uint32_t SM_BAR = SM_IO + BM * IO_ROW;
+static_assert(SM_K1_LO + 32768 <= SM_BAR, "second key stage overruns the staging region");
 constexpr uint32_t SM_TOTAL = SM_BAR + 256;
 static_assert(SM_TOTAL <= 232448, "exceeds the 227 KB per-CTA limit");
 
 // ---- TMEM columns ----
+// merge role
 constexpr uint32_t TM_S = 0;      // 2 x 64: scores
 constexpr uint32_t TM_P = 128;    // 2 x 32: fp16 probabilities, two per column
-constexpr uint32_t TM_O = 256;    // 2 x 128: P.V of one tile
+constexpr uint32_t TM_O = 256;    // 2 x 128: P.V of one unit
+// stream role
+constexpr uint32_t TS_S = 0;      // 2 x 128: scores
+constexpr uint32_t TS_P = 256;    // 2 x 64: fp16 probabilities
+constexpr uint32_t TS_O = 384;    // 128: O~ accumulated over the tiles of a unit
 constexpr uint32_t TM_COLS = 512;
 
 enum {
   BAR_Q_FULL = 0, BAR_Q_FREE,
-  BAR_KV_FULL, BAR_KV_FULL1, BAR_KV_FREE, BAR_KV_FREE1,
+  BAR_KV_FULL, BAR_KV_FULL1, BAR_KV_FREE, BAR_KV_FREE1,   // merge role: 2 stages
+  BAR_K_FULL = BAR_KV_FULL, BAR_V_FULL = BAR_KV_FULL1,    // stream role: keys / values
+  BAR_K_FREE = BAR_KV_FREE, BAR_V_FREE = BAR_KV_FREE1,
   BAR_S_FULL, BAR_S_FULL1, BAR_P_FULL, BAR_P_FULL1,
   BAR_O_FULL, BAR_O_FULL1, BAR_O_FREE, BAR_O_FREE1,
-  BAR_IO_FULL, BAR_IO_FREE, BAR_EPI, BAR_DONE, N_BARS
+  BAR_IO_FULL, BAR_IO_FREE, BAR_EPI, BAR_DONE,
+  BAR_K_FULL1, BAR_K_FREE1,  // stream role, second key stage (block-query units)
+  BAR_PAIR,  // 4 barriers: the two warps that share a TMEM lane quadrant
+  N_BARS = BAR_PAIR + 4
 };
 
 enum { EPI_STATE = 0, EPI_OUT = 1, EPI_PARTIAL = 2 };
@@ -186,8 +213,41 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]),
+               "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16], int) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
       "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
@@ -324,38 +384,41 @@ __device__ __forceinline__ int next_tile(const Unit& un, int t) {
   return t;
 }
 
-__device__ __forceinline__ void issue_s_mma(const Cta& c, uint32_t kv_base, uint32_t s_tmem, uint32_t q_box,
-                                            uint32_t idesc) {
+// S (+)= Q' K'^T as hi.hi + hi.lo + lo.hi; Q planes at q_base (lo at +32 KB) with
+// boxes of q_box bytes, K planes at k_hi / k_lo with boxes of k_box bytes.
+__device__ __forceinline__ void issue_s_mma(uint32_t q_base, uint32_t q_box, uint32_t k_hi, uint32_t k_lo,
+                                            uint32_t k_box, uint32_t s_tmem, uint32_t idesc) {
   uint32_t acc = 0;
 #pragma unroll
-  for (int term = 0; term < 3; ++term) {  // hi.hi, hi.lo, lo.hi
-    const uint32_t qa = c.base + SM_Q + (term == 2 ? SM_Q_LO : 0u);
-    const uint32_t ka = kv_base + (term == 1 ? KV_KLO : 0u);
+  for (int term = 0; term < 3; ++term) {
+    const uint32_t qa = q_base + (term == 2 ? 2u * q_box : 0u);
+    const uint32_t ka = term == 1 ? k_lo : k_hi;
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
       uint32_t qoff = (ks >> 2) * q_box + (ks & 3) * 32;
-      uint32_t koff = (ks >> 2) * K_BOX + (ks & 3) * 32;
+      uint32_t koff = (ks >> 2) * k_box + (ks & 3) * 32;
       mma_ss(s_tmem, smem_desc(qa + qoff, 16, 1024), smem_desc(ka + koff, 16, 1024), idesc, acc);
       acc = 1;
     }
   }
 }
-__device__ __forceinline__ void issue_pv_mma(uint32_t kv_base, uint32_t p_tmem, uint32_t o_tmem, int ksteps) {
+// O (+)= P~ V: A = P~ in TMEM (16 keys = 8 columns per step), B = V tile, MN-major:
+// 64 features contiguous (128 B), the next 64 features v_box bytes further (LBO),
+// groups of 8 keys 1 KB apart (SBO); 16 keys = 2 KB.
+__device__ __forceinline__ void issue_pv_mma(uint32_t v_base, uint32_t v_box, uint32_t p_tmem, uint32_t o_tmem,
+                                             int ksteps, uint32_t accumulate) {
   constexpr uint32_t idesc = idesc_f16(0u /*fp16*/, 1u, BM, D);
-  for (int ks = 0; ks < ksteps; ++ks) {
-    // B = V tile, MN-major: 64 features contiguous (128 B), the next 64 features
-    // 8 KB further (LBO), groups of 8 keys 1 KB apart (SBO); 16 keys = 2 KB.
-    mma_ts(o_tmem, p_tmem + 8 * ks, smem_desc(kv_base + KV_V + ks * 2048, K_BOX, 1024), idesc, ks > 0 ? 1u : 0u);
-  }
+  for (int ks = 0; ks < ksteps; ++ks)
+    mma_ts(o_tmem, p_tmem + 8 * ks, smem_desc(v_base + ks * 2048, v_box, 1024), idesc, (ks > 0) ? 1u : accumulate);
 }
 __device__ __forceinline__ void load_kv_tile(const TcMaps& maps, uint32_t kv_base, uint32_t bar, int krow, int kh) {
   mbar_expect_tx(bar, 6 * K_BOX);
-  tma_load_3d(kv_base, &maps.k_hi, bar, 0, krow, kh);
-  tma_load_3d(kv_base + K_BOX, &maps.k_hi, bar, 64, krow, kh);
-  tma_load_3d(kv_base + KV_KLO, &maps.k_lo, bar, 0, krow, kh);
-  tma_load_3d(kv_base + KV_KLO + K_BOX, &maps.k_lo, bar, 64, krow, kh);
-  tma_load_3d(kv_base + KV_V, &maps.v, bar, 0, krow, kh);
-  tma_load_3d(kv_base + KV_V + K_BOX, &maps.v, bar, 64, krow, kh);
+  tma_load_3d(kv_base, &maps.k64_hi, bar, 0, krow, kh);
+  tma_load_3d(kv_base + K_BOX, &maps.k64_hi, bar, 64, krow, kh);
+  tma_load_3d(kv_base + KV_KLO, &maps.k64_lo, bar, 0, krow, kh);
+  tma_load_3d(kv_base + KV_KLO + K_BOX, &maps.k64_lo, bar, 64, krow, kh);
+  tma_load_3d(kv_base + KV_V, &maps.v64, bar, 0, krow, kh);
+  tma_load_3d(kv_base + KV_V + K_BOX, &maps.v64, bar, 64, krow, kh);
 }
 __device__ __forceinline__ void load_q_tile(const Cta& c, const TcMaps& maps, int q_rows, int row0, int h) {
   const uint32_t bar = c.bar(BAR_Q_FULL);
@@ -365,8 +428,8 @@ __device__ __forceinline__ void load_q_tile(const Cta& c, const TcMaps& maps, in
   mbar_expect_tx(bar, 4 * box);
   tma_load_3d(c.base + SM_Q, mh, bar, 0, row0, h);
   tma_load_3d(c.base + SM_Q + box, mh, bar, 64, row0, h);
-  tma_load_3d(c.base + SM_Q + SM_Q_LO, ml, bar, 0, row0, h);
-  tma_load_3d(c.base + SM_Q + SM_Q_LO + box, ml, bar, 64, row0, h);
+  tma_load_3d(c.base + SM_Q + 2 * box, ml, bar, 0, row0, h);
+  tma_load_3d(c.base + SM_Q + 3 * box, ml, bar, 64, row0, h);
 }
 
 // ===========================================================================
@@ -374,6 +437,7 @@ __device__ __forceinline__ void load_q_tile(const Cta& c, const TcMaps& maps, in
 // ===========================================================================
 __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a,
                                 int first, int stride, int n_units, WorkItem it) {
+  const bool ks2 = a.mode == MODE_STEP;  // block-query units have room for two key stages
   int uu = 0, jj = 0;
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
@@ -382,20 +446,40 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
     if (uu >= 1 && !wait_bar(c, BAR_Q_FREE, (uu - 1) & 1, LOC_WAIT_Q)) return;
     load_q_tile(c, maps, un.q_rows, un.row0, un.h);
     for (int t = next_tile(un, un.t0); t < un.t1; t = next_tile(un, t + 1), ++jj) {
-      const int b = jj & 1, k = jj >> 1;
-      if (k >= 1 && !wait_bar(c, BAR_KV_FREE + b, (k - 1) & 1, LOC_WAIT_K)) return;
-      load_kv_tile(maps, c.base + SM_KV + b * KV_STAGE, c.bar(BAR_KV_FULL + b), un.key_base + t * BN, un.kh);
+      const int krow = un.key_base + t * BN;
+      // keys: a stage is free as soon as the scores that read it have been computed
+      {
+        const int sk = ks2 ? (jj & 1) : 0, kuse = ks2 ? (jj >> 1) : jj;
+        if (kuse >= 1 && !wait_bar(c, sk ? BAR_K_FREE1 : BAR_K_FREE, (kuse - 1) & 1, LOC_WAIT_K)) return;
+        const uint32_t bar = c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL);
+        const uint32_t khi = c.base + (sk ? SM_K1_HI : SM_K), klo = c.base + (sk ? SM_K1_LO : SM_K + SK_LO);
+        mbar_expect_tx(bar, 4 * KS_BOX);
+        tma_load_3d(khi, &maps.k_hi, bar, 0, krow, un.kh);
+        tma_load_3d(khi + KS_BOX, &maps.k_hi, bar, 64, krow, un.kh);
+        tma_load_3d(klo, &maps.k_lo, bar, 0, krow, un.kh);
+        tma_load_3d(klo + KS_BOX, &maps.k_lo, bar, 64, krow, un.kh);
+      }
+      // values: free once P~V of the previous tile has been computed
+      if (jj >= 1 && !wait_bar(c, BAR_V_FREE, (jj - 1) & 1, LOC_WAIT_V)) return;
+      {
+        const uint32_t bar = c.bar(BAR_V_FULL), vb = c.base + SM_V;
+        mbar_expect_tx(bar, 2 * KS_BOX);
+        tma_load_3d(vb, &maps.v, bar, 0, krow, un.kh);
+        tma_load_3d(vb + KS_BOX, &maps.v, bar, 64, krow, un.kh);
+      }
     }
     it = nxt;
   }
 }
 
 // The MMA thread issues whichever product is ready: P~V of the oldest pending
-// tile as soon as its probabilities are in TMEM, else the scores of the next
-// tile as soon as its keys have landed (at most two score tiles in flight).
+// tile as soon as its probabilities are in TMEM and its values have landed,
+// else the scores of the next tile as soon as its keys have landed (at most two
+// score tiles in flight).  O~ accumulates in TMEM across the tiles of a unit.
 __device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units,
                            WorkItem it) {
   constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
+  const bool ks2 = a.mode == MODE_STEP;
   int uu = 0, js = 0, jp = 0;  // global counters of score tiles / PV tiles issued
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
@@ -404,28 +488,37 @@ __device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, i
     const uint32_t q_box = (uint32_t)un.q_rows * 128u;
     if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
     int ts = next_tile(un, un.t0), tp = ts;
-    bool q_released = false;
+    bool q_released = false, first_pv = true;
+    bool o_free_pending = uu >= 1;  // O_FREE of the previous unit is observed exactly once, in order
     long long t_idle = 0;
     while (tp < un.t1) {
       bool did = false;
       if (js > jp) {  // scores of tile jp issued: its P~V may be ready
-        const int b = jp & 1, k = jp >> 1;
-        if (mbar_test(c.bar(BAR_P_FULL + b), k & 1) && (k < 1 || mbar_test(c.bar(BAR_O_FREE + b), (k - 1) & 1))) {
+        const int b = jp & 1;
+        if (mbar_test(c.bar(BAR_P_FULL + b), (jp >> 1) & 1) && mbar_test(c.bar(BAR_V_FULL), jp & 1)) {
+          if (o_free_pending) {  // the row threads have read the previous unit's O~
+            if (!wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
+            o_free_pending = false;
+          }
           tc_fence_after();
-          issue_pv_mma(c.base + SM_KV + b * KV_STAGE, c.tmem + TM_P + 32 * b, c.tmem + TM_O + 128 * b, BN / 16);
-          tc_commit(c.bar(BAR_O_FULL + b));
-          tc_commit(c.bar(BAR_KV_FREE + b));
+          issue_pv_mma(c.base + SM_V, KS_BOX, c.tmem + TS_P + 64 * b, c.tmem + TS_O, BN / 16, first_pv ? 0u : 1u);
+          tc_commit(c.bar(BAR_O_FULL));
+          tc_commit(c.bar(BAR_V_FREE));
+          first_pv = false;
           tp = next_tile(un, tp + 1);
           ++jp;
           did = true;
         }
       }
       if (!did && ts < un.t1 && js - jp < 2) {
-        const int b = js & 1;
-        if (mbar_test(c.bar(BAR_KV_FULL + b), (js >> 1) & 1)) {
+        const int sk = ks2 ? (js & 1) : 0, kuse = ks2 ? (js >> 1) : js;
+        if (mbar_test(c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL), kuse & 1)) {
+          const int b = js & 1;
+          const uint32_t khi = c.base + (sk ? SM_K1_HI : SM_K), klo = c.base + (sk ? SM_K1_LO : SM_K + SK_LO);
           tc_fence_after();
-          issue_s_mma(c, c.base + SM_KV + b * KV_STAGE, c.tmem + TM_S + 64 * b, q_box, IDESC_S);
+          issue_s_mma(c.base + SM_Q, q_box, khi, klo, KS_BOX, c.tmem + TS_S + 128 * b, IDESC_S);
           tc_commit(c.bar(BAR_S_FULL + b));
+          tc_commit(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE));
           ts = next_tile(un, ts + 1);
           ++js;
           if (ts >= un.t1) {  // every score MMA of this unit has been issued
@@ -450,6 +543,7 @@ __device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, i
       }
     }
     if (!q_released) tc_commit(c.bar(BAR_Q_FREE));  // a unit without key tiles
+    if (o_free_pending && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
     it = nxt;
   }
 }
@@ -462,20 +556,15 @@ __device__ __forceinline__ bool epi_sync(const Cta& c, uint32_t& phase) {
   return ok;
 }
 
-// Writes this thread's 64 features (times mul) into its staging half-row and
-// sends them to global memory as one 256-byte bulk copy.
-__device__ __forceinline__ void stage_and_store(const Cta& c, int r, int half, const float (&o)[64], float mul,
-                                                float* gdst, bool valid) {
-  bulk_wait_read();  // an earlier copy out of this half-row must have been read
-  const uint32_t off = SM_IO + r * IO_ROW + half * 256;
-  float4* s4 = reinterpret_cast<float4*>(c.gen + off);
-#pragma unroll
-  for (int i = 0; i < 16; ++i)
-    s4[i] = make_float4(o[4 * i] * mul, o[4 * i + 1] * mul, o[4 * i + 2] * mul, o[4 * i + 3] * mul);
-  fence_async_smem();
-  if (valid) {
-    bulk_store(gdst, c.base + off, 256);
-    bulk_commit();
+// Cooperative, fully coalesced copy of the first nrows staging rows (512 B of
+// payload each) to rows of `stride` floats in global memory: every warp-wide
+// store writes one whole row.
+__device__ __forceinline__ void coop_store_rows(const Cta& c, float* gbase, size_t stride, int nrows) {
+  const int t = threadIdx.x - 64;
+  for (int i = t; i < nrows * 32; i += ROW_THREADS) {
+    const int rr = i >> 5, ch = i & 31;
+    float4 v = *reinterpret_cast<const float4*>(c.gen + SM_IO + rr * IO_ROW + ch * 16);
+    *reinterpret_cast<float4*>(gbase + (size_t)rr * stride + ch * 4) = v;
   }
 }
 
@@ -483,12 +572,13 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
                             WorkItem it) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int quad = warp & 3;
-  const int half = (warp - 2) >> 2;         // 0: columns/features of the first half, 1: the rest
+  const int half = (warp - 2) >> 2;         // 0: first 64 columns / features, 1: the rest
   const int r = quad * 32 + lane;           // row of the tile = TMEM lane
   const uint32_t tlane = c.tmem + ((uint32_t)(quad * 32) << 16);
   const float LN2 = 0.69314718055994530942f;
   volatile float* xch = reinterpret_cast<volatile float*>(c.gen + SM_IO + r * IO_ROW + 512);  // row padding
-  uint32_t epi_phase = 0, epi_unit = 0;
+  float4* const stage4 = reinterpret_cast<float4*>(c.gen + SM_IO + r * IO_ROW + half * 256);
+  uint32_t epi_phase = 0, epi_unit = 0, pair_phase = 0;
   int jj = 0;
   for (int u = first; u < n_units; u += stride) {
     WorkItem nxt = it;
@@ -497,159 +587,245 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     it = nxt;
     const int row = un.row0 + r;
     const bool row_valid = r < un.nrows;
-    float m_run = -INFINITY, l_part = 0.f;
-    float o_acc[64];
-#pragma unroll
-    for (int i = 0; i < 64; ++i) o_acc[i] = 0.f;
+    const bool active = quad * 32 < un.nrows;  // this warp holds at least one real row
+    float m_ref = -INFINITY, l_part = 0.f;
+    bool first_tile = true;
 
     for (int t = next_tile(un, un.t0); t < un.t1; t = next_tile(un, t + 1), ++jj) {
-      const int b = jj & 1, par = (jj >> 1) & 1;
-      const int tile_lo = un.key_base + t * BN;
-      const int v_lo = max(un.k0 - tile_lo, 0), v_hi = min(un.k1 - tile_lo, BN);
-      const int e_lo = un.x0 - tile_lo, e_hi = un.x1 - tile_lo;
-      const bool all_valid = v_lo == 0 && v_hi == BN && (un.x1 <= un.x0 || e_hi <= 0 || e_lo >= BN);
-      auto col_valid = [&](int j) { return j >= v_lo && j < v_hi && !(j >= e_lo && j < e_hi); };
-      if (!wait_bar(c, BAR_S_FULL + b, par, LOC_WAIT_S)) return;
+      const int b = jj & 1;
+      if (!wait_bar(c, BAR_S_FULL + b, (jj >> 1) & 1, LOC_WAIT_S)) return;
       tc_fence_after();
-      // row maximum over all 64 columns (both threads of the pair compute it);
-      // the thread's own 32 columns are read last and kept
-      float mx = -INFINITY;
-      uint32_t rr[32];
-      {
-        const int oc = 32 * (1 - half);
-        tmem_ld32(tlane + TM_S + 64 * b + oc, rr);
-        tmem_ld_wait();
-        if (all_valid) {
+      // every thread observes every completion of O_FULL exactly once and in
+      // order (parity waits must never skip a phase): here, for P~V of the
+      // previous tile, either before an in-place rescale or at the end of the tile
+      bool o_waited = first_tile;
+      if (active) {
+        const int tile_lo = un.key_base + t * BN;
+        const int v_lo = max(un.k0 - tile_lo, 0), v_hi = min(un.k1 - tile_lo, BN);
+        const int e_lo = un.x0 - tile_lo, e_hi = un.x1 - tile_lo;
+        const bool all_valid = v_lo == 0 && v_hi == BN && (un.x1 <= un.x0 || e_hi <= 0 || e_lo >= BN);
+        auto col_valid = [&](int j) { return j >= v_lo && j < v_hi && !(j >= e_lo && j < e_hi); };
+        const uint32_t s_addr = tlane + TS_S + 128 * b;
+        const int mc = 64 * half;   // this thread's 64 columns
+        // Pass 1: maximum over this thread's columns.  Instruction count on
+        // these threads is what limits the kernel, so a tile with no masked
+        // column (the common case) takes a path with no per-column tests, and
+        // the maximum runs as four independent chains.
+        float mx = -INFINITY;
+        {
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll 1
+          for (int cb = 0; cb < 2; ++cb) {
+            uint32_t rr[32];
+            tmem_ld32(s_addr + mc + 32 * cb, rr);
+            tmem_ld_wait();
+            if (all_valid) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(rr[j]));
-        } else {
+              for (int j = 0; j < 32; j += 4) {
+                m0 = fmaxf(m0, __uint_as_float(rr[j]));
+                m1 = fmaxf(m1, __uint_as_float(rr[j + 1]));
+                m2 = fmaxf(m2, __uint_as_float(rr[j + 2]));
+                m3 = fmaxf(m3, __uint_as_float(rr[j + 3]));
+              }
+            } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (col_valid(oc + j)) mx = fmaxf(mx, __uint_as_float(rr[j]));
+              for (int j = 0; j < 32; ++j)
+                if (col_valid(mc + 32 * cb + j)) m0 = fmaxf(m0, __uint_as_float(rr[j]));
+            }
+          }
+          mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
         }
-      }
-      const int mc = 32 * half;
-      tmem_ld32(tlane + TM_S + 64 * b + mc, rr);
-      tmem_ld_wait();
-      if (all_valid) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(rr[j]));
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (col_valid(mc + j)) mx = fmaxf(mx, __uint_as_float(rr[j]));
-      }
-      const float m_new = fmaxf(m_run, ceilf(mx * g.scale_log2));
-      const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-      const float alpha = (m_run == -INFINITY) ? 0.f : ex2(m_run - m_new);
-      // probabilities of this thread's 32 columns
-      float psum = 0.f;
-      uint32_t pk[16];
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        float p0 = ex2(fmaf(__uint_as_float(rr[2 * j]), g.scale_log2, -m_ref));
-        float p1 = ex2(fmaf(__uint_as_float(rr[2 * j + 1]), g.scale_log2, -m_ref));
-        if (!all_valid) {
-          if (!col_valid(mc + 2 * j)) p0 = 0.f;
-          if (!col_valid(mc + 2 * j + 1)) p1 = 0.f;
+        {
+          // exchange slots live in the row's staging payload (idle during the tile
+          // loop) and alternate between consecutive tiles
+          volatile float* mxch = reinterpret_cast<volatile float*>(c.gen + SM_IO + r * IO_ROW) + 2 * (pair_phase & 1u);
+          mxch[half] = mx;
+          mbar_arrive(c.bar(BAR_PAIR + quad));
+          if (!wait_bar(c, BAR_PAIR + quad, pair_phase & 1, LOC_WAIT_S)) return;
+          ++pair_phase;
+          mx = fmaxf(mxch[0], mxch[1]);
         }
-        p0 = round_to_half_bits(p0);
-        p1 = round_to_half_bits(p1);
-        psum += p0 + p1;  // the normaliser sums exactly what the MMA multiplies
-        __half2 hp = __floats2half2_rn(p0, p1);
-        pk[j] = *reinterpret_cast<uint32_t*>(&hp);
+        // integer reference exponent, moved only when the row maximum outgrows it
+        // by more than RESCALE_SLACK (so P~ <= 2^RESCALE_SLACK and rescales are rare)
+        const float cand = ceilf(mx * g.scale_log2);
+        float m_new = m_ref;
+        if (m_ref == -INFINITY || cand > m_ref + RESCALE_SLACK) m_new = fmaxf(m_ref, cand);
+        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+        float alpha = 1.f;
+        if (m_new != m_ref) alpha = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
+        if (!first_tile && __any_sync(0xffffffffu, alpha != 1.f)) {
+          // O~ in TMEM is rescaled in place: P~V of the previous tile must be done
+          if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
+          o_waited = true;
+          tc_fence_after();
+#pragma unroll 1
+          for (int cb = 0; cb < 4; ++cb) {
+            uint32_t rr[16];
+            tmem_ld16(tlane + TS_O + 64 * half + 16 * cb, rr);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) rr[j] = __float_as_uint(__uint_as_float(rr[j]) * alpha);
+            tmem_st16(tlane + TS_O + 64 * half + 16 * cb, rr, 0);
+          }
+        }
+        // Pass 2: probabilities of this thread's 64 columns.
+        float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll 1
+        for (int cb = 0; cb < 2; ++cb) {
+          uint32_t rr[32], pk[16];
+          tmem_ld32(s_addr + mc + 32 * cb, rr);
+          tmem_ld_wait();
+          if (all_valid) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              float p0 = round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j]), g.scale_log2, -m_use)));
+              float p1 = round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j + 1]), g.scale_log2, -m_use)));
+              ps0 += p0;  // the normaliser sums exactly what the MMA multiplies
+              ps1 += p1;
+              __half2 hp = __floats2half2_rn(p0, p1);
+              pk[j] = *reinterpret_cast<uint32_t*>(&hp);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int cidx = mc + 32 * cb + 2 * j;
+              float p0 = col_valid(cidx) ? round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j]), g.scale_log2, -m_use))) : 0.f;
+              float p1 = col_valid(cidx + 1) ? round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j + 1]), g.scale_log2, -m_use))) : 0.f;
+              ps0 += p0;
+              ps1 += p1;
+              __half2 hp = __floats2half2_rn(p0, p1);
+              pk[j] = *reinterpret_cast<uint32_t*>(&hp);
+            }
+          }
+          tmem_st16(tlane + TS_P + 64 * b + 32 * half + 16 * cb, pk);
+        }
+        const float psum = ps0 + ps1;
+        l_part = l_part * alpha + psum;
+        m_ref = m_new;
       }
-      tmem_st16(tlane + TM_P + 32 * b + 16 * half, pk);
       tmem_st_wait();
+      // (before the arrive below: P~V of this tile cannot have been issued yet,
+      // so O_FULL is at most one phase ahead of the one waited for)
+      if (!o_waited && !wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
       tc_fence_before();
       mbar_arrive(c.bar(BAR_P_FULL + b));
-      l_part = l_part * alpha + psum;
-      m_run = m_new;
-      // O~ = alpha O~ + P~ V for this thread's 64 features
-      if (!wait_bar(c, BAR_O_FULL + b, par, LOC_WAIT_O)) return;
-      tc_fence_after();
-#pragma unroll
-      for (int q2 = 0; q2 < 2; ++q2) {
-        tmem_ld32(tlane + TM_O + 128 * b + 64 * half + 32 * q2, rr);
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) o_acc[32 * q2 + j] = fmaf(o_acc[32 * q2 + j], alpha, __uint_as_float(rr[j]));
-      }
-      tc_fence_before();
-      mbar_arrive(c.bar(BAR_O_FREE + b));
+      first_tile = false;
     }
 
-    // ---- epilogue: combine the pair's normaliser, then store ----
+    // ---- epilogue ----
+    if (!first_tile) {  // the unit had key tiles: wait for the last P~V
+      if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
+      tc_fence_after();
+    }
+    // the pair's normaliser halves are combined through the row's padding
     // (slots alternate between consecutive units so a fast thread of the next
     // unit cannot overwrite a value its partner has not read yet)
     const int xs = 2 * (int)(epi_unit & 1u);
     ++epi_unit;
-    xch[xs + half] = l_part;
+    // (block-query units keep a key stage in the upper half of the staging
+    // region: only rows below 64 may touch their staging row there)
+    const bool own_stage = un.q_rows == BM || r < 64;
+    if (own_stage) xch[xs + half] = l_part;
     if (!epi_sync(c, epi_phase)) return;
-    const float l_run = xch[xs] + xch[xs + 1];
+    const float l_run = own_stage ? xch[xs] + xch[xs + 1] : 1.f;
+    const float mul = (un.epi == EPI_OUT) ? 1.f / l_run : 1.f;
+    // O~ (this thread's 64 features) from TMEM to the staging row
+#pragma unroll 1
+    for (int cb = 0; cb < 4; ++cb) {
+      uint32_t rr[16];
+      if (!first_tile) {
+        tmem_ld16(tlane + TS_O + 64 * half + 16 * cb, rr);
+        tmem_ld_wait();
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) rr[j] = 0u;
+      }
+      if (own_stage) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          stage4[4 * cb + i] = make_float4(__uint_as_float(rr[4 * i]) * mul, __uint_as_float(rr[4 * i + 1]) * mul,
+                                           __uint_as_float(rr[4 * i + 2]) * mul, __uint_as_float(rr[4 * i + 3]) * mul);
+      }
+    }
+    tc_fence_before();
+    mbar_arrive(c.bar(BAR_O_FREE));  // the next unit may overwrite O~
     if (un.epi == EPI_STATE) {
-      size_t srow = (size_t)un.h * g.Tp + row;
-      if (row_valid && half == 0) { a.st.m[srow] = m_run; a.st.l[srow] = l_run; }
-      stage_and_store(c, r, half, o_acc, 1.f, a.st.o + srow * D + 64 * half, row_valid);
+      const size_t srow = (size_t)un.h * g.Tp + row;
+      if (row_valid && half == 0) { a.st.m[srow] = m_ref; a.st.l[srow] = l_run; }
+      if (!epi_sync(c, epi_phase)) return;
+      coop_store_rows(c, a.st.o + ((size_t)un.h * g.Tp + un.row0) * D, D, un.nrows);
     } else if (un.epi == EPI_OUT) {
-      size_t orow = (size_t)row * g.Hq + un.h;
-      if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_run + log2f(l_run)) * LN2;
-      stage_and_store(c, r, half, o_acc, 1.f / l_run, a.out + orow * D + 64 * half, row_valid);
+      const size_t orow = (size_t)row * g.Hq + un.h;
+      if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_ref + log2f(l_run)) * LN2;
+      if (!epi_sync(c, epi_phase)) return;
+      coop_store_rows(c, a.out + ((size_t)un.row0 * g.Hq + un.h) * D, (size_t)g.Hq * D, un.nrows);
     } else {
       // partial state of this key chunk; the last chunk of the (sequence, head)
       // to arrive merges all of them
-      const size_t p0 = (((size_t)un.seq * g.Hq + un.h) * a.max_chunks) * g.block_len + r;
-      if (row_valid) {
-        const size_t pr = p0 + (size_t)un.chunk * g.block_len;
-        if (half == 0) { a.part_m[pr] = m_run; a.part_l[pr] = l_run; }
-        float4* dst = reinterpret_cast<float4*>(a.part_o + pr * D + 64 * half);
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-          dst[i] = make_float4(o_acc[4 * i], o_acc[4 * i + 1], o_acc[4 * i + 2], o_acc[4 * i + 3]);
-      }
-      __threadfence();
+      const size_t pbase = ((size_t)un.seq * g.Hq + un.h) * a.max_chunks;  // [chunk][block_len]
+      const size_t prow0 = (pbase + un.chunk) * g.block_len;
+      if (row_valid && half == 0) { a.part_m[prow0 + r] = m_ref; a.part_l[prow0 + r] = l_run; }
       if (!epi_sync(c, epi_phase)) return;
+      coop_store_rows(c, a.part_o + prow0 * D, D, un.nrows);
+      if (!epi_sync(c, epi_phase)) return;  // every partial store of the CTA happens-before thread 64's fence
       if (threadIdx.x == 64) {
+        __threadfence();  // cumulative: publishes the whole CTA's partial state before the count
         int* cnt = &a.counters[un.seq * g.Hq + un.h];
         int old = atomicAdd(cnt, 1);
         int last = (old == un.nchunks - 1) ? 1 : 0;
-        if (last) *cnt = 0;
+        if (last) {
+          *cnt = 0;
+          __threadfence();  // the other chunks' partial states are visible from here on
+        }
         *c.flag = (uint32_t)last;
-        __threadfence();
       }
       if (!epi_sync(c, epi_phase)) return;
-      // the flag is rewritten only after every row thread has passed two more
-      // rendezvous of a later unit, so reading it here is race-free
-      const bool last = *c.flag != 0;
-      if (last) {
-        __threadfence();
-        float M = -INFINITY, L = 0.f;
-        if (row_valid) {
-          for (int ch = 0; ch < un.nchunks; ++ch) M = fmaxf(M, __ldcg(a.part_m + p0 + (size_t)ch * g.block_len));
+      if (*c.flag != 0) {
+        // merge: thread t owns 16 bytes of one row; all partial rows are read
+        // with coalesced loads straight from L2
+        const int t = threadIdx.x - 64;
+        for (int i = t; i < un.nrows * 32; i += ROW_THREADS) {
+          const int rr = i >> 5, ch = i & 31;
+          float M = -INFINITY;
+          {
+            float mv[16];  // at most 16 chunks: all loads in flight together
 #pragma unroll
-          for (int i = 0; i < 64; ++i) o_acc[i] = 0.f;
-          for (int ch = 0; ch < un.nchunks; ++ch) {
-            const size_t pr = p0 + (size_t)ch * g.block_len;
-            const float mcv = __ldcg(a.part_m + pr);
-            if (mcv == -INFINITY) continue;
-            const float w = ex2(mcv - M);
-            L = fmaf(__ldcg(a.part_l + pr), w, L);
-            const float4* src = reinterpret_cast<const float4*>(a.part_o + pr * D + 64 * half);
+            for (int cc = 0; cc < 16; ++cc)
+              mv[cc] = __ldcg(a.part_m + (pbase + min(cc, un.nchunks - 1)) * g.block_len + rr);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              float4 v = __ldcg(src + i);
-              o_acc[4 * i] = fmaf(v.x, w, o_acc[4 * i]);
-              o_acc[4 * i + 1] = fmaf(v.y, w, o_acc[4 * i + 1]);
-              o_acc[4 * i + 2] = fmaf(v.z, w, o_acc[4 * i + 2]);
-              o_acc[4 * i + 3] = fmaf(v.w, w, o_acc[4 * i + 3]);
+            for (int cc = 0; cc < 16; ++cc) M = fmaxf(M, mv[cc]);
+          }
+          float L = 0.f;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int c0 = 0; c0 < un.nchunks; c0 += 4) {
+            float w[4];
+            float4 v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const int cc = min(c0 + k, un.nchunks - 1);
+              const size_t pr = (pbase + cc) * g.block_len + rr;
+              const float mcv = __ldcg(a.part_m + pr);
+              w[k] = (c0 + k < un.nchunks && mcv != -INFINITY) ? ex2(mcv - M) : 0.f;
+              L = fmaf(__ldcg(a.part_l + pr), w[k], L);
+              v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + pr * D) + ch);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              acc.x = fmaf(v[k].x, w[k], acc.x);
+              acc.y = fmaf(v[k].y, w[k], acc.y);
+              acc.z = fmaf(v[k].z, w[k], acc.z);
+              acc.w = fmaf(v[k].w, w[k], acc.w);
             }
           }
+          const float inv = 1.f / L;
+          const size_t orow = (size_t)(un.row0 + rr) * g.Hq + un.h;
+          *reinterpret_cast<float4*>(a.out + orow * D + ch * 4) =
+              make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+          if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
         }
-        size_t orow = (size_t)row * g.Hq + un.h;
-        if (row_valid && half == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
-        stage_and_store(c, r, half, o_acc, row_valid ? 1.f / L : 0.f, a.out + orow * D + 64 * half, row_valid);
       }
     }
+    if (!epi_sync(c, epi_phase)) return;  // the staging rows may be rewritten
   }
 }
 
@@ -687,7 +863,7 @@ __device__ void merge_mma(const Cta& c, const Geometry& g, const AttnArgs& a, in
     if (!wait_bar(c, BAR_Q_FULL, 0, LOC_WAIT_Q)) return;
     if (!wait_bar(c, BAR_KV_FULL, 0, LOC_WAIT_K)) return;
     tc_fence_after();
-    issue_s_mma(c, c.base + SM_KV, c.tmem + TM_S, BM * 128u, idesc_s);
+    issue_s_mma(c.base + SM_Q, BM * 128u, c.base + SM_KV, c.base + SM_KV + KV_KLO, K_BOX, c.tmem + TM_S, idesc_s);
     tc_commit(c.bar(BAR_S_FULL));
     tc_commit(c.bar(BAR_Q_FREE));
   }
@@ -696,7 +872,8 @@ __device__ void merge_mma(const Cta& c, const Geometry& g, const AttnArgs& a, in
     if (!wait_bar(c, BAR_P_FULL + b, k & 1, LOC_WAIT_S)) return;
     if (k >= 1 && !wait_bar(c, BAR_O_FREE + b, (k - 1) & 1, LOC_WAIT_O)) return;
     tc_fence_after();
-    issue_pv_mma(c.base + SM_KV + b * KV_STAGE, c.tmem + TM_P + 32 * b, c.tmem + TM_O + 128 * b, n_s / 16);
+    issue_pv_mma(c.base + SM_KV + b * KV_STAGE + KV_V, K_BOX, c.tmem + TM_P + 32 * b, c.tmem + TM_O + 128 * b, n_s / 16,
+                 0u);
     tc_commit(c.bar(BAR_O_FULL + b));
     tc_commit(c.bar(BAR_KV_FREE + b));
     if (u + stride < n_units) {  // scores of the next unit as soon as its tiles land
@@ -704,7 +881,8 @@ __device__ void merge_mma(const Cta& c, const Geometry& g, const AttnArgs& a, in
       if (!wait_bar(c, BAR_Q_FULL, (uu + 1) & 1, LOC_WAIT_Q)) return;
       if (!wait_bar(c, BAR_KV_FULL + bn, ((uu + 1) >> 1) & 1, LOC_WAIT_K)) return;
       tc_fence_after();
-      issue_s_mma(c, c.base + SM_KV + bn * KV_STAGE, c.tmem + TM_S + 64 * bn, BM * 128u, idesc_s);
+      issue_s_mma(c.base + SM_Q, BM * 128u, c.base + SM_KV + bn * KV_STAGE, c.base + SM_KV + bn * KV_STAGE + KV_KLO, K_BOX,
+                  c.tmem + TM_S + 64 * bn, idesc_s);
       tc_commit(c.bar(BAR_S_FULL + bn));
       tc_commit(c.bar(BAR_Q_FREE));
     }
@@ -871,6 +1049,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
       if (i == BAR_P_FULL || i == BAR_P_FULL1 || i == BAR_O_FREE || i == BAR_O_FREE1 || i == BAR_EPI)
         count = ROW_THREADS;
       if (i == BAR_DONE) count = THREADS;
+      if (i >= BAR_PAIR) count = 64;
       mbar_init(c.bar(i), count);
     }
     words[1] = 0;
@@ -997,6 +1176,9 @@ TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, c
             make_plane_map(&m->k_hi, rot.k_hi, g.Hkv, g.Tp, BN, false, err, errlen) &&
             make_plane_map(&m->k_lo, rot.k_lo, g.Hkv, g.Tp, BN, false, err, errlen) &&
             make_plane_map(&m->v, rot.v, g.Hkv, g.Tp, BN, true, err, errlen) &&
+            make_plane_map(&m->k64_hi, rot.k_hi, g.Hkv, g.Tp, 64, false, err, errlen) &&
+            make_plane_map(&m->k64_lo, rot.k_lo, g.Hkv, g.Tp, 64, false, err, errlen) &&
+            make_plane_map(&m->v64, rot.v, g.Hkv, g.Tp, 64, true, err, errlen) &&
             make_f32_map(&m->st_o, state_o, (cuuint64_t)g.Tp, (cuuint64_t)g.Hq, BM, 1, err, errlen);
   if (!ok) { delete m; return nullptr; }
   return m;
