@@ -195,10 +195,38 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   const bool tc = c->engine == LACACHE_ENGINE_TCGEN05;
   const int R = tc ? TC_ROWS : SIMT_ROWS;
   std::vector<WorkItem> items;
-  // block-query units: chunks of `tpc` key tiles, balanced over the sequence,
-  // at most 16 chunks (the partial-state merge reads them all)
+  // Block-query units: the keys of each (sequence, head) are cut into balanced
+  // chunks of `tpc` tiles.  Unless the caller fixes it, pick the chunk size and
+  // the role split together from a small cost model (times in microseconds,
+  // measured on B200: a stream unit costs ~5 + 3.5 per key tile, a merge unit
+  // ~3.4 after a ~4 us cold start), at most 16 chunks per sequence.
   int tpc = cfg->sc_tiles_per_chunk;
   if (const char* e = getenv("LACACHE_SC_TILES")) tpc = atoi(e);
+  if (tc && tpc <= 0) {
+    int max_nkt = 1;
+    long long rows_u = 0;
+    for (int b = 0; b < g.B; ++b) {
+      max_nkt = std::max(max_nkt, (c->cu[b + 1] - c->cu[b] + TC_KEYS - 1) / TC_KEYS);
+      int n_u = c->cu[b + 1] - c->cu[b] - g.block_len;
+      rows_u += (n_u + TC_ROWS - 1) / TC_ROWS + 1;
+    }
+    const int sms = 148;
+    const double units_m = (double)rows_u * g.Hq;
+    double best = 1e30;
+    for (int cand = 1; cand <= max_nkt; ++cand) {
+      double units_s = 0;
+      for (int b = 0; b < g.B; ++b) {
+        int nkt = (c->cu[b + 1] - c->cu[b] + TC_KEYS - 1) / TC_KEYS;
+        units_s += std::min(16, (nkt + cand - 1) / cand) * (double)g.Hq;
+      }
+      for (int ns = 8; ns <= sms - 8; ns += 4) {
+        double ts = ceil(units_s / ns) * (5.0 + 3.5 * cand);
+        double tm = 4.0 + ceil(units_m / (sms - ns)) * 3.4;
+        double t = std::max(ts, tm);
+        if (t < best - 1e-9) { best = t; tpc = cand; }
+      }
+    }
+  }
   if (tpc <= 0) tpc = 2;
   c->max_chunks = 1;
   for (int k = 0; k < g.n_blk; ++k) {
@@ -340,14 +368,20 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       a.items_merge = c->d_items + ml.off;
       a.n_items_merge = ml.n;
       long long units_merge = (long long)ml.n * Hq;
-      double cost_stream = 0.0;
+      int total = (int)std::min<long long>(c->num_sms, units_stream + units_merge);
+      int max_tiles = 1;
       for (int i = 0; i < list.n; ++i) {
         const WorkItem& w = c->items_host[list.off + i];
-        cost_stream += Hq * (1.5 + 1.0 * (w.kt1 - w.kt0));
+        max_tiles = std::max(max_tiles, w.kt1 - w.kt0);
       }
-      double cost_merge = 2.5 * (double)units_merge;
-      int total = (int)std::min<long long>(c->num_sms, units_stream + units_merge);
-      int ns = (int)lround(total * cost_stream / std::max(1e-9, cost_stream + cost_merge));
+      int ns = 1;
+      double best = 1e30;
+      for (int cand = 1; cand < total; ++cand) {
+        double ts = ceil((double)units_stream / cand) * (5.0 + 3.5 * max_tiles);
+        double tm = 4.0 + ceil((double)units_merge / (total - cand)) * 3.4;
+        double t = std::max(ts, tm);
+        if (t < best - 1e-9) { best = t; ns = cand; }
+      }
       if (c->stream_ctas_override > 0) ns = c->stream_ctas_override;
       if (units_merge == 0) ns = total;
       else ns = std::max(1, std::min(ns, total - 1));
