@@ -128,6 +128,43 @@ lacache_status lacache_full_recompute(lacache_ctx* ctx, const void* q_pre, const
                                       void* cuda_stream);
 
 /*
+ * Plain attention for ONE sequence (batch 1, all rows x all keys, the same
+ * result as lacache_full_recompute on a one-sequence context) for callers that
+ * must not allocate device memory.  The paper has no counterpart.
+ *
+ * Some callers cannot call cudaMalloc at all: code running inside a memory
+ * pool or arena that owns the whole device heap, plugins whose host forbids
+ * allocation after start-up, and latency-critical sections where an
+ * allocation's implicit device synchronisation is not acceptable.  They cannot
+ * create a context either (that allocates the caches).  This entry point needs
+ * no context and calls no cudaMalloc, cudaFree or other allocating routine:
+ * every piece of scratch (rotated q/k/v planes in fp32, RoPE tables, positions,
+ * the work list) lives in one fixed array inside the library's device image --
+ * about 18 MiB, held by every GPU that loads the library until the process
+ * exits.  The caller passes inputs and outputs only.
+ *
+ *   - q_pre [n_tokens, n_q_heads, head_dim], k_pre / v_pre [n_tokens,
+ *     n_kv_heads, head_dim] of `dtype`; out [n_tokens, n_q_heads, head_dim]
+ *     fp32; lse [n_tokens, n_q_heads] fp32 or NULL.  Device pointers, 16-byte
+ *     aligned.  softmax_scale <= 0 means 1/sqrt(head_dim).
+ *   - Limits: n_tokens <= 4096 and n_tokens * (n_q_heads + 2 * n_kv_heads) *
+ *     head_dim <= 4 Mi elements.  Anything larger returns LACACHE_ERR_SHAPE
+ *     (text in lacache_last_error(NULL)) and launches nothing.
+ *   - The first call on each device resolves the array's device address (with
+ *     that device current) and sets kernel attributes; make that first call
+ *     before starting any stream capture.
+ *   - All calls share the one array.  Nothing in it has to start at zero: each
+ *     call overwrites what it reads, and the previous call's contents are
+ *     simply left behind.  Two calls that overlap on the GPU (different
+ *     streams, or different host threads) race on it: serialise them.
+ *   - Runs the fp32 CUDA-core kernels (any dtype).
+ */
+lacache_status lacache_full_recompute_static(int dtype, int n_tokens, int n_q_heads, int n_kv_heads,
+                                             int head_dim, float rope_theta, float softmax_scale,
+                                             const void* q_pre, const void* k_pre, const void* v_pre,
+                                             float* out, float* lse, void* cuda_stream);
+
+/*
  * Same operations with HOST buffers: inputs are copied host->device and
  * results device->host on `cuda_stream` inside the call (asynchronously when
  * the host memory is pinned).  Staging is allocated on first use.  The caller

@@ -20,7 +20,8 @@ EXPORTS = [
     "lacache_version", "lacache_create", "lacache_destroy", "lacache_build", "lacache_step",
     "lacache_full_recompute", "lacache_build_host", "lacache_step_host", "lacache_export_state",
     "lacache_export_rope_cache", "lacache_export_index_meta", "lacache_total_tokens",
-    "lacache_last_launch_count", "lacache_engine", "lacache_set_timing_events", "lacache_poll_status", "lacache_last_error",
+    "lacache_last_launch_count", "lacache_engine", "lacache_set_timing_events",
+    "lacache_full_recompute_static", "lacache_poll_status", "lacache_last_error",
 ]
 
 
@@ -66,6 +67,8 @@ def load():
     lib.lacache_export_rope_cache.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_export_index_meta.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_set_timing_events.argtypes = [vp, vp, vp]
+    lib.lacache_full_recompute_static.argtypes = [ip, ip, ip, ip, ip, ctypes.c_float, ctypes.c_float, vp, vp, vp, vp,
+                                                  vp, vp]
     lib.lacache_total_tokens.argtypes = [vp]
     lib.lacache_last_launch_count.argtypes = [vp]
     lib.lacache_engine.argtypes = [vp]
@@ -88,6 +91,19 @@ def _stream(stream):
         import torch
         stream = torch.cuda.current_stream()
     return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def full_recompute_static(dtype, n_q_heads, n_kv_heads, head_dim, rope_theta, q_pre, k_pre, v_pre, out,
+                          lse=None, softmax_scale=0.0, stream=None):
+    """Plain attention for one sequence without any device allocation (the
+    scratch is a fixed array inside the library).  Mirrors
+    ``lacache_full_recompute_static``; raises LacacheError on a non-zero status."""
+    lib = load()
+    st = lib.lacache_full_recompute_static(int(dtype), int(q_pre.shape[0]), int(n_q_heads), int(n_kv_heads),
+                                           int(head_dim), float(rope_theta), float(softmax_scale), _ptr(q_pre),
+                                           _ptr(k_pre), _ptr(v_pre), _ptr(out), _ptr(lse), _stream(stream))
+    if st != OK:
+        raise LacacheError(st, (lib.lacache_last_error(None) or b"").decode())
 
 
 class Context:

@@ -445,6 +445,11 @@ lacache_status ensure_staging(lacache_ctx* c) {
 
 }  // namespace
 
+namespace lacache {
+// lets other translation units of the library set the text behind lacache_last_error(NULL)
+void set_thread_error(const char* msg) { snprintf(g_create_err, sizeof(g_create_err), "%s", msg); }
+}  // namespace lacache
+
 extern "C" {
 
 int lacache_version(void) { return 100; }
