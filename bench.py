@@ -415,9 +415,12 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
-# per-launch DRAM traffic of the step attention kernel from the committed ncu
-# capture (profiles/), bytes; None where no capture exists for the workload
-TRAFFIC_PER_LAUNCH = {}
+# per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the
+# step attention kernel from the committed ncu capture
+# (profiles/tc_attn_kernel_cfg2_ncu_full.txt), bytes; None where no capture
+# exists for the workload.  The fp32 output (12.6 MB) is still in L2 when the
+# kernel ends, so the figure is dominated by reads.
+TRAFFIC_PER_LAUNCH = {2: 45104000}
 
 
 # ----------------------------------------------------------------------------
