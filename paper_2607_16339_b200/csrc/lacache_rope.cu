@@ -76,6 +76,10 @@ __device__ __forceinline__ void store8_f16(void* plane, size_t off, const float 
 // [Hq,Hq+Hkv) k heads, [Hq+Hkv,Hq+2Hkv) v heads.
 template <bool TC>
 __global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a) {
+  // the attention kernel that follows may be launched programmatically
+  // dependent: let it start its prologue now (it waits for this grid's writes
+  // before it touches them)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int chunks = g.d / 16;
   const int slots = g.Hq + 2 * g.Hkv;
   const long long total = (long long)a.n_src_rows * slots * chunks;

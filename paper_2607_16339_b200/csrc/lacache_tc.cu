@@ -178,6 +178,10 @@ __device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t byt
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Programmatic dependent launch: blocks until the grid launched before this one
+// in the stream has completed and its writes are visible (returns at once when
+// the kernel was launched the ordinary way).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -439,6 +443,9 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
                                 int first, int stride, int n_units, WorkItem it) {
   const bool ks2 = a.mode == MODE_STEP;  // block-query units have room for two key stages
   int uu = 0, jj = 0;
+  // everything this role loads was written by the RoPE kernel launched just
+  // before this one: wait for that grid (this kernel may have started early)
+  grid_dependency_wait();
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
@@ -842,8 +849,6 @@ __device__ void merge_producer(const Cta& c, const TcMaps& maps, const Geometry&
     const int b = uu & 1, k = uu >> 1;
     if (uu >= 1 && !wait_bar(c, BAR_Q_FREE, (uu - 1) & 1, LOC_WAIT_Q)) return;
     load_q_tile(c, maps, BM, it.row0, h);
-    if (k >= 1 && !wait_bar(c, BAR_KV_FREE + b, (k - 1) & 1, LOC_WAIT_K)) return;
-    load_kv_tile(maps, c.base + SM_KV + b * KV_STAGE, c.bar(BAR_KV_FULL + b), it.blk_start, h / g.group);
     // cached O~ tile: four boxes of 32 features x 128 rows (rows past nrows are
     // read but never used)
     if (uu >= 1 && !wait_bar(c, BAR_IO_FREE, (uu - 1) & 1, LOC_WAIT_V)) return;
@@ -851,6 +856,11 @@ __device__ void merge_producer(const Cta& c, const TcMaps& maps, const Geometry&
 #pragma unroll
     for (int cb = 0; cb < 4; ++cb)
       tma_load_3d(c.base + SM_IO + cb * IO_BOX, &maps.st_o, c.bar(BAR_IO_FULL), 32 * cb, it.row0, h);
+    // the block's keys and values are the only thing here that the RoPE kernel
+    // launched just before this one writes: wait for that grid once
+    if (uu == 0) grid_dependency_wait();
+    if (k >= 1 && !wait_bar(c, BAR_KV_FREE + b, (k - 1) & 1, LOC_WAIT_K)) return;
+    load_kv_tile(maps, c.base + SM_KV + b * KV_STAGE, c.bar(BAR_KV_FULL + b), it.blk_start, h / g.group);
     it = nxt;
   }
 }
@@ -1188,8 +1198,19 @@ void tc_free_maps(TcMaps* m) { delete m; }
 
 cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* maps, cudaStream_t s) {
   if (a.n_ctas <= 0) return cudaSuccess;
-  tc_attn_kernel<<<a.n_ctas, THREADS, SM_TOTAL, s>>>(*maps, g, a);
-  return cudaGetLastError();
+  // launched programmatically dependent on the RoPE kernel enqueued just before:
+  // set-up and every load that does not depend on it overlap that kernel
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(a.n_ctas);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = SM_TOTAL;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, tc_attn_kernel, *maps, g, a);
 }
 
 }  // namespace lacache
