@@ -66,29 +66,31 @@ constexpr int ROW_THREADS = ROW_WARPS * 32;
 constexpr int THREADS = 64 + ROW_THREADS;
 
 // ---- shared memory map (bytes from a 1024-aligned base) ----
-constexpr uint32_t SM_Q = 0;                      // Q hi plane, then lo plane at +32 KB
-constexpr uint32_t SM_Q_LO = 32768;
-// stream role: one tile of 128 keys: K hi (2 boxes of 16 KB), K lo, then V
+constexpr uint32_t SM_Q = 0;                      // Q hi plane (two boxes), then the lo plane
+// stream role: two stages of one 128-key tile {K hi (2 boxes of 16 KB), K lo}, one V tile
 constexpr uint32_t SM_K = 65536;
+constexpr uint32_t K_STAGE = 65536;
 constexpr uint32_t SK_LO = 32768;
-constexpr uint32_t SM_V = SM_K + 65536;
+constexpr uint32_t SM_V = SM_K + 2 * K_STAGE;
 constexpr uint32_t KS_BOX = 128 * 128;            // one [128 rows][64 cols] 16-bit box
-// merge role: the same 96 KB hold 2 stages of the block's keys: {K hi, K lo, V} of 64 rows
+// The stream role stages its epilogue (128 rows x 512 B, 16-byte chunks XOR-swizzled
+// by the row so row-wise writes and row-wise reads are both conflict-free) in the
+// Q region: in all of it for 128-row units (the next unit's Q load waits for the
+// epilogue), in its upper half for 64-row units (whose Q tile needs only the lower half).
+constexpr uint32_t STAGE_ROW = 512;
+// merge role: the 96 KB after Q hold 2 stages of the block's keys {K hi, K lo, V} of 64
+// rows, then the staging tile of the cached O~ / the output
 constexpr uint32_t SM_KV = SM_K;
 constexpr uint32_t KV_STAGE = 49152;
 constexpr uint32_t KV_KLO = 16384;
 constexpr uint32_t KV_V = 32768;
 constexpr uint32_t K_BOX = 64 * 128;              // one [64 rows][64 cols] 16-bit box
-constexpr uint32_t SM_IO = SM_V + 32768;          // staging: 128 rows x (512 + 16) bytes
-constexpr uint32_t IO_ROW = 528;
-constexpr uint32_t IO_BOX = 128 * 128;            // merge role: one swizzled box of 32 fp32 columns x 128 rows
-// stream role, block-query units only (64-row Q tile, at most 64 staging rows): a second
-// key stage in the unused halves of the Q and staging regions
-constexpr uint32_t SM_K1_HI = SM_Q + 32768;
-constexpr uint32_t SM_K1_LO = SM_IO + 64 * IO_ROW;
-static_assert(SM_K1_LO % 1024 == 0, "swizzled tiles need 1024-byte alignment");
-constexpr uint32_t SM_BAR = SM_IO + BM * IO_ROW;
-static_assert(SM_K1_LO + 32768 <= SM_BAR, "second key stage overruns the staging region");
+constexpr uint32_t SM_IO = SM_KV + 2 * KV_STAGE;  // four swizzled boxes of 32 fp32 columns x 128 rows
+constexpr uint32_t IO_BOX = 128 * 128;
+// both roles: 16 bytes per row for exchanges between the two threads of a row
+constexpr uint32_t SM_XCH = SM_V + 32768;
+static_assert(SM_IO + 4 * IO_BOX <= SM_XCH, "merge-role staging overruns");
+constexpr uint32_t SM_BAR = SM_XCH + BM * 16;
 constexpr uint32_t SM_TOTAL = SM_BAR + 256;
 static_assert(SM_TOTAL <= 232448, "exceeds the 227 KB per-CTA limit");
 
@@ -441,7 +443,6 @@ __device__ __forceinline__ void load_q_tile(const Cta& c, const TcMaps& maps, in
 // ===========================================================================
 __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a,
                                 int first, int stride, int n_units, WorkItem it) {
-  const bool ks2 = a.mode == MODE_STEP;  // block-query units have room for two key stages
   int uu = 0, jj = 0;
   // everything this role loads was written by the RoPE kernel launched just
   // before this one: wait for that grid (this kernel may have started early)
@@ -456,10 +457,10 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
       const int krow = un.key_base + t * BN;
       // keys: a stage is free as soon as the scores that read it have been computed
       {
-        const int sk = ks2 ? (jj & 1) : 0, kuse = ks2 ? (jj >> 1) : jj;
+        const int sk = jj & 1, kuse = jj >> 1;
         if (kuse >= 1 && !wait_bar(c, sk ? BAR_K_FREE1 : BAR_K_FREE, (kuse - 1) & 1, LOC_WAIT_K)) return;
         const uint32_t bar = c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL);
-        const uint32_t khi = c.base + (sk ? SM_K1_HI : SM_K), klo = c.base + (sk ? SM_K1_LO : SM_K + SK_LO);
+        const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
         mbar_expect_tx(bar, 4 * KS_BOX);
         tma_load_3d(khi, &maps.k_hi, bar, 0, krow, un.kh);
         tma_load_3d(khi + KS_BOX, &maps.k_hi, bar, 64, krow, un.kh);
@@ -486,7 +487,6 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
 __device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units,
                            WorkItem it) {
   constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
-  const bool ks2 = a.mode == MODE_STEP;
   int uu = 0, js = 0, jp = 0;  // global counters of score tiles / PV tiles issued
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
@@ -518,10 +518,10 @@ __device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, i
         }
       }
       if (!did && ts < un.t1 && js - jp < 2) {
-        const int sk = ks2 ? (js & 1) : 0, kuse = ks2 ? (js >> 1) : js;
+        const int sk = js & 1, kuse = js >> 1;
         if (mbar_test(c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL), kuse & 1)) {
           const int b = js & 1;
-          const uint32_t khi = c.base + (sk ? SM_K1_HI : SM_K), klo = c.base + (sk ? SM_K1_LO : SM_K + SK_LO);
+          const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
           tc_fence_after();
           issue_s_mma(c.base + SM_Q, q_box, khi, klo, KS_BOX, c.tmem + TS_S + 128 * b, IDESC_S);
           tc_commit(c.bar(BAR_S_FULL + b));
@@ -563,14 +563,15 @@ __device__ __forceinline__ bool epi_sync(const Cta& c, uint32_t& phase) {
   return ok;
 }
 
-// Cooperative, fully coalesced copy of the first nrows staging rows (512 B of
-// payload each) to rows of `stride` floats in global memory: every warp-wide
-// store writes one whole row.
-__device__ __forceinline__ void coop_store_rows(const Cta& c, float* gbase, size_t stride, int nrows) {
+// Cooperative, fully coalesced copy of the first nrows staging rows (512 B each,
+// chunks XOR-swizzled by the row) to rows of `stride` floats in global memory:
+// every warp-wide store writes one whole row.
+__device__ __forceinline__ void coop_store_rows(const Cta& c, uint32_t stage_off, float* gbase, size_t stride,
+                                                int nrows) {
   const int t = threadIdx.x - 64;
   for (int i = t; i < nrows * 32; i += ROW_THREADS) {
     const int rr = i >> 5, ch = i & 31;
-    float4 v = *reinterpret_cast<const float4*>(c.gen + SM_IO + rr * IO_ROW + ch * 16);
+    float4 v = *reinterpret_cast<const float4*>(c.gen + stage_off + rr * STAGE_ROW + ((ch ^ (rr & 7)) << 4));
     *reinterpret_cast<float4*>(gbase + (size_t)rr * stride + ch * 4) = v;
   }
 }
@@ -583,9 +584,8 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
   const int r = quad * 32 + lane;           // row of the tile = TMEM lane
   const uint32_t tlane = c.tmem + ((uint32_t)(quad * 32) << 16);
   const float LN2 = 0.69314718055994530942f;
-  volatile float* xch = reinterpret_cast<volatile float*>(c.gen + SM_IO + r * IO_ROW + 512);  // row padding
-  float4* const stage4 = reinterpret_cast<float4*>(c.gen + SM_IO + r * IO_ROW + half * 256);
-  uint32_t epi_phase = 0, epi_unit = 0, pair_phase = 0;
+  volatile float* xch = reinterpret_cast<volatile float*>(c.gen + SM_XCH + r * 16);  // 4 exchange slots per row
+  uint32_t epi_phase = 0, epi_unit = 0, pair_phase = 0, xslot = 0;
   int jj = 0;
   for (int u = first; u < n_units; u += stride) {
     WorkItem nxt = it;
@@ -643,9 +643,9 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
           mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
         }
         {
-          // exchange slots live in the row's staging payload (idle during the tile
-          // loop) and alternate between consecutive tiles
-          volatile float* mxch = reinterpret_cast<volatile float*>(c.gen + SM_IO + r * IO_ROW) + 2 * (pair_phase & 1u);
+          // the slots alternate between consecutive exchanges
+          volatile float* mxch = xch + 2 * (xslot & 1u);
+          ++xslot;
           mxch[half] = mx;
           mbar_arrive(c.bar(BAR_PAIR + quad));
           if (!wait_bar(c, BAR_PAIR + quad, pair_phase & 1, LOC_WAIT_S)) return;
@@ -720,23 +720,29 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     }
 
     // ---- epilogue ----
+    // second arrival on Q_FREE (the first is the MMA thread's commit): a 64-row
+    // unit stages outside its Q tile, so its Q region may be reloaded at once
+    if (un.q_rows != BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));
     if (!first_tile) {  // the unit had key tiles: wait for the last P~V
       if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
       tc_fence_after();
     }
-    // the pair's normaliser halves are combined through the row's padding
-    // (slots alternate between consecutive units so a fast thread of the next
-    // unit cannot overwrite a value its partner has not read yet)
-    const int xs = 2 * (int)(epi_unit & 1u);
+    // the pair combines its normaliser halves (same alternating slots as the
+    // per-tile maximum exchange, which is over for this unit)
     ++epi_unit;
-    // (block-query units keep a key stage in the upper half of the staging
-    // region: only rows below 64 may touch their staging row there)
-    const bool own_stage = un.q_rows == BM || r < 64;
-    if (own_stage) xch[xs + half] = l_part;
+    volatile float* lx = xch + 2 * (xslot & 1u);
+    ++xslot;
+    lx[half] = l_part;
     if (!epi_sync(c, epi_phase)) return;
-    const float l_run = own_stage ? xch[xs] + xch[xs + 1] : 1.f;
+    const float l_run = lx[0] + lx[1];
     const float mul = (un.epi == EPI_OUT) ? 1.f / l_run : 1.f;
-    // O~ (this thread's 64 features) from TMEM to the staging row
+    // O~ (this thread's 64 features) from TMEM to its staging row.  The staging
+    // area is the Q region (every score MMA of the unit is complete: the last
+    // P~V, waited for above, was issued after them); 64-row units use its upper
+    // half, which their Q tiles never touch.
+    const uint32_t stage_off = SM_Q + (un.q_rows == BM ? 0u : 32768u);
+    const bool own_stage = un.q_rows == BM || r < 64;
+    uint8_t* const srow = c.gen + stage_off + r * STAGE_ROW;
 #pragma unroll 1
     for (int cb = 0; cb < 4; ++cb) {
       uint32_t rr[16];
@@ -749,9 +755,12 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       }
       if (own_stage) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-          stage4[4 * cb + i] = make_float4(__uint_as_float(rr[4 * i]) * mul, __uint_as_float(rr[4 * i + 1]) * mul,
-                                           __uint_as_float(rr[4 * i + 2]) * mul, __uint_as_float(rr[4 * i + 3]) * mul);
+        for (int i = 0; i < 4; ++i) {
+          const int ch = 16 * half + 4 * cb + i;
+          *reinterpret_cast<float4*>(srow + ((ch ^ (r & 7)) << 4)) =
+              make_float4(__uint_as_float(rr[4 * i]) * mul, __uint_as_float(rr[4 * i + 1]) * mul,
+                          __uint_as_float(rr[4 * i + 2]) * mul, __uint_as_float(rr[4 * i + 3]) * mul);
+        }
       }
     }
     tc_fence_before();
@@ -760,12 +769,12 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       const size_t srow = (size_t)un.h * g.Tp + row;
       if (row_valid && half == 0) { a.st.m[srow] = m_ref; a.st.l[srow] = l_run; }
       if (!epi_sync(c, epi_phase)) return;
-      coop_store_rows(c, a.st.o + ((size_t)un.h * g.Tp + un.row0) * D, D, un.nrows);
+      coop_store_rows(c, stage_off, a.st.o + ((size_t)un.h * g.Tp + un.row0) * D, D, un.nrows);
     } else if (un.epi == EPI_OUT) {
       const size_t orow = (size_t)row * g.Hq + un.h;
       if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_ref + log2f(l_run)) * LN2;
       if (!epi_sync(c, epi_phase)) return;
-      coop_store_rows(c, a.out + ((size_t)un.row0 * g.Hq + un.h) * D, (size_t)g.Hq * D, un.nrows);
+      coop_store_rows(c, stage_off, a.out + ((size_t)un.row0 * g.Hq + un.h) * D, (size_t)g.Hq * D, un.nrows);
     } else {
       // partial state of this key chunk; the last chunk of the (sequence, head)
       // to arrive merges all of them
@@ -773,7 +782,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       const size_t prow0 = (pbase + un.chunk) * g.block_len;
       if (row_valid && half == 0) { a.part_m[prow0 + r] = m_ref; a.part_l[prow0 + r] = l_run; }
       if (!epi_sync(c, epi_phase)) return;
-      coop_store_rows(c, a.part_o + prow0 * D, D, un.nrows);
+      coop_store_rows(c, stage_off, a.part_o + prow0 * D, D, un.nrows);
       if (!epi_sync(c, epi_phase)) return;  // every partial store of the CTA happens-before thread 64's fence
       if (threadIdx.x == 64) {
         __threadfence();  // cumulative: publishes the whole CTA's partial state before the count
@@ -832,7 +841,8 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         }
       }
     }
-    if (!epi_sync(c, epi_phase)) return;  // the staging rows may be rewritten
+    if (!epi_sync(c, epi_phase)) return;  // the staging rows have been read
+    if (un.q_rows == BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));  // the Q region may be reloaded
   }
 }
 
@@ -1059,6 +1069,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
       if (i == BAR_P_FULL || i == BAR_P_FULL1 || i == BAR_O_FREE || i == BAR_O_FREE1 || i == BAR_EPI)
         count = ROW_THREADS;
       if (i == BAR_DONE) count = THREADS;
+      if (i == BAR_Q_FREE && stream) count = 2;  // score MMAs done + epilogue staging read
       if (i >= BAR_PAIR) count = 64;
       mbar_init(c.bar(i), count);
     }
