@@ -198,8 +198,9 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   // Block-query units: the keys of each (sequence, head) are cut into balanced
   // chunks of `tpc` tiles.  Unless the caller fixes it, pick the chunk size and
   // the role split together from a small cost model (times in microseconds,
-  // measured on B200: a stream unit costs ~5 + 3.5 per key tile, a merge unit
-  // ~3.4 after a ~4 us cold start), at most 16 chunks per sequence.
+  // measured on B200: a stream unit costs ~2 + 2.1 per key tile, plus ~4 + 1.2
+  // per chunk when partial states have to be merged; a merge unit ~3.4
+  // after a ~4 us cold start), at most 16 chunks per sequence.
   int tpc = cfg->sc_tiles_per_chunk;
   if (const char* e = getenv("LACACHE_SC_TILES")) tpc = atoi(e);
   if (tc && tpc <= 0) {
@@ -215,12 +216,16 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     double best = 1e30;
     for (int cand = 1; cand <= max_nkt; ++cand) {
       double units_s = 0;
+      int max_ch = 1;
       for (int b = 0; b < g.B; ++b) {
         int nkt = (c->cu[b + 1] - c->cu[b] + TC_KEYS - 1) / TC_KEYS;
-        units_s += std::min(16, (nkt + cand - 1) / cand) * (double)g.Hq;
+        int ch = std::min(16, (nkt + cand - 1) / cand);
+        max_ch = std::max(max_ch, ch);
+        units_s += ch * (double)g.Hq;
       }
+      const double merge_cost = max_ch > 1 ? 4.0 + 1.2 * max_ch : 0.0;
       for (int ns = 8; ns <= sms - 8; ns += 4) {
-        double ts = ceil(units_s / ns) * (5.0 + 3.5 * cand);
+        double ts = ceil(units_s / ns) * (2.0 + 2.1 * cand + merge_cost);
         double tm = 4.0 + ceil(units_m / (sms - ns)) * 3.4;
         double t = std::max(ts, tm);
         if (t < best - 1e-9) { best = t; tpc = cand; }
@@ -377,7 +382,7 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       int ns = 1;
       double best = 1e30;
       for (int cand = 1; cand < total; ++cand) {
-        double ts = ceil((double)units_stream / cand) * (5.0 + 3.5 * max_tiles);
+        double ts = ceil((double)units_stream / cand) * (2.0 + 2.1 * max_tiles + (c->max_chunks > 1 ? 4.0 + 1.2 * c->max_chunks : 0.0));
         double tm = 4.0 + ceil((double)units_merge / (total - cand)) * 3.4;
         double t = std::max(ts, tm);
         if (t < best - 1e-9) { best = t; ns = cand; }

@@ -123,7 +123,7 @@ void tc_free_maps(TcMaps* m);
 
 constexpr int SIMT_ROWS = 32;    // query rows per SIMT work item
 constexpr int TC_ROWS = 128;     // query rows per tcgen05 work item
-constexpr int TC_KEYS = 128;     // keys per tcgen05 key tile (stream role)
+constexpr int TC_KEYS = 96;      // keys per tcgen05 key tile (stream role)
 constexpr int TC_MAX_BLOCK = 64; // largest block length the tcgen05 merge role handles
 
 }  // namespace lacache

@@ -34,6 +34,7 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <stdio.h>
+#include <stdlib.h>
 
 #include "lacache_internal.h"
 
@@ -59,7 +60,9 @@ namespace {
 
 constexpr int D = 128;
 constexpr int BM = TC_ROWS;   // 128 query rows (TMEM lanes)
-constexpr int BN = TC_KEYS;   // 128 keys per tile (stream role)
+constexpr int BN = TC_KEYS;   // 96 keys per tile (stream role): two stages of keys AND of values fit
+constexpr int HC = BN / 2;    // columns per row thread
+static_assert(BN % 32 == 0 && BN <= 128, "tile width");
 constexpr float RESCALE_SLACK = 3.f;
 constexpr int ROW_WARPS = 8;
 constexpr int ROW_THREADS = ROW_WARPS * 32;
@@ -67,12 +70,14 @@ constexpr int THREADS = 64 + ROW_THREADS;
 
 // ---- shared memory map (bytes from a 1024-aligned base) ----
 constexpr uint32_t SM_Q = 0;                      // Q hi plane (two boxes), then the lo plane
-// stream role: two stages of one 128-key tile {K hi (2 boxes of 16 KB), K lo}, one V tile
+// stream role: two stages of one key tile {K hi (2 boxes), K lo (2 boxes)}, two stages of V
 constexpr uint32_t SM_K = 65536;
-constexpr uint32_t K_STAGE = 65536;
-constexpr uint32_t SK_LO = 32768;
-constexpr uint32_t SM_V = SM_K + 2 * K_STAGE;
-constexpr uint32_t KS_BOX = 128 * 128;            // one [128 rows][64 cols] 16-bit box
+constexpr uint32_t KS_BOX = BN * 128;             // one [BN rows][64 cols] 16-bit box
+constexpr uint32_t K_STAGE = 4 * KS_BOX;          // K hi (2 boxes), K lo (2 boxes)
+constexpr uint32_t SK_LO = 2 * KS_BOX;
+constexpr uint32_t SM_V = SM_K + 2 * K_STAGE;     // two stages of V (2 boxes each)
+constexpr uint32_t V_STAGE = 2 * KS_BOX;
+static_assert(KS_BOX % 1024 == 0, "swizzled boxes need 1024-byte alignment");
 // The stream role stages its epilogue (128 rows x 512 B, 16-byte chunks XOR-swizzled
 // by the row so row-wise writes and row-wise reads are both conflict-free) in the
 // Q region: in all of it for 128-row units (the next unit's Q load waits for the
@@ -88,7 +93,8 @@ constexpr uint32_t K_BOX = 64 * 128;              // one [64 rows][64 cols] 16-b
 constexpr uint32_t SM_IO = SM_KV + 2 * KV_STAGE;  // four swizzled boxes of 32 fp32 columns x 128 rows
 constexpr uint32_t IO_BOX = 128 * 128;
 // both roles: 16 bytes per row for exchanges between the two threads of a row
-constexpr uint32_t SM_XCH = SM_V + 32768;
+constexpr uint32_t SM_XCH = 229376;
+static_assert(SM_V + 2 * V_STAGE <= SM_XCH, "stream-role tiles overrun");
 static_assert(SM_IO + 4 * IO_BOX <= SM_XCH, "merge-role staging overruns");
 constexpr uint32_t SM_BAR = SM_XCH + BM * 16;
 constexpr uint32_t SM_TOTAL = SM_BAR + 256;
@@ -100,8 +106,8 @@ constexpr uint32_t TM_S = 0;      // 2 x 64: scores
 constexpr uint32_t TM_P = 128;    // 2 x 32: fp16 probabilities, two per column
 constexpr uint32_t TM_O = 256;    // 2 x 128: P.V of one unit
 // stream role
-constexpr uint32_t TS_S = 0;      // 2 x 128: scores
-constexpr uint32_t TS_P = 256;    // 2 x 64: fp16 probabilities
+constexpr uint32_t TS_S = 0;      // 2 x 128 (BN used): scores
+constexpr uint32_t TS_P = 256;    // 2 x 64 (BN/2 used): fp16 probabilities
 constexpr uint32_t TS_O = 384;    // 128: O~ accumulated over the tiles of a unit
 constexpr uint32_t TM_COLS = 512;
 
@@ -113,7 +119,7 @@ enum {
   BAR_S_FULL, BAR_S_FULL1, BAR_P_FULL, BAR_P_FULL1,
   BAR_O_FULL, BAR_O_FULL1, BAR_O_FREE, BAR_O_FREE1,
   BAR_IO_FULL, BAR_IO_FREE, BAR_EPI, BAR_DONE,
-  BAR_K_FULL1, BAR_K_FREE1,  // stream role, second key stage (block-query units)
+  BAR_K_FULL1, BAR_K_FREE1, BAR_V_FULL1, BAR_V_FREE1,  // stream role, second key / value stage
   BAR_PAIR,  // 4 barriers: the two warps that share a TMEM lane quadrant
   N_BARS = BAR_PAIR + 4
 };
@@ -390,20 +396,26 @@ __device__ __forceinline__ int next_tile(const Unit& un, int t) {
   return t;
 }
 
-// S (+)= Q' K'^T as hi.hi + hi.lo + lo.hi; Q planes at q_base (lo at +32 KB) with
-// boxes of q_box bytes, K planes at k_hi / k_lo with boxes of k_box bytes.
+// S (+)= Q' K'^T as hi.hi + hi.lo + lo.hi; Q planes at q_base (lo plane after the hi
+// plane's two boxes) with boxes of q_box bytes, K planes at k_hi / k_lo with boxes of
+// k_box bytes.  The four base descriptors are built once; each MMA adds a small
+// constant to the start-address field (a single thread issues these back to back,
+// so every instruction saved here shortens the critical path).
 __device__ __forceinline__ void issue_s_mma(uint32_t q_base, uint32_t q_box, uint32_t k_hi, uint32_t k_lo,
                                             uint32_t k_box, uint32_t s_tmem, uint32_t idesc) {
+  const uint64_t qd[2] = {smem_desc(q_base, 16, 1024), smem_desc(q_base + 2u * q_box, 16, 1024)};
+  const uint64_t kd[2] = {smem_desc(k_hi, 16, 1024), smem_desc(k_lo, 16, 1024)};
+  const uint32_t qb16 = q_box >> 4, kb16 = k_box >> 4;
   uint32_t acc = 0;
 #pragma unroll
   for (int term = 0; term < 3; ++term) {
-    const uint32_t qa = q_base + (term == 2 ? 2u * q_box : 0u);
-    const uint32_t ka = term == 1 ? k_lo : k_hi;
+    const uint64_t qa = qd[term == 2 ? 1 : 0];
+    const uint64_t ka = kd[term == 1 ? 1 : 0];
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
-      uint32_t qoff = (ks >> 2) * q_box + (ks & 3) * 32;
-      uint32_t koff = (ks >> 2) * k_box + (ks & 3) * 32;
-      mma_ss(s_tmem, smem_desc(qa + qoff, 16, 1024), smem_desc(ka + koff, 16, 1024), idesc, acc);
+      const uint32_t qoff = (ks >> 2) * qb16 + (ks & 3) * 2;
+      const uint32_t koff = (ks >> 2) * kb16 + (ks & 3) * 2;
+      mma_ss(s_tmem, qa + qoff, ka + koff, idesc, acc);
       acc = 1;
     }
   }
@@ -414,8 +426,9 @@ __device__ __forceinline__ void issue_s_mma(uint32_t q_base, uint32_t q_box, uin
 __device__ __forceinline__ void issue_pv_mma(uint32_t v_base, uint32_t v_box, uint32_t p_tmem, uint32_t o_tmem,
                                              int ksteps, uint32_t accumulate) {
   constexpr uint32_t idesc = idesc_f16(0u /*fp16*/, 1u, BM, D);
+  const uint64_t vd = smem_desc(v_base, v_box, 1024);
   for (int ks = 0; ks < ksteps; ++ks)
-    mma_ts(o_tmem, p_tmem + 8 * ks, smem_desc(v_base + ks * 2048, v_box, 1024), idesc, (ks > 0) ? 1u : accumulate);
+    mma_ts(o_tmem, p_tmem + 8 * ks, vd + (uint64_t)(ks * (2048 >> 4)), idesc, (ks > 0) ? 1u : accumulate);
 }
 __device__ __forceinline__ void load_kv_tile(const TcMaps& maps, uint32_t kv_base, uint32_t bar, int krow, int kh) {
   mbar_expect_tx(bar, 6 * K_BOX);
@@ -467,10 +480,11 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         tma_load_3d(klo, &maps.k_lo, bar, 0, krow, un.kh);
         tma_load_3d(klo + KS_BOX, &maps.k_lo, bar, 64, krow, un.kh);
       }
-      // values: free once P~V of the previous tile has been computed
-      if (jj >= 1 && !wait_bar(c, BAR_V_FREE, (jj - 1) & 1, LOC_WAIT_V)) return;
+      // values: a stage is free once the P~V that read it has been computed
       {
-        const uint32_t bar = c.bar(BAR_V_FULL), vb = c.base + SM_V;
+        const int sv = jj & 1, vuse = jj >> 1;
+        if (vuse >= 1 && !wait_bar(c, sv ? BAR_V_FREE1 : BAR_V_FREE, (vuse - 1) & 1, LOC_WAIT_V)) return;
+        const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
         mbar_expect_tx(bar, 2 * KS_BOX);
         tma_load_3d(vb, &maps.v, bar, 0, krow, un.kh);
         tma_load_3d(vb + KS_BOX, &maps.v, bar, 64, krow, un.kh);
@@ -502,15 +516,18 @@ __device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, i
       bool did = false;
       if (js > jp) {  // scores of tile jp issued: its P~V may be ready
         const int b = jp & 1;
-        if (mbar_test(c.bar(BAR_P_FULL + b), (jp >> 1) & 1) && mbar_test(c.bar(BAR_V_FULL), jp & 1)) {
+        const int sv = jp & 1;
+        if (mbar_test(c.bar(BAR_P_FULL + b), (jp >> 1) & 1) &&
+            mbar_test(c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), (jp >> 1) & 1)) {
           if (o_free_pending) {  // the row threads have read the previous unit's O~
             if (!wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
             o_free_pending = false;
           }
           tc_fence_after();
-          issue_pv_mma(c.base + SM_V, KS_BOX, c.tmem + TS_P + 64 * b, c.tmem + TS_O, BN / 16, first_pv ? 0u : 1u);
+          issue_pv_mma(c.base + SM_V + sv * V_STAGE, KS_BOX, c.tmem + TS_P + 64 * b, c.tmem + TS_O, BN / 16,
+                       first_pv ? 0u : 1u);
           tc_commit(c.bar(BAR_O_FULL));
-          tc_commit(c.bar(BAR_V_FREE));
+          tc_commit(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE));
           first_pv = false;
           tp = next_tile(un, tp + 1);
           ++jp;
@@ -613,7 +630,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         const bool all_valid = v_lo == 0 && v_hi == BN && (un.x1 <= un.x0 || e_hi <= 0 || e_lo >= BN);
         auto col_valid = [&](int j) { return j >= v_lo && j < v_hi && !(j >= e_lo && j < e_hi); };
         const uint32_t s_addr = tlane + TS_S + 128 * b;
-        const int mc = 64 * half;   // this thread's 64 columns
+        const int mc = HC * half;   // this thread's columns
         // Pass 1: maximum over this thread's columns.  Instruction count on
         // these threads is what limits the kernel, so a tile with no masked
         // column (the common case) takes a path with no per-column tests, and
@@ -622,13 +639,13 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         {
           float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll 1
-          for (int cb = 0; cb < 2; ++cb) {
-            uint32_t rr[32];
-            tmem_ld32(s_addr + mc + 32 * cb, rr);
+          for (int cb = 0; cb < HC / 16; ++cb) {
+            uint32_t rr[16];
+            tmem_ld16(s_addr + mc + 16 * cb, rr);
             tmem_ld_wait();
             if (all_valid) {
 #pragma unroll
-              for (int j = 0; j < 32; j += 4) {
+              for (int j = 0; j < 16; j += 4) {
                 m0 = fmaxf(m0, __uint_as_float(rr[j]));
                 m1 = fmaxf(m1, __uint_as_float(rr[j + 1]));
                 m2 = fmaxf(m2, __uint_as_float(rr[j + 2]));
@@ -636,8 +653,8 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
               }
             } else {
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (col_valid(mc + 32 * cb + j)) m0 = fmaxf(m0, __uint_as_float(rr[j]));
+              for (int j = 0; j < 16; ++j)
+                if (col_valid(mc + 16 * cb + j)) m0 = fmaxf(m0, __uint_as_float(rr[j]));
             }
           }
           mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
@@ -678,13 +695,13 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         // Pass 2: probabilities of this thread's 64 columns.
         float ps0 = 0.f, ps1 = 0.f;
 #pragma unroll 1
-        for (int cb = 0; cb < 2; ++cb) {
-          uint32_t rr[32], pk[16];
-          tmem_ld32(s_addr + mc + 32 * cb, rr);
+        for (int cb = 0; cb < HC / 16; ++cb) {
+          uint32_t rr[16], pk[8];
+          tmem_ld16(s_addr + mc + 16 * cb, rr);
           tmem_ld_wait();
           if (all_valid) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
+            for (int j = 0; j < 8; ++j) {
               float p0 = round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j]), g.scale_log2, -m_use)));
               float p1 = round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j + 1]), g.scale_log2, -m_use)));
               ps0 += p0;  // the normaliser sums exactly what the MMA multiplies
@@ -694,8 +711,8 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
             }
           } else {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int cidx = mc + 32 * cb + 2 * j;
+            for (int j = 0; j < 8; ++j) {
+              const int cidx = mc + 16 * cb + 2 * j;
               float p0 = col_valid(cidx) ? round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j]), g.scale_log2, -m_use))) : 0.f;
               float p1 = col_valid(cidx + 1) ? round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j + 1]), g.scale_log2, -m_use))) : 0.f;
               ps0 += p0;
@@ -704,7 +721,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
               pk[j] = *reinterpret_cast<uint32_t*>(&hp);
             }
           }
-          tmem_st16(tlane + TS_P + 64 * b + 32 * half + 16 * cb, pk);
+          tmem_st8(tlane + TS_P + 64 * b + (HC / 2) * half + 8 * cb, pk);
         }
         const float psum = ps0 + ps1;
         l_part = l_part * alpha + psum;
@@ -859,18 +876,28 @@ __device__ void merge_producer(const Cta& c, const TcMaps& maps, const Geometry&
     const int b = uu & 1, k = uu >> 1;
     if (uu >= 1 && !wait_bar(c, BAR_Q_FREE, (uu - 1) & 1, LOC_WAIT_Q)) return;
     load_q_tile(c, maps, BM, it.row0, h);
-    // cached O~ tile: four boxes of 32 features x 128 rows (rows past nrows are
-    // read but never used)
-    if (uu >= 1 && !wait_bar(c, BAR_IO_FREE, (uu - 1) & 1, LOC_WAIT_V)) return;
-    mbar_expect_tx(c.bar(BAR_IO_FULL), 4 * IO_BOX);
+    if (uu == 0) {
+      // first unit: the cached O~ tile does not depend on the RoPE kernel launched
+      // just before this one, the block's keys and values do: wait for that grid
+      // only now (this kernel may have started early)
+      mbar_expect_tx(c.bar(BAR_IO_FULL), 4 * IO_BOX);
 #pragma unroll
-    for (int cb = 0; cb < 4; ++cb)
-      tma_load_3d(c.base + SM_IO + cb * IO_BOX, &maps.st_o, c.bar(BAR_IO_FULL), 32 * cb, it.row0, h);
-    // the block's keys and values are the only thing here that the RoPE kernel
-    // launched just before this one writes: wait for that grid once
-    if (uu == 0) grid_dependency_wait();
-    if (k >= 1 && !wait_bar(c, BAR_KV_FREE + b, (k - 1) & 1, LOC_WAIT_K)) return;
-    load_kv_tile(maps, c.base + SM_KV + b * KV_STAGE, c.bar(BAR_KV_FULL + b), it.blk_start, h / g.group);
+      for (int cb = 0; cb < 4; ++cb)
+        tma_load_3d(c.base + SM_IO + cb * IO_BOX, &maps.st_o, c.bar(BAR_IO_FULL), 32 * cb, it.row0, h);
+      grid_dependency_wait();
+      load_kv_tile(maps, c.base + SM_KV, c.bar(BAR_KV_FULL), it.blk_start, h / g.group);
+    } else {
+      // later units: keys first (their stage frees early), then the cached O~
+      // tile (four boxes of 32 features x 128 rows; rows past nrows are read but
+      // never used) once the previous unit's output has left the staging tile
+      if (k >= 1 && !wait_bar(c, BAR_KV_FREE + b, (k - 1) & 1, LOC_WAIT_K)) return;
+      load_kv_tile(maps, c.base + SM_KV + b * KV_STAGE, c.bar(BAR_KV_FULL + b), it.blk_start, h / g.group);
+      if (!wait_bar(c, BAR_IO_FREE, (uu - 1) & 1, LOC_WAIT_V)) return;
+      mbar_expect_tx(c.bar(BAR_IO_FULL), 4 * IO_BOX);
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb)
+        tma_load_3d(c.base + SM_IO + cb * IO_BOX, &maps.st_o, c.bar(BAR_IO_FULL), 32 * cb, it.row0, h);
+    }
     it = nxt;
   }
 }
@@ -1220,7 +1247,8 @@ cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* map
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  static const bool no_pdl = getenv("LACACHE_NO_PDL") != nullptr;
+  cfg.numAttrs = no_pdl ? 0 : 1;
   return cudaLaunchKernelEx(&cfg, tc_attn_kernel, *maps, g, a);
 }
 
