@@ -90,7 +90,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -266,12 +266,12 @@ def run_cuda(args):
                 step_pairs.append((e0, e1)); launches += ctx.last_launch_count
 
     # warm-up starts at a block boundary so the cache is built before the first step
+    clocks.start()
     run_range(0, W, False)
     if W % S != 0:   # make the timed region start with a valid cache for its block
         blk = (W // S) % sched.n_blocks_used
         ctx.build(blk, *sched.full[blk])
     torch.cuda.synchronize(); barrier()
-    clocks.start()
     t_wall0 = time.perf_counter()
     # the timed range re-enters mid-block if W % S != 0: builds happen only at s == 0
     run_range(W, W + K, True)
@@ -496,7 +496,9 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": W, "ms_per_step": round(total / K / frac * 1e3, 3), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "cfg%d %s" % (wl.cfg, wl.name)},
+            "config": {"workload": "cfg%d %s" % (wl.cfg, wl.name), "batch": wl.batch, "prompt_lens": list(wl.prompt_lens),
+                       "gen_len": wl.gen_len, "block_len": wl.block_len, "steps_per_block": wl.steps_per_block,
+                       "heads": "%d/%d" % (wl.n_q_heads, wl.n_kv_heads), "head_dim": wl.head_dim},
             "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

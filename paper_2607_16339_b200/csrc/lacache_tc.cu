@@ -454,43 +454,104 @@ __device__ __forceinline__ void load_q_tile(const Cta& c, const TcMaps& maps, in
 // ===========================================================================
 // stream role
 // ===========================================================================
+// The producer walks the (unit, tile) sequence twice, with independent cursors for
+// keys (with the unit's Q tile) and for values, and issues whichever load has a
+// free stage: waiting for a value stage must not hold back the next key tile.
+struct TileCursor {
+  int u, uu, t, jj;   // unit index, ordinal of the unit in this CTA, tile, global tile ordinal
+  WorkItem it;
+  Unit un;
+  bool valid, q_done, loads_q;
+};
+__device__ __forceinline__ void cursor_load_unit(const Geometry& g, const AttnArgs& a, TileCursor& cu, int n_units) {
+  cu.valid = cu.u < n_units;
+  if (!cu.valid) return;
+  cu.it = load_item(a.items + cu.u % a.n_items);
+  cu.un = decode_stream(g, a, cu.it, cu.u);
+  cu.t = next_tile(cu.un, cu.un.t0);
+  cu.q_done = !cu.loads_q;
+}
+__device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs& a, TileCursor& cu, int stride,
+                                               int n_units) {
+  // move to the next tile; cross into the next unit(s) when this one is exhausted
+  if (cu.t < cu.un.t1) {
+    cu.t = next_tile(cu.un, cu.t + 1);
+    ++cu.jj;
+  }
+  while (cu.valid && cu.t >= cu.un.t1 && cu.q_done) {
+    cu.u += stride;
+    ++cu.uu;
+    cursor_load_unit(g, a, cu, n_units);
+  }
+}
+
 __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a,
                                 int first, int stride, int n_units, WorkItem it) {
-  int uu = 0, jj = 0;
   // everything this role loads was written by the RoPE kernel launched just
   // before this one: wait for that grid (this kernel may have started early)
   grid_dependency_wait();
-  for (int u = first; u < n_units; u += stride, ++uu) {
-    WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
-    const Unit un = decode_stream(g, a, it, u);
-    if (uu >= 1 && !wait_bar(c, BAR_Q_FREE, (uu - 1) & 1, LOC_WAIT_Q)) return;
-    load_q_tile(c, maps, un.q_rows, un.row0, un.h);
-    for (int t = next_tile(un, un.t0); t < un.t1; t = next_tile(un, t + 1), ++jj) {
-      const int krow = un.key_base + t * BN;
-      // keys: a stage is free as soon as the scores that read it have been computed
-      {
-        const int sk = jj & 1, kuse = jj >> 1;
-        if (kuse >= 1 && !wait_bar(c, sk ? BAR_K_FREE1 : BAR_K_FREE, (kuse - 1) & 1, LOC_WAIT_K)) return;
-        const uint32_t bar = c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL);
-        const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
-        mbar_expect_tx(bar, 4 * KS_BOX);
-        tma_load_3d(khi, &maps.k_hi, bar, 0, krow, un.kh);
-        tma_load_3d(khi + KS_BOX, &maps.k_hi, bar, 64, krow, un.kh);
-        tma_load_3d(klo, &maps.k_lo, bar, 0, krow, un.kh);
-        tma_load_3d(klo + KS_BOX, &maps.k_lo, bar, 64, krow, un.kh);
-      }
-      // values: a stage is free once the P~V that read it has been computed
-      {
-        const int sv = jj & 1, vuse = jj >> 1;
-        if (vuse >= 1 && !wait_bar(c, sv ? BAR_V_FREE1 : BAR_V_FREE, (vuse - 1) & 1, LOC_WAIT_V)) return;
-        const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
-        mbar_expect_tx(bar, 2 * KS_BOX);
-        tma_load_3d(vb, &maps.v, bar, 0, krow, un.kh);
-        tma_load_3d(vb + KS_BOX, &maps.v, bar, 64, krow, un.kh);
+  TileCursor ck, cv;
+  ck.u = first; ck.uu = 0; ck.jj = 0; ck.loads_q = true;
+  cursor_load_unit(g, a, ck, n_units);
+  cv = ck;
+  cv.loads_q = false;  // the value cursor never loads Q
+  cv.q_done = true;
+  if (cv.valid && cv.t >= cv.un.t1) cursor_advance(g, a, cv, stride, n_units);
+  // a unit without key tiles still needs its Q load (the MMA thread waits for it)
+  long long t_idle = 0;
+  while (ck.valid || cv.valid) {
+    bool did = false;
+    if (ck.valid) {
+      if (!ck.q_done) {
+        if (ck.uu == 0 || mbar_test(c.bar(BAR_Q_FREE), (ck.uu - 1) & 1)) {
+          load_q_tile(c, maps, ck.un.q_rows, ck.un.row0, ck.un.h);
+          ck.q_done = true;
+          if (ck.t >= ck.un.t1) cursor_advance(g, a, ck, stride, n_units);  // no key tiles at all
+          did = true;
+        }
+      } else if (ck.t < ck.un.t1) {
+        const int sk = ck.jj & 1, kuse = ck.jj >> 1;
+        if (kuse == 0 || mbar_test(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE), (kuse - 1) & 1)) {
+          const int krow = ck.un.key_base + ck.t * BN;
+          const uint32_t bar = c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL);
+          const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
+          mbar_expect_tx(bar, 4 * KS_BOX);
+          tma_load_3d(khi, &maps.k_hi, bar, 0, krow, ck.un.kh);
+          tma_load_3d(khi + KS_BOX, &maps.k_hi, bar, 64, krow, ck.un.kh);
+          tma_load_3d(klo, &maps.k_lo, bar, 0, krow, ck.un.kh);
+          tma_load_3d(klo + KS_BOX, &maps.k_lo, bar, 64, krow, ck.un.kh);
+          cursor_advance(g, a, ck, stride, n_units);
+          did = true;
+        }
       }
     }
-    it = nxt;
+    if (cv.valid) {
+      if (cv.t < cv.un.t1) {
+        const int sv = cv.jj & 1, vuse = cv.jj >> 1;
+        if (vuse == 0 || mbar_test(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE), (vuse - 1) & 1)) {
+          const int krow = cv.un.key_base + cv.t * BN;
+          const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
+          mbar_expect_tx(bar, 2 * KS_BOX);
+          tma_load_3d(vb, &maps.v, bar, 0, krow, cv.un.kh);
+          tma_load_3d(vb + KS_BOX, &maps.v, bar, 64, krow, cv.un.kh);
+          cursor_advance(g, a, cv, stride, n_units);
+          did = true;
+        }
+      }
+    }
+    if (did) {
+      t_idle = 0;
+    } else {  // nothing free: bounded idle
+      if (t_idle == 0) t_idle = clock64();
+      if (*c.abort_flag) return;
+      if (clock64() - t_idle > WAIT_CYCLES) {
+        *c.abort_flag = 1;
+        if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
+          c.status[1] = LOC_WAIT_K; c.status[2] = blockIdx.x; c.status[3] = threadIdx.x;
+        }
+        return;
+      }
+    }
   }
 }
 
@@ -590,6 +651,88 @@ __device__ __forceinline__ void coop_store_rows(const Cta& c, uint32_t stage_off
     const int rr = i >> 5, ch = i & 31;
     float4 v = *reinterpret_cast<const float4*>(c.gen + stage_off + rr * STAGE_ROW + ((ch ^ (rr & 7)) << 4));
     *reinterpret_cast<float4*>(gbase + (size_t)rr * stride + ch * 4) = v;
+  }
+}
+
+// Merge of the partial states of all key chunks of one (sequence, head) by the
+// last chunk to arrive: thread t owns 16 bytes of one row; the partial rows are
+// read with coalesced loads straight from L2 and the normalised rows written out.
+__device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs& a, size_t pbase, int nchunks,
+                                               int block_len, int row0, int h) {
+  const float LN2 = 0.69314718055994530942f;
+  const int t = threadIdx.x - 64;
+  if (nchunks <= 4) {
+    // few chunks: every load of a row (references, normalisers, 16 bytes of each
+    // partial O~) is issued before any is used -- one L2 round trip in all
+    for (int i = t; i < block_len * 32; i += ROW_THREADS) {
+      const int rr = i >> 5, ch = i & 31;
+      float mv[4], lv[4];
+      float4 v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const size_t pr = (pbase + min(k, nchunks - 1)) * block_len + rr;
+        mv[k] = __ldcg(a.part_m + pr);
+        lv[k] = __ldcg(a.part_l + pr);
+        v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + pr * D) + ch);
+      }
+      float M = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (k < nchunks) M = fmaxf(M, mv[k]);
+      float L = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float w = (k < nchunks && mv[k] != -INFINITY) ? ex2(mv[k] - M) : 0.f;
+        L = fmaf(lv[k], w, L);
+        acc.x = fmaf(v[k].x, w, acc.x);
+        acc.y = fmaf(v[k].y, w, acc.y);
+        acc.z = fmaf(v[k].z, w, acc.z);
+        acc.w = fmaf(v[k].w, w, acc.w);
+      }
+      const float inv = 1.f / L;
+      const size_t orow = (size_t)(row0 + rr) * g.Hq + h;
+      *reinterpret_cast<float4*>(a.out + orow * D + ch * 4) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+      if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
+    }
+    return;
+  }
+  for (int i = t; i < block_len * 32; i += ROW_THREADS) {
+    const int rr = i >> 5, ch = i & 31;
+    float M = -INFINITY;
+    {
+      float mv[16];  // at most 16 chunks: all loads in flight together
+#pragma unroll
+      for (int cc = 0; cc < 16; ++cc) mv[cc] = __ldcg(a.part_m + (pbase + min(cc, nchunks - 1)) * block_len + rr);
+#pragma unroll
+      for (int cc = 0; cc < 16; ++cc) M = fmaxf(M, mv[cc]);
+    }
+    float L = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c0 = 0; c0 < nchunks; c0 += 4) {
+      float w[4];
+      float4 v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int cc = min(c0 + k, nchunks - 1);
+        const size_t pr = (pbase + cc) * block_len + rr;
+        const float mcv = __ldcg(a.part_m + pr);
+        w[k] = (c0 + k < nchunks && mcv != -INFINITY) ? ex2(mcv - M) : 0.f;
+        L = fmaf(__ldcg(a.part_l + pr), w[k], L);
+        v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + pr * D) + ch);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        acc.x = fmaf(v[k].x, w[k], acc.x);
+        acc.y = fmaf(v[k].y, w[k], acc.y);
+        acc.z = fmaf(v[k].z, w[k], acc.z);
+        acc.w = fmaf(v[k].w, w[k], acc.w);
+      }
+    }
+    const float inv = 1.f / L;
+    const size_t orow = (size_t)(row0 + rr) * g.Hq + h;
+    *reinterpret_cast<float4*>(a.out + orow * D + ch * 4) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+    if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
   }
 }
 
@@ -814,48 +957,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       }
       if (!epi_sync(c, epi_phase)) return;
       if (*c.flag != 0) {
-        // merge: thread t owns 16 bytes of one row; all partial rows are read
-        // with coalesced loads straight from L2
-        const int t = threadIdx.x - 64;
-        for (int i = t; i < un.nrows * 32; i += ROW_THREADS) {
-          const int rr = i >> 5, ch = i & 31;
-          float M = -INFINITY;
-          {
-            float mv[16];  // at most 16 chunks: all loads in flight together
-#pragma unroll
-            for (int cc = 0; cc < 16; ++cc)
-              mv[cc] = __ldcg(a.part_m + (pbase + min(cc, un.nchunks - 1)) * g.block_len + rr);
-#pragma unroll
-            for (int cc = 0; cc < 16; ++cc) M = fmaxf(M, mv[cc]);
-          }
-          float L = 0.f;
-          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-          for (int c0 = 0; c0 < un.nchunks; c0 += 4) {
-            float w[4];
-            float4 v[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const int cc = min(c0 + k, un.nchunks - 1);
-              const size_t pr = (pbase + cc) * g.block_len + rr;
-              const float mcv = __ldcg(a.part_m + pr);
-              w[k] = (c0 + k < un.nchunks && mcv != -INFINITY) ? ex2(mcv - M) : 0.f;
-              L = fmaf(__ldcg(a.part_l + pr), w[k], L);
-              v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + pr * D) + ch);
-            }
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              acc.x = fmaf(v[k].x, w[k], acc.x);
-              acc.y = fmaf(v[k].y, w[k], acc.y);
-              acc.z = fmaf(v[k].z, w[k], acc.z);
-              acc.w = fmaf(v[k].w, w[k], acc.w);
-            }
-          }
-          const float inv = 1.f / L;
-          const size_t orow = (size_t)(un.row0 + rr) * g.Hq + un.h;
-          *reinterpret_cast<float4*>(a.out + orow * D + ch * 4) =
-              make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-          if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
-        }
+        merge_partials(g, a, pbase, un.nchunks, g.block_len, un.row0, un.h);
       }
     }
     if (!epi_sync(c, epi_phase)) return;  // the staging rows have been read
