@@ -393,6 +393,11 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       ns = (int)std::min<long long>(ns, units_stream);
       a.n_ctas_stream = ns;
       a.n_ctas = ns + (int)std::min<long long>(units_merge, std::max(0, c->num_sms - ns));
+      {
+        const int n_merge_ctas = a.n_ctas - ns;
+        const long long per_cta = n_merge_ctas > 0 ? (units_merge + n_merge_ctas - 1) / n_merge_ctas : 0;
+        a.merge_deep = (c->g.block_len <= 32 && per_cta <= TC_DEEP_MAX_UNITS && !getenv("LACACHE_NO_DEEP")) ? 1 : 0;
+      }
     } else {
       a.n_ctas_stream = (int)std::min<long long>(c->num_sms, units_stream);
       a.n_ctas = a.n_ctas_stream;

@@ -85,6 +85,7 @@ struct AttnArgs {
   // tcgen05 only: items of the merge role (fixed rows of a step), CTA split
   const WorkItem* items_merge; int n_items_merge;
   int n_ctas_stream; int n_ctas;
+  int merge_deep;            // merge role runs its pipelined variant (block_len <= 32, bounded units per CTA)
   const int32_t* cu;         // [B+1]
   const int32_t* blk_start;  // [B] absolute token index of the block's first row
   RotBuffers rot;
@@ -124,6 +125,7 @@ void tc_free_maps(TcMaps* m);
 constexpr int SIMT_ROWS = 32;    // query rows per SIMT work item
 constexpr int TC_ROWS = 128;     // query rows per tcgen05 work item
 constexpr int TC_KEYS = 96;      // keys per tcgen05 key tile (stream role)
-constexpr int TC_MAX_BLOCK = 64; // largest block length the tcgen05 merge role handles
+constexpr int TC_MAX_BLOCK = 64;
+constexpr int TC_DEEP_MAX_UNITS = 512;  // units per CTA the pipelined merge role can tabulate // largest block length the tcgen05 merge role handles
 
 }  // namespace lacache

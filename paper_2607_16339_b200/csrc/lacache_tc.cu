@@ -51,6 +51,9 @@ struct TcMaps {
   alignas(64) CUtensorMap k64_hi;  // box 64 rows (the block's keys, merge role)
   alignas(64) CUtensorMap k64_lo;
   alignas(64) CUtensorMap v64;
+  alignas(64) CUtensorMap k32_hi;  // box 32 rows (the block's keys, pipelined merge role)
+  alignas(64) CUtensorMap k32_lo;
+  alignas(64) CUtensorMap v32;
   alignas(64) CUtensorMap st_o;    // cached O~ [Hq][Tp][128] fp32, box 32 cols x 128 rows
   alignas(64) CUtensorMap out;     // caller's out [T][Hq][128] fp32, box 32 cols x 1 head x 128 rows
   const void* out_ptr;             // the buffer `out` was encoded for
@@ -120,6 +123,7 @@ enum {
   BAR_O_FULL, BAR_O_FULL1, BAR_O_FREE, BAR_O_FREE1,
   BAR_IO_FULL, BAR_IO_FREE, BAR_EPI, BAR_DONE,
   BAR_K_FULL1, BAR_K_FREE1, BAR_V_FULL1, BAR_V_FREE1,  // stream role, second key / value stage
+  BAR_IO_FULL1, BAR_OUT_RDY, BAR_OUT_RDY1,  // pipelined merge role: second staging tile; output tile b is complete
   BAR_PAIR,  // 4 barriers: the two warps that share a TMEM lane quadrant
   N_BARS = BAR_PAIR + 4
 };
@@ -182,6 +186,9 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 __device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes)
                : "memory");
+}
+__device__ __forceinline__ void prefetch_map(const CUtensorMap* m) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(m) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
@@ -487,9 +494,6 @@ __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs
 
 __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a,
                                 int first, int stride, int n_units, WorkItem it) {
-  // everything this role loads was written by the RoPE kernel launched just
-  // before this one: wait for that grid (this kernel may have started early)
-  grid_dependency_wait();
   TileCursor ck, cv;
   ck.u = first; ck.uu = 0; ck.jj = 0; ck.loads_q = true;
   cursor_load_unit(g, a, ck, n_units);
@@ -497,6 +501,9 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
   cv.loads_q = false;  // the value cursor never loads Q
   cv.q_done = true;
   if (cv.valid && cv.t >= cv.un.t1) cursor_advance(g, a, cv, stride, n_units);
+  // everything this role loads was written by the RoPE kernel launched just
+  // before this one: wait for that grid (this kernel may have started early)
+  grid_dependency_wait();
   // a unit without key tiles still needs its Q load (the MMA thread waits for it)
   long long t_idle = 0;
   while (ck.valid || cv.valid) {
@@ -1164,6 +1171,255 @@ __device__ void merge_rows(const Cta& c, const TcMaps& maps, const Geometry& g, 
 }
 
 // ===========================================================================
+// ===========================================================================
+// merge role, pipelined variant for block_len <= 32.  The block's keys and
+// values need only 24 KB, which leaves room for two staging tiles of cached
+// O~: the tile of unit u + 1 streams in while unit u is combined and while the
+// output of unit u - 1 streams out, so a CTA keeps ~190 KB of loads and stores
+// in flight instead of one tile at a time.  Keys and values have separate
+// barriers (single stage each: the next unit's keys load as soon as the
+// current scores are done).  The producer thread also issues the output
+// stores, and every role reads the CTA's units from a table in shared memory.
+// ===========================================================================
+constexpr uint32_t DM_IO = 65536;                      // two staging tiles of 4 boxes (64 KB each)
+constexpr uint32_t DM_IO_TILE = 4 * IO_BOX;
+constexpr uint32_t DM_KBOX = 32 * 128;                 // one [32 rows][64 cols] 16-bit box
+constexpr uint32_t DM_K = DM_IO + 2 * DM_IO_TILE;      // K hi (2 boxes), K lo (2 boxes)
+constexpr uint32_t DM_V = DM_K + 4 * DM_KBOX;          // V (2 boxes)
+constexpr uint32_t DM_TAB = DM_V + 2 * DM_KBOX;        // unit table: {row0, nrows, blk_start, head}
+constexpr int DM_MAX_UNITS = (int)((SM_XCH - DM_TAB) / 16);
+static_assert(DM_TAB % 16 == 0 && DM_MAX_UNITS >= TC_DEEP_MAX_UNITS, "unit table");
+
+struct DUnit { int row0, nrows, blk_start, h; };
+__device__ __forceinline__ DUnit deep_unit(const Cta& c, int i) {
+  const int4 v = *reinterpret_cast<const int4*>(c.gen + DM_TAB + 16 * i);
+  return DUnit{v.x, v.y, v.z, v.w};
+}
+
+__device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& g, int n_my) {
+  if (n_my == 0) return;
+  auto load_q = [&](int i) {
+    const DUnit un = deep_unit(c, i);
+    load_q_tile(c, maps, BM, un.row0, un.h);
+  };
+  auto load_io = [&](int i) {
+    const DUnit un = deep_unit(c, i);
+    const uint32_t bar = c.bar((i & 1) ? BAR_IO_FULL1 : BAR_IO_FULL);
+    const uint32_t dst = c.base + DM_IO + (i & 1) * DM_IO_TILE;
+    mbar_expect_tx(bar, DM_IO_TILE);
+#pragma unroll
+    for (int cb = 0; cb < 4; ++cb) tma_load_3d(dst + cb * IO_BOX, &maps.st_o, bar, 32 * cb, un.row0, un.h);
+  };
+  auto load_k = [&](int i) {
+    const DUnit un = deep_unit(c, i);
+    const uint32_t bar = c.bar(BAR_KV_FULL), kb = c.base + DM_K;
+    const int kh = un.h / g.group;
+    mbar_expect_tx(bar, 4 * DM_KBOX);
+    tma_load_3d(kb, &maps.k32_hi, bar, 0, un.blk_start, kh);
+    tma_load_3d(kb + DM_KBOX, &maps.k32_hi, bar, 64, un.blk_start, kh);
+    tma_load_3d(kb + 2 * DM_KBOX, &maps.k32_lo, bar, 0, un.blk_start, kh);
+    tma_load_3d(kb + 3 * DM_KBOX, &maps.k32_lo, bar, 64, un.blk_start, kh);
+  };
+  auto load_v = [&](int i) {
+    const DUnit un = deep_unit(c, i);
+    const uint32_t bar = c.bar(BAR_KV_FULL1), vb = c.base + DM_V;
+    const int kh = un.h / g.group;
+    mbar_expect_tx(bar, 2 * DM_KBOX);
+    tma_load_3d(vb, &maps.v32, bar, 0, un.blk_start, kh);
+    tma_load_3d(vb + DM_KBOX, &maps.v32, bar, 64, un.blk_start, kh);
+  };
+  // Q' and cached O~ of fixed rows do not depend on the RoPE kernel launched
+  // just before this one; the block's keys and values do
+  load_q(0);
+  load_io(0);
+  if (n_my > 1) load_io(1);
+  grid_dependency_wait();
+  load_k(0);
+  load_v(0);
+  int qu = 1, ku = 1, vu = 1, iu = 2, su = 0;
+  bool pending_read = false;  // an output store may still be reading its staging tile
+  long long t_idle = 0;
+  while (su < n_my) {
+    bool did = false;
+    if (qu < n_my && mbar_test(c.bar(BAR_Q_FREE), (qu - 1) & 1)) { load_q(qu); ++qu; did = true; }
+    if (ku < n_my && mbar_test(c.bar(BAR_KV_FREE), (ku - 1) & 1)) { load_k(ku); ++ku; did = true; }
+    if (vu < n_my && mbar_test(c.bar(BAR_KV_FREE1), (vu - 1) & 1)) { load_v(vu); ++vu; did = true; }
+    if (mbar_test(c.bar((su & 1) ? BAR_OUT_RDY1 : BAR_OUT_RDY), (su >> 1) & 1)) {
+      const DUnit un = deep_unit(c, su);
+      if (un.nrows == BM) {  // clipped tiles were written row by row by the row threads
+        const uint32_t src = c.base + DM_IO + (su & 1) * DM_IO_TILE;
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) tma_store_3d(&maps.out, src + cb * IO_BOX, 32 * cb, un.h, un.row0);
+        bulk_commit();
+        pending_read = true;
+      }
+      ++su;
+      did = true;
+    }
+    if (!did && iu < n_my && su > iu - 2) {  // the tile of unit iu - 2 has been handed to its store
+      if (pending_read) { bulk_wait_read(); pending_read = false; }
+      load_io(iu);
+      ++iu;
+      did = true;
+    }
+    if (did) {
+      t_idle = 0;
+    } else {
+      if (t_idle == 0) t_idle = clock64();
+      if (*c.abort_flag) break;
+      if (clock64() - t_idle > WAIT_CYCLES) {
+        *c.abort_flag = 1;
+        if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
+          c.status[1] = LOC_WAIT_V; c.status[2] = blockIdx.x; c.status[3] = threadIdx.x;
+        }
+        break;
+      }
+    }
+  }
+  bulk_wait_read();  // shared memory stays valid until the last store has read it
+}
+
+__device__ void deep_mma(const Cta& c, const Geometry& g, int n_my) {
+  if (n_my == 0) return;
+  const int n_s = (g.block_len + 15) & ~15;
+  const uint32_t idesc_s = idesc_f16(1u, 0u, BM, (uint32_t)n_s);
+  const uint32_t kb = c.base + DM_K;
+  if (!wait_bar(c, BAR_Q_FULL, 0, LOC_WAIT_Q)) return;
+  if (!wait_bar(c, BAR_KV_FULL, 0, LOC_WAIT_K)) return;
+  tc_fence_after();
+  issue_s_mma(c.base + SM_Q, BM * 128u, kb, kb + 2 * DM_KBOX, DM_KBOX, c.tmem + TM_S, idesc_s);
+  tc_commit(c.bar(BAR_S_FULL));
+  tc_commit(c.bar(BAR_Q_FREE));
+  tc_commit(c.bar(BAR_KV_FREE));
+  for (int uu = 0; uu < n_my; ++uu) {
+    const int b = uu & 1, k = uu >> 1;
+    if (!wait_bar(c, BAR_P_FULL + b, k & 1, LOC_WAIT_S)) return;
+    if (k >= 1 && !wait_bar(c, BAR_O_FREE + b, (k - 1) & 1, LOC_WAIT_O)) return;
+    if (!wait_bar(c, BAR_KV_FULL1, uu & 1, LOC_WAIT_V)) return;
+    tc_fence_after();
+    issue_pv_mma(c.base + DM_V, DM_KBOX, c.tmem + TM_P + 32 * b, c.tmem + TM_O + 128 * b, n_s / 16, 0u);
+    tc_commit(c.bar(BAR_O_FULL + b));
+    tc_commit(c.bar(BAR_KV_FREE1));
+    if (uu + 1 < n_my) {  // scores of the next unit as soon as its tiles land
+      const int bn = (uu + 1) & 1;
+      if (!wait_bar(c, BAR_Q_FULL, (uu + 1) & 1, LOC_WAIT_Q)) return;
+      if (!wait_bar(c, BAR_KV_FULL, (uu + 1) & 1, LOC_WAIT_K)) return;
+      tc_fence_after();
+      issue_s_mma(c.base + SM_Q, BM * 128u, kb, kb + 2 * DM_KBOX, DM_KBOX, c.tmem + TM_S + 64 * bn, idesc_s);
+      tc_commit(c.bar(BAR_S_FULL + bn));
+      tc_commit(c.bar(BAR_Q_FREE));
+      tc_commit(c.bar(BAR_KV_FREE));
+    }
+  }
+}
+
+__device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, int n_my) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int quad = warp & 3;
+  const int half = (warp - 2) >> 2;
+  const int r = quad * 32 + lane;
+  const uint32_t tlane = c.tmem + ((uint32_t)(quad * 32) << 16);
+  const float LN2 = 0.69314718055994530942f;
+  const int L = g.block_len;
+  const int sw = r & 7;
+  // the cached (m, l) of a unit's rows are fetched one unit ahead
+  float m_nx = -INFINITY, l_nx = 0.f;
+  if (n_my > 0) {
+    const DUnit un = deep_unit(c, 0);
+    if (r < un.nrows) {
+      const size_t srow = (size_t)un.h * g.Tp + un.row0 + r;
+      m_nx = __ldg(a.st.m + srow);
+      l_nx = __ldg(a.st.l + srow);
+    }
+  }
+  for (int uu = 0; uu < n_my; ++uu) {
+    const DUnit un = deep_unit(c, uu);
+    const int b = uu & 1, par = (uu >> 1) & 1;
+    const int row = un.row0 + r;
+    const bool row_valid = r < un.nrows;
+    const float m_c = m_nx, l_c = l_nx;
+    m_nx = -INFINITY; l_nx = 0.f;
+    if (uu + 1 < n_my) {
+      const DUnit nx = deep_unit(c, uu + 1);
+      if (r < nx.nrows) {
+        const size_t srow = (size_t)nx.h * g.Tp + nx.row0 + r;
+        m_nx = __ldg(a.st.m + srow);
+        l_nx = __ldg(a.st.l + srow);
+      }
+    }
+    // staging tile b (as TMA writes and reads it): box cb = features [32 cb, 32 cb + 32),
+    // row r at +128 r, its 16-byte chunk j at ((j ^ (r & 7)) << 4)
+    uint8_t* const sbox = c.gen + DM_IO + b * DM_IO_TILE + (2 * half) * IO_BOX + r * 128;
+
+    if (!wait_bar(c, BAR_S_FULL + b, par, LOC_WAIT_S)) return;
+    tc_fence_after();
+    float mx = -INFINITY;
+    uint32_t s0[32];
+    tmem_ld32(tlane + TM_S + 64 * b, s0);
+    tmem_ld_wait();
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j < L) mx = fmaxf(mx, __uint_as_float(s0[j]));
+    const float m_new = fmaxf(m_c, ceilf(mx * g.scale_log2));
+    const float alpha = (m_c == -INFINITY) ? 0.f : ex2(m_c - m_new);
+    float psum = 0.f;
+    {
+      uint32_t pk[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        float p0 = (2 * j < L) ? round_to_half_bits(ex2(fmaf(__uint_as_float(s0[2 * j]), g.scale_log2, -m_new))) : 0.f;
+        float p1 = (2 * j + 1 < L) ? round_to_half_bits(ex2(fmaf(__uint_as_float(s0[2 * j + 1]), g.scale_log2, -m_new))) : 0.f;
+        psum += p0 + p1;
+        __half2 hp = __floats2half2_rn(p0, p1);
+        pk[j] = *reinterpret_cast<uint32_t*>(&hp);
+      }
+      if (half == 0) tmem_st16(tlane + TM_P + 32 * b, pk);
+    }
+    tmem_st_wait();
+    tc_fence_before();
+    mbar_arrive(c.bar(BAR_P_FULL + b));
+    const float l_new = fmaf(l_c, alpha, psum);
+    const float inv = 1.f / l_new;
+    const float a_inv = alpha * inv;
+
+    if (!wait_bar(c, BAR_O_FULL + b, par, LOC_WAIT_O)) return;
+    if (!wait_bar(c, b ? BAR_IO_FULL1 : BAR_IO_FULL, par, LOC_WAIT_V)) return;
+    tc_fence_after();
+    // out = (alpha O~_cache + P~V) / l, in place in the staging tile
+#pragma unroll
+    for (int q2 = 0; q2 < 2; ++q2) {
+      uint32_t rr[32];
+      tmem_ld32(tlane + TM_O + 128 * b + 64 * half + 32 * q2, rr);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float4* p4 = reinterpret_cast<float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
+        float4 oc = *p4;
+        oc.x = fmaf(oc.x, a_inv, __uint_as_float(rr[4 * i]) * inv);
+        oc.y = fmaf(oc.y, a_inv, __uint_as_float(rr[4 * i + 1]) * inv);
+        oc.z = fmaf(oc.z, a_inv, __uint_as_float(rr[4 * i + 2]) * inv);
+        oc.w = fmaf(oc.w, a_inv, __uint_as_float(rr[4 * i + 3]) * inv);
+        *p4 = oc;
+      }
+    }
+    tc_fence_before();
+    mbar_arrive(c.bar(BAR_O_FREE + b));
+    const size_t orow = (size_t)row * g.Hq + un.h;
+    if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_new + log2f(l_new)) * LN2;
+    if (un.nrows != BM && row_valid) {
+      // a tile clipped by the block or the sequence end: rows go out one by one
+      float4* dst = reinterpret_cast<float4*>(a.out + orow * D + 64 * half);
+#pragma unroll
+      for (int q2 = 0; q2 < 2; ++q2)
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          dst[8 * q2 + i] = *reinterpret_cast<const float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
+    }
+    fence_async_smem();  // the producer thread's bulk store reads this tile
+    mbar_arrive(c.bar(b ? BAR_OUT_RDY1 : BAR_OUT_RDY));
+  }
+}
+
 __global__ void __launch_bounds__(THREADS, 1)
 tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const AttnArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -1178,16 +1434,32 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   c.status = a.status;
   // role and unit range of this CTA; the first work item is fetched before the
   // set-up below so its latency overlaps it
-  const bool stream = (int)blockIdx.x < a.n_ctas_stream;
+  // merge-role CTAs take the low block indices: they are scheduled first and have
+  // loads to issue that do not depend on the preceding RoPE kernel
+  const int n_ctas_merge = (int)gridDim.x - a.n_ctas_stream;
+  const bool stream = (int)blockIdx.x >= n_ctas_merge;
   int first, stride, n_units;
   if (stream) {
-    first = blockIdx.x; stride = a.n_ctas_stream; n_units = a.n_items * g.Hq;
+    first = blockIdx.x - n_ctas_merge; stride = a.n_ctas_stream; n_units = a.n_items * g.Hq;
   } else {
-    first = blockIdx.x - a.n_ctas_stream; stride = gridDim.x - a.n_ctas_stream; n_units = a.n_items_merge * g.Hq;
+    first = blockIdx.x; stride = n_ctas_merge; n_units = a.n_items_merge * g.Hq;
   }
+  const bool deep = !stream && a.merge_deep != 0;
+  if (tid == 0) {  // descriptor fetches overlap the set-up below
+    if (stream) {
+      prefetch_map(a.mode == MODE_STEP ? &maps.q64_hi : &maps.q_hi);
+      prefetch_map(a.mode == MODE_STEP ? &maps.q64_lo : &maps.q_lo);
+      prefetch_map(&maps.k_hi); prefetch_map(&maps.k_lo); prefetch_map(&maps.v);
+    } else {
+      prefetch_map(&maps.q_hi); prefetch_map(&maps.q_lo); prefetch_map(&maps.st_o); prefetch_map(&maps.out);
+      if (deep) { prefetch_map(&maps.k32_hi); prefetch_map(&maps.k32_lo); prefetch_map(&maps.v32); }
+      else { prefetch_map(&maps.k64_hi); prefetch_map(&maps.k64_lo); prefetch_map(&maps.v64); }
+    }
+  }
+  const int n_my = first < n_units ? (n_units - first + stride - 1) / stride : 0;
   WorkItem it0{};
-  if (first < n_units) it0 = stream ? load_item(a.items + first % a.n_items)
-                                    : load_item(a.items_merge + first % a.n_items_merge);
+  if (!deep && first < n_units) it0 = stream ? load_item(a.items + first % a.n_items)
+                                             : load_item(a.items_merge + first % a.n_items_merge);
   if ((c.base & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = LOC_SMEM_ALIGN;
     return;
@@ -1195,7 +1467,8 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   if (tid == 0) {
     for (int i = 0; i < N_BARS; ++i) {
       uint32_t count = 1;
-      if (i == BAR_P_FULL || i == BAR_P_FULL1 || i == BAR_O_FREE || i == BAR_O_FREE1 || i == BAR_EPI)
+      if (i == BAR_P_FULL || i == BAR_P_FULL1 || i == BAR_O_FREE || i == BAR_O_FREE1 || i == BAR_EPI ||
+          i == BAR_OUT_RDY || i == BAR_OUT_RDY1)
         count = ROW_THREADS;
       if (i == BAR_DONE) count = THREADS;
       if (i == BAR_Q_FREE && stream) count = 2;  // score MMAs done + epilogue staging read
@@ -1206,6 +1479,14 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     words[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
+  }
+  if (deep) {
+    // this CTA's units, read by every role from shared memory
+    for (int i = tid; i < n_my; i += THREADS) {
+      const int u = first + i * stride;
+      const WorkItem w = load_item(a.items_merge + u % a.n_items_merge);
+      *reinterpret_cast<int4*>(smem_raw + DM_TAB + 16 * i) = make_int4(w.row0, w.nrows, w.blk_start, u / a.n_items_merge);
+    }
   }
   __syncwarp();
   if (warp == 0) {
@@ -1222,16 +1503,20 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   if (warp == 0) {
     if (stream) {
       if (tid == 0) stream_producer(c, maps, g, a, first, stride, n_units, it0);
+    } else if (deep) {
+      if (tid == 0) deep_producer(c, maps, g, n_my);
     } else {
       if (tid == 0) merge_producer(c, maps, g, a, first, stride, n_units, it0);
     }
   } else if (warp == 1) {
     if (tid == 32) {
       if (stream) stream_mma(c, g, a, first, stride, n_units, it0);
+      else if (deep) deep_mma(c, g, n_my);
       else merge_mma(c, g, a, first, stride, n_units);
     }
   } else {
     if (stream) stream_rows(c, g, a, first, stride, n_units, it0);
+    else if (deep) deep_rows(c, g, a, n_my);
     else merge_rows(c, maps, g, a, first, stride, n_units, it0);
     bulk_wait_read();
   }
@@ -1329,6 +1614,9 @@ TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, c
             make_plane_map(&m->k64_hi, rot.k_hi, g.Hkv, g.Tp, 64, false, err, errlen) &&
             make_plane_map(&m->k64_lo, rot.k_lo, g.Hkv, g.Tp, 64, false, err, errlen) &&
             make_plane_map(&m->v64, rot.v, g.Hkv, g.Tp, 64, true, err, errlen) &&
+            make_plane_map(&m->k32_hi, rot.k_hi, g.Hkv, g.Tp, 32, false, err, errlen) &&
+            make_plane_map(&m->k32_lo, rot.k_lo, g.Hkv, g.Tp, 32, false, err, errlen) &&
+            make_plane_map(&m->v32, rot.v, g.Hkv, g.Tp, 32, true, err, errlen) &&
             make_f32_map(&m->st_o, state_o, (cuuint64_t)g.Tp, (cuuint64_t)g.Hq, BM, 1, err, errlen);
   if (!ok) { delete m; return nullptr; }
   return m;
