@@ -38,6 +38,10 @@ struct lacache_ctx {
   int32_t* d_pos = nullptr;
   float* d_cos = nullptr;
   float* d_sin = nullptr;
+  // per block: destination token and cos/sin rows of the block's B * block_len rows
+  int32_t* d_blk_tok = nullptr;
+  float* d_blk_cos = nullptr;
+  float* d_blk_sin = nullptr;
   WorkItem* d_items = nullptr;
   RotBuffers rot{}, rot_scratch{};
   StateBuffers st{};
@@ -119,13 +123,13 @@ lacache_status alloc_rot(lacache_ctx* c, RotBuffers* r) {
   const Geometry& g = c->g;
   size_t nq = (size_t)g.Hq * g.Tp * g.d, nk = (size_t)g.Hkv * g.Tp * g.d;
   if (c->engine == LACACHE_ENGINE_TCGEN05) {
-    uint16_t *a, *b, *cc, *d, *e;
-    CU_TRY(c, dev_alloc(c, &a, nq, true));
-    CU_TRY(c, dev_alloc(c, &b, nq, true));
-    CU_TRY(c, dev_alloc(c, &cc, nk, true));
-    CU_TRY(c, dev_alloc(c, &d, nk, true));
+    // hi and lo planes of a tensor share one allocation (the lo plane starts
+    // right after the hi plane): the tensor maps address them as one 5-D tensor
+    uint16_t *a, *cc, *e;
+    CU_TRY(c, dev_alloc(c, &a, 2 * nq, true));
+    CU_TRY(c, dev_alloc(c, &cc, 2 * nk, true));
     CU_TRY(c, dev_alloc(c, &e, nk, true));
-    *r = RotBuffers{a, b, cc, d, e};
+    *r = RotBuffers{a, a + nq, cc, cc + nk, e};
   } else {
     float *a, *b, *cc;
     CU_TRY(c, dev_alloc(c, &a, nq, true));
@@ -315,6 +319,26 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     CU_TRY(c, dev_alloc(c, &c->d_sin, sn.size()));
     CU_TRY(c, cudaMemcpy(c->d_cos, cs.data(), sizeof(float) * cs.size(), cudaMemcpyHostToDevice));
     CU_TRY(c, cudaMemcpy(c->d_sin, sn.data(), sizeof(float) * sn.size(), cudaMemcpyHostToDevice));
+    // the same rows gathered per block row (row r of block k: sequence r / block_len,
+    // offset r % block_len), so the step's RoPE kernel needs no dependent look-ups
+    const size_t rows = (size_t)g.n_blk * g.B * g.block_len;
+    std::vector<int32_t> btok(rows);
+    std::vector<float> bcs(rows * half), bsn(rows * half);
+    for (int k = 0; k < g.n_blk; ++k)
+      for (int r = 0; r < g.B * g.block_len; ++r) {
+        const size_t row = (size_t)k * g.B * g.block_len + r;
+        const int tok = c->blk_start_all[(size_t)k * g.B + r / g.block_len] + r % g.block_len;
+        const int pos = c->pos_of_tok[tok];
+        btok[row] = tok;
+        std::copy(cs.begin() + (size_t)pos * half, cs.begin() + (size_t)(pos + 1) * half, bcs.begin() + row * half);
+        std::copy(sn.begin() + (size_t)pos * half, sn.begin() + (size_t)(pos + 1) * half, bsn.begin() + row * half);
+      }
+    CU_TRY(c, dev_alloc(c, &c->d_blk_tok, rows));
+    CU_TRY(c, dev_alloc(c, &c->d_blk_cos, rows * half));
+    CU_TRY(c, dev_alloc(c, &c->d_blk_sin, rows * half));
+    CU_TRY(c, cudaMemcpy(c->d_blk_tok, btok.data(), sizeof(int32_t) * rows, cudaMemcpyHostToDevice));
+    CU_TRY(c, cudaMemcpy(c->d_blk_cos, bcs.data(), sizeof(float) * bcs.size(), cudaMemcpyHostToDevice));
+    CU_TRY(c, cudaMemcpy(c->d_blk_sin, bsn.data(), sizeof(float) * bsn.size(), cudaMemcpyHostToDevice));
   }
   lacache_status st = alloc_rot(c, &c->rot);
   if (st != LACACHE_OK) return st;
@@ -522,6 +546,12 @@ lacache_status lacache_step(lacache_ctx* c, const void* q, const void* k, const 
   r.blk_start = c->d_blk_start_all + (size_t)blk * c->g.B;
   r.block_len = c->g.block_len;
   r.pos_of_tok = c->d_pos; r.cos_tab = c->d_cos; r.sin_tab = c->d_sin;
+  {
+    const size_t row0 = (size_t)blk * c->g.B * c->g.block_len;
+    r.row_tok = c->d_blk_tok + row0;
+    r.row_cos = c->d_blk_cos + row0 * (c->g.d / 2);
+    r.row_sin = c->d_blk_sin + row0 * (c->g.d / 2);
+  }
   r.dst = c->rot;
   r.in_dtype = c->cfg.dtype;
   CU_TRY(c, rope_write(c->g, r, c->engine, s));

@@ -75,6 +75,9 @@ struct RopeArgs {
   const int32_t* blk_start; int block_len;
   const int32_t* pos_of_tok;
   const float* cos_tab; const float* sin_tab;  // [maxN][d/2]
+  // optional (block rows of a step): destination token and cos/sin rows of source
+  // row r, gathered ahead of time so that no load of the kernel depends on another
+  const int32_t* row_tok; const float* row_cos; const float* row_sin;  // [n_src_rows], [n_src_rows][d/2]
   RotBuffers dst;
   int in_dtype;
 };

@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a)
   long long t = idx / chunks;
   int slot = (int)(t % slots);
   int r = (int)(t / slots);
-  int tok = a.blk_start ? a.blk_start[r / a.block_len] + r % a.block_len : r;
+  int tok = a.row_tok ? a.row_tok[r] : (a.blk_start ? a.blk_start[r / a.block_len] + r % a.block_len : r);
   const int half = g.d / 2;
   const int c0 = chunk * 8;
 
@@ -105,9 +105,15 @@ __global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a)
   load8(src, soff + c0, a.in_dtype, x1);
   load8(src, soff + c0 + half, a.in_dtype, x2);
   if (which < 2) {
-    int pos = a.pos_of_tok[tok];
-    const float4* cp = reinterpret_cast<const float4*>(a.cos_tab + (size_t)pos * half + c0);
-    const float4* sp = reinterpret_cast<const float4*>(a.sin_tab + (size_t)pos * half + c0);
+    const float4 *cp, *sp;
+    if (a.row_cos) {
+      cp = reinterpret_cast<const float4*>(a.row_cos + (size_t)r * half + c0);
+      sp = reinterpret_cast<const float4*>(a.row_sin + (size_t)r * half + c0);
+    } else {
+      int pos = a.pos_of_tok[tok];
+      cp = reinterpret_cast<const float4*>(a.cos_tab + (size_t)pos * half + c0);
+      sp = reinterpret_cast<const float4*>(a.sin_tab + (size_t)pos * half + c0);
+    }
     float4 ca = cp[0], cb = cp[1], sa = sp[0], sb = sp[1];
     float cs[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
     float sn[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
@@ -123,15 +129,18 @@ __global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a)
   }
   size_t doff = ((size_t)h * g.Tp + tok) * g.d;
   if (TC) {
+    // tcgen05 storage: [head][feature half][Tp][64] (d = 128), each half of a row one 128-byte line
+    const size_t o1 = ((size_t)(2 * h) * g.Tp + tok) * 64 + c0;
+    const size_t o2 = ((size_t)(2 * h + 1) * g.Tp + tok) * 64 + c0;
     if (which == 0) {
-      store8_split(a.dst.q_hi, a.dst.q_lo, doff + c0, y1);
-      store8_split(a.dst.q_hi, a.dst.q_lo, doff + c0 + half, y2);
+      store8_split(a.dst.q_hi, a.dst.q_lo, o1, y1);
+      store8_split(a.dst.q_hi, a.dst.q_lo, o2, y2);
     } else if (which == 1) {
-      store8_split(a.dst.k_hi, a.dst.k_lo, doff + c0, y1);
-      store8_split(a.dst.k_hi, a.dst.k_lo, doff + c0 + half, y2);
+      store8_split(a.dst.k_hi, a.dst.k_lo, o1, y1);
+      store8_split(a.dst.k_hi, a.dst.k_lo, o2, y2);
     } else {
-      store8_f16(a.dst.v, doff + c0, y1);
-      store8_f16(a.dst.v, doff + c0 + half, y2);
+      store8_f16(a.dst.v, o1, y1);
+      store8_f16(a.dst.v, o2, y2);
     }
   } else {
     void* plane = which == 0 ? a.dst.q_hi : (which == 1 ? a.dst.k_hi : a.dst.v);
@@ -159,9 +168,11 @@ __global__ void __launch_bounds__(256) export_kernel(Geometry g, ExportArgs a) {
   long long t = idx / g.d;
   int h = (int)(t % g.Hq);
   int tok = (int)(t / g.Hq);
-  size_t src = ((size_t)h * g.Tp + tok) * g.d + c;
+  const size_t srow = ((size_t)h * g.Tp + tok) * g.d + c;   // state: [head][Tp][d]
+  // rotated planes: the tcgen05 engine stores [head][feature half][Tp][64]
+  const size_t src = TC ? ((size_t)(2 * h + c / 64) * g.Tp + tok) * 64 + c % 64 : srow;
   const float LN2 = 0.69314718055994530942f;
-  if (a.o) a.o[idx] = a.st.o[src];
+  if (a.o) a.o[idx] = a.st.o[srow];
   if (c == 0) {
     if (a.m) a.m[(size_t)tok * g.Hq + h] = a.st.m[(size_t)h * g.Tp + tok] * LN2;
     if (a.l) a.l[(size_t)tok * g.Hq + h] = a.st.l[(size_t)h * g.Tp + tok];

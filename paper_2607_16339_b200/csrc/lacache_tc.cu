@@ -41,18 +41,17 @@
 namespace lacache {
 
 struct TcMaps {
-  alignas(64) CUtensorMap q_hi;    // box 128 rows
-  alignas(64) CUtensorMap q_lo;
-  alignas(64) CUtensorMap q64_hi;  // box 64 rows (block queries)
-  alignas(64) CUtensorMap q64_lo;
-  alignas(64) CUtensorMap k_hi;    // box 128 rows (stream role)
-  alignas(64) CUtensorMap k_lo;
+  // rotated Q' / K': 5-D views {64 features, Tp rows, 2 feature halves, heads, 2 planes (hi, lo)} of the
+  // split-bf16 storage [plane][head][half][Tp][64]; one box = both planes and both halves of `rows` rows
+  // of one head, laid out in shared memory as [plane][half][rows][64] (128-byte swizzle)
+  alignas(64) CUtensorMap q;       // box 128 rows
+  alignas(64) CUtensorMap q64;     // box 64 rows (block queries)
+  alignas(64) CUtensorMap k;       // box TC_KEYS rows (stream role)
+  alignas(64) CUtensorMap k64;     // box 64 rows (the block's keys, merge role)
+  alignas(64) CUtensorMap k32;     // box 32 rows (the block's keys, pipelined merge role)
+  // V: 4-D views {64, Tp, 2 halves, heads} of the fp16 storage [head][half][Tp][64]
   alignas(64) CUtensorMap v;
-  alignas(64) CUtensorMap k64_hi;  // box 64 rows (the block's keys, merge role)
-  alignas(64) CUtensorMap k64_lo;
   alignas(64) CUtensorMap v64;
-  alignas(64) CUtensorMap k32_hi;  // box 32 rows (the block's keys, pipelined merge role)
-  alignas(64) CUtensorMap k32_lo;
   alignas(64) CUtensorMap v32;
   alignas(64) CUtensorMap st_o;    // cached O~ [Hq][Tp][128] fp32, box 32 cols x 128 rows
   alignas(64) CUtensorMap out;     // caller's out [T][Hq][128] fp32, box 32 cols x 1 head x 128 rows
@@ -171,6 +170,27 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+// both planes and both feature halves of `rows` rows of head h, starting at row `row`
+__device__ __forceinline__ void load_qk_box(uint32_t dst, const CUtensorMap* map, uint32_t bar, int row, int h) {
+  tma_load_5d(dst, map, bar, 0, row, 0, h, 0);
+}
+__device__ __forceinline__ void load_v_box(uint32_t dst, const CUtensorMap* map, uint32_t bar, int row, int h) {
+  tma_load_4d(dst, map, bar, 0, row, 0, h);
 }
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(map),
@@ -438,24 +458,16 @@ __device__ __forceinline__ void issue_pv_mma(uint32_t v_base, uint32_t v_box, ui
     mma_ts(o_tmem, p_tmem + 8 * ks, vd + (uint64_t)(ks * (2048 >> 4)), idesc, (ks > 0) ? 1u : accumulate);
 }
 __device__ __forceinline__ void load_kv_tile(const TcMaps& maps, uint32_t kv_base, uint32_t bar, int krow, int kh) {
+  static_assert(KV_KLO == 2 * K_BOX && KV_V == 4 * K_BOX, "K hi, K lo and V boxes are contiguous");
   mbar_expect_tx(bar, 6 * K_BOX);
-  tma_load_3d(kv_base, &maps.k64_hi, bar, 0, krow, kh);
-  tma_load_3d(kv_base + K_BOX, &maps.k64_hi, bar, 64, krow, kh);
-  tma_load_3d(kv_base + KV_KLO, &maps.k64_lo, bar, 0, krow, kh);
-  tma_load_3d(kv_base + KV_KLO + K_BOX, &maps.k64_lo, bar, 64, krow, kh);
-  tma_load_3d(kv_base + KV_V, &maps.v64, bar, 0, krow, kh);
-  tma_load_3d(kv_base + KV_V + K_BOX, &maps.v64, bar, 64, krow, kh);
+  load_qk_box(kv_base, &maps.k64, bar, krow, kh);
+  load_v_box(kv_base + KV_V, &maps.v64, bar, krow, kh);
 }
 __device__ __forceinline__ void load_q_tile(const Cta& c, const TcMaps& maps, int q_rows, int row0, int h) {
   const uint32_t bar = c.bar(BAR_Q_FULL);
   const uint32_t box = (uint32_t)q_rows * 128u;
-  const CUtensorMap* mh = q_rows == 64 ? &maps.q64_hi : &maps.q_hi;
-  const CUtensorMap* ml = q_rows == 64 ? &maps.q64_lo : &maps.q_lo;
   mbar_expect_tx(bar, 4 * box);
-  tma_load_3d(c.base + SM_Q, mh, bar, 0, row0, h);
-  tma_load_3d(c.base + SM_Q + box, mh, bar, 64, row0, h);
-  tma_load_3d(c.base + SM_Q + 2 * box, ml, bar, 0, row0, h);
-  tma_load_3d(c.base + SM_Q + 3 * box, ml, bar, 64, row0, h);
+  load_qk_box(c.base + SM_Q, q_rows == 64 ? &maps.q64 : &maps.q, bar, row0, h);
 }
 
 // ===========================================================================
@@ -521,12 +533,9 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         if (kuse == 0 || mbar_test(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE), (kuse - 1) & 1)) {
           const int krow = ck.un.key_base + ck.t * BN;
           const uint32_t bar = c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL);
-          const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
+          const uint32_t khi = c.base + SM_K + sk * K_STAGE;
           mbar_expect_tx(bar, 4 * KS_BOX);
-          tma_load_3d(khi, &maps.k_hi, bar, 0, krow, ck.un.kh);
-          tma_load_3d(khi + KS_BOX, &maps.k_hi, bar, 64, krow, ck.un.kh);
-          tma_load_3d(klo, &maps.k_lo, bar, 0, krow, ck.un.kh);
-          tma_load_3d(klo + KS_BOX, &maps.k_lo, bar, 64, krow, ck.un.kh);
+          load_qk_box(khi, &maps.k, bar, krow, ck.un.kh);  // the lo plane lands at khi + SK_LO
           cursor_advance(g, a, ck, stride, n_units);
           did = true;
         }
@@ -539,8 +548,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
           const int krow = cv.un.key_base + cv.t * BN;
           const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
           mbar_expect_tx(bar, 2 * KS_BOX);
-          tma_load_3d(vb, &maps.v, bar, 0, krow, cv.un.kh);
-          tma_load_3d(vb + KS_BOX, &maps.v, bar, 64, krow, cv.un.kh);
+          load_v_box(vb, &maps.v, bar, krow, cv.un.kh);
           cursor_advance(g, a, cv, stride, n_units);
           did = true;
         }
@@ -1215,18 +1223,14 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
     const uint32_t bar = c.bar(BAR_KV_FULL), kb = c.base + DM_K;
     const int kh = un.h / g.group;
     mbar_expect_tx(bar, 4 * DM_KBOX);
-    tma_load_3d(kb, &maps.k32_hi, bar, 0, un.blk_start, kh);
-    tma_load_3d(kb + DM_KBOX, &maps.k32_hi, bar, 64, un.blk_start, kh);
-    tma_load_3d(kb + 2 * DM_KBOX, &maps.k32_lo, bar, 0, un.blk_start, kh);
-    tma_load_3d(kb + 3 * DM_KBOX, &maps.k32_lo, bar, 64, un.blk_start, kh);
+    load_qk_box(kb, &maps.k32, bar, un.blk_start, kh);
   };
   auto load_v = [&](int i) {
     const DUnit un = deep_unit(c, i);
     const uint32_t bar = c.bar(BAR_KV_FULL1), vb = c.base + DM_V;
     const int kh = un.h / g.group;
     mbar_expect_tx(bar, 2 * DM_KBOX);
-    tma_load_3d(vb, &maps.v32, bar, 0, un.blk_start, kh);
-    tma_load_3d(vb + DM_KBOX, &maps.v32, bar, 64, un.blk_start, kh);
+    load_v_box(vb, &maps.v32, bar, un.blk_start, kh);
   };
   // Q' and cached O~ of fixed rows do not depend on the RoPE kernel launched
   // just before this one; the block's keys and values do
@@ -1447,13 +1451,11 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   const bool deep = !stream && a.merge_deep != 0;
   if (tid == 0) {  // descriptor fetches overlap the set-up below
     if (stream) {
-      prefetch_map(a.mode == MODE_STEP ? &maps.q64_hi : &maps.q_hi);
-      prefetch_map(a.mode == MODE_STEP ? &maps.q64_lo : &maps.q_lo);
-      prefetch_map(&maps.k_hi); prefetch_map(&maps.k_lo); prefetch_map(&maps.v);
+      prefetch_map(a.mode == MODE_STEP ? &maps.q64 : &maps.q);
+      prefetch_map(&maps.k); prefetch_map(&maps.v);
     } else {
-      prefetch_map(&maps.q_hi); prefetch_map(&maps.q_lo); prefetch_map(&maps.st_o); prefetch_map(&maps.out);
-      if (deep) { prefetch_map(&maps.k32_hi); prefetch_map(&maps.k32_lo); prefetch_map(&maps.v32); }
-      else { prefetch_map(&maps.k64_hi); prefetch_map(&maps.k64_lo); prefetch_map(&maps.v64); }
+      prefetch_map(&maps.q); prefetch_map(&maps.st_o); prefetch_map(&maps.out);
+      prefetch_map(deep ? &maps.k32 : &maps.k64); prefetch_map(deep ? &maps.v32 : &maps.v64);
     }
   }
   const int n_my = first < n_units ? (n_units - first + stride - 1) / stride : 0;
@@ -1573,17 +1575,33 @@ bool make_f32_map(CUtensorMap* m, void* base, cuuint64_t d1, cuuint64_t d2, cuui
   return true;
 }
 
-bool make_plane_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, bool fp16, char* err, int errlen) {
+// Split-bf16 planes [plane][H][2][Tp][64] (hi plane at `base`, lo plane `plane_elems` further) as a 5-D
+// tensor; fp16 values [H][2][Tp][64] as a 4-D tensor.  Box: `box_rows` rows of one head, both feature
+// halves (and both planes).
+bool make_qk_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* err, int errlen) {
   EncodeTiledFn enc = get_encode();
   if (!enc) { snprintf(err, errlen, "cuTensorMapEncodeTiled entry point not found"); return false; }
-  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)Tp, (cuuint64_t)H};
-  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)Tp * D * 2};
-  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = enc(m, fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims,
-                   strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) { snprintf(err, errlen, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r); return false; }
+  cuuint64_t dims[5] = {64, (cuuint64_t)Tp, 2, (cuuint64_t)H, 2};
+  cuuint64_t strides[4] = {128, (cuuint64_t)Tp * 128, (cuuint64_t)Tp * 256, (cuuint64_t)H * Tp * 256};
+  cuuint32_t box[5] = {64, (cuuint32_t)box_rows, 2, 1, 2};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { snprintf(err, errlen, "cuTensorMapEncodeTiled (5-D) failed with CUresult %d", (int)r); return false; }
+  return true;
+}
+bool make_v_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* err, int errlen) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) { snprintf(err, errlen, "cuTensorMapEncodeTiled entry point not found"); return false; }
+  cuuint64_t dims[4] = {64, (cuuint64_t)Tp, 2, (cuuint64_t)H};
+  cuuint64_t strides[3] = {128, (cuuint64_t)Tp * 128, (cuuint64_t)Tp * 256};
+  cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 2, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, base, dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { snprintf(err, errlen, "cuTensorMapEncodeTiled (4-D) failed with CUresult %d", (int)r); return false; }
   return true;
 }
 
@@ -1604,19 +1622,15 @@ TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, c
   TcMaps* m = new TcMaps();
   m->out_ptr = nullptr;
   m->out = CUtensorMap{};
-  bool ok = make_plane_map(&m->q_hi, rot.q_hi, g.Hq, g.Tp, BM, false, err, errlen) &&
-            make_plane_map(&m->q_lo, rot.q_lo, g.Hq, g.Tp, BM, false, err, errlen) &&
-            make_plane_map(&m->q64_hi, rot.q_hi, g.Hq, g.Tp, 64, false, err, errlen) &&
-            make_plane_map(&m->q64_lo, rot.q_lo, g.Hq, g.Tp, 64, false, err, errlen) &&
-            make_plane_map(&m->k_hi, rot.k_hi, g.Hkv, g.Tp, BN, false, err, errlen) &&
-            make_plane_map(&m->k_lo, rot.k_lo, g.Hkv, g.Tp, BN, false, err, errlen) &&
-            make_plane_map(&m->v, rot.v, g.Hkv, g.Tp, BN, true, err, errlen) &&
-            make_plane_map(&m->k64_hi, rot.k_hi, g.Hkv, g.Tp, 64, false, err, errlen) &&
-            make_plane_map(&m->k64_lo, rot.k_lo, g.Hkv, g.Tp, 64, false, err, errlen) &&
-            make_plane_map(&m->v64, rot.v, g.Hkv, g.Tp, 64, true, err, errlen) &&
-            make_plane_map(&m->k32_hi, rot.k_hi, g.Hkv, g.Tp, 32, false, err, errlen) &&
-            make_plane_map(&m->k32_lo, rot.k_lo, g.Hkv, g.Tp, 32, false, err, errlen) &&
-            make_plane_map(&m->v32, rot.v, g.Hkv, g.Tp, 32, true, err, errlen) &&
+  // (the lo planes follow the hi planes at a fixed distance: see alloc_rot)
+  bool ok = make_qk_map(&m->q, rot.q_hi, g.Hq, g.Tp, BM, err, errlen) &&
+            make_qk_map(&m->q64, rot.q_hi, g.Hq, g.Tp, 64, err, errlen) &&
+            make_qk_map(&m->k, rot.k_hi, g.Hkv, g.Tp, BN, err, errlen) &&
+            make_qk_map(&m->k64, rot.k_hi, g.Hkv, g.Tp, 64, err, errlen) &&
+            make_qk_map(&m->k32, rot.k_hi, g.Hkv, g.Tp, 32, err, errlen) &&
+            make_v_map(&m->v, rot.v, g.Hkv, g.Tp, BN, err, errlen) &&
+            make_v_map(&m->v64, rot.v, g.Hkv, g.Tp, 64, err, errlen) &&
+            make_v_map(&m->v32, rot.v, g.Hkv, g.Tp, 32, err, errlen) &&
             make_f32_map(&m->st_o, state_o, (cuuint64_t)g.Tp, (cuuint64_t)g.Hq, BM, 1, err, errlen);
   if (!ok) { delete m; return nullptr; }
   return m;
