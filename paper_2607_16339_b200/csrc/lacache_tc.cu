@@ -506,53 +506,71 @@ __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs
 
 __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a,
                                 int first, int stride, int n_units, WorkItem it) {
-  TileCursor ck, cv;
-  ck.u = first; ck.uu = 0; ck.jj = 0; ck.loads_q = true;
-  cursor_load_unit(g, a, ck, n_units);
+  // three independent cursors: Q tiles (one per unit), key tiles, value tiles
+  TileCursor cq, ck, cv;
+  cq.u = first; cq.uu = 0; cq.jj = 0; cq.loads_q = true;
+  cursor_load_unit(g, a, cq, n_units);
+  ck = cq;
+  ck.loads_q = false;  // the key and value cursors never load Q
+  ck.q_done = true;
+  if (ck.valid && ck.t >= ck.un.t1) cursor_advance(g, a, ck, stride, n_units);
   cv = ck;
-  cv.loads_q = false;  // the value cursor never loads Q
-  cv.q_done = true;
-  if (cv.valid && cv.t >= cv.un.t1) cursor_advance(g, a, cv, stride, n_units);
-  // everything this role loads was written by the RoPE kernel launched just
-  // before this one: wait for that grid (this kernel may have started early)
-  grid_dependency_wait();
-  // a unit without key tiles still needs its Q load (the MMA thread waits for it)
+  // What the RoPE kernel launched just before this one writes must not be loaded
+  // before that grid has completed (this kernel may have started early): in a step
+  // that is the block's rows -- every Q tile of this role and the key/value tiles
+  // that overlap the block -- so tiles of fixed tokens are requested at once and
+  // the wait comes only when nothing else can be issued.
+  bool dep_done = false;
+  auto tile_depends = [&](const TileCursor& cu) {
+    if (a.mode != MODE_STEP) return true;
+    const int krow = cu.un.key_base + cu.t * BN;
+    return krow < cu.it.blk_start + g.block_len && krow + BN > cu.it.blk_start;
+  };
   long long t_idle = 0;
-  while (ck.valid || cv.valid) {
-    bool did = false;
-    if (ck.valid) {
-      if (!ck.q_done) {
-        if (ck.uu == 0 || mbar_test(c.bar(BAR_Q_FREE), (ck.uu - 1) & 1)) {
-          load_q_tile(c, maps, ck.un.q_rows, ck.un.row0, ck.un.h);
-          ck.q_done = true;
-          if (ck.t >= ck.un.t1) cursor_advance(g, a, ck, stride, n_units);  // no key tiles at all
-          did = true;
-        }
-      } else if (ck.t < ck.un.t1) {
-        const int sk = ck.jj & 1, kuse = ck.jj >> 1;
-        if (kuse == 0 || mbar_test(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE), (kuse - 1) & 1)) {
-          const int krow = ck.un.key_base + ck.t * BN;
-          const uint32_t bar = c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL);
-          const uint32_t khi = c.base + SM_K + sk * K_STAGE;
-          mbar_expect_tx(bar, 4 * KS_BOX);
-          load_qk_box(khi, &maps.k, bar, krow, ck.un.kh);  // the lo plane lands at khi + SK_LO
-          cursor_advance(g, a, ck, stride, n_units);
-          did = true;
-        }
+  while (cq.valid || ck.valid || cv.valid) {
+    bool did = false, blocked_on_dep = false;
+    if (cq.valid) {  // a unit without key tiles still needs its Q load (the MMA thread waits for it)
+      if (!dep_done) {
+        blocked_on_dep = true;
+      } else if (cq.uu == 0 || mbar_test(c.bar(BAR_Q_FREE), (cq.uu - 1) & 1)) {
+        load_q_tile(c, maps, cq.un.q_rows, cq.un.row0, cq.un.h);
+        cq.q_done = true;
+        cq.t = cq.un.t1;
+        cursor_advance(g, a, cq, stride, n_units);
+        did = true;
       }
     }
-    if (cv.valid) {
-      if (cv.t < cv.un.t1) {
-        const int sv = cv.jj & 1, vuse = cv.jj >> 1;
-        if (vuse == 0 || mbar_test(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE), (vuse - 1) & 1)) {
-          const int krow = cv.un.key_base + cv.t * BN;
-          const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
-          mbar_expect_tx(bar, 2 * KS_BOX);
-          load_v_box(vb, &maps.v, bar, krow, cv.un.kh);
-          cursor_advance(g, a, cv, stride, n_units);
-          did = true;
-        }
+    if (ck.valid && ck.t < ck.un.t1) {
+      const int sk = ck.jj & 1, kuse = ck.jj >> 1;
+      if (!dep_done && tile_depends(ck)) {
+        blocked_on_dep = true;
+      } else if (kuse == 0 || mbar_test(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE), (kuse - 1) & 1)) {
+        const int krow = ck.un.key_base + ck.t * BN;
+        const uint32_t bar = c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL);
+        const uint32_t khi = c.base + SM_K + sk * K_STAGE;
+        mbar_expect_tx(bar, 4 * KS_BOX);
+        load_qk_box(khi, &maps.k, bar, krow, ck.un.kh);  // the lo plane lands at khi + SK_LO
+        cursor_advance(g, a, ck, stride, n_units);
+        did = true;
       }
+    }
+    if (cv.valid && cv.t < cv.un.t1) {
+      const int sv = cv.jj & 1, vuse = cv.jj >> 1;
+      if (!dep_done && tile_depends(cv)) {
+        blocked_on_dep = true;
+      } else if (vuse == 0 || mbar_test(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE), (vuse - 1) & 1)) {
+        const int krow = cv.un.key_base + cv.t * BN;
+        const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
+        mbar_expect_tx(bar, 2 * KS_BOX);
+        load_v_box(vb, &maps.v, bar, krow, cv.un.kh);
+        cursor_advance(g, a, cv, stride, n_units);
+        did = true;
+      }
+    }
+    if (!did && blocked_on_dep) {
+      grid_dependency_wait();
+      dep_done = true;
+      did = true;
     }
     if (did) {
       t_idle = 0;
@@ -568,6 +586,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
       }
     }
   }
+  // (a CTA without units never touches memory the RoPE kernel writes)
 }
 
 // The MMA thread issues whichever product is ready: P~V of the oldest pending
