@@ -688,6 +688,59 @@ __device__ __forceinline__ void coop_store_rows(const Cta& c, uint32_t stage_off
   }
 }
 
+// Few chunks (at most NC): each thread takes BATCH (row, 16-byte column) items at a
+// time and issues every load of the batch -- references, normalisers, 16 bytes of
+// each partial O~ -- before any is used: one L2 round trip per batch.
+template <int NC, int BATCH>
+__device__ __forceinline__ void merge_few(const Geometry& g, const AttnArgs& a, size_t pbase, int nchunks,
+                                          int block_len, int row0, int h) {
+  const float LN2 = 0.69314718055994530942f;
+  const int t = threadIdx.x - 64;
+  const int n_items = block_len * 32;
+  for (int i0 = t; i0 < n_items; i0 += BATCH * ROW_THREADS) {
+    float mv[BATCH][NC], lv[BATCH][NC];
+    float4 v[BATCH][NC];
+#pragma unroll
+    for (int bi = 0; bi < BATCH; ++bi) {
+      const int i = min(i0 + bi * ROW_THREADS, n_items - 1);
+      const int rr = i >> 5, ch = i & 31;
+#pragma unroll
+      for (int k = 0; k < NC; ++k) {
+        const size_t pr = (pbase + min(k, nchunks - 1)) * block_len + rr;
+        mv[bi][k] = __ldcg(a.part_m + pr);
+        lv[bi][k] = __ldcg(a.part_l + pr);
+        v[bi][k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + pr * D) + ch);
+      }
+    }
+#pragma unroll
+    for (int bi = 0; bi < BATCH; ++bi) {
+      const int i = i0 + bi * ROW_THREADS;
+      if (i >= n_items) break;
+      const int rr = i >> 5, ch = i & 31;
+      float M = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < NC; ++k)
+        if (k < nchunks) M = fmaxf(M, mv[bi][k]);
+      float L = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int k = 0; k < NC; ++k) {
+        const float w = (k < nchunks && mv[bi][k] != -INFINITY) ? ex2(mv[bi][k] - M) : 0.f;
+        L = fmaf(lv[bi][k], w, L);
+        acc.x = fmaf(v[bi][k].x, w, acc.x);
+        acc.y = fmaf(v[bi][k].y, w, acc.y);
+        acc.z = fmaf(v[bi][k].z, w, acc.z);
+        acc.w = fmaf(v[bi][k].w, w, acc.w);
+      }
+      const float inv = 1.f / L;
+      const size_t orow = (size_t)(row0 + rr) * g.Hq + h;
+      *reinterpret_cast<float4*>(a.out + orow * D + ch * 4) =
+          make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+      if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
+    }
+  }
+}
+
 // Merge of the partial states of all key chunks of one (sequence, head) by the
 // last chunk to arrive: thread t owns 16 bytes of one row; the partial rows are
 // read with coalesced loads straight from L2 and the normalised rows written out.
@@ -695,40 +748,12 @@ __device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs
                                                int block_len, int row0, int h) {
   const float LN2 = 0.69314718055994530942f;
   const int t = threadIdx.x - 64;
+  if (nchunks <= 2) {
+    merge_few<2, 4>(g, a, pbase, nchunks, block_len, row0, h);
+    return;
+  }
   if (nchunks <= 4) {
-    // few chunks: every load of a row (references, normalisers, 16 bytes of each
-    // partial O~) is issued before any is used -- one L2 round trip in all
-    for (int i = t; i < block_len * 32; i += ROW_THREADS) {
-      const int rr = i >> 5, ch = i & 31;
-      float mv[4], lv[4];
-      float4 v[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const size_t pr = (pbase + min(k, nchunks - 1)) * block_len + rr;
-        mv[k] = __ldcg(a.part_m + pr);
-        lv[k] = __ldcg(a.part_l + pr);
-        v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + pr * D) + ch);
-      }
-      float M = -INFINITY;
-#pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (k < nchunks) M = fmaxf(M, mv[k]);
-      float L = 0.f;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float w = (k < nchunks && mv[k] != -INFINITY) ? ex2(mv[k] - M) : 0.f;
-        L = fmaf(lv[k], w, L);
-        acc.x = fmaf(v[k].x, w, acc.x);
-        acc.y = fmaf(v[k].y, w, acc.y);
-        acc.z = fmaf(v[k].z, w, acc.z);
-        acc.w = fmaf(v[k].w, w, acc.w);
-      }
-      const float inv = 1.f / L;
-      const size_t orow = (size_t)(row0 + rr) * g.Hq + h;
-      *reinterpret_cast<float4*>(a.out + orow * D + ch * 4) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-      if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
-    }
+    merge_few<4, 2>(g, a, pbase, nchunks, block_len, row0, h);
     return;
   }
   for (int i = t; i < block_len * 32; i += ROW_THREADS) {
@@ -930,6 +955,51 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     if (!epi_sync(c, epi_phase)) return;
     const float l_run = lx[0] + lx[1];
     const float mul = (un.epi == EPI_OUT) ? 1.f / l_run : 1.f;
+    if (un.epi == EPI_PARTIAL) {
+      // Partial state of this key chunk, straight from TMEM to global memory (each
+      // thread 256 contiguous bytes of its row); the last chunk of the (sequence,
+      // head) to arrive merges all of them.
+      const size_t pbase = ((size_t)un.seq * g.Hq + un.h) * a.max_chunks;  // [chunk][block_len]
+      const size_t prow0 = (pbase + un.chunk) * g.block_len;
+      if (row_valid) {
+        float4* dst = reinterpret_cast<float4*>(a.part_o + (prow0 + r) * D + 64 * half);
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t rr[16];
+          if (!first_tile) {
+            tmem_ld16(tlane + TS_O + 64 * half + 16 * cb, rr);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) rr[j] = 0u;
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            dst[4 * cb + i] = make_float4(__uint_as_float(rr[4 * i]), __uint_as_float(rr[4 * i + 1]),
+                                          __uint_as_float(rr[4 * i + 2]), __uint_as_float(rr[4 * i + 3]));
+        }
+        if (half == 0) { a.part_m[prow0 + r] = m_ref; a.part_l[prow0 + r] = l_run; }
+      }
+      tc_fence_before();
+      mbar_arrive(c.bar(BAR_O_FREE));  // the next unit may overwrite O~
+      if (!epi_sync(c, epi_phase)) return;  // every partial store of the CTA happens-before thread 64's fence
+      if (threadIdx.x == 64) {
+        __threadfence();  // cumulative: publishes the whole CTA's partial state before the count
+        int* cnt = &a.counters[un.seq * g.Hq + un.h];
+        int old = atomicAdd(cnt, 1);
+        int last = (old == un.nchunks - 1) ? 1 : 0;
+        if (last) {
+          *cnt = 0;
+          __threadfence();  // the other chunks' partial states are visible from here on
+        }
+        *c.flag = (uint32_t)last;
+      }
+      if (!epi_sync(c, epi_phase)) return;
+      if (*c.flag != 0) merge_partials(g, a, pbase, un.nchunks, g.block_len, un.row0, un.h);
+      if (!epi_sync(c, epi_phase)) return;  // the flag may be rewritten
+      if (un.q_rows == BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));
+      continue;
+    }
     // O~ (this thread's 64 features) from TMEM to its staging row.  The staging
     // area is the Q region (every score MMA of the unit is complete: the last
     // P~V, waited for above, was issued after them); 64-row units use its upper
@@ -969,30 +1039,6 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_ref + log2f(l_run)) * LN2;
       if (!epi_sync(c, epi_phase)) return;
       coop_store_rows(c, stage_off, a.out + ((size_t)un.row0 * g.Hq + un.h) * D, (size_t)g.Hq * D, un.nrows);
-    } else {
-      // partial state of this key chunk; the last chunk of the (sequence, head)
-      // to arrive merges all of them
-      const size_t pbase = ((size_t)un.seq * g.Hq + un.h) * a.max_chunks;  // [chunk][block_len]
-      const size_t prow0 = (pbase + un.chunk) * g.block_len;
-      if (row_valid && half == 0) { a.part_m[prow0 + r] = m_ref; a.part_l[prow0 + r] = l_run; }
-      if (!epi_sync(c, epi_phase)) return;
-      coop_store_rows(c, stage_off, a.part_o + prow0 * D, D, un.nrows);
-      if (!epi_sync(c, epi_phase)) return;  // every partial store of the CTA happens-before thread 64's fence
-      if (threadIdx.x == 64) {
-        __threadfence();  // cumulative: publishes the whole CTA's partial state before the count
-        int* cnt = &a.counters[un.seq * g.Hq + un.h];
-        int old = atomicAdd(cnt, 1);
-        int last = (old == un.nchunks - 1) ? 1 : 0;
-        if (last) {
-          *cnt = 0;
-          __threadfence();  // the other chunks' partial states are visible from here on
-        }
-        *c.flag = (uint32_t)last;
-      }
-      if (!epi_sync(c, epi_phase)) return;
-      if (*c.flag != 0) {
-        merge_partials(g, a, pbase, un.nchunks, g.block_len, un.row0, un.h);
-      }
     }
     if (!epi_sync(c, epi_phase)) return;  // the staging rows have been read
     if (un.q_rows == BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));  // the Q region may be reloaded
