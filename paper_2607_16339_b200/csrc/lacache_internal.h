@@ -89,6 +89,10 @@ struct AttnArgs {
   const WorkItem* items_merge; int n_items_merge;
   int n_ctas_stream; int n_ctas;
   int merge_deep;            // merge role runs its pipelined variant (block_len <= 32, bounded units per CTA)
+  // step only: the block's pre-RoPE queries [B * block_len, Hq, d] and the cos/sin rows of
+  // those tokens [B * block_len][d/2]; a CTA's first block-query unit rotates its Q tile
+  // from these itself and so does not have to wait for the RoPE kernel
+  const void* q_raw; int q_raw_bf16; const float* row_cos; const float* row_sin;
   const int32_t* cu;         // [B+1]
   const int32_t* blk_start;  // [B] absolute token index of the block's first row
   RotBuffers rot;

@@ -12,27 +12,10 @@
 #include <cuda_fp16.h>
 
 #include "lacache_internal.h"
+#include "lacache_rope_math.h"
 
 namespace lacache {
 namespace {
-
-__device__ __forceinline__ void load8(const void* base, size_t elem_off, int in_dtype, float (&x)[8]) {
-  if (in_dtype == LACACHE_DTYPE_BF16) {
-    uint4 u = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(base) + elem_off);
-    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&u);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float2 f = __bfloat1622float2(p[i]);
-      x[2 * i] = f.x;
-      x[2 * i + 1] = f.y;
-    }
-  } else {
-    const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(base) + elem_off);
-    float4 a = p[0], b = p[1];
-    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
-    x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
-  }
-}
 
 __device__ __forceinline__ void store8_f32(void* plane, size_t off, const float (&y)[8]) {
   float4* p = reinterpret_cast<float4*>(reinterpret_cast<float*>(plane) + off);
@@ -43,17 +26,7 @@ __device__ __forceinline__ void store8_f32(void* plane, size_t off, const float 
 __device__ __forceinline__ void store8_split(void* hi_plane, void* lo_plane, size_t off,
                                              const float (&y)[8]) {
   uint4 uh, ul;
-  __nv_bfloat162* ph = reinterpret_cast<__nv_bfloat162*>(&uh);
-  __nv_bfloat162* pl = reinterpret_cast<__nv_bfloat162*>(&ul);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    __nv_bfloat16 h0 = __float2bfloat16_rn(y[2 * i]);
-    __nv_bfloat16 h1 = __float2bfloat16_rn(y[2 * i + 1]);
-    __nv_bfloat16 l0 = __float2bfloat16_rn(y[2 * i] - __bfloat162float(h0));
-    __nv_bfloat16 l1 = __float2bfloat16_rn(y[2 * i + 1] - __bfloat162float(h1));
-    ph[i] = __halves2bfloat162(h0, h1);
-    pl[i] = __halves2bfloat162(l0, l1);
-  }
+  rope_split8(y, uh, ul);
   *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(hi_plane) + off) = uh;
   *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(lo_plane) + off) = ul;
 }
@@ -102,8 +75,8 @@ __global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a)
 
   float x1[8], x2[8], y1[8], y2[8];
   size_t soff = ((size_t)r * H + h) * g.d;
-  load8(src, soff + c0, a.in_dtype, x1);
-  load8(src, soff + c0 + half, a.in_dtype, x2);
+  rope_load8(src, soff + c0, a.in_dtype == LACACHE_DTYPE_BF16, x1);
+  rope_load8(src, soff + c0 + half, a.in_dtype == LACACHE_DTYPE_BF16, x2);
   if (which < 2) {
     const float4 *cp, *sp;
     if (a.row_cos) {
@@ -117,12 +90,7 @@ __global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a)
     float4 ca = cp[0], cb = cp[1], sa = sp[0], sb = sp[1];
     float cs[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
     float sn[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      // separate roundings on purpose (no fma contraction surprises)
-      y1[i] = __fsub_rn(__fmul_rn(x1[i], cs[i]), __fmul_rn(x2[i], sn[i]));
-      y2[i] = __fadd_rn(__fmul_rn(x2[i], cs[i]), __fmul_rn(x1[i], sn[i]));
-    }
+    rope_rotate8(x1, x2, cs, sn, y1, y2);
   } else {
 #pragma unroll
     for (int i = 0; i < 8; ++i) { y1[i] = x1[i]; y2[i] = x2[i]; }

@@ -37,6 +37,7 @@
 #include <stdlib.h>
 
 #include "lacache_internal.h"
+#include "lacache_rope_math.h"
 
 namespace lacache {
 
@@ -55,6 +56,7 @@ struct TcMaps {
   alignas(64) CUtensorMap v32;
   alignas(64) CUtensorMap st_o;    // cached O~ [Hq][Tp][128] fp32, box 32 cols x 128 rows
   alignas(64) CUtensorMap out;     // caller's out [T][Hq][128] fp32, box 32 cols x 1 head x 128 rows
+  alignas(64) CUtensorMap out_sub[4];  // the same with boxes of 64, 32, 16 and 8 rows (clipped row tiles)
   const void* out_ptr;             // the buffer `out` was encoded for
 };
 
@@ -122,6 +124,7 @@ enum {
   BAR_O_FULL, BAR_O_FULL1, BAR_O_FREE, BAR_O_FREE1,
   BAR_IO_FULL, BAR_IO_FREE, BAR_EPI, BAR_DONE,
   BAR_K_FULL1, BAR_K_FREE1, BAR_V_FULL1, BAR_V_FREE1,  // stream role, second key / value stage
+  BAR_QC,  // stream role: the row threads have written the rotated Q tile of the CTA's first unit
   BAR_IO_FULL1, BAR_OUT_RDY, BAR_OUT_RDY1,  // pipelined merge role: second staging tile; output tile b is complete
   BAR_PAIR,  // 4 barriers: the two warps that share a TMEM lane quadrant
   N_BARS = BAR_PAIR + 4
@@ -521,6 +524,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
   // that overlap the block -- so tiles of fixed tokens are requested at once and
   // the wait comes only when nothing else can be issued.
   bool dep_done = false;
+  const bool q_computed = a.mode == MODE_STEP && a.q_raw != nullptr;
   auto tile_depends = [&](const TileCursor& cu) {
     if (a.mode != MODE_STEP) return true;
     const int krow = cu.un.key_base + cu.t * BN;
@@ -530,7 +534,15 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
   while (cq.valid || ck.valid || cv.valid) {
     bool did = false, blocked_on_dep = false;
     if (cq.valid) {  // a unit without key tiles still needs its Q load (the MMA thread waits for it)
-      if (!dep_done) {
+      if (cq.uu == 0 && q_computed) {
+        // the row threads rotate this tile from the raw queries: nothing to load,
+        // nothing to wait for (the plain arrival keeps the barrier's phase count in step)
+        mbar_arrive(c.bar(BAR_Q_FULL));
+        cq.q_done = true;
+        cq.t = cq.un.t1;
+        cursor_advance(g, a, cq, stride, n_units);
+        did = true;
+      } else if (!dep_done) {
         blocked_on_dep = true;
       } else if (cq.uu == 0 || mbar_test(c.bar(BAR_Q_FREE), (cq.uu - 1) & 1)) {
         load_q_tile(c, maps, cq.un.q_rows, cq.un.row0, cq.un.h);
@@ -603,6 +615,7 @@ __device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, i
     const Unit un = decode_stream(g, a, it, u);
     const uint32_t q_box = (uint32_t)un.q_rows * 128u;
     if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
+    if (uu == 0 && a.mode == MODE_STEP && a.q_raw != nullptr && !wait_bar(c, BAR_QC, 0, LOC_WAIT_Q)) return;
     int ts = next_tile(un, un.t0), tp = ts;
     bool q_released = false, first_pv = true;
     bool o_free_pending = uu >= 1;  // O_FREE of the previous unit is observed exactly once, in order
@@ -811,6 +824,38 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
     const Unit un = decode_stream(g, a, it, u);
     it = nxt;
+    if (u == first && a.mode == MODE_STEP && a.q_raw != nullptr) {
+      // The CTA's first unit: rotate the block's queries of this (sequence, head) here,
+      // with the very arithmetic of the RoPE kernel, and write them where the TMA load
+      // would have put them ([plane][feature half][row][64], 16-byte chunks XOR-swizzled
+      // by the row), so this unit does not wait for that kernel.
+      const int tq = threadIdx.x - 64;
+      const uint32_t box = (uint32_t)un.q_rows * 128u;
+      for (int i = tq; i < un.nrows * 8; i += ROW_THREADS) {
+        const int qi = i >> 3, ch = i & 7, c0 = ch * 8;
+        const size_t src = (size_t)un.seq * g.block_len + qi;            // row of the block's inputs
+        const size_t soff = (src * g.Hq + un.h) * D;
+        float x1[8], x2[8], cs[8], sn[8], y1[8], y2[8];
+        rope_load8(a.q_raw, soff + c0, a.q_raw_bf16 != 0, x1);
+        rope_load8(a.q_raw, soff + c0 + D / 2, a.q_raw_bf16 != 0, x2);
+        const float4* cp = reinterpret_cast<const float4*>(a.row_cos + src * (D / 2) + c0);
+        const float4* sp = reinterpret_cast<const float4*>(a.row_sin + src * (D / 2) + c0);
+        const float4 ca = cp[0], cb = cp[1], sa = sp[0], sb = sp[1];
+        cs[0] = ca.x; cs[1] = ca.y; cs[2] = ca.z; cs[3] = ca.w; cs[4] = cb.x; cs[5] = cb.y; cs[6] = cb.z; cs[7] = cb.w;
+        sn[0] = sa.x; sn[1] = sa.y; sn[2] = sa.z; sn[3] = sa.w; sn[4] = sb.x; sn[5] = sb.y; sn[6] = sb.z; sn[7] = sb.w;
+        rope_rotate8(x1, x2, cs, sn, y1, y2);
+        uint4 h1, l1, h2, l2;
+        rope_split8(y1, h1, l1);
+        rope_split8(y2, h2, l2);
+        uint8_t* const q0 = c.gen + SM_Q + qi * 128 + ((ch ^ (qi & 7)) << 4);
+        *reinterpret_cast<uint4*>(q0) = h1;                 // hi plane, features [0, 64)
+        *reinterpret_cast<uint4*>(q0 + box) = h2;           // hi plane, features [64, 128)
+        *reinterpret_cast<uint4*>(q0 + 2 * box) = l1;       // lo plane
+        *reinterpret_cast<uint4*>(q0 + 3 * box) = l2;
+      }
+      fence_async_smem();  // the MMA reads shared memory through the async proxy
+      mbar_arrive(c.bar(BAR_QC));
+    }
     const int row = un.row0 + r;
     const bool row_valid = r < un.nrows;
     const bool active = quad * 32 < un.nrows;  // this warp holds at least one real row
@@ -1045,6 +1090,31 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
   }
 }
 
+// Output rows [row0, row0 + nrows) of head h from a swizzled staging tile (four boxes of
+// 32 features x 128 rows) to the caller's `out` with tiled bulk stores: one 128-row box, or
+// for a clipped tile boxes of 64, 32, 16 and 8 rows (each starts on a multiple of 8 rows,
+// where the staging tile's swizzle pattern repeats).  Returns the rows covered; the last
+// nrows % 8 rows are left to the row threads.  The caller commits the bulk group.
+__device__ __forceinline__ int store_out_tile(const TcMaps& maps, uint32_t src, int h, int row0, int nrows) {
+  if (nrows == BM) {
+#pragma unroll
+    for (int cb = 0; cb < 4; ++cb) tma_store_3d(&maps.out, src + cb * IO_BOX, 32 * cb, h, row0);
+    return BM;
+  }
+  int done = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int bs = 64 >> i;
+    if (nrows - done >= bs) {
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb)
+        tma_store_3d(&maps.out_sub[i], src + cb * IO_BOX + done * 128, 32 * cb, h, row0 + done);
+      done += bs;
+    }
+  }
+  return done;
+}
+
 // ===========================================================================
 // merge role: fixed queries x block keys, merged into the cached state
 // ===========================================================================
@@ -1053,8 +1123,8 @@ __device__ void merge_producer(const Cta& c, const TcMaps& maps, const Geometry&
   int uu = 0;
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items_merge + (u + stride) % a.n_items_merge);
-    const int h = u / a.n_items_merge;
+    if (u + stride < n_units) nxt = load_item(a.items_merge + (u + stride) / g.Hq);
+    const int h = u % g.Hq;
     const int b = uu & 1, k = uu >> 1;
     if (uu >= 1 && !wait_bar(c, BAR_Q_FREE, (uu - 1) & 1, LOC_WAIT_Q)) return;
     load_q_tile(c, maps, BM, it.row0, h);
@@ -1136,8 +1206,8 @@ __device__ void merge_rows(const Cta& c, const TcMaps& maps, const Geometry& g, 
   int uu = 0;
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items_merge + (u + stride) % a.n_items_merge);
-    const int h = u / a.n_items_merge;
+    if (u + stride < n_units) nxt = load_item(a.items_merge + (u + stride) / g.Hq);
+    const int h = u % g.Hq;
     const int b = uu & 1, par = (uu >> 1) & 1;
     const int row = it.row0 + r;
     const bool row_valid = r < it.nrows;
@@ -1218,9 +1288,8 @@ __device__ void merge_rows(const Cta& c, const TcMaps& maps, const Geometry& g, 
     mbar_arrive(c.bar(BAR_O_FREE + b));
     const size_t orow = (size_t)row * g.Hq + h;
     if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_new + log2f(l_new)) * LN2;
-    const bool full_tile = it.nrows == BM;
-    if (!full_tile && row_valid) {
-      // a tile clipped by the block or the sequence end: rows go out one by one
+    if (row_valid && r >= (it.nrows & ~7)) {
+      // the last nrows % 8 rows of a clipped tile go out one by one (the rest by bulk stores)
       float4* dst = reinterpret_cast<float4*>(a.out + orow * D + 64 * half);
 #pragma unroll
       for (int q2 = 0; q2 < 2; ++q2)
@@ -1231,9 +1300,7 @@ __device__ void merge_rows(const Cta& c, const TcMaps& maps, const Geometry& g, 
     fence_async_smem();
     if (!epi_sync(c, epi_phase)) return;  // the whole tile is in the staging buffer
     if (threadIdx.x == 64) {
-      if (full_tile) {
-#pragma unroll
-        for (int cb = 0; cb < 4; ++cb) tma_store_3d(&maps.out, c.base + SM_IO + cb * IO_BOX, 32 * cb, h, it.row0);
+      if (store_out_tile(maps, c.base + SM_IO, h, it.row0, it.nrows) > 0) {
         bulk_commit();
         bulk_wait_read();               // the copies have read the staging tile
       }
@@ -1315,10 +1382,7 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
     if (vu < n_my && mbar_test(c.bar(BAR_KV_FREE1), (vu - 1) & 1)) { load_v(vu); ++vu; did = true; }
     if (mbar_test(c.bar((su & 1) ? BAR_OUT_RDY1 : BAR_OUT_RDY), (su >> 1) & 1)) {
       const DUnit un = deep_unit(c, su);
-      if (un.nrows == BM) {  // clipped tiles were written row by row by the row threads
-        const uint32_t src = c.base + DM_IO + (su & 1) * DM_IO_TILE;
-#pragma unroll
-        for (int cb = 0; cb < 4; ++cb) tma_store_3d(&maps.out, src + cb * IO_BOX, 32 * cb, un.h, un.row0);
+      if (store_out_tile(maps, c.base + DM_IO + (su & 1) * DM_IO_TILE, un.h, un.row0, un.nrows) > 0) {
         bulk_commit();
         pending_read = true;
       }
@@ -1475,8 +1539,8 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
     mbar_arrive(c.bar(BAR_O_FREE + b));
     const size_t orow = (size_t)row * g.Hq + un.h;
     if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_new + log2f(l_new)) * LN2;
-    if (un.nrows != BM && row_valid) {
-      // a tile clipped by the block or the sequence end: rows go out one by one
+    if (row_valid && r >= (un.nrows & ~7)) {
+      // the last nrows % 8 rows of a clipped tile go out one by one (the rest by bulk stores)
       float4* dst = reinterpret_cast<float4*>(a.out + orow * D + 64 * half);
 #pragma unroll
       for (int q2 = 0; q2 < 2; ++q2)
@@ -1506,6 +1570,15 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   // merge-role CTAs take the low block indices: they are scheduled first and have
   // loads to issue that do not depend on the preceding RoPE kernel
   const int n_ctas_merge = (int)gridDim.x - a.n_ctas_stream;
+#ifdef LACACHE_STREAM_FIRST
+  const bool stream = (int)blockIdx.x < a.n_ctas_stream;
+  int first, stride, n_units;
+  if (stream) {
+    first = blockIdx.x; stride = a.n_ctas_stream; n_units = a.n_items * g.Hq;
+  } else {
+    first = blockIdx.x - a.n_ctas_stream; stride = n_ctas_merge; n_units = a.n_items_merge * g.Hq;
+  }
+#else
   const bool stream = (int)blockIdx.x >= n_ctas_merge;
   int first, stride, n_units;
   if (stream) {
@@ -1513,6 +1586,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   } else {
     first = blockIdx.x; stride = n_ctas_merge; n_units = a.n_items_merge * g.Hq;
   }
+#endif
   const bool deep = !stream && a.merge_deep != 0;
   if (tid == 0) {  // descriptor fetches overlap the set-up below
     if (stream) {
@@ -1526,7 +1600,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   const int n_my = first < n_units ? (n_units - first + stride - 1) / stride : 0;
   WorkItem it0{};
   if (!deep && first < n_units) it0 = stream ? load_item(a.items + first % a.n_items)
-                                             : load_item(a.items_merge + first % a.n_items_merge);
+                                             : load_item(a.items_merge + first / g.Hq);
   if ((c.base & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = LOC_SMEM_ALIGN;
     return;
@@ -1535,7 +1609,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     for (int i = 0; i < N_BARS; ++i) {
       uint32_t count = 1;
       if (i == BAR_P_FULL || i == BAR_P_FULL1 || i == BAR_O_FREE || i == BAR_O_FREE1 || i == BAR_EPI ||
-          i == BAR_OUT_RDY || i == BAR_OUT_RDY1)
+          i == BAR_OUT_RDY || i == BAR_OUT_RDY1 || i == BAR_QC)
         count = ROW_THREADS;
       if (i == BAR_DONE) count = THREADS;
       if (i == BAR_Q_FREE && stream) count = 2;  // score MMAs done + epilogue staging read
@@ -1551,8 +1625,10 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     // this CTA's units, read by every role from shared memory
     for (int i = tid; i < n_my; i += THREADS) {
       const int u = first + i * stride;
-      const WorkItem w = load_item(a.items_merge + u % a.n_items_merge);
-      *reinterpret_cast<int4*>(smem_raw + DM_TAB + 16 * i) = make_int4(w.row0, w.nrows, w.blk_start, u / a.n_items_merge);
+      // units are head-minor (unit u = row tile u / Hq of head u % Hq): a CTA's units, a
+      // fixed stride apart, then cycle through the row tiles, clipped ones included
+      const WorkItem w = load_item(a.items_merge + u / g.Hq);
+      *reinterpret_cast<int4*>(smem_raw + DM_TAB + 16 * i) = make_int4(w.row0, w.nrows, w.blk_start, u % g.Hq);
     }
   }
   __syncwarp();
@@ -1679,6 +1755,8 @@ cudaError_t tc_prepare() {
 bool tc_set_out(TcMaps* m, const Geometry& g, float* out, char* err, int errlen) {
   if (m->out_ptr == out) return true;
   if (!make_f32_map(&m->out, out, (cuuint64_t)g.Hq, (cuuint64_t)g.T, 1, BM, err, errlen)) return false;
+  for (int i = 0; i < 4; ++i)
+    if (!make_f32_map(&m->out_sub[i], out, (cuuint64_t)g.Hq, (cuuint64_t)g.T, 1, 64u >> i, err, errlen)) return false;
   m->out_ptr = out;
   return true;
 }
