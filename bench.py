@@ -7,10 +7,12 @@ A "step" is one denoising step of the block schedule: `lacache_step` (RoPE-on-
 write of the block, fixed queries x block keys merged with the cached state,
 block queries x all keys); the first step of every block is preceded by that
 block's `lacache_build`, which is inside the timed region.  The headline value
-is denoising steps/s with every timed call starting from a flushed L2 (in a
-real model 31 other layers run between two calls of this one); a warm-L2 figure
-from one CUDA-graph replay of the same calls is reported beside it, and `e2e`
-times the same schedule through the host-buffer entry points.
+is denoising steps/s over K calls issued back to back on several replicas of
+the cache state visited round-robin, so that every call finds its inputs in
+HBM rather than in L2 (inputs larger than L2; in a real model 31 other layers
+run between two calls of this one).  Beside it: the old per-call figure with a
+flushed L2, a warm-L2 figure from one CUDA-graph replay on one replica, and
+`e2e`, the same schedule through the host-buffer entry points.
 
 With N > 1 (one process per GPU under torchrun) every rank runs its own seeded
 batch of the same workload: the path has no exchange step, so there is no
@@ -84,13 +86,14 @@ class ClockSampler:
     def __init__(self, index):
         self.index = index
         self.samples = []
+        self.window = []
         self.proc = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
-                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "5"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -98,7 +101,11 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.samples.append(line.strip())
+            self.samples.append((time.perf_counter(), line.strip()))
+
+    def mark(self):
+        """Start (first call) / end (second call) of the window whose samples count."""
+        self.window.append(time.perf_counter())
 
     def stop(self):
         if not self.proc:
@@ -110,7 +117,11 @@ class ClockSampler:
             pass
         sm, mx, reasons = [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for s in self.samples:
+        lo, hi = (self.window + [None, None])[:2]
+        inside = [l for t, l in self.samples if (lo is None or t >= lo) and (hi is None or t <= hi + 0.01)]
+        if len(inside) < 3:      # a very short window: fall back to every sample taken
+            inside = [l for _, l in self.samples]
+        for s in inside:
             f = [x.strip() for x in s.split(",")]
             if len(f) < 6:
                 continue
@@ -212,6 +223,17 @@ class DeviceSchedule:
 # ----------------------------------------------------------------------------
 # the CUDA arm
 # ----------------------------------------------------------------------------
+L2_BYTES = 126 << 20
+
+
+def n_replicas(step_bytes):
+    """Cache states visited round-robin so that a state's lines have left the L2
+    before it is touched again: the other replicas' steps move at least twice
+    the L2 capacity in between."""
+    import math
+    return max(3, math.ceil(2.0 * L2_BYTES / max(step_bytes, 1)) + 1)
+
+
 def run_cuda(args):
     import torch
     from paper_2607_16339_b200 import binding
@@ -230,86 +252,117 @@ def run_cuda(args):
     S = wl.steps_per_block
     counts = flops_and_bytes(wl)
     peaks = load_peaks()
-
-    sched = DeviceSchedule(wl, rank_seed(args.seed, rank), dev, W + K)
-    ctx = binding.Context.from_workload(wl)
     T = wl.total_tokens
-    out = torch.empty(T, wl.n_q_heads, wl.head_dim, device=dev)
-    lse = torch.empty(T, wl.n_q_heads, device=dev)
-    flush = torch.empty(256 << 20, dtype=torch.int8, device=dev)   # 2x the 126 MB L2
     stream = torch.cuda.current_stream()
     mk = lambda: torch.cuda.Event(enable_timing=True)
 
-    # ---- cold-L2 timing: every call individually bracketed by events, L2 flushed before it ----
-    k_ev0, k_ev1 = mk(), mk()
-    k_ev0.record(); k_ev1.record()
+    # ---- replicas: independent cache states of the same workload, visited round-robin ----
+    # Every call then finds its inputs (cached state, rotated planes) in HBM, not in L2,
+    # while the calls run back to back as they do in a denoising loop.
+    R = args.replicas or n_replicas(counts["step_attn_bytes"])
+    stagger = max(1, S // R)                       # replica c starts c * stagger steps into its block
+    nk = min(K, 256)                               # calls of the per-kernel timing pass
+    local_steps = (R - 1) * stagger + (W + K + nk + R - 1) // R + 1
+    sched = DeviceSchedule(wl, rank_seed(args.seed, rank), dev, local_steps)
+    ctxs = [binding.Context.from_workload(wl) for _ in range(R)]
+    outs = [(torch.empty(T, wl.n_q_heads, wl.head_dim, device=dev), torch.empty(T, wl.n_q_heads, device=dev))
+            for _ in range(R)]
+    ctx = ctxs[0]
+
+    def call_of(i):
+        """Global call i -> (replica, block, step in block, block inputs)."""
+        c = i % R
+        blk, s, tens = sched.step_inputs(c * stagger + i // R)
+        return c, blk, s, tens
+
+    for c in range(R):   # every replica starts with a valid cache for the block it is in
+        blk = sched.step_inputs(c * stagger)[0]
+        ctxs[c].build(blk, *sched.full[blk])
+    torch.cuda.synchronize()
+
     launches = 0
-    step_pairs, build_pairs = [], []
-    kern_step_ms, kern_build_ms = [], []
-    clocks = ClockSampler(local_rank)
+    n_builds = 0
 
-    def run_range(lo, hi, timed):
-        nonlocal launches
+    def run_range(lo, hi, timed, events=None):
+        nonlocal launches, n_builds
         for i in range(lo, hi):
-            blk, s, (qb, kb, vb) = sched.step_inputs(i)
-            if s == 0:
-                fq, fk, fv = sched.full[blk]
-                flush.add_(1)
-                e0, e1 = mk(), mk()
-                e0.record(); ctx.build(blk, fq, fk, fv); e1.record()
+            c, blk, s, (qb, kb, vb) = call_of(i)
+            if s == 0 and i >= R:      # a replica's very first call had its build above
+                if events is not None:
+                    e = (mk(), mk()); e[0].record(); e[1].record()
+                    ctxs[c].set_timing_events(*e); events.append(("build", e))
+                ctxs[c].build(blk, *sched.full[blk])
                 if timed:
-                    build_pairs.append((e0, e1)); launches += ctx.last_launch_count
-            flush.add_(1)
-            e0, e1 = mk(), mk()
-            e0.record(); ctx.step(qb, kb, vb, out, lse); e1.record()
+                    launches += ctxs[c].last_launch_count; n_builds += 1
+            if events is not None:
+                e = (mk(), mk()); e[0].record(); e[1].record()
+                ctxs[c].set_timing_events(*e); events.append(("step", e))
+            ctxs[c].step(qb, kb, vb, *outs[c])
             if timed:
-                step_pairs.append((e0, e1)); launches += ctx.last_launch_count
+                launches += ctxs[c].last_launch_count
 
-    # warm-up starts at a block boundary so the cache is built before the first step
+    clocks = ClockSampler(local_rank)
     clocks.start()
+    time.sleep(0.05)   # let the sampler come up
+    # ---- headline: K calls back to back, builds included, one event pair around the region ----
     run_range(0, W, False)
-    if W % S != 0:   # make the timed region start with a valid cache for its block
-        blk = (W // S) % sched.n_blocks_used
-        ctx.build(blk, *sched.full[blk])
     torch.cuda.synchronize(); barrier()
+    clocks.mark()
     t_wall0 = time.perf_counter()
-    # the timed range re-enters mid-block if W % S != 0: builds happen only at s == 0
+    ev0, ev1 = mk(), mk()
+    ev0.record()
     run_range(W, W + K, True)
+    ev1.record()
     torch.cuda.synchronize(); barrier()
     t_wall = time.perf_counter() - t_wall0
-    step_ms = [a.elapsed_time(b) for a, b in step_pairs]
-    build_ms = [a.elapsed_time(b) for a, b in build_pairs]
-    cold_total_ms = sum(step_ms) + sum(build_ms)
+    total_ms = ev0.elapsed_time(ev1)
 
-    # ---- per-kernel durations of the attention kernels (events recorded inside the library) ----
-    ctx.set_timing_events(k_ev0, k_ev1)
-    for i in range(W, W + min(K, 64)):
-        blk, s, (qb, kb, vb) = sched.step_inputs(i)
-        if s == 0 or i == W:
-            flush.add_(1)
-            ctx.build(blk, *sched.full[blk]); torch.cuda.synchronize()
-            kern_build_ms.append(k_ev0.elapsed_time(k_ev1))
+    # ---- per-kernel durations of the attention kernels: the same calls again, with an event
+    # pair recorded inside the library around each attention kernel (no host sync in between) ----
+    events = []
+    run_range(W + K, W + K + nk, False, events)
+    torch.cuda.synchronize()
+    for c in range(R):
+        ctxs[c].set_timing_events(None, None)
+    kern_step_ms = [a.elapsed_time(b) for kind, (a, b) in events if kind == "step"]
+    kern_build_ms = [a.elapsed_time(b) for kind, (a, b) in events if kind == "build"]
+    if not kern_build_ms:     # no block boundary in the range: time one build on its own
+        e = (mk(), mk()); e[0].record(); e[1].record()
+        c, blk, s, _ = call_of(W + K + nk)
+        ctxs[c].set_timing_events(*e)
+        ctxs[c].build(blk, *sched.full[blk]); torch.cuda.synchronize()
+        ctxs[c].set_timing_events(None, None)
+        kern_build_ms.append(e[0].elapsed_time(e[1]))
+
+    # ---- for comparison: one replica, L2 flushed (256 MiB write) before every call, each call
+    # bracketed by its own events (the launch latency after the flush kernel is inside) ----
+    flush = torch.empty(256 << 20, dtype=torch.int8, device=dev)
+    blk0 = sched.step_inputs(0)[0]
+    ctx.build(blk0, *sched.full[blk0])
+    fl_pairs = []
+    for i in range(8 + min(K, 64)):
+        _, s, (qb, kb, vb) = sched.step_inputs(i % S)
         flush.add_(1)
-        ctx.step(qb, kb, vb, out, lse); torch.cuda.synchronize()
-        kern_step_ms.append(k_ev0.elapsed_time(k_ev1))
-    ctx.set_timing_events(None, None)
+        e = (mk(), mk())
+        e[0].record(); ctx.step(qb, kb, vb, *outs[0]); e[1].record()
+        if i >= 8:
+            fl_pairs.append(e)
+    torch.cuda.synchronize()
+    flush_step_ms = statistics.mean(a.elapsed_time(b) for a, b in fl_pairs)
+    del flush
+    clocks.mark()      # window: the headline region, the per-kernel pass and the flushed pass (GPU busy throughout)
     clock_info = clocks.stop()
 
-    # ---- warm-L2: the same K calls captured once in a CUDA graph and replayed ----
+    # ---- warm L2: the same replica stepped K times from one CUDA-graph replay ----
     warm_ms = None
     try:
-        blk0 = (W // S) % sched.n_blocks_used
-        ctx.build(blk0, *sched.full[blk0])
-        torch.cuda.synchronize()
         gs = torch.cuda.Stream()
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.stream(gs):
             with torch.cuda.graph(graph, stream=gs):
-                for i in range(W, W + K):
-                    blk, s, (qb, kb, vb) = sched.step_inputs(i)
-                    if s == 0:
-                        ctx.build(blk, *sched.full[blk], stream=gs)
-                    ctx.step(qb, kb, vb, out, lse, stream=gs)
+                for i in range(K):
+                    _, s, (qb, kb, vb) = sched.step_inputs(i % S)
+                    ctx.step(qb, kb, vb, *outs[0], stream=gs)
             for _ in range(3):
                 graph.replay()
             gs.synchronize()
@@ -327,27 +380,24 @@ def run_cuda(args):
     pin = lambda t: t.cpu().pin_memory()
     h_full = {}
     h_steps = []
-    for i in range(W, W + n_e2e):
+    for i in range(n_e2e):
         blk, s, tens = sched.step_inputs(i)
         if s == 0 and blk not in h_full:
             h_full[blk] = tuple(pin(t) for t in sched.full[blk])
         h_steps.append(tuple(pin(t) for t in tens))
-    blk_first = sched.step_inputs(W)[0]
-    if blk_first not in h_full:
-        h_full[blk_first] = tuple(pin(t) for t in sched.full[blk_first])
     out_h = torch.empty(T, wl.n_q_heads, wl.head_dim).pin_memory()
     lse_h = torch.empty(T, wl.n_q_heads).pin_memory()
-    ctx.build_host(blk_first, *h_full[blk_first])
+    ctx.build_host(0, *h_full[0])
     ctx.step_host(*h_steps[0], out_h, lse_h)     # allocates staging, warms the path
     torch.cuda.synchronize(); barrier()
     e0, e1 = mk(), mk()
     e0.record()
     n_builds_e2e = 0
-    for j, i in enumerate(range(W, W + n_e2e)):
+    for i in range(n_e2e):
         blk, s, _ = sched.step_inputs(i)
         if s == 0:
             ctx.build_host(blk, *h_full[blk]); n_builds_e2e += 1
-        ctx.step_host(*h_steps[j], out_h, lse_h)
+        ctx.step_host(*h_steps[i], out_h, lse_h)
     e1.record()
     torch.cuda.synchronize(); barrier()
     e2e_ms = e0.elapsed_time(e1)
@@ -357,21 +407,21 @@ def run_cuda(args):
     h2d = blk_in + full_in * n_builds_e2e / max(n_e2e, 1)
     d2h = T * wl.n_q_heads * wl.head_dim * 4 + T * wl.n_q_heads * 4
 
-    st, msg = ctx.poll_status()
-    if st != 0:
-        raise SystemExit("device status: %s" % msg)
+    for c in range(R):
+        st, msg = ctxs[c].poll_status()
+        if st != 0:
+            raise SystemExit("device status: %s" % msg)
 
     # ---- reduce over ranks (timing only) ----
-    cold_total_ms = reduce_max(cold_total_ms, dev)
+    total_ms = reduce_max(total_ms, dev)
     e2e_ms = reduce_max(e2e_ms, dev)
     if warm_ms is not None:
         warm_ms = reduce_max(warm_ms, dev)
-    value = world * K / (cold_total_ms * 1e-3)
+    value = world * K / (total_ms * 1e-3)
 
     if rank == 0:
         step_k = statistics.mean(kern_step_ms) * 1e-3
         build_k = statistics.mean(kern_build_ms) * 1e-3 if kern_build_ms else None
-        n_builds = len(build_ms)
         total_flops = K * counts["step_flops"] + n_builds * counts["build_flops"]
         ach = counts["step_attn_bytes"] / step_k / 1e9
         roof = {"kernel": "tc_attn_kernel (step: fixed rows x block keys + merge, block rows x all keys)",
@@ -381,18 +431,24 @@ def run_cuda(args):
                 "algorithmic_bytes_per_launch": counts["step_attn_bytes"]}
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
-            "ms_per_step": round(cold_total_ms / K, 5), "higher_is_better": True, "scaling": "weak",
+            "ms_per_step": round(total_ms / K, 5), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": "cfg%d %s" % (wl.cfg, wl.name), "batch": wl.batch, "prompt_lens": list(wl.prompt_lens),
                        "gen_len": wl.gen_len, "block_len": wl.block_len, "steps_per_block": S,
                        "heads": "%d/%d" % (wl.n_q_heads, wl.n_kv_heads), "head_dim": wl.head_dim,
-                       "builds_in_timed_region": n_builds, "l2": "flushed before every timed call (256 MiB write)",
+                       "builds_in_timed_region": n_builds,
+                       "l2": "inputs larger than L2: %d replicas of the cache state visited round-robin "
+                             "(%.0f MB of algorithmic traffic between two visits of a replica, L2 is 126 MB), "
+                             "calls back to back, no flush" % (R, (R - 1) * counts["step_attn_bytes"] / 1e6),
+                       "replicas": R,
                        "out_dtype": "f32", "engine": "tcgen05" if ctx.engine == binding.ENGINE_TCGEN05 else "simt"},
-            "tflops": round(total_flops / (cold_total_ms * 1e-3) / 1e12, 2),
-            "step_us": {"mean": round(statistics.mean(step_ms) * 1e3, 2), "median": round(statistics.median(step_ms) * 1e3, 2)},
-            "build_us": {"mean": round(statistics.mean(build_ms) * 1e3, 2)} if build_ms else None,
+            "tflops": round(total_flops / (total_ms * 1e-3) / 1e12, 2),
+            "flushed_l2": {"value": round(world * 1e3 / flush_step_ms, 1), "unit": UNIT,
+                           "step_us": round(flush_step_ms * 1e3, 2),
+                           "how": "one replica, 256 MiB write before every call, each call bracketed by its own events"},
             "warm_l2": None if warm_ms is None else {
-                "value": round(world * K / (warm_ms * 1e-3), 1), "unit": UNIT, "how": "one CUDA-graph replay of the same K calls, no flush"},
+                "value": round(world * K / (warm_ms * 1e-3), 1), "unit": UNIT,
+                "how": "one replica stepped K times from one CUDA-graph replay"},
             "roofline": roof,
             "roofline_build": None if build_k is None else {
                 "kernel": "tc_attn_kernel (build: fixed rows x fixed keys -> cached state)", "bound": "tensor",
@@ -409,7 +465,8 @@ def run_cuda(args):
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(wl, budget_s=12.0)
         print(json.dumps(line), flush=True)
-    ctx.destroy()
+    for c in ctxs:
+        c.destroy()
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
@@ -509,12 +566,13 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--steps", type=int, default=1024)
     ap.add_argument("--warmup", type=int, default=32)
     ap.add_argument("--workload", type=int, default=2, help="config number 1..5 (2 = the headline LLaDA-8B shape)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--replicas", type=int, default=0, help="cache-state replicas visited round-robin (0 = sized from the L2)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
