@@ -559,6 +559,8 @@ lacache_status lacache_step(lacache_ctx* c, const void* q, const void* k, const 
   AttnArgs a = attn_args(c, MODE_STEP, c->step_list[blk], blk, c->rot, out, lse);
   if (!getenv("LACACHE_NO_QCOMP")) {
     a.q_raw = q;
+    a.k_raw = k;
+    a.v_raw = v;
     a.q_raw_bf16 = c->cfg.dtype == LACACHE_DTYPE_BF16 ? 1 : 0;
     a.row_cos = r.row_cos;
     a.row_sin = r.row_sin;

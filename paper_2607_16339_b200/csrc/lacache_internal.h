@@ -93,6 +93,9 @@ struct AttnArgs {
   // those tokens [B * block_len][d/2]; a CTA's first block-query unit rotates its Q tile
   // from these itself and so does not have to wait for the RoPE kernel
   const void* q_raw; int q_raw_bf16; const float* row_cos; const float* row_sin;
+  // likewise the block's pre-RoPE keys and values [B * block_len, Hkv, d]: the first unit of a
+  // pipelined merge-role CTA rotates the block's keys / converts its values itself
+  const void* k_raw; const void* v_raw;
   const int32_t* cu;         // [B+1]
   const int32_t* blk_start;  // [B] absolute token index of the block's first row
   RotBuffers rot;

@@ -32,16 +32,7 @@ __device__ __forceinline__ void store8_split(void* hi_plane, void* lo_plane, siz
 }
 
 __device__ __forceinline__ void store8_f16(void* plane, size_t off, const float (&y)[8]) {
-  uint4 u;
-  __half2* p = reinterpret_cast<__half2*>(&u);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    // saturate to the finite fp16 range
-    float a = fminf(fmaxf(y[2 * i], -65504.f), 65504.f);
-    float b = fminf(fmaxf(y[2 * i + 1], -65504.f), 65504.f);
-    p[i] = __floats2half2_rn(a, b);
-  }
-  *reinterpret_cast<uint4*>(reinterpret_cast<__half*>(plane) + off) = u;
+  *reinterpret_cast<uint4*>(reinterpret_cast<__half*>(plane) + off) = rope_half8(y);
 }
 
 // One thread: 8 features c0..c0+7 of the first half and their partners at

@@ -53,4 +53,17 @@ __device__ __forceinline__ void rope_split8(const float (&y)[8], uint4& hi, uint
   }
 }
 
+// 8 values as fp16, saturated to the finite fp16 range (the storage format of V)
+__device__ __forceinline__ uint4 rope_half8(const float (&y)[8]) {
+  uint4 u;
+  __half2* p = reinterpret_cast<__half2*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float a = fminf(fmaxf(y[2 * i], -65504.f), 65504.f);
+    float b = fminf(fmaxf(y[2 * i + 1], -65504.f), 65504.f);
+    p[i] = __floats2half2_rn(a, b);
+  }
+  return u;
+}
+
 }  // namespace lacache

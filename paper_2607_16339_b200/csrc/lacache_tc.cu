@@ -1330,13 +1330,13 @@ constexpr uint32_t DM_TAB = DM_V + 2 * DM_KBOX;        // unit table: {row0, nro
 constexpr int DM_MAX_UNITS = (int)((SM_XCH - DM_TAB) / 16);
 static_assert(DM_TAB % 16 == 0 && DM_MAX_UNITS >= TC_DEEP_MAX_UNITS, "unit table");
 
-struct DUnit { int row0, nrows, blk_start, h; };
+struct DUnit { int row0, nrows, blk_start, h, seq; };
 __device__ __forceinline__ DUnit deep_unit(const Cta& c, int i) {
   const int4 v = *reinterpret_cast<const int4*>(c.gen + DM_TAB + 16 * i);
-  return DUnit{v.x, v.y, v.z, v.w};
+  return DUnit{v.x, v.y, v.z, v.w & 0xFFFF, v.w >> 16};
 }
 
-__device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& g, int n_my) {
+__device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& g, int n_my, bool kv_computed) {
   if (n_my == 0) return;
   auto load_q = [&](int i) {
     const DUnit un = deep_unit(c, i);
@@ -1369,17 +1369,32 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
   load_q(0);
   load_io(0);
   if (n_my > 1) load_io(1);
-  grid_dependency_wait();
-  load_k(0);
-  load_v(0);
+  bool dep_done = false;
+  if (kv_computed) {
+    // the row threads rotate / convert the block's keys and values of the first unit
+    // from the raw inputs (plain arrivals keep the barriers' phase counts in step)
+    mbar_arrive(c.bar(BAR_KV_FULL));
+    mbar_arrive(c.bar(BAR_KV_FULL1));
+  } else {
+    grid_dependency_wait();
+    dep_done = true;
+    load_k(0);
+    load_v(0);
+  }
   int qu = 1, ku = 1, vu = 1, iu = 2, su = 0;
   bool pending_read = false;  // an output store may still be reading its staging tile
   long long t_idle = 0;
   while (su < n_my) {
     bool did = false;
     if (qu < n_my && mbar_test(c.bar(BAR_Q_FREE), (qu - 1) & 1)) { load_q(qu); ++qu; did = true; }
-    if (ku < n_my && mbar_test(c.bar(BAR_KV_FREE), (ku - 1) & 1)) { load_k(ku); ++ku; did = true; }
-    if (vu < n_my && mbar_test(c.bar(BAR_KV_FREE1), (vu - 1) & 1)) { load_v(vu); ++vu; did = true; }
+    if (ku < n_my && mbar_test(c.bar(BAR_KV_FREE), (ku - 1) & 1)) {
+      if (!dep_done) { grid_dependency_wait(); dep_done = true; }  // long over by now
+      load_k(ku); ++ku; did = true;
+    }
+    if (vu < n_my && mbar_test(c.bar(BAR_KV_FREE1), (vu - 1) & 1)) {
+      if (!dep_done) { grid_dependency_wait(); dep_done = true; }
+      load_v(vu); ++vu; did = true;
+    }
     if (mbar_test(c.bar((su & 1) ? BAR_OUT_RDY1 : BAR_OUT_RDY), (su >> 1) & 1)) {
       const DUnit un = deep_unit(c, su);
       if (store_out_tile(maps, c.base + DM_IO + (su & 1) * DM_IO_TILE, un.h, un.row0, un.nrows) > 0) {
@@ -1412,13 +1427,14 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
   bulk_wait_read();  // shared memory stays valid until the last store has read it
 }
 
-__device__ void deep_mma(const Cta& c, const Geometry& g, int n_my) {
+__device__ void deep_mma(const Cta& c, const Geometry& g, int n_my, bool kv_computed) {
   if (n_my == 0) return;
   const int n_s = (g.block_len + 15) & ~15;
   const uint32_t idesc_s = idesc_f16(1u, 0u, BM, (uint32_t)n_s);
   const uint32_t kb = c.base + DM_K;
   if (!wait_bar(c, BAR_Q_FULL, 0, LOC_WAIT_Q)) return;
   if (!wait_bar(c, BAR_KV_FULL, 0, LOC_WAIT_K)) return;
+  if (kv_computed && !wait_bar(c, BAR_QC, 0, LOC_WAIT_K)) return;  // keys and values written by the row threads
   tc_fence_after();
   issue_s_mma(c.base + SM_Q, BM * 128u, kb, kb + 2 * DM_KBOX, DM_KBOX, c.tmem + TM_S, idesc_s);
   tc_commit(c.bar(BAR_S_FULL));
@@ -1464,6 +1480,57 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
       m_nx = __ldg(a.st.m + srow);
       l_nx = __ldg(a.st.l + srow);
     }
+  }
+  if (n_my > 0 && a.k_raw != nullptr) {
+    // First unit: the block's keys (rotated, split bf16) and values (fp16) of this head,
+    // computed here with the RoPE kernel's own arithmetic and written where the TMA loads
+    // would have put them ([plane][feature half][row][64], 16-byte chunks XOR-swizzled by
+    // the row), so the unit does not wait for that kernel.
+    const DUnit un = deep_unit(c, 0);
+    const int kh = un.h / g.group;
+    const int tq = threadIdx.x - 64;
+    for (int i = tq; i < L * 8; i += ROW_THREADS) {
+      const int ki = i >> 3, ch = i & 7, c0 = ch * 8;
+      const size_t src = (size_t)un.seq * L + ki;
+      const size_t soff = (src * g.Hkv + kh) * D;
+      float x1[8], x2[8], cs[8], sn[8], y1[8], y2[8];
+      rope_load8(a.k_raw, soff + c0, a.q_raw_bf16 != 0, x1);
+      rope_load8(a.k_raw, soff + c0 + D / 2, a.q_raw_bf16 != 0, x2);
+      const float4* cp = reinterpret_cast<const float4*>(a.row_cos + src * (D / 2) + c0);
+      const float4* sp = reinterpret_cast<const float4*>(a.row_sin + src * (D / 2) + c0);
+      const float4 ca = cp[0], cb = cp[1], sa = sp[0], sb = sp[1];
+      cs[0] = ca.x; cs[1] = ca.y; cs[2] = ca.z; cs[3] = ca.w; cs[4] = cb.x; cs[5] = cb.y; cs[6] = cb.z; cs[7] = cb.w;
+      sn[0] = sa.x; sn[1] = sa.y; sn[2] = sa.z; sn[3] = sa.w; sn[4] = sb.x; sn[5] = sb.y; sn[6] = sb.z; sn[7] = sb.w;
+      rope_rotate8(x1, x2, cs, sn, y1, y2);
+      uint4 h1, l1, h2, l2;
+      rope_split8(y1, h1, l1);
+      rope_split8(y2, h2, l2);
+      uint8_t* const k0 = c.gen + DM_K + ki * 128 + ((ch ^ (ki & 7)) << 4);
+      *reinterpret_cast<uint4*>(k0) = h1;
+      *reinterpret_cast<uint4*>(k0 + DM_KBOX) = h2;
+      *reinterpret_cast<uint4*>(k0 + 2 * DM_KBOX) = l1;
+      *reinterpret_cast<uint4*>(k0 + 3 * DM_KBOX) = l2;
+      // values: the same two 8-feature chunks of row ki, unrotated
+      float v1[8], v2[8];
+      rope_load8(a.v_raw, soff + c0, a.q_raw_bf16 != 0, v1);
+      rope_load8(a.v_raw, soff + c0 + D / 2, a.q_raw_bf16 != 0, v2);
+      uint8_t* const v0 = c.gen + DM_V + ki * 128 + ((ch ^ (ki & 7)) << 4);
+      *reinterpret_cast<uint4*>(v0) = rope_half8(v1);
+      *reinterpret_cast<uint4*>(v0 + DM_KBOX) = rope_half8(v2);
+    }
+    // rows [L, 32) of the boxes (block_len < 32) are never multiplied by a non-zero P~
+    // but must not hold NaN or Inf patterns: clear them
+    for (int i = tq + L * 8; i < 32 * 8; i += ROW_THREADS) {
+      const int ki = i >> 3, ch = i & 7;
+      const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+      uint8_t* const k0 = c.gen + DM_K + ki * 128 + ((ch ^ (ki & 7)) << 4);
+      *reinterpret_cast<uint4*>(k0) = z; *reinterpret_cast<uint4*>(k0 + DM_KBOX) = z;
+      *reinterpret_cast<uint4*>(k0 + 2 * DM_KBOX) = z; *reinterpret_cast<uint4*>(k0 + 3 * DM_KBOX) = z;
+      uint8_t* const v0 = c.gen + DM_V + ki * 128 + ((ch ^ (ki & 7)) << 4);
+      *reinterpret_cast<uint4*>(v0) = z; *reinterpret_cast<uint4*>(v0 + DM_KBOX) = z;
+    }
+    fence_async_smem();  // the MMAs read shared memory through the async proxy
+    mbar_arrive(c.bar(BAR_QC));
   }
   for (int uu = 0; uu < n_my; ++uu) {
     const DUnit un = deep_unit(c, uu);
@@ -1567,10 +1634,9 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   c.status = a.status;
   // role and unit range of this CTA; the first work item is fetched before the
   // set-up below so its latency overlaps it
-  // merge-role CTAs take the low block indices: they are scheduled first and have
-  // loads to issue that do not depend on the preceding RoPE kernel
   const int n_ctas_merge = (int)gridDim.x - a.n_ctas_stream;
-#ifdef LACACHE_STREAM_FIRST
+  // stream-role CTAs take the low block indices (they are scheduled first: the block
+  // queries' chain of key tiles is the longest dependent chain of a step)
   const bool stream = (int)blockIdx.x < a.n_ctas_stream;
   int first, stride, n_units;
   if (stream) {
@@ -1578,15 +1644,6 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   } else {
     first = blockIdx.x - a.n_ctas_stream; stride = n_ctas_merge; n_units = a.n_items_merge * g.Hq;
   }
-#else
-  const bool stream = (int)blockIdx.x >= n_ctas_merge;
-  int first, stride, n_units;
-  if (stream) {
-    first = blockIdx.x - n_ctas_merge; stride = a.n_ctas_stream; n_units = a.n_items * g.Hq;
-  } else {
-    first = blockIdx.x; stride = n_ctas_merge; n_units = a.n_items_merge * g.Hq;
-  }
-#endif
   const bool deep = !stream && a.merge_deep != 0;
   if (tid == 0) {  // descriptor fetches overlap the set-up below
     if (stream) {
@@ -1628,7 +1685,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
       // units are head-minor (unit u = row tile u / Hq of head u % Hq): a CTA's units, a
       // fixed stride apart, then cycle through the row tiles, clipped ones included
       const WorkItem w = load_item(a.items_merge + u / g.Hq);
-      *reinterpret_cast<int4*>(smem_raw + DM_TAB + 16 * i) = make_int4(w.row0, w.nrows, w.blk_start, u % g.Hq);
+      *reinterpret_cast<int4*>(smem_raw + DM_TAB + 16 * i) = make_int4(w.row0, w.nrows, w.blk_start, (u % g.Hq) | (w.seq << 16));
     }
   }
   __syncwarp();
@@ -1647,14 +1704,14 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     if (stream) {
       if (tid == 0) stream_producer(c, maps, g, a, first, stride, n_units, it0);
     } else if (deep) {
-      if (tid == 0) deep_producer(c, maps, g, n_my);
+      if (tid == 0) deep_producer(c, maps, g, n_my, a.k_raw != nullptr);
     } else {
       if (tid == 0) merge_producer(c, maps, g, a, first, stride, n_units, it0);
     }
   } else if (warp == 1) {
     if (tid == 32) {
       if (stream) stream_mma(c, g, a, first, stride, n_units, it0);
-      else if (deep) deep_mma(c, g, n_my);
+      else if (deep) deep_mma(c, g, n_my, a.k_raw != nullptr);
       else merge_mma(c, g, a, first, stride, n_units);
     }
   } else {
