@@ -289,6 +289,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   cudaDeviceProp prop;
   CU_TRY(c, cudaGetDeviceProperties(&prop, c->device));
   c->num_sms = prop.multiProcessorCount;
+  if (const char* e = getenv("LACACHE_MAX_CTAS")) c->num_sms = std::max(1, std::min(c->num_sms, atoi(e)));  // experiments
   if (const char* e = getenv("LACACHE_STREAM_CTAS")) c->stream_ctas_override = atoi(e);
   if (tc && prop.major != 10)
     return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs an sm_100 device, found sm_%d%d", prop.major, prop.minor);
