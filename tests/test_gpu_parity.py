@@ -30,6 +30,8 @@ def _small_cases():
     c["oneblock"] = dict(prompt_lens=(131,), gen_len=32, block_len=32, steps=2, hq=2, hkv=2)
     # key outliers as in the long-generation config
     c["outliers"] = dict(prompt_lens=(300,), gen_len=64, block_len=32, steps=1, hq=4, hkv=4, outlier_frac=0.02)
+    # GQA with a 32-row block (pipelined merge role: the block's keys of a KV head serve its query heads)
+    c["gqa32"] = dict(prompt_lens=(150, 61), gen_len=64, block_len=32, steps=2, hq=8, hkv=2)
     # tiny block
     c["blk16"] = dict(prompt_lens=(50, 64), gen_len=48, block_len=16, steps=1, hq=2, hkv=2)
     return c
