@@ -134,7 +134,10 @@ void tc_free_maps(TcMaps* m);
 
 constexpr int SIMT_ROWS = 32;    // query rows per SIMT work item
 constexpr int TC_ROWS = 128;     // query rows per tcgen05 work item
-constexpr int TC_KEYS = 96;      // keys per tcgen05 key tile (stream role)
+#ifndef LACACHE_TC_KEYS
+#define LACACHE_TC_KEYS 96
+#endif
+constexpr int TC_KEYS = LACACHE_TC_KEYS;   // keys per tile of the tcgen05 stream role
 constexpr int TC_MAX_BLOCK = 64;
 constexpr int TC_DEEP_MAX_UNITS = 512;  // units per CTA the pipelined merge role can tabulate // largest block length the tcgen05 merge role handles
 

@@ -417,14 +417,9 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
   }
   return un;
 }
-__device__ __forceinline__ bool tile_skipped(const Unit& un, int t) {
-  int lo = un.key_base + t * BN, hi = min(lo + BN, un.k1);
-  return un.x1 > un.x0 && lo >= un.x0 && hi <= un.x1;
-}
-__device__ __forceinline__ int next_tile(const Unit& un, int t) {
-  while (t < un.t1 && tile_skipped(un, t)) ++t;
-  return t;
-}
+// (A key tile is wider than a block -- BN > TC_MAX_BLOCK -- so no tile lies wholly inside the keys a
+// build excludes: every tile in [t0, t1) is processed, excluded columns are masked by the row threads.)
+static_assert(BN > TC_MAX_BLOCK, "a key tile could fall wholly inside the excluded block");
 
 // S (+)= Q' K'^T as hi.hi + hi.lo + lo.hi; Q planes at q_base (lo plane after the hi
 // plane's two boxes) with boxes of q_box bytes, K planes at k_hi / k_lo with boxes of
@@ -490,14 +485,14 @@ __device__ __forceinline__ void cursor_load_unit(const Geometry& g, const AttnAr
   if (!cu.valid) return;
   cu.it = load_item(a.items + cu.u % a.n_items);
   cu.un = decode_stream(g, a, cu.it, cu.u);
-  cu.t = next_tile(cu.un, cu.un.t0);
+  cu.t = cu.un.t0;
   cu.q_done = !cu.loads_q;
 }
 __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs& a, TileCursor& cu, int stride,
                                                int n_units) {
   // move to the next tile; cross into the next unit(s) when this one is exhausted
   if (cu.t < cu.un.t1) {
-    cu.t = next_tile(cu.un, cu.t + 1);
+    ++cu.t;
     ++cu.jj;
   }
   while (cu.valid && cu.t >= cu.un.t1 && cu.q_done) {
@@ -601,81 +596,56 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
   // (a CTA without units never touches memory the RoPE kernel writes)
 }
 
-// The MMA thread issues whichever product is ready: P~V of the oldest pending
-// tile as soon as its probabilities are in TMEM and its values have landed,
-// else the scores of the next tile as soon as its keys have landed (at most two
-// score tiles in flight).  O~ accumulates in TMEM across the tiles of a unit.
+// The MMA thread runs a fixed software pipeline with blocking (bounded) waits: the scores of the
+// unit's first two tiles, then per tile j: P~V of tile j (its probabilities are in TMEM, its values have
+// landed), then the scores of tile j + 2 (its keys have landed; the score buffer it overwrites was read
+// for tile j, whose probabilities have just been waited for).  A single thread's scalar code runs at a
+// few tens of instructions per 100 ns, so the loop carries no polling and no per-tile bookkeeping beyond
+// the stage toggles.  O~ accumulates in TMEM across the tiles of a unit.
 __device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units,
                            WorkItem it) {
   constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
-  int uu = 0, js = 0, jp = 0;  // global counters of score tiles / PV tiles issued
+  int uu = 0;
+  uint32_t js = 0, jp = 0;  // score tiles / P~V tiles issued so far (stage = j & 1, phase = (j >> 1) & 1)
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
     const Unit un = decode_stream(g, a, it, u);
     const uint32_t q_box = (uint32_t)un.q_rows * 128u;
+    const int n_tiles = un.t1 - un.t0;
     if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
     if (uu == 0 && a.mode == MODE_STEP && a.q_raw != nullptr && !wait_bar(c, BAR_QC, 0, LOC_WAIT_Q)) return;
-    int ts = next_tile(un, un.t0), tp = ts;
-    bool q_released = false, first_pv = true;
-    bool o_free_pending = uu >= 1;  // O_FREE of the previous unit is observed exactly once, in order
-    long long t_idle = 0;
-    while (tp < un.t1) {
-      bool did = false;
-      if (js > jp) {  // scores of tile jp issued: its P~V may be ready
-        const int b = jp & 1;
-        const int sv = jp & 1;
-        if (mbar_test(c.bar(BAR_P_FULL + b), (jp >> 1) & 1) &&
-            mbar_test(c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), (jp >> 1) & 1)) {
-          if (o_free_pending) {  // the row threads have read the previous unit's O~
-            if (!wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
-            o_free_pending = false;
-          }
-          tc_fence_after();
-          issue_pv_mma(c.base + SM_V + sv * V_STAGE, KS_BOX, c.tmem + TS_P + 64 * b, c.tmem + TS_O, BN / 16,
-                       first_pv ? 0u : 1u);
-          tc_commit(c.bar(BAR_O_FULL));
-          tc_commit(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE));
-          first_pv = false;
-          tp = next_tile(un, tp + 1);
-          ++jp;
-          did = true;
-        }
-      }
-      if (!did && ts < un.t1 && js - jp < 2) {
-        const int sk = js & 1, kuse = js >> 1;
-        if (mbar_test(c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL), kuse & 1)) {
-          const int b = js & 1;
-          const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
-          tc_fence_after();
-          issue_s_mma(c.base + SM_Q, q_box, khi, klo, KS_BOX, c.tmem + TS_S + 128 * b, IDESC_S);
-          tc_commit(c.bar(BAR_S_FULL + b));
-          tc_commit(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE));
-          ts = next_tile(un, ts + 1);
-          ++js;
-          if (ts >= un.t1) {  // every score MMA of this unit has been issued
-            tc_commit(c.bar(BAR_Q_FREE));
-            q_released = true;
-          }
-          did = true;
-        }
-      }
-      if (did) {
-        t_idle = 0;
-      } else {  // nothing ready: bounded idle
-        if (t_idle == 0) t_idle = clock64();
-        if (*c.abort_flag) return;
-        if (clock64() - t_idle > WAIT_CYCLES) {
-          *c.abort_flag = 1;
-          if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
-            c.status[1] = LOC_WAIT_S; c.status[2] = blockIdx.x; c.status[3] = threadIdx.x;
-          }
-          return;
-        }
+    if (n_tiles == 0) tc_commit(c.bar(BAR_Q_FREE));  // a unit without key tiles
+    // issue order S0, S1, PV0, S2, PV1, S3, ...; one copy of each code block (the unrolled
+    // MMA sequences are large, and cold instruction fetches are slow)
+    int n_s = 0, n_pv = 0;
+    while (n_pv < n_tiles) {
+      if (n_s < n_tiles && n_s < n_pv + 2) {
+        const uint32_t sk = js & 1u, b = js & 1u;
+        if (!wait_bar(c, sk ? BAR_K_FULL1 : BAR_K_FULL, (js >> 1) & 1u, LOC_WAIT_K)) return;
+        const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
+        tc_fence_after();
+        issue_s_mma(c.base + SM_Q, q_box, khi, klo, KS_BOX, c.tmem + TS_S + 128 * b, IDESC_S);
+        tc_commit(c.bar(BAR_S_FULL + b));
+        tc_commit(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE));
+        ++js;
+        if (++n_s == n_tiles) tc_commit(c.bar(BAR_Q_FREE));  // every score MMA of this unit has been issued
+      } else {
+        const uint32_t b = jp & 1u, sv = jp & 1u, ph = (jp >> 1) & 1u;
+        if (!wait_bar(c, BAR_P_FULL + b, ph, LOC_WAIT_S)) return;
+        if (!wait_bar(c, sv ? BAR_V_FULL1 : BAR_V_FULL, ph, LOC_WAIT_V)) return;
+        if (n_pv == 0 && uu >= 1 && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;  // O~ of the previous unit was read
+        tc_fence_after();
+        issue_pv_mma(c.base + SM_V + sv * V_STAGE, KS_BOX, c.tmem + TS_P + 64 * b, c.tmem + TS_O, BN / 16,
+                     n_pv == 0 ? 0u : 1u);
+        tc_commit(c.bar(BAR_O_FULL));
+        tc_commit(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE));
+        ++jp;
+        ++n_pv;
       }
     }
-    if (!q_released) tc_commit(c.bar(BAR_Q_FREE));  // a unit without key tiles
-    if (o_free_pending && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
+    // (a unit without key tiles still consumes O_FREE of its predecessor in order)
+    if (n_tiles == 0 && uu >= 1 && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
     it = nxt;
   }
 }
@@ -862,7 +832,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     float m_ref = -INFINITY, l_part = 0.f;
     bool first_tile = true;
 
-    for (int t = next_tile(un, un.t0); t < un.t1; t = next_tile(un, t + 1), ++jj) {
+    for (int t = un.t0; t < un.t1; ++t, ++jj) {
       const int b = jj & 1;
       if (!wait_bar(c, BAR_S_FULL + b, (jj >> 1) & 1, LOC_WAIT_S)) return;
       tc_fence_after();
