@@ -70,7 +70,8 @@ static_assert(BN % 32 == 0 && BN <= 128, "tile width");
 constexpr float RESCALE_SLACK = 3.f;
 constexpr int ROW_WARPS = 8;
 constexpr int ROW_THREADS = ROW_WARPS * 32;
-constexpr int THREADS = 64 + ROW_THREADS;
+constexpr int THREADS = 64 + ROW_THREADS + 32;   // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: row threads,
+                                                  // warp 10: second MMA issuer (P~V products of the stream role)
 
 // ---- shared memory map (bytes from a 1024-aligned base) ----
 constexpr uint32_t SM_Q = 0;                      // Q hi plane (two boxes), then the lo plane
@@ -596,17 +597,18 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
   // (a CTA without units never touches memory the RoPE kernel writes)
 }
 
-// The MMA thread runs a fixed software pipeline with blocking (bounded) waits: the scores of the
-// unit's first two tiles, then per tile j: P~V of tile j (its probabilities are in TMEM, its values have
-// landed), then the scores of tile j + 2 (its keys have landed; the score buffer it overwrites was read
-// for tile j, whose probabilities have just been waited for).  A single thread's scalar code runs at a
-// few tens of instructions per 100 ns, so the loop carries no polling and no per-tile bookkeeping beyond
-// the stage toggles.  O~ accumulates in TMEM across the tiles of a unit.
-__device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units,
-                           WorkItem it) {
+// Two threads issue the stream role's MMAs, each a fixed pipeline with blocking (bounded) waits: one
+// the score products, the other the P~V products.  tcgen05.mma accepts the next instruction only when the
+// tensor pipe has room, so a single issuer leaves the pipe idle while it runs the scalar code between two
+// batches (barrier waits, commits); with two issuers one thread's bookkeeping overlaps the other's MMAs.
+// Scores of tile j need its keys and the score buffer of tile j - 2 read (= the probabilities of tile
+// j - 2 written); P~V of tile j needs its probabilities and its values.  Each code block exists once
+// (the unrolled MMA sequences are large, and cold instruction fetches are slow).
+__device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
+                                  int n_units, WorkItem it) {
   constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
   int uu = 0;
-  uint32_t js = 0, jp = 0;  // score tiles / P~V tiles issued so far (stage = j & 1, phase = (j >> 1) & 1)
+  uint32_t js = 0;  // score tiles issued so far (stage and buffer = js & 1, phase = (js >> 1) & 1)
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
@@ -615,37 +617,44 @@ __device__ void stream_mma(const Cta& c, const Geometry& g, const AttnArgs& a, i
     const int n_tiles = un.t1 - un.t0;
     if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
     if (uu == 0 && a.mode == MODE_STEP && a.q_raw != nullptr && !wait_bar(c, BAR_QC, 0, LOC_WAIT_Q)) return;
-    if (n_tiles == 0) tc_commit(c.bar(BAR_Q_FREE));  // a unit without key tiles
-    // issue order S0, S1, PV0, S2, PV1, S3, ...; one copy of each code block (the unrolled
-    // MMA sequences are large, and cold instruction fetches are slow)
-    int n_s = 0, n_pv = 0;
-    while (n_pv < n_tiles) {
-      if (n_s < n_tiles && n_s < n_pv + 2) {
-        const uint32_t sk = js & 1u, b = js & 1u;
-        if (!wait_bar(c, sk ? BAR_K_FULL1 : BAR_K_FULL, (js >> 1) & 1u, LOC_WAIT_K)) return;
-        const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
-        tc_fence_after();
-        issue_s_mma(c.base + SM_Q, q_box, khi, klo, KS_BOX, c.tmem + TS_S + 128 * b, IDESC_S);
-        tc_commit(c.bar(BAR_S_FULL + b));
-        tc_commit(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE));
-        ++js;
-        if (++n_s == n_tiles) tc_commit(c.bar(BAR_Q_FREE));  // every score MMA of this unit has been issued
-      } else {
-        const uint32_t b = jp & 1u, sv = jp & 1u, ph = (jp >> 1) & 1u;
-        if (!wait_bar(c, BAR_P_FULL + b, ph, LOC_WAIT_S)) return;
-        if (!wait_bar(c, sv ? BAR_V_FULL1 : BAR_V_FULL, ph, LOC_WAIT_V)) return;
-        if (n_pv == 0 && uu >= 1 && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;  // O~ of the previous unit was read
-        tc_fence_after();
-        issue_pv_mma(c.base + SM_V + sv * V_STAGE, KS_BOX, c.tmem + TS_P + 64 * b, c.tmem + TS_O, BN / 16,
-                     n_pv == 0 ? 0u : 1u);
-        tc_commit(c.bar(BAR_O_FULL));
-        tc_commit(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE));
-        ++jp;
-        ++n_pv;
-      }
+    for (int j = 0; j < n_tiles; ++j, ++js) {
+      const uint32_t sk = js & 1u, b = js & 1u;
+      // the score buffer was last used two tiles ago (possibly by the previous unit): its
+      // probabilities have been written, so its scores have been read
+      if (js >= 2 && !wait_bar(c, BAR_P_FULL + b, ((js - 2) >> 1) & 1u, LOC_WAIT_S)) return;
+      if (!wait_bar(c, sk ? BAR_K_FULL1 : BAR_K_FULL, (js >> 1) & 1u, LOC_WAIT_K)) return;
+      const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
+      tc_fence_after();
+      issue_s_mma(c.base + SM_Q, q_box, khi, klo, KS_BOX, c.tmem + TS_S + 128 * b, IDESC_S);
+      tc_commit(c.bar(BAR_S_FULL + b));
+      tc_commit(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE));
     }
-    // (a unit without key tiles still consumes O_FREE of its predecessor in order)
-    if (n_tiles == 0 && uu >= 1 && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
+    tc_commit(c.bar(BAR_Q_FREE));  // every score MMA of this unit has been issued (or it had no key tiles)
+    it = nxt;
+  }
+}
+
+__device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
+                              int n_units, WorkItem it) {
+  int uu = 0;
+  uint32_t jp = 0;  // P~V tiles issued so far
+  for (int u = first; u < n_units; u += stride, ++uu) {
+    WorkItem nxt = it;
+    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
+    const Unit un = decode_stream(g, a, it, u);
+    const int n_tiles = un.t1 - un.t0;
+    // O~ of the previous unit has been read by the row threads (observed once per unit, in order)
+    if (uu >= 1 && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
+    for (int j = 0; j < n_tiles; ++j, ++jp) {
+      const uint32_t b = jp & 1u, sv = jp & 1u, ph = (jp >> 1) & 1u;
+      if (!wait_bar(c, BAR_P_FULL + b, ph, LOC_WAIT_S)) return;
+      if (!wait_bar(c, sv ? BAR_V_FULL1 : BAR_V_FULL, ph, LOC_WAIT_V)) return;
+      tc_fence_after();
+      issue_pv_mma(c.base + SM_V + sv * V_STAGE, KS_BOX, c.tmem + TS_P + 64 * b, c.tmem + TS_O, BN / 16,
+                   j == 0 ? 0u : 1u);
+      tc_commit(c.bar(BAR_O_FULL));
+      tc_commit(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE));
+    }
     it = nxt;
   }
 }
@@ -1680,10 +1689,12 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     }
   } else if (warp == 1) {
     if (tid == 32) {
-      if (stream) stream_mma(c, g, a, first, stride, n_units, it0);
+      if (stream) stream_mma_scores(c, g, a, first, stride, n_units, it0);
       else if (deep) deep_mma(c, g, n_my, a.k_raw != nullptr);
       else merge_mma(c, g, a, first, stride, n_units);
     }
+  } else if (warp == 10) {
+    if (tid == 320 && stream) stream_mma_pv(c, g, a, first, stride, n_units, it0);
   } else {
     if (stream) stream_rows(c, g, a, first, stride, n_units, it0);
     else if (deep) deep_rows(c, g, a, n_my);
