@@ -477,7 +477,7 @@ def run_cuda(args):
 # (profiles/tc_attn_kernel_cfg2_ncu_full.txt), bytes; None where no capture
 # exists for the workload.  The fp32 output (12.6 MB) is still in L2 when the
 # kernel ends, so the figure is dominated by reads.
-TRAFFIC_PER_LAUNCH = {2: 45104000}
+TRAFFIC_PER_LAUNCH = {2: 45356544}
 
 
 # ----------------------------------------------------------------------------
