@@ -70,8 +70,8 @@ static_assert(BN % 32 == 0 && BN <= 128, "tile width");
 constexpr float RESCALE_SLACK = 3.f;
 constexpr int ROW_WARPS = 8;
 constexpr int ROW_THREADS = ROW_WARPS * 32;
-constexpr int THREADS = 64 + ROW_THREADS + 64;   // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: row threads,
-                                                  // warps 10, 11: further MMA issuers of the stream role
+constexpr int THREADS = 64 + ROW_THREADS + 32;   // warp 0: TMA producer, warp 1: MMA issuer, warps 2-9: row threads,
+                                                  // warp 10: second MMA issuer (P~V products of the stream role)
 
 // ---- shared memory map (bytes from a 1024-aligned base) ----
 constexpr uint32_t SM_Q = 0;                      // Q hi plane (two boxes), then the lo plane
@@ -371,10 +371,6 @@ __device__ __noinline__ bool wait_slow(const Cta& c, uint32_t bar, uint32_t pari
     }
   }
 }
-__device__ __forceinline__ bool wait_slow_or_fast(const Cta& c, uint32_t b, uint32_t parity, int loc) {
-  if (mbar_try(b, parity)) return true;
-  return wait_slow(c, b, parity, loc);
-}
 __device__ __forceinline__ bool wait_bar(const Cta& c, int slot, uint32_t parity, int loc) {
   uint32_t b = c.bar(slot);
   if (mbar_try(b, parity)) return true;
@@ -609,37 +605,31 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
 // j - 2 written); P~V of tile j needs its probabilities and its values.  Each code block exists once
 // (the unrolled MMA sequences are large, and cold instruction fetches are slow).
 __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
-                                  int n_units, WorkItem it, uint32_t parity) {
-  // One of two score issuers: this one issues the tiles whose global ordinal has the given parity, i.e.
-  // it owns key stage `parity` and score buffer `parity`.  A lone thread issues an MMA every ~65 cycles
-  // (scalar work per instruction) while the tensor pipe needs ~48 for N = 96: two issuers keep it fed,
-  // and every tile's products still come from one thread in a fixed order (bit-reproducible sums).
+                                  int n_units, WorkItem it) {
   constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
-  const uint32_t b = parity;
-  const uint32_t khi = c.base + SM_K + b * K_STAGE, klo = khi + SK_LO;
-  const uint32_t bar_kfull = c.bar(b ? BAR_K_FULL1 : BAR_K_FULL), bar_kfree = c.bar(b ? BAR_K_FREE1 : BAR_K_FREE);
   int uu = 0;
-  uint32_t js0 = 0;  // global ordinal of the unit's first tile
+  uint32_t js = 0;  // score tiles issued so far (stage and buffer = js & 1, phase = (js >> 1) & 1)
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
     const Unit un = decode_stream(g, a, it, u);
     const uint32_t q_box = (uint32_t)un.q_rows * 128u;
-    const uint32_t n_tiles = (uint32_t)(un.t1 - un.t0);
+    const int n_tiles = un.t1 - un.t0;
     if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
     if (uu == 0 && a.mode == MODE_STEP && a.q_raw != nullptr && !wait_bar(c, BAR_QC, 0, LOC_WAIT_Q)) return;
-    for (uint32_t js = js0 + ((js0 ^ parity) & 1u); js < js0 + n_tiles; js += 2) {
+    for (int j = 0; j < n_tiles; ++j, ++js) {
+      const uint32_t sk = js & 1u, b = js & 1u;
       // the score buffer was last used two tiles ago (possibly by the previous unit): its
       // probabilities have been written, so its scores have been read
       if (js >= 2 && !wait_bar(c, BAR_P_FULL + b, ((js - 2) >> 1) & 1u, LOC_WAIT_S)) return;
-      if (!wait_slow_or_fast(c, bar_kfull, (js >> 1) & 1u, LOC_WAIT_K)) return;
+      if (!wait_bar(c, sk ? BAR_K_FULL1 : BAR_K_FULL, (js >> 1) & 1u, LOC_WAIT_K)) return;
+      const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
       tc_fence_after();
       issue_s_mma(c.base + SM_Q, q_box, khi, klo, KS_BOX, c.tmem + TS_S + 128 * b, IDESC_S);
       tc_commit(c.bar(BAR_S_FULL + b));
-      tc_commit(bar_kfree);
+      tc_commit(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE));
     }
-    js0 += n_tiles;
-    tc_commit(c.bar(BAR_Q_FREE));  // this issuer's score MMAs of the unit have been issued (count 2: both issuers)
+    tc_commit(c.bar(BAR_Q_FREE));  // every score MMA of this unit has been issued (or it had no key tiles)
     it = nxt;
   }
 }
@@ -1658,7 +1648,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
           i == BAR_OUT_RDY || i == BAR_OUT_RDY1 || i == BAR_QC)
         count = ROW_THREADS;
       if (i == BAR_DONE) count = THREADS;
-      if (i == BAR_Q_FREE && stream) count = 3;  // score MMAs of both issuers done + epilogue staging read
+      if (i == BAR_Q_FREE && stream) count = 2;  // score MMAs done + epilogue staging read
       if (i >= BAR_PAIR) count = 64;
       mbar_init(c.bar(i), count);
     }
@@ -1697,12 +1687,11 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     } else {
       if (tid == 0) merge_producer(c, maps, g, a, first, stride, n_units, it0);
     }
-  } else if (warp == 1 || warp == 11) {
-    // one call site for both score issuers: the unrolled MMA block exists once
-    if ((tid & 31) == 0) {
-      if (stream) stream_mma_scores(c, g, a, first, stride, n_units, it0, warp == 11 ? 1u : 0u);
-      else if (warp == 1 && deep) deep_mma(c, g, n_my, a.k_raw != nullptr);
-      else if (warp == 1) merge_mma(c, g, a, first, stride, n_units);
+  } else if (warp == 1) {
+    if (tid == 32) {
+      if (stream) stream_mma_scores(c, g, a, first, stride, n_units, it0);
+      else if (deep) deep_mma(c, g, n_my, a.k_raw != nullptr);
+      else merge_mma(c, g, a, first, stride, n_units);
     }
   } else if (warp == 10) {
     if (tid == 320 && stream) stream_mma_pv(c, g, a, first, stride, n_units, it0);
