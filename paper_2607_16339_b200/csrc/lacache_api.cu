@@ -202,9 +202,10 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   // Block-query units: the keys of each (sequence, head) are cut into balanced
   // chunks of `tpc` tiles.  Unless the caller fixes it, pick the chunk size and
   // the role split together from a small cost model (times in microseconds,
-  // measured on B200: a stream unit costs ~2 + 2.1 per key tile, plus ~4 + 1.2
-  // per chunk when partial states have to be merged; a merge unit ~3.4
-  // after a ~4 us cold start), at most 16 chunks per sequence.
+  // measured on B200: a stream unit costs ~3 + 1.6 per key tile, plus ~2 + 0.8
+  // per chunk when partial states have to be merged; a merge unit ~2.6
+  // (pipelined variant, block_len <= 32, few units per CTA) or ~3.4 after a ~4 us cold start),
+  // at most 16 chunks per sequence.
   int tpc = cfg->sc_tiles_per_chunk;
   if (const char* e = getenv("LACACHE_SC_TILES")) tpc = atoi(e);
   if (tc && tpc <= 0) {
@@ -219,18 +220,27 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     const double units_m = (double)rows_u * g.Hq;
     double best = 1e30;
     for (int cand = 1; cand <= max_nkt; ++cand) {
-      double units_s = 0;
-      int max_ch = 1;
+      // the chunks this candidate would produce (balanced within a sequence, as below); a CTA
+      // draws short and long units alike, so a unit is costed between the mean and the longest
+      double units_s = 0, sum_t = 0;
+      int max_ch = 1, max_t = 1;
       for (int b = 0; b < g.B; ++b) {
         int nkt = (c->cu[b + 1] - c->cu[b] + TC_KEYS - 1) / TC_KEYS;
         int ch = std::min(16, (nkt + cand - 1) / cand);
+        int per = (nkt + ch - 1) / ch;
+        ch = (nkt + per - 1) / per;
         max_ch = std::max(max_ch, ch);
+        max_t = std::max(max_t, per);
         units_s += ch * (double)g.Hq;
+        sum_t += nkt;
       }
-      const double merge_cost = max_ch > 1 ? 4.0 + 1.2 * max_ch : 0.0;
+      const double eff_tiles = 0.5 * (sum_t * g.Hq / units_s + max_t);
+      const double merge_cost = max_ch > 1 ? 2.0 + 0.8 * max_ch : 0.0;
       for (int ns = 8; ns <= sms - 8; ns += 4) {
-        double ts = ceil(units_s / ns) * (2.0 + 2.1 * cand + merge_cost);
-        double tm = 4.0 + ceil(units_m / (sms - ns)) * 3.4;
+        double ts = ceil(units_s / ns) * (3.0 + 1.6 * eff_tiles + merge_cost);
+        // (a CTA with many merge units runs in the HBM-saturated regime, where a unit costs more)
+        const double per_cta = ceil(units_m / (sms - ns));
+        double tm = 4.0 + per_cta * ((g.block_len <= 32 && per_cta <= 8) ? 2.6 : 3.4);
         double t = std::max(ts, tm);
         if (t < best - 1e-9) { best = t; tpc = cand; }
       }
@@ -399,16 +409,20 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       a.n_items_merge = ml.n;
       long long units_merge = (long long)ml.n * Hq;
       int total = (int)std::min<long long>(c->num_sms, units_stream + units_merge);
-      int max_tiles = 1;
+      double sum_tiles = 0;   // ragged batches mix short and long units on a CTA: cost a unit between mean and longest
+      int longest = 1;
       for (int i = 0; i < list.n; ++i) {
         const WorkItem& w = c->items_host[list.off + i];
-        max_tiles = std::max(max_tiles, w.kt1 - w.kt0);
+        sum_tiles += w.kt1 - w.kt0;
+        longest = std::max(longest, w.kt1 - w.kt0);
       }
+      const double max_tiles = list.n > 0 ? 0.5 * (sum_tiles / list.n + longest) : 1.0;
       int ns = 1;
       double best = 1e30;
       for (int cand = 1; cand < total; ++cand) {
-        double ts = ceil((double)units_stream / cand) * (2.0 + 2.1 * max_tiles + (c->max_chunks > 1 ? 4.0 + 1.2 * c->max_chunks : 0.0));
-        double tm = 4.0 + ceil((double)units_merge / (total - cand)) * 3.4;
+        double ts = ceil((double)units_stream / cand) * (3.0 + 1.6 * max_tiles + (c->max_chunks > 1 ? 2.0 + 0.8 * c->max_chunks : 0.0));
+        const double per_cta = ceil((double)units_merge / (total - cand));
+        double tm = 4.0 + per_cta * ((c->g.block_len <= 32 && per_cta <= 8) ? 2.6 : 3.4);
         double t = std::max(ts, tm);
         if (t < best - 1e-9) { best = t; ns = cand; }
       }
@@ -417,6 +431,10 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       else ns = std::max(1, std::min(ns, total - 1));
       ns = (int)std::min<long long>(ns, units_stream);
       a.n_ctas_stream = ns;
+      if (getenv("LACACHE_VERBOSE")) {
+        static int printed = 0;
+        if (printed++ < 2) fprintf(stderr, "lacache: step plan: %lld stream units (max %d chunks), %lld merge units, %d stream CTAs of %d\n", units_stream, c->max_chunks, units_merge, ns, total);
+      }
       a.n_ctas = ns + (int)std::min<long long>(units_merge, std::max(0, c->num_sms - ns));
       {
         const int n_merge_ctas = a.n_ctas - ns;

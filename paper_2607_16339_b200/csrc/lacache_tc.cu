@@ -388,7 +388,8 @@ struct Unit {
 
 __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs& a, const WorkItem& it, int u) {
   Unit un;
-  un.h = u / a.n_items;
+  un.h = u % g.Hq;   // units are head-minor: unit u = item u / Hq of head u % Hq (a CTA's units, a fixed
+                     // stride apart, then cycle through the items instead of drawing one item's heads)
   un.kh = un.h / g.group;
   un.seq = it.seq;
   un.row0 = it.row0;
@@ -484,7 +485,7 @@ struct TileCursor {
 __device__ __forceinline__ void cursor_load_unit(const Geometry& g, const AttnArgs& a, TileCursor& cu, int n_units) {
   cu.valid = cu.u < n_units;
   if (!cu.valid) return;
-  cu.it = load_item(a.items + cu.u % a.n_items);
+  cu.it = load_item(a.items + cu.u / g.Hq);
   cu.un = decode_stream(g, a, cu.it, cu.u);
   cu.t = cu.un.t0;
   cu.q_done = !cu.loads_q;
@@ -611,7 +612,7 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   uint32_t js = 0;  // score tiles issued so far (stage and buffer = js & 1, phase = (js >> 1) & 1)
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
+    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / g.Hq);
     const Unit un = decode_stream(g, a, it, u);
     const uint32_t q_box = (uint32_t)un.q_rows * 128u;
     const int n_tiles = un.t1 - un.t0;
@@ -640,7 +641,7 @@ __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a
   uint32_t jp = 0;  // P~V tiles issued so far
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
+    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / g.Hq);
     const Unit un = decode_stream(g, a, it, u);
     const int n_tiles = un.t1 - un.t0;
     // O~ of the previous unit has been read by the row threads (observed once per unit, in order)
@@ -800,7 +801,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
   int jj = 0;
   for (int u = first; u < n_units; u += stride) {
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) % a.n_items);
+    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / g.Hq);
     const Unit un = decode_stream(g, a, it, u);
     it = nxt;
     if (u == first && a.mode == MODE_STEP && a.q_raw != nullptr) {
@@ -1635,7 +1636,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   }
   const int n_my = first < n_units ? (n_units - first + stride - 1) / stride : 0;
   WorkItem it0{};
-  if (!deep && first < n_units) it0 = stream ? load_item(a.items + first % a.n_items)
+  if (!deep && first < n_units) it0 = stream ? load_item(a.items + first / g.Hq)
                                              : load_item(a.items_merge + first / g.Hq);
   if ((c.base & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = LOC_SMEM_ALIGN;
