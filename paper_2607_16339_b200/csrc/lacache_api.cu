@@ -571,11 +571,13 @@ lacache_status lacache_step(lacache_ctx* c, const void* q, const void* k, const 
     r.row_cos = c->d_blk_cos + row0 * (c->g.d / 2);
     r.row_sin = c->d_blk_sin + row0 * (c->g.d / 2);
   }
+  r.pdl = 1;   // may start while the previous step's attention kernel drains (it waits before its stores)
   r.dst = c->rot;
   r.in_dtype = c->cfg.dtype;
   CU_TRY(c, rope_write(c->g, r, c->engine, s));
   c->last_launches++;
   AttnArgs a = attn_args(c, MODE_STEP, c->step_list[blk], blk, c->rot, out, lse);
+  a.step_overlap = (getenv("LACACHE_NO_PDL") || getenv("LACACHE_NO_STEP_OVERLAP")) ? 0 : 1;
   if (!getenv("LACACHE_NO_QCOMP")) {
     a.q_raw = q;
     a.k_raw = k;

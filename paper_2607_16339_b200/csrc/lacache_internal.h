@@ -80,6 +80,9 @@ struct RopeArgs {
   const int32_t* row_tok; const float* row_cos; const float* row_sin;  // [n_src_rows], [n_src_rows][d/2]
   RotBuffers dst;
   int in_dtype;
+  // launch programmatically dependent on the kernel before it in the stream (a step's attention
+  // kernel lets its successors start early): the kernel then waits before its first store
+  int pdl;
 };
 
 struct AttnArgs {
@@ -96,6 +99,7 @@ struct AttnArgs {
   // likewise the block's pre-RoPE keys and values [B * block_len, Hkv, d]: the first unit of a
   // pipelined merge-role CTA rotates the block's keys / converts its values itself
   const void* k_raw; const void* v_raw;
+  int step_overlap;          // step: let the next step's kernels be scheduled while this one drains
   const int32_t* cu;         // [B+1]
   const int32_t* blk_start;  // [B] absolute token index of the block's first row
   RotBuffers rot;

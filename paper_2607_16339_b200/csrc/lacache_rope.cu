@@ -11,6 +11,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <cstdlib>
+
 #include "lacache_internal.h"
 #include "lacache_rope_math.h"
 
@@ -86,6 +88,10 @@ __global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a)
 #pragma unroll
     for (int i = 0; i < 8; ++i) { y1[i] = x1[i]; y2[i] = x2[i]; }
   }
+  // Everything above read only this call's inputs and constant tables.  The stores below overwrite
+  // cache rows that the previous step's attention kernel may still be reading when this kernel was
+  // launched programmatically dependent on it: wait for that grid first (returns at once otherwise).
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   size_t doff = ((size_t)h * g.Tp + tok) * g.d;
   if (TC) {
     // tcgen05 storage: [head][feature half][Tp][64] (d = 128), each half of a row one 128-byte line
@@ -153,10 +159,20 @@ cudaError_t rope_write(const Geometry& g, const RopeArgs& a, int engine, cudaStr
   long long total = (long long)a.n_src_rows * (g.Hq + 2 * g.Hkv) * (g.d / 16);
   if (total == 0) return cudaSuccess;
   unsigned blocks = (unsigned)((total + 255) / 256);
-  if (engine == LACACHE_ENGINE_TCGEN05)
-    rope_write_kernel<true><<<blocks, 256, 0, s>>>(g, a);
-  else
-    rope_write_kernel<false><<<blocks, 256, 0, s>>>(g, a);
+  if (engine == LACACHE_ENGINE_TCGEN05) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    static const bool no_pdl = getenv("LACACHE_NO_PDL") != nullptr || getenv("LACACHE_NO_STEP_OVERLAP") != nullptr;
+    cfg.numAttrs = (a.pdl && !no_pdl) ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, rope_write_kernel<true>, g, a);
+  }
+  rope_write_kernel<false><<<blocks, 256, 0, s>>>(g, a);
   return cudaGetLastError();
 }
 

@@ -964,6 +964,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     }
 
     // ---- epilogue ----
+    grid_dependency_wait();  // no global store before the preceding grids are complete (see kernel entry)
     // second arrival on Q_FREE (the first is the MMA thread's commit): a 64-row
     // unit stages outside its Q tile, so its Q region may be reloaded at once
     if (un.q_rows != BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));
@@ -1266,6 +1267,7 @@ __device__ void merge_rows(const Cta& c, const TcMaps& maps, const Geometry& g, 
     }
     tc_fence_before();
     mbar_arrive(c.bar(BAR_O_FREE + b));
+    grid_dependency_wait();  // no global store before the preceding grids are complete
     const size_t orow = (size_t)row * g.Hq + h;
     if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_new + log2f(l_new)) * LN2;
     if (row_valid && r >= (it.nrows & ~7)) {
@@ -1280,6 +1282,7 @@ __device__ void merge_rows(const Cta& c, const TcMaps& maps, const Geometry& g, 
     fence_async_smem();
     if (!epi_sync(c, epi_phase)) return;  // the whole tile is in the staging buffer
     if (threadIdx.x == 64) {
+      grid_dependency_wait();
       if (store_out_tile(maps, c.base + SM_IO, h, it.row0, it.nrows) > 0) {
         bulk_commit();
         bulk_wait_read();               // the copies have read the staging tile
@@ -1377,6 +1380,7 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
     }
     if (mbar_test(c.bar((su & 1) ? BAR_OUT_RDY1 : BAR_OUT_RDY), (su >> 1) & 1)) {
       const DUnit un = deep_unit(c, su);
+      if (!dep_done) { grid_dependency_wait(); dep_done = true; }  // no store before the preceding grids are complete
       if (store_out_tile(maps, c.base + DM_IO + (su & 1) * DM_IO_TILE, un.h, un.row0, un.nrows) > 0) {
         bulk_commit();
         pending_read = true;
@@ -1584,6 +1588,7 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
     }
     tc_fence_before();
     mbar_arrive(c.bar(BAR_O_FREE + b));
+    grid_dependency_wait();  // no global store before the preceding grids are complete
     const size_t orow = (size_t)row * g.Hq + un.h;
     if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_new + log2f(l_new)) * LN2;
     if (row_valid && r >= (un.nrows & ~7)) {
@@ -1605,6 +1610,11 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
+  // A step reads only state that stays fixed until the next build plus what the RoPE kernel before it
+  // wrote, and every global store below comes after a wait on that kernel: the next step's kernels may
+  // therefore be scheduled as SMs free up (they, too, wait before their first store).  A build or a
+  // full recompute writes what a following step would read early, so they do not trigger.
+  if (a.mode == MODE_STEP && a.step_overlap) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   Cta c;
   c.base = smem_u32(smem_raw);
   c.gen = smem_raw;

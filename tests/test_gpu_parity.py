@@ -190,6 +190,57 @@ def test_runs_are_bit_reproducible():
         assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
 
 
+@pytest.mark.parametrize("cfg", [2, 4])
+def test_back_to_back_steps_match_synchronised_steps(cfg):
+    """Consecutive steps overlap on the device (the next step's kernels are scheduled while
+    the previous attention kernel drains).  A stream of steps and builds issued without any
+    host synchronisation must give, bit for bit, what the same calls give when the host
+    waits after each one -- with a separate output buffer per step and with one reused."""
+    wl = WORKLOADS[cfg]
+    S = min(wl.steps_per_block, 6)
+    calls = []   # ("build", blk, q, k, v) / ("step", qb, kb, vb)
+    sch = SyntheticSchedule(wl, seed=21)
+    for blk in (0, 1):
+        q, k, v = sch.begin_block(blk)
+        calls.append(("build", blk, to_dev(q, wl), to_dev(k, wl), to_dev(v, wl)))
+        for s in range(1, S + 1):
+            qb, kb, vb = sch.draw_step(blk, s)
+            calls.append(("step", to_dev(qb, wl), to_dev(kb, wl), to_dev(vb, wl)))
+    n_steps = sum(1 for c in calls if c[0] == "step")
+
+    def run(sync, one_buffer):
+        ctx = make_ctx(wl, engine=ENGINES["tc"])
+        bufs = [new_outputs(wl) for _ in range(1 if one_buffer else n_steps)]
+        res, i = [], 0
+        for c in calls:
+            if c[0] == "build":
+                ctx.build(c[1], c[2], c[3], c[4])
+            else:
+                out, lse = bufs[0 if one_buffer else i]
+                ctx.step(c[1], c[2], c[3], out, lse)
+                i += 1
+                if sync:
+                    torch.cuda.synchronize()
+                    res.append((out.clone(), lse.clone()))
+            if sync:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        st, msg = ctx.poll_status()
+        assert st == 0, msg
+        if not sync:
+            res = [(o.clone(), l.clone()) for o, l in bufs]
+        ctx.destroy()
+        return res
+
+    ref = run(sync=True, one_buffer=False)
+    for rep in range(3):
+        got = run(sync=False, one_buffer=False)
+        for i, ((o0, l0), (o1, l1)) in enumerate(zip(ref, got)):
+            assert torch.equal(o0, o1) and torch.equal(l0, l1), "step %d differs when issued back to back" % i
+        last = run(sync=False, one_buffer=True)
+        assert torch.equal(ref[-1][0], last[0][0]) and torch.equal(ref[-1][1], last[0][1])
+
+
 def test_error_paths():
     wl = small_workload(prompt_lens=(40,), gen_len=64, block_len=32, steps=1, hq=2, hkv=2, d=128)
     sch = SyntheticSchedule(wl, seed=1)
