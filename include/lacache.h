@@ -113,6 +113,14 @@ lacache_status lacache_build(lacache_ctx* ctx, int block_idx, const void* q_pre,
  * out [T,Hq,d] fp32 for ALL T rows and, if lse != NULL, lse [T,Hq].  The
  * (m, l, O~) cache is read-only here.  Requires a preceding lacache_build for
  * the same block, else LACACHE_ERR_STATE.
+ *
+ * Stream semantics: the work is enqueued on `cuda_stream` and is complete, with
+ * out / lse fully written, before any later operation of that stream that this
+ * library did not enqueue (a kernel, a copy, an event) runs.  Two lacache_step
+ * calls in a row on one stream may overlap on the device (the second call's
+ * kernels are launched programmatically dependent and store nothing before the
+ * first call's kernels have completed); q_blk / k_blk / v_blk must stay
+ * unchanged until the call's work has completed, as for any stream-ordered call.
  */
 lacache_status lacache_step(lacache_ctx* ctx, const void* q_blk, const void* k_blk,
                             const void* v_blk, float* out, float* lse, void* cuda_stream);
