@@ -190,7 +190,7 @@ def test_runs_are_bit_reproducible():
         assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
 
 
-@pytest.mark.parametrize("cfg", [2, 4])
+@pytest.mark.parametrize("cfg", [2, 4, 5])
 def test_back_to_back_steps_match_synchronised_steps(cfg):
     """Consecutive steps overlap on the device (the next step's kernels are scheduled while
     the previous attention kernel drains).  A stream of steps and builds issued without any
