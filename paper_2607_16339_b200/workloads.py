@@ -96,7 +96,8 @@ def round_to_dtype(x, dtype):
     raise ValueError(dtype)
 
 
-_TENSOR_IDS = {"q": 1, "k": 2, "v": 3, "scale": 4, "mask": 5, "outlier": 6}
+_TENSOR_IDS = {"q": 1, "k": 2, "v": 3, "scale": 4, "mask": 5, "outlier": 6,
+               "embed": 7, "norm_w": 8, "w_qkv": 9, "ids": 10, "channels": 11}
 
 
 def _rng(seed, cfg, tensor, block=0, step=0):
@@ -228,3 +229,75 @@ def small_workload(name="small", dtype="bf16", prompt_lens=(70,), gen_len=64, bl
     finishes in seconds."""
     return Workload(cfg, name, dtype, tuple(prompt_lens), gen_len, block_len, steps, hq, hkv, d,
                     theta, scale_mode, outlier_frac, 4.0 if outlier_frac > 0 else 1.0)
+
+
+@dataclass
+class TokenModel:
+    """Seeded synthetic weights of the token-wise operators in front of the
+    first-layer attention (embedding table, norm weight, stacked Q/K/V
+    projection) and the token ids a block-wise denoising run feeds them.
+
+    They stand in for the trained first-layer weights of the models the paper
+    evaluates, which are not available.  Shapes follow those models: ``d_model``
+    4096 with 32 heads (LLaDA-8B), 3584 with 28/4 heads (Dream-7B).  Values: the
+    embedding rows are N(0, 1) with a few seeded channels 20x larger (trained
+    LLM embeddings carry such outlier channels, and the norm in front of the
+    projection is what they stress); the norm weight is U(0.5, 1.5); projection
+    rows are N(0, 1/d_model) times the per-head scale of the attention workload,
+    so the projected q/k/v have the spread of the workload's own q/k/v.  All
+    values are rounded to bf16 (returned as float32).  The last table row is
+    the [MASK] token.  The vocabulary size does not change the work of a call
+    (a call gathers one row per token), so it may be chosen small.
+    """
+    wl: Workload
+    d_model: int
+    vocab: int
+    seed: int = 0
+    rms_eps: float = 1e-5
+    embed: Optional[np.ndarray] = None
+    norm_weight: Optional[np.ndarray] = None
+    w_qkv: Optional[np.ndarray] = None
+
+    def __post_init__(self):
+        wl, dm = self.wl, self.d_model
+        d, Hq, Hkv = wl.head_dim, wl.n_q_heads, wl.n_kv_heads
+        e = _rng(self.seed, wl.cfg, "embed").standard_normal((self.vocab, dm), dtype=np.float32)
+        ch = _rng(self.seed, wl.cfg, "channels").choice(dm, size=max(1, dm // 1024), replace=False)
+        e[:, ch] *= 20.0
+        self.embed = round_to_bf16(e)
+        self.norm_weight = round_to_bf16(_rng(self.seed, wl.cfg, "norm_w").uniform(0.5, 1.5, dm))
+        if wl.scale_mode == "inv_sqrt_d":
+            sq, skv = np.full(Hq, 1.0 / np.sqrt(d)), np.full(Hkv, 1.0 / np.sqrt(d))
+        else:
+            c = _rng(self.seed, wl.cfg, "scale").uniform(0.5, 2.0, Hq)
+            sq, skv = c, c[::Hq // Hkv].copy()
+        row_scale = np.concatenate([np.repeat(sq, d), np.repeat(skv, d), np.repeat(skv, d)])
+        w = _rng(self.seed, wl.cfg, "w_qkv").standard_normal(((Hq + 2 * Hkv) * d, dm), dtype=np.float32)
+        w *= (row_scale / np.sqrt(dm)).astype(np.float32)[:, None]
+        self.w_qkv = round_to_bf16(w)
+
+    @property
+    def mask_id(self):
+        return self.vocab - 1
+
+    def full_ids(self, b):
+        """Token ids of all T packed tokens as the build of block b sees them:
+        seeded prompt and already decoded ids, [MASK] from block b on."""
+        wl = self.wl
+        ids = _rng(self.seed, wl.cfg, "ids").integers(0, self.vocab - 1, wl.total_tokens).astype(np.int32)
+        cu = wl.cu_seqlens
+        for s, P in enumerate(wl.prompt_lens):
+            ids[cu[s] + P + b * wl.block_len:cu[s + 1]] = self.mask_id
+        return ids
+
+    def block_ids(self, b, s):
+        """Ids of the block's B * L_b tokens at step s (1-based): a seeded subset
+        of about s / steps_per_block of the positions is decoded, the rest is
+        still [MASK].  Sequence-major."""
+        wl = self.wl
+        n = wl.batch * wl.block_len
+        r = _rng(self.seed, wl.cfg, "ids", b + 1, s)
+        ids = r.integers(0, self.vocab - 1, n).astype(np.int32)
+        still_masked = r.uniform(size=n) >= s / wl.steps_per_block
+        ids[still_masked] = self.mask_id
+        return ids
