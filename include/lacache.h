@@ -186,6 +186,85 @@ lacache_status lacache_step_host(lacache_ctx* ctx, const void* q_blk_host, const
                                  void* cuda_stream);
 
 /*
+ * Token-wise producer (Sec. 3.3.2, EmbedCache and RoPECache; Eq. 1): the operators that act on
+ * each token alone in front of the first-layer attention.  For a list of tokens it computes
+ * H = Embed(x) (or takes H as given), H^ = RMSNorm(H) and the pre-rotation projections
+ * H^ W_Q, H^ W_K, H^ W_V; the rotation of Eq. 1 is applied by lacache_build / lacache_step, which
+ * consume the result.  With it a denoising step feeds only the current block's token ids (or
+ * hidden states): everything token-wise for the fixed tokens stays in the caches.
+ *
+ * Arithmetic: bf16 weights and activations; the norm is evaluated in fp32 and rounded once to
+ * bf16; the projections accumulate in fp32 on the tensor cores and are rounded once to bf16.
+ *
+ * Config pointers are DEVICE pointers to bf16 data that the caller owns and keeps alive and
+ * unchanged for the life of the handle (they are not copied):
+ *   embed        [vocab, d_model]; NULL with vocab == 0 when only hidden states will be fed
+ *   norm_weight  [d_model]
+ *   w_qkv        [(n_q_heads + 2 n_kv_heads) * head_dim, d_model], one row per output feature
+ *                (the layout of a torch Linear weight): Q heads, then K heads, then V heads
+ * d_model is a multiple of 64, at most 8192; head_dim is 128; max_tokens bounds n_tokens of every
+ * later call.  Needs an sm_100 device.
+ */
+typedef struct lacache_qkv lacache_qkv;
+typedef struct {
+  int vocab;
+  int d_model;
+  int n_q_heads;
+  int n_kv_heads;
+  int head_dim;
+  float rms_eps;
+  int max_tokens;
+  const void* embed;
+  const void* norm_weight;
+  const void* w_qkv;
+} lacache_qkv_config;
+
+/* Allocates the handle's scratch (operand rows, stream-K workspace, projected rows for the
+ * *_tokens calls) and encodes the TMA descriptors.  The only allocating call of the producer.
+ * On failure *out is NULL and lacache_qkv_last_error(NULL) has the text. */
+lacache_status lacache_qkv_create(const lacache_qkv_config* cfg, lacache_qkv** out);
+/* Synchronises the device, then frees what the handle owns (not the weights). */
+lacache_status lacache_qkv_destroy(lacache_qkv* p);
+
+/*
+ * Projects n_tokens tokens (0 <= n_tokens <= max_tokens).  Exactly one of token_ids (DEVICE
+ * int32 [n_tokens], each in [0, vocab)) and hidden (DEVICE bf16 [n_tokens, d_model]) is non-NULL.
+ * Writes bf16 q [n_tokens, Hq, d], k and v [n_tokens, Hkv, d] (pre-rotation) and, if h_out is
+ * non-NULL, the embedding rows H [n_tokens, d_model] bf16 (the EmbedCache content).  Enqueues two
+ * kernels on `cuda_stream` and returns without synchronising.  A token id outside the table is
+ * reported by lacache_qkv_poll_status (LACACHE_ERR_INVALID_ARG); its rows are zero.
+ * The result does not depend on how the work was split over the SMs: equal inputs give equal bits.
+ */
+lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, const void* hidden,
+                                   int n_tokens, void* q, void* k, void* v, void* h_out,
+                                   void* cuda_stream);
+
+/*
+ * lacache_build / lacache_step fed by the producer: the tokens are projected into the handle's
+ * scratch and the attention call consumes it on the same stream.  build takes all T tokens
+ * (token_ids [T] or hidden [T, d_model], packed like q_pre), step the block's B * L_b tokens
+ * (sequence-major like q_blk).  The context must be bf16 with the same heads and head_dim as
+ * the producer, and max_tokens must cover the call (else LACACHE_ERR_SHAPE).  Consecutive
+ * calls on one stream are ordered; unlike lacache_step, a step fed this way starts after the
+ * previous step has completed.
+ */
+lacache_status lacache_build_tokens(lacache_ctx* ctx, lacache_qkv* p, int block_idx,
+                                    const int32_t* token_ids, const void* hidden,
+                                    void* cuda_stream);
+lacache_status lacache_step_tokens(lacache_ctx* ctx, lacache_qkv* p, const int32_t* blk_token_ids,
+                                   const void* blk_hidden, float* out, float* lse,
+                                   void* cuda_stream);
+
+/* Profiling hook like lacache_set_timing_events, around the projection (GEMM) kernel. */
+lacache_status lacache_qkv_set_timing_events(lacache_qkv* p, void* ev_start, void* ev_stop);
+/* Kernels launched by the last lacache_qkv_project. */
+int lacache_qkv_last_launch_count(const lacache_qkv* p);
+/* Synchronises the device and reads the producer's status word (bounded waits, token ids). */
+lacache_status lacache_qkv_poll_status(lacache_qkv* p);
+/* Text of the last error of this handle; with NULL, of the last failed lacache_qkv_create. */
+const char* lacache_qkv_last_error(const lacache_qkv* p);
+
+/*
  * Test hooks.  All outputs are device pointers, token-major fp32.
  *   export_state: the cached triple in natural-log units, m [T,Hq], l [T,Hq],
  *     o_acc [T,Hq,d].  The triple is not unique (any reference m gives the same

@@ -22,6 +22,9 @@ EXPORTS = [
     "lacache_export_rope_cache", "lacache_export_index_meta", "lacache_total_tokens",
     "lacache_last_launch_count", "lacache_engine", "lacache_set_timing_events",
     "lacache_full_recompute_static", "lacache_poll_status", "lacache_last_error",
+    "lacache_qkv_create", "lacache_qkv_destroy", "lacache_qkv_project", "lacache_build_tokens",
+    "lacache_step_tokens", "lacache_qkv_set_timing_events", "lacache_qkv_last_launch_count",
+    "lacache_qkv_poll_status", "lacache_qkv_last_error",
 ]
 
 
@@ -33,6 +36,15 @@ class LacacheConfig(ctypes.Structure):
         ("batch", ctypes.c_int), ("prompt_lens", ctypes.POINTER(ctypes.c_int32)),
         ("gen_len", ctypes.c_int), ("block_len", ctypes.c_int),
         ("sc_tiles_per_chunk", ctypes.c_int),
+    ]
+
+
+class LacacheQkvConfig(ctypes.Structure):
+    _fields_ = [
+        ("vocab", ctypes.c_int), ("d_model", ctypes.c_int), ("n_q_heads", ctypes.c_int),
+        ("n_kv_heads", ctypes.c_int), ("head_dim", ctypes.c_int), ("rms_eps", ctypes.c_float),
+        ("max_tokens", ctypes.c_int), ("embed", ctypes.c_void_p), ("norm_weight", ctypes.c_void_p),
+        ("w_qkv", ctypes.c_void_p),
     ]
 
 
@@ -75,8 +87,18 @@ def load():
     lib.lacache_poll_status.argtypes = [vp]
     lib.lacache_last_error.argtypes = [vp]
     lib.lacache_last_error.restype = ctypes.c_char_p
+    lib.lacache_qkv_create.argtypes = [ctypes.POINTER(LacacheQkvConfig), ctypes.POINTER(vp)]
+    lib.lacache_qkv_destroy.argtypes = [vp]
+    lib.lacache_qkv_project.argtypes = [vp, vp, vp, ip, vp, vp, vp, vp, vp]
+    lib.lacache_build_tokens.argtypes = [vp, vp, ip, vp, vp, vp]
+    lib.lacache_step_tokens.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.lacache_qkv_set_timing_events.argtypes = [vp, vp, vp]
+    lib.lacache_qkv_last_launch_count.argtypes = [vp]
+    lib.lacache_qkv_poll_status.argtypes = [vp]
+    lib.lacache_qkv_last_error.argtypes = [vp]
+    lib.lacache_qkv_last_error.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name != "lacache_last_error":
+        if name not in ("lacache_last_error", "lacache_qkv_last_error"):
             getattr(lib, name).restype = ip
     _lib = lib
     return lib
@@ -192,6 +214,14 @@ class Context:
         self._check(self._lib.lacache_export_index_meta(self._h, p(seq), p(pos), p(isb), p(kvh)))
         return seq, pos, isb, kvh
 
+    def build_tokens(self, producer, block_idx, token_ids=None, hidden=None, stream=None):
+        self._check(self._lib.lacache_build_tokens(self._h, producer._h, int(block_idx), _ptr(token_ids),
+                                                   _ptr(hidden), _stream(stream)))
+
+    def step_tokens(self, producer, out, lse=None, blk_token_ids=None, blk_hidden=None, stream=None):
+        self._check(self._lib.lacache_step_tokens(self._h, producer._h, _ptr(blk_token_ids), _ptr(blk_hidden),
+                                                  _ptr(out), _ptr(lse), _stream(stream)))
+
     def set_timing_events(self, ev_start, ev_stop):
         """torch.cuda.Event pair (already recorded once) or (None, None)."""
         h = lambda e: None if e is None else ctypes.c_void_p(e.cuda_event)
@@ -200,3 +230,54 @@ class Context:
     def poll_status(self):
         st = self._lib.lacache_poll_status(self._h)
         return st, (self._lib.lacache_last_error(self._h) or b"").decode()
+
+
+class QkvProducer:
+    """Owns one ``lacache_qkv`` (the token-wise producer).  The weight tensors
+    (bf16, on the device) are kept referenced here because the library does not
+    copy them."""
+
+    def __init__(self, embed, norm_weight, w_qkv, n_q_heads, n_kv_heads, head_dim, rms_eps, max_tokens):
+        self._lib = load()
+        self._h = ctypes.c_void_p()
+        self._weights = (embed, norm_weight, w_qkv)
+        vocab = 0 if embed is None else int(embed.shape[0])
+        cfg = LacacheQkvConfig(vocab, int(w_qkv.shape[1]), int(n_q_heads), int(n_kv_heads), int(head_dim),
+                               float(rms_eps), int(max_tokens),
+                               None if embed is None else embed.data_ptr(), norm_weight.data_ptr(),
+                               w_qkv.data_ptr())
+        st = self._lib.lacache_qkv_create(ctypes.byref(cfg), ctypes.byref(self._h))
+        if st != OK:
+            self._h = ctypes.c_void_p()
+            raise LacacheError(st, (self._lib.lacache_qkv_last_error(None) or b"").decode())
+
+    def _check(self, st):
+        if st != OK:
+            raise LacacheError(st, (self._lib.lacache_qkv_last_error(self._h) or b"").decode())
+
+    def destroy(self):
+        if self._h:
+            self._lib.lacache_qkv_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def project(self, n_tokens, q, k, v, token_ids=None, hidden=None, h_out=None, stream=None):
+        self._check(self._lib.lacache_qkv_project(self._h, _ptr(token_ids), _ptr(hidden), int(n_tokens),
+                                                  _ptr(q), _ptr(k), _ptr(v), _ptr(h_out), _stream(stream)))
+
+    def set_timing_events(self, ev_start, ev_stop):
+        h = lambda e: None if e is None else ctypes.c_void_p(e.cuda_event)
+        self._check(self._lib.lacache_qkv_set_timing_events(self._h, h(ev_start), h(ev_stop)))
+
+    @property
+    def last_launch_count(self):
+        return self._lib.lacache_qkv_last_launch_count(self._h)
+
+    def poll_status(self):
+        st = self._lib.lacache_qkv_poll_status(self._h)
+        return st, (self._lib.lacache_qkv_last_error(self._h) or b"").decode()

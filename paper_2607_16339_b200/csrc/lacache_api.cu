@@ -549,8 +549,64 @@ lacache_status lacache_build(lacache_ctx* c, int block_idx, const void* q, const
   return LACACHE_OK;
 }
 
+namespace {
+// inputs_just_written: q / k / v are produced by the kernel enqueued right before this call, so
+// nothing of the step may read them before that kernel has completed
+lacache_status step_impl(lacache_ctx* c, const void* q, const void* k, const void* v, float* out, float* lse,
+                         void* stream, bool inputs_just_written);
+}  // namespace
+
 lacache_status lacache_step(lacache_ctx* c, const void* q, const void* k, const void* v, float* out,
                             float* lse, void* stream) {
+  return step_impl(c, q, k, v, out, lse, stream, false);
+}
+
+namespace {
+// the producer handle fits the context and covers n tokens
+lacache_status check_producer(lacache_ctx* c, lacache_qkv* p, int n) {
+  int hq = 0, hkv = 0, max_tokens = 0;
+  const int d = qkv_heads(p, &hq, &hkv, &max_tokens);
+  if (c->cfg.dtype != LACACHE_DTYPE_BF16) return fail(c, LACACHE_ERR_UNSUPPORTED, "the producer writes bf16: the context must be bf16");
+  if (hq != c->g.Hq || hkv != c->g.Hkv || d != c->g.d)
+    return fail(c, LACACHE_ERR_SHAPE, "producer heads %d/%d x %d, context %d/%d x %d", hq, hkv, d, c->g.Hq, c->g.Hkv, c->g.d);
+  if (n > max_tokens) return fail(c, LACACHE_ERR_SHAPE, "%d tokens, producer max_tokens %d", n, max_tokens);
+  return LACACHE_OK;
+}
+}  // namespace
+
+lacache_status lacache_build_tokens(lacache_ctx* c, lacache_qkv* p, int block_idx, const int32_t* token_ids,
+                                    const void* hidden, void* stream) {
+  if (!c || !p) return LACACHE_ERR_INVALID_ARG;
+  lacache_status st = check_producer(c, p, c->g.T);
+  if (st != LACACHE_OK) return st;
+  void *q, *k, *v;
+  qkv_scratch(p, &q, &k, &v);
+  st = lacache_qkv_project(p, token_ids, hidden, c->g.T, q, k, v, nullptr, stream);
+  if (st != LACACHE_OK) return fail(c, st, "producer: %s", lacache_qkv_last_error(p));
+  st = lacache_build(c, block_idx, q, k, v, stream);
+  if (st == LACACHE_OK) c->last_launches += lacache_qkv_last_launch_count(p);
+  return st;
+}
+
+lacache_status lacache_step_tokens(lacache_ctx* c, lacache_qkv* p, const int32_t* blk_token_ids,
+                                   const void* blk_hidden, float* out, float* lse, void* stream) {
+  if (!c || !p) return LACACHE_ERR_INVALID_ARG;
+  if (c->built_block < 0) return fail(c, LACACHE_ERR_STATE, "lacache_step_tokens before a successful build");
+  const int n = c->g.B * c->g.block_len;
+  lacache_status st = check_producer(c, p, n);
+  if (st != LACACHE_OK) return st;
+  void *q, *k, *v;
+  qkv_scratch(p, &q, &k, &v);
+  st = lacache_qkv_project(p, blk_token_ids, blk_hidden, n, q, k, v, nullptr, stream);
+  if (st != LACACHE_OK) return fail(c, st, "producer: %s", lacache_qkv_last_error(p));
+  st = step_impl(c, q, k, v, out, lse, stream, true);
+  if (st == LACACHE_OK) c->last_launches += lacache_qkv_last_launch_count(p);
+  return st;
+}
+
+namespace {
+lacache_status step_impl(lacache_ctx* c, const void* q, const void* k, const void* v, float* out, float* lse,
+                         void* stream, bool inputs_just_written) {
   if (!c) return LACACHE_ERR_INVALID_ARG;
   if (c->built_block < 0) return fail(c, LACACHE_ERR_STATE, "lacache_step before a successful lacache_build");
   if (!q || !k || !v || !out) return fail(c, LACACHE_ERR_INVALID_ARG, "NULL pointer");
@@ -571,7 +627,9 @@ lacache_status lacache_step(lacache_ctx* c, const void* q, const void* k, const 
     r.row_cos = c->d_blk_cos + row0 * (c->g.d / 2);
     r.row_sin = c->d_blk_sin + row0 * (c->g.d / 2);
   }
-  r.pdl = 1;   // may start while the previous step's attention kernel drains (it waits before its stores)
+  // may start while the previous step's attention kernel drains (it waits before its stores), unless
+  // the kernel before it in the stream is the one that writes its inputs
+  r.pdl = inputs_just_written ? 0 : 1;
   r.dst = c->rot;
   r.in_dtype = c->cfg.dtype;
   CU_TRY(c, rope_write(c->g, r, c->engine, s));
@@ -588,6 +646,7 @@ lacache_status lacache_step(lacache_ctx* c, const void* q, const void* k, const 
   }
   return run_attention(c, a, false, s);
 }
+}  // namespace
 
 lacache_status lacache_full_recompute(lacache_ctx* c, const void* q, const void* k, const void* v, float* out,
                                       float* lse, void* stream) {

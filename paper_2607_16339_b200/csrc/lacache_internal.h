@@ -136,6 +136,11 @@ TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, c
 bool tc_set_out(TcMaps* m, const Geometry& g, float* out, char* err, int errlen);
 void tc_free_maps(TcMaps* m);
 
+// token-wise producer (lacache_qkv.cu): the scratch rows the *_tokens entry points project into,
+// and its head configuration (returns head_dim)
+void qkv_scratch(lacache_qkv* p, void** q, void** k, void** v);
+int qkv_heads(const lacache_qkv* p, int* hq, int* hkv, int* max_tokens);
+
 constexpr int SIMT_ROWS = 32;    // query rows per SIMT work item
 constexpr int TC_ROWS = 128;     // query rows per tcgen05 work item
 #ifndef LACACHE_TC_KEYS

@@ -1,0 +1,637 @@
+// Token-wise producer in front of the first-layer attention (Sec. 3.3.2: embedding, attention norm,
+// Q/K/V projections; the rotation of Eq. 1 is applied by the kernels that consume the result).
+//
+// Two kernels:
+//   qkv_norm_kernel  one CTA per token: gathers the token's embedding row (or takes a given hidden
+//                    state), RMS-normalises it in fp32 and writes the bf16 operand row X^ (and, on
+//                    request, the embedding row itself: what the EmbedCache keeps).
+//   qkv_gemm_kernel  Y^T = W X^T on tcgen05: the 128 output features of one head are the M rows of the
+//                    MMA (A = a [128 x 64] tile of W, K-major, by TMA), the tokens are its N columns
+//                    (B = [TN x 64] tile of X^, K-major, by TMA), fp32 accumulators in TMEM.  With a
+//                    block's 32..64 tokens the kernel is bound by reading W once from HBM, so the work
+//                    is cut stream-K fashion: the (tile, 64-wide k chunk) pairs are dealt out in equal
+//                    contiguous ranges to one persistent CTA per SM.  A CTA that owns only part of a
+//                    tile's chunks leaves its fp32 partial in a workspace; the last CTA to arrive at a
+//                    tile adds the partials in CTA order (the result does not depend on arrival order)
+//                    and writes the bf16 rows.
+// Warp roles of the GEMM: warp 0 (one lane) TMA producer over a ring of stages, warp 1 (one lane) MMA
+// issuer, warps 2..5 epilogue (TMEM lane = output feature).  Two accumulators alternate so that an
+// epilogue overlaps the next segment's MMAs.  Every mbarrier wait is bounded; a wait that runs out sets
+// the status word and the CTA unwinds (TMEM is always freed).
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "lacache_internal.h"
+#include "lacache_ptx.h"
+
+using namespace lacache;
+
+struct lacache_qkv {
+  lacache_qkv_config cfg;
+  int n_ftiles = 0;        // 128-row tiles of W = heads: Hq + 2 Hkv
+  int tokens_pad = 0;      // rows of the operand buffer (max_tokens rounded up to 256)
+  int num_sms = 148;
+  int device = 0;
+  __nv_bfloat16* xhat = nullptr;        // [tokens_pad][d_model]
+  float* ws = nullptr;                  // [2 * num_sms][256 * 128] partial tiles
+  int* counters = nullptr;              // per tile: chunks accumulated so far
+  int32_t* status = nullptr;
+  __nv_bfloat16 *q = nullptr, *k = nullptr, *v = nullptr;   // [max_tokens][H][128] scratch of the *_tokens calls
+  CUtensorMap w_map;
+  CUtensorMap x_map[4];                 // boxes of 32, 64, 128, 256 tokens
+  cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
+  int last_launches = 0;
+  char err[512];
+};
+
+namespace lacache {
+namespace {
+
+using namespace ptx;
+
+constexpr int QD = 128;                 // head_dim = features per tile = MMA M
+constexpr int BK = 64;                  // k chunk: one 128-byte swizzled row of bf16
+constexpr int MAX_TN = 256;
+constexpr int G_THREADS = 192;
+constexpr int EPI_THREADS = 128;
+constexpr uint32_t A_BYTES = QD * BK * 2;
+constexpr int MAX_STAGES = 12;
+constexpr uint32_t RING_BYTES = 229376;
+constexpr uint32_t SMQ_BAR = RING_BYTES;
+enum { QB_FULL = 0, QB_FREE = MAX_STAGES, QB_ACC_FULL = 2 * MAX_STAGES, QB_ACC_FREE = QB_ACC_FULL + 2,
+       QB_N = QB_ACC_FREE + 2 };
+constexpr uint32_t SMQ_TOTAL = SMQ_BAR + 8 * QB_N + 32;
+static_assert(SMQ_TOTAL <= 232448, "exceeds the 227 KB per-CTA limit");
+constexpr long long Q_WAIT_CYCLES = 4000000000ll;  // ~2 s
+enum { QLOC_SMEM_ALIGN = 101, QLOC_WAIT_FULL = 102, QLOC_WAIT_FREE = 103, QLOC_WAIT_ACC_FULL = 104,
+       QLOC_WAIT_ACC_FREE = 105, QLOC_TOKEN_ID = 106 };
+
+struct GemmArgs {
+  int n_tokens, tn, n_ttiles, n_tiles, kc;   // kc = d_model / 64 chunks per tile
+  long long total_chunks;
+  int n_stages;
+  int Hq, Hkv;
+  __nv_bfloat16 *q, *k, *v;
+  float* ws;
+  int* counters;
+  int32_t* status;
+};
+
+struct QCta {
+  uint32_t base;
+  volatile int* abort_flag;
+  int32_t* status;
+  __device__ __forceinline__ uint32_t bar(int slot) const { return base + SMQ_BAR + 8u * slot; }
+};
+
+__device__ __noinline__ bool q_wait_slow(const QCta& c, uint32_t bar, uint32_t parity, int loc) {
+  long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if (*c.abort_flag) return false;
+    if (clock64() - t0 > Q_WAIT_CYCLES) {
+      *c.abort_flag = 1;
+      if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
+        c.status[1] = loc;
+        c.status[2] = blockIdx.x;
+        c.status[3] = threadIdx.x;
+      }
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool q_wait(const QCta& c, int slot, uint32_t parity, int loc) {
+  const uint32_t b = c.bar(slot);
+  if (mbar_try(b, parity)) return true;
+  return q_wait_slow(c, b, parity, loc);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+// first chunk of CTA j's contiguous range of the (tile, chunk) list
+__device__ __forceinline__ long long range_start(const GemmArgs& a, int j) {
+  return (long long)j * a.total_chunks / (long long)gridDim.x;
+}
+// the CTA whose range holds chunk x
+__device__ __forceinline__ int cta_of(const GemmArgs& a, long long x) {
+  return (int)(((x + 1) * (long long)gridDim.x - 1) / a.total_chunks);
+}
+
+// destination of feature tile ft, token t: row of q, k or v
+__device__ __forceinline__ __nv_bfloat16* out_row(const GemmArgs& a, int ft, int t) {
+  if (ft < a.Hq) return a.q + ((size_t)t * a.Hq + ft) * QD;
+  if (ft < a.Hq + a.Hkv) return a.k + ((size_t)t * a.Hkv + (ft - a.Hq)) * QD;
+  return a.v + ((size_t)t * a.Hkv + (ft - a.Hq - a.Hkv)) * QD;
+}
+
+__device__ __forceinline__ void gemm_producer(const QCta& c, const CUtensorMap* w_map, const CUtensorMap* x_map,
+                                              const GemmArgs& a, long long r0, long long r1, uint32_t stage_bytes) {
+  long long it = 0;
+  for (long long x = r0; x < r1;) {
+    const int tile = (int)(x / a.kc), c0 = (int)(x % a.kc);
+    const int c1 = (int)min((long long)a.kc, c0 + (r1 - x));
+    const int ft = tile / a.n_ttiles, tt = tile % a.n_ttiles;
+    for (int ch = c0; ch < c1; ++ch, ++it) {
+      const int s = (int)(it % a.n_stages);
+      const uint32_t ph = (uint32_t)(it / a.n_stages) & 1u;
+      if (!q_wait(c, QB_FREE + s, ph ^ 1u, QLOC_WAIT_FREE)) return;
+      const uint32_t dst = c.base + s * stage_bytes;
+      mbar_expect_tx(c.bar(QB_FULL + s), stage_bytes);
+      tma_load_2d(dst, w_map, c.bar(QB_FULL + s), ch * BK, ft * QD);
+      tma_load_2d(dst + A_BYTES, x_map, c.bar(QB_FULL + s), ch * BK, tt * a.tn);
+    }
+    x += c1 - c0;
+  }
+}
+
+__device__ __forceinline__ void gemm_mma(const QCta& c, const GemmArgs& a, uint32_t tmem, long long r0, long long r1,
+                                         uint32_t stage_bytes) {
+  const uint32_t idesc = idesc_f16(1u /*bf16*/, 0u, QD, (uint32_t)a.tn);
+  long long it = 0;
+  int seg = 0;
+  for (long long x = r0; x < r1; ++seg) {
+    const int c0 = (int)(x % a.kc);
+    const int c1 = (int)min((long long)a.kc, c0 + (r1 - x));
+    const int buf = seg & 1;
+    // the epilogue of the segment that used this accumulator two segments ago has drained it
+    if (!q_wait(c, QB_ACC_FREE + buf, ((uint32_t)(seg >> 1) & 1u) ^ 1u, QLOC_WAIT_ACC_FREE)) return;
+    tc_fence_after();
+    const uint32_t acc = tmem + (uint32_t)(buf * MAX_TN);
+    for (int ch = c0; ch < c1; ++ch, ++it) {
+      const int s = (int)(it % a.n_stages);
+      const uint32_t ph = (uint32_t)(it / a.n_stages) & 1u;
+      if (!q_wait(c, QB_FULL + s, ph, QLOC_WAIT_FULL)) return;
+      tc_fence_after();
+      const uint32_t sa = c.base + s * stage_bytes;
+      const uint64_t ad = smem_desc(sa, 16, 1024), bd = smem_desc(sa + A_BYTES, 16, 1024);
+#pragma unroll
+      for (int ks = 0; ks < BK / 16; ++ks)
+        mma_ss(acc, ad + 2u * ks, bd + 2u * ks, idesc, (ch > c0 || ks > 0) ? 1u : 0u);
+      tc_commit(c.bar(QB_FREE + s));
+    }
+    tc_commit(c.bar(QB_ACC_FULL + buf));
+    x += c1 - c0;
+  }
+}
+
+__device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, uint32_t tmem, long long r0,
+                                              long long r1, volatile uint32_t* flag) {
+  const int tid = threadIdx.x;
+  const int et = tid - 64;                       // 0..127
+  const int quad = (tid >> 5) & 3;               // the TMEM lane quadrant this warp may read
+  const int f = quad * 32 + (tid & 31);          // output feature within the tile
+  const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+  int seg = 0;
+  for (long long x = r0; x < r1; ++seg) {
+    const int tile = (int)(x / a.kc), c0 = (int)(x % a.kc);
+    const int c1 = (int)min((long long)a.kc, c0 + (r1 - x));
+    const int ft = tile / a.n_ttiles, tt = tile % a.n_ttiles;
+    const int t0 = tt * a.tn;
+    const int nt = min(a.tn, a.n_tokens - t0);   // valid tokens of the tile
+    const int buf = seg & 1;
+    const bool whole = (c0 == 0 && c1 == a.kc);
+    if (!q_wait(c, QB_ACC_FULL + buf, (uint32_t)(seg >> 1) & 1u, QLOC_WAIT_ACC_FULL)) return;
+    tc_fence_after();
+    // a CTA's range leaves at most its first and its last segment partial: two workspace slots
+    float* part = a.ws + ((size_t)blockIdx.x * 2 + (seg == 0 ? 0 : 1)) * (size_t)(MAX_TN * QD);
+    for (int g = 0; g * 32 < nt; ++g) {
+      uint32_t r[32];
+      tmem_ld32(tmem + lane_off + (uint32_t)(buf * MAX_TN + g * 32), r);
+      tmem_ld_wait();
+      if (whole) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int t = g * 32 + i;
+          if (t < nt) out_row(a, ft, t0 + t)[f] = __float2bfloat16_rn(__uint_as_float(r[i]));
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int t = g * 32 + i;
+          if (t < nt) part[(size_t)t * QD + f] = __uint_as_float(r[i]);
+        }
+      }
+    }
+    tc_fence_before();
+    mbar_arrive(c.bar(QB_ACC_FREE + buf));
+    if (!whole) {
+      // publish the partial, then count this segment's chunks; whoever completes the tile adds up
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (et == 0) {
+        const int old = atomicAdd(a.counters + tile, c1 - c0);
+        const uint32_t last = (old + (c1 - c0) == a.kc) ? 1u : 0u;
+        if (last) a.counters[tile] = 0;           // ready for the next launch
+        *flag = last;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (*flag) {
+        __threadfence();
+        const long long x_lo = (long long)tile * a.kc, x_hi = x_lo + a.kc;
+        const int j_lo = cta_of(a, x_lo), j_hi = cta_of(a, x_hi - 1);
+        for (int t = 0; t < nt; ++t) {
+          float sum = 0.f;
+          for (int j = j_lo; j <= j_hi; ++j) {
+            const long long s0 = range_start(a, j), s1 = range_start(a, j + 1);
+            if (s1 <= s0) continue;               // a CTA without work
+            const int slot = (s0 >= x_lo) ? 0 : 1;   // the tile holds its first segment, or its last
+            const float* p = a.ws + ((size_t)j * 2 + slot) * (size_t)(MAX_TN * QD);
+            sum += __ldcg(p + (size_t)t * QD + f);
+          }
+          out_row(a, ft, t0 + t)[f] = __float2bfloat16_rn(sum);
+        }
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // the flag word is reused by the next segment
+    }
+    x += c1 - c0;
+  }
+}
+
+__global__ void __launch_bounds__(G_THREADS, 1)
+qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map,
+                const GemmArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5;
+  QCta c;
+  c.base = smem_u32(smem_raw);
+  uint32_t* words = reinterpret_cast<uint32_t*>(smem_raw + SMQ_BAR + 8 * QB_N);  // [0] tmem, [1] abort, [2] flag
+  c.abort_flag = reinterpret_cast<volatile int*>(words + 1);
+  c.status = a.status;
+  if ((c.base & 1023u) != 0) {
+    if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = QLOC_SMEM_ALIGN;
+    return;
+  }
+  if (tid == 0) {
+    prefetch_map(&w_map);
+    prefetch_map(&x_map);
+    for (int i = 0; i < QB_N; ++i) mbar_init(c.bar(i), (i >= QB_ACC_FREE) ? EPI_THREADS : 1);
+    words[1] = 0;
+    words[2] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  __syncwarp();
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(words)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = words[0];
+  // the operand rows X^ come from the kernel launched before this one
+  grid_dependency_wait();
+
+  const long long r0 = range_start(a, blockIdx.x), r1 = range_start(a, blockIdx.x + 1);
+  const uint32_t stage_bytes = A_BYTES + (uint32_t)a.tn * 128u;
+  if (warp == 0) {
+    if (tid == 0) gemm_producer(c, &w_map, &x_map, a, r0, r1, stage_bytes);
+  } else if (warp == 1) {
+    if (tid == 32) gemm_mma(c, a, tmem, r0, r1, stage_bytes);
+  } else {
+    gemm_epilogue(c, a, tmem, r0, r1, words + 2);
+  }
+  __syncwarp();
+  // teardown: free TMEM once every thread is past its last TMEM access
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+constexpr int N_THREADS = 256;
+constexpr int N_MAX_CHUNKS = 4;   // 8-element chunks per thread: d_model <= 8192
+
+struct NormArgs {
+  const int32_t* ids;             // or null
+  const __nv_bfloat16* hidden;    // [n][d_model], used when ids == null
+  const __nv_bfloat16* table;     // [vocab][d_model]
+  const __nv_bfloat16* weight;    // [d_model]
+  __nv_bfloat16* xhat;            // [n][d_model]
+  __nv_bfloat16* h_out;           // [n][d_model] or null
+  int d_model, vocab;
+  float eps;
+  int32_t* status;
+};
+
+__global__ void __launch_bounds__(N_THREADS) qkv_norm_kernel(const NormArgs a) {
+  // the projection kernel may be scheduled now: it waits for this grid before it reads X^
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  __shared__ float red[N_THREADS / 32];
+  const int t = blockIdx.x;
+  const int tid = threadIdx.x;
+  const __nv_bfloat16* src;
+  bool valid = true;
+  if (a.ids) {
+    const int id = a.ids[t];
+    valid = id >= 0 && id < a.vocab;
+    if (!valid && tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_INVALID_ARG) == 0) {
+      a.status[1] = QLOC_TOKEN_ID;
+      a.status[2] = t;
+      a.status[3] = id;
+    }
+    src = a.table + (size_t)(valid ? id : 0) * a.d_model;
+  } else {
+    src = a.hidden + (size_t)t * a.d_model;
+  }
+  const int n_chunks = a.d_model / 8;
+  uint4 raw[N_MAX_CHUNKS];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < N_MAX_CHUNKS; ++i) {
+    const int ch = tid + i * N_THREADS;
+    raw[i] = make_uint4(0, 0, 0, 0);
+    if (ch < n_chunks && valid) raw[i] = __ldg(reinterpret_cast<const uint4*>(src) + ch);
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw[i]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 x = __bfloat1622float2(p[e]);
+      ss = fmaf(x.x, x.x, ss);
+      ss = fmaf(x.y, x.y, ss);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  if ((tid & 31) == 0) red[tid >> 5] = ss;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < N_THREADS / 32; ++i) tot += red[i];
+  // an invalid token id (reported through the status word) yields a zero row
+  const float rinv = valid ? 1.0f / sqrtf(tot / (float)a.d_model + a.eps) : 0.f;
+#pragma unroll
+  for (int i = 0; i < N_MAX_CHUNKS; ++i) {
+    const int ch = tid + i * N_THREADS;
+    if (ch >= n_chunks) continue;
+    const uint4 wraw = __ldg(reinterpret_cast<const uint4*>(a.weight) + ch);
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw[i]);
+    const __nv_bfloat162* w = reinterpret_cast<const __nv_bfloat162*>(&wraw);
+    uint4 o;
+    __nv_bfloat162* q = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 x = __bfloat1622float2(p[e]);
+      const float2 g = __bfloat1622float2(w[e]);
+      q[e] = __floats2bfloat162_rn(x.x * rinv * g.x, x.y * rinv * g.y);
+    }
+    reinterpret_cast<uint4*>(a.xhat + (size_t)t * a.d_model)[ch] = o;
+    if (a.h_out) reinterpret_cast<uint4*>(a.h_out + (size_t)t * a.d_model)[ch] = raw[i];
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+thread_local char g_qkv_create_err[512] = "";
+
+lacache_status qfail(lacache_qkv* p, lacache_status st, const char* fmt, ...) {
+  char* dst = p ? p->err : g_qkv_create_err;
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(dst, 512, fmt, ap);
+  va_end(ap);
+  return st;
+}
+
+#define QCU_TRY(p, expr)                                                               \
+  do {                                                                                 \
+    cudaError_t e_ = (expr);                                                           \
+    if (e_ != cudaSuccess)                                                             \
+      return qfail(p, e_ == cudaErrorMemoryAllocation ? LACACHE_ERR_OOM : LACACHE_ERR_CUDA, \
+                   "%s: %s", #expr, cudaGetErrorString(e_));                           \
+  } while (0)
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 matrix [rows][cols] row-major as a 2-D tensor {cols, rows}; box = 64 columns x box_rows rows
+bool make_bf16_map(lacache_qkv* p, CUtensorMap* m, const void* base, int rows, int cols, int box_rows) {
+  static EncodeTiledFn enc = nullptr;
+  if (!enc) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess) {
+      qfail(p, LACACHE_ERR_CUDA, "cuTensorMapEncodeTiled entry point not found");
+      return false;
+    }
+    enc = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    qfail(p, LACACHE_ERR_CUDA, "cuTensorMapEncodeTiled (2-D bf16) failed with CUresult %d", (int)r);
+    return false;
+  }
+  return true;
+}
+
+void qkv_free(lacache_qkv* p) {
+  if (!p) return;
+  cudaDeviceSynchronize();
+  void* bufs[] = {p->xhat, p->ws, p->counters, p->status, p->q, p->k, p->v};
+  for (void* b : bufs)
+    if (b) cudaFree(b);
+  delete p;
+}
+
+bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+}  // namespace
+
+// scratch rows the *_tokens entry points project into
+void qkv_scratch(lacache_qkv* p, void** q, void** k, void** v) {
+  *q = p->q; *k = p->k; *v = p->v;
+}
+int qkv_heads(const lacache_qkv* p, int* hq, int* hkv, int* max_tokens) {
+  *hq = p->cfg.n_q_heads; *hkv = p->cfg.n_kv_heads; *max_tokens = p->cfg.max_tokens;
+  return p->cfg.head_dim;
+}
+
+}  // namespace lacache
+
+extern "C" {
+
+lacache_status lacache_qkv_create(const lacache_qkv_config* cfg, lacache_qkv** out) {
+  if (out) *out = nullptr;
+  if (!cfg || !out) return qfail(nullptr, LACACHE_ERR_INVALID_ARG, "NULL argument");
+  if (cfg->head_dim != QD) return qfail(nullptr, LACACHE_ERR_UNSUPPORTED, "head_dim %d: only 128", cfg->head_dim);
+  if (cfg->d_model < BK || cfg->d_model % BK != 0 || cfg->d_model > 8 * N_THREADS * N_MAX_CHUNKS)
+    return qfail(nullptr, LACACHE_ERR_SHAPE, "d_model %d: a multiple of 64 in [64, 8192]", cfg->d_model);
+  if (cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads % cfg->n_kv_heads != 0)
+    return qfail(nullptr, LACACHE_ERR_SHAPE, "heads %d / %d", cfg->n_q_heads, cfg->n_kv_heads);
+  if (cfg->max_tokens < 1 || cfg->vocab < 0 || !(cfg->rms_eps >= 0.f))
+    return qfail(nullptr, LACACHE_ERR_INVALID_ARG, "max_tokens %d, vocab %d, rms_eps %g", cfg->max_tokens, cfg->vocab,
+                 (double)cfg->rms_eps);
+  if (!cfg->norm_weight || !cfg->w_qkv || (cfg->vocab > 0 && !cfg->embed))
+    return qfail(nullptr, LACACHE_ERR_INVALID_ARG, "NULL weight pointer");
+  if (misaligned16(cfg->norm_weight) || misaligned16(cfg->w_qkv) || misaligned16(cfg->embed))
+    return qfail(nullptr, LACACHE_ERR_INVALID_ARG, "weight pointer not 16-byte aligned");
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev < 1) {
+    cudaGetLastError();
+    return qfail(nullptr, LACACHE_ERR_CUDA, "no CUDA device");
+  }
+  lacache_qkv* p = new (std::nothrow) lacache_qkv();
+  if (!p) return qfail(nullptr, LACACHE_ERR_OOM, "host allocation failed");
+  p->cfg = *cfg;
+  p->err[0] = 0;
+  p->n_ftiles = cfg->n_q_heads + 2 * cfg->n_kv_heads;
+  p->tokens_pad = (cfg->max_tokens + MAX_TN - 1) / MAX_TN * MAX_TN;
+  lacache_status st = LACACHE_OK;
+  auto attempt = [&]() -> lacache_status {
+    QCU_TRY(p, cudaGetDevice(&p->device));
+    cudaDeviceProp prop;
+    QCU_TRY(p, cudaGetDeviceProperties(&prop, p->device));
+    if (prop.major != 10) return qfail(p, LACACHE_ERR_UNSUPPORTED, "device is sm_%d%d, need sm_100", prop.major, prop.minor);
+    p->num_sms = prop.multiProcessorCount;
+    const size_t d = (size_t)cfg->d_model;
+    QCU_TRY(p, cudaMalloc(&p->xhat, (size_t)p->tokens_pad * d * 2));
+    QCU_TRY(p, cudaMemset(p->xhat, 0, (size_t)p->tokens_pad * d * 2));
+    QCU_TRY(p, cudaMalloc(&p->ws, (size_t)2 * p->num_sms * MAX_TN * QD * 4));
+    const int max_tiles = p->n_ftiles * ((cfg->max_tokens + 31) / 32);
+    QCU_TRY(p, cudaMalloc(&p->counters, (size_t)max_tiles * 4));
+    QCU_TRY(p, cudaMemset(p->counters, 0, (size_t)max_tiles * 4));
+    QCU_TRY(p, cudaMalloc(&p->status, 16));
+    QCU_TRY(p, cudaMemset(p->status, 0, 16));
+    QCU_TRY(p, cudaMalloc(&p->q, (size_t)cfg->max_tokens * cfg->n_q_heads * QD * 2));
+    QCU_TRY(p, cudaMalloc(&p->k, (size_t)cfg->max_tokens * cfg->n_kv_heads * QD * 2));
+    QCU_TRY(p, cudaMalloc(&p->v, (size_t)cfg->max_tokens * cfg->n_kv_heads * QD * 2));
+    if (!make_bf16_map(p, &p->w_map, cfg->w_qkv, p->n_ftiles * QD, cfg->d_model, QD)) return LACACHE_ERR_CUDA;
+    for (int i = 0; i < 4; ++i)
+      if (!make_bf16_map(p, &p->x_map[i], p->xhat, p->tokens_pad, cfg->d_model, 32 << i)) return LACACHE_ERR_CUDA;
+    QCU_TRY(p, cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMQ_TOTAL));
+    return LACACHE_OK;
+  };
+  st = attempt();
+  if (st != LACACHE_OK) {
+    snprintf(g_qkv_create_err, sizeof g_qkv_create_err, "%s", p->err);
+    qkv_free(p);
+    return st;
+  }
+  *out = p;
+  return LACACHE_OK;
+}
+
+lacache_status lacache_qkv_destroy(lacache_qkv* p) {
+  if (!p) return LACACHE_ERR_INVALID_ARG;
+  qkv_free(p);
+  return LACACHE_OK;
+}
+
+lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, const void* hidden, int n_tokens,
+                                   void* q, void* k, void* v, void* h_out, void* stream) {
+  if (!p) return LACACHE_ERR_INVALID_ARG;
+  if ((token_ids == nullptr) == (hidden == nullptr))
+    return qfail(p, LACACHE_ERR_INVALID_ARG, "pass exactly one of token_ids and hidden");
+  if (token_ids && p->cfg.vocab == 0) return qfail(p, LACACHE_ERR_STATE, "token ids given but no embedding table");
+  if (!q || !k || !v) return qfail(p, LACACHE_ERR_INVALID_ARG, "NULL output pointer");
+  if (misaligned16(q) || misaligned16(k) || misaligned16(v) || misaligned16(hidden) || misaligned16(h_out))
+    return qfail(p, LACACHE_ERR_INVALID_ARG, "pointer not 16-byte aligned");
+  if (n_tokens < 0 || n_tokens > p->cfg.max_tokens)
+    return qfail(p, LACACHE_ERR_SHAPE, "n_tokens %d outside [0, %d]", n_tokens, p->cfg.max_tokens);
+  p->last_launches = 0;
+  if (n_tokens == 0) return LACACHE_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+
+  NormArgs na{};
+  na.ids = token_ids;
+  na.hidden = reinterpret_cast<const __nv_bfloat16*>(hidden);
+  na.table = reinterpret_cast<const __nv_bfloat16*>(p->cfg.embed);
+  na.weight = reinterpret_cast<const __nv_bfloat16*>(p->cfg.norm_weight);
+  na.xhat = p->xhat;
+  na.h_out = reinterpret_cast<__nv_bfloat16*>(h_out);
+  na.d_model = p->cfg.d_model;
+  na.vocab = p->cfg.vocab;
+  na.eps = p->cfg.rms_eps;
+  na.status = p->status;
+  qkv_norm_kernel<<<n_tokens, N_THREADS, 0, s>>>(na);
+  QCU_TRY(p, cudaGetLastError());
+  p->last_launches++;
+
+  GemmArgs ga{};
+  int tn_idx = 0;
+  while (tn_idx < 3 && (32 << tn_idx) < n_tokens) ++tn_idx;
+  ga.n_tokens = n_tokens;
+  ga.tn = 32 << tn_idx;
+  ga.n_ttiles = (n_tokens + ga.tn - 1) / ga.tn;
+  ga.n_tiles = p->n_ftiles * ga.n_ttiles;
+  ga.kc = p->cfg.d_model / BK;
+  ga.total_chunks = (long long)ga.n_tiles * ga.kc;
+  ga.n_stages = (int)std::min<uint32_t>(MAX_STAGES, RING_BYTES / (A_BYTES + (uint32_t)ga.tn * 128u));
+  ga.Hq = p->cfg.n_q_heads;
+  ga.Hkv = p->cfg.n_kv_heads;
+  ga.q = reinterpret_cast<__nv_bfloat16*>(q);
+  ga.k = reinterpret_cast<__nv_bfloat16*>(k);
+  ga.v = reinterpret_cast<__nv_bfloat16*>(v);
+  ga.ws = p->ws;
+  ga.counters = p->counters;
+  ga.status = p->status;
+  const int n_ctas = (int)std::min<long long>(p->num_sms, ga.total_chunks);
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_ctas);
+  cfg.blockDim = dim3(G_THREADS);
+  cfg.dynamicSmemBytes = SMQ_TOTAL;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = getenv("LACACHE_NO_PDL") ? 0 : 1;
+  if (p->ev_start && p->ev_stop) {
+    cfg.numAttrs = 0;   // an event between the two kernels: an ordinary launch
+    QCU_TRY(p, cudaEventRecord(p->ev_start, s));
+  }
+  QCU_TRY(p, cudaLaunchKernelEx(&cfg, qkv_gemm_kernel, p->w_map, p->x_map[tn_idx], ga));
+  if (p->ev_start && p->ev_stop) QCU_TRY(p, cudaEventRecord(p->ev_stop, s));
+  p->last_launches++;
+  return LACACHE_OK;
+}
+
+lacache_status lacache_qkv_set_timing_events(lacache_qkv* p, void* ev_start, void* ev_stop) {
+  if (!p) return LACACHE_ERR_INVALID_ARG;
+  p->ev_start = (cudaEvent_t)ev_start;
+  p->ev_stop = (cudaEvent_t)ev_stop;
+  return LACACHE_OK;
+}
+
+int lacache_qkv_last_launch_count(const lacache_qkv* p) { return p ? p->last_launches : -1; }
+
+lacache_status lacache_qkv_poll_status(lacache_qkv* p) {
+  if (!p) return LACACHE_ERR_INVALID_ARG;
+  QCU_TRY(p, cudaDeviceSynchronize());
+  int32_t w[4] = {0, 0, 0, 0};
+  QCU_TRY(p, cudaMemcpy(w, p->status, 16, cudaMemcpyDeviceToHost));
+  if (w[0] == 0) return LACACHE_OK;
+  QCU_TRY(p, cudaMemset(p->status, 0, 16));
+  if (w[1] == QLOC_TOKEN_ID)
+    return qfail(p, (lacache_status)w[0], "token id %d of input row %d is outside the embedding table", w[3], w[2]);
+  return qfail(p, (lacache_status)w[0], "device status %d at location %d (block %d, thread %d)", w[0], w[1], w[2], w[3]);
+}
+
+const char* lacache_qkv_last_error(const lacache_qkv* p) { return p ? p->err : g_qkv_create_err; }
+
+}  // extern "C"

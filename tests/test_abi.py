@@ -59,6 +59,36 @@ def test_create_rejects_bad_configs_without_gpu():
     assert lib.lacache_build(None, 0, None, None, None, None) == binding.ERR_INVALID_ARG
 
 
+def test_producer_create_rejects_bad_configs_without_gpu():
+    lib = binding.load()
+    h = ctypes.c_void_p()
+    dummy = 0x1000   # never dereferenced: validation fails first
+
+    def cfg(**kw):
+        base = dict(vocab=10, d_model=256, n_q_heads=4, n_kv_heads=2, head_dim=128, rms_eps=1e-5,
+                    max_tokens=32, embed=dummy, norm_weight=dummy, w_qkv=dummy)
+        base.update(kw)
+        return binding.LacacheQkvConfig(*[base[f[0]] for f in binding.LacacheQkvConfig._fields_])
+
+    cases = [
+        (cfg(head_dim=64), binding.ERR_UNSUPPORTED),
+        (cfg(d_model=200), binding.ERR_SHAPE),
+        (cfg(d_model=16384), binding.ERR_SHAPE),
+        (cfg(n_kv_heads=3), binding.ERR_SHAPE),
+        (cfg(max_tokens=0), binding.ERR_INVALID_ARG),
+        (cfg(w_qkv=None), binding.ERR_INVALID_ARG),
+        (cfg(embed=None), binding.ERR_INVALID_ARG),
+        (cfg(norm_weight=0x1004), binding.ERR_INVALID_ARG),
+    ]
+    for c, want in cases:
+        st = lib.lacache_qkv_create(ctypes.byref(c), ctypes.byref(h))
+        assert st == want, (st, want, lib.lacache_qkv_last_error(None))
+        assert not h.value and lib.lacache_qkv_last_error(None)
+    assert lib.lacache_qkv_create(None, ctypes.byref(h)) == binding.ERR_INVALID_ARG
+    assert lib.lacache_qkv_project(None, None, None, 0, None, None, None, None, None) == binding.ERR_INVALID_ARG
+    assert lib.lacache_step_tokens(None, None, None, None, None, None, None) == binding.ERR_INVALID_ARG
+
+
 def test_product_path_does_not_touch_the_oracle():
     pkg = os.path.join(ROOT, "paper_2607_16339_b200")
     for dirpath, _, files in os.walk(pkg):
