@@ -470,12 +470,95 @@ def run_cuda(args):
         }
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(wl, budget_s=12.0)
-        print(json.dumps(line), flush=True)
     for c in ctxs:
         c.destroy()
+    del outs, sched
+    if rank == 0:
+        if world == 1 and not args.no_token_path and wl.dtype == "bf16" and wl.n_q_heads in D_MODEL:
+            line["token_path"] = token_path_leg(wl, dev, peaks, args.seed, min(K, 512))
+        print(json.dumps(line), flush=True)
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------
+# the step fed by token ids: embedding gather + RMS norm + Q/K/V projection in front
+# ----------------------------------------------------------------------------
+D_MODEL = {32: 4096, 28: 3584}     # first-layer width of the model a workload is shaped like, by query heads
+QKV_TRAFFIC_PER_LAUNCH = {2: 105807872}   # ncu, profiles/qkv_gemm_kernel_llada_n32_ncu.txt
+
+
+def token_path_leg(wl, dev, peaks, seed, n_steps):
+    """Steps per second of lacache_step_tokens (token ids in, attention output out) and the
+    event-timed duration of its projection kernel, which is bound by reading the stacked
+    Q/K/V weight once per step.  Weight and cache-state replicas are visited round-robin so
+    that every call finds them in HBM."""
+    import torch
+    from paper_2607_16339_b200 import binding
+    from paper_2607_16339_b200.workloads import TokenModel
+    mk = lambda: torch.cuda.Event(enable_timing=True)
+    tm = TokenModel(wl, D_MODEL[wl.n_q_heads], 8192, seed)
+    T, nb, S = wl.total_tokens, wl.batch * wl.block_len, wl.steps_per_block
+    bf = lambda a: torch.from_numpy(a).to(dev).to(torch.bfloat16).contiguous()
+    emb, nw, w0 = bf(tm.embed), bf(tm.norm_weight), bf(tm.w_qkv)
+    w_bytes = w0.numel() * 2
+    R = max(3, -(-2 * L2_BYTES // w_bytes) + 1)
+    prods = [binding.QkvProducer(emb, nw, w0, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, tm.rms_eps, T)
+             for _ in range(R)]      # each handle holds its own re-laid-out copy of the weight
+    ctxs = [binding.Context.from_workload(wl) for _ in range(R)]
+    out = torch.empty(T, wl.n_q_heads, wl.head_dim, device=dev)
+    lse = torch.empty(T, wl.n_q_heads, device=dev)
+    blk = wl.n_blocks // 2
+    ids_full = torch.from_numpy(tm.full_ids(blk)).to(dev)
+    ids_blk = [torch.from_numpy(tm.block_ids(blk, s)).to(dev) for s in range(1, S + 1)]
+    for c in range(R):
+        ctxs[c].build_tokens(prods[c], blk, token_ids=ids_full)
+    torch.cuda.synchronize()
+    e0, e1 = mk(), mk()
+    e0.record()
+    for i in range(2 * R):
+        ctxs[i % R].build_tokens(prods[i % R], blk, token_ids=ids_full)
+    e1.record(); torch.cuda.synchronize()
+    build_us = e0.elapsed_time(e1) / (2 * R) * 1e3
+    launches = 0
+    for i in range(16):
+        ctxs[i % R].step_tokens(prods[i % R], out, lse, blk_token_ids=ids_blk[i % S])
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(n_steps):
+        ctxs[i % R].step_tokens(prods[i % R], out, lse, blk_token_ids=ids_blk[i % S])
+        launches += ctxs[i % R].last_launch_count
+    e1.record(); torch.cuda.synchronize()
+    step_us = e0.elapsed_time(e1) / n_steps * 1e3
+    # the projection kernel alone, event pair recorded inside the library around its launch
+    pairs = []
+    for i in range(min(n_steps, 96)):
+        e = (mk(), mk()); e[0].record(); e[1].record()
+        prods[i % R].set_timing_events(*e); pairs.append(e)
+        ctxs[i % R].step_tokens(prods[i % R], out, lse, blk_token_ids=ids_blk[i % S])
+    torch.cuda.synchronize()
+    gemm_us = statistics.mean(a.elapsed_time(b) for a, b in pairs) * 1e3
+    for o in prods + ctxs:
+        st, msg = o.poll_status()
+        if st != 0:
+            raise SystemExit("device status (token path): %s" % msg)
+        o.destroy()
+    d_model = tm.d_model
+    alg = w_bytes + nb * d_model * 2 + nb * (wl.n_q_heads + 2 * wl.n_kv_heads) * wl.head_dim * 2
+    ach = alg / (gemm_us * 1e-6) / 1e9
+    return {
+        "what": "lacache_step_tokens: token ids -> embedding gather + RMS norm + Q/K/V projection (tcgen05, stream-K) "
+                "-> RoPE + cached attention; synthetic first-layer weights",
+        "d_model": d_model, "tokens_per_step": nb, "replicas": R,
+        "value": round(1e6 / step_us, 1), "unit": UNIT, "step_us": round(step_us, 2),
+        "build_tokens_us": round(build_us, 1), "gpu_launches": launches, "steps": n_steps,
+        "roofline": {"kernel": "qkv_gemm_kernel (one step: %d tokens x %d -> %d features)" % (nb, d_model, w0.shape[0]),
+                     "bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": round(ach / peaks["hbm_gbs"], 4), "peak_source": peaks["source"],
+                     "traffic": QKV_TRAFFIC_PER_LAUNCH.get(wl.cfg), "avg_launch_us": round(gemm_us, 2),
+                     "algorithmic_bytes_per_launch": int(alg)},
+    }
 
 
 # per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the
@@ -578,6 +661,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-token-path", action="store_true", help="skip the extra leg that feeds steps from token ids")
     ap.add_argument("--replicas", type=int, default=0, help="cache-state replicas visited round-robin (0 = sized from the L2)")
     args = ap.parse_args()
     if args.warmup < 3:

@@ -196,12 +196,15 @@ lacache_status lacache_step_host(lacache_ctx* ctx, const void* q_blk_host, const
  * Arithmetic: bf16 weights and activations; the norm is evaluated in fp32 and rounded once to
  * bf16; the projections accumulate in fp32 on the tensor cores and are rounded once to bf16.
  *
- * Config pointers are DEVICE pointers to bf16 data that the caller owns and keeps alive and
- * unchanged for the life of the handle (they are not copied):
+ * Config pointers are DEVICE pointers to bf16 data owned by the caller:
  *   embed        [vocab, d_model]; NULL with vocab == 0 when only hidden states will be fed
  *   norm_weight  [d_model]
  *   w_qkv        [(n_q_heads + 2 n_kv_heads) * head_dim, d_model], one row per output feature
  *                (the layout of a torch Linear weight): Q heads, then K heads, then V heads
+ * embed and norm_weight are referenced, not copied: keep them alive and unchanged for the life
+ * of the handle.  w_qkv is copied at create into the handle, re-laid out in the tile order the
+ * projection kernel streams (same size); the caller's copy may be released afterwards, and a
+ * later change to it has no effect.
  * d_model is a multiple of 64, at most 8192; head_dim is 128; max_tokens bounds n_tokens of every
  * later call.  Needs an sm_100 device.
  */

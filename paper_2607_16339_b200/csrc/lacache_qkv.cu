@@ -6,7 +6,8 @@
 //                    state), RMS-normalises it in fp32 and writes the bf16 operand row X^ (and, on
 //                    request, the embedding row itself: what the EmbedCache keeps).
 //   qkv_gemm_kernel  Y^T = W X^T on tcgen05: the 128 output features of one head are the M rows of the
-//                    MMA (A = a [128 x 64] tile of W, K-major, by TMA), the tokens are its N columns
+//                    MMA (A = a [128 x 64] tile of W, K-major, by TMA from a copy of W re-laid out at
+//                    create so that every such tile is one contiguous 16 KB run), the tokens are its N columns
 //                    (B = [TN x 64] tile of X^, K-major, by TMA), fp32 accumulators in TMEM.  With a
 //                    block's 32..64 tokens the kernel is bound by reading W once from HBM, so the work
 //                    is cut stream-K fashion: the (tile, 64-wide k chunk) pairs are dealt out in equal
@@ -39,6 +40,7 @@ struct lacache_qkv {
   int tokens_pad = 0;      // rows of the operand buffer (max_tokens rounded up to 256)
   int num_sms = 148;
   int device = 0;
+  __nv_bfloat16* w_packed = nullptr;    // W in tile order: [feature tile][k chunk][128 rows][64 columns]
   __nv_bfloat16* xhat = nullptr;        // [tokens_pad][d_model]
   float* ws = nullptr;                  // [2 * num_sms][256 * 128] partial tiles
   int* counters = nullptr;              // per tile: chunks accumulated so far
@@ -138,30 +140,61 @@ __device__ __forceinline__ __nv_bfloat16* out_row(const GemmArgs& a, int ft, int
   return a.v + ((size_t)t * a.Hkv + (ft - a.Hq - a.Hkv)) * QD;
 }
 
-__device__ __forceinline__ void gemm_producer(const QCta& c, const CUtensorMap* w_map, const CUtensorMap* x_map,
-                                              const GemmArgs& a, long long r0, long long r1, uint32_t stage_bytes) {
-  long long it = 0;
-  for (long long x = r0; x < r1;) {
-    const int tile = (int)(x / a.kc), c0 = (int)(x % a.kc);
-    const int c1 = (int)min((long long)a.kc, c0 + (r1 - x));
-    const int ft = tile / a.n_ttiles, tt = tile % a.n_ttiles;
-    for (int ch = c0; ch < c1; ++ch, ++it) {
-      const int s = (int)(it % a.n_stages);
-      const uint32_t ph = (uint32_t)(it / a.n_stages) & 1u;
-      if (!q_wait(c, QB_FREE + s, ph ^ 1u, QLOC_WAIT_FREE)) return;
-      const uint32_t dst = c.base + s * stage_bytes;
-      mbar_expect_tx(c.bar(QB_FULL + s), stage_bytes);
-      tma_load_2d(dst, w_map, c.bar(QB_FULL + s), ch * BK, ft * QD);
-      tma_load_2d(dst + A_BYTES, x_map, c.bar(QB_FULL + s), ch * BK, tt * a.tn);
+// Walks this CTA's chunks in order without divisions: ring stage and phase, tile coordinates, chunk.
+struct ChunkCursor {
+  int s; uint32_t ph;     // ring stage and its phase
+  int ft, tt, ch;         // feature tile, token tile, k chunk
+  __device__ __forceinline__ void init(const GemmArgs& a, long long r0) {
+    s = 0; ph = 0;
+    const int tile = (int)(r0 / a.kc);
+    ch = (int)(r0 % a.kc);
+    ft = tile / a.n_ttiles;
+    tt = tile % a.n_ttiles;
+  }
+  __device__ __forceinline__ void next(const GemmArgs& a) {
+    if (++s == a.n_stages) { s = 0; ph ^= 1u; }
+    if (++ch == a.kc) {
+      ch = 0;
+      if (++tt == a.n_ttiles) { tt = 0; ++ft; }
     }
-    x += c1 - c0;
+  }
+};
+
+// Loads of one chunk into its ring stage: the W tile and / or the X^ tile.  One mbarrier per stage
+// counts the bytes of both.
+__device__ __forceinline__ void load_chunk(const QCta& c, const CUtensorMap* w_map, const CUtensorMap* x_map,
+                                           const GemmArgs& a, const ChunkCursor& k, uint32_t stage_bytes,
+                                           bool load_w, bool load_x) {
+  const uint32_t dst = c.base + k.s * stage_bytes;
+  if (load_w) {
+    mbar_expect_tx(c.bar(QB_FULL + k.s), stage_bytes);
+    tma_load_2d(dst, w_map, c.bar(QB_FULL + k.s), 0, (k.ft * a.kc + k.ch) * QD);   // one contiguous 16 KB tile
+  }
+  if (load_x) tma_load_2d(dst + A_BYTES, x_map, c.bar(QB_FULL + k.s), k.ch * BK, k.tt * a.tn);
+}
+
+// `early` chunks already have their W tile in flight (issued before the wait on the preceding grid)
+__device__ __forceinline__ void gemm_producer(const QCta& c, const CUtensorMap* w_map, const CUtensorMap* x_map,
+                                              const GemmArgs& a, long long r0, long long r1, uint32_t stage_bytes,
+                                              int early) {
+  ChunkCursor k;
+  k.init(a, r0);
+  const int n = (int)(r1 - r0);
+  for (int it = 0; it < n; ++it, k.next(a)) {
+    if (it < early) {
+      load_chunk(c, w_map, x_map, a, k, stage_bytes, false, true);
+      continue;
+    }
+    if (!q_wait(c, QB_FREE + k.s, k.ph ^ 1u, QLOC_WAIT_FREE)) return;
+    load_chunk(c, w_map, x_map, a, k, stage_bytes, true, true);
   }
 }
 
 __device__ __forceinline__ void gemm_mma(const QCta& c, const GemmArgs& a, uint32_t tmem, long long r0, long long r1,
                                          uint32_t stage_bytes) {
   const uint32_t idesc = idesc_f16(1u /*bf16*/, 0u, QD, (uint32_t)a.tn);
-  long long it = 0;
+  int s = 0;
+  uint32_t ph = 0;
   int seg = 0;
   for (long long x = r0; x < r1; ++seg) {
     const int c0 = (int)(x % a.kc);
@@ -171,9 +204,7 @@ __device__ __forceinline__ void gemm_mma(const QCta& c, const GemmArgs& a, uint3
     if (!q_wait(c, QB_ACC_FREE + buf, ((uint32_t)(seg >> 1) & 1u) ^ 1u, QLOC_WAIT_ACC_FREE)) return;
     tc_fence_after();
     const uint32_t acc = tmem + (uint32_t)(buf * MAX_TN);
-    for (int ch = c0; ch < c1; ++ch, ++it) {
-      const int s = (int)(it % a.n_stages);
-      const uint32_t ph = (uint32_t)(it / a.n_stages) & 1u;
+    for (int ch = c0; ch < c1; ++ch) {
       if (!q_wait(c, QB_FULL + s, ph, QLOC_WAIT_FULL)) return;
       tc_fence_after();
       const uint32_t sa = c.base + s * stage_bytes;
@@ -182,6 +213,7 @@ __device__ __forceinline__ void gemm_mma(const QCta& c, const GemmArgs& a, uint3
       for (int ks = 0; ks < BK / 16; ++ks)
         mma_ss(acc, ad + 2u * ks, bd + 2u * ks, idesc, (ch > c0 || ks > 0) ? 1u : 0u);
       tc_commit(c.bar(QB_FREE + s));
+      if (++s == a.n_stages) { s = 0; ph ^= 1u; }
     }
     tc_commit(c.bar(QB_ACC_FULL + buf));
     x += c1 - c0;
@@ -241,18 +273,42 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (*flag) {
         __threadfence();
+        // four features per thread, four token rows per pass of the 128 threads; the loads of eight
+        // passes (32 tokens) are issued together so that the tile costs a few memory round trips
         const long long x_lo = (long long)tile * a.kc, x_hi = x_lo + a.kc;
         const int j_lo = cta_of(a, x_lo), j_hi = cta_of(a, x_hi - 1);
-        for (int t = 0; t < nt; ++t) {
-          float sum = 0.f;
-          for (int j = j_lo; j <= j_hi; ++j) {
+        const int f4 = (et & 31) * 4, tr = et >> 5;
+        for (int tb = 0; tb < nt; tb += 32) {
+          float4 acc[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int j = j_lo; j <= j_hi; ++j) {       // ascending CTA order: a fixed summation order
             const long long s0 = range_start(a, j), s1 = range_start(a, j + 1);
-            if (s1 <= s0) continue;               // a CTA without work
-            const int slot = (s0 >= x_lo) ? 0 : 1;   // the tile holds its first segment, or its last
-            const float* p = a.ws + ((size_t)j * 2 + slot) * (size_t)(MAX_TN * QD);
-            sum += __ldcg(p + (size_t)t * QD + f);
+            if (s1 <= s0) continue;                 // a CTA without work
+            const int slot = (s0 >= x_lo) ? 0 : 1;  // the tile holds its first segment, or its last
+            const float* p = a.ws + ((size_t)j * 2 + slot) * (size_t)(MAX_TN * QD) + f4;
+            float4 v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int t = tb + tr + 4 * i;
+              v[i] = (t < nt) ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)t * QD)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              acc[i].x += v[i].x; acc[i].y += v[i].y; acc[i].z += v[i].z; acc[i].w += v[i].w;
+            }
           }
-          out_row(a, ft, t0 + t)[f] = __float2bfloat16_rn(sum);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int t = tb + tr + 4 * i;
+            if (t < nt) {
+              __nv_bfloat162 lo = __floats2bfloat162_rn(acc[i].x, acc[i].y), hi = __floats2bfloat162_rn(acc[i].z, acc[i].w);
+              uint2 o;
+              o.x = *reinterpret_cast<uint32_t*>(&lo);
+              o.y = *reinterpret_cast<uint32_t*>(&hi);
+              *reinterpret_cast<uint2*>(out_row(a, ft, t0 + t) + f4) = o;
+            }
+          }
         }
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");   // the flag word is reused by the next segment
@@ -276,6 +332,9 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = QLOC_SMEM_ALIGN;
     return;
   }
+  const long long r0 = range_start(a, blockIdx.x), r1 = range_start(a, blockIdx.x + 1);
+  const uint32_t stage_bytes = A_BYTES + (uint32_t)a.tn * 128u;
+  int early = 0;
   if (tid == 0) {
     prefetch_map(&w_map);
     prefetch_map(&x_map);
@@ -284,6 +343,12 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     words[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
+    // the weights do not depend on the kernel before this one: fill the ring with W tiles right away
+    // (the X^ tiles of the same stages follow after the wait below)
+    early = (int)min((long long)a.n_stages, r1 - r0);
+    ChunkCursor k;
+    k.init(a, r0);
+    for (int it = 0; it < early; ++it, k.next(a)) load_chunk(c, &w_map, &x_map, a, k, stage_bytes, true, false);
   }
   __syncwarp();
   if (warp == 0) {
@@ -298,10 +363,8 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
   // the operand rows X^ come from the kernel launched before this one
   grid_dependency_wait();
 
-  const long long r0 = range_start(a, blockIdx.x), r1 = range_start(a, blockIdx.x + 1);
-  const uint32_t stage_bytes = A_BYTES + (uint32_t)a.tn * 128u;
   if (warp == 0) {
-    if (tid == 0) gemm_producer(c, &w_map, &x_map, a, r0, r1, stage_bytes);
+    if (tid == 0) gemm_producer(c, &w_map, &x_map, a, r0, r1, stage_bytes, early);
   } else if (warp == 1) {
     if (tid == 32) gemm_mma(c, a, tmem, r0, r1, stage_bytes);
   } else {
@@ -313,6 +376,19 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
   __syncthreads();
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+}
+
+// W [rows][d_model] -> tile order [rows / 128][d_model / 64][128][64]: every (feature tile, k chunk)
+// operand tile becomes one contiguous 16 KB run, so that the projection streams W from HBM in
+// whole DRAM pages instead of 128-byte pieces a row pitch apart.  Runs once, at create.
+__global__ void qkv_pack_w_kernel(const uint4* __restrict__ w, uint4* __restrict__ wp, int rows, int d_model) {
+  const int per_row = d_model / 8;                       // 16-byte pieces per row
+  const size_t n = (size_t)rows * per_row;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / per_row), p = (int)(i % per_row);
+    const int ft = r / QD, rr = r % QD, ch = p / 8, pp = p % 8;
+    wp[(((size_t)ft * (d_model / BK) + ch) * QD + rr) * 8 + pp] = w[i];
   }
 }
 
@@ -333,8 +409,12 @@ struct NormArgs {
 };
 
 __global__ void __launch_bounds__(N_THREADS) qkv_norm_kernel(const NormArgs a) {
-  // the projection kernel may be scheduled now: it waits for this grid before it reads X^
+  // The projection kernel may be scheduled now: before it waits for this grid it only sets itself up
+  // and starts fetching weights.  This kernel is itself launched programmatically dependent and waits,
+  // before its first load, for everything enqueued ahead of it (whatever wrote the token ids or hidden
+  // states included); the projection kernel's own wait then covers all of that as well.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  grid_dependency_wait();
   __shared__ float red[N_THREADS / 32];
   const int t = blockIdx.x;
   const int tid = threadIdx.x;
@@ -451,7 +531,7 @@ bool make_bf16_map(lacache_qkv* p, CUtensorMap* m, const void* base, int rows, i
 void qkv_free(lacache_qkv* p) {
   if (!p) return;
   cudaDeviceSynchronize();
-  void* bufs[] = {p->xhat, p->ws, p->counters, p->status, p->q, p->k, p->v};
+  void* bufs[] = {p->w_packed, p->xhat, p->ws, p->counters, p->status, p->q, p->k, p->v};
   for (void* b : bufs)
     if (b) cudaFree(b);
   delete p;
@@ -519,7 +599,14 @@ lacache_status lacache_qkv_create(const lacache_qkv_config* cfg, lacache_qkv** o
     QCU_TRY(p, cudaMalloc(&p->q, (size_t)cfg->max_tokens * cfg->n_q_heads * QD * 2));
     QCU_TRY(p, cudaMalloc(&p->k, (size_t)cfg->max_tokens * cfg->n_kv_heads * QD * 2));
     QCU_TRY(p, cudaMalloc(&p->v, (size_t)cfg->max_tokens * cfg->n_kv_heads * QD * 2));
-    if (!make_bf16_map(p, &p->w_map, cfg->w_qkv, p->n_ftiles * QD, cfg->d_model, QD)) return LACACHE_ERR_CUDA;
+    const int w_rows = p->n_ftiles * QD;
+    QCU_TRY(p, cudaMalloc(&p->w_packed, (size_t)w_rows * d * 2));
+    qkv_pack_w_kernel<<<p->num_sms * 8, 256>>>(reinterpret_cast<const uint4*>(cfg->w_qkv),
+                                               reinterpret_cast<uint4*>(p->w_packed), w_rows, cfg->d_model);
+    QCU_TRY(p, cudaGetLastError());
+    QCU_TRY(p, cudaDeviceSynchronize());
+    // the packed copy as a matrix of 64 columns: a tile is 128 consecutive rows
+    if (!make_bf16_map(p, &p->w_map, p->w_packed, w_rows * (cfg->d_model / BK), BK, QD)) return LACACHE_ERR_CUDA;
     for (int i = 0; i < 4; ++i)
       if (!make_bf16_map(p, &p->x_map[i], p->xhat, p->tokens_pad, cfg->d_model, 32 << i)) return LACACHE_ERR_CUDA;
     QCU_TRY(p, cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMQ_TOTAL));
@@ -567,8 +654,19 @@ lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, con
   na.vocab = p->cfg.vocab;
   na.eps = p->cfg.rms_eps;
   na.status = p->status;
-  qkv_norm_kernel<<<n_tokens, N_THREADS, 0, s>>>(na);
-  QCU_TRY(p, cudaGetLastError());
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  const bool no_pdl = getenv("LACACHE_NO_PDL") != nullptr;
+  {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_tokens);
+    cfg.blockDim = dim3(N_THREADS);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = no_pdl ? 0 : 1;
+    QCU_TRY(p, cudaLaunchKernelEx(&cfg, qkv_norm_kernel, na));
+  }
   p->last_launches++;
 
   GemmArgs ga{};
@@ -596,11 +694,8 @@ lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, con
   cfg.blockDim = dim3(G_THREADS);
   cfg.dynamicSmemBytes = SMQ_TOTAL;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = getenv("LACACHE_NO_PDL") ? 0 : 1;
+  cfg.numAttrs = no_pdl ? 0 : 1;
   if (p->ev_start && p->ev_stop) {
     cfg.numAttrs = 0;   // an event between the two kernels: an ordinary launch
     QCU_TRY(p, cudaEventRecord(p->ev_start, s));
