@@ -627,9 +627,9 @@ lacache_status step_impl(lacache_ctx* c, const void* q, const void* k, const voi
     r.row_cos = c->d_blk_cos + row0 * (c->g.d / 2);
     r.row_sin = c->d_blk_sin + row0 * (c->g.d / 2);
   }
-  // may start while the previous step's attention kernel drains (it waits before its stores), unless
-  // the kernel before it in the stream is the one that writes its inputs
-  r.pdl = inputs_just_written ? 0 : 1;
+  // may start while the previous step's attention kernel drains (it waits before its stores); when
+  // the kernel before it in the stream is the one that writes its inputs, it waits for that one first
+  r.pdl = inputs_just_written ? 2 : 1;
   r.dst = c->rot;
   r.in_dtype = c->cfg.dtype;
   CU_TRY(c, rope_write(c->g, r, c->engine, s));

@@ -80,8 +80,9 @@ struct RopeArgs {
   const int32_t* row_tok; const float* row_cos; const float* row_sin;  // [n_src_rows], [n_src_rows][d/2]
   RotBuffers dst;
   int in_dtype;
-  // launch programmatically dependent on the kernel before it in the stream (a step's attention
-  // kernel lets its successors start early): the kernel then waits before its first store
+  // launch programmatically dependent on the kernel before it in the stream.  1: that kernel is a
+  // step's attention kernel, which lets its successors start early; this kernel then waits before its
+  // first store.  2: that kernel writes this kernel's inputs; this kernel waits before anything else.
   int pdl;
 };
 

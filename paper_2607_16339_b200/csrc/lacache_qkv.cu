@@ -278,24 +278,55 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
         const long long x_lo = (long long)tile * a.kc, x_hi = x_lo + a.kc;
         const int j_lo = cta_of(a, x_lo), j_hi = cta_of(a, x_hi - 1);
         const int f4 = (et & 31) * 4, tr = et >> 5;
+        // the tile's parts in ascending CTA order (a fixed summation order); with up to three of them,
+        // the usual case, the loads of all parts are in flight together
+        const float *p0 = nullptr, *p1 = nullptr, *p2 = nullptr;
+        int n_parts = 0;
+        for (int j = j_lo; j <= j_hi; ++j) {
+          const long long s0 = range_start(a, j), s1 = range_start(a, j + 1);
+          if (s1 <= s0) continue;                   // a CTA without work
+          const int slot = (s0 >= x_lo) ? 0 : 1;    // the tile holds its first segment, or its last
+          const float* p = a.ws + ((size_t)j * 2 + slot) * (size_t)(MAX_TN * QD) + f4;
+          if (n_parts == 0) p0 = p; else if (n_parts == 1) p1 = p; else if (n_parts == 2) p2 = p;
+          ++n_parts;
+        }
+        const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int tb = 0; tb < nt; tb += 32) {
           float4 acc[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-          for (int j = j_lo; j <= j_hi; ++j) {       // ascending CTA order: a fixed summation order
-            const long long s0 = range_start(a, j), s1 = range_start(a, j + 1);
-            if (s1 <= s0) continue;                 // a CTA without work
-            const int slot = (s0 >= x_lo) ? 0 : 1;  // the tile holds its first segment, or its last
-            const float* p = a.ws + ((size_t)j * 2 + slot) * (size_t)(MAX_TN * QD) + f4;
-            float4 v[8];
+          if (n_parts <= 3) {
+            float4 v0[8], v1[8], v2[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               const int t = tb + tr + 4 * i;
-              v[i] = (t < nt) ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)t * QD)) : make_float4(0.f, 0.f, 0.f, 0.f);
+              const size_t o = (size_t)t * QD;
+              v0[i] = (t < nt) ? __ldcg(reinterpret_cast<const float4*>(p0 + o)) : zero4;
+              v1[i] = (t < nt && n_parts > 1) ? __ldcg(reinterpret_cast<const float4*>(p1 + o)) : zero4;
+              v2[i] = (t < nt && n_parts > 2) ? __ldcg(reinterpret_cast<const float4*>(p2 + o)) : zero4;
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-              acc[i].x += v[i].x; acc[i].y += v[i].y; acc[i].z += v[i].z; acc[i].w += v[i].w;
+              acc[i].x = 0.f + v0[i].x; acc[i].y = 0.f + v0[i].y; acc[i].z = 0.f + v0[i].z; acc[i].w = 0.f + v0[i].w;
+              if (n_parts > 1) { acc[i].x += v1[i].x; acc[i].y += v1[i].y; acc[i].z += v1[i].z; acc[i].w += v1[i].w; }
+              if (n_parts > 2) { acc[i].x += v2[i].x; acc[i].y += v2[i].y; acc[i].z += v2[i].z; acc[i].w += v2[i].w; }
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = zero4;
+            for (int j = j_lo; j <= j_hi; ++j) {
+              const long long s0 = range_start(a, j), s1 = range_start(a, j + 1);
+              if (s1 <= s0) continue;
+              const int slot = (s0 >= x_lo) ? 0 : 1;
+              const float* p = a.ws + ((size_t)j * 2 + slot) * (size_t)(MAX_TN * QD) + f4;
+              float4 v[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int t = tb + tr + 4 * i;
+                v[i] = (t < nt) ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)t * QD)) : zero4;
+              }
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                acc[i].x += v[i].x; acc[i].y += v[i].y; acc[i].z += v[i].z; acc[i].w += v[i].w;
+              }
             }
           }
 #pragma unroll
@@ -323,6 +354,9 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
+  // a kernel launched programmatically dependent on this one may be scheduled now (it has to wait
+  // for this grid before it touches anything this grid writes)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   QCta c;
   c.base = smem_u32(smem_raw);
   uint32_t* words = reinterpret_cast<uint32_t*>(smem_raw + SMQ_BAR + 8 * QB_N);  // [0] tmem, [1] abort, [2] flag

@@ -45,6 +45,9 @@ __global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a)
   // the attention kernel that follows may be launched programmatically
   // dependent: let it start its prologue now (it waits for this grid's writes
   // before it touches them)
+  // (when the kernel before this one writes this kernel's inputs, they are complete only after the
+  // wait, and the attention kernel, which also reads them early, must not start before that)
+  if (a.pdl == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int chunks = g.d / 16;
   const int slots = g.Hq + 2 * g.Hkv;
