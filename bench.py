@@ -486,7 +486,7 @@ def run_cuda(args):
 # the step fed by token ids: embedding gather + RMS norm + Q/K/V projection in front
 # ----------------------------------------------------------------------------
 D_MODEL = {32: 4096, 28: 3584}     # first-layer width of the model a workload is shaped like, by query heads
-QKV_TRAFFIC_PER_LAUNCH = {2: 105807872}   # ncu, profiles/qkv_gemm_kernel_llada_n32_ncu.txt
+QKV_TRAFFIC_PER_LAUNCH = {2: 104626944}   # ncu, profiles/qkv_gemm_kernel_cfg2_step_ncu_full.txt
 
 
 def token_path_leg(wl, dev, peaks, seed, n_steps):
@@ -494,6 +494,7 @@ def token_path_leg(wl, dev, peaks, seed, n_steps):
     event-timed duration of its projection kernel, which is bound by reading the stacked
     Q/K/V weight once per step.  Weight and cache-state replicas are visited round-robin so
     that every call finds them in HBM."""
+    import numpy as np
     import torch
     from paper_2607_16339_b200 import binding
     from paper_2607_16339_b200.workloads import TokenModel
@@ -521,6 +522,19 @@ def token_path_leg(wl, dev, peaks, seed, n_steps):
         ctxs[i % R].build_tokens(prods[i % R], blk, token_ids=ids_full)
     e1.record(); torch.cuda.synchronize()
     build_us = e0.elapsed_time(e1) / (2 * R) * 1e3
+    # the build of the next block that re-projects only the block just finished
+    rows_prev = torch.from_numpy(np.concatenate(
+        [wl.cu_seqlens[s] + P + (blk - 1) * wl.block_len + np.arange(wl.block_len)
+         for s, P in enumerate(wl.prompt_lens)]).astype("int32")).to(dev)
+    ids_prev = ids_full[rows_prev.long()].contiguous()
+    for c in range(R):
+        ctxs[c].build_tokens_update(prods[c], blk, rows_prev, token_ids=ids_prev)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(2 * R):
+        ctxs[i % R].build_tokens_update(prods[i % R], blk, rows_prev, token_ids=ids_prev)
+    e1.record(); torch.cuda.synchronize()
+    update_us = e0.elapsed_time(e1) / (2 * R) * 1e3
     launches = 0
     for i in range(16):
         ctxs[i % R].step_tokens(prods[i % R], out, lse, blk_token_ids=ids_blk[i % S])
@@ -552,7 +566,8 @@ def token_path_leg(wl, dev, peaks, seed, n_steps):
                 "-> RoPE + cached attention; synthetic first-layer weights",
         "d_model": d_model, "tokens_per_step": nb, "replicas": R,
         "value": round(1e6 / step_us, 1), "unit": UNIT, "step_us": round(step_us, 2),
-        "build_tokens_us": round(build_us, 1), "gpu_launches": launches, "steps": n_steps,
+        "build_tokens_us": round(build_us, 1), "build_tokens_update_us": round(update_us, 1),
+        "gpu_launches": launches, "steps": n_steps,
         "roofline": {"kernel": "qkv_gemm_kernel (one step: %d tokens x %d -> %d features)" % (nb, d_model, w0.shape[0]),
                      "bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": round(ach / peaks["hbm_gbs"], 4), "peak_source": peaks["source"],

@@ -121,9 +121,25 @@ lacache_status lacache_build(lacache_ctx* ctx, int block_idx, const void* q_pre,
  * kernels are launched programmatically dependent and store nothing before the
  * first call's kernels have completed); q_blk / k_blk / v_blk must stay
  * unchanged until the call's work has completed, as for any stream-ordered call.
+ *
+ * Because of that overlap a step reads q_blk / k_blk / v_blk EARLY: possibly
+ * before the operation enqueued just ahead of it has flushed its writes.  That
+ * is safe when the three tensors were complete before the previous
+ * lacache_step of this context was enqueued (precomputed inputs), or were
+ * written by work enqueued on another stream and joined by an event.  When
+ * they are written by work enqueued on the SAME stream between two steps (a
+ * projection kernel run before every step), switch the overlap off with
+ * lacache_set_step_overlap(ctx, 0): every kernel of a step is then ordered
+ * after all earlier work of the stream, as an ordinary launch is.
+ * lacache_step_tokens, which runs such a producer itself, orders its kernels
+ * correctly whatever this setting.
  */
 lacache_status lacache_step(lacache_ctx* ctx, const void* q_blk, const void* k_blk,
                             const void* v_blk, float* out, float* lse, void* cuda_stream);
+
+/* Overlap of consecutive lacache_step calls on the device (see lacache_step): on (non-zero,
+ * the default) or off.  No paper counterpart. */
+lacache_status lacache_set_step_overlap(lacache_ctx* ctx, int enable);
 
 /*
  * Plain attention for all rows over all keys (the definition in Sec. 3.3.3 /
@@ -254,6 +270,26 @@ lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, con
 lacache_status lacache_build_tokens(lacache_ctx* ctx, lacache_qkv* p, int block_idx,
                                     const int32_t* token_ids, const void* hidden,
                                     void* cuda_stream);
+/*
+ * The build of the next block, re-projecting only what changed.  Token-wise results depend on the
+ * token alone (Sec. 3.3.2), so from one block to the next only the tokens whose ids changed need
+ * the embedding, norm and projections again: as a rule the B * L_b tokens of the block just
+ * finished, now decoded.  The producer keeps the pre-rotation rows of all T tokens from the last
+ * lacache_build_tokens / _update of this (ctx, p) pair; this call projects the n_changed tokens
+ * listed in `rows` (DEVICE int32 [n_changed], distinct packed token indices in [0, T)) from
+ * token_ids [n_changed] or hidden [n_changed, d_model], stores them at those rows, and runs
+ * lacache_build on the complete set.  Tokens not listed must be unchanged since that call.
+ * LACACHE_ERR_STATE without such a preceding call (another context's lacache_build_tokens with the
+ * same producer in between invalidates it).  A row outside [0, T) is reported by
+ * lacache_qkv_poll_status and dropped.  n_changed == 0 just rebuilds.
+ * Rows that are not re-projected keep their bits.  A re-projected row can differ in the last bf16
+ * place, in a few elements, from what a projection of all T tokens gives for it: the reduction over
+ * d_model is split over the SMs differently for a different token count, so the fp32 sums round
+ * differently; both are within one unit of the exactly rounded value.
+ */
+lacache_status lacache_build_tokens_update(lacache_ctx* ctx, lacache_qkv* p, int block_idx,
+                                           const int32_t* rows, const int32_t* token_ids,
+                                           const void* hidden, int n_changed, void* cuda_stream);
 lacache_status lacache_step_tokens(lacache_ctx* ctx, lacache_qkv* p, const int32_t* blk_token_ids,
                                    const void* blk_hidden, float* out, float* lse,
                                    void* cuda_stream);

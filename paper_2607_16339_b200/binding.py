@@ -24,7 +24,8 @@ EXPORTS = [
     "lacache_full_recompute_static", "lacache_poll_status", "lacache_last_error",
     "lacache_qkv_create", "lacache_qkv_destroy", "lacache_qkv_project", "lacache_build_tokens",
     "lacache_step_tokens", "lacache_qkv_set_timing_events", "lacache_qkv_last_launch_count",
-    "lacache_qkv_poll_status", "lacache_qkv_last_error",
+    "lacache_qkv_poll_status", "lacache_qkv_last_error", "lacache_set_step_overlap",
+    "lacache_build_tokens_update",
 ]
 
 
@@ -79,6 +80,7 @@ def load():
     lib.lacache_export_rope_cache.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_export_index_meta.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_set_timing_events.argtypes = [vp, vp, vp]
+    lib.lacache_set_step_overlap.argtypes = [vp, ip]
     lib.lacache_full_recompute_static.argtypes = [ip, ip, ip, ip, ip, ctypes.c_float, ctypes.c_float, vp, vp, vp, vp,
                                                   vp, vp]
     lib.lacache_total_tokens.argtypes = [vp]
@@ -92,6 +94,7 @@ def load():
     lib.lacache_qkv_project.argtypes = [vp, vp, vp, ip, vp, vp, vp, vp, vp]
     lib.lacache_build_tokens.argtypes = [vp, vp, ip, vp, vp, vp]
     lib.lacache_step_tokens.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.lacache_build_tokens_update.argtypes = [vp, vp, ip, vp, vp, vp, ip, vp]
     lib.lacache_qkv_set_timing_events.argtypes = [vp, vp, vp]
     lib.lacache_qkv_last_launch_count.argtypes = [vp]
     lib.lacache_qkv_poll_status.argtypes = [vp]
@@ -214,9 +217,17 @@ class Context:
         self._check(self._lib.lacache_export_index_meta(self._h, p(seq), p(pos), p(isb), p(kvh)))
         return seq, pos, isb, kvh
 
+    def set_step_overlap(self, enable):
+        self._check(self._lib.lacache_set_step_overlap(self._h, int(bool(enable))))
+
     def build_tokens(self, producer, block_idx, token_ids=None, hidden=None, stream=None):
         self._check(self._lib.lacache_build_tokens(self._h, producer._h, int(block_idx), _ptr(token_ids),
                                                    _ptr(hidden), _stream(stream)))
+
+    def build_tokens_update(self, producer, block_idx, rows, token_ids=None, hidden=None, stream=None):
+        self._check(self._lib.lacache_build_tokens_update(self._h, producer._h, int(block_idx), _ptr(rows),
+                                                          _ptr(token_ids), _ptr(hidden), int(rows.shape[0]),
+                                                          _stream(stream)))
 
     def step_tokens(self, producer, out, lse=None, blk_token_ids=None, blk_hidden=None, stream=None):
         self._check(self._lib.lacache_step_tokens(self._h, producer._h, _ptr(blk_token_ids), _ptr(blk_hidden),

@@ -56,6 +56,7 @@ struct lacache_ctx {
   float *hs_out = nullptr, *hs_lse = nullptr;
 
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
+  int step_overlap = 1;   // consecutive steps may overlap on the device
   int built_block = -1;
   int last_launches = 0;
   int device = 0;
@@ -580,11 +581,37 @@ lacache_status lacache_build_tokens(lacache_ctx* c, lacache_qkv* p, int block_id
   lacache_status st = check_producer(c, p, c->g.T);
   if (st != LACACHE_OK) return st;
   void *q, *k, *v;
-  qkv_scratch(p, &q, &k, &v);
+  qkv_scratch(p, false, &q, &k, &v);
+  qkv_set_full_owner(p, nullptr, 0);
   st = lacache_qkv_project(p, token_ids, hidden, c->g.T, q, k, v, nullptr, stream);
   if (st != LACACHE_OK) return fail(c, st, "producer: %s", lacache_qkv_last_error(p));
   st = lacache_build(c, block_idx, q, k, v, stream);
-  if (st == LACACHE_OK) c->last_launches += lacache_qkv_last_launch_count(p);
+  if (st != LACACHE_OK) return st;
+  qkv_set_full_owner(p, c, c->g.T);
+  c->last_launches += lacache_qkv_last_launch_count(p);
+  return LACACHE_OK;
+}
+
+lacache_status lacache_build_tokens_update(lacache_ctx* c, lacache_qkv* p, int block_idx, const int32_t* rows,
+                                           const int32_t* token_ids, const void* hidden, int n_changed,
+                                           void* stream) {
+  if (!c || !p) return LACACHE_ERR_INVALID_ARG;
+  if (n_changed < 0 || n_changed > c->g.T) return fail(c, LACACHE_ERR_SHAPE, "n_changed %d outside [0, %d]", n_changed, c->g.T);
+  lacache_status st = check_producer(c, p, c->g.T);
+  if (st != LACACHE_OK) return st;
+  if (!qkv_full_owner_is(p, c, c->g.T))
+    return fail(c, LACACHE_ERR_STATE, "lacache_build_tokens_update needs a preceding lacache_build_tokens of this context with this producer");
+  if (n_changed > 0 && !rows) return fail(c, LACACHE_ERR_INVALID_ARG, "NULL rows");
+  void *q, *k, *v;
+  qkv_scratch(p, false, &q, &k, &v);
+  int producer_launches = 0;
+  if (n_changed > 0) {
+    st = qkv_project_rows(p, token_ids, hidden, n_changed, q, k, v, nullptr, rows, c->g.T, stream);
+    if (st != LACACHE_OK) return fail(c, st, "producer: %s", lacache_qkv_last_error(p));
+    producer_launches = lacache_qkv_last_launch_count(p);
+  }
+  st = lacache_build(c, block_idx, q, k, v, stream);
+  if (st == LACACHE_OK) c->last_launches += producer_launches;
   return st;
 }
 
@@ -596,7 +623,7 @@ lacache_status lacache_step_tokens(lacache_ctx* c, lacache_qkv* p, const int32_t
   lacache_status st = check_producer(c, p, n);
   if (st != LACACHE_OK) return st;
   void *q, *k, *v;
-  qkv_scratch(p, &q, &k, &v);
+  qkv_scratch(p, true, &q, &k, &v);
   st = lacache_qkv_project(p, blk_token_ids, blk_hidden, n, q, k, v, nullptr, stream);
   if (st != LACACHE_OK) return fail(c, st, "producer: %s", lacache_qkv_last_error(p));
   st = step_impl(c, q, k, v, out, lse, stream, true);
@@ -629,13 +656,14 @@ lacache_status step_impl(lacache_ctx* c, const void* q, const void* k, const voi
   }
   // may start while the previous step's attention kernel drains (it waits before its stores); when
   // the kernel before it in the stream is the one that writes its inputs, it waits for that one first
-  r.pdl = inputs_just_written ? 2 : 1;
+  const bool overlap = c->step_overlap && !getenv("LACACHE_NO_PDL") && !getenv("LACACHE_NO_STEP_OVERLAP");
+  r.pdl = inputs_just_written ? 2 : (overlap ? 1 : 0);
   r.dst = c->rot;
   r.in_dtype = c->cfg.dtype;
   CU_TRY(c, rope_write(c->g, r, c->engine, s));
   c->last_launches++;
   AttnArgs a = attn_args(c, MODE_STEP, c->step_list[blk], blk, c->rot, out, lse);
-  a.step_overlap = (getenv("LACACHE_NO_PDL") || getenv("LACACHE_NO_STEP_OVERLAP")) ? 0 : 1;
+  a.step_overlap = overlap ? 1 : 0;
   if (!getenv("LACACHE_NO_QCOMP")) {
     a.q_raw = q;
     a.k_raw = k;
@@ -647,6 +675,12 @@ lacache_status step_impl(lacache_ctx* c, const void* q, const void* k, const voi
   return run_attention(c, a, false, s);
 }
 }  // namespace
+
+lacache_status lacache_set_step_overlap(lacache_ctx* c, int enable) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  c->step_overlap = enable ? 1 : 0;
+  return LACACHE_OK;
+}
 
 lacache_status lacache_full_recompute(lacache_ctx* c, const void* q, const void* k, const void* v, float* out,
                                       float* lse, void* stream) {

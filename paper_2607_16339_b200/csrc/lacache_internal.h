@@ -139,8 +139,14 @@ void tc_free_maps(TcMaps* m);
 
 // token-wise producer (lacache_qkv.cu): the scratch rows the *_tokens entry points project into,
 // and its head configuration (returns head_dim)
-void qkv_scratch(lacache_qkv* p, void** q, void** k, void** v);
+void qkv_scratch(lacache_qkv* p, bool block, void** q, void** k, void** v);
 int qkv_heads(const lacache_qkv* p, int* hq, int* hkv, int* max_tokens);
+// lacache_qkv_project with a scatter: input token t is written to output row dst_rows[t] (null: t)
+lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const void* hidden, int n_tokens, void* q,
+                                void* k, void* v, void* h_out, const int32_t* dst_rows, int max_rows, void* stream);
+// which context's tokens the all-token scratch holds (set by a full projection)
+void qkv_set_full_owner(lacache_qkv* p, const void* ctx, int n_tokens);
+bool qkv_full_owner_is(const lacache_qkv* p, const void* ctx, int n_tokens);
 
 constexpr int SIMT_ROWS = 32;    // query rows per SIMT work item
 constexpr int TC_ROWS = 128;     // query rows per tcgen05 work item

@@ -45,7 +45,12 @@ struct lacache_qkv {
   float* ws = nullptr;                  // [2 * num_sms][256 * 128] partial tiles
   int* counters = nullptr;              // per tile: chunks accumulated so far
   int32_t* status = nullptr;
-  __nv_bfloat16 *q = nullptr, *k = nullptr, *v = nullptr;   // [max_tokens][H][128] scratch of the *_tokens calls
+  // scratch of the *_tokens calls, [max_tokens][H][128] each: the projections of all tokens (kept from
+  // one build to the next, so that a build re-projects only the tokens that changed) and of a block
+  __nv_bfloat16 *q = nullptr, *k = nullptr, *v = nullptr;
+  __nv_bfloat16 *qb = nullptr, *kb = nullptr, *vb = nullptr;
+  const void* full_owner = nullptr;     // the context whose tokens q / k / v currently hold
+  int full_tokens = 0;
   CUtensorMap w_map;
   CUtensorMap x_map[4];                 // boxes of 32, 64, 128, 256 tokens
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
@@ -73,7 +78,7 @@ constexpr uint32_t SMQ_TOTAL = SMQ_BAR + 8 * QB_N + 32;
 static_assert(SMQ_TOTAL <= 232448, "exceeds the 227 KB per-CTA limit");
 constexpr long long Q_WAIT_CYCLES = 4000000000ll;  // ~2 s
 enum { QLOC_SMEM_ALIGN = 101, QLOC_WAIT_FULL = 102, QLOC_WAIT_FREE = 103, QLOC_WAIT_ACC_FULL = 104,
-       QLOC_WAIT_ACC_FREE = 105, QLOC_TOKEN_ID = 106 };
+       QLOC_WAIT_ACC_FREE = 105, QLOC_TOKEN_ID = 106, QLOC_ROW = 107 };
 
 struct GemmArgs {
   int n_tokens, tn, n_ttiles, n_tiles, kc;   // kc = d_model / 64 chunks per tile
@@ -81,6 +86,8 @@ struct GemmArgs {
   int n_stages;
   int Hq, Hkv;
   __nv_bfloat16 *q, *k, *v;
+  const int32_t* dst_rows;   // output row of input token t (null: t); rows outside [0, max_rows) are dropped
+  int max_rows;
   float* ws;
   int* counters;
   int32_t* status;
@@ -133,8 +140,12 @@ __device__ __forceinline__ int cta_of(const GemmArgs& a, long long x) {
   return (int)(((x + 1) * (long long)gridDim.x - 1) / a.total_chunks);
 }
 
-// destination of feature tile ft, token t: row of q, k or v
+// destination of feature tile ft, input token t: a row of q, k or v (null: the row is dropped)
 __device__ __forceinline__ __nv_bfloat16* out_row(const GemmArgs& a, int ft, int t) {
+  if (a.dst_rows) {
+    t = __ldg(a.dst_rows + t);
+    if ((unsigned)t >= (unsigned)a.max_rows) return nullptr;   // reported by the norm kernel
+  }
   if (ft < a.Hq) return a.q + ((size_t)t * a.Hq + ft) * QD;
   if (ft < a.Hq + a.Hkv) return a.k + ((size_t)t * a.Hkv + (ft - a.Hq)) * QD;
   return a.v + ((size_t)t * a.Hkv + (ft - a.Hq - a.Hkv)) * QD;
@@ -248,7 +259,10 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const int t = g * 32 + i;
-          if (t < nt) out_row(a, ft, t0 + t)[f] = __float2bfloat16_rn(__uint_as_float(r[i]));
+          if (t < nt) {
+            __nv_bfloat16* dst = out_row(a, ft, t0 + t);
+            if (dst) dst[f] = __float2bfloat16_rn(__uint_as_float(r[i]));
+          }
         }
       } else {
 #pragma unroll
@@ -337,7 +351,8 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
               uint2 o;
               o.x = *reinterpret_cast<uint32_t*>(&lo);
               o.y = *reinterpret_cast<uint32_t*>(&hi);
-              *reinterpret_cast<uint2*>(out_row(a, ft, t0 + t) + f4) = o;
+              __nv_bfloat16* dst = out_row(a, ft, t0 + t);
+              if (dst) *reinterpret_cast<uint2*>(dst + f4) = o;
             }
           }
         }
@@ -437,6 +452,8 @@ struct NormArgs {
   const __nv_bfloat16* weight;    // [d_model]
   __nv_bfloat16* xhat;            // [n][d_model]
   __nv_bfloat16* h_out;           // [n][d_model] or null
+  const int32_t* dst_rows;        // or null; checked against max_rows here
+  int max_rows;
   int d_model, vocab;
   float eps;
   int32_t* status;
@@ -454,6 +471,14 @@ __global__ void __launch_bounds__(N_THREADS) qkv_norm_kernel(const NormArgs a) {
   const int tid = threadIdx.x;
   const __nv_bfloat16* src;
   bool valid = true;
+  if (a.dst_rows && tid == 0) {
+    const int row = a.dst_rows[t];
+    if ((unsigned)row >= (unsigned)a.max_rows && atomicCAS(a.status, 0, (int)LACACHE_ERR_INVALID_ARG) == 0) {
+      a.status[1] = QLOC_ROW;
+      a.status[2] = t;
+      a.status[3] = row;
+    }
+  }
   if (a.ids) {
     const int id = a.ids[t];
     valid = id >= 0 && id < a.vocab;
@@ -565,7 +590,7 @@ bool make_bf16_map(lacache_qkv* p, CUtensorMap* m, const void* base, int rows, i
 void qkv_free(lacache_qkv* p) {
   if (!p) return;
   cudaDeviceSynchronize();
-  void* bufs[] = {p->w_packed, p->xhat, p->ws, p->counters, p->status, p->q, p->k, p->v};
+  void* bufs[] = {p->w_packed, p->xhat, p->ws, p->counters, p->status, p->q, p->k, p->v, p->qb, p->kb, p->vb};
   for (void* b : bufs)
     if (b) cudaFree(b);
   delete p;
@@ -575,9 +600,13 @@ bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u)
 
 }  // namespace
 
-// scratch rows the *_tokens entry points project into
-void qkv_scratch(lacache_qkv* p, void** q, void** k, void** v) {
-  *q = p->q; *k = p->k; *v = p->v;
+// scratch rows the *_tokens entry points project into: all tokens of a context, or a block
+void qkv_scratch(lacache_qkv* p, bool block, void** q, void** k, void** v) {
+  *q = block ? p->qb : p->q; *k = block ? p->kb : p->k; *v = block ? p->vb : p->v;
+}
+void qkv_set_full_owner(lacache_qkv* p, const void* ctx, int n_tokens) { p->full_owner = ctx; p->full_tokens = n_tokens; }
+bool qkv_full_owner_is(const lacache_qkv* p, const void* ctx, int n_tokens) {
+  return p->full_owner == ctx && p->full_tokens == n_tokens;
 }
 int qkv_heads(const lacache_qkv* p, int* hq, int* hkv, int* max_tokens) {
   *hq = p->cfg.n_q_heads; *hkv = p->cfg.n_kv_heads; *max_tokens = p->cfg.max_tokens;
@@ -633,6 +662,9 @@ lacache_status lacache_qkv_create(const lacache_qkv_config* cfg, lacache_qkv** o
     QCU_TRY(p, cudaMalloc(&p->q, (size_t)cfg->max_tokens * cfg->n_q_heads * QD * 2));
     QCU_TRY(p, cudaMalloc(&p->k, (size_t)cfg->max_tokens * cfg->n_kv_heads * QD * 2));
     QCU_TRY(p, cudaMalloc(&p->v, (size_t)cfg->max_tokens * cfg->n_kv_heads * QD * 2));
+    QCU_TRY(p, cudaMalloc(&p->qb, (size_t)cfg->max_tokens * cfg->n_q_heads * QD * 2));
+    QCU_TRY(p, cudaMalloc(&p->kb, (size_t)cfg->max_tokens * cfg->n_kv_heads * QD * 2));
+    QCU_TRY(p, cudaMalloc(&p->vb, (size_t)cfg->max_tokens * cfg->n_kv_heads * QD * 2));
     const int w_rows = p->n_ftiles * QD;
     QCU_TRY(p, cudaMalloc(&p->w_packed, (size_t)w_rows * d * 2));
     qkv_pack_w_kernel<<<p->num_sms * 8, 256>>>(reinterpret_cast<const uint4*>(cfg->w_qkv),
@@ -664,6 +696,14 @@ lacache_status lacache_qkv_destroy(lacache_qkv* p) {
 
 lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, const void* hidden, int n_tokens,
                                    void* q, void* k, void* v, void* h_out, void* stream) {
+  return lacache::qkv_project_rows(p, token_ids, hidden, n_tokens, q, k, v, h_out, nullptr, 0, stream);
+}
+
+}  // extern "C"
+
+namespace lacache {
+lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const void* hidden, int n_tokens, void* q,
+                                void* k, void* v, void* h_out, const int32_t* dst_rows, int max_rows, void* stream) {
   if (!p) return LACACHE_ERR_INVALID_ARG;
   if ((token_ids == nullptr) == (hidden == nullptr))
     return qfail(p, LACACHE_ERR_INVALID_ARG, "pass exactly one of token_ids and hidden");
@@ -684,6 +724,8 @@ lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, con
   na.weight = reinterpret_cast<const __nv_bfloat16*>(p->cfg.norm_weight);
   na.xhat = p->xhat;
   na.h_out = reinterpret_cast<__nv_bfloat16*>(h_out);
+  na.dst_rows = dst_rows;
+  na.max_rows = max_rows;
   na.d_model = p->cfg.d_model;
   na.vocab = p->cfg.vocab;
   na.eps = p->cfg.rms_eps;
@@ -718,6 +760,8 @@ lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, con
   ga.q = reinterpret_cast<__nv_bfloat16*>(q);
   ga.k = reinterpret_cast<__nv_bfloat16*>(k);
   ga.v = reinterpret_cast<__nv_bfloat16*>(v);
+  ga.dst_rows = dst_rows;
+  ga.max_rows = max_rows;
   ga.ws = p->ws;
   ga.counters = p->counters;
   ga.status = p->status;
@@ -739,6 +783,9 @@ lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, con
   p->last_launches++;
   return LACACHE_OK;
 }
+}  // namespace lacache
+
+extern "C" {
 
 lacache_status lacache_qkv_set_timing_events(lacache_qkv* p, void* ev_start, void* ev_stop) {
   if (!p) return LACACHE_ERR_INVALID_ARG;
@@ -758,6 +805,8 @@ lacache_status lacache_qkv_poll_status(lacache_qkv* p) {
   QCU_TRY(p, cudaMemset(p->status, 0, 16));
   if (w[1] == QLOC_TOKEN_ID)
     return qfail(p, (lacache_status)w[0], "token id %d of input row %d is outside the embedding table", w[3], w[2]);
+  if (w[1] == QLOC_ROW)
+    return qfail(p, (lacache_status)w[0], "destination row %d of input row %d is out of range", w[3], w[2]);
   return qfail(p, (lacache_status)w[0], "device status %d at location %d (block %d, thread %d)", w[0], w[1], w[2], w[3]);
 }
 

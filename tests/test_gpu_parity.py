@@ -241,6 +241,38 @@ def test_back_to_back_steps_match_synchronised_steps(cfg):
         assert torch.equal(ref[-1][0], last[0][0]) and torch.equal(ref[-1][1], last[0][1])
 
 
+@pytest.mark.parametrize("cfg", [2, 5])
+def test_steps_fed_by_same_stream_writes_with_overlap_off(cfg):
+    """Block inputs that are written on the stream between two steps (here: copied into one reused
+    trio of buffers right before each step) with the cross-step overlap switched off: every kernel
+    of a step is then ordered after the copy.  Bit for bit what synchronised steps give."""
+    wl = WORKLOADS[cfg]
+    S = min(wl.steps_per_block, 5)
+    sch = SyntheticSchedule(wl, seed=33)
+    q, k, v = (to_dev(a, wl) for a in sch.begin_block(0))
+    steps = [tuple(to_dev(a, wl) for a in sch.draw_step(0, s)) for s in range(1, S + 1)]
+    ctx = make_ctx(wl, engine=ENGINES["tc"])
+    ctx.build(0, q, k, v)
+    ref = []
+    for qb, kb, vb in steps:
+        out, lse = new_outputs(wl)
+        ctx.step(qb, kb, vb, out, lse)
+        torch.cuda.synchronize()
+        ref.append((out, lse))
+    ctx.set_step_overlap(False)
+    qs, ks, vs = (torch.empty_like(t) for t in steps[0])
+    for rep in range(3):
+        got = [new_outputs(wl) for _ in steps]
+        for (qb, kb, vb), (out, lse) in zip(steps, got):
+            qs.copy_(qb); ks.copy_(kb); vs.copy_(vb)      # same stream, no host wait
+            ctx.step(qs, ks, vs, out, lse)
+        torch.cuda.synchronize()
+        for i, ((o0, l0), (o1, l1)) in enumerate(zip(ref, got)):
+            assert torch.equal(o0, o1) and torch.equal(l0, l1), "step %d" % i
+    assert ctx.poll_status()[0] == 0
+    ctx.destroy()
+
+
 def test_error_paths():
     wl = small_workload(prompt_lens=(40,), gen_len=64, block_len=32, steps=1, hq=2, hkv=2, d=128)
     sch = SyntheticSchedule(wl, seed=1)

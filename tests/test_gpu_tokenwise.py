@@ -229,3 +229,86 @@ def test_build_and_step_from_token_ids(shape):
     assert e.value.status == binding.ERR_SHAPE
     for o in (prod_bad, prod, ctx, ctx2):
         o.destroy()
+
+
+def test_build_update_reprojects_only_changed_rows():
+    """From one block to the next only the finished block's tokens change: an update that re-projects
+    those rows alone must leave the context in the state a build from all T token ids leaves it in.
+    Untouched rows are bit-identical.  Re-projected rows may differ in the last bf16 place in a few
+    elements (the reduction over d_model is split over the SMs differently for 64 tokens than for T,
+    so the fp32 sums round differently); a step taken from either state meets the oracle tolerance."""
+    wl = W.small_workload(prompt_lens=(130, 75), gen_len=96, block_len=32, steps=2, hq=8, hkv=4)
+    tm = TokenModel(wl, 384, 2000)
+    T, nb = wl.total_tokens, wl.batch * wl.block_len
+    sch = SyntheticSchedule(wl)   # index sets only
+    prod_a, prod_b = make_producer(tm, T), make_producer(tm, T)
+    ctx_a, ctx_b = make_ctx(wl), make_ctx(wl)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    ids0, ids1 = tm.full_ids(0).copy(), tm.full_ids(1).copy()
+    rows = sch.block_rows(0).astype(np.int32)
+    ids0[rows] = tm.mask_id                       # block 0 still masked at its build
+    assert np.array_equal(np.flatnonzero(ids0 != ids1), np.sort(rows))
+    # an update needs the all-token rows of a preceding build of the same pair
+    with pytest.raises(binding.LacacheError) as e:
+        ctx_a.build_tokens_update(prod_a, 1, dev(rows), token_ids=dev(ids1[rows]))
+    assert e.value.status == binding.ERR_STATE
+    ctx_a.build_tokens(prod_a, 0, token_ids=dev(ids0))
+    out, lse = new_outputs(wl)
+    ctx_a.step_tokens(prod_a, out, lse, blk_token_ids=dev(tm.block_ids(0, 1)))   # block scratch must not disturb it
+    perm = np.random.default_rng(3).permutation(len(rows))                        # any order of the changed rows
+    ctx_a.build_tokens_update(prod_a, 1, dev(rows[perm]), token_ids=dev(ids1[rows[perm]]))
+    assert ctx_a.last_launch_count == 4
+    ctx_b.build_tokens(prod_b, 1, token_ids=dev(ids1))
+    caches = []
+    for ctx in (ctx_a, ctx_b):
+        qr = torch.empty(T, wl.n_q_heads, wl.head_dim, device="cuda")
+        kr = torch.empty(T, wl.n_kv_heads, wl.head_dim, device="cuda")
+        vr = torch.empty_like(kr)
+        ctx.export_rope_cache(qr, kr, vr)
+        caches.append((qr, kr, vr))
+    keep = torch.ones(T, dtype=torch.bool, device="cuda")
+    keep[torch.from_numpy(rows.astype(np.int64)).cuda()] = False
+    for x, y in zip(*caches):
+        assert torch.equal(x[keep], y[keep])
+        d = (x[~keep] - y[~keep]).abs()
+        assert float(d.max()) <= 2.0 ** -7 * float(y[~keep].abs().max())
+        assert float((d != 0).float().mean()) <= 0.03
+    ids_blk = dev(tm.block_ids(1, 2))
+    res = []
+    for ctx, prod in ((ctx_a, prod_a), (ctx_b, prod_b)):
+        out, lse = new_outputs(wl)
+        ctx.step_tokens(prod, out, lse, blk_token_ids=ids_blk)
+        torch.cuda.synchronize()
+        res.append((out, lse))
+    _, qf, kf, vf = oracle_qkv(tm, ids=ids1)
+    _, qb, kb, vb = oracle_qkv(tm, ids=tm.block_ids(1, 2))
+    brows = sch.block_rows(1)
+    qf[brows], kf[brows], vf[brows] = qb, kb, vb
+    ref, rlse = oracle.attention(qf, kf, vf, wl.cu_seqlens, wl.rope_theta, wl.head_dim ** -0.5)
+    for out, lse in res:
+        err = np.abs(out.cpu().numpy().astype(np.float64) - ref)
+        assert err.max() <= TOL["bf16"][0] and err.mean() <= TOL["bf16"][1], (err.max(), err.mean())
+        assert np.abs(lse.cpu().numpy() - rlse).max() <= TOL["bf16"][0]
+    assert float((res[0][0] - res[1][0]).abs().max()) <= TOL["bf16"][0]
+    # hidden-state entry of the update, and n_changed = 0
+    ctx_a.build_tokens_update(prod_a, 1, dev(rows), hidden=dev_bf16(tm.embed[ids1[rows]]))
+    ctx_a.build_tokens_update(prod_a, 1, dev(rows[:0]), token_ids=dev(ids1[:0]))
+    out, lse = new_outputs(wl)
+    ctx_a.step_tokens(prod_a, out, lse, blk_token_ids=ids_blk)
+    torch.cuda.synchronize()
+    assert torch.equal(out, res[0][0])      # the same update again: the same bits
+    # a row outside [0, T): reported, dropped, the other rows still written
+    bad = rows.copy()
+    bad[3] = T
+    ctx_a.build_tokens_update(prod_a, 1, dev(bad), token_ids=dev(ids1[rows]))
+    torch.cuda.synchronize()
+    st, msg = prod_a.poll_status()
+    assert st == binding.ERR_INVALID_ARG and "destination row" in msg, (st, msg)
+    # another context's build with the same producer invalidates the kept rows
+    ctx_b.build_tokens(prod_a, 1, token_ids=dev(ids1))
+    with pytest.raises(binding.LacacheError) as e:
+        ctx_a.build_tokens_update(prod_a, 1, dev(rows), token_ids=dev(ids1[rows]))
+    assert e.value.status == binding.ERR_STATE
+    assert ctx_a.poll_status()[0] == binding.OK and ctx_b.poll_status()[0] == binding.OK
+    for o in (prod_a, prod_b, ctx_a, ctx_b):
+        o.destroy()
