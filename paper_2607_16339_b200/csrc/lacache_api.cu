@@ -57,6 +57,7 @@ struct lacache_ctx {
 
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
   int step_overlap = 1;   // consecutive steps may overlap on the device
+  int steps_since_build = 0;
   int built_block = -1;
   int last_launches = 0;
   int device = 0;
@@ -547,6 +548,7 @@ lacache_status lacache_build(lacache_ctx* c, int block_idx, const void* q, const
   st = run_attention(c, a, false, s);
   if (st != LACACHE_OK) return st;
   c->built_block = block_idx;
+  c->steps_since_build = 0;
   return LACACHE_OK;
 }
 
@@ -657,7 +659,10 @@ lacache_status step_impl(lacache_ctx* c, const void* q, const void* k, const voi
   // may start while the previous step's attention kernel drains (it waits before its stores); when
   // the kernel before it in the stream is the one that writes its inputs, it waits for that one first
   const bool overlap = c->step_overlap && !getenv("LACACHE_NO_PDL") && !getenv("LACACHE_NO_STEP_OVERLAP");
-  r.pdl = inputs_just_written ? 2 : (overlap ? 1 : 0);
+  // (the first step after a build is launched the ordinary way: the build's cached state, which the
+  // attention kernel reads before it waits on anything, is then complete and flushed)
+  r.pdl = inputs_just_written ? 2 : ((overlap && c->steps_since_build > 0) ? 1 : 0);
+  c->steps_since_build++;
   r.dst = c->rot;
   r.in_dtype = c->cfg.dtype;
   CU_TRY(c, rope_write(c->g, r, c->engine, s));
