@@ -166,61 +166,6 @@ def rank_seed(base_seed, rank):
 
 
 # ----------------------------------------------------------------------------
-# synthetic inputs on the device (same distributions as the parity workloads)
-# ----------------------------------------------------------------------------
-class DeviceSchedule:
-    """All inputs of the block schedule, resident in HBM before timing starts:
-    per block the full pre-RoPE arrays the build sees, per step the block's
-    fresh tensors."""
-
-    def __init__(self, wl, seed, device, n_steps):
-        import torch
-        self.wl = wl
-        g = torch.Generator(device=device).manual_seed(seed)
-        tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
-        d, Hq, Hkv = wl.head_dim, wl.n_q_heads, wl.n_kv_heads
-        grp = Hq // Hkv
-        if wl.scale_mode == "inv_sqrt_d":
-            cq = torch.full((Hq,), d ** -0.5, device=device)
-        else:
-            cq = torch.rand(Hq, generator=g, device=device) * 1.5 + 0.5
-        ckv = cq[::grp].contiguous()
-        T = wl.total_tokens
-        rn = lambda n, H, c: (torch.randn(n, H, d, generator=g, device=device) * c[None, :, None])
-        q, k, v = rn(T, Hq, cq), rn(T, Hkv, ckv), rn(T, Hkv, ckv)
-        cu = wl.cu_seqlens
-        if wl.key_outlier_frac > 0:
-            for b, P in enumerate(wl.prompt_lens):
-                n_out = int(wl.key_outlier_frac * P)
-                idx = torch.randperm(P, generator=g, device=device)[:n_out] + int(cu[b])
-                k[idx] *= wl.key_outlier_mult
-        mq, mk, mv = rn(1, Hq, cq)[0], rn(1, Hkv, ckv)[0], rn(1, Hkv, ckv)[0]
-        for b, P in enumerate(wl.prompt_lens):
-            q[cu[b] + P:cu[b + 1]] = mq; k[cu[b] + P:cu[b + 1]] = mk; v[cu[b] + P:cu[b + 1]] = mv
-        S, Lb, B = wl.steps_per_block, wl.block_len, wl.batch
-        self.n_blocks_used = min(wl.n_blocks, (n_steps + S - 1) // S)
-        self.full = []    # per block: (q, k, v) as the build sees them
-        self.steps = []   # per step: (q_blk, k_blk, v_blk)
-        rows_of = lambda blk: torch.cat([torch.arange(cu[b] + P + blk * Lb, cu[b] + P + (blk + 1) * Lb)
-                                         for b, P in enumerate(wl.prompt_lens)]).to(device)
-        for blk in range(self.n_blocks_used):
-            self.full.append((q.to(tdt).contiguous(), k.to(tdt).contiguous(), v.to(tdt).contiguous()))
-            last = None
-            for s in range(S):
-                last = (rn(B * Lb, Hq, cq).to(tdt).contiguous(), rn(B * Lb, Hkv, ckv).to(tdt).contiguous(),
-                        rn(B * Lb, Hkv, ckv).to(tdt).contiguous())
-                self.steps.append(last)
-            rows = rows_of(blk)
-            q[rows], k[rows], v[rows] = last[0].float(), last[1].float(), last[2].float()
-
-    def step_inputs(self, i):
-        S = self.wl.steps_per_block
-        n = self.n_blocks_used * S
-        i = i % n
-        return i // S, i % S, self.steps[i]
-
-
-# ----------------------------------------------------------------------------
 # the CUDA arm
 # ----------------------------------------------------------------------------
 L2_BYTES = 126 << 20
@@ -231,13 +176,15 @@ def n_replicas(step_bytes):
     before it is touched again: the other replicas' steps move at least twice
     the L2 capacity in between."""
     import math
+    if step_bytes >= 8 * L2_BYTES:      # one step alone moves many times the L2
+        return 1
     return max(3, math.ceil(2.0 * L2_BYTES / max(step_bytes, 1)) + 1)
 
 
 def run_cuda(args):
     import torch
     from paper_2607_16339_b200 import binding
-    from paper_2607_16339_b200.workloads import WORKLOADS
+    from paper_2607_16339_b200.workloads import WORKLOADS, DeviceSchedule
 
     rank, local_rank, world = dist_env()
     if not torch.cuda.is_available():
@@ -474,7 +421,8 @@ def run_cuda(args):
         c.destroy()
     del outs, sched
     if rank == 0:
-        if world == 1 and not args.no_token_path and wl.dtype == "bf16" and wl.n_q_heads in D_MODEL:
+        if (world == 1 and not args.no_token_path and wl.dtype == "bf16" and wl.n_q_heads in D_MODEL
+                and wl.total_tokens <= 65536):     # (its replicas of the all-token scratch would not fit beyond that)
             line["token_path"] = token_path_leg(wl, dev, peaks, args.seed, min(K, 512))
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -672,7 +620,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1024)
     ap.add_argument("--warmup", type=int, default=32)
-    ap.add_argument("--workload", type=int, default=2, help="config number 1..5 (2 = the headline LLaDA-8B shape)")
+    ap.add_argument("--workload", type=int, default=2, help="config number 1..6 (2 = the headline LLaDA-8B shape; 6 = the large-batch extension)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")

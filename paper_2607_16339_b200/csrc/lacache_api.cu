@@ -384,6 +384,14 @@ void destroy_impl(lacache_ctx* c) {
   delete c;
 }
 
+// Units per CTA the pipelined merge variant takes in one launch (its table size; LACACHE_DEEP_UNITS
+// lowers it so that small cases exercise the multi-launch path).
+int deep_unit_cap() {
+  const char* e = getenv("LACACHE_DEEP_UNITS");
+  const int v = e ? atoi(e) : TC_DEEP_MAX_UNITS;
+  return std::max(1, std::min(v, (int)TC_DEEP_MAX_UNITS));
+}
+
 AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk, const RotBuffers& rot,
                    float* out, float* lse) {
   AttnArgs a{};
@@ -421,11 +429,18 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       const double max_tiles = list.n > 0 ? 0.5 * (sum_tiles / list.n + longest) : 1.0;
       int ns = 1;
       double best = 1e30;
+      const bool deep_ok = c->g.block_len <= 32 && !getenv("LACACHE_NO_DEEP");
+      const int deep_cap = deep_unit_cap();
       for (int cand = 1; cand < total; ++cand) {
         double ts = ceil((double)units_stream / cand) * (3.0 + 1.6 * max_tiles + (c->max_chunks > 1 ? 2.0 + 0.8 * c->max_chunks : 0.0));
-        const double per_cta = ceil((double)units_merge / (total - cand));
+        double per_cta = ceil((double)units_merge / (total - cand));
+        double rest = 0.0;   // merge units beyond what one launch of the pipelined variant takes: further launches, all SMs
+        if (deep_ok && per_cta > deep_cap) {
+          rest = (double)units_merge - (double)deep_cap * (total - cand);
+          per_cta = deep_cap;
+        }
         double tm = 4.0 + per_cta * ((c->g.block_len <= 32 && per_cta <= 8) ? 2.6 : 3.4);
-        double t = std::max(ts, tm);
+        double t = std::max(ts, tm) + (rest > 0 ? 4.0 + ceil(rest / c->num_sms) * 3.4 : 0.0);
         if (t < best - 1e-9) { best = t; ns = cand; }
       }
       if (c->stream_ctas_override > 0) ns = c->stream_ctas_override;
@@ -441,7 +456,8 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       {
         const int n_merge_ctas = a.n_ctas - ns;
         const long long per_cta = n_merge_ctas > 0 ? (units_merge + n_merge_ctas - 1) / n_merge_ctas : 0;
-        a.merge_deep = (c->g.block_len <= 32 && per_cta <= TC_DEEP_MAX_UNITS && !getenv("LACACHE_NO_DEEP")) ? 1 : 0;
+        a.merge_deep = (deep_ok && per_cta <= deep_cap) ? 1 : 0;
+        a.split_merge = (deep_ok && per_cta > deep_cap) ? 1 : 0;
       }
     } else {
       a.n_ctas_stream = (int)std::min<long long>(c->num_sms, units_stream);
@@ -456,12 +472,47 @@ lacache_status run_attention(lacache_ctx* c, const AttnArgs& a, bool scratch, cu
     if (!tc_set_out(scratch ? c->maps_scratch : c->maps, c->g, a.out, c->err, sizeof(c->err))) return LACACHE_ERR_CUDA;
   }
   if (c->ev_start) CU_TRY(c, cudaEventRecord(c->ev_start, s));
-  if (c->engine == LACACHE_ENGINE_TCGEN05)
-    CU_TRY(c, tc_attention(c->g, a, scratch ? c->maps_scratch : c->maps, s));
-  else
-    CU_TRY(c, simt_attention(c->g, a, s));
+  if (c->engine == LACACHE_ENGINE_TCGEN05 && a.split_merge) {
+    // The pipelined merge variant tabulates at most TC_DEEP_MAX_UNITS units per CTA.  A step with more
+    // fixed rows than that goes out in several launches: the first carries the block queries and as
+    // many row tiles as its merge CTAs can tabulate, the others row tiles only, on all SMs.
+    const TcMaps* maps = scratch ? c->maps_scratch : c->maps;
+    const int Hq = c->g.Hq;
+    const int deep_cap = deep_unit_cap();
+    AttnArgs b = a;
+    b.merge_deep = 1;
+    const int m0 = a.n_ctas - a.n_ctas_stream;
+    int done = std::min(a.n_items_merge, std::max(1, deep_cap * m0 / Hq));
+    b.n_items_merge = done;
+    b.n_ctas = a.n_ctas_stream + (int)std::min<long long>((long long)done * Hq, m0);
+    CU_TRY(c, tc_attention(c->g, b, maps, s));
+    c->last_launches++;
+    const int rest = a.n_items_merge - done;
+    if (rest > 0) {
+      const int cap = std::max(1, deep_cap * c->num_sms / Hq);
+      const int n_more = (rest + cap - 1) / cap;
+      const int per = (rest + n_more - 1) / n_more;
+      while (done < a.n_items_merge) {
+        AttnArgs m = a;
+        m.merge_deep = 1;
+        m.n_items = 0;
+        m.n_ctas_stream = 0;
+        m.items_merge = a.items_merge + done;
+        m.n_items_merge = std::min(per, a.n_items_merge - done);
+        m.n_ctas = (int)std::min<long long>(c->num_sms, (long long)m.n_items_merge * Hq);
+        CU_TRY(c, tc_attention(c->g, m, maps, s));
+        c->last_launches++;
+        done += m.n_items_merge;
+      }
+    }
+  } else {
+    if (c->engine == LACACHE_ENGINE_TCGEN05)
+      CU_TRY(c, tc_attention(c->g, a, scratch ? c->maps_scratch : c->maps, s));
+    else
+      CU_TRY(c, simt_attention(c->g, a, s));
+    c->last_launches++;
+  }
   if (c->ev_stop) CU_TRY(c, cudaEventRecord(c->ev_stop, s));
-  c->last_launches++;
   return LACACHE_OK;
 }
 

@@ -93,6 +93,8 @@ struct AttnArgs {
   const WorkItem* items_merge; int n_items_merge;
   int n_ctas_stream; int n_ctas;
   int merge_deep;            // merge role runs its pipelined variant (block_len <= 32, bounded units per CTA)
+  int split_merge;           // host only: more merge units per CTA than the pipelined variant tabulates, so the
+                             // fixed rows of the step go out in several launches of that variant
   // step only: the block's pre-RoPE queries [B * block_len, Hq, d] and the cos/sin rows of
   // those tokens [B * block_len][d/2]; a CTA's first block-query unit rotates its Q tile
   // from these itself and so does not have to wait for the RoPE kernel

@@ -65,6 +65,9 @@ class Workload:
 
 # prompt lengths of the ragged config: Philox(key=4).integers(256, 1025, 8)
 _RAGGED_PROMPTS = (500, 256, 798, 584, 526, 932, 396, 371)
+# prompt lengths of the large-batch extension: 256 few-shot prompts of 600..1000 tokens
+_LARGE_BATCH_PROMPTS = tuple(int(x) for x in
+                             np.random.Generator(np.random.Philox(key=6)).integers(600, 1001, 256))
 
 WORKLOADS = {
     1: Workload(1, "tiny-fp32", "fp32", (48,), 64, 16, 4, 4, 4, 64, 1.0e4, "inv_sqrt_d"),
@@ -76,6 +79,11 @@ WORKLOADS = {
                 "per_head_u(0.5,2)"),
     5: Workload(5, "dream7b-l1-gqa-p4096-g1024", "bf16", (4096,), 1024, 64, 64, 28, 4, 128, 1.0e6,
                 "inv_sqrt_d"),
+    # extension beyond the five named configurations: the large-batch setting in which the paper
+    # isolates FACache (batch 256, block 32, a 28/4-head GQA model, few-shot prompts; App. table
+    # "FACache only"); not a headline configuration
+    6: Workload(6, "gqa-l1-batch256-p600to1000-g320", "bf16", _LARGE_BATCH_PROMPTS, 320, 32, 8, 28, 4, 128,
+                1.0e6, "inv_sqrt_d"),
 }
 
 
@@ -301,3 +309,57 @@ class TokenModel:
         still_masked = r.uniform(size=n) >= s / wl.steps_per_block
         ids[still_masked] = self.mask_id
         return ids
+
+
+class DeviceSchedule:
+    """The same kind of schedule as SyntheticSchedule, drawn on the device with
+    torch's generator (data generation only; for sizes where numpy on the host
+    would take minutes): all inputs of the block schedule resident in HBM, per
+    block the full pre-RoPE arrays the build sees, per step the block's fresh
+    tensors."""
+
+    def __init__(self, wl, seed, device, n_steps):
+        import torch
+        self.wl = wl
+        g = torch.Generator(device=device).manual_seed(seed)
+        tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+        d, Hq, Hkv = wl.head_dim, wl.n_q_heads, wl.n_kv_heads
+        grp = Hq // Hkv
+        if wl.scale_mode == "inv_sqrt_d":
+            cq = torch.full((Hq,), d ** -0.5, device=device)
+        else:
+            cq = torch.rand(Hq, generator=g, device=device) * 1.5 + 0.5
+        ckv = cq[::grp].contiguous()
+        T = wl.total_tokens
+        rn = lambda n, H, c: (torch.randn(n, H, d, generator=g, device=device) * c[None, :, None])
+        q, k, v = rn(T, Hq, cq), rn(T, Hkv, ckv), rn(T, Hkv, ckv)
+        cu = wl.cu_seqlens
+        if wl.key_outlier_frac > 0:
+            for b, P in enumerate(wl.prompt_lens):
+                n_out = int(wl.key_outlier_frac * P)
+                idx = torch.randperm(P, generator=g, device=device)[:n_out] + int(cu[b])
+                k[idx] *= wl.key_outlier_mult
+        mq, mk, mv = rn(1, Hq, cq)[0], rn(1, Hkv, ckv)[0], rn(1, Hkv, ckv)[0]
+        for b, P in enumerate(wl.prompt_lens):
+            q[cu[b] + P:cu[b + 1]] = mq; k[cu[b] + P:cu[b + 1]] = mk; v[cu[b] + P:cu[b + 1]] = mv
+        S, Lb, B = wl.steps_per_block, wl.block_len, wl.batch
+        self.n_blocks_used = min(wl.n_blocks, (n_steps + S - 1) // S)
+        self.full = []    # per block: (q, k, v) as the build sees them
+        self.steps = []   # per step: (q_blk, k_blk, v_blk)
+        rows_of = lambda blk: torch.cat([torch.arange(cu[b] + P + blk * Lb, cu[b] + P + (blk + 1) * Lb)
+                                         for b, P in enumerate(wl.prompt_lens)]).to(device)
+        for blk in range(self.n_blocks_used):
+            self.full.append((q.to(tdt).contiguous(), k.to(tdt).contiguous(), v.to(tdt).contiguous()))
+            last = None
+            for s in range(S):
+                last = (rn(B * Lb, Hq, cq).to(tdt).contiguous(), rn(B * Lb, Hkv, ckv).to(tdt).contiguous(),
+                        rn(B * Lb, Hkv, ckv).to(tdt).contiguous())
+                self.steps.append(last)
+            rows = rows_of(blk)
+            q[rows], k[rows], v[rows] = last[0].float(), last[1].float(), last[2].float()
+
+    def step_inputs(self, i):
+        S = self.wl.steps_per_block
+        n = self.n_blocks_used * S
+        i = i % n
+        return i // S, i % S, self.steps[i]

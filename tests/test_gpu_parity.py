@@ -273,6 +273,84 @@ def test_steps_fed_by_same_stream_writes_with_overlap_off(cfg):
     ctx.destroy()
 
 
+@pytest.mark.parametrize("cfg", [3, 4])
+def test_step_split_over_several_launches(cfg, monkeypatch):
+    """A step with more fixed-row tiles per CTA than the pipelined merge variant tabulates goes out in
+    several launches (block queries and the first row tiles, then row tiles only on all SMs).  Forced
+    here with a tiny table: the result must be, bit for bit, that of the single launch."""
+    wl = WORKLOADS[cfg]
+    sch = SyntheticSchedule(wl, seed=5)
+    b = 1
+    q, k, v = (to_dev(a, wl) for a in advance_to_block(sch, b))
+    steps = [tuple(to_dev(a, wl) for a in sch.draw_step(b, s)) for s in (1, 2, 3)]
+    ctx = make_ctx(wl, engine=ENGINES["tc"])
+    ctx.build(b, q, k, v)
+    ref = []
+    for qb, kb, vb in steps:
+        out, lse = new_outputs(wl)
+        ctx.step(qb, kb, vb, out, lse)
+        ref.append((out, lse))
+    torch.cuda.synchronize()
+    assert ctx.last_launch_count == 2
+    for cap in ("3", "1"):
+        monkeypatch.setenv("LACACHE_DEEP_UNITS", cap)
+        got = []
+        for qb, kb, vb in steps:              # back to back: the launches of consecutive steps overlap
+            out, lse = new_outputs(wl)
+            ctx.step(qb, kb, vb, out, lse)
+            got.append((out, lse))
+        torch.cuda.synchronize()
+        assert ctx.last_launch_count >= 3, ctx.last_launch_count
+        for (o0, l0), (o1, l1) in zip(ref, got):
+            assert torch.equal(o0, o1) and torch.equal(l0, l1)
+    monkeypatch.delenv("LACACHE_DEEP_UNITS")
+    assert ctx.poll_status()[0] == 0
+    check_against_oracle(wl, sch, got[-1][0], got[-1][1], rows=sample_rows(wl, sch, b), what="split step")
+    ctx.destroy()
+
+
+def test_large_batch_extension_full_size():
+    """The large-batch extension (256 sequences, 28/4 heads, ~287k tokens) at full size, in the
+    launch configuration the bench times: the step's fixed rows exceed one launch of the pipelined
+    merge variant and go out in several.  Cached path vs full recompute on every row; vs the oracle
+    on all rows of three sequences (first, longest, last)."""
+    from paper_2607_16339_b200.workloads import DeviceSchedule
+    wl = WORKLOADS[6]
+    S = 3
+    sched = DeviceSchedule(wl, 17, torch.device("cuda"), S)
+    ctx = make_ctx(wl, engine=ENGINES["tc"])
+    q, k, v = sched.full[0]
+    ctx.build(0, q, k, v)
+    out, lse = new_outputs(wl)
+    for s in range(S):
+        qb, kb, vb = sched.steps[s]
+        ctx.step(qb, kb, vb, out, lse)
+    torch.cuda.synchronize()
+    assert ctx.last_launch_count >= 3            # RoPE + more than one attention launch
+    assert ctx.poll_status()[0] == 0
+    cu = wl.cu_seqlens
+    rows = torch.cat([torch.arange(cu[b] + P, cu[b] + P + wl.block_len) for b, P in enumerate(wl.prompt_lens)]).cuda()
+    qf, kf, vf = q.clone(), k.clone(), v.clone()
+    qf[rows], kf[rows], vf[rows] = qb, kb, vb
+    out2, lse2 = new_outputs(wl)
+    ctx.full_recompute(qf, kf, vf, out2, lse2)
+    torch.cuda.synchronize()
+    assert float((out - out2).abs().max()) <= TOL_CACHED_VS_FULL["bf16"]
+    assert float((lse - lse2).abs().max()) <= TOL_CACHED_VS_FULL["bf16"]
+    seqs = sorted({0, int(np.argmax(wl.prompt_lens)), wl.batch - 1})
+    idx = np.concatenate([np.arange(cu[b], cu[b + 1]) for b in seqs])
+    sub_cu = np.concatenate([[0], np.cumsum([cu[b + 1] - cu[b] for b in seqs])]).astype(np.int32)
+    t_idx = torch.from_numpy(idx).cuda()
+    host = lambda t: t[t_idx].float().cpu().numpy().astype(np.float64)
+    ref, rlse = oracle.attention(host(qf), host(kf), host(vf), sub_cu, wl.rope_theta, wl.head_dim ** -0.5)
+    err = np.abs(out[t_idx].cpu().numpy().astype(np.float64) - ref)
+    assert err.max() <= TOL["bf16"][0] and err.mean() <= TOL["bf16"][1], (err.max(), err.mean())
+    # the outputs here are small (values ~ N(0,1)/sqrt(d), near-uniform attention): also relative to their scale
+    assert err.max() <= 2e-2 * np.abs(ref).max(), (err.max(), np.abs(ref).max())
+    assert np.abs(lse[t_idx].cpu().numpy() - rlse).max() <= TOL["bf16"][0]
+    ctx.destroy()
+
+
 def test_error_paths():
     wl = small_workload(prompt_lens=(40,), gen_len=64, block_len=32, steps=1, hq=2, hkv=2, d=128)
     sch = SyntheticSchedule(wl, seed=1)
