@@ -222,7 +222,9 @@ lacache_status lacache_step_host(lacache_ctx* ctx, const void* q_blk_host, const
  * projection kernel streams (same size); the caller's copy may be released afterwards, and a
  * later change to it has no effect.
  * d_model is a multiple of 64, at most 8192; head_dim is 128; max_tokens bounds n_tokens of every
- * later call.  Needs an sm_100 device.
+ * later call.  Needs an sm_100 device.  A handle is not thread-safe, and its calls share one
+ * workspace: enqueue them on one stream at a time (calls on one stream are ordered and may follow
+ * each other without synchronising).
  */
 typedef struct lacache_qkv lacache_qkv;
 typedef struct {

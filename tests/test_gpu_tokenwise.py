@@ -312,3 +312,22 @@ def test_build_update_reprojects_only_changed_rows():
     assert ctx_a.poll_status()[0] == binding.OK and ctx_b.poll_status()[0] == binding.OK
     for o in (prod_a, prod_b, ctx_a, ctx_b):
         o.destroy()
+
+
+@pytest.mark.parametrize("d_model,hq,hkv,n", [(64, 1, 1, 1), (64, 2, 1, 33), (192, 3, 1, 257), (1024, 6, 2, 130),
+                                              (8192, 2, 2, 20)])
+def test_projection_odd_shapes(d_model, hq, hkv, n):
+    """Corners of the work split: a single k chunk per tile (every segment covers its tile alone),
+    fewer chunks than SMs, one token, token counts just past a tile, the widest row the norm
+    kernel takes."""
+    wl = W.small_workload(name="odd", hq=hq, hkv=hkv, scale_mode="inv_sqrt_d")
+    tm = TokenModel(wl, d_model, 300, seed=d_model + n)
+    prod = make_producer(tm, n)
+    ids = np.random.default_rng(n).integers(0, tm.vocab, n).astype(np.int32)
+    st, msg, q, k, v, h = project(prod, tm, n, ids=ids, want_h=True)
+    assert st == binding.OK, msg
+    hr = check_qkv(tm, q, k, v, ids=ids, what="d_model=%d n=%d" % (d_model, n))
+    assert np.array_equal(h.float().cpu().numpy(), hr.astype(np.float32))
+    st, msg, q2, k2, v2, _ = project(prod, tm, n, ids=ids)
+    assert torch.equal(q, q2) and torch.equal(k, k2) and torch.equal(v, v2)
+    prod.destroy()
