@@ -45,6 +45,7 @@ enum StatusLoc : int32_t {
   LOC_WAIT_V = 4,
   LOC_WAIT_S = 5,
   LOC_WAIT_O = 6,
+  LOC_UNIT_TABLE = 7,
 };
 
 struct Geometry {

@@ -1489,6 +1489,10 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = LOC_SMEM_ALIGN;
     return;
   }
+  if (deep && n_my > TC_DEEP_MAX_UNITS) {  // the host sizes launches so that the unit table never overflows
+    if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) { a.status[1] = LOC_UNIT_TABLE; a.status[2] = n_my; }
+    return;
+  }
   if (tid == 0) {
     for (int i = 0; i < N_BARS; ++i) {
       uint32_t count = 1;
