@@ -824,7 +824,9 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       // head) to arrive merges all of them.
       const size_t pbase = ((size_t)un.seq * g.Hq + un.h) * a.max_chunks;  // [chunk][block_len]
       const size_t prow0 = (pbase + un.chunk) * g.block_len;
-      if (row_valid) {
+      {
+        // (the TMEM loads are warp-wide: rows past the block take part in them and only skip the
+        // stores, so a block length that is not a multiple of 32 cannot split a warp around them)
         float4* dst = reinterpret_cast<float4*>(a.part_o + (prow0 + r) * D + 64 * half);
 #pragma unroll 1
         for (int cb = 0; cb < 4; ++cb) {
@@ -836,12 +838,14 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
 #pragma unroll
             for (int j = 0; j < 16; ++j) rr[j] = 0u;
           }
+          if (row_valid) {
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            dst[4 * cb + i] = make_float4(__uint_as_float(rr[4 * i]), __uint_as_float(rr[4 * i + 1]),
-                                          __uint_as_float(rr[4 * i + 2]), __uint_as_float(rr[4 * i + 3]));
+            for (int i = 0; i < 4; ++i)
+              dst[4 * cb + i] = make_float4(__uint_as_float(rr[4 * i]), __uint_as_float(rr[4 * i + 1]),
+                                            __uint_as_float(rr[4 * i + 2]), __uint_as_float(rr[4 * i + 3]));
+          }
         }
-        if (half == 0) { a.part_m[prow0 + r] = m_ref; a.part_l[prow0 + r] = l_run; }
+        if (row_valid && half == 0) { a.part_m[prow0 + r] = m_ref; a.part_l[prow0 + r] = l_run; }
       }
       tc_fence_before();
       mbar_arrive(c.bar(BAR_O_FREE));  // the next unit may overwrite O~
@@ -861,6 +865,36 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       if (*c.flag != 0) merge_partials(g, a, pbase, un.nchunks, g.block_len, un.row0, un.h);
       if (!epi_sync(c, epi_phase)) return;  // the flag may be rewritten
       if (un.q_rows == BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));
+      continue;
+    }
+    if (un.epi == EPI_STATE && un.q_rows == BM) {
+      // Cached state of a build unit, straight from TMEM to global memory (each thread 256
+      // contiguous bytes of its row).  Nothing is staged in the Q region, so the next unit's Q
+      // tile may be loaded while this epilogue runs.
+      if (threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));
+      const size_t srow = (size_t)un.h * g.Tp + row;
+      float4* dst = reinterpret_cast<float4*>(a.st.o + srow * D + 64 * half);
+#pragma unroll 1
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t rr[16];
+        if (!first_tile) {   // (uniform over the CTA; the TMEM load is warp-wide, so rows past the
+                             // end of a clipped tile take part in it and only skip the stores)
+          tmem_ld16(tlane + TS_O + 64 * half + 16 * cb, rr);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) rr[j] = 0u;
+        }
+        if (row_valid) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            dst[4 * cb + i] = make_float4(__uint_as_float(rr[4 * i]), __uint_as_float(rr[4 * i + 1]),
+                                          __uint_as_float(rr[4 * i + 2]), __uint_as_float(rr[4 * i + 3]));
+        }
+      }
+      if (row_valid && half == 0) { a.st.m[srow] = m_ref; a.st.l[srow] = l_run; }
+      tc_fence_before();
+      mbar_arrive(c.bar(BAR_O_FREE));  // the next unit may overwrite O~
       continue;
     }
     // O~ (this thread's 64 features) from TMEM to its staging row.  The staging

@@ -44,9 +44,9 @@ def _engines_for(dtype, d):
     return ["simt", "tc"] if (dtype == "bf16" and d == 128) else ["simt"]
 
 
-def _run_points(wl, engine, seed, blocks=None, rows_fn=None, check_full=True, check_state=True):
+def _run_points(wl, engine, seed, blocks=None, rows_fn=None, check_full=True, check_state=True, **ctx_kw):
     sch = SyntheticSchedule(wl, seed=seed)
-    ctx = make_ctx(wl, engine=ENGINES[engine])
+    ctx = make_ctx(wl, engine=ENGINES[engine], **ctx_kw)
     out, lse = new_outputs(wl)
     fout, flse = new_outputs(wl)
     blocks = list(range(wl.n_blocks)) if blocks is None else blocks
@@ -108,6 +108,16 @@ def test_small_cases(case, dtype):
         wl = small_workload(name=case, dtype=dtype, d=d, **kw)
         for engine in _engines_for(dtype, d):
             _run_points(wl, engine, seed=5)
+
+
+@pytest.mark.parametrize("block_len", [16, 48])
+def test_block_lengths_that_split_a_warp(block_len):
+    """Blocks of 16 and 48 rows on the tcgen05 engine with the block queries' keys cut into several
+    chunks: the rows of the block end in the middle of a warp of row threads, which must still take
+    part in the warp-wide TMEM loads of the partial-state epilogue."""
+    wl = small_workload(name="blk%d" % block_len, prompt_lens=(700, 333), gen_len=96, block_len=block_len,
+                        steps=2, hq=4, hkv=2)
+    _run_points(wl, "tc", seed=8, blocks=[0, wl.n_blocks - 1], sc_tiles_per_chunk=2)
 
 
 @pytest.mark.parametrize("engine", ["simt", "tc"])
