@@ -145,6 +145,12 @@ __device__ __forceinline__ void load_qk_box(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void load_v_box(uint32_t dst, const CUtensorMap* map, uint32_t bar, int row, int h) {
   tma_load_4d(dst, map, bar, 0, row, 0, h);
 }
+// one 32-byte store of 8 words (the address is 32-byte aligned)
+__device__ __forceinline__ void st_global_v8(void* dst, const uint32_t* r) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(r[0]), "r"(r[1]), "r"(r[2]),
+               "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -874,23 +880,20 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       if (threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));
       const size_t srow = (size_t)un.h * g.Tp + row;
       float4* dst = reinterpret_cast<float4*>(a.st.o + srow * D + 64 * half);
-#pragma unroll 1
-      for (int cb = 0; cb < 4; ++cb) {
-        uint32_t rr[16];
-        if (!first_tile) {   // (uniform over the CTA; the TMEM load is warp-wide, so rows past the
-                             // end of a clipped tile take part in it and only skip the stores)
-          tmem_ld16(tlane + TS_O + 64 * half + 16 * cb, rr);
-          tmem_ld_wait();
-        } else {
+      // (the TMEM loads are warp-wide: rows past the end of a clipped tile take part in them and
+      // only skip the stores; first_tile is uniform over the CTA)
+      uint32_t rr[64];
+      if (!first_tile) {
+        tmem_ld32(tlane + TS_O + 64 * half, *reinterpret_cast<uint32_t(*)[32]>(rr));
+        tmem_ld32(tlane + TS_O + 64 * half + 32, *reinterpret_cast<uint32_t(*)[32]>(rr + 32));
+        tmem_ld_wait();
+      } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) rr[j] = 0u;
-        }
-        if (row_valid) {
+        for (int j = 0; j < 64; ++j) rr[j] = 0u;
+      }
+      if (row_valid) {   // 32-byte stores: whole sectors, half as many instructions
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            dst[4 * cb + i] = make_float4(__uint_as_float(rr[4 * i]), __uint_as_float(rr[4 * i + 1]),
-                                          __uint_as_float(rr[4 * i + 2]), __uint_as_float(rr[4 * i + 3]));
-        }
+        for (int i = 0; i < 8; ++i) st_global_v8(dst + 2 * i, rr + 8 * i);
       }
       if (row_valid && half == 0) { a.st.m[srow] = m_ref; a.st.l[srow] = l_run; }
       tc_fence_before();
