@@ -131,8 +131,9 @@ lacache_status lacache_build(lacache_ctx* ctx, int block_idx, const void* q_pre,
  * projection kernel run before every step), switch the overlap off with
  * lacache_set_step_overlap(ctx, 0): every kernel of a step is then ordered
  * after all earlier work of the stream, as an ordinary launch is.
- * lacache_step_tokens, which runs such a producer itself, orders its kernels
- * correctly whatever this setting.
+ * lacache_step_tokens runs such a producer itself and orders its own kernels
+ * correctly whatever this setting; what it reads early with the overlap on
+ * is blk_token_ids / blk_hidden, to which the same rule applies.
  */
 lacache_status lacache_step(lacache_ctx* ctx, const void* q_blk, const void* k_blk,
                             const void* v_blk, float* out, float* lse, void* cuda_stream);
@@ -266,8 +267,9 @@ lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, con
  * (token_ids [T] or hidden [T, d_model], packed like q_pre), step the block's B * L_b tokens
  * (sequence-major like q_blk).  The context must be bf16 with the same heads and head_dim as
  * the producer, and max_tokens must cover the call (else LACACHE_ERR_SHAPE).  Consecutive
- * calls on one stream are ordered; unlike lacache_step, a step fed this way starts after the
- * previous step has completed.
+ * calls on one stream are ordered.  A step fed this way does not overlap the previous one, except
+ * that its norm kernel runs alongside the previous step's attention kernel when the overlap of
+ * lacache_set_step_overlap is on: blk_token_ids / blk_hidden are then read early (see lacache_step).
  */
 lacache_status lacache_build_tokens(lacache_ctx* ctx, lacache_qkv* p, int block_idx,
                                     const int32_t* token_ids, const void* hidden,

@@ -659,7 +659,7 @@ lacache_status lacache_build_tokens_update(lacache_ctx* c, lacache_qkv* p, int b
   qkv_scratch(p, false, &q, &k, &v);
   int producer_launches = 0;
   if (n_changed > 0) {
-    st = qkv_project_rows(p, token_ids, hidden, n_changed, q, k, v, nullptr, rows, c->g.T, stream);
+    st = qkv_project_rows(p, token_ids, hidden, n_changed, q, k, v, nullptr, rows, c->g.T, false, stream);
     if (st != LACACHE_OK) return fail(c, st, "producer: %s", lacache_qkv_last_error(p));
     producer_launches = lacache_qkv_last_launch_count(p);
   }
@@ -677,7 +677,11 @@ lacache_status lacache_step_tokens(lacache_ctx* c, lacache_qkv* p, const int32_t
   if (st != LACACHE_OK) return st;
   void *q, *k, *v;
   qkv_scratch(p, true, &q, &k, &v);
-  st = lacache_qkv_project(p, blk_token_ids, blk_hidden, n, q, k, v, nullptr, stream);
+  // with the cross-step overlap on (and not right after a build) the norm kernel reads the ids while the
+  // previous step's attention kernel still runs: the same contract as for q_blk / k_blk / v_blk of lacache_step
+  const bool early = c->step_overlap && c->steps_since_build > 0 && !getenv("LACACHE_NO_PDL") &&
+                     !getenv("LACACHE_NO_STEP_OVERLAP");
+  st = qkv_project_rows(p, blk_token_ids, blk_hidden, n, q, k, v, nullptr, nullptr, 0, early, stream);
   if (st != LACACHE_OK) return fail(c, st, "producer: %s", lacache_qkv_last_error(p));
   st = step_impl(c, q, k, v, out, lse, stream, true);
   if (st == LACACHE_OK) c->last_launches += lacache_qkv_last_launch_count(p);

@@ -145,8 +145,11 @@ void tc_free_maps(TcMaps* m);
 void qkv_scratch(lacache_qkv* p, bool block, void** q, void** k, void** v);
 int qkv_heads(const lacache_qkv* p, int* hq, int* hkv, int* max_tokens);
 // lacache_qkv_project with a scatter: input token t is written to output row dst_rows[t] (null: t)
+// early_inputs: token_ids / hidden were complete before the grid ahead in the stream was enqueued, so the
+// norm kernel may read them while that grid still runs (it waits for it at its end instead).
 lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const void* hidden, int n_tokens, void* q,
-                                void* k, void* v, void* h_out, const int32_t* dst_rows, int max_rows, void* stream);
+                                void* k, void* v, void* h_out, const int32_t* dst_rows, int max_rows, bool early_inputs,
+                                void* stream);
 // which context's tokens the all-token scratch holds (set by a full projection)
 void qkv_set_full_owner(lacache_qkv* p, const void* ctx, int n_tokens);
 bool qkv_full_owner_is(const lacache_qkv* p, const void* ctx, int n_tokens);

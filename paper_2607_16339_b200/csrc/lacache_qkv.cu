@@ -454,6 +454,7 @@ struct NormArgs {
   __nv_bfloat16* h_out;           // [n][d_model] or null
   const int32_t* dst_rows;        // or null; checked against max_rows here
   int max_rows;
+  int early_inputs;               // the inputs were complete before the preceding grid started: read them at once
   int d_model, vocab;
   float eps;
   int32_t* status;
@@ -464,8 +465,12 @@ __global__ void __launch_bounds__(N_THREADS) qkv_norm_kernel(const NormArgs a) {
   // and starts fetching weights.  This kernel is itself launched programmatically dependent and waits,
   // before its first load, for everything enqueued ahead of it (whatever wrote the token ids or hidden
   // states included); the projection kernel's own wait then covers all of that as well.
+  // (A caller that vouches for inputs that were complete before the grid ahead was even enqueued gets
+  // the wait at the end instead: this kernel then runs alongside that grid, and still does not complete
+  // before it, which is what the projection kernel's wait relies on.  The operand rows X^ it writes are
+  // read by nothing but the projection kernel of this call.)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  grid_dependency_wait();
+  if (!a.early_inputs) grid_dependency_wait();
   __shared__ float red[N_THREADS / 32];
   const int t = blockIdx.x;
   const int tid = threadIdx.x;
@@ -532,7 +537,17 @@ __global__ void __launch_bounds__(N_THREADS) qkv_norm_kernel(const NormArgs a) {
       q[e] = __floats2bfloat162_rn(x.x * rinv * g.x, x.y * rinv * g.y);
     }
     reinterpret_cast<uint4*>(a.xhat + (size_t)t * a.d_model)[ch] = o;
-    if (a.h_out) reinterpret_cast<uint4*>(a.h_out + (size_t)t * a.d_model)[ch] = raw[i];
+    if (a.h_out && !a.early_inputs) reinterpret_cast<uint4*>(a.h_out + (size_t)t * a.d_model)[ch] = raw[i];
+  }
+  if (a.early_inputs) {
+    grid_dependency_wait();
+    if (a.h_out) {   // a caller's buffer: not before the grids ahead are complete
+#pragma unroll
+      for (int i = 0; i < N_MAX_CHUNKS; ++i) {
+        const int ch = tid + i * N_THREADS;
+        if (ch < n_chunks) reinterpret_cast<uint4*>(a.h_out + (size_t)t * a.d_model)[ch] = raw[i];
+      }
+    }
   }
 }
 
@@ -696,14 +711,15 @@ lacache_status lacache_qkv_destroy(lacache_qkv* p) {
 
 lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, const void* hidden, int n_tokens,
                                    void* q, void* k, void* v, void* h_out, void* stream) {
-  return lacache::qkv_project_rows(p, token_ids, hidden, n_tokens, q, k, v, h_out, nullptr, 0, stream);
+  return lacache::qkv_project_rows(p, token_ids, hidden, n_tokens, q, k, v, h_out, nullptr, 0, false, stream);
 }
 
 }  // extern "C"
 
 namespace lacache {
 lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const void* hidden, int n_tokens, void* q,
-                                void* k, void* v, void* h_out, const int32_t* dst_rows, int max_rows, void* stream) {
+                                void* k, void* v, void* h_out, const int32_t* dst_rows, int max_rows, bool early_inputs,
+                                void* stream) {
   if (!p) return LACACHE_ERR_INVALID_ARG;
   if ((token_ids == nullptr) == (hidden == nullptr))
     return qfail(p, LACACHE_ERR_INVALID_ARG, "pass exactly one of token_ids and hidden");
@@ -726,6 +742,7 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   na.h_out = reinterpret_cast<__nv_bfloat16*>(h_out);
   na.dst_rows = dst_rows;
   na.max_rows = max_rows;
+  na.early_inputs = early_inputs ? 1 : 0;
   na.d_model = p->cfg.d_model;
   na.vocab = p->cfg.vocab;
   na.eps = p->cfg.rms_eps;

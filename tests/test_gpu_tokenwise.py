@@ -331,3 +331,38 @@ def test_projection_odd_shapes(d_model, hq, hkv, n):
     st, msg, q2, k2, v2, _ = project(prod, tm, n, ids=ids)
     assert torch.equal(q, q2) and torch.equal(k, k2) and torch.equal(v, v2)
     prod.destroy()
+
+
+def test_back_to_back_token_steps_match_synchronised_ones():
+    """Token-fed steps issued without any host synchronisation (the norm kernel of a step then runs
+    alongside the previous step's attention kernel) give, bit for bit, what the same calls give when
+    the host waits after each."""
+    wl = W.small_workload(prompt_lens=(300, 170), gen_len=64, block_len=32, steps=6, hq=8, hkv=4)
+    tm = TokenModel(wl, 512, 1500)
+    T = wl.total_tokens
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    ids_full = dev(tm.full_ids(0))
+    ids_steps = [dev(tm.block_ids(0, s)) for s in range(1, wl.steps_per_block + 1)]
+
+    def run(sync):
+        prod = make_producer(tm, T)
+        ctx = make_ctx(wl)
+        ctx.build_tokens(prod, 0, token_ids=ids_full)
+        res = []
+        for ids in ids_steps:
+            out, lse = new_outputs(wl)
+            ctx.step_tokens(prod, out, lse, blk_token_ids=ids)
+            if sync:
+                torch.cuda.synchronize()
+            res.append((out, lse))
+        torch.cuda.synchronize()
+        assert ctx.poll_status()[0] == binding.OK and prod.poll_status()[0] == binding.OK
+        ctx.destroy()
+        prod.destroy()
+        return res
+
+    ref = run(True)
+    for rep in range(3):
+        got = run(False)
+        for i, ((o0, l0), (o1, l1)) in enumerate(zip(ref, got)):
+            assert torch.equal(o0, o1) and torch.equal(l0, l1), "step %d differs when issued back to back" % i
