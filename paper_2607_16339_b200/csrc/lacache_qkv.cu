@@ -44,6 +44,8 @@ struct lacache_qkv {
   __nv_bfloat16* xhat = nullptr;        // [tokens_pad][d_model]
   float* ws = nullptr;                  // [2 * num_sms][256 * 128] partial tiles
   int* counters = nullptr;              // per tile: chunks accumulated so far
+  int* ready = nullptr;                 // operand rows written so far, over all calls (wraps)
+  unsigned ready_target = 0;            // what `ready` reads when the rows of the latest call are complete
   int32_t* status = nullptr;
   // scratch of the *_tokens calls, [max_tokens][H][128] each: the projections of all tokens (kept from
   // one build to the next, so that a build re-projects only the tokens that changed) and of a block
@@ -78,7 +80,7 @@ constexpr uint32_t SMQ_TOTAL = SMQ_BAR + 8 * QB_N + 32;
 static_assert(SMQ_TOTAL <= 232448, "exceeds the 227 KB per-CTA limit");
 constexpr long long Q_WAIT_CYCLES = 4000000000ll;  // ~2 s
 enum { QLOC_SMEM_ALIGN = 101, QLOC_WAIT_FULL = 102, QLOC_WAIT_FREE = 103, QLOC_WAIT_ACC_FULL = 104,
-       QLOC_WAIT_ACC_FREE = 105, QLOC_TOKEN_ID = 106, QLOC_ROW = 107 };
+       QLOC_WAIT_ACC_FREE = 105, QLOC_TOKEN_ID = 106, QLOC_ROW = 107, QLOC_WAIT_ROWS = 108 };
 
 struct GemmArgs {
   int n_tokens, tn, n_ttiles, n_tiles, kc;   // kc = d_model / 64 chunks per tile
@@ -88,6 +90,8 @@ struct GemmArgs {
   __nv_bfloat16 *q, *k, *v;
   const int32_t* dst_rows;   // output row of input token t (null: t); rows outside [0, max_rows) are dropped
   int max_rows;
+  const int* ready;          // count of operand rows the norm kernels have written (all calls, wraps)
+  int ready_target;          // its value once this call's rows are complete
   float* ws;
   int* counters;
   int32_t* status;
@@ -188,6 +192,28 @@ __device__ __forceinline__ void load_chunk(const QCta& c, const CUtensorMap* w_m
 __device__ __forceinline__ void gemm_producer(const QCta& c, const CUtensorMap* w_map, const CUtensorMap* x_map,
                                               const GemmArgs& a, long long r0, long long r1, uint32_t stage_bytes,
                                               int early) {
+  // The operand rows X^ are written by the norm kernel launched just ahead, which counts the rows it has
+  // completed.  Waiting for that count rather than for the whole grid lets this kernel work while grids
+  // further ahead in the stream (a previous step's attention kernel, which the norm kernel may run
+  // alongside) are still draining.  Every CTA of the norm kernel is resident by the time this kernel
+  // starts (it lets its dependents launch at entry), so the count always arrives; the wait is bounded anyway.
+  {
+    const long long t_start = clock64();
+    for (;;) {
+      int cnt;
+      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(cnt) : "l"(a.ready) : "memory");
+      if (cnt - a.ready_target >= 0) break;
+      if (*c.abort_flag) return;
+      if (clock64() - t_start > Q_WAIT_CYCLES) {
+        *c.abort_flag = 1;
+        if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
+          c.status[1] = QLOC_WAIT_ROWS; c.status[2] = blockIdx.x; c.status[3] = cnt;
+        }
+        return;
+      }
+    }
+    asm volatile("fence.proxy.async.global;" ::: "memory");   // the rows are read through the async proxy (TMA)
+  }
   ChunkCursor k;
   k.init(a, r0);
   const int n = (int)(r1 - r0);
@@ -256,6 +282,7 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
       tmem_ld32(tmem + lane_off + (uint32_t)(buf * MAX_TN + g * 32), r);
       tmem_ld_wait();
       if (whole) {
+        grid_dependency_wait();   // results may overwrite rows that a grid ahead in the stream still reads
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const int t = g * 32 + i;
@@ -286,6 +313,7 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (*flag) {
+        grid_dependency_wait();   // results may overwrite rows that a grid ahead in the stream still reads
         __threadfence();
         // four features per thread, four token rows per pass of the 128 threads; the loads of eight
         // passes (32 tokens) are issued together so that the tile costs a few memory round trips
@@ -409,8 +437,6 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = words[0];
-  // the operand rows X^ come from the kernel launched before this one
-  grid_dependency_wait();
 
   if (warp == 0) {
     if (tid == 0) gemm_producer(c, &w_map, &x_map, a, r0, r1, stage_bytes, early);
@@ -420,6 +446,8 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     gemm_epilogue(c, a, tmem, r0, r1, words + 2);
   }
   __syncwarp();
+  // this grid must not complete before the grids ahead of it have: whatever waits for it relies on that
+  grid_dependency_wait();
   // teardown: free TMEM once every thread is past its last TMEM access
   tc_fence_before();
   __syncthreads();
@@ -454,6 +482,7 @@ struct NormArgs {
   __nv_bfloat16* h_out;           // [n][d_model] or null
   const int32_t* dst_rows;        // or null; checked against max_rows here
   int max_rows;
+  int* ready;                     // incremented once this row of X^ is complete and visible
   int early_inputs;               // the inputs were complete before the preceding grid started: read them at once
   int d_model, vocab;
   float eps;
@@ -539,6 +568,10 @@ __global__ void __launch_bounds__(N_THREADS) qkv_norm_kernel(const NormArgs a) {
     reinterpret_cast<uint4*>(a.xhat + (size_t)t * a.d_model)[ch] = o;
     if (a.h_out && !a.early_inputs) reinterpret_cast<uint4*>(a.h_out + (size_t)t * a.d_model)[ch] = raw[i];
   }
+  // publish the row: every thread's stores, then one count
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) atomicAdd(a.ready, 1);
   if (a.early_inputs) {
     grid_dependency_wait();
     if (a.h_out) {   // a caller's buffer: not before the grids ahead are complete
@@ -605,7 +638,7 @@ bool make_bf16_map(lacache_qkv* p, CUtensorMap* m, const void* base, int rows, i
 void qkv_free(lacache_qkv* p) {
   if (!p) return;
   cudaDeviceSynchronize();
-  void* bufs[] = {p->w_packed, p->xhat, p->ws, p->counters, p->status, p->q, p->k, p->v, p->qb, p->kb, p->vb};
+  void* bufs[] = {p->w_packed, p->xhat, p->ws, p->counters, p->ready, p->status, p->q, p->k, p->v, p->qb, p->kb, p->vb};
   for (void* b : bufs)
     if (b) cudaFree(b);
   delete p;
@@ -672,6 +705,8 @@ lacache_status lacache_qkv_create(const lacache_qkv_config* cfg, lacache_qkv** o
     const int max_tiles = p->n_ftiles * ((cfg->max_tokens + 31) / 32);
     QCU_TRY(p, cudaMalloc(&p->counters, (size_t)max_tiles * 4));
     QCU_TRY(p, cudaMemset(p->counters, 0, (size_t)max_tiles * 4));
+    QCU_TRY(p, cudaMalloc(&p->ready, 4));
+    QCU_TRY(p, cudaMemset(p->ready, 0, 4));
     QCU_TRY(p, cudaMalloc(&p->status, 16));
     QCU_TRY(p, cudaMemset(p->status, 0, 16));
     QCU_TRY(p, cudaMalloc(&p->q, (size_t)cfg->max_tokens * cfg->n_q_heads * QD * 2));
@@ -743,6 +778,8 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   na.dst_rows = dst_rows;
   na.max_rows = max_rows;
   na.early_inputs = early_inputs ? 1 : 0;
+  na.ready = p->ready;
+  p->ready_target += (unsigned)n_tokens;
   na.d_model = p->cfg.d_model;
   na.vocab = p->cfg.vocab;
   na.eps = p->cfg.rms_eps;
@@ -779,6 +816,8 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   ga.v = reinterpret_cast<__nv_bfloat16*>(v);
   ga.dst_rows = dst_rows;
   ga.max_rows = max_rows;
+  ga.ready = p->ready;
+  ga.ready_target = (int)p->ready_target;
   ga.ws = p->ws;
   ga.counters = p->counters;
   ga.status = p->status;
