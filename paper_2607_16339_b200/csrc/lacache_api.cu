@@ -56,6 +56,10 @@ struct lacache_ctx {
   float *hs_out = nullptr, *hs_lse = nullptr;
 
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
+  // the role split of a step is planned once per (block, table size) and reused: a step is called
+  // thousands of times per second and the host must stay ahead of the device
+  struct StepPlan { int deep_cap = -1, ns = 0; };
+  std::vector<StepPlan> step_plan;
   int step_overlap = 1;   // consecutive steps may overlap on the device
   int steps_since_build = 0;
   int built_block = -1;
@@ -419,19 +423,22 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       a.n_items_merge = ml.n;
       long long units_merge = (long long)ml.n * Hq;
       int total = (int)std::min<long long>(c->num_sms, units_stream + units_merge);
+      const bool deep_ok = c->g.block_len <= 32 && !getenv("LACACHE_NO_DEEP");
+      const int deep_cap = deep_unit_cap();
+      if (c->step_plan.empty()) c->step_plan.resize(c->g.n_blk);
+      lacache_ctx::StepPlan& plan = c->step_plan[blk];
+      const bool planned = plan.deep_cap == deep_cap;
       double sum_tiles = 0;   // ragged batches mix short and long units on a CTA: cost a unit between mean and longest
       int longest = 1;
-      for (int i = 0; i < list.n; ++i) {
+      for (int i = 0; i < list.n && !planned; ++i) {
         const WorkItem& w = c->items_host[list.off + i];
         sum_tiles += w.kt1 - w.kt0;
         longest = std::max(longest, w.kt1 - w.kt0);
       }
       const double max_tiles = list.n > 0 ? 0.5 * (sum_tiles / list.n + longest) : 1.0;
-      int ns = 1;
+      int ns = planned ? plan.ns : 1;
       double best = 1e30;
-      const bool deep_ok = c->g.block_len <= 32 && !getenv("LACACHE_NO_DEEP");
-      const int deep_cap = deep_unit_cap();
-      for (int cand = 1; cand < total; ++cand) {
+      for (int cand = 1; cand < total && !planned; ++cand) {
         double ts = ceil((double)units_stream / cand) * (3.0 + 1.6 * max_tiles + (c->max_chunks > 1 ? 2.0 + 0.8 * c->max_chunks : 0.0));
         double per_cta = ceil((double)units_merge / (total - cand));
         double rest = 0.0;   // merge units beyond what one launch of the pipelined variant takes: further launches, all SMs
@@ -447,6 +454,8 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       if (units_merge == 0) ns = total;
       else ns = std::max(1, std::min(ns, total - 1));
       ns = (int)std::min<long long>(ns, units_stream);
+      plan.deep_cap = deep_cap;
+      plan.ns = ns;
       a.n_ctas_stream = ns;
       if (getenv("LACACHE_VERBOSE")) {
         static int printed = 0;
