@@ -42,7 +42,7 @@ struct lacache_qkv {
   int device = 0;
   __nv_bfloat16* w_packed = nullptr;    // W in tile order: [feature tile][k chunk][128 rows][64 columns]
   __nv_bfloat16* xhat = nullptr;        // [tokens_pad][d_model]
-  float* ws = nullptr;                  // [2 * num_sms][256 * 128] partial tiles
+  float* ws = nullptr;                  // [3 * num_sms][256 * 128] partial tiles
   int* counters = nullptr;              // per tile: chunks accumulated so far
   int* ready = nullptr;                 // operand rows written so far, over all calls (wraps)
   unsigned ready_target = 0;            // what `ready` reads when the rows of the latest call are complete
@@ -72,6 +72,7 @@ constexpr int G_THREADS = 192;
 constexpr int EPI_THREADS = 128;
 constexpr uint32_t A_BYTES = QD * BK * 2;
 constexpr int MAX_STAGES = 12;
+constexpr int WS_SLOTS = 3;             // partial tiles a CTA may publish
 constexpr uint32_t RING_BYTES = 229376;
 constexpr uint32_t SMQ_BAR = RING_BYTES;
 enum { QB_FULL = 0, QB_FREE = MAX_STAGES, QB_ACC_FULL = 2 * MAX_STAGES, QB_ACC_FREE = QB_ACC_FULL + 2,
@@ -80,11 +81,19 @@ constexpr uint32_t SMQ_TOTAL = SMQ_BAR + 8 * QB_N + 32;
 static_assert(SMQ_TOTAL <= 232448, "exceeds the 227 KB per-CTA limit");
 constexpr long long Q_WAIT_CYCLES = 4000000000ll;  // ~2 s
 enum { QLOC_SMEM_ALIGN = 101, QLOC_WAIT_FULL = 102, QLOC_WAIT_FREE = 103, QLOC_WAIT_ACC_FULL = 104,
-       QLOC_WAIT_ACC_FREE = 105, QLOC_TOKEN_ID = 106, QLOC_ROW = 107, QLOC_WAIT_ROWS = 108 };
+       QLOC_WAIT_ACC_FREE = 105, QLOC_TOKEN_ID = 106, QLOC_ROW = 107, QLOC_WAIT_ROWS = 108, QLOC_WAIT_PARTS = 109 };
 
 struct GemmArgs {
   int n_tokens, tn, n_ttiles, n_tiles, kc;   // kc = d_model / 64 chunks per tile
   long long total_chunks;
+  // Closer / helper split (hp > 0), used when there are more CTAs than tiles and fewer than twice as
+  // many: n_tiles of the CTAs ("closers", the high block indices) own the last kc - hp chunks of one tile
+  // each and finish it; the other CTAs ("helpers", placed first) share the first hp chunks of all tiles
+  // in equal contiguous ranges and only publish partial tiles.  Helpers start earlier and get less work
+  // than closers, so their parts are published by the time a closer is through: the closer fetches them
+  // ahead of its last MMA and finishes its tile straight from TMEM, with no publish / count / read-back
+  // round trips at the end of the kernel.
+  int hp;
   int n_stages;
   int Hq, Hkv;
   __nv_bfloat16 *q, *k, *v;
@@ -100,6 +109,7 @@ struct GemmArgs {
 struct QCta {
   uint32_t base;
   volatile int* abort_flag;
+  volatile int* rows_ready;   // set by the producer once the operand rows of this launch are complete
   int32_t* status;
   __device__ __forceinline__ uint32_t bar(int slot) const { return base + SMQ_BAR + 8u * slot; }
 };
@@ -135,13 +145,47 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
-// first chunk of CTA j's contiguous range of the (tile, chunk) list
-__device__ __forceinline__ long long range_start(const GemmArgs& a, int j) {
-  return (long long)j * a.total_chunks / (long long)gridDim.x;
+// The CTAs that share a list of (tile, chunk) pairs in equal contiguous ranges: all CTAs and kc chunks per
+// tile in the plain stream-K split; the helpers and the first hp chunks per tile in the closer / helper split.
+struct Sharing {
+  int n_ctas;        // CTAs that share the list
+  int first_cta;     // block index of the first of them
+  int kce;           // chunks per tile in the list
+  long long total;   // n_tiles * kce
+};
+__device__ __forceinline__ Sharing sharing(const GemmArgs& a) {
+  Sharing sh;
+  if (a.hp > 0) { sh.n_ctas = (int)gridDim.x - a.n_tiles; sh.first_cta = 0; sh.kce = a.hp; }   // helpers are placed first
+  else { sh.n_ctas = (int)gridDim.x; sh.first_cta = 0; sh.kce = a.kc; }
+  sh.total = (long long)a.n_tiles * sh.kce;
+  return sh;
 }
-// the CTA whose range holds chunk x
-__device__ __forceinline__ int cta_of(const GemmArgs& a, long long x) {
-  return (int)(((x + 1) * (long long)gridDim.x - 1) / a.total_chunks);
+// first list position of the j-th sharing CTA
+__device__ __forceinline__ long long range_start(const Sharing& sh, int j) {
+  return (long long)j * sh.total / (long long)sh.n_ctas;
+}
+// the sharing CTA (ordinal) whose range holds list position x
+__device__ __forceinline__ int cta_of(const Sharing& sh, long long x) {
+  return (int)(((x + 1) * (long long)sh.n_ctas - 1) / sh.total);
+}
+// This CTA's work: list positions [r0, r1) of a list with kce chunks per tile, whose chunk c is chunk
+// coff + c of the tile.  A closer's list is its own: the last kc - hp chunks of every tile.
+struct Work { long long r0, r1; int kce, coff; bool closer, helper; };
+__device__ __forceinline__ Work my_work(const GemmArgs& a) {
+  Work w;
+  const int b = (int)blockIdx.x;
+  const int n_helpers = a.hp > 0 ? (int)gridDim.x - a.n_tiles : 0;
+  w.closer = a.hp > 0 && b >= n_helpers;
+  w.helper = a.hp > 0 && b < n_helpers;
+  if (w.closer) {
+    w.kce = a.kc - a.hp; w.coff = a.hp;
+    w.r0 = (long long)(b - n_helpers) * w.kce; w.r1 = w.r0 + w.kce;
+  } else {
+    const Sharing sh = sharing(a);
+    w.kce = sh.kce; w.coff = 0;
+    w.r0 = range_start(sh, b - sh.first_cta); w.r1 = range_start(sh, b - sh.first_cta + 1);
+  }
+  return w;
 }
 
 // destination of feature tile ft, input token t: a row of q, k or v (null: the row is dropped)
@@ -159,16 +203,18 @@ __device__ __forceinline__ __nv_bfloat16* out_row(const GemmArgs& a, int ft, int
 struct ChunkCursor {
   int s; uint32_t ph;     // ring stage and its phase
   int ft, tt, ch;         // feature tile, token tile, k chunk
-  __device__ __forceinline__ void init(const GemmArgs& a, long long r0) {
+  int kce, coff;          // chunks per tile in this CTA's list; its chunk ch is chunk coff + ch of the tile
+  __device__ __forceinline__ void init(const GemmArgs& a, const Work& w) {
     s = 0; ph = 0;
-    const int tile = (int)(r0 / a.kc);
-    ch = (int)(r0 % a.kc);
+    kce = w.kce; coff = w.coff;
+    const int tile = (int)(w.r0 / kce);
+    ch = (int)(w.r0 % kce);
     ft = tile / a.n_ttiles;
     tt = tile % a.n_ttiles;
   }
   __device__ __forceinline__ void next(const GemmArgs& a) {
     if (++s == a.n_stages) { s = 0; ph ^= 1u; }
-    if (++ch == a.kc) {
+    if (++ch == kce) {
       ch = 0;
       if (++tt == a.n_ttiles) { tt = 0; ++ft; }
     }
@@ -183,15 +229,14 @@ __device__ __forceinline__ void load_chunk(const QCta& c, const CUtensorMap* w_m
   const uint32_t dst = c.base + k.s * stage_bytes;
   if (load_w) {
     mbar_expect_tx(c.bar(QB_FULL + k.s), stage_bytes);
-    tma_load_2d(dst, w_map, c.bar(QB_FULL + k.s), 0, (k.ft * a.kc + k.ch) * QD);   // one contiguous 16 KB tile
+    tma_load_2d(dst, w_map, c.bar(QB_FULL + k.s), 0, (k.ft * a.kc + k.coff + k.ch) * QD);   // one contiguous 16 KB tile
   }
-  if (load_x) tma_load_2d(dst + A_BYTES, x_map, c.bar(QB_FULL + k.s), k.ch * BK, k.tt * a.tn);
+  if (load_x) tma_load_2d(dst + A_BYTES, x_map, c.bar(QB_FULL + k.s), (k.coff + k.ch) * BK, k.tt * a.tn);
 }
 
 // `early` chunks already have their W tile in flight (issued before the wait on the preceding grid)
 __device__ __forceinline__ void gemm_producer(const QCta& c, const CUtensorMap* w_map, const CUtensorMap* x_map,
-                                              const GemmArgs& a, long long r0, long long r1, uint32_t stage_bytes,
-                                              int early) {
+                                              const GemmArgs& a, const Work& w, uint32_t stage_bytes, int early) {
   // The operand rows X^ are written by the norm kernel launched just ahead, which counts the rows it has
   // completed.  Waiting for that count rather than for the whole grid lets this kernel work while grids
   // further ahead in the stream (a previous step's attention kernel, which the norm kernel may run
@@ -213,10 +258,11 @@ __device__ __forceinline__ void gemm_producer(const QCta& c, const CUtensorMap* 
       }
     }
     asm volatile("fence.proxy.async.global;" ::: "memory");   // the rows are read through the async proxy (TMA)
+    *c.rows_ready = 1;
   }
   ChunkCursor k;
-  k.init(a, r0);
-  const int n = (int)(r1 - r0);
+  k.init(a, w);
+  const int n = (int)(w.r1 - w.r0);
   for (int it = 0; it < n; ++it, k.next(a)) {
     if (it < early) {
       load_chunk(c, w_map, x_map, a, k, stage_bytes, false, true);
@@ -227,15 +273,16 @@ __device__ __forceinline__ void gemm_producer(const QCta& c, const CUtensorMap* 
   }
 }
 
-__device__ __forceinline__ void gemm_mma(const QCta& c, const GemmArgs& a, uint32_t tmem, long long r0, long long r1,
+__device__ __forceinline__ void gemm_mma(const QCta& c, const GemmArgs& a, uint32_t tmem, const Work& w,
                                          uint32_t stage_bytes) {
+  const long long r0 = w.r0, r1 = w.r1;
   const uint32_t idesc = idesc_f16(1u /*bf16*/, 0u, QD, (uint32_t)a.tn);
   int s = 0;
   uint32_t ph = 0;
   int seg = 0;
   for (long long x = r0; x < r1; ++seg) {
-    const int c0 = (int)(x % a.kc);
-    const int c1 = (int)min((long long)a.kc, c0 + (r1 - x));
+    const int c0 = (int)(x % w.kce);
+    const int c1 = (int)min((long long)w.kce, c0 + (r1 - x));
     const int buf = seg & 1;
     // the epilogue of the segment that used this accumulator two segments ago has drained it
     if (!q_wait(c, QB_ACC_FREE + buf, ((uint32_t)(seg >> 1) & 1u) ^ 1u, QLOC_WAIT_ACC_FREE)) return;
@@ -257,8 +304,102 @@ __device__ __forceinline__ void gemm_mma(const QCta& c, const GemmArgs& a, uint3
   }
 }
 
-__device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, uint32_t tmem, long long r0,
-                                              long long r1, volatile uint32_t* flag) {
+// A closer finishes its tile: the helpers' parts of the tile (published earlier, as a rule) are fetched
+// ahead of the last MMA, then added to the accumulator straight from TMEM in ascending chunk order
+// (helper parts first, then this CTA's chunks), rounded and stored.
+__device__ __forceinline__ void closer_epilogue(const QCta& c, const GemmArgs& a, uint32_t tmem, const Work& w,
+                                                volatile uint32_t* flag) {
+  const int tid = threadIdx.x;
+  const int et = tid - 64;
+  const int quad = (tid >> 5) & 3;
+  const int f = quad * 32 + (tid & 31);
+  const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
+  const int tile = (int)blockIdx.x - ((int)gridDim.x - a.n_tiles);
+  const int ft = tile / a.n_ttiles, tt = tile % a.n_ttiles;
+  const int t0 = tt * a.tn;
+  const int nt = min(a.tn, a.n_tokens - t0);
+  // Every helper part of the tile has been published once the tile's counter shows all hp chunks.  The
+  // counter is looked at only after this launch's operand rows are complete: every earlier launch of the
+  // handle (whose closer may not have reset the counter yet) is then over.
+  if (et == 0) {
+    const long long t_start = clock64();
+    uint32_t ok = 1;
+    for (;;) {
+      int cnt = -1;
+      if (*c.rows_ready)
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(cnt) : "l"(a.counters + tile) : "memory");
+      if (cnt == a.hp) break;
+      if (*c.abort_flag) { ok = 0; break; }
+      if (clock64() - t_start > Q_WAIT_CYCLES) {
+        *c.abort_flag = 1;
+        if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
+          c.status[1] = QLOC_WAIT_PARTS; c.status[2] = blockIdx.x; c.status[3] = cnt;
+        }
+        ok = 0;
+        break;
+      }
+    }
+    if (ok) a.counters[tile] = 0;                  // ready for the next launch
+    *flag = ok;
+  }
+  asm volatile("bar.sync 1, 128;" ::: "memory");
+  if (*flag == 0) return;
+  __threadfence();
+  // the helpers whose ranges touch the first hp chunks of this tile, in ascending order (at most three:
+  // a helper's range is at least hp long)
+  const Sharing sh = sharing(a);
+  const long long x_lo = (long long)tile * sh.kce;
+  const int j_lo = cta_of(sh, x_lo), j_hi = cta_of(sh, x_lo + sh.kce - 1);
+  const float *p0 = nullptr, *p1 = nullptr, *p2 = nullptr;
+  int n_parts = 0;
+  for (int j = j_lo; j <= j_hi; ++j) {
+    const long long s0 = range_start(sh, j), s1 = range_start(sh, j + 1);
+    if (s1 <= s0) continue;
+    const int slot = tile - (int)(s0 / sh.kce);    // the ordinal of this tile among the helper's segments
+    const float* p = a.ws + ((size_t)(sh.first_cta + j) * WS_SLOTS + slot) * (size_t)(MAX_TN * QD) + f;
+    if (n_parts == 0) p0 = p; else if (n_parts == 1) p1 = p; else p2 = p;
+    ++n_parts;
+  }
+  for (int g = 0; g * 32 < nt; ++g) {
+    float pre0[32], pre1[32], pre2[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int t = g * 32 + i;
+      const size_t o = (size_t)t * QD;
+      pre0[i] = (t < nt && n_parts > 0) ? __ldcg(p0 + o) : 0.f;
+      pre1[i] = (t < nt && n_parts > 1) ? __ldcg(p1 + o) : 0.f;
+      pre2[i] = (t < nt && n_parts > 2) ? __ldcg(p2 + o) : 0.f;
+    }
+    if (g == 0) {
+      if (!q_wait(c, QB_ACC_FULL, 0, QLOC_WAIT_ACC_FULL)) return;
+      tc_fence_after();
+      grid_dependency_wait();   // results may overwrite rows that a grid ahead in the stream still reads
+    }
+    uint32_t r[32];
+    tmem_ld32(tmem + lane_off + (uint32_t)(g * 32), r);
+    tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int t = g * 32 + i;
+      float sum = 0.f + pre0[i];
+      if (n_parts > 1) sum += pre1[i];
+      if (n_parts > 2) sum += pre2[i];
+      sum += __uint_as_float(r[i]);
+      if (t < nt) {
+        __nv_bfloat16* dst = out_row(a, ft, t0 + t);
+        if (dst) dst[f] = __float2bfloat16_rn(sum);
+      }
+    }
+  }
+  tc_fence_before();
+  mbar_arrive(c.bar(QB_ACC_FREE));
+}
+
+__device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, uint32_t tmem, const Work& w,
+                                              volatile uint32_t* flag) {
+  if (w.closer) { closer_epilogue(c, a, tmem, w, flag); return; }
+  const long long r0 = w.r0, r1 = w.r1;
+  const Sharing sh = sharing(a);
   const int tid = threadIdx.x;
   const int et = tid - 64;                       // 0..127
   const int quad = (tid >> 5) & 3;               // the TMEM lane quadrant this warp may read
@@ -266,17 +407,18 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
   const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
   int seg = 0;
   for (long long x = r0; x < r1; ++seg) {
-    const int tile = (int)(x / a.kc), c0 = (int)(x % a.kc);
-    const int c1 = (int)min((long long)a.kc, c0 + (r1 - x));
+    const int tile = (int)(x / w.kce), c0 = (int)(x % w.kce);
+    const int c1 = (int)min((long long)w.kce, c0 + (r1 - x));
     const int ft = tile / a.n_ttiles, tt = tile % a.n_ttiles;
     const int t0 = tt * a.tn;
     const int nt = min(a.tn, a.n_tokens - t0);   // valid tokens of the tile
     const int buf = seg & 1;
-    const bool whole = (c0 == 0 && c1 == a.kc);
+    const bool whole = !w.helper && (c0 == 0 && c1 == a.kc);
     if (!q_wait(c, QB_ACC_FULL + buf, (uint32_t)(seg >> 1) & 1u, QLOC_WAIT_ACC_FULL)) return;
     tc_fence_after();
-    // a CTA's range leaves at most its first and its last segment partial: two workspace slots
-    float* part = a.ws + ((size_t)blockIdx.x * 2 + (seg == 0 ? 0 : 1)) * (size_t)(MAX_TN * QD);
+    // plain split: a CTA's range leaves at most its first and its last segment partial (slots 0 and 1);
+    // a helper publishes every segment, of which it has at most three
+    float* part = a.ws + ((size_t)blockIdx.x * WS_SLOTS + (w.helper ? seg : (seg == 0 ? 0 : 1))) * (size_t)(MAX_TN * QD);
     for (int g = 0; g * 32 < nt; ++g) {
       uint32_t r[32];
       tmem_ld32(tmem + lane_off + (uint32_t)(buf * MAX_TN + g * 32), r);
@@ -307,7 +449,8 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (et == 0) {
         const int old = atomicAdd(a.counters + tile, c1 - c0);
-        const uint32_t last = (old + (c1 - c0) == a.kc) ? 1u : 0u;
+        // (a helper's tiles are finished by their closers)
+        const uint32_t last = (!w.helper && old + (c1 - c0) == a.kc) ? 1u : 0u;
         if (last) a.counters[tile] = 0;           // ready for the next launch
         *flag = last;
       }
@@ -318,17 +461,17 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
         // four features per thread, four token rows per pass of the 128 threads; the loads of eight
         // passes (32 tokens) are issued together so that the tile costs a few memory round trips
         const long long x_lo = (long long)tile * a.kc, x_hi = x_lo + a.kc;
-        const int j_lo = cta_of(a, x_lo), j_hi = cta_of(a, x_hi - 1);
+        const int j_lo = cta_of(sh, x_lo), j_hi = cta_of(sh, x_hi - 1);
         const int f4 = (et & 31) * 4, tr = et >> 5;
         // the tile's parts in ascending CTA order (a fixed summation order); with up to three of them,
         // the usual case, the loads of all parts are in flight together
         const float *p0 = nullptr, *p1 = nullptr, *p2 = nullptr;
         int n_parts = 0;
         for (int j = j_lo; j <= j_hi; ++j) {
-          const long long s0 = range_start(a, j), s1 = range_start(a, j + 1);
+          const long long s0 = range_start(sh, j), s1 = range_start(sh, j + 1);
           if (s1 <= s0) continue;                   // a CTA without work
           const int slot = (s0 >= x_lo) ? 0 : 1;    // the tile holds its first segment, or its last
-          const float* p = a.ws + ((size_t)j * 2 + slot) * (size_t)(MAX_TN * QD) + f4;
+          const float* p = a.ws + ((size_t)j * WS_SLOTS + slot) * (size_t)(MAX_TN * QD) + f4;
           if (n_parts == 0) p0 = p; else if (n_parts == 1) p1 = p; else if (n_parts == 2) p2 = p;
           ++n_parts;
         }
@@ -355,10 +498,10 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
 #pragma unroll
             for (int i = 0; i < 8; ++i) acc[i] = zero4;
             for (int j = j_lo; j <= j_hi; ++j) {
-              const long long s0 = range_start(a, j), s1 = range_start(a, j + 1);
+              const long long s0 = range_start(sh, j), s1 = range_start(sh, j + 1);
               if (s1 <= s0) continue;
               const int slot = (s0 >= x_lo) ? 0 : 1;
-              const float* p = a.ws + ((size_t)j * 2 + slot) * (size_t)(MAX_TN * QD) + f4;
+              const float* p = a.ws + ((size_t)j * WS_SLOTS + slot) * (size_t)(MAX_TN * QD) + f4;
               float4 v[8];
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
@@ -404,12 +547,14 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
   c.base = smem_u32(smem_raw);
   uint32_t* words = reinterpret_cast<uint32_t*>(smem_raw + SMQ_BAR + 8 * QB_N);  // [0] tmem, [1] abort, [2] flag
   c.abort_flag = reinterpret_cast<volatile int*>(words + 1);
+  c.rows_ready = reinterpret_cast<volatile int*>(words + 3);
   c.status = a.status;
   if ((c.base & 1023u) != 0) {
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = QLOC_SMEM_ALIGN;
     return;
   }
-  const long long r0 = range_start(a, blockIdx.x), r1 = range_start(a, blockIdx.x + 1);
+  const Work w = my_work(a);
+  const long long r0 = w.r0, r1 = w.r1;
   const uint32_t stage_bytes = A_BYTES + (uint32_t)a.tn * 128u;
   int early = 0;
   if (tid == 0) {
@@ -418,13 +563,14 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     for (int i = 0; i < QB_N; ++i) mbar_init(c.bar(i), (i >= QB_ACC_FREE) ? EPI_THREADS : 1);
     words[1] = 0;
     words[2] = 0;
+    words[3] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
     // the weights do not depend on the kernel before this one: fill the ring with W tiles right away
     // (the X^ tiles of the same stages follow after the wait below)
     early = (int)min((long long)a.n_stages, r1 - r0);
     ChunkCursor k;
-    k.init(a, r0);
+    k.init(a, w);
     for (int it = 0; it < early; ++it, k.next(a)) load_chunk(c, &w_map, &x_map, a, k, stage_bytes, true, false);
   }
   __syncwarp();
@@ -439,11 +585,11 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
   const uint32_t tmem = words[0];
 
   if (warp == 0) {
-    if (tid == 0) gemm_producer(c, &w_map, &x_map, a, r0, r1, stage_bytes, early);
+    if (tid == 0) gemm_producer(c, &w_map, &x_map, a, w, stage_bytes, early);
   } else if (warp == 1) {
-    if (tid == 32) gemm_mma(c, a, tmem, r0, r1, stage_bytes);
+    if (tid == 32) gemm_mma(c, a, tmem, w, stage_bytes);
   } else {
-    gemm_epilogue(c, a, tmem, r0, r1, words + 2);
+    gemm_epilogue(c, a, tmem, w, words + 2);
   }
   __syncwarp();
   // this grid must not complete before the grids ahead of it have: whatever waits for it relies on that
@@ -701,7 +847,7 @@ lacache_status lacache_qkv_create(const lacache_qkv_config* cfg, lacache_qkv** o
     const size_t d = (size_t)cfg->d_model;
     QCU_TRY(p, cudaMalloc(&p->xhat, (size_t)p->tokens_pad * d * 2));
     QCU_TRY(p, cudaMemset(p->xhat, 0, (size_t)p->tokens_pad * d * 2));
-    QCU_TRY(p, cudaMalloc(&p->ws, (size_t)2 * p->num_sms * MAX_TN * QD * 4));
+    QCU_TRY(p, cudaMalloc(&p->ws, (size_t)WS_SLOTS * p->num_sms * MAX_TN * QD * 4));
     const int max_tiles = p->n_ftiles * ((cfg->max_tokens + 31) / 32);
     QCU_TRY(p, cudaMalloc(&p->counters, (size_t)max_tiles * 4));
     QCU_TRY(p, cudaMemset(p->counters, 0, (size_t)max_tiles * 4));
@@ -822,6 +968,16 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   ga.counters = p->counters;
   ga.status = p->status;
   const int n_ctas = (int)std::min<long long>(p->num_sms, ga.total_chunks);
+  ga.hp = 0;
+  if (ga.tn <= 64 && n_ctas > ga.n_tiles && n_ctas < 2 * ga.n_tiles && !getenv("LACACHE_QKV_PLAIN_SPLIT")) {
+    // closers take `per_closer` chunks each, helpers about HEAD_START chunks fewer
+    const int HEAD_START = 8;
+    const int n_helpers = n_ctas - ga.n_tiles;
+    const long long num = ga.total_chunks + (long long)n_helpers * HEAD_START;
+    const int per_closer = (int)((num + n_ctas - 1) / n_ctas);
+    const int hp = ga.kc - per_closer;
+    if (hp >= 1 && (long long)ga.n_tiles * hp >= n_helpers) ga.hp = hp;
+  }
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_ctas);
