@@ -434,7 +434,7 @@ def run_cuda(args):
 # the step fed by token ids: embedding gather + RMS norm + Q/K/V projection in front
 # ----------------------------------------------------------------------------
 D_MODEL = {32: 4096, 28: 3584}     # first-layer width of the model a workload is shaped like, by query heads
-QKV_TRAFFIC_PER_LAUNCH = {2: 104626944}   # ncu, profiles/qkv_gemm_kernel_cfg2_step_ncu_full.txt
+QKV_TRAFFIC_PER_LAUNCH = {2: 104751872}   # ncu, profiles/qkv_gemm_kernel_cfg2_step_ncu_full.txt
 
 
 def token_path_leg(wl, dev, peaks, seed, n_steps):
