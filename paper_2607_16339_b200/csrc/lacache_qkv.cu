@@ -14,7 +14,10 @@
 //                    contiguous ranges to one persistent CTA per SM.  A CTA that owns only part of a
 //                    tile's chunks leaves its fp32 partial in a workspace; the last CTA to arrive at a
 //                    tile adds the partials in CTA order (the result does not depend on arrival order)
-//                    and writes the bf16 rows.
+//                    and writes the bf16 rows.  With more CTAs than tiles and fewer than twice as many
+//                    (a step at LLaDA width) the cut is by role instead, see GemmArgs::hp.  The kernel
+//                    does not wait for the norm grid but for the count of operand rows it publishes,
+//                    and for the grids ahead of it only before its final stores and its exit.
 // Warp roles of the GEMM: warp 0 (one lane) TMA producer over a ring of stages, warp 1 (one lane) MMA
 // issuer, warps 2..5 epilogue (TMEM lane = output feature).  Two accumulators alternate so that an
 // epilogue overlaps the next segment's MMAs.  Every mbarrier wait is bounded; a wait that runs out sets
