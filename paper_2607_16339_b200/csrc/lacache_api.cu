@@ -416,7 +416,17 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
     // persistent grid: one CTA per SM, split between the two roles by a cost
     // estimate (units x per-unit cost, in arbitrary time units)
     const int Hq = c->g.Hq;
-    long long units_stream = (long long)list.n * Hq;
+    a.stream_slots = Hq; a.pack = 1; a.pack_rows = 0;
+    if (mode == MODE_STEP && c->g.group >= 2 && !getenv("LACACHE_NO_PACK")) {
+      // block queries of a GQA model: heads of one KV group side by side in the 128 lanes of a tile
+      const int rows = c->g.block_len <= 32 ? 32 : 64;
+      const int pack = std::min(128 / rows, c->g.group);
+      if (pack >= 2) {
+        a.pack = pack; a.pack_rows = rows;
+        a.stream_slots = c->g.Hkv * ((c->g.group + pack - 1) / pack);
+      }
+    }
+    long long units_stream = (long long)list.n * a.stream_slots;
     if (mode == MODE_STEP) {
       lacache_ctx::ListRef ml = c->merge_list[blk];
       a.items_merge = c->d_items + ml.off;

@@ -93,6 +93,10 @@ struct AttnArgs {
   // tcgen05 only: items of the merge role (fixed rows of a step), CTA split
   const WorkItem* items_merge; int n_items_merge;
   int n_ctas_stream; int n_ctas;
+  // tcgen05, stream role: units per item.  Normally one per query head.  In a step of a GQA model the
+  // block rows of `pack` query heads of one KV group share a 128-row tile (they read the same keys and
+  // values): units then count (KV head, group of `pack` heads) pairs, each head taking `pack_rows` lanes.
+  int stream_slots; int pack; int pack_rows;
   int merge_deep;            // merge role runs its pipelined variant (block_len <= 32, bounded units per CTA)
   int split_merge;           // host only: more merge units per CTA than the pipelined variant tabulates, so the
                              // fixed rows of the step go out in several launches of that variant

@@ -48,6 +48,9 @@ struct TcMaps {
   // of one head, laid out in shared memory as [plane][half][rows][64] (128-byte swizzle)
   alignas(64) CUtensorMap q;       // box 128 rows
   alignas(64) CUtensorMap q64;     // box 64 rows (block queries)
+  // block queries of `pack` heads of one KV group side by side: dimensions ordered {64, rows, heads, halves,
+  // planes}, box {64, pack_rows, pack, 2, 2}: lands as [plane][half][head][row][64], i.e. one 128-row tile
+  alignas(64) CUtensorMap q_pack;
   alignas(64) CUtensorMap k;       // box TC_KEYS rows (stream role)
   alignas(64) CUtensorMap k64;     // box 64 rows (the block's keys, merge role)
   alignas(64) CUtensorMap k32;     // box 32 rows (the block's keys, pipelined merge role)
@@ -227,13 +230,37 @@ struct Unit {
   int k0, k1, x0, x1;     // valid keys [k0, k1) minus [x0, x1)
   int epi, chunk, nchunks;
   int q_rows;             // rows of the Q box: 128 or 64
+  int nh, rh;             // packed block queries: nh heads h, h + 1, ... of one KV group, rh lanes each (rh = 0: one head)
 };
+// head and row within the head's rows of tile row r; whether r holds a real query row (rh is 0, 32 or 64)
+__device__ __forceinline__ int unit_head(const Unit& un, int r) { return un.rh ? un.h + (r >> (un.rh == 64 ? 6 : 5)) : un.h; }
+__device__ __forceinline__ int unit_row(const Unit& un, int r) { return un.rh ? (r & (un.rh - 1)) : r; }
+__device__ __forceinline__ bool unit_row_valid(const Unit& un, int r) {
+  return un.rh ? ((r >> (un.rh == 64 ? 6 : 5)) < un.nh && (r & (un.rh - 1)) < un.nrows) : r < un.nrows;
+}
 
+// PACKED (a.pack > 1): the units are block queries of several heads side by side in one tile.  A template
+// parameter of the whole kernel, so that the kernel a build or an MHA step runs carries none of the per-row
+// head arithmetic: this kernel is sensitive to its code size.
+template <bool PACKED>
 __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs& a, const WorkItem& it, int u) {
   Unit un;
-  un.h = u % g.Hq;   // units are head-minor: unit u = item u / Hq of head u % Hq (a CTA's units, a fixed
-                     // stride apart, then cycle through the items instead of drawing one item's heads)
-  un.kh = un.h / g.group;
+  // units are head-minor: unit u = item u / slots of head (or head group) u % slots (a CTA's units, a
+  // fixed stride apart, then cycle through the items instead of drawing one item's heads)
+  const int slot = u % (PACKED ? a.stream_slots : g.Hq);
+  if (PACKED) {
+    const int per_kv = (g.group + a.pack - 1) / a.pack;
+    un.kh = slot / per_kv;
+    const int s = slot % per_kv;
+    un.h = un.kh * g.group + s * a.pack;
+    un.nh = min(a.pack, g.group - s * a.pack);
+    un.rh = a.pack_rows;
+  } else {
+    un.h = slot;
+    un.kh = un.h / g.group;
+    un.nh = 1;
+    un.rh = 0;
+  }
   un.seq = it.seq;
   un.row0 = it.row0;
   un.nrows = it.nrows;
@@ -256,7 +283,7 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
     un.chunk = it.chunk;
     un.nchunks = it.pad;
     un.epi = it.pad > 1 ? EPI_PARTIAL : EPI_OUT;
-    un.q_rows = 64;
+    un.q_rows = un.rh ? BM : 64;
   } else {
     un.epi = EPI_OUT;
   }
@@ -306,11 +333,13 @@ __device__ __forceinline__ void load_kv_tile(const TcMaps& maps, uint32_t kv_bas
   load_qk_box(kv_base, &maps.k64, bar, krow, kh);
   load_v_box(kv_base + KV_V, &maps.v64, bar, krow, kh);
 }
-__device__ __forceinline__ void load_q_tile(const Cta& c, const TcMaps& maps, int q_rows, int row0, int h) {
+__device__ __forceinline__ void load_q_tile(const Cta& c, const TcMaps& maps, int q_rows, int row0, int h,
+                                            bool packed = false) {
   const uint32_t bar = c.bar(BAR_Q_FULL);
   const uint32_t box = (uint32_t)q_rows * 128u;
   mbar_expect_tx(bar, 4 * box);
-  load_qk_box(c.base + SM_Q, q_rows == 64 ? &maps.q64 : &maps.q, bar, row0, h);
+  if (packed) tma_load_5d(c.base + SM_Q, &maps.q_pack, bar, 0, row0, h, 0, 0);   // heads h, h + 1, ... side by side
+  else load_qk_box(c.base + SM_Q, q_rows == 64 ? &maps.q64 : &maps.q, bar, row0, h);
 }
 
 // ===========================================================================
@@ -325,14 +354,16 @@ struct TileCursor {
   Unit un;
   bool valid, q_done, loads_q;
 };
+template <bool PACKED>
 __device__ __forceinline__ void cursor_load_unit(const Geometry& g, const AttnArgs& a, TileCursor& cu, int n_units) {
   cu.valid = cu.u < n_units;
   if (!cu.valid) return;
-  cu.it = load_item(a.items + cu.u / g.Hq);
-  cu.un = decode_stream(g, a, cu.it, cu.u);
+  cu.it = load_item(a.items + cu.u / (PACKED ? a.stream_slots : g.Hq));
+  cu.un = decode_stream<PACKED>(g, a, cu.it, cu.u);
   cu.t = cu.un.t0;
   cu.q_done = !cu.loads_q;
 }
+template <bool PACKED>
 __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs& a, TileCursor& cu, int stride,
                                                int n_units) {
   // move to the next tile; cross into the next unit(s) when this one is exhausted
@@ -343,20 +374,21 @@ __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs
   while (cu.valid && cu.t >= cu.un.t1 && cu.q_done) {
     cu.u += stride;
     ++cu.uu;
-    cursor_load_unit(g, a, cu, n_units);
+    cursor_load_unit<PACKED>(g, a, cu, n_units);
   }
 }
 
+template <bool PACKED>
 __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a,
                                 int first, int stride, int n_units, WorkItem it) {
   // three independent cursors: Q tiles (one per unit), key tiles, value tiles
   TileCursor cq, ck, cv;
   cq.u = first; cq.uu = 0; cq.jj = 0; cq.loads_q = true;
-  cursor_load_unit(g, a, cq, n_units);
+  cursor_load_unit<PACKED>(g, a, cq, n_units);
   ck = cq;
   ck.loads_q = false;  // the key and value cursors never load Q
   ck.q_done = true;
-  if (ck.valid && ck.t >= ck.un.t1) cursor_advance(g, a, ck, stride, n_units);
+  if (ck.valid && ck.t >= ck.un.t1) cursor_advance<PACKED>(g, a, ck, stride, n_units);
   cv = ck;
   // What the RoPE kernel launched just before this one writes must not be loaded
   // before that grid has completed (this kernel may have started early): in a step
@@ -380,15 +412,15 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         mbar_arrive(c.bar(BAR_Q_FULL));
         cq.q_done = true;
         cq.t = cq.un.t1;
-        cursor_advance(g, a, cq, stride, n_units);
+        cursor_advance<PACKED>(g, a, cq, stride, n_units);
         did = true;
       } else if (!dep_done) {
         blocked_on_dep = true;
       } else if (cq.uu == 0 || mbar_test(c.bar(BAR_Q_FREE), (cq.uu - 1) & 1)) {
-        load_q_tile(c, maps, cq.un.q_rows, cq.un.row0, cq.un.h);
+        load_q_tile(c, maps, cq.un.q_rows, cq.un.row0, cq.un.h, cq.un.rh != 0);
         cq.q_done = true;
         cq.t = cq.un.t1;
-        cursor_advance(g, a, cq, stride, n_units);
+        cursor_advance<PACKED>(g, a, cq, stride, n_units);
         did = true;
       }
     }
@@ -402,7 +434,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         const uint32_t khi = c.base + SM_K + sk * K_STAGE;
         mbar_expect_tx(bar, 4 * KS_BOX);
         load_qk_box(khi, &maps.k, bar, krow, ck.un.kh);  // the lo plane lands at khi + SK_LO
-        cursor_advance(g, a, ck, stride, n_units);
+        cursor_advance<PACKED>(g, a, ck, stride, n_units);
         did = true;
       }
     }
@@ -415,7 +447,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
         mbar_expect_tx(bar, 2 * KS_BOX);
         load_v_box(vb, &maps.v, bar, krow, cv.un.kh);
-        cursor_advance(g, a, cv, stride, n_units);
+        cursor_advance<PACKED>(g, a, cv, stride, n_units);
         did = true;
       }
     }
@@ -448,6 +480,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
 // Scores of tile j need its keys and the score buffer of tile j - 2 read (= the probabilities of tile
 // j - 2 written); P~V of tile j needs its probabilities and its values.  Each code block exists once
 // (the unrolled MMA sequences are large, and cold instruction fetches are slow).
+template <bool PACKED>
 __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
                                   int n_units, WorkItem it) {
   constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
@@ -455,8 +488,8 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   uint32_t js = 0;  // score tiles issued so far (stage and buffer = js & 1, phase = (js >> 1) & 1)
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / g.Hq);
-    const Unit un = decode_stream(g, a, it, u);
+    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
+    const Unit un = decode_stream<PACKED>(g, a, it, u);
     const uint32_t q_box = (uint32_t)un.q_rows * 128u;
     const int n_tiles = un.t1 - un.t0;
     if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
@@ -478,14 +511,15 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   }
 }
 
+template <bool PACKED>
 __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
                               int n_units, WorkItem it) {
   int uu = 0;
   uint32_t jp = 0;  // P~V tiles issued so far
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / g.Hq);
-    const Unit un = decode_stream(g, a, it, u);
+    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
+    const Unit un = decode_stream<PACKED>(g, a, it, u);
     const int n_tiles = un.t1 - un.t0;
     // O~ of the previous unit has been read by the row threads (observed once per unit, in order)
     if (uu >= 1 && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
@@ -631,6 +665,7 @@ __device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs
   }
 }
 
+template <bool PACKED>
 __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units,
                             WorkItem it) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -644,8 +679,8 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
   int jj = 0;
   for (int u = first; u < n_units; u += stride) {
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / g.Hq);
-    const Unit un = decode_stream(g, a, it, u);
+    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
+    const Unit un = decode_stream<PACKED>(g, a, it, u);
     it = nxt;
     if (u == first && a.mode == MODE_STEP && a.q_raw != nullptr) {
       // The CTA's first unit: rotate the block's queries of this (sequence, head) here,
@@ -654,10 +689,12 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       // by the row), so this unit does not wait for that kernel.
       const int tq = threadIdx.x - 64;
       const uint32_t box = (uint32_t)un.q_rows * 128u;
-      for (int i = tq; i < un.nrows * 8; i += ROW_THREADS) {
+      const int tile_rows = PACKED ? un.nh * un.rh : un.nrows;
+      for (int i = tq; i < tile_rows * 8; i += ROW_THREADS) {
         const int qi = i >> 3, ch = i & 7, c0 = ch * 8;
-        const size_t src = (size_t)un.seq * g.block_len + qi;            // row of the block's inputs
-        const size_t soff = (src * g.Hq + un.h) * D;
+        if (PACKED && !unit_row_valid(un, qi)) continue;   // lanes between a short block and the next head's rows
+        const size_t src = (size_t)un.seq * g.block_len + unit_row(un, qi);   // row of the block's inputs
+        const size_t soff = (src * g.Hq + unit_head(un, qi)) * D;
         float x1[8], x2[8], cs[8], sn[8], y1[8], y2[8];
         rope_load8(a.q_raw, soff + c0, a.q_raw_bf16 != 0, x1);
         rope_load8(a.q_raw, soff + c0 + D / 2, a.q_raw_bf16 != 0, x2);
@@ -679,9 +716,10 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       fence_async_smem();  // the MMA reads shared memory through the async proxy
       mbar_arrive(c.bar(BAR_QC));
     }
-    const int row = un.row0 + r;
-    const bool row_valid = r < un.nrows;
-    const bool active = quad * 32 < un.nrows;  // this warp holds at least one real row
+    const int row = un.row0 + unit_row(un, r);   // token of this tile row
+    const int hrow = unit_head(un, r);           // and its query head
+    const bool row_valid = unit_row_valid(un, r);
+    const bool active = unit_row_valid(un, quad * 32);  // this warp holds at least one real row (its first)
     float m_ref = -INFINITY, l_part = 0.f;
     bool first_tile = true;
 
@@ -828,12 +866,13 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       // Partial state of this key chunk, straight from TMEM to global memory (each
       // thread 256 contiguous bytes of its row); the last chunk of the (sequence,
       // head) to arrive merges all of them.
-      const size_t pbase = ((size_t)un.seq * g.Hq + un.h) * a.max_chunks;  // [chunk][block_len]
+      const size_t pbase = ((size_t)un.seq * g.Hq + hrow) * a.max_chunks;  // [chunk][block_len], of this row's head
       const size_t prow0 = (pbase + un.chunk) * g.block_len;
+      const int r_blk = unit_row(un, r);
       {
         // (the TMEM loads are warp-wide: rows past the block take part in them and only skip the
         // stores, so a block length that is not a multiple of 32 cannot split a warp around them)
-        float4* dst = reinterpret_cast<float4*>(a.part_o + (prow0 + r) * D + 64 * half);
+        float4* dst = reinterpret_cast<float4*>(a.part_o + (prow0 + r_blk) * D + 64 * half);
 #pragma unroll 1
         for (int cb = 0; cb < 4; ++cb) {
           uint32_t rr[16];
@@ -851,24 +890,33 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
                                             __uint_as_float(rr[4 * i + 2]), __uint_as_float(rr[4 * i + 3]));
           }
         }
-        if (row_valid && half == 0) { a.part_m[prow0 + r] = m_ref; a.part_l[prow0 + r] = l_run; }
+        if (row_valid && half == 0) { a.part_m[prow0 + r_blk] = m_ref; a.part_l[prow0 + r_blk] = l_run; }
       }
       tc_fence_before();
       mbar_arrive(c.bar(BAR_O_FREE));  // the next unit may overwrite O~
       if (!epi_sync(c, epi_phase)) return;  // every partial store of the CTA happens-before thread 64's fence
       if (threadIdx.x == 64) {
-        __threadfence();  // cumulative: publishes the whole CTA's partial state before the count
-        int* cnt = &a.counters[un.seq * g.Hq + un.h];
-        int old = atomicAdd(cnt, 1);
-        int last = (old == un.nchunks - 1) ? 1 : 0;
-        if (last) {
-          *cnt = 0;
-          __threadfence();  // the other chunks' partial states are visible from here on
+        __threadfence();  // cumulative: publishes the whole CTA's partial state before the counts
+        uint32_t last_bits = 0;   // bit j: this chunk was the last of head un.h + j to arrive
+        for (int j = 0; j < un.nh; ++j) {
+          int* cnt = &a.counters[un.seq * g.Hq + un.h + j];
+          const int old = atomicAdd(cnt, 1);
+          if (old == un.nchunks - 1) {
+            *cnt = 0;
+            last_bits |= 1u << j;
+          }
         }
-        *c.flag = (uint32_t)last;
+        if (last_bits) __threadfence();  // the other chunks' partial states are visible from here on
+        *c.flag = last_bits;
       }
       if (!epi_sync(c, epi_phase)) return;
-      if (*c.flag != 0) merge_partials(g, a, pbase, un.nchunks, g.block_len, un.row0, un.h);
+      {
+        const uint32_t last_bits = *c.flag;
+        for (int j = 0; j < un.nh; ++j)
+          if (last_bits & (1u << j))
+            merge_partials(g, a, ((size_t)un.seq * g.Hq + un.h + j) * a.max_chunks, un.nchunks, g.block_len, un.row0,
+                           un.h + j);
+      }
       if (!epi_sync(c, epi_phase)) return;  // the flag may be rewritten
       if (un.q_rows == BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));
       continue;
@@ -935,10 +983,12 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       if (!epi_sync(c, epi_phase)) return;
       coop_store_rows(c, stage_off, a.st.o + ((size_t)un.h * g.Tp + un.row0) * D, D, un.nrows);
     } else if (un.epi == EPI_OUT) {
-      const size_t orow = (size_t)row * g.Hq + un.h;
+      const size_t orow = (size_t)row * g.Hq + hrow;
       if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_ref + log2f(l_run)) * LN2;
       if (!epi_sync(c, epi_phase)) return;
-      coop_store_rows(c, stage_off, a.out + ((size_t)un.row0 * g.Hq + un.h) * D, (size_t)g.Hq * D, un.nrows);
+      for (int j = 0; j < un.nh; ++j)   // one head's rows at a time (a single head unless block queries are packed)
+        coop_store_rows(c, stage_off + (uint32_t)(j * un.rh) * STAGE_ROW, a.out + ((size_t)un.row0 * g.Hq + un.h + j) * D,
+                        (size_t)g.Hq * D, un.nrows);
     }
     if (!epi_sync(c, epi_phase)) return;  // the staging rows have been read
     if (un.q_rows == BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));  // the Q region may be reloaded
@@ -1479,8 +1529,11 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
   }
 }
 
+template <bool PACKED>
 __global__ void __launch_bounds__(THREADS, 1)
 tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const AttnArgs a) {
+  // (instantiated twice, as two kernels: PACKED for the steps of a GQA model whose block queries share
+  // tiles across heads, see decode_stream)
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -1504,14 +1557,14 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   const bool stream = (int)blockIdx.x < a.n_ctas_stream;
   int first, stride, n_units;
   if (stream) {
-    first = blockIdx.x; stride = a.n_ctas_stream; n_units = a.n_items * g.Hq;
+    first = blockIdx.x; stride = a.n_ctas_stream; n_units = a.n_items * (PACKED ? a.stream_slots : g.Hq);
   } else {
     first = blockIdx.x - a.n_ctas_stream; stride = n_ctas_merge; n_units = a.n_items_merge * g.Hq;
   }
   const bool deep = !stream && a.merge_deep != 0;
   if (tid == 0) {  // descriptor fetches overlap the set-up below
     if (stream) {
-      prefetch_map(a.mode == MODE_STEP ? &maps.q64 : &maps.q);
+      prefetch_map(a.mode == MODE_STEP ? (PACKED ? &maps.q_pack : &maps.q64) : &maps.q);
       prefetch_map(&maps.k); prefetch_map(&maps.v);
     } else {
       prefetch_map(&maps.q); prefetch_map(&maps.st_o); prefetch_map(&maps.out);
@@ -1520,7 +1573,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   }
   const int n_my = first < n_units ? (n_units - first + stride - 1) / stride : 0;
   WorkItem it0{};
-  if (!deep && first < n_units) it0 = stream ? load_item(a.items + first / g.Hq)
+  if (!deep && first < n_units) it0 = stream ? load_item(a.items + first / (PACKED ? a.stream_slots : g.Hq))
                                              : load_item(a.items_merge + first / g.Hq);
   if ((c.base & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = LOC_SMEM_ALIGN;
@@ -1570,7 +1623,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
 
   if (warp == 0) {
     if (stream) {
-      if (tid == 0) stream_producer(c, maps, g, a, first, stride, n_units, it0);
+      if (tid == 0) stream_producer<PACKED>(c, maps, g, a, first, stride, n_units, it0);
     } else if (deep) {
       if (tid == 0) deep_producer(c, maps, g, n_my, a.k_raw != nullptr);
     } else {
@@ -1578,14 +1631,14 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     }
   } else if (warp == 1) {
     if (tid == 32) {
-      if (stream) stream_mma_scores(c, g, a, first, stride, n_units, it0);
+      if (stream) stream_mma_scores<PACKED>(c, g, a, first, stride, n_units, it0);
       else if (deep) deep_mma(c, g, n_my, a.k_raw != nullptr);
       else merge_mma(c, g, a, first, stride, n_units);
     }
   } else if (warp == 10) {
-    if (tid == 320 && stream) stream_mma_pv(c, g, a, first, stride, n_units, it0);
+    if (tid == 320 && stream) stream_mma_pv<PACKED>(c, g, a, first, stride, n_units, it0);
   } else {
-    if (stream) stream_rows(c, g, a, first, stride, n_units, it0);
+    if (stream) stream_rows<PACKED>(c, g, a, first, stride, n_units, it0);
     else if (deep) deep_rows(c, g, a, n_my);
     else merge_rows(c, maps, g, a, first, stride, n_units, it0);
     bulk_wait_read();
@@ -1659,6 +1712,21 @@ bool make_qk_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* 
   if (r != CUDA_SUCCESS) { snprintf(err, errlen, "cuTensorMapEncodeTiled (5-D) failed with CUresult %d", (int)r); return false; }
   return true;
 }
+// The same planes with the head dimension inside the half dimension, so that a box of `pack` heads x
+// `rows` rows lands as one [plane][half][pack * rows][64] tile.
+bool make_qpack_map(CUtensorMap* m, void* base, int H, int Tp, int rows, int pack, char* err, int errlen) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) { snprintf(err, errlen, "cuTensorMapEncodeTiled entry point not found"); return false; }
+  cuuint64_t dims[5] = {64, (cuuint64_t)Tp, (cuuint64_t)H, 2, 2};
+  cuuint64_t strides[4] = {128, (cuuint64_t)Tp * 256, (cuuint64_t)Tp * 128, (cuuint64_t)H * Tp * 256};
+  cuuint32_t box[5] = {64, (cuuint32_t)rows, (cuuint32_t)pack, 2, 2};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { snprintf(err, errlen, "cuTensorMapEncodeTiled (packed heads) failed with CUresult %d", (int)r); return false; }
+  return true;
+}
 bool make_v_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* err, int errlen) {
   EncodeTiledFn enc = get_encode();
   if (!enc) { snprintf(err, errlen, "cuTensorMapEncodeTiled entry point not found"); return false; }
@@ -1676,7 +1744,9 @@ bool make_v_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* e
 }  // namespace
 
 cudaError_t tc_prepare() {
-  return cudaFuncSetAttribute(tc_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
+  cudaError_t e = cudaFuncSetAttribute(tc_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(tc_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
 }
 
 bool tc_set_out(TcMaps* m, const Geometry& g, float* out, char* err, int errlen) {
@@ -1695,6 +1765,8 @@ TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, c
   // (the lo planes follow the hi planes at a fixed distance: see alloc_rot)
   bool ok = make_qk_map(&m->q, rot.q_hi, g.Hq, g.Tp, BM, err, errlen) &&
             make_qk_map(&m->q64, rot.q_hi, g.Hq, g.Tp, 64, err, errlen) &&
+            make_qpack_map(&m->q_pack, rot.q_hi, g.Hq, g.Tp, g.block_len <= 32 ? 32 : 64,
+                           std::max(1, std::min(g.block_len <= 32 ? 4 : 2, g.group)), err, errlen) &&
             make_qk_map(&m->k, rot.k_hi, g.Hkv, g.Tp, BN, err, errlen) &&
             make_qk_map(&m->k64, rot.k_hi, g.Hkv, g.Tp, 64, err, errlen) &&
             make_qk_map(&m->k32, rot.k_hi, g.Hkv, g.Tp, 32, err, errlen) &&
@@ -1723,7 +1795,8 @@ cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* map
   cfg.attrs = attr;
   static const bool no_pdl = getenv("LACACHE_NO_PDL") != nullptr;
   cfg.numAttrs = no_pdl ? 0 : 1;
-  return cudaLaunchKernelEx(&cfg, tc_attn_kernel, *maps, g, a);
+  if (a.pack > 1) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true>, *maps, g, a);
+  return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false>, *maps, g, a);
 }
 
 }  // namespace lacache
