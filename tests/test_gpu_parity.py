@@ -120,6 +120,17 @@ def test_block_lengths_that_split_a_warp(block_len):
     _run_points(wl, "tc", seed=8, blocks=[0, wl.n_blocks - 1], sc_tiles_per_chunk=2)
 
 
+@pytest.mark.parametrize("hq,hkv,block_len", [(6, 2, 64), (10, 2, 32), (7, 1, 64), (14, 2, 16)])
+def test_packed_block_queries_odd_groups(hq, hkv, block_len):
+    """GQA steps put the block rows of two (blocks of 33..64 rows) or four (up to 32 rows) heads of a KV
+    group into one tile.  Groups that do not divide evenly leave a last, partly filled tile; with the
+    keys cut into chunks every head of a tile has its own arrival counter and is merged on its own."""
+    wl = small_workload(name="pack%d_%d_%d" % (hq, hkv, block_len), prompt_lens=(420, 150), gen_len=64,
+                        block_len=block_len, steps=2, hq=hq, hkv=hkv, scale_mode="inv_sqrt_d")
+    for tiles_per_chunk in (0, 2):
+        _run_points(wl, "tc", seed=12, blocks=[0, wl.n_blocks - 1], sc_tiles_per_chunk=tiles_per_chunk)
+
+
 @pytest.mark.parametrize("engine", ["simt", "tc"])
 def test_cached_state_matches_oracle_state(engine):
     wl = small_workload(prompt_lens=(150, 40), gen_len=96, block_len=32, steps=1, hq=4, hkv=2, d=128)
