@@ -242,7 +242,7 @@ __device__ __forceinline__ bool unit_row_valid(const Unit& un, int r) {
 // PACKED (a.pack > 1): the units are block queries of several heads side by side in one tile.  A template
 // parameter of the whole kernel, so that the kernel a build or an MHA step runs carries none of the per-row
 // head arithmetic: this kernel is sensitive to its code size.
-template <bool PACKED>
+template <bool PACKED, bool STEP>
 __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs& a, const WorkItem& it, int u) {
   Unit un;
   // units are head-minor: unit u = item u / slots of head (or head group) u % slots (a CTA's units, a
@@ -273,11 +273,11 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
   un.chunk = 0;
   un.nchunks = 1;
   un.q_rows = BM;
-  if (a.mode == MODE_BUILD) {
+  if (!STEP && a.mode == MODE_BUILD) {
     un.x0 = it.blk_start;
     un.x1 = it.blk_start + g.block_len;
     un.epi = EPI_STATE;
-  } else if (a.mode == MODE_STEP) {
+  } else if (STEP) {
     un.t0 = it.kt0;
     un.t1 = it.kt1;
     un.chunk = it.chunk;
@@ -354,16 +354,16 @@ struct TileCursor {
   Unit un;
   bool valid, q_done, loads_q;
 };
-template <bool PACKED>
+template <bool PACKED, bool STEP>
 __device__ __forceinline__ void cursor_load_unit(const Geometry& g, const AttnArgs& a, TileCursor& cu, int n_units) {
   cu.valid = cu.u < n_units;
   if (!cu.valid) return;
   cu.it = load_item(a.items + cu.u / (PACKED ? a.stream_slots : g.Hq));
-  cu.un = decode_stream<PACKED>(g, a, cu.it, cu.u);
+  cu.un = decode_stream<PACKED, STEP>(g, a, cu.it, cu.u);
   cu.t = cu.un.t0;
   cu.q_done = !cu.loads_q;
 }
-template <bool PACKED>
+template <bool PACKED, bool STEP>
 __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs& a, TileCursor& cu, int stride,
                                                int n_units) {
   // move to the next tile; cross into the next unit(s) when this one is exhausted
@@ -374,21 +374,21 @@ __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs
   while (cu.valid && cu.t >= cu.un.t1 && cu.q_done) {
     cu.u += stride;
     ++cu.uu;
-    cursor_load_unit<PACKED>(g, a, cu, n_units);
+    cursor_load_unit<PACKED, STEP>(g, a, cu, n_units);
   }
 }
 
-template <bool PACKED>
+template <bool PACKED, bool STEP>
 __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a,
                                 int first, int stride, int n_units, WorkItem it) {
   // three independent cursors: Q tiles (one per unit), key tiles, value tiles
   TileCursor cq, ck, cv;
   cq.u = first; cq.uu = 0; cq.jj = 0; cq.loads_q = true;
-  cursor_load_unit<PACKED>(g, a, cq, n_units);
+  cursor_load_unit<PACKED, STEP>(g, a, cq, n_units);
   ck = cq;
   ck.loads_q = false;  // the key and value cursors never load Q
   ck.q_done = true;
-  if (ck.valid && ck.t >= ck.un.t1) cursor_advance<PACKED>(g, a, ck, stride, n_units);
+  if (ck.valid && ck.t >= ck.un.t1) cursor_advance<PACKED, STEP>(g, a, ck, stride, n_units);
   cv = ck;
   // What the RoPE kernel launched just before this one writes must not be loaded
   // before that grid has completed (this kernel may have started early): in a step
@@ -396,9 +396,9 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
   // that overlap the block -- so tiles of fixed tokens are requested at once and
   // the wait comes only when nothing else can be issued.
   bool dep_done = false;
-  const bool q_computed = a.mode == MODE_STEP && a.q_raw != nullptr;
+  const bool q_computed = STEP && a.q_raw != nullptr;
   auto tile_depends = [&](const TileCursor& cu) {
-    if (a.mode != MODE_STEP) return true;
+    if (!STEP) return true;
     const int krow = cu.un.key_base + cu.t * BN;
     return krow < cu.it.blk_start + g.block_len && krow + BN > cu.it.blk_start;
   };
@@ -412,7 +412,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         mbar_arrive(c.bar(BAR_Q_FULL));
         cq.q_done = true;
         cq.t = cq.un.t1;
-        cursor_advance<PACKED>(g, a, cq, stride, n_units);
+        cursor_advance<PACKED, STEP>(g, a, cq, stride, n_units);
         did = true;
       } else if (!dep_done) {
         blocked_on_dep = true;
@@ -420,7 +420,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         load_q_tile(c, maps, cq.un.q_rows, cq.un.row0, cq.un.h, cq.un.rh != 0);
         cq.q_done = true;
         cq.t = cq.un.t1;
-        cursor_advance<PACKED>(g, a, cq, stride, n_units);
+        cursor_advance<PACKED, STEP>(g, a, cq, stride, n_units);
         did = true;
       }
     }
@@ -434,7 +434,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         const uint32_t khi = c.base + SM_K + sk * K_STAGE;
         mbar_expect_tx(bar, 4 * KS_BOX);
         load_qk_box(khi, &maps.k, bar, krow, ck.un.kh);  // the lo plane lands at khi + SK_LO
-        cursor_advance<PACKED>(g, a, ck, stride, n_units);
+        cursor_advance<PACKED, STEP>(g, a, ck, stride, n_units);
         did = true;
       }
     }
@@ -447,7 +447,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
         mbar_expect_tx(bar, 2 * KS_BOX);
         load_v_box(vb, &maps.v, bar, krow, cv.un.kh);
-        cursor_advance<PACKED>(g, a, cv, stride, n_units);
+        cursor_advance<PACKED, STEP>(g, a, cv, stride, n_units);
         did = true;
       }
     }
@@ -480,7 +480,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
 // Scores of tile j need its keys and the score buffer of tile j - 2 read (= the probabilities of tile
 // j - 2 written); P~V of tile j needs its probabilities and its values.  Each code block exists once
 // (the unrolled MMA sequences are large, and cold instruction fetches are slow).
-template <bool PACKED>
+template <bool PACKED, bool STEP>
 __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
                                   int n_units, WorkItem it) {
   constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
@@ -489,11 +489,11 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
-    const Unit un = decode_stream<PACKED>(g, a, it, u);
+    const Unit un = decode_stream<PACKED, STEP>(g, a, it, u);
     const uint32_t q_box = (uint32_t)un.q_rows * 128u;
     const int n_tiles = un.t1 - un.t0;
     if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
-    if (uu == 0 && a.mode == MODE_STEP && a.q_raw != nullptr && !wait_bar(c, BAR_QC, 0, LOC_WAIT_Q)) return;
+    if (uu == 0 && STEP && a.q_raw != nullptr && !wait_bar(c, BAR_QC, 0, LOC_WAIT_Q)) return;
     for (int j = 0; j < n_tiles; ++j, ++js) {
       const uint32_t sk = js & 1u, b = js & 1u;
       // the score buffer was last used two tiles ago (possibly by the previous unit): its
@@ -511,7 +511,7 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   }
 }
 
-template <bool PACKED>
+template <bool PACKED, bool STEP>
 __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
                               int n_units, WorkItem it) {
   int uu = 0;
@@ -519,7 +519,7 @@ __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
-    const Unit un = decode_stream<PACKED>(g, a, it, u);
+    const Unit un = decode_stream<PACKED, STEP>(g, a, it, u);
     const int n_tiles = un.t1 - un.t0;
     // O~ of the previous unit has been read by the row threads (observed once per unit, in order)
     if (uu >= 1 && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
@@ -665,7 +665,7 @@ __device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs
   }
 }
 
-template <bool PACKED>
+template <bool PACKED, bool STEP>
 __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units,
                             WorkItem it) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -680,9 +680,9 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
   for (int u = first; u < n_units; u += stride) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
-    const Unit un = decode_stream<PACKED>(g, a, it, u);
+    const Unit un = decode_stream<PACKED, STEP>(g, a, it, u);
     it = nxt;
-    if (u == first && a.mode == MODE_STEP && a.q_raw != nullptr) {
+    if (u == first && STEP && a.q_raw != nullptr) {
       // The CTA's first unit: rotate the block's queries of this (sequence, head) here,
       // with the very arithmetic of the RoPE kernel, and write them where the TMA load
       // would have put them ([plane][feature half][row][64], 16-byte chunks XOR-swizzled
@@ -1529,7 +1529,7 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
   }
 }
 
-template <bool PACKED>
+template <bool PACKED, bool STEP>
 __global__ void __launch_bounds__(THREADS, 1)
 tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const AttnArgs a) {
   // (instantiated twice, as two kernels: PACKED for the steps of a GQA model whose block queries share
@@ -1541,7 +1541,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   // wrote, and every global store below comes after a wait on that kernel: the next step's kernels may
   // therefore be scheduled as SMs free up (they, too, wait before their first store).  A build or a
   // full recompute writes what a following step would read early, so they do not trigger.
-  if (a.mode == MODE_STEP && a.step_overlap) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (STEP && a.step_overlap) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   Cta c;
   c.base = smem_u32(smem_raw);
   c.gen = smem_raw;
@@ -1554,7 +1554,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   const int n_ctas_merge = (int)gridDim.x - a.n_ctas_stream;
   // stream-role CTAs take the low block indices (they are scheduled first: the block
   // queries' chain of key tiles is the longest dependent chain of a step)
-  const bool stream = (int)blockIdx.x < a.n_ctas_stream;
+  const bool stream = !STEP || (int)blockIdx.x < a.n_ctas_stream;   // (only a step has fixed rows to merge)
   int first, stride, n_units;
   if (stream) {
     first = blockIdx.x; stride = a.n_ctas_stream; n_units = a.n_items * (PACKED ? a.stream_slots : g.Hq);
@@ -1564,7 +1564,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   const bool deep = !stream && a.merge_deep != 0;
   if (tid == 0) {  // descriptor fetches overlap the set-up below
     if (stream) {
-      prefetch_map(a.mode == MODE_STEP ? (PACKED ? &maps.q_pack : &maps.q64) : &maps.q);
+      prefetch_map(STEP ? (PACKED ? &maps.q_pack : &maps.q64) : &maps.q);
       prefetch_map(&maps.k); prefetch_map(&maps.v);
     } else {
       prefetch_map(&maps.q); prefetch_map(&maps.st_o); prefetch_map(&maps.out);
@@ -1623,7 +1623,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
 
   if (warp == 0) {
     if (stream) {
-      if (tid == 0) stream_producer<PACKED>(c, maps, g, a, first, stride, n_units, it0);
+      if (tid == 0) stream_producer<PACKED, STEP>(c, maps, g, a, first, stride, n_units, it0);
     } else if (deep) {
       if (tid == 0) deep_producer(c, maps, g, n_my, a.k_raw != nullptr);
     } else {
@@ -1631,14 +1631,14 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     }
   } else if (warp == 1) {
     if (tid == 32) {
-      if (stream) stream_mma_scores<PACKED>(c, g, a, first, stride, n_units, it0);
+      if (stream) stream_mma_scores<PACKED, STEP>(c, g, a, first, stride, n_units, it0);
       else if (deep) deep_mma(c, g, n_my, a.k_raw != nullptr);
       else merge_mma(c, g, a, first, stride, n_units);
     }
   } else if (warp == 10) {
-    if (tid == 320 && stream) stream_mma_pv<PACKED>(c, g, a, first, stride, n_units, it0);
+    if (tid == 320 && stream) stream_mma_pv<PACKED, STEP>(c, g, a, first, stride, n_units, it0);
   } else {
-    if (stream) stream_rows<PACKED>(c, g, a, first, stride, n_units, it0);
+    if (stream) stream_rows<PACKED, STEP>(c, g, a, first, stride, n_units, it0);
     else if (deep) deep_rows(c, g, a, n_my);
     else merge_rows(c, maps, g, a, first, stride, n_units, it0);
     bulk_wait_read();
@@ -1744,9 +1744,11 @@ bool make_v_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* e
 }  // namespace
 
 cudaError_t tc_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(tc_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
+  cudaError_t e = cudaFuncSetAttribute(tc_attn_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(tc_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
+  e = cudaFuncSetAttribute(tc_attn_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(tc_attn_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
 }
 
 bool tc_set_out(TcMaps* m, const Geometry& g, float* out, char* err, int errlen) {
@@ -1795,8 +1797,10 @@ cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* map
   cfg.attrs = attr;
   static const bool no_pdl = getenv("LACACHE_NO_PDL") != nullptr;
   cfg.numAttrs = no_pdl ? 0 : 1;
-  if (a.pack > 1) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true>, *maps, g, a);
-  return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false>, *maps, g, a);
+  // three instantiations: build / full recompute, the step of an MHA model, the step of a GQA model
+  if (a.mode != MODE_STEP) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, false>, *maps, g, a);
+  if (a.pack > 1) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true, true>, *maps, g, a);
+  return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, true>, *maps, g, a);
 }
 
 }  // namespace lacache
