@@ -1529,7 +1529,7 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
   }
 }
 
-template <bool PACKED, bool STEP>
+template <bool PACKED, bool STEP, bool DEEP>
 __global__ void __launch_bounds__(THREADS, 1)
 tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const AttnArgs a) {
   // (instantiated twice, as two kernels: PACKED for the steps of a GQA model whose block queries share
@@ -1561,7 +1561,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   } else {
     first = blockIdx.x - a.n_ctas_stream; stride = n_ctas_merge; n_units = a.n_items_merge * g.Hq;
   }
-  const bool deep = !stream && a.merge_deep != 0;
+  const bool deep = !stream && DEEP;   // (DEEP: a.merge_deep, which variant of the merge role this launch runs)
   if (tid == 0) {  // descriptor fetches overlap the set-up below
     if (stream) {
       prefetch_map(STEP ? (PACKED ? &maps.q_pack : &maps.q64) : &maps.q);
@@ -1744,11 +1744,14 @@ bool make_v_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* e
 }  // namespace
 
 cudaError_t tc_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(tc_attn_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(tc_attn_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(tc_attn_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
+  const void* kernels[] = {(const void*)tc_attn_kernel<false, false, false>, (const void*)tc_attn_kernel<false, true, false>,
+                           (const void*)tc_attn_kernel<false, true, true>, (const void*)tc_attn_kernel<true, true, false>,
+                           (const void*)tc_attn_kernel<true, true, true>};
+  for (const void* k : kernels) {
+    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 bool tc_set_out(TcMaps* m, const Geometry& g, float* out, char* err, int errlen) {
@@ -1797,10 +1800,15 @@ cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* map
   cfg.attrs = attr;
   static const bool no_pdl = getenv("LACACHE_NO_PDL") != nullptr;
   cfg.numAttrs = no_pdl ? 0 : 1;
-  // three instantiations: build / full recompute, the step of an MHA model, the step of a GQA model
-  if (a.mode != MODE_STEP) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, false>, *maps, g, a);
-  if (a.pack > 1) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true, true>, *maps, g, a);
-  return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, true>, *maps, g, a);
+  // five instantiations: build / full recompute; the step of an MHA and of a GQA model, each with
+  // either variant of the merge role
+  if (a.mode != MODE_STEP) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, false, false>, *maps, g, a);
+  if (a.pack > 1) {
+    if (a.merge_deep) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true, true, true>, *maps, g, a);
+    return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true, true, false>, *maps, g, a);
+  }
+  if (a.merge_deep) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, true, true>, *maps, g, a);
+  return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, true, false>, *maps, g, a);
 }
 
 }  // namespace lacache
