@@ -529,7 +529,7 @@ def token_path_leg(wl, dev, peaks, seed, n_steps):
 # (profiles/tc_attn_kernel_cfg2_ncu_full.txt, tc_attn_kernel_cfg{3,4,5}_step_ncu_full.txt),
 # bytes; None where no capture exists for the workload.  The fp32 output (12.6 MB) is still in L2 when the
 # kernel ends, so the figure is dominated by reads.
-TRAFFIC_PER_LAUNCH = {2: 45288448, 3: 93736960, 4: 456532736, 5: 208314880}
+TRAFFIC_PER_LAUNCH = {2: 45337856, 3: 93736960, 4: 456532736, 5: 208314880}
 
 
 # ----------------------------------------------------------------------------
