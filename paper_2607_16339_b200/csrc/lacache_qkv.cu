@@ -174,12 +174,15 @@ __device__ __forceinline__ int cta_of(const Sharing& sh, long long x) {
 // This CTA's work: list positions [r0, r1) of a list with kce chunks per tile, whose chunk c is chunk
 // coff + c of the tile.  A closer's list is its own: the last kc - hp chunks of every tile.
 struct Work { long long r0, r1; int kce, coff; bool closer, helper; };
+// BY_ROLE: the closer / helper split (a.hp > 0); a template parameter of the kernel, which then carries
+// only the epilogue code of the split it runs
+template <bool BY_ROLE>
 __device__ __forceinline__ Work my_work(const GemmArgs& a) {
   Work w;
   const int b = (int)blockIdx.x;
-  const int n_helpers = a.hp > 0 ? (int)gridDim.x - a.n_tiles : 0;
-  w.closer = a.hp > 0 && b >= n_helpers;
-  w.helper = a.hp > 0 && b < n_helpers;
+  const int n_helpers = BY_ROLE ? (int)gridDim.x - a.n_tiles : 0;
+  w.closer = BY_ROLE && b >= n_helpers;
+  w.helper = BY_ROLE && b < n_helpers;
   if (w.closer) {
     w.kce = a.kc - a.hp; w.coff = a.hp;
     w.r0 = (long long)(b - n_helpers) * w.kce; w.r1 = w.r0 + w.kce;
@@ -398,9 +401,10 @@ __device__ __forceinline__ void closer_epilogue(const QCta& c, const GemmArgs& a
   mbar_arrive(c.bar(QB_ACC_FREE));
 }
 
+template <bool BY_ROLE>
 __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, uint32_t tmem, const Work& w,
                                               volatile uint32_t* flag) {
-  if (w.closer) { closer_epilogue(c, a, tmem, w, flag); return; }
+  if (BY_ROLE && w.closer) { closer_epilogue(c, a, tmem, w, flag); return; }
   const long long r0 = w.r0, r1 = w.r1;
   const Sharing sh = sharing(a);
   const int tid = threadIdx.x;
@@ -416,12 +420,12 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
     const int t0 = tt * a.tn;
     const int nt = min(a.tn, a.n_tokens - t0);   // valid tokens of the tile
     const int buf = seg & 1;
-    const bool whole = !w.helper && (c0 == 0 && c1 == a.kc);
+    const bool whole = !BY_ROLE && (c0 == 0 && c1 == a.kc);
     if (!q_wait(c, QB_ACC_FULL + buf, (uint32_t)(seg >> 1) & 1u, QLOC_WAIT_ACC_FULL)) return;
     tc_fence_after();
     // plain split: a CTA's range leaves at most its first and its last segment partial (slots 0 and 1);
     // a helper publishes every segment, of which it has at most three
-    float* part = a.ws + ((size_t)blockIdx.x * WS_SLOTS + (w.helper ? seg : (seg == 0 ? 0 : 1))) * (size_t)(MAX_TN * QD);
+    float* part = a.ws + ((size_t)blockIdx.x * WS_SLOTS + (BY_ROLE ? seg : (seg == 0 ? 0 : 1))) * (size_t)(MAX_TN * QD);
     for (int g = 0; g * 32 < nt; ++g) {
       uint32_t r[32];
       tmem_ld32(tmem + lane_off + (uint32_t)(buf * MAX_TN + g * 32), r);
@@ -453,7 +457,7 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
       if (et == 0) {
         const int old = atomicAdd(a.counters + tile, c1 - c0);
         // (a helper's tiles are finished by their closers)
-        const uint32_t last = (!w.helper && old + (c1 - c0) == a.kc) ? 1u : 0u;
+        const uint32_t last = (!BY_ROLE && old + (c1 - c0) == a.kc) ? 1u : 0u;
         if (last) a.counters[tile] = 0;           // ready for the next launch
         *flag = last;
       }
@@ -537,6 +541,7 @@ __device__ __forceinline__ void gemm_epilogue(const QCta& c, const GemmArgs& a, 
   }
 }
 
+template <bool BY_ROLE>
 __global__ void __launch_bounds__(G_THREADS, 1)
 qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant__ CUtensorMap x_map,
                 const GemmArgs a) {
@@ -556,7 +561,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = QLOC_SMEM_ALIGN;
     return;
   }
-  const Work w = my_work(a);
+  const Work w = my_work<BY_ROLE>(a);
   const long long r0 = w.r0, r1 = w.r1;
   const uint32_t stage_bytes = A_BYTES + (uint32_t)a.tn * 128u;
   int early = 0;
@@ -592,7 +597,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
   } else if (warp == 1) {
     if (tid == 32) gemm_mma(c, a, tmem, w, stage_bytes);
   } else {
-    gemm_epilogue(c, a, tmem, w, words + 2);
+    gemm_epilogue<BY_ROLE>(c, a, tmem, w, words + 2);
   }
   __syncwarp();
   // this grid must not complete before the grids ahead of it have: whatever waits for it relies on that
@@ -874,7 +879,8 @@ lacache_status lacache_qkv_create(const lacache_qkv_config* cfg, lacache_qkv** o
     if (!make_bf16_map(p, &p->w_map, p->w_packed, w_rows * (cfg->d_model / BK), BK, QD)) return LACACHE_ERR_CUDA;
     for (int i = 0; i < 4; ++i)
       if (!make_bf16_map(p, &p->x_map[i], p->xhat, p->tokens_pad, cfg->d_model, 32 << i)) return LACACHE_ERR_CUDA;
-    QCU_TRY(p, cudaFuncSetAttribute(qkv_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMQ_TOTAL));
+    QCU_TRY(p, cudaFuncSetAttribute(qkv_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMQ_TOTAL));
+    QCU_TRY(p, cudaFuncSetAttribute(qkv_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMQ_TOTAL));
     return LACACHE_OK;
   };
   st = attempt();
@@ -993,7 +999,8 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
     cfg.numAttrs = 0;   // an event between the two kernels: an ordinary launch
     QCU_TRY(p, cudaEventRecord(p->ev_start, s));
   }
-  QCU_TRY(p, cudaLaunchKernelEx(&cfg, qkv_gemm_kernel, p->w_map, p->x_map[tn_idx], ga));
+  if (ga.hp > 0) QCU_TRY(p, cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<true>, p->w_map, p->x_map[tn_idx], ga));
+  else QCU_TRY(p, cudaLaunchKernelEx(&cfg, qkv_gemm_kernel<false>, p->w_map, p->x_map[tn_idx], ga));
   if (p->ev_start && p->ev_stop) QCU_TRY(p, cudaEventRecord(p->ev_stop, s));
   p->last_launches++;
   return LACACHE_OK;
