@@ -747,7 +747,6 @@ lacache_status step_impl(lacache_ctx* c, const void* q, const void* k, const voi
     a.q_raw = q;
     a.k_raw = k;
     a.v_raw = v;
-    a.q_raw_bf16 = c->cfg.dtype == LACACHE_DTYPE_BF16 ? 1 : 0;
     a.row_cos = r.row_cos;
     a.row_sin = r.row_sin;
   }

@@ -103,7 +103,7 @@ struct AttnArgs {
   // step only: the block's pre-RoPE queries [B * block_len, Hq, d] and the cos/sin rows of
   // those tokens [B * block_len][d/2]; a CTA's first block-query unit rotates its Q tile
   // from these itself and so does not have to wait for the RoPE kernel
-  const void* q_raw; int q_raw_bf16; const float* row_cos; const float* row_sin;
+  const void* q_raw; const float* row_cos; const float* row_sin;   // (bf16: the tcgen05 engine takes bf16 inputs only)
   // likewise the block's pre-RoPE keys and values [B * block_len, Hkv, d]: the first unit of a
   // pipelined merge-role CTA rotates the block's keys / converts its values itself
   const void* k_raw; const void* v_raw;

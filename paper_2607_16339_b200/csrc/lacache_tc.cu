@@ -696,8 +696,8 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         const size_t src = (size_t)un.seq * g.block_len + unit_row(un, qi);   // row of the block's inputs
         const size_t soff = (src * g.Hq + unit_head(un, qi)) * D;
         float x1[8], x2[8], cs[8], sn[8], y1[8], y2[8];
-        rope_load8(a.q_raw, soff + c0, a.q_raw_bf16 != 0, x1);
-        rope_load8(a.q_raw, soff + c0 + D / 2, a.q_raw_bf16 != 0, x2);
+        rope_load8(a.q_raw, soff + c0, true, x1);
+        rope_load8(a.q_raw, soff + c0 + D / 2, true, x2);
         const float4* cp = reinterpret_cast<const float4*>(a.row_cos + src * (D / 2) + c0);
         const float4* sp = reinterpret_cast<const float4*>(a.row_sin + src * (D / 2) + c0);
         const float4 ca = cp[0], cb = cp[1], sa = sp[0], sb = sp[1];
@@ -1402,8 +1402,8 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
       const size_t src = (size_t)un.seq * L + ki;
       const size_t soff = (src * g.Hkv + kh) * D;
       float x1[8], x2[8], cs[8], sn[8], y1[8], y2[8];
-      rope_load8(a.k_raw, soff + c0, a.q_raw_bf16 != 0, x1);
-      rope_load8(a.k_raw, soff + c0 + D / 2, a.q_raw_bf16 != 0, x2);
+      rope_load8(a.k_raw, soff + c0, true, x1);
+      rope_load8(a.k_raw, soff + c0 + D / 2, true, x2);
       const float4* cp = reinterpret_cast<const float4*>(a.row_cos + src * (D / 2) + c0);
       const float4* sp = reinterpret_cast<const float4*>(a.row_sin + src * (D / 2) + c0);
       const float4 ca = cp[0], cb = cp[1], sa = sp[0], sb = sp[1];
@@ -1420,8 +1420,8 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
       *reinterpret_cast<uint4*>(k0 + 3 * DM_KBOX) = l2;
       // values: the same two 8-feature chunks of row ki, unrotated
       float v1[8], v2[8];
-      rope_load8(a.v_raw, soff + c0, a.q_raw_bf16 != 0, v1);
-      rope_load8(a.v_raw, soff + c0 + D / 2, a.q_raw_bf16 != 0, v2);
+      rope_load8(a.v_raw, soff + c0, true, v1);
+      rope_load8(a.v_raw, soff + c0 + D / 2, true, v2);
       uint8_t* const v0 = c.gen + DM_V + ki * 128 + ((ch ^ (ki & 7)) << 4);
       *reinterpret_cast<uint4*>(v0) = rope_half8(v1);
       *reinterpret_cast<uint4*>(v0 + DM_KBOX) = rope_half8(v2);
