@@ -582,7 +582,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
     for (int it = 0; it < early; ++it, k.next(a)) load_chunk(c, &w_map, &x_map, a, k, stage_bytes, true, false);
   }
   __syncwarp();
-  if (warp == 0) {
+  if (warp == 1) {  // (warp 1 allocates while thread 0 is still initialising barriers and requesting weights)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(words)), "r"(512)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -605,7 +605,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
   // teardown: free TMEM once every thread is past its last TMEM access
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == 1) {  // the warp that allocated
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
   }
 }

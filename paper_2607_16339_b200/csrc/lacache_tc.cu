@@ -1610,7 +1610,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     }
   }
   __syncwarp();
-  if (warp == 0) {
+  if (warp == 1) {  // (warp 1 allocates while thread 0 is still initialising the barriers)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(words)),
                  "r"(TM_COLS)
                  : "memory");
@@ -1648,7 +1648,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   // teardown: free TMEM once every thread is past its last TMEM access
   tc_fence_before();
   mbar_arrive(c.bar(BAR_DONE));
-  if (warp == 0) {
+  if (warp == 1) {  // the warp that allocated
     wait_bar(c, BAR_DONE, 0, LOC_WAIT_O);
     __syncwarp();
     tc_fence_after();
