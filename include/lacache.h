@@ -106,6 +106,34 @@ lacache_status lacache_build(lacache_ctx* ctx, int block_idx, const void* q_pre,
                              const void* k_pre, const void* v_pre, void* cuda_stream);
 
 /*
+ * Incremental rebuild across blocks (an extension: the paper refills the cache for every block,
+ * Sec. 3.3.1 "recomputed once per block"; the result is the state of Eq. 2-6 over the same key
+ * set, reached in another order).  Between block b and block b + 1 of a sequence the fixed set
+ * changes by U_{b+1} = U_b + C_b - C_{b+1}, and only the rows of C_b change their Q/K/V (their
+ * tokens were decoded).  Online softmax (Eq. 2-6) can add keys to a state but not take them out, so
+ * the context keeps a second state per token, the *prefix state*: (m, l, O~) over the keys before
+ * the current block.  Then
+ *   - prefix state of block b + 1 = prefix state of block b, extended by the keys of C_b (rows of
+ *     C_b themselves are computed over all keys before block b + 1 from scratch);
+ *   - cached state of block b + 1 = that prefix state, extended by the keys after block b + 1.
+ * Work per advance is N x (L_b + suffix length) score columns per row instead of N x (N - L_b).
+ *
+ * lacache_build_incremental: as lacache_build (same arguments, same cached state up to rounding
+ * order), and leaves the prefix state of block_idx behind.  Allocates the prefix state (the size of
+ * the (m, l, O~) cache) on first use: LACACHE_ERR_OOM if that fails.
+ * lacache_build_advance: from the block the context holds (built by lacache_build_incremental or by
+ * an earlier advance; LACACHE_ERR_STATE otherwise, or when it is the last block) to the next one.
+ * q_fin [B*L_b,Hq,d], k_fin / v_fin [B*L_b,Hkv,d] of `dtype` are the pre-RoPE rows of the FINISHED
+ * block (layout of lacache_step's inputs); all other tokens must be unchanged since the build.
+ * Afterwards lacache_step serves the next block.  tcgen05 engine only (LACACHE_ERR_UNSUPPORTED
+ * otherwise).  Device pointers, 16-byte aligned, borrowed for the duration of the enqueued work.
+ */
+lacache_status lacache_build_incremental(lacache_ctx* ctx, int block_idx, const void* q_pre,
+                                         const void* k_pre, const void* v_pre, void* cuda_stream);
+lacache_status lacache_build_advance(lacache_ctx* ctx, const void* q_fin, const void* k_fin,
+                                     const void* v_fin, void* cuda_stream);
+
+/*
  * Algorithm 1 with GenStep = False (Sec. 3.3.3, last paragraph).  Rotates the
  * block's fresh q_blk [B*L_b,Hq,d], k_blk / v_blk [B*L_b,Hkv,d] into the
  * block's cache slots; fixed queries start from the cached state, visit only

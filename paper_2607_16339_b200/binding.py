@@ -25,7 +25,7 @@ EXPORTS = [
     "lacache_qkv_create", "lacache_qkv_destroy", "lacache_qkv_project", "lacache_build_tokens",
     "lacache_step_tokens", "lacache_qkv_set_timing_events", "lacache_qkv_last_launch_count",
     "lacache_qkv_poll_status", "lacache_qkv_last_error", "lacache_set_step_overlap",
-    "lacache_build_tokens_update",
+    "lacache_build_tokens_update", "lacache_build_incremental", "lacache_build_advance",
 ]
 
 
@@ -73,6 +73,8 @@ def load():
     lib.lacache_destroy.argtypes = [vp]
     lib.lacache_build.argtypes = [vp, ip, vp, vp, vp, vp]
     lib.lacache_step.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.lacache_build_incremental.argtypes = [vp, ip, vp, vp, vp, vp]
+    lib.lacache_build_advance.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_full_recompute.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.lacache_build_host.argtypes = [vp, ip, vp, vp, vp, vp]
     lib.lacache_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -184,6 +186,14 @@ class Context:
     def build(self, block_idx, q_pre, k_pre, v_pre, stream=None):
         self._check(self._lib.lacache_build(self._h, int(block_idx), _ptr(q_pre), _ptr(k_pre),
                                             _ptr(v_pre), _stream(stream)))
+
+    def build_incremental(self, block_idx, q_pre, k_pre, v_pre, stream=None):
+        self._check(self._lib.lacache_build_incremental(self._h, int(block_idx), _ptr(q_pre), _ptr(k_pre),
+                                                        _ptr(v_pre), _stream(stream)))
+
+    def build_advance(self, q_fin, k_fin, v_fin, stream=None):
+        self._check(self._lib.lacache_build_advance(self._h, _ptr(q_fin), _ptr(k_fin), _ptr(v_fin),
+                                                    _stream(stream)))
 
     def step(self, q_blk, k_blk, v_blk, out, lse=None, stream=None):
         self._check(self._lib.lacache_step(self._h, _ptr(q_blk), _ptr(k_blk), _ptr(v_blk), _ptr(out),

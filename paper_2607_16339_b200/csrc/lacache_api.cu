@@ -25,6 +25,11 @@ struct lacache_ctx {
   struct ListRef { int off, n; };
   std::vector<ListRef> build_list, step_list;  // per block (step_list: SIMT all items; tcgen05 block-chunk items)
   std::vector<ListRef> merge_list;             // per block: fixed-row items of a step (tcgen05)
+  // per block, tcgen05: row tiles x key windows of the incremental build (prefix state from scratch;
+  // cached state = prefix state + the keys after the block; prefix state advanced by one block)
+  std::vector<ListRef> inc_prefix, inc_comb, inc_adv;
+  StateBuffers pst{};      // prefix state of every token: its keys before the current block (allocated on first use)
+  int prefix_block = -1;   // block pst is valid for
   int num_sms = 148;
   int stream_ctas_override = 0;
   ListRef full_list;
@@ -292,6 +297,51 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
       c->merge_list.push_back({0, 0});
     }
     c->build_list.push_back({rows_off, (int)items.size() - rows_off});
+  }
+  for (int k = 0; k < g.n_blk && tc; ++k) {
+    // Incremental build.  With s the block's first token and e one past its last, of a sequence
+    // [cs, ce): the prefix state holds keys [cs, s); the cached state adds keys [e, ce); advancing
+    // from block k - 1 adds that block's keys [s - L_b, s) to the rows outside it and computes the
+    // rows inside it (whose queries changed) over [cs, s) from scratch.
+    auto window = [&](int from, int k0, int k1, bool init) {
+      for (size_t i = from; i < items.size(); ++i) {
+        items[i].kind = ITEM_ROWS_WINDOW;
+        items[i].kt0 = k0;
+        items[i].kt1 = k1;
+        items[i].chunk = init ? 1 : 0;
+      }
+    };
+    int off = (int)items.size();
+    for (int b = 0; b < g.B; ++b) {
+      const int cs = c->cu[b], ce = c->cu[b + 1], s0 = c->blk_start_all[(size_t)k * g.B + b], e0 = s0 + g.block_len;
+      const int from = (int)items.size();
+      add_row_tiles(items, b, cs, s0, R, cs, ce, s0);
+      add_row_tiles(items, b, e0, ce, R, cs, ce, s0);
+      window(from, cs, s0, false);
+    }
+    c->inc_prefix.push_back({off, (int)items.size() - off});
+    off = (int)items.size();
+    for (int b = 0; b < g.B; ++b) {
+      const int cs = c->cu[b], ce = c->cu[b + 1], s0 = c->blk_start_all[(size_t)k * g.B + b], e0 = s0 + g.block_len;
+      const int from = (int)items.size();
+      add_row_tiles(items, b, cs, s0, R, cs, ce, s0);
+      add_row_tiles(items, b, e0, ce, R, cs, ce, s0);
+      window(from, e0, ce, true);
+    }
+    c->inc_comb.push_back({off, (int)items.size() - off});
+    off = (int)items.size();
+    for (int b = 0; b < g.B && k > 0; ++b) {
+      const int cs = c->cu[b], ce = c->cu[b + 1], s0 = c->blk_start_all[(size_t)k * g.B + b], e0 = s0 + g.block_len;
+      const int sp = s0 - g.block_len;   // the finished block (blocks are consecutive)
+      int from = (int)items.size();
+      add_row_tiles(items, b, cs, sp, R, cs, ce, s0);
+      add_row_tiles(items, b, e0, ce, R, cs, ce, s0);
+      window(from, sp, s0, true);
+      from = (int)items.size();
+      add_row_tiles(items, b, sp, s0, R, cs, ce, s0);
+      window(from, cs, s0, false);
+    }
+    c->inc_adv.push_back({off, (int)items.size() - off});
   }
   {
     int off = (int)items.size();
@@ -612,12 +662,103 @@ lacache_status lacache_build(lacache_ctx* c, int block_idx, const void* q, const
   cudaStream_t s = (cudaStream_t)stream;
   c->last_launches = 0;
   c->built_block = -1;
+  c->prefix_block = -1;
   lacache_status st = rope_all(c, q, k, v, c->rot, s);
   if (st != LACACHE_OK) return st;
   AttnArgs a = attn_args(c, MODE_BUILD, c->build_list[block_idx], block_idx, c->rot, nullptr, nullptr);
   st = run_attention(c, a, false, s);
   if (st != LACACHE_OK) return st;
   c->built_block = block_idx;
+  c->steps_since_build = 0;
+  return LACACHE_OK;
+}
+
+namespace {
+// the prefix state's buffers, allocated when the incremental build is first used
+lacache_status ensure_prefix_state(lacache_ctx* c) {
+  if (c->engine != LACACHE_ENGINE_TCGEN05)
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "the incremental build needs the tcgen05 engine");
+  if (c->pst.o) return LACACHE_OK;
+  const Geometry& g = c->g;
+  CU_TRY(c, dev_alloc(c, &c->pst.m, (size_t)g.Hq * g.Tp, true));
+  CU_TRY(c, dev_alloc(c, &c->pst.l, (size_t)g.Hq * g.Tp, true));
+  CU_TRY(c, dev_alloc(c, &c->pst.o, (size_t)g.Hq * g.Tp * g.d, true));
+  return LACACHE_OK;
+}
+// one launch over a list of key-window items: dst = (init +) the window's keys
+lacache_status run_window(lacache_ctx* c, lacache_ctx::ListRef list, int blk, const StateBuffers& init,
+                          const StateBuffers& dst, cudaStream_t s) {
+  if (list.n == 0) return LACACHE_OK;
+  AttnArgs a = attn_args(c, MODE_BUILD, list, blk, c->rot, nullptr, nullptr);
+  a.init = init;
+  a.st = dst;
+  return run_attention(c, a, false, s);
+}
+}  // namespace
+
+lacache_status lacache_build_incremental(lacache_ctx* c, int block_idx, const void* q, const void* k, const void* v,
+                                         void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if (!q || !k || !v) return fail(c, LACACHE_ERR_INVALID_ARG, "NULL input pointer");
+  if (misaligned(q) || misaligned(k) || misaligned(v)) return fail(c, LACACHE_ERR_INVALID_ARG, "input pointer not 16-byte aligned");
+  if (block_idx < 0 || block_idx >= c->g.n_blk)
+    return fail(c, LACACHE_ERR_INVALID_ARG, "block_idx %d outside [0, %d)", block_idx, c->g.n_blk);
+  lacache_status st = ensure_prefix_state(c);
+  if (st != LACACHE_OK) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  c->last_launches = 0;
+  c->built_block = -1;
+  c->prefix_block = -1;
+  st = rope_all(c, q, k, v, c->rot, s);
+  if (st != LACACHE_OK) return st;
+  st = run_window(c, c->inc_prefix[block_idx], block_idx, StateBuffers{}, c->pst, s);
+  if (st != LACACHE_OK) return st;
+  st = run_window(c, c->inc_comb[block_idx], block_idx, c->pst, c->st, s);
+  if (st != LACACHE_OK) return st;
+  c->built_block = block_idx;
+  c->prefix_block = block_idx;
+  c->steps_since_build = 0;
+  return LACACHE_OK;
+}
+
+lacache_status lacache_build_advance(lacache_ctx* c, const void* q, const void* k, const void* v, void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if (c->built_block < 0 || c->prefix_block != c->built_block)
+    return fail(c, LACACHE_ERR_STATE, "lacache_build_advance needs the state of lacache_build_incremental or of an earlier advance");
+  if (c->built_block + 1 >= c->g.n_blk)
+    return fail(c, LACACHE_ERR_STATE, "block %d is the last one", c->built_block);
+  if (!q || !k || !v) return fail(c, LACACHE_ERR_INVALID_ARG, "NULL input pointer");
+  if (misaligned(q) || misaligned(k) || misaligned(v)) return fail(c, LACACHE_ERR_INVALID_ARG, "input pointer not 16-byte aligned");
+  cudaStream_t s = (cudaStream_t)stream;
+  const int done = c->built_block, blk = done + 1;
+  c->last_launches = 0;
+  c->built_block = -1;
+  c->prefix_block = -1;
+  // the finished block's rows, rotated into the cache (an ordinary launch: everything ahead in the
+  // stream, a step that still reads the cached state included, completes first)
+  RopeArgs r{};
+  r.q = q; r.k = k; r.v = v;
+  r.n_src_rows = c->g.B * c->g.block_len;
+  r.blk_start = c->d_blk_start_all + (size_t)done * c->g.B;
+  r.block_len = c->g.block_len;
+  r.pos_of_tok = c->d_pos; r.cos_tab = c->d_cos; r.sin_tab = c->d_sin;
+  {
+    const size_t row0 = (size_t)done * c->g.B * c->g.block_len;
+    r.row_tok = c->d_blk_tok + row0;
+    r.row_cos = c->d_blk_cos + row0 * (c->g.d / 2);
+    r.row_sin = c->d_blk_sin + row0 * (c->g.d / 2);
+  }
+  r.pdl = 0;
+  r.dst = c->rot;
+  r.in_dtype = c->cfg.dtype;
+  CU_TRY(c, rope_write(c->g, r, c->engine, s));
+  c->last_launches++;
+  lacache_status st = run_window(c, c->inc_adv[blk], blk, c->pst, c->pst, s);
+  if (st != LACACHE_OK) return st;
+  st = run_window(c, c->inc_comb[blk], blk, c->pst, c->st, s);
+  if (st != LACACHE_OK) return st;
+  c->built_block = blk;
+  c->prefix_block = blk;
   c->steps_since_build = 0;
   return LACACHE_OK;
 }

@@ -12,6 +12,8 @@ namespace lacache {
 enum ItemKind : int32_t {
   ITEM_ROWS = 0,   // a tile of query rows [row0, row0 + nrows) of one sequence
   ITEM_BLOCK_CHUNK = 1,  // the block's query rows x one chunk of key tiles
+  ITEM_ROWS_WINDOW = 2,  // (build) a tile of query rows x the keys [kt0, kt1) of its sequence, given as token
+                         // indices; chunk bit 0: continue from the rows' state in AttnArgs::init
 };
 struct WorkItem {
   int32_t kind;   // ItemKind
@@ -112,6 +114,7 @@ struct AttnArgs {
   const int32_t* blk_start;  // [B] absolute token index of the block's first row
   RotBuffers rot;
   StateBuffers st;
+  StateBuffers init;         // build over key windows: the state units with the init bit start from (may alias st)
   float* out; float* lse;    // token-major [T,Hq,d], [T,Hq]
   // split-key partial states of block queries and their arrival counters
   float* part_m; float* part_l; float* part_o; int* counters; int max_chunks;

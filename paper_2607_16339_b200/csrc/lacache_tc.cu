@@ -231,6 +231,7 @@ struct Unit {
   int epi, chunk, nchunks;
   int q_rows;             // rows of the Q box: 128 or 64
   int nh, rh;             // packed block queries: nh heads h, h + 1, ... of one KV group, rh lanes each (rh = 0: one head)
+  int init;               // build over a key window: the unit starts from the rows' state in a.init instead of an empty one
 };
 // head and row within the head's rows of tile row r; whether r holds a real query row (rh is 0, 32 or 64)
 __device__ __forceinline__ int unit_head(const Unit& un, int r) { return un.rh ? un.h + (r >> (un.rh == 64 ? 6 : 5)) : un.h; }
@@ -273,7 +274,15 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
   un.chunk = 0;
   un.nchunks = 1;
   un.q_rows = BM;
-  if (!STEP && a.mode == MODE_BUILD) {
+  un.init = 0;
+  if (!STEP && it.kind == ITEM_ROWS_WINDOW) {
+    // keys [kt0, kt1) of the sequence (token indices), tiles counted from the window's first key
+    un.key_base = un.k0 = it.kt0;
+    un.k1 = it.kt1;
+    un.t1 = it.kt1 > it.kt0 ? (it.kt1 - it.kt0 + BN - 1) / BN : 0;
+    un.epi = EPI_STATE;
+    un.init = it.chunk & 1;
+  } else if (!STEP && a.mode == MODE_BUILD) {
     un.x0 = it.blk_start;
     un.x1 = it.blk_start + g.block_len;
     un.epi = EPI_STATE;
@@ -529,7 +538,7 @@ __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a
       if (!wait_bar(c, sv ? BAR_V_FULL1 : BAR_V_FULL, ph, LOC_WAIT_V)) return;
       tc_fence_after();
       issue_pv_mma(c.base + SM_V + sv * V_STAGE, KS_BOX, c.tmem + TS_P + 64 * b, c.tmem + TS_O, BN / 16,
-                   j == 0 ? 0u : 1u);
+                   (j == 0 && !(!STEP && un.init)) ? 0u : 1u);
       tc_commit(c.bar(BAR_O_FULL));
       tc_commit(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE));
     }
@@ -722,6 +731,33 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     const bool active = unit_row_valid(un, quad * 32);  // this warp holds at least one real row (its first)
     float m_ref = -INFINITY, l_part = 0.f;
     bool first_tile = true;
+    bool have_o = false;   // O~ in TMEM holds something before the unit's first P~V
+    if (!STEP && un.init) {
+      // The unit continues from a stored state (m, l, O~) of its rows: the reference exponent and the
+      // normaliser go to registers (the normaliser to the first thread of the pair), O~ to the
+      // accumulator columns this thread owns.  Nobody else reads or writes those cells between units
+      // (the previous unit's P~V products are complete, and its epilogue read them from this thread).
+      // The TMEM stores are warp-wide: rows past the end of a clipped tile store zeros.
+      const size_t srow = (size_t)un.h * g.Tp + row;
+      if (row_valid) {
+        m_ref = a.init.m[srow];
+        if (half == 0) l_part = a.init.l[srow];
+      }
+      const float4* src = reinterpret_cast<const float4*>(a.init.o + srow * D + 64 * half);
+#pragma unroll 1
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t rr[16];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 x = row_valid ? src[4 * cb + i] : make_float4(0.f, 0.f, 0.f, 0.f);   // (plain loads: the launch may update these rows in place)
+          rr[4 * i] = __float_as_uint(x.x); rr[4 * i + 1] = __float_as_uint(x.y);
+          rr[4 * i + 2] = __float_as_uint(x.z); rr[4 * i + 3] = __float_as_uint(x.w);
+        }
+        tmem_st16(tlane + TS_O + 64 * half + 16 * cb, rr, 0);
+      }
+      tmem_st_wait();
+      have_o = true;
+    }
 
     for (int t = un.t0; t < un.t1; ++t, ++jj) {
       const int b = jj & 1;
@@ -785,11 +821,13 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
         float alpha = 1.f;
         if (m_new != m_ref) alpha = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
-        if (!first_tile && __any_sync(0xffffffffu, alpha != 1.f)) {
+        if ((!first_tile || (!STEP && have_o)) && __any_sync(0xffffffffu, alpha != 1.f)) {
           // O~ in TMEM is rescaled in place: P~V of the previous tile must be done
-          if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
-          o_waited = true;
-          tc_fence_after();
+          if (!first_tile) {
+            if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
+            o_waited = true;
+            tc_fence_after();
+          }
 #pragma unroll 1
           for (int cb = 0; cb < 4; ++cb) {
             uint32_t rr[16];
@@ -931,7 +969,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       // (the TMEM loads are warp-wide: rows past the end of a clipped tile take part in them and
       // only skip the stores; first_tile is uniform over the CTA)
       uint32_t rr[64];
-      if (!first_tile) {
+      if (!first_tile || (!STEP && have_o)) {
         tmem_ld32(tlane + TS_O + 64 * half, *reinterpret_cast<uint32_t(*)[32]>(rr));
         tmem_ld32(tlane + TS_O + 64 * half + 32, *reinterpret_cast<uint32_t(*)[32]>(rr + 32));
         tmem_ld_wait();
