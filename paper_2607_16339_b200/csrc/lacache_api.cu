@@ -26,8 +26,9 @@ struct lacache_ctx {
   std::vector<ListRef> build_list, step_list;  // per block (step_list: SIMT all items; tcgen05 block-chunk items)
   std::vector<ListRef> merge_list;             // per block: fixed-row items of a step (tcgen05)
   // per block, tcgen05: row tiles x key windows of the incremental build (prefix state from scratch;
-  // cached state = prefix state + the keys after the block; prefix state advanced by one block)
-  std::vector<ListRef> inc_prefix, inc_comb, inc_adv;
+  // cached state = prefix state + the keys after the block; the finished block's rows from scratch;
+  // every other row advanced by the finished block's keys and completed by the keys after the block)
+  std::vector<ListRef> inc_prefix, inc_comb, inc_fresh, inc_fused;
   StateBuffers pst{};      // prefix state of every token: its keys before the current block (allocated on first use)
   int prefix_block = -1;   // block pst is valid for
   int num_sms = 148;
@@ -303,21 +304,23 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     // [cs, ce): the prefix state holds keys [cs, s); the cached state adds keys [e, ce); advancing
     // from block k - 1 adds that block's keys [s - L_b, s) to the rows outside it and computes the
     // rows inside it (whose queries changed) over [cs, s) from scratch.
-    auto window = [&](int from, int k0, int k1, bool init) {
+    auto window = [&](int from, int base, int k0, int k1, int flags) {
       for (size_t i = from; i < items.size(); ++i) {
         items[i].kind = ITEM_ROWS_WINDOW;
+        items[i].pad = base;
         items[i].kt0 = k0;
         items[i].kt1 = k1;
-        items[i].chunk = init ? 1 : 0;
+        items[i].chunk = flags;
       }
     };
+    enum { W_INIT = 1, W_SNAP = 2, W_SKIP_BLOCK = 4 };
     int off = (int)items.size();
     for (int b = 0; b < g.B; ++b) {
       const int cs = c->cu[b], ce = c->cu[b + 1], s0 = c->blk_start_all[(size_t)k * g.B + b], e0 = s0 + g.block_len;
       const int from = (int)items.size();
       add_row_tiles(items, b, cs, s0, R, cs, ce, s0);
       add_row_tiles(items, b, e0, ce, R, cs, ce, s0);
-      window(from, cs, s0, false);
+      window(from, cs, cs, s0, 0);
     }
     c->inc_prefix.push_back({off, (int)items.size() - off});
     off = (int)items.size();
@@ -326,22 +329,35 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
       const int from = (int)items.size();
       add_row_tiles(items, b, cs, s0, R, cs, ce, s0);
       add_row_tiles(items, b, e0, ce, R, cs, ce, s0);
-      window(from, e0, ce, true);
+      window(from, e0, e0, ce, W_INIT);
     }
     c->inc_comb.push_back({off, (int)items.size() - off});
+    // advancing from block k - 1 (rows [sp, s0), blocks are consecutive), in two launches:
+    off = (int)items.size();
+    for (int b = 0; b < g.B && k > 0; ++b) {
+      // its rows changed their queries: prefix state over every key before block k, from scratch
+      const int cs = c->cu[b], ce = c->cu[b + 1], s0 = c->blk_start_all[(size_t)k * g.B + b];
+      const int from = (int)items.size();
+      add_row_tiles(items, b, s0 - g.block_len, s0, R, cs, ce, s0);
+      window(from, cs, cs, s0, 0);
+    }
+    c->inc_fresh.push_back({off, (int)items.size() - off});
     off = (int)items.size();
     for (int b = 0; b < g.B && k > 0; ++b) {
       const int cs = c->cu[b], ce = c->cu[b + 1], s0 = c->blk_start_all[(size_t)k * g.B + b], e0 = s0 + g.block_len;
-      const int sp = s0 - g.block_len;   // the finished block (blocks are consecutive)
+      const int sp = s0 - g.block_len;
+      // every other fixed row: old prefix state + the finished block's keys (exactly the first key
+      // tile, which ends at s0) = new prefix state, stored; + the keys after block k = cached state
       int from = (int)items.size();
       add_row_tiles(items, b, cs, sp, R, cs, ce, s0);
       add_row_tiles(items, b, e0, ce, R, cs, ce, s0);
-      window(from, sp, s0, true);
+      window(from, s0 - TC_KEYS, sp, ce > e0 ? ce : s0, W_INIT | W_SNAP | W_SKIP_BLOCK);
+      // the finished block's rows: their new prefix state + the keys after block k
       from = (int)items.size();
       add_row_tiles(items, b, sp, s0, R, cs, ce, s0);
-      window(from, cs, s0, false);
+      window(from, e0, e0, ce, W_INIT);
     }
-    c->inc_adv.push_back({off, (int)items.size() - off});
+    c->inc_fused.push_back({off, (int)items.size() - off});
   }
   {
     int off = (int)items.size();
@@ -687,11 +703,12 @@ lacache_status ensure_prefix_state(lacache_ctx* c) {
 }
 // one launch over a list of key-window items: dst = (init +) the window's keys
 lacache_status run_window(lacache_ctx* c, lacache_ctx::ListRef list, int blk, const StateBuffers& init,
-                          const StateBuffers& dst, cudaStream_t s) {
+                          const StateBuffers& dst, const StateBuffers& snap, cudaStream_t s) {
   if (list.n == 0) return LACACHE_OK;
   AttnArgs a = attn_args(c, MODE_BUILD, list, blk, c->rot, nullptr, nullptr);
   a.init = init;
   a.st = dst;
+  a.snap = snap;
   return run_attention(c, a, false, s);
 }
 }  // namespace
@@ -711,9 +728,9 @@ lacache_status lacache_build_incremental(lacache_ctx* c, int block_idx, const vo
   c->prefix_block = -1;
   st = rope_all(c, q, k, v, c->rot, s);
   if (st != LACACHE_OK) return st;
-  st = run_window(c, c->inc_prefix[block_idx], block_idx, StateBuffers{}, c->pst, s);
+  st = run_window(c, c->inc_prefix[block_idx], block_idx, StateBuffers{}, c->pst, StateBuffers{}, s);
   if (st != LACACHE_OK) return st;
-  st = run_window(c, c->inc_comb[block_idx], block_idx, c->pst, c->st, s);
+  st = run_window(c, c->inc_comb[block_idx], block_idx, c->pst, c->st, StateBuffers{}, s);
   if (st != LACACHE_OK) return st;
   c->built_block = block_idx;
   c->prefix_block = block_idx;
@@ -753,9 +770,9 @@ lacache_status lacache_build_advance(lacache_ctx* c, const void* q, const void* 
   r.in_dtype = c->cfg.dtype;
   CU_TRY(c, rope_write(c->g, r, c->engine, s));
   c->last_launches++;
-  lacache_status st = run_window(c, c->inc_adv[blk], blk, c->pst, c->pst, s);
+  lacache_status st = run_window(c, c->inc_fresh[blk], blk, StateBuffers{}, c->pst, StateBuffers{}, s);
   if (st != LACACHE_OK) return st;
-  st = run_window(c, c->inc_comb[blk], blk, c->pst, c->st, s);
+  st = run_window(c, c->inc_fused[blk], blk, c->pst, c->st, c->pst, s);
   if (st != LACACHE_OK) return st;
   c->built_block = blk;
   c->prefix_block = blk;

@@ -13,7 +13,10 @@ enum ItemKind : int32_t {
   ITEM_ROWS = 0,   // a tile of query rows [row0, row0 + nrows) of one sequence
   ITEM_BLOCK_CHUNK = 1,  // the block's query rows x one chunk of key tiles
   ITEM_ROWS_WINDOW = 2,  // (build) a tile of query rows x the keys [kt0, kt1) of its sequence, given as token
-                         // indices; chunk bit 0: continue from the rows' state in AttnArgs::init
+                         // indices; key tiles are counted from token `pad` (<= kt0, may be negative).
+                         // chunk bit 0: continue from the rows' state in AttnArgs::init; bit 1: store the
+                         // state after the first key tile to AttnArgs::snap; bit 2: leave out the keys of
+                         // the block at blk_start
 };
 struct WorkItem {
   int32_t kind;   // ItemKind
@@ -115,6 +118,8 @@ struct AttnArgs {
   RotBuffers rot;
   StateBuffers st;
   StateBuffers init;         // build over key windows: the state units with the init bit start from (may alias st)
+  StateBuffers snap;         // ... and where units with the snapshot bit store their state after the first key tile
+                             // (may alias init: a unit loads its rows before it stores them)
   float* out; float* lse;    // token-major [T,Hq,d], [T,Hq]
   // split-key partial states of block queries and their arrival counters
   float* part_m; float* part_l; float* part_o; int* counters; int max_chunks;

@@ -232,6 +232,7 @@ struct Unit {
   int q_rows;             // rows of the Q box: 128 or 64
   int nh, rh;             // packed block queries: nh heads h, h + 1, ... of one KV group, rh lanes each (rh = 0: one head)
   int init;               // build over a key window: the unit starts from the rows' state in a.init instead of an empty one
+  int snap;               // ... and stores the state it has after its first key tile to a.snap
 };
 // head and row within the head's rows of tile row r; whether r holds a real query row (rh is 0, 32 or 64)
 __device__ __forceinline__ int unit_head(const Unit& un, int r) { return un.rh ? un.h + (r >> (un.rh == 64 ? 6 : 5)) : un.h; }
@@ -274,14 +275,22 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
   un.chunk = 0;
   un.nchunks = 1;
   un.q_rows = BM;
-  un.init = 0;
+  un.init = un.snap = 0;
   if (!STEP && it.kind == ITEM_ROWS_WINDOW) {
-    // keys [kt0, kt1) of the sequence (token indices), tiles counted from the window's first key
-    un.key_base = un.k0 = it.kt0;
+    // keys [kt0, kt1) of the sequence (token indices), optionally without the block's; tiles are
+    // counted from token `pad`, which may lie before the window (and before token 0: those key rows
+    // load as zeros and are masked like every key outside the window)
+    un.key_base = it.pad;
+    un.k0 = it.kt0;
     un.k1 = it.kt1;
-    un.t1 = it.kt1 > it.kt0 ? (it.kt1 - it.kt0 + BN - 1) / BN : 0;
+    un.t1 = it.kt1 > it.pad ? (it.kt1 - it.pad + BN - 1) / BN : 0;
+    if (it.chunk & 4) {
+      un.x0 = it.blk_start;
+      un.x1 = it.blk_start + g.block_len;
+    }
     un.epi = EPI_STATE;
     un.init = it.chunk & 1;
+    un.snap = (it.chunk >> 1) & 1;
   } else if (!STEP && a.mode == MODE_BUILD) {
     un.x0 = it.blk_start;
     un.x1 = it.blk_start + g.block_len;
@@ -430,6 +439,9 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         cq.q_done = true;
         cq.t = cq.un.t1;
         cursor_advance<PACKED, STEP>(g, a, cq, stride, n_units);
+        // a build's Q tiles come from HBM once the batch outgrows L2: the next unit's tile is asked
+        // into L2 a whole unit ahead of its load
+        if (!STEP && cq.valid) tma_prefetch_5d(&maps.q, 0, cq.un.row0, 0, cq.un.h, 0);
         did = true;
       }
     }
@@ -757,6 +769,13 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       }
       tmem_st_wait();
       have_o = true;
+      if (u + stride < n_units && it.kind == ITEM_ROWS_WINDOW && (it.chunk & 1) && r < it.nrows) {
+        // the next unit's rows of that state, asked into L2 now (`it` already holds its item)
+        const char* nx = reinterpret_cast<const char*>(
+            a.init.o + ((size_t)((u + stride) % g.Hq) * g.Tp + it.row0 + r) * D + 64 * half);
+        prefetch_l2(nx);
+        prefetch_l2(nx + 128);
+      }
     }
 
     for (int t = un.t0; t < un.t1; ++t, ++jj) {
@@ -768,13 +787,48 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       // previous tile, either before an in-place rescale or at the end of the tile
       bool o_waited = first_tile;
       if (active) {
+        if (!STEP && un.snap && t == un.t0 + 1) {
+          // The state after the unit's first key tile goes to a.snap before this tile changes it:
+          // P~V of that tile must be complete; the pair adds up its normaliser halves.
+          if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
+          o_waited = true;
+          tc_fence_after();
+          volatile float* lxs = xch + 2 * (xslot & 1u);
+          ++xslot;
+          lxs[half] = l_part;
+          mbar_arrive(c.bar(BAR_PAIR + quad));
+          if (!wait_bar(c, BAR_PAIR + quad, pair_phase & 1, LOC_WAIT_S)) return;
+          ++pair_phase;
+          const float l_sum = lxs[0] + lxs[1];
+          const size_t srow = (size_t)un.h * g.Tp + row;
+          float4* dst = reinterpret_cast<float4*>(a.snap.o + srow * D + 64 * half);
+          uint32_t rr[64];   // (warp-wide loads; rows past the end of a clipped tile only skip the stores)
+          tmem_ld32(tlane + TS_O + 64 * half, *reinterpret_cast<uint32_t(*)[32]>(rr));
+          tmem_ld32(tlane + TS_O + 64 * half + 32, *reinterpret_cast<uint32_t(*)[32]>(rr + 32));
+          tmem_ld_wait();
+          if (row_valid) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) st_global_v8(dst + 2 * i, rr + 8 * i);
+            if (half == 0) { a.snap.m[srow] = m_ref; a.snap.l[srow] = l_sum; }
+          }
+        }
         const int tile_lo = un.key_base + t * BN;
         const int v_lo = max(un.k0 - tile_lo, 0), v_hi = min(un.k1 - tile_lo, BN);
         const int e_lo = un.x0 - tile_lo, e_hi = un.x1 - tile_lo;
         const bool all_valid = v_lo == 0 && v_hi == BN && (un.x1 <= un.x0 || e_hi <= 0 || e_lo >= BN);
-        auto col_valid = [&](int j) { return j >= v_lo && j < v_hi && !(j >= e_lo && j < e_hi); };
-        const uint32_t s_addr = tlane + TS_S + 128 * b;
+        // the masks of a tile are the same for every row: one bit per column of this thread's half
+        // (bit j: column mc + j takes part), built once per tile
         const int mc = HC * half;   // this thread's columns
+        auto span_bits = [](int lo, int hi) -> uint64_t {   // bits [lo, hi) of 64
+          lo = max(lo, 0);
+          hi = min(hi, 64);
+          if (hi <= lo) return 0ull;
+          return (hi - lo == 64 ? ~0ull : ((1ull << (hi - lo)) - 1ull)) << lo;
+        };
+        const uint64_t col_bits = all_valid ? ~0ull
+                                            : (span_bits(v_lo - mc, v_hi - mc) &
+                                               ~((un.x1 > un.x0) ? span_bits(e_lo - mc, e_hi - mc) : 0ull));
+        const uint32_t s_addr = tlane + TS_S + 128 * b;
         // Pass 1: maximum over this thread's columns.  Instruction count on
         // these threads is what limits the kernel, so a tile with no masked
         // column (the common case) takes a path with no per-column tests, and
@@ -796,9 +850,14 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
                 m3 = fmaxf(m3, __uint_as_float(rr[j + 3]));
               }
             } else {
+              const uint32_t bits = (uint32_t)(col_bits >> (16 * cb)) & 0xffffu;
 #pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (col_valid(mc + 16 * cb + j)) m0 = fmaxf(m0, __uint_as_float(rr[j]));
+              for (int j = 0; j < 16; j += 4) {
+                m0 = fmaxf(m0, ((bits >> j) & 1u) ? __uint_as_float(rr[j]) : -INFINITY);
+                m1 = fmaxf(m1, ((bits >> (j + 1)) & 1u) ? __uint_as_float(rr[j + 1]) : -INFINITY);
+                m2 = fmaxf(m2, ((bits >> (j + 2)) & 1u) ? __uint_as_float(rr[j + 2]) : -INFINITY);
+                m3 = fmaxf(m3, ((bits >> (j + 3)) & 1u) ? __uint_as_float(rr[j + 3]) : -INFINITY);
+              }
             }
           }
           mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
@@ -823,7 +882,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         if (m_new != m_ref) alpha = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
         if ((!first_tile || (!STEP && have_o)) && __any_sync(0xffffffffu, alpha != 1.f)) {
           // O~ in TMEM is rescaled in place: P~V of the previous tile must be done
-          if (!first_tile) {
+          if (!o_waited) {
             if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
             o_waited = true;
             tc_fence_after();
@@ -856,11 +915,13 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
               pk[j] = *reinterpret_cast<uint32_t*>(&hp);
             }
           } else {
+            const uint32_t bits = (uint32_t)(col_bits >> (16 * cb)) & 0xffffu;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-              const int cidx = mc + 16 * cb + 2 * j;
-              float p0 = col_valid(cidx) ? round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j]), g.scale_log2, -m_use))) : 0.f;
-              float p1 = col_valid(cidx + 1) ? round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j + 1]), g.scale_log2, -m_use))) : 0.f;
+              float p0 = round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j]), g.scale_log2, -m_use)));
+              float p1 = round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j + 1]), g.scale_log2, -m_use)));
+              p0 = ((bits >> (2 * j)) & 1u) ? p0 : 0.f;
+              p1 = ((bits >> (2 * j + 1)) & 1u) ? p1 : 0.f;
               ps0 += p0;
               ps1 += p1;
               __half2 hp = __floats2half2_rn(p0, p1);
@@ -982,6 +1043,15 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         for (int i = 0; i < 8; ++i) st_global_v8(dst + 2 * i, rr + 8 * i);
       }
       if (row_valid && half == 0) { a.st.m[srow] = m_ref; a.st.l[srow] = l_run; }
+      if (!STEP && un.snap && un.t1 - un.t0 <= 1) {
+        // a single key tile: the state after it is the final one as well
+        float4* sdst = reinterpret_cast<float4*>(a.snap.o + srow * D + 64 * half);
+        if (row_valid) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) st_global_v8(sdst + 2 * i, rr + 8 * i);
+          if (half == 0) { a.snap.m[srow] = m_ref; a.snap.l[srow] = l_run; }
+        }
+      }
       tc_fence_before();
       mbar_arrive(c.bar(BAR_O_FREE));  // the next unit may overwrite O~
       continue;
