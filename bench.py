@@ -424,10 +424,68 @@ def run_cuda(args):
         if (world == 1 and not args.no_token_path and wl.dtype == "bf16" and wl.n_q_heads in D_MODEL
                 and wl.total_tokens <= 65536):     # (its replicas of the all-token scratch would not fit beyond that)
             line["token_path"] = token_path_leg(wl, dev, peaks, args.seed, min(K, 512))
+        if world == 1 and not args.no_incremental and wl.dtype == "bf16" and wl.head_dim == 128 and wl.n_blocks >= 2:
+            line["incremental"] = incremental_leg(wl, dev, args.seed, R)
         print(json.dumps(line), flush=True)
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------
+# one whole generation, the cache rebuilt for every block or advanced from block to block
+# ----------------------------------------------------------------------------
+def incremental_leg(wl, dev, seed, R):
+    """Steps per second over one generation (every block, every step of it) of R independent cache
+    states visited round-robin, twice: with lacache_build at the start of every block, and with
+    lacache_build_incremental at block 0 and lacache_build_advance between blocks.  Also the mean
+    device time of one rebuild and of one advance (events around the calls)."""
+    import torch
+    from paper_2607_16339_b200 import binding
+    from paper_2607_16339_b200.workloads import DeviceSchedule
+    mk = lambda: torch.cuda.Event(enable_timing=True)
+    S, nb, T = wl.steps_per_block, wl.n_blocks, wl.total_tokens
+    sched = DeviceSchedule(wl, seed + 17, dev, nb * S)
+    ctxs = [binding.Context.from_workload(wl) for _ in range(R)]
+    outs = [(torch.empty(T, wl.n_q_heads, wl.head_dim, device=dev), torch.empty(T, wl.n_q_heads, device=dev))
+            for _ in range(R)]
+    res = {}
+    for mode in ("rebuild", "advance", "rebuild", "advance"):     # (the first pass of each warms up)
+        pairs = []
+        e0, e1 = mk(), mk()
+        torch.cuda.synchronize()
+        e0.record()
+        for b in range(nb):
+            for c in range(R):
+                ev = (mk(), mk())
+                ev[0].record()
+                if mode == "rebuild":
+                    ctxs[c].build(b, *sched.full[b])
+                elif b == 0:
+                    ctxs[c].build_incremental(0, *sched.full[0])
+                else:
+                    ctxs[c].build_advance(*sched.steps[b * S - 1])
+                ev[1].record()
+                if b > 0:
+                    pairs.append(ev)
+            for s in range(S):
+                for c in range(R):
+                    ctxs[c].step(*sched.steps[b * S + s], *outs[c])
+        e1.record()
+        torch.cuda.synchronize()
+        for c in ctxs:
+            st, msg = c.poll_status()
+            if st != 0:
+                raise SystemExit("bench.py: device status %d in the incremental leg: %s" % (st, msg))
+        ms = e0.elapsed_time(e1)
+        res[mode] = (R * nb * S / (ms * 1e-3), sum(a.elapsed_time(b_) for a, b_ in pairs) / len(pairs) * 1e3)
+    for c in ctxs:
+        c.destroy()
+    return {"what": "one generation of %d blocks x %d steps on %d cache states round-robin: lacache_build per block "
+                    "against lacache_build_incremental + lacache_build_advance" % (nb, S, R),
+            "value": round(res["advance"][0], 1), "rebuild_value": round(res["rebuild"][0], 1), "unit": UNIT,
+            "advance_us": round(res["advance"][1], 1), "rebuild_us": round(res["rebuild"][1], 1),
+            "blocks": nb, "steps": R * nb * S, "replicas": R}
 
 
 # ----------------------------------------------------------------------------
@@ -625,6 +683,8 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-token-path", action="store_true", help="skip the extra leg that feeds steps from token ids")
+    ap.add_argument("--no-incremental", action="store_true",
+                    help="skip the extra leg that compares rebuilding the cache per block with advancing it")
     ap.add_argument("--replicas", type=int, default=0, help="cache-state replicas visited round-robin (0 = sized from the L2)")
     args = ap.parse_args()
     if args.warmup < 3:
