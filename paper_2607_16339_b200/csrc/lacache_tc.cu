@@ -756,16 +756,17 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         if (half == 0) l_part = a.init.l[srow];
       }
       const float4* src = reinterpret_cast<const float4*>(a.init.o + srow * D + 64 * half);
-#pragma unroll 1
-      for (int cb = 0; cb < 4; ++cb) {
-        uint32_t rr[16];
+      {
+        // all sixteen loads of the row half are in flight together (one round trip, not four)
+        uint32_t rr[64];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float4 x = row_valid ? src[4 * cb + i] : make_float4(0.f, 0.f, 0.f, 0.f);   // (plain loads: the launch may update these rows in place)
+        for (int i = 0; i < 16; ++i) {
+          const float4 x = row_valid ? src[i] : make_float4(0.f, 0.f, 0.f, 0.f);   // (plain loads: the launch may update these rows in place)
           rr[4 * i] = __float_as_uint(x.x); rr[4 * i + 1] = __float_as_uint(x.y);
           rr[4 * i + 2] = __float_as_uint(x.z); rr[4 * i + 3] = __float_as_uint(x.w);
         }
-        tmem_st16(tlane + TS_O + 64 * half + 16 * cb, rr, 0);
+        tmem_st32(tlane + TS_O + 64 * half, *reinterpret_cast<uint32_t(*)[32]>(rr));
+        tmem_st32(tlane + TS_O + 64 * half + 32, *reinterpret_cast<uint32_t(*)[32]>(rr + 32));
       }
       tmem_st_wait();
       have_o = true;
