@@ -154,6 +154,13 @@ __device__ __forceinline__ void st_global_v8(void* dst, const uint32_t* r) {
                "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
                : "memory");
 }
+// one 32-byte load of 8 words (the address is 32-byte aligned)
+__device__ __forceinline__ void ld_global_v8(const void* src, uint32_t* r) {
+  asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "l"(src)
+               : "memory");
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -758,12 +765,15 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       const float4* src = reinterpret_cast<const float4*>(a.init.o + srow * D + 64 * half);
       {
         // all sixteen loads of the row half are in flight together (one round trip, not four)
+        // (32-byte loads: a warp's load touches 32 rows whatever its width, so wider loads mean
+        // fewer passes through the L1 tags; plain loads, not the read-only path: the launch may update
+        // these rows in place)
         uint32_t rr[64];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float4 x = row_valid ? src[i] : make_float4(0.f, 0.f, 0.f, 0.f);   // (plain loads: the launch may update these rows in place)
-          rr[4 * i] = __float_as_uint(x.x); rr[4 * i + 1] = __float_as_uint(x.y);
-          rr[4 * i + 2] = __float_as_uint(x.z); rr[4 * i + 3] = __float_as_uint(x.w);
+        for (int i = 0; i < 64; ++i) rr[i] = 0u;
+        if (row_valid) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) ld_global_v8(src + 2 * i, rr + 8 * i);
         }
         tmem_st32(tlane + TS_O + 64 * half, *reinterpret_cast<uint32_t(*)[32]>(rr));
         tmem_st32(tlane + TS_O + 64 * half + 32, *reinterpret_cast<uint32_t(*)[32]>(rr + 32));
