@@ -303,6 +303,19 @@ lacache_status lacache_build_tokens(lacache_ctx* ctx, lacache_qkv* p, int block_
                                     const int32_t* token_ids, const void* hidden,
                                     void* cuda_stream);
 /*
+ * The incremental rebuild (see lacache_build_incremental / lacache_build_advance) fed by tokens:
+ * lacache_build_tokens_incremental projects all T tokens like lacache_build_tokens;
+ * lacache_build_advance_tokens projects the B*L_b FINAL tokens of the finished block (ids or hidden
+ * rows, layout of lacache_step_tokens' inputs) and advances to the next block.  Same errors as the
+ * calls they combine.
+ */
+lacache_status lacache_build_tokens_incremental(lacache_ctx* ctx, lacache_qkv* p, int block_idx,
+                                                const int32_t* token_ids, const void* hidden,
+                                                void* cuda_stream);
+lacache_status lacache_build_advance_tokens(lacache_ctx* ctx, lacache_qkv* p, const int32_t* fin_token_ids,
+                                            const void* fin_hidden, void* cuda_stream);
+
+/*
  * The build of the next block, re-projecting only what changed.  Token-wise results depend on the
  * token alone (Sec. 3.3.2), so from one block to the next only the tokens whose ids changed need
  * the embedding, norm and projections again: as a rule the B * L_b tokens of the block just

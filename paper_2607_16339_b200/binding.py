@@ -26,6 +26,7 @@ EXPORTS = [
     "lacache_step_tokens", "lacache_qkv_set_timing_events", "lacache_qkv_last_launch_count",
     "lacache_qkv_poll_status", "lacache_qkv_last_error", "lacache_set_step_overlap",
     "lacache_build_tokens_update", "lacache_build_incremental", "lacache_build_advance",
+    "lacache_build_tokens_incremental", "lacache_build_advance_tokens",
 ]
 
 
@@ -95,6 +96,8 @@ def load():
     lib.lacache_qkv_destroy.argtypes = [vp]
     lib.lacache_qkv_project.argtypes = [vp, vp, vp, ip, vp, vp, vp, vp, vp]
     lib.lacache_build_tokens.argtypes = [vp, vp, ip, vp, vp, vp]
+    lib.lacache_build_tokens_incremental.argtypes = [vp, vp, ip, vp, vp, vp]
+    lib.lacache_build_advance_tokens.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_step_tokens.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.lacache_build_tokens_update.argtypes = [vp, vp, ip, vp, vp, vp, ip, vp]
     lib.lacache_qkv_set_timing_events.argtypes = [vp, vp, vp]
@@ -233,6 +236,14 @@ class Context:
     def build_tokens(self, producer, block_idx, token_ids=None, hidden=None, stream=None):
         self._check(self._lib.lacache_build_tokens(self._h, producer._h, int(block_idx), _ptr(token_ids),
                                                    _ptr(hidden), _stream(stream)))
+
+    def build_tokens_incremental(self, producer, block_idx, token_ids=None, hidden=None, stream=None):
+        self._check(self._lib.lacache_build_tokens_incremental(self._h, producer._h, int(block_idx),
+                                                               _ptr(token_ids), _ptr(hidden), _stream(stream)))
+
+    def build_advance_tokens(self, producer, fin_token_ids=None, fin_hidden=None, stream=None):
+        self._check(self._lib.lacache_build_advance_tokens(self._h, producer._h, _ptr(fin_token_ids),
+                                                           _ptr(fin_hidden), _stream(stream)))
 
     def build_tokens_update(self, producer, block_idx, rows, token_ids=None, hidden=None, stream=None):
         self._check(self._lib.lacache_build_tokens_update(self._h, producer._h, int(block_idx), _ptr(rows),

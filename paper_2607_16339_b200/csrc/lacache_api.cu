@@ -845,6 +845,39 @@ lacache_status lacache_build_tokens_update(lacache_ctx* c, lacache_qkv* p, int b
   return st;
 }
 
+lacache_status lacache_build_tokens_incremental(lacache_ctx* c, lacache_qkv* p, int block_idx,
+                                                const int32_t* token_ids, const void* hidden, void* stream) {
+  if (!c || !p) return LACACHE_ERR_INVALID_ARG;
+  lacache_status st = check_producer(c, p, c->g.T);
+  if (st != LACACHE_OK) return st;
+  void *q, *k, *v;
+  qkv_scratch(p, false, &q, &k, &v);
+  qkv_set_full_owner(p, nullptr, 0);
+  st = lacache_qkv_project(p, token_ids, hidden, c->g.T, q, k, v, nullptr, stream);
+  if (st != LACACHE_OK) return fail(c, st, "producer: %s", lacache_qkv_last_error(p));
+  st = lacache_build_incremental(c, block_idx, q, k, v, stream);
+  if (st == LACACHE_OK) c->last_launches += lacache_qkv_last_launch_count(p);
+  return st;
+}
+
+lacache_status lacache_build_advance_tokens(lacache_ctx* c, lacache_qkv* p, const int32_t* fin_token_ids,
+                                            const void* fin_hidden, void* stream) {
+  if (!c || !p) return LACACHE_ERR_INVALID_ARG;
+  if (c->built_block < 0 || c->prefix_block != c->built_block)
+    return fail(c, LACACHE_ERR_STATE, "lacache_build_advance_tokens needs the state of an incremental build or of an earlier advance");
+  const int n = c->g.B * c->g.block_len;
+  lacache_status st = check_producer(c, p, n);
+  if (st != LACACHE_OK) return st;
+  void *q, *k, *v;
+  qkv_scratch(p, true, &q, &k, &v);
+  // (the RoPE launch of the advance is an ordinary one: it starts when the projection has completed)
+  st = qkv_project_rows(p, fin_token_ids, fin_hidden, n, q, k, v, nullptr, nullptr, 0, false, stream);
+  if (st != LACACHE_OK) return fail(c, st, "producer: %s", lacache_qkv_last_error(p));
+  st = lacache_build_advance(c, q, k, v, stream);
+  if (st == LACACHE_OK) c->last_launches += lacache_qkv_last_launch_count(p);
+  return st;
+}
+
 lacache_status lacache_step_tokens(lacache_ctx* c, lacache_qkv* p, const int32_t* blk_token_ids,
                                    const void* blk_hidden, float* out, float* lse, void* stream) {
   if (!c || !p) return LACACHE_ERR_INVALID_ARG;

@@ -142,3 +142,40 @@ def test_advance_needs_an_incremental_state():
         simt.build_incremental(0, to_dev(q, wl), to_dev(k, wl), to_dev(v, wl))
     assert e.value.status == binding.ERR_UNSUPPORTED
     simt.destroy()
+
+
+def test_token_fed_generation_advances():
+    """The incremental rebuild fed by token ids: all T tokens projected once at block 0, afterwards only
+    the finished block's final tokens (projection -> RoPE-on-write -> advance); every block's last step
+    against the oracle chain (token-wise oracle at model precision -> attention oracle)."""
+    import oracle
+    from paper_2607_16339_b200.workloads import TokenModel
+    from test_gpu_tokenwise import make_producer, oracle_qkv
+    wl = small_workload(name="tokgen", prompt_lens=(150, 61), gen_len=96, block_len=32, steps=2, hq=4, hkv=2)
+    tm = TokenModel(wl, 512, 3000)
+    prod = make_producer(tm, wl.total_tokens)
+    ctx = make_ctx(wl, engine=binding.ENGINE_TCGEN05)
+    sch = SyntheticSchedule(wl)   # index sets only
+    out, lse = new_outputs(wl)
+    ids = tm.full_ids(0).copy()
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    ctx.build_tokens_incremental(prod, 0, token_ids=dev(ids))
+    fin = None
+    for b in range(wl.n_blocks):
+        if b > 0:
+            ctx.build_advance_tokens(prod, fin_token_ids=dev(fin))
+        fin = tm.block_ids(b, wl.steps_per_block)      # the block's last step sees its final tokens
+        assert not (fin == tm.mask_id).any()
+        ctx.step_tokens(prod, out, lse, blk_token_ids=dev(fin))
+        torch.cuda.synchronize()
+        for o in (ctx, prod):
+            st, msg = o.poll_status()
+            assert st == binding.OK, msg
+        ids[sch.block_rows(b)] = fin
+        _, qf, kf, vf = oracle_qkv(tm, ids=ids)
+        ref, rlse = oracle.attention(qf, kf, vf, wl.cu_seqlens, wl.rope_theta, wl.head_dim ** -0.5)
+        err = np.abs(out.cpu().numpy().astype(np.float64) - ref)
+        assert err.max() <= 2e-2 and err.mean() <= 2e-3, (b, err.max(), err.mean())
+        assert np.abs(lse.cpu().numpy() - rlse).max() <= 2e-2
+    ctx.destroy()
+    prod.destroy()
