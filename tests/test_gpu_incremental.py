@@ -179,3 +179,47 @@ def test_token_fed_generation_advances():
         assert np.abs(lse.cpu().numpy() - rlse).max() <= 2e-2
     ctx.destroy()
     prod.destroy()
+
+
+@pytest.mark.parametrize("cfg,n_adv", [(3, 3), (5, 2), (6, 2)])
+def test_full_size_advance(cfg, n_adv):
+    """Full-size workloads (the long-generation and the GQA long-prompt configurations, and the
+    large-batch extension) advanced n_adv blocks from an incremental build: the step after the last
+    advance against a full recompute of the same inputs on every row, and against the oracle on all
+    rows of up to three whole sequences (first, longest, last)."""
+    import oracle
+    from paper_2607_16339_b200.workloads import WORKLOADS, DeviceSchedule
+    from lacache_testlib import TOL
+    wl = WORKLOADS[cfg]
+    S = wl.steps_per_block
+    sched = DeviceSchedule(wl, 23, torch.device("cuda"), n_adv * S + 1)
+    ctx = make_ctx(wl, engine=binding.ENGINE_TCGEN05)
+    ctx.build_incremental(0, *sched.full[0])
+    for b in range(1, n_adv + 1):
+        ctx.build_advance(*sched.steps[b * S - 1])     # the finished block's rows as its last step saw them
+    out, lse = new_outputs(wl)
+    qb, kb, vb = sched.steps[n_adv * S]
+    ctx.step(qb, kb, vb, out, lse)
+    torch.cuda.synchronize()
+    st, msg = ctx.poll_status()
+    assert st == 0, msg
+    cu = wl.cu_seqlens
+    rows = torch.cat([torch.arange(cu[b] + P + n_adv * wl.block_len, cu[b] + P + (n_adv + 1) * wl.block_len)
+                      for b, P in enumerate(wl.prompt_lens)]).cuda()
+    qf, kf, vf = (x.clone() for x in sched.full[n_adv])
+    qf[rows], kf[rows], vf[rows] = qb, kb, vb
+    out2, lse2 = new_outputs(wl)
+    ctx.full_recompute(qf, kf, vf, out2, lse2)
+    torch.cuda.synchronize()
+    assert float((out - out2).abs().max()) <= TOL_CACHED_VS_FULL["bf16"]
+    assert float((lse - lse2).abs().max()) <= TOL_CACHED_VS_FULL["bf16"]
+    seqs = sorted({0, int(np.argmax(wl.prompt_lens)), wl.batch - 1})
+    idx = np.concatenate([np.arange(cu[b], cu[b + 1]) for b in seqs])
+    sub_cu = np.concatenate([[0], np.cumsum([cu[b + 1] - cu[b] for b in seqs])]).astype(np.int32)
+    t_idx = torch.from_numpy(idx).cuda()
+    host = lambda t: t[t_idx].float().cpu().numpy().astype(np.float64)
+    ref, rlse = oracle.attention(host(qf), host(kf), host(vf), sub_cu, wl.rope_theta, wl.head_dim ** -0.5)
+    err = np.abs(out[t_idx].cpu().numpy().astype(np.float64) - ref)
+    assert err.max() <= TOL["bf16"][0] and err.mean() <= TOL["bf16"][1], (err.max(), err.mean())
+    assert np.abs(lse[t_idx].cpu().numpy() - rlse).max() <= TOL["bf16"][0]
+    ctx.destroy()
