@@ -706,6 +706,7 @@ lacache_status run_window(lacache_ctx* c, lacache_ctx::ListRef list, int blk, co
                           const StateBuffers& dst, const StateBuffers& snap, cudaStream_t s) {
   if (list.n == 0) return LACACHE_OK;
   AttnArgs a = attn_args(c, MODE_BUILD, list, blk, c->rot, nullptr, nullptr);
+  a.window = 1;
   a.init = init;
   a.st = dst;
   a.snap = snap;

@@ -117,6 +117,7 @@ struct AttnArgs {
   const int32_t* blk_start;  // [B] absolute token index of the block's first row
   RotBuffers rot;
   StateBuffers st;
+  int window;                // build: the items are ITEM_ROWS_WINDOW (the kernel instantiation that knows them)
   StateBuffers init;         // build over key windows: the state units with the init bit start from (may alias st)
   StateBuffers snap;         // ... and where units with the snapshot bit store their state after the first key tile
                              // (may alias init: a unit loads its rows before it stores them)

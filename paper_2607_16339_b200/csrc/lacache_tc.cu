@@ -231,6 +231,11 @@ __device__ __forceinline__ bool wait_bar(const Cta& c, int slot, uint32_t parity
 }
 
 // One unit of work of the stream role, decoded identically by every warp role.
+// What the stream role's templates are instantiated for: a build or a full recompute; a step; a build
+// over key windows (units may start from a stored state and store a snapshot: the incremental rebuild).
+// Separate kernels, so that the plain build and the step carry none of the window code.
+enum StreamKind : int { KIND_BUILD = 0, KIND_STEP = 1, KIND_WINDOW = 2 };
+
 struct Unit {
   int row0, nrows, h, kh, seq;
   int key_base, t0, t1;   // key tiles [t0, t1): tile t holds keys key_base + 64 t ...
@@ -251,8 +256,11 @@ __device__ __forceinline__ bool unit_row_valid(const Unit& un, int r) {
 // PACKED (a.pack > 1): the units are block queries of several heads side by side in one tile.  A template
 // parameter of the whole kernel, so that the kernel a build or an MHA step runs carries none of the per-row
 // head arithmetic: this kernel is sensitive to its code size.
-template <bool PACKED, bool STEP>
+template <bool PACKED, int KIND>
 __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs& a, const WorkItem& it, int u) {
+  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool WINDOW = KIND == KIND_WINDOW;
+  (void)WINDOW;
   Unit un;
   // units are head-minor: unit u = item u / slots of head (or head group) u % slots (a CTA's units, a
   // fixed stride apart, then cycle through the items instead of drawing one item's heads)
@@ -283,7 +291,7 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
   un.nchunks = 1;
   un.q_rows = BM;
   un.init = un.snap = 0;
-  if (!STEP && it.kind == ITEM_ROWS_WINDOW) {
+  if (WINDOW) {
     // keys [kt0, kt1) of the sequence (token indices), optionally without the block's; tiles are
     // counted from token `pad`, which may lie before the window (and before token 0: those key rows
     // load as zeros and are masked like every key outside the window)
@@ -379,18 +387,24 @@ struct TileCursor {
   Unit un;
   bool valid, q_done, loads_q;
 };
-template <bool PACKED, bool STEP>
+template <bool PACKED, int KIND>
 __device__ __forceinline__ void cursor_load_unit(const Geometry& g, const AttnArgs& a, TileCursor& cu, int n_units) {
+  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool WINDOW = KIND == KIND_WINDOW;
+  (void)WINDOW;
   cu.valid = cu.u < n_units;
   if (!cu.valid) return;
   cu.it = load_item(a.items + cu.u / (PACKED ? a.stream_slots : g.Hq));
-  cu.un = decode_stream<PACKED, STEP>(g, a, cu.it, cu.u);
+  cu.un = decode_stream<PACKED, KIND>(g, a, cu.it, cu.u);
   cu.t = cu.un.t0;
   cu.q_done = !cu.loads_q;
 }
-template <bool PACKED, bool STEP>
+template <bool PACKED, int KIND>
 __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs& a, TileCursor& cu, int stride,
                                                int n_units) {
+  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool WINDOW = KIND == KIND_WINDOW;
+  (void)WINDOW;
   // move to the next tile; cross into the next unit(s) when this one is exhausted
   if (cu.t < cu.un.t1) {
     ++cu.t;
@@ -399,21 +413,24 @@ __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs
   while (cu.valid && cu.t >= cu.un.t1 && cu.q_done) {
     cu.u += stride;
     ++cu.uu;
-    cursor_load_unit<PACKED, STEP>(g, a, cu, n_units);
+    cursor_load_unit<PACKED, KIND>(g, a, cu, n_units);
   }
 }
 
-template <bool PACKED, bool STEP>
+template <bool PACKED, int KIND>
 __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a,
                                 int first, int stride, int n_units, WorkItem it) {
+  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool WINDOW = KIND == KIND_WINDOW;
+  (void)WINDOW;
   // three independent cursors: Q tiles (one per unit), key tiles, value tiles
   TileCursor cq, ck, cv;
   cq.u = first; cq.uu = 0; cq.jj = 0; cq.loads_q = true;
-  cursor_load_unit<PACKED, STEP>(g, a, cq, n_units);
+  cursor_load_unit<PACKED, KIND>(g, a, cq, n_units);
   ck = cq;
   ck.loads_q = false;  // the key and value cursors never load Q
   ck.q_done = true;
-  if (ck.valid && ck.t >= ck.un.t1) cursor_advance<PACKED, STEP>(g, a, ck, stride, n_units);
+  if (ck.valid && ck.t >= ck.un.t1) cursor_advance<PACKED, KIND>(g, a, ck, stride, n_units);
   cv = ck;
   // What the RoPE kernel launched just before this one writes must not be loaded
   // before that grid has completed (this kernel may have started early): in a step
@@ -437,7 +454,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         mbar_arrive(c.bar(BAR_Q_FULL));
         cq.q_done = true;
         cq.t = cq.un.t1;
-        cursor_advance<PACKED, STEP>(g, a, cq, stride, n_units);
+        cursor_advance<PACKED, KIND>(g, a, cq, stride, n_units);
         did = true;
       } else if (!dep_done) {
         blocked_on_dep = true;
@@ -445,7 +462,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         load_q_tile(c, maps, cq.un.q_rows, cq.un.row0, cq.un.h, cq.un.rh != 0);
         cq.q_done = true;
         cq.t = cq.un.t1;
-        cursor_advance<PACKED, STEP>(g, a, cq, stride, n_units);
+        cursor_advance<PACKED, KIND>(g, a, cq, stride, n_units);
         // a build's Q tiles come from HBM once the batch outgrows L2: the next unit's tile is asked
         // into L2 a whole unit ahead of its load
         if (!STEP && cq.valid) tma_prefetch_5d(&maps.q, 0, cq.un.row0, 0, cq.un.h, 0);
@@ -462,7 +479,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         const uint32_t khi = c.base + SM_K + sk * K_STAGE;
         mbar_expect_tx(bar, 4 * KS_BOX);
         load_qk_box(khi, &maps.k, bar, krow, ck.un.kh);  // the lo plane lands at khi + SK_LO
-        cursor_advance<PACKED, STEP>(g, a, ck, stride, n_units);
+        cursor_advance<PACKED, KIND>(g, a, ck, stride, n_units);
         did = true;
       }
     }
@@ -475,7 +492,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
         mbar_expect_tx(bar, 2 * KS_BOX);
         load_v_box(vb, &maps.v, bar, krow, cv.un.kh);
-        cursor_advance<PACKED, STEP>(g, a, cv, stride, n_units);
+        cursor_advance<PACKED, KIND>(g, a, cv, stride, n_units);
         did = true;
       }
     }
@@ -508,16 +525,19 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
 // Scores of tile j need its keys and the score buffer of tile j - 2 read (= the probabilities of tile
 // j - 2 written); P~V of tile j needs its probabilities and its values.  Each code block exists once
 // (the unrolled MMA sequences are large, and cold instruction fetches are slow).
-template <bool PACKED, bool STEP>
+template <bool PACKED, int KIND>
 __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
                                   int n_units, WorkItem it) {
+  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool WINDOW = KIND == KIND_WINDOW;
+  (void)WINDOW;
   constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
   int uu = 0;
   uint32_t js = 0;  // score tiles issued so far (stage and buffer = js & 1, phase = (js >> 1) & 1)
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
-    const Unit un = decode_stream<PACKED, STEP>(g, a, it, u);
+    const Unit un = decode_stream<PACKED, KIND>(g, a, it, u);
     const uint32_t q_box = (uint32_t)un.q_rows * 128u;
     const int n_tiles = un.t1 - un.t0;
     if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
@@ -539,15 +559,18 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   }
 }
 
-template <bool PACKED, bool STEP>
+template <bool PACKED, int KIND>
 __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
                               int n_units, WorkItem it) {
+  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool WINDOW = KIND == KIND_WINDOW;
+  (void)WINDOW;
   int uu = 0;
   uint32_t jp = 0;  // P~V tiles issued so far
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
-    const Unit un = decode_stream<PACKED, STEP>(g, a, it, u);
+    const Unit un = decode_stream<PACKED, KIND>(g, a, it, u);
     const int n_tiles = un.t1 - un.t0;
     // O~ of the previous unit has been read by the row threads (observed once per unit, in order)
     if (uu >= 1 && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
@@ -557,7 +580,7 @@ __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a
       if (!wait_bar(c, sv ? BAR_V_FULL1 : BAR_V_FULL, ph, LOC_WAIT_V)) return;
       tc_fence_after();
       issue_pv_mma(c.base + SM_V + sv * V_STAGE, KS_BOX, c.tmem + TS_P + 64 * b, c.tmem + TS_O, BN / 16,
-                   (j == 0 && !(!STEP && un.init)) ? 0u : 1u);
+                   (j == 0 && !(WINDOW && un.init)) ? 0u : 1u);
       tc_commit(c.bar(BAR_O_FULL));
       tc_commit(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE));
     }
@@ -693,9 +716,12 @@ __device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs
   }
 }
 
-template <bool PACKED, bool STEP>
+template <bool PACKED, int KIND>
 __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units,
                             WorkItem it) {
+  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool WINDOW = KIND == KIND_WINDOW;
+  (void)WINDOW;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int quad = warp & 3;
   const int half = (warp - 2) >> 2;         // 0: first 64 columns / features, 1: the rest
@@ -708,7 +734,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
   for (int u = first; u < n_units; u += stride) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
-    const Unit un = decode_stream<PACKED, STEP>(g, a, it, u);
+    const Unit un = decode_stream<PACKED, KIND>(g, a, it, u);
     it = nxt;
     if (u == first && STEP && a.q_raw != nullptr) {
       // The CTA's first unit: rotate the block's queries of this (sequence, head) here,
@@ -751,7 +777,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     float m_ref = -INFINITY, l_part = 0.f;
     bool first_tile = true;
     bool have_o = false;   // O~ in TMEM holds something before the unit's first P~V
-    if (!STEP && un.init) {
+    if (WINDOW && un.init) {
       // The unit continues from a stored state (m, l, O~) of its rows: the reference exponent and the
       // normaliser go to registers (the normaliser to the first thread of the pair), O~ to the
       // accumulator columns this thread owns.  Nobody else reads or writes those cells between units
@@ -780,7 +806,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       }
       tmem_st_wait();
       have_o = true;
-      if (u + stride < n_units && it.kind == ITEM_ROWS_WINDOW && (it.chunk & 1) && r < it.nrows) {
+      if (u + stride < n_units && (it.chunk & 1) && r < it.nrows) {
         // the next unit's rows of that state, asked into L2 now (`it` already holds its item)
         const char* nx = reinterpret_cast<const char*>(
             a.init.o + ((size_t)((u + stride) % g.Hq) * g.Tp + it.row0 + r) * D + 64 * half);
@@ -798,7 +824,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       // previous tile, either before an in-place rescale or at the end of the tile
       bool o_waited = first_tile;
       if (active) {
-        if (!STEP && un.snap && t == un.t0 + 1) {
+        if (WINDOW && un.snap && t == un.t0 + 1) {
           // The state after the unit's first key tile goes to a.snap before this tile changes it:
           // P~V of that tile must be complete; the pair adds up its normaliser halves.
           if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
@@ -891,7 +917,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
         float alpha = 1.f;
         if (m_new != m_ref) alpha = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
-        if ((!first_tile || (!STEP && have_o)) && __any_sync(0xffffffffu, alpha != 1.f)) {
+        if ((!first_tile || (WINDOW && have_o)) && __any_sync(0xffffffffu, alpha != 1.f)) {
           // O~ in TMEM is rescaled in place: P~V of the previous tile must be done
           if (!o_waited) {
             if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
@@ -1041,7 +1067,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       // (the TMEM loads are warp-wide: rows past the end of a clipped tile take part in them and
       // only skip the stores; first_tile is uniform over the CTA)
       uint32_t rr[64];
-      if (!first_tile || (!STEP && have_o)) {
+      if (!first_tile || (WINDOW && have_o)) {
         tmem_ld32(tlane + TS_O + 64 * half, *reinterpret_cast<uint32_t(*)[32]>(rr));
         tmem_ld32(tlane + TS_O + 64 * half + 32, *reinterpret_cast<uint32_t(*)[32]>(rr + 32));
         tmem_ld_wait();
@@ -1054,7 +1080,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         for (int i = 0; i < 8; ++i) st_global_v8(dst + 2 * i, rr + 8 * i);
       }
       if (row_valid && half == 0) { a.st.m[srow] = m_ref; a.st.l[srow] = l_run; }
-      if (!STEP && un.snap && un.t1 - un.t0 <= 1) {
+      if (WINDOW && un.snap && un.t1 - un.t0 <= 1) {
         // a single key tile: the state after it is the final one as well
         float4* sdst = reinterpret_cast<float4*>(a.snap.o + srow * D + 64 * half);
         if (row_valid) {
@@ -1648,11 +1674,12 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
   }
 }
 
-template <bool PACKED, bool STEP, bool DEEP>
+template <bool PACKED, int KIND, bool DEEP>
 __global__ void __launch_bounds__(THREADS, 1)
 tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const AttnArgs a) {
-  // (instantiated twice, as two kernels: PACKED for the steps of a GQA model whose block queries share
-  // tiles across heads, see decode_stream)
+  constexpr bool STEP = KIND == KIND_STEP;
+  // (PACKED: the steps of a GQA model whose block queries share tiles across heads, see decode_stream;
+  // KIND: see StreamKind; DEEP: which variant of the merge role a step runs)
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const int tid = threadIdx.x;
   const int warp = tid >> 5;
@@ -1742,7 +1769,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
 
   if (warp == 0) {
     if (stream) {
-      if (tid == 0) stream_producer<PACKED, STEP>(c, maps, g, a, first, stride, n_units, it0);
+      if (tid == 0) stream_producer<PACKED, KIND>(c, maps, g, a, first, stride, n_units, it0);
     } else if (deep) {
       if (tid == 0) deep_producer(c, maps, g, n_my, a.k_raw != nullptr);
     } else {
@@ -1750,14 +1777,14 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     }
   } else if (warp == 1) {
     if (tid == 32) {
-      if (stream) stream_mma_scores<PACKED, STEP>(c, g, a, first, stride, n_units, it0);
+      if (stream) stream_mma_scores<PACKED, KIND>(c, g, a, first, stride, n_units, it0);
       else if (deep) deep_mma(c, g, n_my, a.k_raw != nullptr);
       else merge_mma(c, g, a, first, stride, n_units);
     }
   } else if (warp == 10) {
-    if (tid == 320 && stream) stream_mma_pv<PACKED, STEP>(c, g, a, first, stride, n_units, it0);
+    if (tid == 320 && stream) stream_mma_pv<PACKED, KIND>(c, g, a, first, stride, n_units, it0);
   } else {
-    if (stream) stream_rows<PACKED, STEP>(c, g, a, first, stride, n_units, it0);
+    if (stream) stream_rows<PACKED, KIND>(c, g, a, first, stride, n_units, it0);
     else if (deep) deep_rows(c, g, a, n_my);
     else merge_rows(c, maps, g, a, first, stride, n_units, it0);
     bulk_wait_read();
@@ -1863,9 +1890,9 @@ bool make_v_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* e
 }  // namespace
 
 cudaError_t tc_prepare() {
-  const void* kernels[] = {(const void*)tc_attn_kernel<false, false, false>, (const void*)tc_attn_kernel<false, true, false>,
-                           (const void*)tc_attn_kernel<false, true, true>, (const void*)tc_attn_kernel<true, true, false>,
-                           (const void*)tc_attn_kernel<true, true, true>};
+  const void* kernels[] = {(const void*)tc_attn_kernel<false, KIND_BUILD, false>, (const void*)tc_attn_kernel<false, KIND_WINDOW, false>,
+                           (const void*)tc_attn_kernel<false, KIND_STEP, false>, (const void*)tc_attn_kernel<false, KIND_STEP, true>,
+                           (const void*)tc_attn_kernel<true, KIND_STEP, false>, (const void*)tc_attn_kernel<true, KIND_STEP, true>};
   for (const void* k : kernels) {
     cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
     if (e != cudaSuccess) return e;
@@ -1919,15 +1946,18 @@ cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* map
   cfg.attrs = attr;
   static const bool no_pdl = getenv("LACACHE_NO_PDL") != nullptr;
   cfg.numAttrs = no_pdl ? 0 : 1;
-  // five instantiations: build / full recompute; the step of an MHA and of a GQA model, each with
-  // either variant of the merge role
-  if (a.mode != MODE_STEP) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, false, false>, *maps, g, a);
-  if (a.pack > 1) {
-    if (a.merge_deep) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true, true, true>, *maps, g, a);
-    return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true, true, false>, *maps, g, a);
+  // six instantiations: build / full recompute; build over key windows; the step of an MHA and of a
+  // GQA model, each with either variant of the merge role
+  if (a.mode != MODE_STEP) {
+    if (a.window) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, KIND_WINDOW, false>, *maps, g, a);
+    return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, KIND_BUILD, false>, *maps, g, a);
   }
-  if (a.merge_deep) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, true, true>, *maps, g, a);
-  return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, true, false>, *maps, g, a);
+  if (a.pack > 1) {
+    if (a.merge_deep) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true, KIND_STEP, true>, *maps, g, a);
+    return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true, KIND_STEP, false>, *maps, g, a);
+  }
+  if (a.merge_deep) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, KIND_STEP, true>, *maps, g, a);
+  return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, KIND_STEP, false>, *maps, g, a);
 }
 
 }  // namespace lacache
