@@ -313,7 +313,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
         items[i].chunk = flags;
       }
     };
-    enum { W_INIT = 1, W_SNAP = 2, W_SKIP_BLOCK = 4 };
+    enum { W_INIT = 1, W_SNAP = 2, W_SKIP_BLOCK = 4, W_JUMP_BLOCK = 8 };
     int off = (int)items.size();
     for (int b = 0; b < g.B; ++b) {
       const int cs = c->cu[b], ce = c->cu[b + 1], s0 = c->blk_start_all[(size_t)k * g.B + b], e0 = s0 + g.block_len;
@@ -351,7 +351,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
       int from = (int)items.size();
       add_row_tiles(items, b, cs, sp, R, cs, ce, s0);
       add_row_tiles(items, b, e0, ce, R, cs, ce, s0);
-      window(from, s0 - TC_KEYS, sp, ce > e0 ? ce : s0, W_INIT | W_SNAP | W_SKIP_BLOCK);
+      window(from, s0 - TC_KEYS, sp, ce > e0 ? ce : s0, W_INIT | W_SNAP | W_JUMP_BLOCK);
       // the finished block's rows: their new prefix state + the keys after block k
       from = (int)items.size();
       add_row_tiles(items, b, sp, s0, R, cs, ce, s0);

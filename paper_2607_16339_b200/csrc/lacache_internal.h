@@ -16,7 +16,8 @@ enum ItemKind : int32_t {
                          // indices; key tiles are counted from token `pad` (<= kt0, may be negative).
                          // chunk bit 0: continue from the rows' state in AttnArgs::init; bit 1: store the
                          // state after the first key tile to AttnArgs::snap; bit 2: leave out the keys of
-                         // the block at blk_start
+                         // the block at blk_start; bit 3: the first tile ends at blk_start (pad = blk_start -
+                         // tile width) and the tiles after it are counted from the end of that block
 };
 struct WorkItem {
   int32_t kind;   // ItemKind

@@ -245,7 +245,14 @@ struct Unit {
   int nh, rh;             // packed block queries: nh heads h, h + 1, ... of one KV group, rh lanes each (rh = 0: one head)
   int init;               // build over a key window: the unit starts from the rows' state in a.init instead of an empty one
   int snap;               // ... and stores the state it has after its first key tile to a.snap
+  int base1;              // >= 0: key tiles after the first are counted from this token instead of key_base + BN
 };
+// first key (token index) of key tile t of a unit
+template <int KIND>
+__device__ __forceinline__ int tile_key_row(const Unit& un, int t) {
+  if (KIND == KIND_WINDOW && un.base1 >= 0 && t > 0) return un.base1 + (t - 1) * BN;
+  return un.key_base + t * BN;
+}
 // head and row within the head's rows of tile row r; whether r holds a real query row (rh is 0, 32 or 64)
 __device__ __forceinline__ int unit_head(const Unit& un, int r) { return un.rh ? un.h + (r >> (un.rh == 64 ? 6 : 5)) : un.h; }
 __device__ __forceinline__ int unit_row(const Unit& un, int r) { return un.rh ? (r & (un.rh - 1)) : r; }
@@ -291,6 +298,7 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
   un.nchunks = 1;
   un.q_rows = BM;
   un.init = un.snap = 0;
+  un.base1 = -1;
   if (WINDOW) {
     // keys [kt0, kt1) of the sequence (token indices), optionally without the block's; tiles are
     // counted from token `pad`, which may lie before the window (and before token 0: those key rows
@@ -302,6 +310,11 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
     if (it.chunk & 4) {
       un.x0 = it.blk_start;
       un.x1 = it.blk_start + g.block_len;
+    }
+    if (it.chunk & 8) {
+      // the first tile ends where the block starts; the others start right after the block
+      un.base1 = it.blk_start + g.block_len;
+      un.t1 = 1 + (it.kt1 > un.base1 ? (it.kt1 - un.base1 + BN - 1) / BN : 0);
     }
     un.epi = EPI_STATE;
     un.init = it.chunk & 1;
@@ -474,7 +487,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
       if (!dep_done && tile_depends(ck)) {
         blocked_on_dep = true;
       } else if (kuse == 0 || mbar_test(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE), (kuse - 1) & 1)) {
-        const int krow = ck.un.key_base + ck.t * BN;
+        const int krow = tile_key_row<KIND>(ck.un, ck.t);
         const uint32_t bar = c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL);
         const uint32_t khi = c.base + SM_K + sk * K_STAGE;
         mbar_expect_tx(bar, 4 * KS_BOX);
@@ -488,7 +501,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
       if (!dep_done && tile_depends(cv)) {
         blocked_on_dep = true;
       } else if (vuse == 0 || mbar_test(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE), (vuse - 1) & 1)) {
-        const int krow = cv.un.key_base + cv.t * BN;
+        const int krow = tile_key_row<KIND>(cv.un, cv.t);
         const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
         mbar_expect_tx(bar, 2 * KS_BOX);
         load_v_box(vb, &maps.v, bar, krow, cv.un.kh);
@@ -849,7 +862,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
             if (half == 0) { a.snap.m[srow] = m_ref; a.snap.l[srow] = l_sum; }
           }
         }
-        const int tile_lo = un.key_base + t * BN;
+        const int tile_lo = tile_key_row<KIND>(un, t);
         const int v_lo = max(un.k0 - tile_lo, 0), v_hi = min(un.k1 - tile_lo, BN);
         const int e_lo = un.x0 - tile_lo, e_hi = un.x1 - tile_lo;
         const bool all_valid = v_lo == 0 && v_hi == BN && (un.x1 <= un.x0 || e_hi <= 0 || e_lo >= BN);
