@@ -166,6 +166,21 @@ lacache_status lacache_build_advance(lacache_ctx* ctx, const void* q_fin, const 
 lacache_status lacache_step(lacache_ctx* ctx, const void* q_blk, const void* k_blk,
                             const void* v_blk, float* out, float* lse, void* cuda_stream);
 
+/*
+ * Sampling-stage truncation (Sec. 3.4, last paragraph; the caption of the figure of one inference
+ * step): the float softmax over the vocabulary is evaluated on the rows of the current block only.
+ * logits [T, vocab] of `dtype` (LACACHE_DTYPE_BF16 or _FP32; DEVICE, row-major, every token's row
+ * present as the model's head writes them) -- only the B*L_b rows of the block the context was last
+ * built for (or advanced to) are read.  Per block row, in the order of lacache_step's inputs
+ * (sequence-major): token = the most probable vocabulary entry (the lowest id among entries of
+ * exactly equal logit), conf = its probability, lse = log sum_v exp(logit_v) (lse may be NULL).
+ * conf / token / lse are DEVICE arrays [B*L_b] (fp32, int32, fp32).  A logit of -inf contributes
+ * nothing.  fp32 arithmetic.  LACACHE_ERR_STATE before a build.  Allocates a small scratch on first
+ * use.  Calls on one context must not overlap on the GPU (they share that scratch).
+ */
+lacache_status lacache_sample_block(lacache_ctx* ctx, const void* logits, int dtype, int vocab,
+                                    float* conf, int32_t* token, float* lse, void* cuda_stream);
+
 /* Overlap of consecutive lacache_step calls on the device (see lacache_step): on (non-zero,
  * the default) or off.  No paper counterpart. */
 lacache_status lacache_set_step_overlap(lacache_ctx* ctx, int enable);

@@ -26,7 +26,7 @@ EXPORTS = [
     "lacache_step_tokens", "lacache_qkv_set_timing_events", "lacache_qkv_last_launch_count",
     "lacache_qkv_poll_status", "lacache_qkv_last_error", "lacache_set_step_overlap",
     "lacache_build_tokens_update", "lacache_build_incremental", "lacache_build_advance",
-    "lacache_build_tokens_incremental", "lacache_build_advance_tokens",
+    "lacache_build_tokens_incremental", "lacache_build_advance_tokens", "lacache_sample_block",
 ]
 
 
@@ -84,6 +84,7 @@ def load():
     lib.lacache_export_index_meta.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_set_timing_events.argtypes = [vp, vp, vp]
     lib.lacache_set_step_overlap.argtypes = [vp, ip]
+    lib.lacache_sample_block.argtypes = [vp, vp, ip, ip, vp, vp, vp, vp]
     lib.lacache_full_recompute_static.argtypes = [ip, ip, ip, ip, ip, ctypes.c_float, ctypes.c_float, vp, vp, vp, vp,
                                                   vp, vp]
     lib.lacache_total_tokens.argtypes = [vp]
@@ -253,6 +254,13 @@ class Context:
     def step_tokens(self, producer, out, lse=None, blk_token_ids=None, blk_hidden=None, stream=None):
         self._check(self._lib.lacache_step_tokens(self._h, producer._h, _ptr(blk_token_ids), _ptr(blk_hidden),
                                                   _ptr(out), _ptr(lse), _stream(stream)))
+
+    def sample_block(self, logits, conf, token, lse=None, stream=None):
+        """logits [T, vocab] bf16 or fp32; conf fp32 / token int32 / lse fp32 [B * L_b]."""
+        import torch
+        dt = DTYPE_BF16 if logits.dtype == torch.bfloat16 else DTYPE_FP32
+        self._check(self._lib.lacache_sample_block(self._h, _ptr(logits), dt, int(logits.shape[-1]), _ptr(conf),
+                                                   _ptr(token), _ptr(lse), _stream(stream)))
 
     def set_timing_events(self, ev_start, ev_stop):
         """torch.cuda.Event pair (already recorded once) or (None, None)."""

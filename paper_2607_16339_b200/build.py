@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "liblacache.so")
-SOURCES = ["lacache_api.cu", "lacache_rope.cu", "lacache_simt.cu", "lacache_tc.cu", "lacache_static.cu", "lacache_qkv.cu"]
+SOURCES = ["lacache_api.cu", "lacache_rope.cu", "lacache_simt.cu", "lacache_tc.cu", "lacache_static.cu", "lacache_qkv.cu", "lacache_sample.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -29,6 +29,8 @@ struct lacache_ctx {
   // cached state = prefix state + the keys after the block; the finished block's rows from scratch;
   // every other row advanced by the finished block's keys and completed by the keys after the block)
   std::vector<ListRef> inc_prefix, inc_comb, inc_fresh, inc_fused;
+  float* sample_part = nullptr;   // scratch of lacache_sample_block (allocated on first use)
+  int* sample_counters = nullptr;
   StateBuffers pst{};      // prefix state of every token: its keys before the current block (allocated on first use)
   int prefix_block = -1;   // block pst is valid for
   int num_sms = 148;
@@ -945,6 +947,41 @@ lacache_status step_impl(lacache_ctx* c, const void* q, const void* k, const voi
   return run_attention(c, a, false, s);
 }
 }  // namespace
+
+lacache_status lacache_sample_block(lacache_ctx* c, const void* logits, int dtype, int vocab, float* conf,
+                                    int32_t* token, float* lse, void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if (c->built_block < 0) return fail(c, LACACHE_ERR_STATE, "lacache_sample_block before a successful build");
+  if (!logits || !conf || !token) return fail(c, LACACHE_ERR_INVALID_ARG, "NULL pointer");
+  if (dtype != LACACHE_DTYPE_BF16 && dtype != LACACHE_DTYPE_FP32) return fail(c, LACACHE_ERR_INVALID_ARG, "dtype %d", dtype);
+  if (vocab <= 0) return fail(c, LACACHE_ERR_INVALID_ARG, "vocab %d", vocab);
+  constexpr int MAX_SPLITS = 64;
+  const int n = c->g.B * c->g.block_len;
+  if (!c->sample_part) {
+    CU_TRY(c, dev_alloc(c, &c->sample_part, (size_t)n * MAX_SPLITS * 4));
+    CU_TRY(c, dev_alloc(c, &c->sample_counters, (size_t)n, true));
+  }
+  SampleArgs a{};
+  a.logits = logits; a.dtype = dtype;
+  a.n_tokens = c->g.T; a.vocab = vocab;
+  a.rows = c->d_blk_tok + (size_t)c->built_block * n;
+  a.n_rows = n;
+  // enough CTAs for two per SM, each with at least 2048 entries, slices a multiple of 8 entries
+  int splits = std::max(1, std::min(MAX_SPLITS, (2 * c->num_sms + n - 1) / n));
+  splits = std::min(splits, std::max(1, vocab / 2048));
+  int slice = ((vocab + splits - 1) / splits + 7) / 8 * 8;
+  splits = (vocab + slice - 1) / slice;
+  a.splits = splits; a.slice = slice;
+  const size_t row_bytes = (size_t)vocab * elem_size(dtype);
+  a.vector_ok = (row_bytes % 16 == 0 && !misaligned(logits)) ? 1 : 0;
+  a.part = c->sample_part; a.counters = c->sample_counters;
+  a.conf = conf; a.token = token; a.lse = lse;
+  a.status = c->d_status;
+  c->last_launches = 0;
+  CU_TRY(c, sample_rows(a, (cudaStream_t)stream));
+  c->last_launches++;
+  return LACACHE_OK;
+}
 
 lacache_status lacache_set_step_overlap(lacache_ctx* c, int enable) {
   if (!c) return LACACHE_ERR_INVALID_ARG;

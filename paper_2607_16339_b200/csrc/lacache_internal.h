@@ -52,6 +52,7 @@ enum StatusLoc : int32_t {
   LOC_WAIT_S = 5,
   LOC_WAIT_O = 6,
   LOC_UNIT_TABLE = 7,
+  LOC_SAMPLE_ROW = 8,
 };
 
 struct Geometry {
@@ -127,6 +128,18 @@ struct AttnArgs {
   float* part_m; float* part_l; float* part_o; int* counters; int max_chunks;
   int32_t* status;
 };
+
+struct SampleArgs {
+  const void* logits; int dtype;   // [n_tokens, vocab], bf16 or fp32
+  int n_tokens, vocab;
+  const int32_t* rows; int n_rows; // the rows to sample (device)
+  int splits, slice;               // CTAs per row and vocabulary entries per CTA (splits * slice >= vocab)
+  int vector_ok;                   // rows start on 16-byte boundaries and `slice` is a multiple of the vector width
+  float* part; int* counters;      // [n_rows][splits][4] partial results, [n_rows] arrival counters (zero between launches)
+  float* conf; int32_t* token; float* lse;   // [n_rows]; lse may be null
+  int32_t* status;
+};
+cudaError_t sample_rows(const SampleArgs& a, cudaStream_t s);
 
 struct ExportArgs {
   RotBuffers rot; StateBuffers st;

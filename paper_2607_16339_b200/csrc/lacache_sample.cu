@@ -1,0 +1,132 @@
+// Sampling-stage truncation (Sec. 3.4, last paragraph): the float softmax over the vocabulary runs on
+// the rows of the current block only.  Per block row: the most probable token (lowest id among equal
+// logits), its probability and the log normaliser.  HBM-bound: every logit of the block's rows is read
+// once, nothing else of the [T, vocab] array is touched.
+//
+// A row is cut into `splits` slices of the vocabulary, one CTA each (a block has few rows: one CTA per
+// row would leave most SMs idle).  A CTA reduces its slice to (max, sum of exp relative to that max,
+// index of the first maximum) with one pass and one exponential per element; the last CTA of a row to
+// arrive (one counter per row, reset by that CTA) combines the slices in slice order, so the result
+// does not depend on the arrival order.
+#include <cuda_bf16.h>
+
+#include "lacache_internal.h"
+
+namespace lacache {
+namespace {
+
+constexpr int SAMPLE_THREADS = 256;
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2F = 0.69314718055994531f;
+
+struct Acc {
+  float m, s;   // running maximum; sum of 2^((x - m) log2 e) over the elements seen
+  int idx;      // index of the first element equal to m
+};
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void acc_add(Acc& a, float x, int i) {
+  if (x > a.m) {   // (strict: an equal logit further on does not move the index)
+    a.s = a.s * ex2f((a.m - x) * LOG2E) + 1.f;
+    a.m = x;
+    a.idx = i;
+  } else if (x != -INFINITY) {   // (a masked vocabulary entry adds nothing, also before any finite logit)
+    a.s += ex2f((x - a.m) * LOG2E);
+  }
+}
+// a and b cover disjoint index ranges
+__device__ __forceinline__ Acc acc_merge(const Acc& a, const Acc& b) {
+  Acc r;
+  if (b.m > a.m || (b.m == a.m && b.idx < a.idx)) {
+    r.m = b.m; r.idx = b.idx;
+  } else {
+    r.m = a.m; r.idx = a.idx;
+  }
+  const float sa = a.m == -INFINITY ? 0.f : a.s * ex2f((a.m - r.m) * LOG2E);
+  const float sb = b.m == -INFINITY ? 0.f : b.s * ex2f((b.m - r.m) * LOG2E);
+  r.s = sa + sb;
+  return r;
+}
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <class T>
+__global__ void __launch_bounds__(SAMPLE_THREADS) sample_rows_kernel(SampleArgs a) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  const int r = blockIdx.y, sp = blockIdx.x;
+  const int row = a.rows[r];
+  __shared__ Acc warp_acc[SAMPLE_THREADS / 32];
+  const bool bad = row < 0 || row >= a.n_tokens;
+  Acc acc{-INFINITY, 0.f, 0x7fffffff};
+  if (!bad) {
+    const T* x = reinterpret_cast<const T*>(a.logits) + (size_t)row * a.vocab;
+    const int lo = sp * a.slice, hi = min(lo + a.slice, a.vocab);
+    if (a.vector_ok) {   // rows start on 16-byte boundaries and the slice is a multiple of the vector width
+      const int hi_v = lo + (max(hi - lo, 0) / VEC) * VEC;
+      for (int i = lo + threadIdx.x * VEC; i < hi_v; i += SAMPLE_THREADS * VEC) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(x + i);
+        const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) acc_add(acc, to_float(e[j]), i + j);
+      }
+      for (int i = hi_v + threadIdx.x; i < hi; i += SAMPLE_THREADS) acc_add(acc, to_float(x[i]), i);
+    } else {
+      for (int i = lo + threadIdx.x; i < hi; i += SAMPLE_THREADS) acc_add(acc, to_float(x[i]), i);
+    }
+  }
+  // CTA reduction
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    Acc b;
+    b.m = __shfl_xor_sync(0xffffffffu, acc.m, o);
+    b.s = __shfl_xor_sync(0xffffffffu, acc.s, o);
+    b.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
+    acc = acc_merge(acc, b);
+  }
+  if ((threadIdx.x & 31) == 0) warp_acc[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    Acc t = warp_acc[0];
+    for (int w = 1; w < SAMPLE_THREADS / 32; ++w) t = acc_merge(t, warp_acc[w]);
+    float* p = a.part + ((size_t)r * a.splits + sp) * 4;
+    p[0] = t.m; p[1] = t.s; p[2] = __int_as_float(t.idx);
+    __threadfence();
+    const int old = atomicAdd(a.counters + r, 1);
+    if (old == a.splits - 1) {
+      a.counters[r] = 0;
+      __threadfence();   // the other slices' partial results are visible from here on
+      const volatile float* q = a.part + (size_t)r * a.splits * 4;
+      Acc all{-INFINITY, 0.f, 0x7fffffff};
+      for (int s2 = 0; s2 < a.splits; ++s2) {   // slice order: independent of who arrived when
+        Acc b{q[4 * s2], q[4 * s2 + 1], __float_as_int(q[4 * s2 + 2])};
+        all = acc_merge(all, b);
+      }
+      if (bad) {
+        a.token[r] = -1; a.conf[r] = 0.f;
+        if (a.lse) a.lse[r] = 0.f;
+        if (atomicCAS(a.status, 0, (int)LACACHE_ERR_INVALID_ARG) == 0) { a.status[1] = LOC_SAMPLE_ROW; a.status[2] = r; a.status[3] = row; }
+      } else {
+        a.token[r] = all.idx;
+        a.conf[r] = 1.f / all.s;                       // exp(x_max - x_max) / sum
+        if (a.lse) a.lse[r] = all.m + log2f(all.s) * LN2F;
+      }
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t sample_rows(const SampleArgs& a, cudaStream_t s) {
+  if (a.n_rows == 0) return cudaSuccess;
+  dim3 grid(a.splits, a.n_rows);
+  if (a.dtype == LACACHE_DTYPE_BF16) sample_rows_kernel<__nv_bfloat16><<<grid, SAMPLE_THREADS, 0, s>>>(a);
+  else sample_rows_kernel<float><<<grid, SAMPLE_THREADS, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace lacache
