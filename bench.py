@@ -424,12 +424,64 @@ def run_cuda(args):
         if (world == 1 and not args.no_token_path and wl.dtype == "bf16" and wl.n_q_heads in D_MODEL
                 and wl.total_tokens <= 65536):     # (its replicas of the all-token scratch would not fit beyond that)
             line["token_path"] = token_path_leg(wl, dev, peaks, args.seed, min(K, 512))
+        if world == 1 and not args.no_sampler and wl.n_q_heads in VOCAB and wl.total_tokens * VOCAB[wl.n_q_heads] * 2 <= 8e9:
+            line["sampler"] = sampler_leg(wl, dev, peaks, args.seed)
         if world == 1 and not args.no_incremental and wl.dtype == "bf16" and wl.head_dim == 128 and wl.n_blocks >= 2:
             line["incremental"] = incremental_leg(wl, dev, args.seed, R)
         print(json.dumps(line), flush=True)
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------
+# sampling-stage truncation: softmax over the vocabulary on the current block's rows only
+# ----------------------------------------------------------------------------
+VOCAB = {32: 126464, 28: 152064}     # vocabulary of the model a workload is shaped like, by query heads
+
+
+def sampler_leg(wl, dev, peaks, seed):
+    """Device time of lacache_sample_block on bf16 logits [T, vocab] (synthetic, N(0, 3)): every call
+    preceded by a 256 MiB write so that the block's rows come from HBM, each call bracketed by its own
+    events; the median.  Algorithmic bytes = block rows x vocab x 2."""
+    import torch
+    from paper_2607_16339_b200 import binding
+    from paper_2607_16339_b200.workloads import DeviceSchedule
+    mk = lambda: torch.cuda.Event(enable_timing=True)
+    V, T, n = VOCAB[wl.n_q_heads], wl.total_tokens, wl.batch * wl.block_len
+    g = torch.Generator(device=dev).manual_seed(seed + 5)
+    logits = torch.empty(T, V, device=dev, dtype=torch.bfloat16)
+    for lo in range(0, T, 1024):      # (in pieces: the fp32 draw of all rows at once would be twice the array)
+        logits[lo:lo + 1024] = (torch.randn(min(1024, T - lo), V, generator=g, device=dev) * 3).to(torch.bfloat16)
+    sched = DeviceSchedule(wl, seed + 6, dev, 1)
+    ctx = binding.Context.from_workload(wl)
+    ctx.build(0, *sched.full[0])
+    conf = torch.empty(n, device=dev); tok = torch.empty(n, device=dev, dtype=torch.int32); lse = torch.empty(n, device=dev)
+    flush = torch.empty(256 << 20, device=dev, dtype=torch.int8)
+    times = []
+    for i in range(3 + 21):
+        flush.add_(1)
+        e = (mk(), mk())
+        e[0].record()
+        ctx.sample_block(logits, conf, tok, lse)
+        e[1].record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            times.append(e[0].elapsed_time(e[1]) * 1e3)
+    st, msg = ctx.poll_status()
+    if st != 0:
+        raise SystemExit("bench.py: device status %d in the sampler leg: %s" % (st, msg))
+    ctx.destroy()
+    us = sorted(times)[len(times) // 2]
+    nbytes = n * V * 2
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"what": "lacache_sample_block: softmax over the vocabulary on the current block's rows only (token, "
+                    "probability, log normaliser), bf16 logits, flushed L2",
+            "rows": n, "of_rows": T, "vocab": V, "launch_us": round(us, 2),
+            "roofline": {"kernel": "sample_rows_kernel", "bound": "hbm", "achieved": round(gbs, 1),
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(gbs / peaks["hbm_gbs"], 4),
+                         "peak_source": peaks["source"], "traffic": None, "avg_launch_us": round(us, 2),
+                         "algorithmic_bytes_per_launch": nbytes}}
 
 
 # ----------------------------------------------------------------------------
@@ -683,6 +735,7 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-token-path", action="store_true", help="skip the extra leg that feeds steps from token ids")
+    ap.add_argument("--no-sampler", action="store_true", help="skip the extra leg that times the sampling-stage truncation")
     ap.add_argument("--no-incremental", action="store_true",
                     help="skip the extra leg that compares rebuilding the cache per block with advancing it")
     ap.add_argument("--replicas", type=int, default=0, help="cache-state replicas visited round-robin (0 = sized from the L2)")

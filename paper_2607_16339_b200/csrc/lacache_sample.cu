@@ -68,7 +68,22 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) sample_rows_kernel(SampleArgs 
     const int lo = sp * a.slice, hi = min(lo + a.slice, a.vocab);
     if (a.vector_ok) {   // rows start on 16-byte boundaries and the slice is a multiple of the vector width
       const int hi_v = lo + (max(hi - lo, 0) / VEC) * VEC;
-      for (int i = lo + threadIdx.x * VEC; i < hi_v; i += SAMPLE_THREADS * VEC) {
+      // four independent 16-byte loads in flight per thread before any of them is used (the reduction
+      // below them is one dependent chain, which would otherwise serialise the loads' latencies)
+      constexpr int STEP = SAMPLE_THREADS * VEC;
+      int i = lo + threadIdx.x * VEC;
+      for (; i + 3 * STEP < hi_v; i += 4 * STEP) {
+        uint4 raw[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) raw[u] = *reinterpret_cast<const uint4*>(x + i + u * STEP);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const T* e = reinterpret_cast<const T*>(&raw[u]);
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) acc_add(acc, to_float(e[j]), i + u * STEP + j);
+        }
+      }
+      for (; i < hi_v; i += STEP) {
         const uint4 raw = *reinterpret_cast<const uint4*>(x + i);
         const T* e = reinterpret_cast<const T*>(&raw);
 #pragma unroll
@@ -90,6 +105,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) sample_rows_kernel(SampleArgs 
   }
   if ((threadIdx.x & 31) == 0) warp_acc[threadIdx.x >> 5] = acc;
   __syncthreads();
+  __shared__ int is_last;
   if (threadIdx.x == 0) {
     Acc t = warp_acc[0];
     for (int w = 1; w < SAMPLE_THREADS / 32; ++w) t = acc_merge(t, warp_acc[w]);
@@ -97,25 +113,39 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) sample_rows_kernel(SampleArgs 
     p[0] = t.m; p[1] = t.s; p[2] = __int_as_float(t.idx);
     __threadfence();
     const int old = atomicAdd(a.counters + r, 1);
-    if (old == a.splits - 1) {
+    is_last = old == a.splits - 1;
+    if (is_last) {
       a.counters[r] = 0;
       __threadfence();   // the other slices' partial results are visible from here on
-      const volatile float* q = a.part + (size_t)r * a.splits * 4;
-      Acc all{-INFINITY, 0.f, 0x7fffffff};
-      for (int s2 = 0; s2 < a.splits; ++s2) {   // slice order: independent of who arrived when
-        Acc b{q[4 * s2], q[4 * s2 + 1], __float_as_int(q[4 * s2 + 2])};
-        all = acc_merge(all, b);
-      }
-      if (bad) {
-        a.token[r] = -1; a.conf[r] = 0.f;
-        if (a.lse) a.lse[r] = 0.f;
-        if (atomicCAS(a.status, 0, (int)LACACHE_ERR_INVALID_ARG) == 0) { a.status[1] = LOC_SAMPLE_ROW; a.status[2] = r; a.status[3] = row; }
-      } else {
-        a.token[r] = all.idx;
-        a.conf[r] = 1.f / all.s;                       // exp(x_max - x_max) / sum
-        if (a.lse) a.lse[r] = all.m + log2f(all.s) * LN2F;
-      }
     }
+  }
+  __syncthreads();
+  if (!is_last || threadIdx.x >= 32) return;
+  // The last CTA of the row to arrive: its first warp combines the slices, lane l slices l and l + 32,
+  // then a fixed shuffle tree -- the result does not depend on who arrived when.
+  const float* q = a.part + (size_t)r * a.splits * 4;
+  Acc all{-INFINITY, 0.f, 0x7fffffff};
+  for (int s2 = threadIdx.x; s2 < a.splits; s2 += 32) {
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(q + 4 * s2));
+    all = acc_merge(all, Acc{v.x, v.y, __float_as_int(v.z)});
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    Acc b;
+    b.m = __shfl_xor_sync(0xffffffffu, all.m, o);
+    b.s = __shfl_xor_sync(0xffffffffu, all.s, o);
+    b.idx = __shfl_xor_sync(0xffffffffu, all.idx, o);
+    all = acc_merge(all, b);
+  }
+  if (threadIdx.x != 0) return;
+  if (bad) {
+    a.token[r] = -1; a.conf[r] = 0.f;
+    if (a.lse) a.lse[r] = 0.f;
+    if (atomicCAS(a.status, 0, (int)LACACHE_ERR_INVALID_ARG) == 0) { a.status[1] = LOC_SAMPLE_ROW; a.status[2] = r; a.status[3] = row; }
+  } else {
+    a.token[r] = all.idx;
+    a.conf[r] = 1.f / all.s;                       // exp(x_max - x_max) / sum
+    if (a.lse) a.lse[r] = all.m + log2f(all.s) * LN2F;
   }
 }
 
