@@ -966,9 +966,9 @@ lacache_status lacache_sample_block(lacache_ctx* c, const void* logits, int dtyp
   a.n_tokens = c->g.T; a.vocab = vocab;
   a.rows = c->d_blk_tok + (size_t)c->built_block * n;
   a.n_rows = n;
-  // enough CTAs for eight per SM (a CTA is 256 threads with a few loads in flight each: HBM latency
-  // is hidden by many resident CTAs), each with at least 2048 entries, slices a multiple of 8 entries
-  int splits = std::max(1, std::min(MAX_SPLITS, (8 * c->num_sms + n - 1) / n));
+  // as many CTAs as are resident at once (four per SM), each with at least 2048 entries, slices a
+  // multiple of 8 entries (rounded down: no second wave of a few stragglers)
+  int splits = std::max(1, std::min(MAX_SPLITS, 4 * c->num_sms / n));
   splits = std::min(splits, std::max(1, vocab / 2048));
   int slice = ((vocab + splits - 1) / splits + 7) / 8 * 8;
   splits = (vocab + slice - 1) / slice;

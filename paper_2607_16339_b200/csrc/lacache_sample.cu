@@ -52,11 +52,34 @@ __device__ __forceinline__ Acc acc_merge(const Acc& a, const Acc& b) {
   return r;
 }
 
+// NV vectors of VEC elements each (vector u starts at index i0 + u * step) added without a per-element
+// branch or rescale: maximum and its first index (compare + selects), one rescale of the sum, then one
+// exponential per element.
+template <int NV, int VEC>
+__device__ __forceinline__ void batch_add(Acc& acc, const float (&f)[NV * VEC], int i0, int step) {
+  float best = acc.m;
+  int bidx = acc.idx;
+#pragma unroll
+  for (int u = 0; u < NV; ++u) {
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+      const bool up = f[u * VEC + j] > best;   // (strict: an equal logit further on does not move the index)
+      best = up ? f[u * VEC + j] : best;
+      bidx = up ? i0 + u * step + j : bidx;
+    }
+  }
+  const float m_use = best == -INFINITY ? 0.f : best;   // (only -inf so far: every term below is 0)
+  float sum = acc.m == -INFINITY ? 0.f : acc.s * ex2f((acc.m - m_use) * LOG2E);
+#pragma unroll
+  for (int k = 0; k < NV * VEC; ++k) sum += ex2f((f[k] - m_use) * LOG2E);
+  acc.m = best; acc.idx = bidx; acc.s = sum;
+}
+
 __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
 
 template <class T>
-__global__ void __launch_bounds__(SAMPLE_THREADS) sample_rows_kernel(SampleArgs a) {
+__global__ void __launch_bounds__(SAMPLE_THREADS, 4) sample_rows_kernel(SampleArgs a) {
   constexpr int VEC = 16 / (int)sizeof(T);
   const int r = blockIdx.y, sp = blockIdx.x;
   const int row = a.rows[r];
@@ -68,8 +91,10 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) sample_rows_kernel(SampleArgs 
     const int lo = sp * a.slice, hi = min(lo + a.slice, a.vocab);
     if (a.vector_ok) {   // rows start on 16-byte boundaries and the slice is a multiple of the vector width
       const int hi_v = lo + (max(hi - lo, 0) / VEC) * VEC;
-      // four independent 16-byte loads in flight per thread before any of them is used (the reduction
-      // below them is one dependent chain, which would otherwise serialise the loads' latencies)
+      // Four independent 16-byte loads in flight per thread, then two batches of two vectors each
+      // (batch_add: the lanes of a warp move their running maxima at different elements, so a
+      // per-element branch would run both of its sides -- two exponentials, and the exponential
+      // unit is what bounds this kernel -- nearly every time).
       constexpr int STEP = SAMPLE_THREADS * VEC;
       int i = lo + threadIdx.x * VEC;
       for (; i + 3 * STEP < hi_v; i += 4 * STEP) {
@@ -77,17 +102,24 @@ __global__ void __launch_bounds__(SAMPLE_THREADS) sample_rows_kernel(SampleArgs 
 #pragma unroll
         for (int u = 0; u < 4; ++u) raw[u] = *reinterpret_cast<const uint4*>(x + i + u * STEP);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const T* e = reinterpret_cast<const T*>(&raw[u]);
+        for (int h = 0; h < 2; ++h) {
+          float f[2 * VEC];
 #pragma unroll
-          for (int j = 0; j < VEC; ++j) acc_add(acc, to_float(e[j]), i + u * STEP + j);
+          for (int u = 0; u < 2; ++u) {
+            const T* e = reinterpret_cast<const T*>(&raw[2 * h + u]);
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) f[u * VEC + j] = to_float(e[j]);
+          }
+          batch_add<2, VEC>(acc, f, i + 2 * h * STEP, STEP);
         }
       }
       for (; i < hi_v; i += STEP) {
         const uint4 raw = *reinterpret_cast<const uint4*>(x + i);
         const T* e = reinterpret_cast<const T*>(&raw);
+        float f[VEC];
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) acc_add(acc, to_float(e[j]), i + j);
+        for (int j = 0; j < VEC; ++j) f[j] = to_float(e[j]);
+        batch_add<1, VEC>(acc, f, i, STEP);
       }
       for (int i = hi_v + threadIdx.x; i < hi; i += SAMPLE_THREADS) acc_add(acc, to_float(x[i]), i);
     } else {
