@@ -438,7 +438,7 @@ def run_cuda(args):
 # sampling-stage truncation: softmax over the vocabulary on the current block's rows only
 # ----------------------------------------------------------------------------
 VOCAB = {32: 126464, 28: 152064}     # vocabulary of the model a workload is shaped like, by query heads
-SAMPLER_TRAFFIC_PER_LAUNCH = {4: 65654016}   # ncu, profiles/sample_rows_kernel_cfg4_ncu_full.txt (read + write)
+SAMPLER_TRAFFIC_PER_LAUNCH = {4: 66288640}   # ncu, profiles/sample_rows_kernel_cfg4_ncu_full.txt (read + write)
 
 
 def sampler_leg(wl, dev, peaks, seed):
