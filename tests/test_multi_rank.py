@@ -62,6 +62,7 @@ def test_single_process_helpers_are_identity():
     bench.barrier()
     from paper_2607_16339_b200.workloads import WORKLOADS
     c = bench.flops_and_bytes(WORKLOADS[2])
-    # step 0.789 GFLOP, build 8.88 GFLOP at the LLaDA-8B shape
+    # hand count at the LLaDA-8B shape (N = 768, L_b = 32, 32 heads x 128): a step is 4 d Hq L_b (2N - L_b)
+    # = 0.789 GFLOP, a build 4 d Hq (N - L_b)^2 = 8.88 GFLOP
     assert abs(c["step_flops"] / 1e9 - 0.789) < 0.002 and abs(c["build_flops"] / 1e9 - 8.88) < 0.01
     assert abs(c["step_bytes"] / 1e6 - 45.0) < 0.5
