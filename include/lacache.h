@@ -85,8 +85,10 @@ int lacache_version(void);
  * position), builds the RoPE cos/sin table in double precision (Eq. 1) and
  * allocates every cache: rotated Q/K/V (RoPECache), (m, l, O~) (FACache;
  * RowMaxcache / RowSumcache / Ocache of Algorithm 1) and scratch.  This is the
- * only call that allocates device memory (the *_host calls allocate staging
- * on first use).  Uses the current CUDA device.  On failure *out is NULL.
+ * only call that allocates device memory, with three documented exceptions
+ * that allocate once, on their first use: the *_host calls (staging),
+ * lacache_build_incremental (the prefix state) and lacache_sample_block (a
+ * small scratch).  Uses the current CUDA device.  On failure *out is NULL.
  */
 lacache_status lacache_create(const lacache_config* cfg, lacache_ctx** out);
 
