@@ -957,6 +957,7 @@ lacache_status lacache_sample_block(lacache_ctx* c, const void* logits, int dtyp
   if (vocab <= 0) return fail(c, LACACHE_ERR_INVALID_ARG, "vocab %d", vocab);
   constexpr int MAX_SPLITS = 64;
   const int n = c->g.B * c->g.block_len;
+  if (n > 65535) return fail(c, LACACHE_ERR_UNSUPPORTED, "%d block rows: the sampler's grid takes at most 65535", n);
   if (!c->sample_part) {
     CU_TRY(c, dev_alloc(c, &c->sample_part, (size_t)n * MAX_SPLITS * 4));
     CU_TRY(c, dev_alloc(c, &c->sample_counters, (size_t)n, true));
