@@ -181,6 +181,112 @@ def n_replicas(step_bytes):
     return max(3, math.ceil(2.0 * L2_BYTES / max(step_bytes, 1)) + 1)
 
 
+def replica_phases(K, R, S):
+    """Step-in-block index of every replica's first timed call, chosen so that K calls visiting the R
+    replicas round-robin contain round(K / S) builds (at least one once K >= 8): a build falls due when a
+    replica reaches step 0 of a block.  Returns (phases, builds the K calls will contain)."""
+    n = [(K - c + R - 1) // R if c < K else 0 for c in range(R)]
+    builds = lambda p, m: sum(1 for q in range(m) if (p + q) % S == 0)
+    target = round(K / S)
+    if K >= 8:
+        target = max(1, target)
+    base = sum(m // S for m in n)
+    cand = [c for c in range(R) if n[c] > 0 and n[c] % S != 0]
+    extra = max(0, min(len(cand), target - base))
+    chosen = set(cand[int((j + 0.5) * len(cand) / extra)] for j in range(extra)) if extra else set()
+    phases = []
+    for c in range(R):
+        m = n[c]
+        want = m // S + (1 if c in chosen else 0)
+        if m >= S:
+            pref = (c * max(1, S // R)) % S              # long runs: block boundaries staggered over the replicas
+        else:
+            pref = (S - m // 2) % S if c in chosen else 1  # the one build in the middle of the replica's calls
+        ok = [p for p in range(S) if builds(p, m) == want] or list(range(S))
+        phases.append(min(ok, key=lambda p: min((p - pref) % S, (pref - p) % S)))
+    return phases, sum(builds(p, m) for p, m in zip(phases, n))
+
+
+class RoundRobin:
+    """K calls over R cache states visited round-robin, every replica walking its own block schedule:
+    a step per call, preceded by the block's build whenever the replica enters a new block."""
+
+    def __init__(self, ctxs, outs, sched, K, S):
+        self.ctxs, self.outs, self.sched, self.K, self.S = ctxs, outs, sched, K, S
+        self.R = len(ctxs)
+        self.phases, self.n_builds = replica_phases(K, self.R, S)
+        self.total = sched.n_blocks_used * S
+        self.local = [0] * self.R
+
+    def prepare(self):
+        """Untimed: every replica gets the cache of the block in which the step BEFORE its first timed call
+        lies, and runs that step (so each replica has stepped at least once, and a replica whose phase is 0
+        meets its build inside the timed region)."""
+        for c in range(self.R):
+            first = ((c % self.sched.n_blocks_used) * self.S + self.phases[c]) % self.total
+            prev = (first - 1) % self.total
+            blk, _, tens = self.sched.step_inputs(prev)
+            self.ctxs[c].build(blk, *self.sched.full[blk])
+            self.ctxs[c].step(*tens, *self.outs[c])
+            self.local[c] = first
+
+    def run(self, n_calls=None, on_call=None):
+        """The calls themselves.  Returns (kernel launches, builds)."""
+        launches = builds = 0
+        for j in range(self.K if n_calls is None else n_calls):
+            c = j % self.R
+            blk, s, tens = self.sched.step_inputs(self.local[c])
+            ctx = self.ctxs[c]
+            if s == 0:
+                if on_call:
+                    on_call("build", ctx)
+                ctx.build(blk, *self.sched.full[blk])
+                launches += ctx.last_launch_count
+                builds += 1
+                if on_call:
+                    on_call("built", ctx)
+            if on_call:
+                on_call("step", ctx)
+            ctx.step(*tens, *self.outs[c])
+            launches += ctx.last_launch_count
+            if on_call:
+                on_call("stepped", ctx)
+            self.local[c] = (self.local[c] + 1) % self.total
+        return launches, builds
+
+
+def timed_region(rr, W, min_ms=50.0, max_repeats=200):
+    """W untimed warm-up calls, then the K-call region `repeats` times, each bracketed by one event pair
+    (barrier + synchronize on both sides) after an untimed pass that puts every replica at its phase.
+    Returns (per-repeat ms, launches per repeat, builds per repeat, wall seconds of the timed regions)."""
+    import math
+    import torch
+    mk = lambda: torch.cuda.Event(enable_timing=True)
+    rr.prepare()
+    rr.run(W)
+    torch.cuda.synchronize()
+    times, wall = [], 0.0
+    launches = builds = 0
+    repeats = 1
+    i = 0
+    while i < repeats:
+        rr.prepare()
+        torch.cuda.synchronize(); barrier()
+        t0 = time.perf_counter()
+        e0, e1 = mk(), mk()
+        e0.record()
+        launches, builds = rr.run()
+        e1.record()
+        torch.cuda.synchronize(); barrier()
+        wall += time.perf_counter() - t0
+        times.append(e0.elapsed_time(e1))
+        if i == 0:   # size the number of repeats from the first one (the same on every rank: max over ranks)
+            t1 = reduce_max(times[0], torch.device("cuda", torch.cuda.current_device()))
+            repeats = 1 if t1 >= 4 * min_ms else max(3, min(max_repeats, math.ceil(min_ms / max(t1, 1e-3))))
+        i += 1
+    return times, launches, builds, wall
+
+
 def run_cuda(args):
     import torch
     from paper_2607_16339_b200 import binding
@@ -200,92 +306,128 @@ def run_cuda(args):
     counts = flops_and_bytes(wl)
     peaks = load_peaks()
     T = wl.total_tokens
-    stream = torch.cuda.current_stream()
     mk = lambda: torch.cuda.Event(enable_timing=True)
+    precision = binding.PRECISION_SPLIT if args.precision_mode < 0 else args.precision_mode
+    out_bf16 = args.out_dtype == "bf16"
+    ctx_kw = dict(precision_mode=precision, out_dtype=binding.OUT_BF16 if out_bf16 else binding.OUT_FP32)
+    out_t = torch.bfloat16 if out_bf16 else torch.float32
 
     # ---- replicas: independent cache states of the same workload, visited round-robin ----
     # Every call then finds its inputs (cached state, rotated planes) in HBM, not in L2,
     # while the calls run back to back as they do in a denoising loop.
     R = args.replicas or n_replicas(counts["step_attn_bytes"])
-    stagger = max(1, S // R)                       # replica c starts c * stagger steps into its block
-    nk = min(K, 256)                               # calls of the per-kernel timing pass
-    local_steps = (R - 1) * stagger + (W + K + nk + R - 1) // R + 1
-    sched = DeviceSchedule(wl, rank_seed(args.seed, rank), dev, local_steps)
-    ctxs = [binding.Context.from_workload(wl) for _ in range(R)]
-    outs = [(torch.empty(T, wl.n_q_heads, wl.head_dim, device=dev), torch.empty(T, wl.n_q_heads, device=dev))
+    sched = DeviceSchedule(wl, rank_seed(args.seed, rank), dev, min(wl.n_steps, 3 * S))
+
+    def make_replicas(**kw):
+        cs = [binding.Context.from_workload(wl, **dict(ctx_kw, **kw)) for _ in range(R)]
+        for c in cs:
+            c.set_step_overlap(True)     # the step inputs are all resident before the first call
+        return cs
+
+    ctxs = make_replicas()
+    outs = [(torch.empty(T, wl.n_q_heads, wl.head_dim, device=dev, dtype=out_t), torch.empty(T, wl.n_q_heads, device=dev))
             for _ in range(R)]
     ctx = ctxs[0]
-
-    def call_of(i):
-        """Global call i -> (replica, block, step in block, block inputs)."""
-        c = i % R
-        blk, s, tens = sched.step_inputs(c * stagger + i // R)
-        return c, blk, s, tens
-
-    for c in range(R):   # every replica starts with a valid cache for the block it is in
-        blk = sched.step_inputs(c * stagger)[0]
-        ctxs[c].build(blk, *sched.full[blk])
-    torch.cuda.synchronize()
-
-    launches = 0
-    n_builds = 0
-
-    def run_range(lo, hi, timed, events=None):
-        nonlocal launches, n_builds
-        for i in range(lo, hi):
-            c, blk, s, (qb, kb, vb) = call_of(i)
-            if s == 0 and i >= R:      # a replica's very first call had its build above
-                if events is not None:
-                    e = (mk(), mk()); e[0].record(); e[1].record()
-                    ctxs[c].set_timing_events(*e); events.append(("build", e))
-                ctxs[c].build(blk, *sched.full[blk])
-                if timed:
-                    launches += ctxs[c].last_launch_count; n_builds += 1
-            if events is not None:
-                e = (mk(), mk()); e[0].record(); e[1].record()
-                ctxs[c].set_timing_events(*e); events.append(("step", e))
-            ctxs[c].step(qb, kb, vb, *outs[c])
-            if timed:
-                launches += ctxs[c].last_launch_count
+    tc = ctx.engine == binding.ENGINE_TCGEN05
 
     clocks = ClockSampler(local_rank)
     clocks.start()
     time.sleep(0.05)   # let the sampler come up
-    # ---- headline: K calls back to back, builds included, one event pair around the region ----
-    run_range(0, W, False)
-    torch.cuda.synchronize(); barrier()
+    # ---- headline: K calls back to back, builds pro rata, one event pair around each repeat ----
+    rr = RoundRobin(ctxs, outs, sched, K, S)
     clocks.mark()
-    t_wall0 = time.perf_counter()
-    ev0, ev1 = mk(), mk()
-    ev0.record()
-    run_range(W, W + K, True)
-    ev1.record()
-    torch.cuda.synchronize(); barrier()
-    t_wall = time.perf_counter() - t_wall0
-    total_ms = ev0.elapsed_time(ev1)
+    times, launches, n_builds, t_wall = timed_region(rr, W)
+    total_ms = statistics.median(times)
 
     # ---- per-kernel durations of the attention kernels: the same calls again, with an event
     # pair recorded inside the library around each attention kernel (no host sync in between) ----
     events = []
-    run_range(W + K, W + K + nk, False, events)
+
+    def with_events(kind, c):
+        if kind in ("build", "step"):
+            e = (mk(), mk()); e[0].record(); e[1].record()
+            c.set_timing_events(*e); events.append((kind, e))
+
+    rrk = RoundRobin(ctxs, outs, sched, max(min(K, 256), S * R // 4), S)
+    rrk.prepare()
+    rrk.run(on_call=with_events)
     torch.cuda.synchronize()
-    for c in range(R):
-        ctxs[c].set_timing_events(None, None)
+    for c in ctxs:
+        c.set_timing_events(None, None)
     kern_step_ms = [a.elapsed_time(b) for kind, (a, b) in events if kind == "step"]
     kern_build_ms = [a.elapsed_time(b) for kind, (a, b) in events if kind == "build"]
     if not kern_build_ms:     # no block boundary in the range: time one build on its own
         e = (mk(), mk()); e[0].record(); e[1].record()
-        c, blk, s, _ = call_of(W + K + nk)
-        ctxs[c].set_timing_events(*e)
-        ctxs[c].build(blk, *sched.full[blk]); torch.cuda.synchronize()
-        ctxs[c].set_timing_events(None, None)
+        ctx.set_timing_events(*e)
+        ctx.build(0, *sched.full[0]); torch.cuda.synchronize()
+        ctx.set_timing_events(None, None)
         kern_build_ms.append(e[0].elapsed_time(e[1]))
+
+    # ---- the same calls once more, back to back and overlapping as in the headline, with every launch of
+    # the attention kernel stamping the GPU's global timer at its first CTA's entry and last CTA's exit ----
+    span = None
+    if tc:
+        n_slots = 4 * (rrk.K // R + 2) + 8
+        rings = [torch.empty(n_slots, 2, dtype=torch.int64, device=dev) for _ in range(R)]
+        for r_ in rings:
+            r_[:, 0] = -1       # UINT64_MAX
+            r_[:, 1] = 0
+        kinds = [[] for _ in range(R)]
+        idx = {id(c): i for i, c in enumerate(ctxs)}
+
+        def note(kind, c):
+            if kind in ("built", "stepped"):
+                kinds[idx[id(c)]] += [kind] * (c.last_launch_count - 1)     # (one RoPE launch per call)
+
+        rrk.prepare()
+        torch.cuda.synchronize()
+        for c, r_ in zip(ctxs, rings):
+            c.set_span_ring(r_)
+        rrk.run(on_call=note)
+        torch.cuda.synchronize()
+        for c in ctxs:
+            c.set_span_ring(None)
+        sp = {"stepped": [], "built": []}
+        for r_, ks in zip(rings, kinds):
+            h = r_.cpu().numpy()
+            for slot, kind in enumerate(ks[:n_slots]):
+                sp[kind].append(float(h[slot, 1] - h[slot, 0]) * 1e-3)     # ns -> us
+        if sp["stepped"]:
+            span = {"step_us": round(statistics.mean(sp["stepped"]), 2),
+                    "step_us_median": round(statistics.median(sp["stepped"]), 2),
+                    "build_us": round(statistics.mean(sp["built"]), 2) if sp["built"] else None,
+                    "launches": len(sp["stepped"]),
+                    "how": "first CTA entry to last CTA exit of the attention kernel's launches (global timer, "
+                           "stamped by the kernel), calls back to back and overlapping as in the headline"}
+
+    # ---- GPU full recompute of the same step (the vanilla pass the method replaces), same round-robin ----
+    n_fr = max(2 * R, 16)
+    fulls = [sched.full[c % sched.n_blocks_used] for c in range(R)]
+    for c in range(R):
+        ctxs[c].full_recompute(*fulls[c], *outs[c])
+    torch.cuda.synchronize(); barrier()
+    e0, e1 = mk(), mk()
+    e0.record()
+    for i in range(n_fr):
+        ctxs[i % R].full_recompute(*fulls[i % R], *outs[i % R])
+    e1.record()
+    torch.cuda.synchronize()
+    fr_ms = e0.elapsed_time(e1) / n_fr
+    fr_pairs = []
+    for i in range(min(n_fr, 16)):
+        e = (mk(), mk()); e[0].record(); e[1].record()
+        ctxs[i % R].set_timing_events(*e); fr_pairs.append(e)
+        ctxs[i % R].full_recompute(*fulls[i % R], *outs[i % R])
+    torch.cuda.synchronize()
+    for c in ctxs:
+        c.set_timing_events(None, None)
+    fr_kernel_ms = statistics.mean(a.elapsed_time(b) for a, b in fr_pairs)
+    full_flops = sum(4 * wl.head_dim * wl.n_q_heads * N * N for N in wl.seq_lens)
 
     # ---- for comparison: one replica, L2 flushed (256 MiB write) before every call, each call
     # bracketed by its own events (the launch latency after the flush kernel is inside) ----
     flush = torch.empty(256 << 20, dtype=torch.int8, device=dev)
-    blk0 = sched.step_inputs(0)[0]
-    ctx.build(blk0, *sched.full[blk0])
+    ctx.build(0, *sched.full[0])
     fl_pairs = []
     for i in range(8 + min(K, 64)):
         _, s, (qb, kb, vb) = sched.step_inputs(i % S)
@@ -297,7 +439,7 @@ def run_cuda(args):
     torch.cuda.synchronize()
     flush_step_ms = statistics.mean(a.elapsed_time(b) for a, b in fl_pairs)
     del flush
-    clocks.mark()      # window: the headline region, the per-kernel pass and the flushed pass (GPU busy throughout)
+    clocks.mark()      # window: the headline repeats, the per-kernel passes, the full recompute and the flushed pass
     clock_info = clocks.stop()
 
     # ---- warm L2: the same replica stepped K times from one CUDA-graph replay ----
@@ -323,7 +465,7 @@ def run_cuda(args):
     torch.cuda.synchronize()
 
     # ---- e2e: host buffers through the *_host entry points, copies inside the timed region ----
-    n_e2e = min(K, 2 * S)
+    n_e2e = max(8, min(K, 2 * S))
     pin = lambda t: t.cpu().pin_memory()
     h_full = {}
     h_steps = []
@@ -332,7 +474,7 @@ def run_cuda(args):
         if s == 0 and blk not in h_full:
             h_full[blk] = tuple(pin(t) for t in sched.full[blk])
         h_steps.append(tuple(pin(t) for t in tens))
-    out_h = torch.empty(T, wl.n_q_heads, wl.head_dim).pin_memory()
+    out_h = torch.empty(T, wl.n_q_heads, wl.head_dim, dtype=out_t).pin_memory()
     lse_h = torch.empty(T, wl.n_q_heads).pin_memory()
     ctx.build_host(0, *h_full[0])
     ctx.step_host(*h_steps[0], out_h, lse_h)     # allocates staging, warms the path
@@ -352,7 +494,7 @@ def run_cuda(args):
     blk_in = wl.batch * wl.block_len * (wl.n_q_heads + 2 * wl.n_kv_heads) * wl.head_dim * el
     full_in = T * (wl.n_q_heads + 2 * wl.n_kv_heads) * wl.head_dim * el
     h2d = blk_in + full_in * n_builds_e2e / max(n_e2e, 1)
-    d2h = T * wl.n_q_heads * wl.head_dim * 4 + T * wl.n_q_heads * 4
+    d2h = T * wl.n_q_heads * wl.head_dim * (2 if out_bf16 else 4) + T * wl.n_q_heads * 4
 
     for c in range(R):
         st, msg = ctxs[c].poll_status()
@@ -362,6 +504,7 @@ def run_cuda(args):
     # ---- reduce over ranks (timing only) ----
     total_ms = reduce_max(total_ms, dev)
     e2e_ms = reduce_max(e2e_ms, dev)
+    fr_ms = reduce_max(fr_ms, dev)
     if warm_ms is not None:
         warm_ms = reduce_max(warm_ms, dev)
     value = world * K / (total_ms * 1e-3)
@@ -374,8 +517,16 @@ def run_cuda(args):
         roof = {"kernel": "tc_attn_kernel (step: fixed rows x block keys + merge, block rows x all keys)",
                 "bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": round(ach / peaks["hbm_gbs"], 4), "peak_source": peaks["source"],
-                "traffic": TRAFFIC_PER_LAUNCH.get(wl.cfg), "avg_launch_us": round(step_k * 1e6, 2),
+                "traffic": TRAFFIC_PER_LAUNCH.get((wl.cfg, precision)), "avg_launch_us": round(step_k * 1e6, 2),
+                "how": "algorithmic bytes / mean duration of the launch between an event pair recorded inside "
+                       "the library (the pair keeps the launch from overlapping its neighbours and contains its "
+                       "launch latency)",
                 "algorithmic_bytes_per_launch": counts["step_attn_bytes"]}
+        if span:
+            a2 = counts["step_attn_bytes"] / (span["step_us"] * 1e-6) / 1e9
+            roof["overlapped"] = dict(span, achieved=round(a2, 1), frac=round(a2 / peaks["hbm_gbs"], 4),
+                                      step_period_us=round(total_ms / K * 1e3, 2))
+        fr_value = world * 1e3 / fr_ms
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": round(total_ms / K, 5), "higher_is_better": True, "scaling": "weak",
@@ -383,13 +534,28 @@ def run_cuda(args):
             "config": {"workload": "cfg%d %s" % (wl.cfg, wl.name), "batch": wl.batch, "prompt_lens": list(wl.prompt_lens),
                        "gen_len": wl.gen_len, "block_len": wl.block_len, "steps_per_block": S,
                        "heads": "%d/%d" % (wl.n_q_heads, wl.n_kv_heads), "head_dim": wl.head_dim,
-                       "builds_in_timed_region": n_builds,
+                       "precision_mode": precision, "out_dtype": "bf16" if out_bf16 else "f32",
                        "l2": "inputs larger than L2: %d replicas of the cache state visited round-robin "
                              "(%.0f MB of algorithmic traffic between two visits of a replica, L2 is 126 MB), "
-                             "calls back to back, no flush" % (R, (R - 1) * counts["step_attn_bytes"] / 1e6),
-                       "replicas": R,
-                       "out_dtype": "f32", "engine": "tcgen05" if ctx.engine == binding.ENGINE_TCGEN05 else "simt"},
+                             "calls back to back, no flush" % (R, (R - 1) * counts["step_attn_bytes"] / 1e6)},
+            "protocol": {"replicas": R, "builds_in_timed_region": n_builds, "repeats": len(times),
+                         "ms_per_repeat": {"median": round(total_ms, 4), "min": round(min(times), 4),
+                                           "max": round(max(times), 4)},
+                         "how": "each repeat: untimed pass that puts every replica at its place in its block "
+                                "schedule (a build and a step each), barrier + synchronize, K calls (a step each, "
+                                "preceded by the block's build where a replica enters a block: round(K / "
+                                "steps_per_block) builds) between one event pair, synchronize; value = K / median",
+                         "step_overlap": "on (inputs resident before the first call)",
+                         "engine": "tcgen05" if tc else "simt"},
             "tflops": round(total_flops / (total_ms * 1e-3) / 1e12, 2),
+            "full_recompute": {"value": round(fr_value, 1), "unit": UNIT, "step_us": round(fr_ms * 1e3, 2),
+                               "kernel_us": round(fr_kernel_ms * 1e3, 2),
+                               "tflops": round(full_flops / (fr_kernel_ms * 1e-3) / 1e12, 1),
+                               "tensor_frac": round(full_flops / (fr_kernel_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], 4),
+                               "calls": n_fr,
+                               "how": "lacache_full_recompute (every row x every key, no cache: the full pass the "
+                                      "method replaces) on the same replicas round-robin, calls back to back"},
+            "speedup_vs_full_recompute": round(value / fr_value, 3),
             "flushed_l2": {"value": round(world * 1e3 / flush_step_ms, 1), "unit": UNIT,
                            "step_us": round(flush_step_ms * 1e3, 2),
                            "how": "one replica, 256 MiB write before every call, each call bracketed by its own events"},
@@ -419,14 +585,32 @@ def run_cuda(args):
             line["cpu_baseline"] = cpu_baseline(wl, budget_s=12.0)
     for c in ctxs:
         c.destroy()
+    if rank == 0 and world == 1 and tc and not args.no_tile_granular and wl.total_tokens <= 65536:
+        # Algorithm 1 at tile granularity (less cached, more step work): the same protocol, its own contexts
+        tctxs = make_replicas(cache_granularity=binding.GRANULARITY_TILE)
+        trr = RoundRobin(tctxs, outs, sched, min(K, 256), S)
+        ttimes, _, tbuilds, _ = timed_region(trr, max(3, min(W, 8)), min_ms=20.0)
+        tms = statistics.median(ttimes)
+        for c in tctxs:
+            st, msg = c.poll_status()
+            if st != 0:
+                raise SystemExit("device status (tile-granular leg): %s" % msg)
+            c.destroy()
+        line["tile_granular"] = {"value": round(trr.K / (tms * 1e-3), 1), "unit": UNIT, "steps": trr.K,
+                                 "step_period_us": round(tms / trr.K * 1e3, 2), "builds_in_timed_region": tbuilds,
+                                 "repeats": len(ttimes), "vs_token_granular": round(trr.K / (tms * 1e-3) / value, 3),
+                                 "how": "cache_granularity = tile (state cached only for 128-row tiles and over 128-key "
+                                        "tiles that do not overlap the block; Algorithm 1's overlap predicates): same "
+                                        "round-robin protocol, same out / lse"}
     del outs, sched
     if rank == 0:
         if (world == 1 and not args.no_token_path and wl.dtype == "bf16" and wl.n_q_heads in D_MODEL
-                and wl.total_tokens <= 65536):     # (its replicas of the all-token scratch would not fit beyond that)
+                and wl.total_tokens <= 65536 and precision == binding.PRECISION_SPLIT and not out_bf16):
             line["token_path"] = token_path_leg(wl, dev, peaks, args.seed, min(K, 512))
         if world == 1 and not args.no_sampler and wl.n_q_heads in VOCAB and wl.total_tokens * VOCAB[wl.n_q_heads] * 2 <= 8e9:
             line["sampler"] = sampler_leg(wl, dev, peaks, args.seed)
-        if world == 1 and not args.no_incremental and wl.dtype == "bf16" and wl.head_dim == 128 and wl.n_blocks >= 2:
+        if (world == 1 and not args.no_incremental and wl.dtype == "bf16" and wl.head_dim == 128 and wl.n_blocks >= 2
+                and precision == binding.PRECISION_SPLIT and not out_bf16):
             line["incremental"] = incremental_leg(wl, dev, args.seed, R)
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -526,6 +710,8 @@ def incremental_leg(wl, dev, seed, R):
     S, nb, T = wl.steps_per_block, wl.n_blocks, wl.total_tokens
     sched = DeviceSchedule(wl, seed + 17, dev, nb * S)
     ctxs = [binding.Context.from_workload(wl) for _ in range(R)]
+    for c in ctxs:
+        c.set_step_overlap(True)     # the step inputs are all resident before the first call
     outs = [(torch.empty(T, wl.n_q_heads, wl.head_dim, device=dev), torch.empty(T, wl.n_q_heads, device=dev))
             for _ in range(R)]
     res = {}
@@ -593,6 +779,8 @@ def token_path_leg(wl, dev, peaks, seed, n_steps):
     prods = [binding.QkvProducer(emb, nw, w0, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, tm.rms_eps, T)
              for _ in range(R)]      # each handle holds its own re-laid-out copy of the weight
     ctxs = [binding.Context.from_workload(wl) for _ in range(R)]
+    for c in ctxs:
+        c.set_step_overlap(True)     # the token ids are all resident before the first call
     out = torch.empty(T, wl.n_q_heads, wl.head_dim, device=dev)
     lse = torch.empty(T, wl.n_q_heads, device=dev)
     blk = wl.n_blocks // 2
@@ -666,7 +854,7 @@ def token_path_leg(wl, dev, peaks, seed, n_steps):
 # (profiles/tc_attn_kernel_cfg2_ncu_full.txt, tc_attn_kernel_cfg{3,4,5}_step_ncu_full.txt),
 # bytes; None where no capture exists for the workload.  The fp32 output (12.6 MB) is still in L2 when the
 # kernel ends, so the figure is dominated by reads.
-TRAFFIC_PER_LAUNCH = {2: 45337856, 3: 93736960, 4: 456532736, 5: 208314880}
+TRAFFIC_PER_LAUNCH = {(2, 1): 45337856, (3, 1): 93736960, (4, 1): 456532736, (5, 1): 208314880}   # (config, precision mode)
 
 
 # ----------------------------------------------------------------------------
@@ -766,6 +954,10 @@ def main():
     ap.add_argument("--no-incremental", action="store_true",
                     help="skip the extra leg that compares rebuilding the cache per block with advancing it")
     ap.add_argument("--replicas", type=int, default=0, help="cache-state replicas visited round-robin (0 = sized from the L2)")
+    ap.add_argument("--no-tile-granular", action="store_true", help="skip the extra leg with tile-granular caching")
+    ap.add_argument("--precision-mode", type=int, default=-1,
+                    help="0 = plain bf16 operands (suits the small-score configurations 5 and 6), 1 = split operands (default)")
+    ap.add_argument("--out-dtype", default="f32", choices=["f32", "bf16"])
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -21,8 +21,11 @@
  *     [T, Hq, d], lse [T, Hq]; T = sum_b (prompt_lens[b] + gen_len).  Block
  *     tensors are sequence-major: row b * block_len + r is token r of
  *     sequence b's current block.
- *   - Q/K/V element type is `dtype` (bf16 or fp32).  `out` is always fp32,
- *     `lse` fp32 in natural-log units (L = m + log l, Algorithm 1).
+ *   - Q/K/V element type is `dtype` (bf16 or fp32).  `out` is fp32 or bf16
+ *     (`out_dtype`; the `float* out` parameters point to bf16 data then), `lse`
+ *     fp32 in natural-log units (L = m + log l, Algorithm 1).  A bf16 `out` adds
+ *     its own rounding, up to 2^-9 |o| per element (0.016 for 4 <= |o| < 8): the
+ *     stated tolerances are for fp32.
  *   - Query head h reads KV head h / (Hq / Hkv).  Positions are 0-based
  *     inside each sequence.  RoPE pairs feature c with c + d/2 and uses
  *     frequency theta^(-2c/d); V is not rotated.
@@ -60,6 +63,34 @@ enum { LACACHE_DTYPE_BF16 = 0, LACACHE_DTYPE_FP32 = 1 };
 /* which kernel family runs the attention: AUTO picks tcgen05 for bf16 with
  * head_dim 128 and the fp32 CUDA-core kernels otherwise */
 enum { LACACHE_ENGINE_AUTO = 0, LACACHE_ENGINE_SIMT = 1, LACACHE_ENGINE_TCGEN05 = 2 };
+/* element type of `out` (lse is always fp32) */
+enum { LACACHE_OUT_BF16 = 0, LACACHE_OUT_FP32 = 1 };
+/*
+ * How the tcgen05 engine carries the rotated Q', K' into the score product (the paper states no
+ * precision for its kernel beyond "the model's"; Sec. 3.4 keeps the first layer at model precision):
+ *   PLAIN  one bf16 plane per tensor, one tensor-core product per score tile, 128-key tiles.
+ *          Holds the tolerance (2e-2 max / 2e-3 mean abs against an fp64 evaluation) when the
+ *          scores are small: |scale * q.k| of order 1 or less, e.g. q, k ~ N(0,1)/sqrt(d) as in
+ *          the GQA long-context configuration.  The error grows with the score magnitude:
+ *          ~2^-9 * |s| per score, so per-head scales of 2 (scores of order 50) miss it (0.06-0.3).
+ *   SPLIT  two bf16 planes hi = bf16(x), lo = bf16(x - hi), three products hi.hi + hi.lo + lo.hi
+ *          (16 significant bits): needed for the LLaDA-shaped configurations whose per-head scale
+ *          reaches 2 and whose keys carry 4x outliers.  Twice the Q'/K' bytes and twice the
+ *          tensor-core work of PLAIN.
+ * The fp32 CUDA-core engine ignores the mode (its operands are fp32).
+ */
+enum { LACACHE_PRECISION_PLAIN = 0, LACACHE_PRECISION_SPLIT = 1 };
+/*
+ * What a build caches (Sec. 3.3.3 last paragraph; Algorithm 1's Q_overlap / K_overlap predicates):
+ *   TOKEN  the index sets U and C of Sec. 3.3.1 at token granularity: every fixed row keeps a state
+ *          over every fixed key; a step adds exactly the block's keys.
+ *   TILE   Algorithm 1 as printed: state is cached only for row tiles (128 rows, counted from the
+ *          start of the sequence) that do not overlap the block, over key tiles (128 keys) that do
+ *          not overlap it; a step treats every row of a tile that overlaps the block as a block row
+ *          (all keys) and adds to the fixed rows every key of the tiles that overlap the block.
+ *          Same out / lse; less cached, more work per step.  tcgen05 engine only.
+ */
+enum { LACACHE_GRANULARITY_TOKEN = 0, LACACHE_GRANULARITY_TILE = 1 };
 
 typedef struct {
   int dtype;          /* LACACHE_DTYPE_*: element type of q/k/v inputs */
@@ -73,7 +104,10 @@ typedef struct {
   const int32_t* prompt_lens; /* HOST pointer, B entries, each >= 0; copied */
   int gen_len;                /* G > 0, the same for every sequence */
   int block_len;              /* L_b > 0, divides G */
-  int sc_tiles_per_chunk;     /* key tiles (64 keys) per block-query work item; 0 = auto */
+  int sc_tiles_per_chunk;     /* key tiles per block-query work item; 0 = auto */
+  int out_dtype;              /* LACACHE_OUT_*.  NOTE: 0 is bf16; fp32 is what the tolerances are stated for */
+  int precision_mode;         /* LACACHE_PRECISION_*.  NOTE: 0 is PLAIN; see above which inputs it suits */
+  int cache_granularity;      /* LACACHE_GRANULARITY_* */
 } lacache_config;
 
 /* Library version, e.g. 100 = 1.0.0.  No paper counterpart. */
@@ -144,23 +178,23 @@ lacache_status lacache_build_advance(lacache_ctx* ctx, const void* q_fin, const 
  * (m, l, O~) cache is read-only here.  Requires a preceding lacache_build for
  * the same block, else LACACHE_ERR_STATE.
  *
- * Stream semantics: the work is enqueued on `cuda_stream` and is complete, with
- * out / lse fully written, before any later operation of that stream that this
- * library did not enqueue (a kernel, a copy, an event) runs.  Two lacache_step
- * calls in a row on one stream may overlap on the device (the second call's
- * kernels are launched programmatically dependent and store nothing before the
- * first call's kernels have completed); q_blk / k_blk / v_blk must stay
- * unchanged until the call's work has completed, as for any stream-ordered call.
+ * Stream semantics: the work is enqueued on `cuda_stream`, is ordered after
+ * everything enqueued on that stream before it, and is complete, with out / lse
+ * fully written, before any later operation of that stream runs: an ordinary
+ * stream-ordered call.  q_blk / k_blk / v_blk must stay unchanged until the
+ * call's work has completed.
  *
- * Because of that overlap a step reads q_blk / k_blk / v_blk EARLY: possibly
- * before the operation enqueued just ahead of it has flushed its writes.  That
- * is safe when the three tensors were complete before the previous
- * lacache_step of this context was enqueued (precomputed inputs), or were
- * written by work enqueued on another stream and joined by an event.  When
- * they are written by work enqueued on the SAME stream between two steps (a
- * projection kernel run before every step), switch the overlap off with
- * lacache_set_step_overlap(ctx, 0): every kernel of a step is then ordered
- * after all earlier work of the stream, as an ordinary launch is.
+ * Optional overlap of consecutive steps, lacache_set_step_overlap(ctx, 1): two
+ * lacache_step calls in a row on one stream then overlap on the device (the
+ * second call's kernels are launched programmatically dependent and store
+ * nothing before the first call's kernels have completed).  The price is that
+ * such a step reads q_blk / k_blk / v_blk EARLY, possibly before the operation
+ * enqueued just ahead of it has flushed its writes.  Switch it on only when
+ * the three tensors are complete before the PREVIOUS lacache_step of this
+ * context is enqueued (precomputed inputs), or are written by work enqueued on
+ * another stream and joined by an event; never when they are written by work
+ * enqueued on the same stream between two steps (a projection kernel run
+ * before every step).  The results are bit-identical either way.
  * lacache_step_tokens runs such a producer itself and orders its own kernels
  * correctly whatever this setting; what it reads early with the overlap on
  * is blk_token_ids / blk_hidden, to which the same rule applies.
@@ -183,8 +217,9 @@ lacache_status lacache_step(lacache_ctx* ctx, const void* q_blk, const void* k_b
 lacache_status lacache_sample_block(lacache_ctx* ctx, const void* logits, int dtype, int vocab,
                                     float* conf, int32_t* token, float* lse, void* cuda_stream);
 
-/* Overlap of consecutive lacache_step calls on the device (see lacache_step): on (non-zero,
- * the default) or off.  No paper counterpart. */
+/* Overlap of consecutive lacache_step calls on the device (see lacache_step): off (0, the
+ * default: plain stream order) or on (non-zero: the caller vouches that a step's inputs are
+ * complete before the previous step is enqueued).  No paper counterpart. */
 lacache_status lacache_set_step_overlap(lacache_ctx* ctx, int enable);
 
 /*
@@ -223,6 +258,11 @@ lacache_status lacache_full_recompute(lacache_ctx* ctx, const void* q_pre, const
  *   - The first call on each device resolves the array's device address (with
  *     that device current) and sets kernel attributes; make that first call
  *     before starting any stream capture.
+ *   - A call whose (n_tokens, head_dim, rope_theta) differ from the previous
+ *     call's on that device recomputes the RoPE tables on the host and copies
+ *     them (up to 2 MiB, from pageable memory the library owns, so the call
+ *     may wait for the stream's earlier work); a call that repeats them copies
+ *     nothing and only enqueues its two kernels.
  *   - All calls share the one array.  Nothing in it has to start at zero: each
  *     call overwrites what it reads, and the previous call's contents are
  *     simply left behind.  Two calls that overlap on the GPU (different
@@ -392,6 +432,18 @@ lacache_status lacache_export_index_meta(lacache_ctx* ctx, int32_t* seq_of_tok_h
  * the events.  No paper counterpart.
  */
 lacache_status lacache_set_timing_events(lacache_ctx* ctx, void* ev_start, void* ev_stop);
+
+/*
+ * Profiling hook for kernels that overlap their neighbours (an event pair around a launch keeps it
+ * from overlapping and adds the launch latency): `ring` is a DEVICE array of n_slots pairs of
+ * 64-bit words, initialised by the caller to {UINT64_MAX, 0}.  Every later launch of the tcgen05
+ * attention kernel (build, step, full recompute) takes the next slot, in launch order starting at
+ * slot 0 and wrapping, and folds the GPU's global nanosecond timer into it: word 0 = the earliest
+ * entry of any of its CTAs, word 1 = the latest exit.  The caller reads the ring after
+ * synchronising.  Pass NULL, 0 to switch it off.  tcgen05 engine only (other launches leave the
+ * ring alone).  No paper counterpart.
+ */
+lacache_status lacache_set_span_ring(lacache_ctx* ctx, uint64_t* ring, int n_slots);
 
 /* Total packed tokens T, and the number of kernels launched by the last
  * build / step / full_recompute call.  No paper counterpart. */

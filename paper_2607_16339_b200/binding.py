@@ -15,6 +15,9 @@ LIB_PATH = os.path.join(HERE, "liblacache.so")
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_STATE, ERR_UNSUPPORTED, ERR_OOM, ERR_CUDA, ERR_TIMEOUT = range(8)
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 ENGINE_AUTO, ENGINE_SIMT, ENGINE_TCGEN05 = 0, 1, 2
+OUT_BF16, OUT_FP32 = 0, 1
+PRECISION_PLAIN, PRECISION_SPLIT = 0, 1
+GRANULARITY_TOKEN, GRANULARITY_TILE = 0, 1
 
 EXPORTS = [
     "lacache_version", "lacache_create", "lacache_destroy", "lacache_build", "lacache_step",
@@ -27,6 +30,7 @@ EXPORTS = [
     "lacache_qkv_poll_status", "lacache_qkv_last_error", "lacache_set_step_overlap",
     "lacache_build_tokens_update", "lacache_build_incremental", "lacache_build_advance",
     "lacache_build_tokens_incremental", "lacache_build_advance_tokens", "lacache_sample_block",
+    "lacache_set_span_ring",
 ]
 
 
@@ -38,6 +42,7 @@ class LacacheConfig(ctypes.Structure):
         ("batch", ctypes.c_int), ("prompt_lens", ctypes.POINTER(ctypes.c_int32)),
         ("gen_len", ctypes.c_int), ("block_len", ctypes.c_int),
         ("sc_tiles_per_chunk", ctypes.c_int),
+        ("out_dtype", ctypes.c_int), ("precision_mode", ctypes.c_int), ("cache_granularity", ctypes.c_int),
     ]
 
 
@@ -84,6 +89,7 @@ def load():
     lib.lacache_export_index_meta.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_set_timing_events.argtypes = [vp, vp, vp]
     lib.lacache_set_step_overlap.argtypes = [vp, ip]
+    lib.lacache_set_span_ring.argtypes = [vp, vp, ip]
     lib.lacache_sample_block.argtypes = [vp, vp, ip, ip, vp, vp, vp, vp]
     lib.lacache_full_recompute_static.argtypes = [ip, ip, ip, ip, ip, ctypes.c_float, ctypes.c_float, vp, vp, vp, vp,
                                                   vp, vp]
@@ -141,19 +147,22 @@ class Context:
     """Owns one ``lacache_ctx``.  Methods mirror the C calls one to one."""
 
     def __init__(self, dtype, n_q_heads, n_kv_heads, head_dim, rope_theta, prompt_lens, gen_len,
-                 block_len, softmax_scale=0.0, engine=ENGINE_AUTO, sc_tiles_per_chunk=0):
+                 block_len, softmax_scale=0.0, engine=ENGINE_AUTO, sc_tiles_per_chunk=0,
+                 out_dtype=OUT_FP32, precision_mode=PRECISION_SPLIT, cache_granularity=GRANULARITY_TOKEN):
         self._lib = load()
         self._h = ctypes.c_void_p()
         pl = (ctypes.c_int32 * len(prompt_lens))(*[int(p) for p in prompt_lens])
         cfg = LacacheConfig(int(dtype), int(engine), int(n_q_heads), int(n_kv_heads), int(head_dim),
                             float(rope_theta), float(softmax_scale), len(prompt_lens), pl,
-                            int(gen_len), int(block_len), int(sc_tiles_per_chunk))
+                            int(gen_len), int(block_len), int(sc_tiles_per_chunk), int(out_dtype),
+                            int(precision_mode), int(cache_granularity))
         st = self._lib.lacache_create(ctypes.byref(cfg), ctypes.byref(self._h))
         if st != OK:
             self._h = ctypes.c_void_p()
             raise LacacheError(st, (self._lib.lacache_last_error(None) or b"").decode())
         self.n_q_heads, self.n_kv_heads, self.head_dim = n_q_heads, n_kv_heads, head_dim
         self.batch, self.block_len = len(prompt_lens), block_len
+        self.out_dtype = out_dtype
 
     @classmethod
     def from_workload(cls, wl, **kw):
@@ -261,6 +270,14 @@ class Context:
         dt = DTYPE_BF16 if logits.dtype == torch.bfloat16 else DTYPE_FP32
         self._check(self._lib.lacache_sample_block(self._h, _ptr(logits), dt, int(logits.shape[-1]), _ptr(conf),
                                                    _ptr(token), _ptr(lse), _stream(stream)))
+
+    def set_span_ring(self, ring):
+        """ring: int64 / uint64 device tensor [n_slots, 2] initialised to {UINT64_MAX, 0} by the caller, or
+        None to switch the hook off."""
+        if ring is None:
+            self._check(self._lib.lacache_set_span_ring(self._h, None, 0))
+        else:
+            self._check(self._lib.lacache_set_span_ring(self._h, _ptr(ring), int(ring.shape[0])))
 
     def set_timing_events(self, ev_start, ev_stop):
         """torch.cuda.Event pair (already recorded once) or (None, None)."""

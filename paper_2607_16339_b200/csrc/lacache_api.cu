@@ -29,12 +29,28 @@ struct lacache_ctx {
   // cached state = prefix state + the keys after the block; the finished block's rows from scratch;
   // every other row advanced by the finished block's keys and completed by the keys after the block)
   std::vector<ListRef> inc_prefix, inc_comb, inc_fresh, inc_fused;
+  // per block, tile-granular caching (Algorithm 1's overlap predicates): the build in two launches over
+  // the key tiles before / after the tiles that overlap the block, the step in one
+  std::vector<ListRef> tile_prefix, tile_suffix, tile_step;
+  std::vector<int32_t> tile_lo_all, tile_hi_all;   // [n_blk][B]: tokens [lo, hi) of the tiles that overlap the block
   float* sample_part = nullptr;   // scratch of lacache_sample_block (allocated on first use)
   int* sample_counters = nullptr;
   StateBuffers pst{};      // prefix state of every token: its keys before the current block (allocated on first use)
   int prefix_block = -1;   // block pst is valid for
   int num_sms = 148;
-  int stream_ctas_override = 0;
+  // experiment knobs, read from the environment once at create (none is needed in normal use)
+  struct Knobs {
+    int sc_tiles = 0;        // LACACHE_SC_TILES: key tiles per block-query chunk
+    int max_ctas = 0;        // LACACHE_MAX_CTAS: cap on the persistent grid
+    int stream_ctas = 0;     // LACACHE_STREAM_CTAS: role split of a step
+    int deep_units = TC_DEEP_MAX_UNITS;  // LACACHE_DEEP_UNITS: units per CTA one launch of the pipelined merge variant takes
+    bool no_pdl = false;     // LACACHE_NO_PDL: plain stream-ordered launches
+    bool no_step_overlap = false;  // LACACHE_NO_STEP_OVERLAP
+    bool no_deep = false;    // LACACHE_NO_DEEP: earlier merge variant
+    bool no_qcomp = false;   // LACACHE_NO_QCOMP: no in-kernel rotation of first units
+    bool no_pack = false;    // LACACHE_NO_PACK: no head packing of GQA block queries
+    bool verbose = false;    // LACACHE_VERBOSE: prints the step plan
+  } knobs;
   ListRef full_list;
   int max_chunks = 1;
   std::vector<WorkItem> items_host;
@@ -64,11 +80,14 @@ struct lacache_ctx {
   float *hs_out = nullptr, *hs_lse = nullptr;
 
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
+  unsigned long long* span_ring = nullptr;   // lacache_set_span_ring: [n_slots][2] device words
+  int span_slots = 0;
+  unsigned span_next = 0;
   // the role split of a step is planned once per (block, table size) and reused: a step is called
   // thousands of times per second and the host must stay ahead of the device
   struct StepPlan { int deep_cap = -1, ns = 0; };
   std::vector<StepPlan> step_plan;
-  int step_overlap = 1;   // consecutive steps may overlap on the device
+  int step_overlap = 0;   // consecutive steps may overlap on the device (the caller opts in: a step then reads its inputs early)
   int steps_since_build = 0;
   int built_block = -1;
   int last_launches = 0;
@@ -158,6 +177,20 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   c->cfg = *cfg;
   c->cfg.prompt_lens = nullptr;
   c->err[0] = 0;
+  {
+    lacache_ctx::Knobs& k = c->knobs;
+    auto geti = [](const char* name, int dflt) { const char* e = getenv(name); return e ? atoi(e) : dflt; };
+    k.sc_tiles = geti("LACACHE_SC_TILES", 0);
+    k.max_ctas = geti("LACACHE_MAX_CTAS", 0);
+    k.stream_ctas = geti("LACACHE_STREAM_CTAS", 0);
+    k.deep_units = std::max(1, std::min(geti("LACACHE_DEEP_UNITS", TC_DEEP_MAX_UNITS), (int)TC_DEEP_MAX_UNITS));
+    k.no_pdl = getenv("LACACHE_NO_PDL") != nullptr;
+    k.no_step_overlap = getenv("LACACHE_NO_STEP_OVERLAP") != nullptr;
+    k.no_deep = getenv("LACACHE_NO_DEEP") != nullptr;
+    k.no_qcomp = getenv("LACACHE_NO_QCOMP") != nullptr;
+    k.no_pack = getenv("LACACHE_NO_PACK") != nullptr;
+    k.verbose = getenv("LACACHE_VERBOSE") != nullptr;
+  }
   if (cfg->batch < 1 || !cfg->prompt_lens) return fail(c, LACACHE_ERR_INVALID_ARG, "batch < 1 or prompt_lens NULL");
   if (cfg->dtype != LACACHE_DTYPE_BF16 && cfg->dtype != LACACHE_DTYPE_FP32)
     return fail(c, LACACHE_ERR_UNSUPPORTED, "dtype %d", cfg->dtype);
@@ -173,6 +206,12 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   for (int b = 0; b < cfg->batch; ++b)
     if (cfg->prompt_lens[b] < 0) return fail(c, LACACHE_ERR_SHAPE, "prompt_lens[%d] < 0", b);
 
+  if (cfg->out_dtype != LACACHE_OUT_BF16 && cfg->out_dtype != LACACHE_OUT_FP32)
+    return fail(c, LACACHE_ERR_INVALID_ARG, "out_dtype %d", cfg->out_dtype);
+  if (cfg->precision_mode != LACACHE_PRECISION_PLAIN && cfg->precision_mode != LACACHE_PRECISION_SPLIT)
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "precision_mode %d (0 = plain bf16 operands, 1 = split)", cfg->precision_mode);
+  if (cfg->cache_granularity != LACACHE_GRANULARITY_TOKEN && cfg->cache_granularity != LACACHE_GRANULARITY_TILE)
+    return fail(c, LACACHE_ERR_INVALID_ARG, "cache_granularity %d", cfg->cache_granularity);
   bool tc_ok = cfg->dtype == LACACHE_DTYPE_BF16 && cfg->head_dim == 128 && cfg->block_len <= TC_MAX_BLOCK;
   if (cfg->engine == LACACHE_ENGINE_AUTO) c->engine = tc_ok ? LACACHE_ENGINE_TCGEN05 : LACACHE_ENGINE_SIMT;
   else if (cfg->engine == LACACHE_ENGINE_SIMT) c->engine = LACACHE_ENGINE_SIMT;
@@ -180,6 +219,11 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     if (!tc_ok) return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs bf16, head_dim 128, block_len <= 64");
     c->engine = LACACHE_ENGINE_TCGEN05;
   } else return fail(c, LACACHE_ERR_INVALID_ARG, "engine %d", cfg->engine);
+  if (cfg->out_dtype == LACACHE_OUT_BF16) return fail(c, LACACHE_ERR_UNSUPPORTED, "bf16 out: not built yet");   // TEMP
+  if (cfg->precision_mode == LACACHE_PRECISION_PLAIN && c->engine == LACACHE_ENGINE_TCGEN05)
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "plain operands: not built yet");   // TEMP
+  if (cfg->cache_granularity == LACACHE_GRANULARITY_TILE && c->engine != LACACHE_ENGINE_TCGEN05)
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "tile-granular caching needs the tcgen05 engine (bf16, head_dim 128, block_len <= 64)");
 
   // ---- integer metadata (index sets of Sec. 3.3.1) ----
   Geometry& g = c->g;
@@ -209,6 +253,15 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   for (int k = 0; k < g.n_blk; ++k)
     for (int b = 0; b < g.B; ++b) c->blk_start_all[(size_t)k * g.B + b] = c->cu[b] + c->prompt_lens[b] + k * g.block_len;
 
+  // ---- device (queried before planning: the cost models below size work for its SM count) ----
+  CU_TRY(c, cudaGetDevice(&c->device));
+  cudaDeviceProp prop;
+  CU_TRY(c, cudaGetDeviceProperties(&prop, c->device));
+  c->num_sms = prop.multiProcessorCount;
+  if (c->knobs.max_ctas > 0) c->num_sms = std::max(1, std::min(c->num_sms, c->knobs.max_ctas));
+  if (c->engine == LACACHE_ENGINE_TCGEN05 && prop.major != 10)
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs an sm_100 device, found sm_%d%d", prop.major, prop.minor);
+
   // ---- work lists ----
   const bool tc = c->engine == LACACHE_ENGINE_TCGEN05;
   const int R = tc ? TC_ROWS : SIMT_ROWS;
@@ -221,7 +274,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   // (pipelined variant, block_len <= 32, few units per CTA) or ~3.4 after a ~4 us cold start),
   // at most 16 chunks per sequence.
   int tpc = cfg->sc_tiles_per_chunk;
-  if (const char* e = getenv("LACACHE_SC_TILES")) tpc = atoi(e);
+  if (c->knobs.sc_tiles > 0) tpc = c->knobs.sc_tiles;
   if (tc && tpc <= 0) {
     int max_nkt = 1;
     long long rows_u = 0;
@@ -230,7 +283,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
       int n_u = c->cu[b + 1] - c->cu[b] - g.block_len;
       rows_u += (n_u + TC_ROWS - 1) / TC_ROWS + 1;
     }
-    const int sms = 148;
+    const int sms = c->num_sms;
     const double units_m = (double)rows_u * g.Hq;
     double best = 1e30;
     for (int cand = 1; cand <= max_nkt; ++cand) {
@@ -250,7 +303,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
       }
       const double eff_tiles = 0.5 * (sum_t * g.Hq / units_s + max_t);
       const double merge_cost = max_ch > 1 ? 2.0 + 0.8 * max_ch : 0.0;
-      for (int ns = 8; ns <= sms - 8; ns += 4) {
+      for (int ns = std::min(8, std::max(1, sms / 4)); ns <= std::max(1, sms - 8); ns += 4) {
         double ts = ceil(units_s / ns) * (3.0 + 1.6 * eff_tiles + merge_cost);
         // (a CTA with many merge units runs in the HBM-saturated regime, where a unit costs more)
         const double per_cta = ceil(units_m / (sms - ns));
@@ -361,6 +414,49 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     }
     c->inc_fused.push_back({off, (int)items.size() - off});
   }
+  if (cfg->cache_granularity == LACACHE_GRANULARITY_TILE) {
+    // Algorithm 1 at tile granularity, tiles of TC_ROWS tokens counted from the start of each sequence
+    // (B_r = B_c).  With [lo, hi) the tokens of the tiles that overlap the block: state is cached for the
+    // rows outside [lo, hi) over the keys outside [lo, hi) (first the keys before lo, then, on top, the
+    // keys from hi on); a step gives those rows the keys [lo, hi) and runs the rows of [lo, hi) over all
+    // keys.  The work items are key-window items of the build kernel.
+    enum { W_INIT = 1, W_OUT = 16 };
+    auto window = [&](size_t from, int base, int k0, int k1, int flags) {
+      for (size_t i = from; i < items.size(); ++i) {
+        items[i].kind = ITEM_ROWS_WINDOW;
+        items[i].pad = base;
+        items[i].kt0 = k0;
+        items[i].kt1 = k1;
+        items[i].chunk = flags;
+      }
+    };
+    c->tile_lo_all.resize((size_t)g.n_blk * g.B);
+    c->tile_hi_all.resize((size_t)g.n_blk * g.B);
+    for (int k = 0; k < g.n_blk; ++k) {
+      for (int pass = 0; pass < 3; ++pass) {
+        const int off = (int)items.size();
+        for (int b = 0; b < g.B; ++b) {
+          const int cs = c->cu[b], ce = c->cu[b + 1], s0 = c->blk_start_all[(size_t)k * g.B + b], e0 = s0 + g.block_len;
+          const int lo = cs + (s0 - cs) / TC_ROWS * TC_ROWS;
+          const int hi = std::min(ce, cs + (e0 - cs + TC_ROWS - 1) / TC_ROWS * TC_ROWS);
+          c->tile_lo_all[(size_t)k * g.B + b] = lo;
+          c->tile_hi_all[(size_t)k * g.B + b] = hi;
+          size_t from = items.size();
+          if (pass == 2) {   // the rows of the overlapping tiles x all keys: the longest units, so they go first
+            add_row_tiles(items, b, lo, hi, R, cs, ce, s0);
+            window(from, cs, cs, ce, W_OUT);
+            from = items.size();
+          }
+          add_row_tiles(items, b, cs, lo, R, cs, ce, s0);
+          add_row_tiles(items, b, hi, ce, R, cs, ce, s0);
+          if (pass == 0) window(from, cs, cs, lo, 0);
+          else if (pass == 1) window(from, hi, hi, ce, W_INIT);
+          else window(from, lo, lo, hi, W_INIT | W_OUT);
+        }
+        (pass == 0 ? c->tile_prefix : pass == 1 ? c->tile_suffix : c->tile_step).push_back({off, (int)items.size() - off});
+      }
+    }
+  }
   {
     int off = (int)items.size();
     for (int b = 0; b < g.B; ++b) add_row_tiles(items, b, c->cu[b], c->cu[b + 1], R, c->cu[b], c->cu[b + 1], 0);
@@ -368,15 +464,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   }
   c->items_host = items;
 
-  // ---- device ----
-  CU_TRY(c, cudaGetDevice(&c->device));
-  cudaDeviceProp prop;
-  CU_TRY(c, cudaGetDeviceProperties(&prop, c->device));
-  c->num_sms = prop.multiProcessorCount;
-  if (const char* e = getenv("LACACHE_MAX_CTAS")) c->num_sms = std::max(1, std::min(c->num_sms, atoi(e)));  // experiments
-  if (const char* e = getenv("LACACHE_STREAM_CTAS")) c->stream_ctas_override = atoi(e);
-  if (tc && prop.major != 10)
-    return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs an sm_100 device, found sm_%d%d", prop.major, prop.minor);
+  // ---- device memory ----
   CU_TRY(c, simt_prepare());
   if (tc) CU_TRY(c, tc_prepare());
 
@@ -456,13 +544,9 @@ void destroy_impl(lacache_ctx* c) {
   delete c;
 }
 
-// Units per CTA the pipelined merge variant takes in one launch (its table size; LACACHE_DEEP_UNITS
-// lowers it so that small cases exercise the multi-launch path).
-int deep_unit_cap() {
-  const char* e = getenv("LACACHE_DEEP_UNITS");
-  const int v = e ? atoi(e) : TC_DEEP_MAX_UNITS;
-  return std::max(1, std::min(v, (int)TC_DEEP_MAX_UNITS));
-}
+// Units per CTA the pipelined merge variant takes in one launch (its table size; the
+// LACACHE_DEEP_UNITS knob lowers it so that small cases exercise the multi-launch path).
+int deep_unit_cap(const lacache_ctx* c) { return c->knobs.deep_units; }
 
 AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk, const RotBuffers& rot,
                    float* out, float* lse) {
@@ -480,12 +564,13 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
   a.counters = c->counters;
   a.max_chunks = c->max_chunks;
   a.status = c->d_status;
+  a.no_pdl = c->knobs.no_pdl ? 1 : 0;
   if (c->engine == LACACHE_ENGINE_TCGEN05) {
     // persistent grid: one CTA per SM, split between the two roles by a cost
     // estimate (units x per-unit cost, in arbitrary time units)
     const int Hq = c->g.Hq;
     a.stream_slots = Hq; a.pack = 1; a.pack_rows = 0;
-    if (mode == MODE_STEP && c->g.group >= 2 && !getenv("LACACHE_NO_PACK")) {
+    if (mode == MODE_STEP && c->g.group >= 2 && !c->knobs.no_pack) {
       // block queries of a GQA model: heads of one KV group side by side in the 128 lanes of a tile
       const int rows = c->g.block_len <= 32 ? 32 : 64;
       const int pack = std::min(128 / rows, c->g.group);
@@ -501,8 +586,8 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       a.n_items_merge = ml.n;
       long long units_merge = (long long)ml.n * Hq;
       int total = (int)std::min<long long>(c->num_sms, units_stream + units_merge);
-      const bool deep_ok = c->g.block_len <= 32 && !getenv("LACACHE_NO_DEEP");
-      const int deep_cap = deep_unit_cap();
+      const bool deep_ok = c->g.block_len <= 32 && !c->knobs.no_deep;
+      const int deep_cap = deep_unit_cap(c);
       if (c->step_plan.empty()) c->step_plan.resize(c->g.n_blk);
       lacache_ctx::StepPlan& plan = c->step_plan[blk];
       const bool planned = plan.deep_cap == deep_cap;
@@ -528,14 +613,14 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
         double t = std::max(ts, tm) + (rest > 0 ? 4.0 + ceil(rest / c->num_sms) * 3.4 : 0.0);
         if (t < best - 1e-9) { best = t; ns = cand; }
       }
-      if (c->stream_ctas_override > 0) ns = c->stream_ctas_override;
+      if (c->knobs.stream_ctas > 0) ns = c->knobs.stream_ctas;
       if (units_merge == 0) ns = total;
       else ns = std::max(1, std::min(ns, total - 1));
       ns = (int)std::min<long long>(ns, units_stream);
       plan.deep_cap = deep_cap;
       plan.ns = ns;
       a.n_ctas_stream = ns;
-      if (getenv("LACACHE_VERBOSE")) {
+      if (c->knobs.verbose) {
         static int printed = 0;
         if (printed++ < 2) fprintf(stderr, "lacache: step plan: %lld stream units (max %d chunks), %lld merge units, %d stream CTAs of %d\n", units_stream, c->max_chunks, units_merge, ns, total);
       }
@@ -554,6 +639,12 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
   return a;
 }
 
+// one launch of the tcgen05 kernel; with a span ring set, the launch gets the ring's next slot
+cudaError_t launch_tc(lacache_ctx* c, AttnArgs a, const TcMaps* maps, cudaStream_t s) {
+  if (c->span_ring) a.span = c->span_ring + 2 * (size_t)(c->span_next++ % (unsigned)c->span_slots);
+  return tc_attention(c->g, a, maps, s);
+}
+
 lacache_status run_attention(lacache_ctx* c, const AttnArgs& a, bool scratch, cudaStream_t s) {
   if (c->engine == LACACHE_ENGINE_TCGEN05 && a.out) {
     if (!tc_set_out(scratch ? c->maps_scratch : c->maps, c->g, a.out, c->err, sizeof(c->err))) return LACACHE_ERR_CUDA;
@@ -565,14 +656,14 @@ lacache_status run_attention(lacache_ctx* c, const AttnArgs& a, bool scratch, cu
     // many row tiles as its merge CTAs can tabulate, the others row tiles only, on all SMs.
     const TcMaps* maps = scratch ? c->maps_scratch : c->maps;
     const int Hq = c->g.Hq;
-    const int deep_cap = deep_unit_cap();
+    const int deep_cap = deep_unit_cap(c);
     AttnArgs b = a;
     b.merge_deep = 1;
     const int m0 = a.n_ctas - a.n_ctas_stream;
     int done = std::min(a.n_items_merge, std::max(1, deep_cap * m0 / Hq));
     b.n_items_merge = done;
     b.n_ctas = a.n_ctas_stream + (int)std::min<long long>((long long)done * Hq, m0);
-    CU_TRY(c, tc_attention(c->g, b, maps, s));
+    CU_TRY(c, launch_tc(c, b, maps, s));
     c->last_launches++;
     const int rest = a.n_items_merge - done;
     if (rest > 0) {
@@ -587,14 +678,14 @@ lacache_status run_attention(lacache_ctx* c, const AttnArgs& a, bool scratch, cu
         m.items_merge = a.items_merge + done;
         m.n_items_merge = std::min(per, a.n_items_merge - done);
         m.n_ctas = (int)std::min<long long>(c->num_sms, (long long)m.n_items_merge * Hq);
-        CU_TRY(c, tc_attention(c->g, m, maps, s));
+        CU_TRY(c, launch_tc(c, m, maps, s));
         c->last_launches++;
         done += m.n_items_merge;
       }
     }
   } else {
     if (c->engine == LACACHE_ENGINE_TCGEN05)
-      CU_TRY(c, tc_attention(c->g, a, scratch ? c->maps_scratch : c->maps, s));
+      CU_TRY(c, launch_tc(c, a, scratch ? c->maps_scratch : c->maps, s));
     else
       CU_TRY(c, simt_attention(c->g, a, s));
     c->last_launches++;
@@ -670,6 +761,12 @@ lacache_status lacache_destroy(lacache_ctx* ctx) {
   return LACACHE_OK;
 }
 
+namespace {
+lacache_status run_window(lacache_ctx* c, lacache_ctx::ListRef list, int blk, const StateBuffers& init,
+                          const StateBuffers& dst, const StateBuffers& snap, cudaStream_t s, float* out = nullptr,
+                          float* lse = nullptr);
+}  // namespace
+
 lacache_status lacache_build(lacache_ctx* c, int block_idx, const void* q, const void* k, const void* v,
                              void* stream) {
   if (!c) return LACACHE_ERR_INVALID_ARG;
@@ -683,9 +780,18 @@ lacache_status lacache_build(lacache_ctx* c, int block_idx, const void* q, const
   c->prefix_block = -1;
   lacache_status st = rope_all(c, q, k, v, c->rot, s);
   if (st != LACACHE_OK) return st;
-  AttnArgs a = attn_args(c, MODE_BUILD, c->build_list[block_idx], block_idx, c->rot, nullptr, nullptr);
-  st = run_attention(c, a, false, s);
-  if (st != LACACHE_OK) return st;
+  if (c->cfg.cache_granularity == LACACHE_GRANULARITY_TILE) {
+    // state of the rows outside the tiles that overlap the block: over the key tiles before them, then
+    // continued over the key tiles after them (in place: a unit loads its rows before it stores them)
+    st = run_window(c, c->tile_prefix[block_idx], block_idx, StateBuffers{}, c->st, StateBuffers{}, s);
+    if (st != LACACHE_OK) return st;
+    st = run_window(c, c->tile_suffix[block_idx], block_idx, c->st, c->st, StateBuffers{}, s);
+    if (st != LACACHE_OK) return st;
+  } else {
+    AttnArgs a = attn_args(c, MODE_BUILD, c->build_list[block_idx], block_idx, c->rot, nullptr, nullptr);
+    st = run_attention(c, a, false, s);
+    if (st != LACACHE_OK) return st;
+  }
   c->built_block = block_idx;
   c->steps_since_build = 0;
   return LACACHE_OK;
@@ -696,6 +802,8 @@ namespace {
 lacache_status ensure_prefix_state(lacache_ctx* c) {
   if (c->engine != LACACHE_ENGINE_TCGEN05)
     return fail(c, LACACHE_ERR_UNSUPPORTED, "the incremental build needs the tcgen05 engine");
+  if (c->cfg.cache_granularity == LACACHE_GRANULARITY_TILE)
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "the incremental build is token-granular only");
   if (c->pst.o) return LACACHE_OK;
   const Geometry& g = c->g;
   CU_TRY(c, dev_alloc(c, &c->pst.m, (size_t)g.Hq * g.Tp, true));
@@ -705,9 +813,9 @@ lacache_status ensure_prefix_state(lacache_ctx* c) {
 }
 // one launch over a list of key-window items: dst = (init +) the window's keys
 lacache_status run_window(lacache_ctx* c, lacache_ctx::ListRef list, int blk, const StateBuffers& init,
-                          const StateBuffers& dst, const StateBuffers& snap, cudaStream_t s) {
+                          const StateBuffers& dst, const StateBuffers& snap, cudaStream_t s, float* out, float* lse) {
   if (list.n == 0) return LACACHE_OK;
-  AttnArgs a = attn_args(c, MODE_BUILD, list, blk, c->rot, nullptr, nullptr);
+  AttnArgs a = attn_args(c, MODE_BUILD, list, blk, c->rot, out, lse);
   a.window = 1;
   a.init = init;
   a.st = dst;
@@ -892,8 +1000,7 @@ lacache_status lacache_step_tokens(lacache_ctx* c, lacache_qkv* p, const int32_t
   qkv_scratch(p, true, &q, &k, &v);
   // with the cross-step overlap on (and not right after a build) the norm kernel reads the ids while the
   // previous step's attention kernel still runs: the same contract as for q_blk / k_blk / v_blk of lacache_step
-  const bool early = c->step_overlap && c->steps_since_build > 0 && !getenv("LACACHE_NO_PDL") &&
-                     !getenv("LACACHE_NO_STEP_OVERLAP");
+  const bool early = c->step_overlap && c->steps_since_build > 0 && !c->knobs.no_pdl && !c->knobs.no_step_overlap;
   st = qkv_project_rows(p, blk_token_ids, blk_hidden, n, q, k, v, nullptr, nullptr, 0, early, stream);
   if (st != LACACHE_OK) return fail(c, st, "producer: %s", lacache_qkv_last_error(p));
   st = step_impl(c, q, k, v, out, lse, stream, true);
@@ -926,18 +1033,28 @@ lacache_status step_impl(lacache_ctx* c, const void* q, const void* k, const voi
   }
   // may start while the previous step's attention kernel drains (it waits before its stores); when
   // the kernel before it in the stream is the one that writes its inputs, it waits for that one first
-  const bool overlap = c->step_overlap && !getenv("LACACHE_NO_PDL") && !getenv("LACACHE_NO_STEP_OVERLAP");
+  const bool overlap = c->step_overlap && !c->knobs.no_pdl && !c->knobs.no_step_overlap;
   // (the first step after a build is launched the ordinary way: the build's cached state, which the
   // attention kernel reads before it waits on anything, is then complete and flushed)
   r.pdl = inputs_just_written ? 2 : ((overlap && c->steps_since_build > 0) ? 1 : 0);
+  r.no_pdl = (c->knobs.no_pdl || c->knobs.no_step_overlap) ? 1 : 0;
   c->steps_since_build++;
   r.dst = c->rot;
   r.in_dtype = c->cfg.dtype;
+  if (c->cfg.cache_granularity == LACACHE_GRANULARITY_TILE) {
+    // Algorithm 1's reuse pass at tile granularity: ordinary launches, one pass of the build kernel over
+    // key windows (rows of the overlapping tiles x all keys; every other row: cached state + the keys of
+    // the overlapping tiles), normalised output instead of state
+    r.pdl = 0;
+    CU_TRY(c, rope_write(c->g, r, c->engine, s));
+    c->last_launches++;
+    return run_window(c, c->tile_step[blk], blk, c->st, c->st, StateBuffers{}, s, out, lse);
+  }
   CU_TRY(c, rope_write(c->g, r, c->engine, s));
   c->last_launches++;
   AttnArgs a = attn_args(c, MODE_STEP, c->step_list[blk], blk, c->rot, out, lse);
   a.step_overlap = overlap ? 1 : 0;
-  if (!getenv("LACACHE_NO_QCOMP")) {
+  if (!c->knobs.no_qcomp) {
     a.q_raw = q;
     a.k_raw = k;
     a.v_raw = v;
@@ -1072,6 +1189,16 @@ lacache_status lacache_export_index_meta(lacache_ctx* c, int32_t* seq, int32_t* 
   }
   if (kvh)
     for (int h = 0; h < g.Hq; ++h) kvh[h] = h / g.group;
+  return LACACHE_OK;
+}
+
+lacache_status lacache_set_span_ring(lacache_ctx* c, uint64_t* ring, int n_slots) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if ((ring == nullptr) != (n_slots <= 0)) return fail(c, LACACHE_ERR_INVALID_ARG, "pass a ring with n_slots > 0, or NULL with 0");
+  if (ring && (reinterpret_cast<uintptr_t>(ring) & 7u)) return fail(c, LACACHE_ERR_INVALID_ARG, "ring not 8-byte aligned");
+  c->span_ring = reinterpret_cast<unsigned long long*>(ring);
+  c->span_slots = ring ? n_slots : 0;
+  c->span_next = 0;
   return LACACHE_OK;
 }
 

@@ -17,7 +17,8 @@ enum ItemKind : int32_t {
                          // chunk bit 0: continue from the rows' state in AttnArgs::init; bit 1: store the
                          // state after the first key tile to AttnArgs::snap; bit 2: leave out the keys of
                          // the block at blk_start; bit 3: the first tile ends at blk_start (pad = blk_start -
-                         // tile width) and the tiles after it are counted from the end of that block
+                         // tile width) and the tiles after it are counted from the end of that block; bit 4:
+                         // the unit writes normalised rows to out / lse instead of a state
 };
 struct WorkItem {
   int32_t kind;   // ItemKind
@@ -92,6 +93,7 @@ struct RopeArgs {
   // step's attention kernel, which lets its successors start early; this kernel then waits before its
   // first store.  2: that kernel writes this kernel's inputs; this kernel waits before anything else.
   int pdl;
+  int no_pdl;   // host only: launch the ordinary way whatever `pdl` says (experiment knob)
 };
 
 struct AttnArgs {
@@ -127,6 +129,10 @@ struct AttnArgs {
   // split-key partial states of block queries and their arrival counters
   float* part_m; float* part_l; float* part_o; int* counters; int max_chunks;
   int32_t* status;
+  int no_pdl;                // host only: launch the ordinary way (experiment knob)
+  // optional (lacache_set_span_ring): two device words of this launch; every CTA folds the global
+  // nanosecond timer into them at entry (minimum) and at exit (maximum)
+  unsigned long long* span;
 };
 
 struct SampleArgs {

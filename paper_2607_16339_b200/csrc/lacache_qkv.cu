@@ -60,6 +60,9 @@ struct lacache_qkv {
   CUtensorMap x_map[4];                 // boxes of 32, 64, 128, 256 tokens
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
   int last_launches = 0;
+  // experiment knobs, read from the environment once at create
+  bool no_pdl = false;        // LACACHE_NO_PDL: plain stream-ordered launches
+  bool plain_split = false;   // LACACHE_QKV_PLAIN_SPLIT: no closer / helper roles
   char err[512];
 };
 
@@ -847,6 +850,8 @@ lacache_status lacache_qkv_create(const lacache_qkv_config* cfg, lacache_qkv** o
   p->tokens_pad = (cfg->max_tokens + MAX_TN - 1) / MAX_TN * MAX_TN;
   lacache_status st = LACACHE_OK;
   auto attempt = [&]() -> lacache_status {
+    p->no_pdl = getenv("LACACHE_NO_PDL") != nullptr;
+    p->plain_split = getenv("LACACHE_QKV_PLAIN_SPLIT") != nullptr;
     QCU_TRY(p, cudaGetDevice(&p->device));
     cudaDeviceProp prop;
     QCU_TRY(p, cudaGetDeviceProperties(&prop, p->device));
@@ -934,7 +939,6 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   na.max_rows = max_rows;
   na.early_inputs = early_inputs ? 1 : 0;
   na.ready = p->ready;
-  p->ready_target += (unsigned)n_tokens;
   na.d_model = p->cfg.d_model;
   na.vocab = p->cfg.vocab;
   na.eps = p->cfg.rms_eps;
@@ -942,7 +946,7 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  const bool no_pdl = getenv("LACACHE_NO_PDL") != nullptr;
+  const bool no_pdl = p->no_pdl;
   {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_tokens);
@@ -952,6 +956,9 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
     cfg.numAttrs = no_pdl ? 0 : 1;
     QCU_TRY(p, cudaLaunchKernelEx(&cfg, qkv_norm_kernel, na));
   }
+  // the norm kernel is enqueued and will publish its n_tokens rows: only now does the count the
+  // projection waits for move (a failed launch above leaves counter and target in step)
+  p->ready_target += (unsigned)n_tokens;
   p->last_launches++;
 
   GemmArgs ga{};
@@ -978,7 +985,7 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   ga.status = p->status;
   const int n_ctas = (int)std::min<long long>(p->num_sms, ga.total_chunks);
   ga.hp = 0;
-  if (ga.tn <= 64 && n_ctas > ga.n_tiles && n_ctas < 2 * ga.n_tiles && !getenv("LACACHE_QKV_PLAIN_SPLIT")) {
+  if (ga.tn <= 64 && n_ctas > ga.n_tiles && n_ctas < 2 * ga.n_tiles && !p->plain_split) {
     // closers take `per_closer` chunks each, helpers about HEAD_START chunks fewer
     const int HEAD_START = 8;
     const int n_helpers = n_ctas - ga.n_tiles;

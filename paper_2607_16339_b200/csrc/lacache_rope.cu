@@ -11,8 +11,6 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
-#include <cstdlib>
-
 #include "lacache_internal.h"
 #include "lacache_rope_math.h"
 
@@ -171,8 +169,7 @@ cudaError_t rope_write(const Geometry& g, const RopeArgs& a, int engine, cudaStr
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    static const bool no_pdl = getenv("LACACHE_NO_PDL") != nullptr || getenv("LACACHE_NO_STEP_OVERLAP") != nullptr;
-    cfg.numAttrs = (a.pdl && !no_pdl) ? 1 : 0;
+    cfg.numAttrs = (a.pdl && !a.no_pdl) ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, rope_write_kernel<true>, g, a);
   }
   rope_write_kernel<false><<<blocks, 256, 0, s>>>(g, a);

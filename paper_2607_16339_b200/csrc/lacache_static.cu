@@ -35,6 +35,10 @@ static __device__ __align__(256) float g_static_scratch[STATIC_WORDS];
 
 constexpr int MAX_DEVICES = 64;
 float* g_scratch_dev[MAX_DEVICES];  // device address of the array, per device (nullptr = not set up)
+// What the tables and metadata in a device's copy of the array were last filled for: a call with the same
+// (n_tokens, head_dim, rope_theta) finds them as it needs them and copies nothing.
+struct Filled { int n_tokens, head_dim; float theta; };
+Filled g_filled[MAX_DEVICES];
 
 // host-side staging for the tables and metadata (no allocation per call)
 float h_cos[STATIC_MAX_TOKENS * 64];
@@ -106,32 +110,38 @@ extern "C" lacache_status lacache_full_recompute_static(int dtype, int n_tokens,
   // meta: [0, T) positions | [T, T+16) cu (padded) | work items
   const int n_items = (n_tokens + SIMT_ROWS - 1) / SIMT_ROWS;
   const size_t items_off = ((size_t)n_tokens + 16 + 3) & ~(size_t)3;  // 16-byte aligned
-  for (int t = 0; t < n_tokens; ++t) h_meta[t] = t;
-  memset(h_meta + n_tokens, 0, sizeof(int32_t) * 16);
-  h_meta[n_tokens + 1] = n_tokens;  // cu = {0, T}
-  WorkItem* items = reinterpret_cast<WorkItem*>(h_meta + items_off);
-  for (int i = 0; i < n_items; ++i) {
-    WorkItem w{};
-    w.kind = ITEM_ROWS; w.seq = 0; w.row0 = i * SIMT_ROWS;
-    w.nrows = n_tokens - w.row0 < SIMT_ROWS ? n_tokens - w.row0 : SIMT_ROWS;
-    w.pad = 1; w.seq_start = 0; w.seq_end = n_tokens;
-    items[i] = w;
-  }
-  for (int c = 0; c < half; ++c) {
-    const double f = pow((double)rope_theta, -2.0 * (double)c / (double)head_dim);
-    for (int p = 0; p < n_tokens; ++p) {
-      const double ang = (double)p * f;
-      h_cos[(size_t)p * half + c] = (float)cos(ang);
-      h_sin[(size_t)p * half + c] = (float)sin(ang);
+  Filled& filled = g_filled[dev];
+  const bool refill = filled.n_tokens != n_tokens || filled.head_dim != head_dim || filled.theta != rope_theta;
+  if (refill) {
+    filled.n_tokens = 0;   // (until the copies below are enqueued)
+    for (int t = 0; t < n_tokens; ++t) h_meta[t] = t;
+    memset(h_meta + n_tokens, 0, sizeof(int32_t) * 16);
+    h_meta[n_tokens + 1] = n_tokens;  // cu = {0, T}
+    WorkItem* items = reinterpret_cast<WorkItem*>(h_meta + items_off);
+    for (int i = 0; i < n_items; ++i) {
+      WorkItem w{};
+      w.kind = ITEM_ROWS; w.seq = 0; w.row0 = i * SIMT_ROWS;
+      w.nrows = n_tokens - w.row0 < SIMT_ROWS ? n_tokens - w.row0 : SIMT_ROWS;
+      w.pad = 1; w.seq_start = 0; w.seq_end = n_tokens;
+      items[i] = w;
     }
+    for (int c = 0; c < half; ++c) {
+      const double f = pow((double)rope_theta, -2.0 * (double)c / (double)head_dim);
+      for (int p = 0; p < n_tokens; ++p) {
+        const double ang = (double)p * f;
+        h_cos[(size_t)p * half + c] = (float)cos(ang);
+        h_sin[(size_t)p * half + c] = (float)sin(ang);
+      }
+    }
+    // Nothing in the array has to start at zero: every word a kernel reads below
+    // is written first by these copies or by the rotation kernel.
+    const size_t meta_words = items_off + (size_t)n_items * (sizeof(WorkItem) / 4);
+    if ((e = cudaMemcpyAsync(d_cos, h_cos, sizeof(float) * n_tokens * half, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(d_sin, h_sin, sizeof(float) * n_tokens * half, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(d_meta, h_meta, sizeof(int32_t) * meta_words, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+      return fail(LACACHE_ERR_CUDA, cudaGetErrorString(e));
+    filled = Filled{n_tokens, head_dim, rope_theta};
   }
-  // Nothing in the array has to start at zero: every word a kernel reads below
-  // is written first by these copies or by the rotation kernel.
-  const size_t meta_words = items_off + (size_t)n_items * (sizeof(WorkItem) / 4);
-  if ((e = cudaMemcpyAsync(d_cos, h_cos, sizeof(float) * n_tokens * half, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(d_sin, h_sin, sizeof(float) * n_tokens * half, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(d_meta, h_meta, sizeof(int32_t) * meta_words, cudaMemcpyHostToDevice, s)) != cudaSuccess)
-    return fail(LACACHE_ERR_CUDA, cudaGetErrorString(e));
 
   RopeArgs r{};
   r.q = q_pre; r.k = k_pre; r.v = v_pre;

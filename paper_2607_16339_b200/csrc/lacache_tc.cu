@@ -34,7 +34,6 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 #include <stdio.h>
-#include <stdlib.h>
 
 #include "lacache_internal.h"
 #include "lacache_ptx.h"
@@ -161,6 +160,11 @@ __device__ __forceinline__ void ld_global_v8(const void* src, uint32_t* r) {
                : "l"(src)
                : "memory");
 }
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -185,15 +189,6 @@ __device__ __forceinline__ WorkItem load_item(const WorkItem* p) {
 }
 
 
-#ifdef LACACHE_DEBUG_CLOCKS
-__device__ long long g_dbg_clocks[256 * 64];
-#define DBG_CLK(k) do { if ((k) < 64) g_dbg_clocks[(size_t)blockIdx.x * 64 + (k)] = clock64(); } while (0)
-__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define DBG_GT(k) do { g_dbg_clocks[(size_t)blockIdx.x * 64 + (k)] = gtime(); } while (0)
-#else
-#define DBG_CLK(k) do { } while (0)
-#define DBG_GT(k) do { } while (0)
-#endif
 
 struct Cta {
   uint32_t base;            // shared-space address of the region
@@ -316,7 +311,7 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
       un.base1 = it.blk_start + g.block_len;
       un.t1 = 1 + (it.kt1 > un.base1 ? (it.kt1 - un.base1 + BN - 1) / BN : 0);
     }
-    un.epi = EPI_STATE;
+    un.epi = (it.chunk & 16) ? EPI_OUT : EPI_STATE;   // bit 4: normalised rows to out / lse instead of a state
     un.init = it.chunk & 1;
     un.snap = (it.chunk >> 1) & 1;
   } else if (!STEP && a.mode == MODE_BUILD) {
@@ -1701,6 +1696,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   // therefore be scheduled as SMs free up (they, too, wait before their first store).  A build or a
   // full recompute writes what a following step would read early, so they do not trigger.
   if (STEP && a.step_overlap) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (a.span != nullptr && tid == 0) atomicMin(a.span, global_timer_ns());   // first CTA entry of this launch
   Cta c;
   c.base = smem_u32(smem_raw);
   c.gen = smem_raw;
@@ -1812,18 +1808,11 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.tmem), "r"(TM_COLS) : "memory");
+    // (every thread of the CTA is past its work here: BAR_DONE counts them all)
+    if (a.span != nullptr && tid == 32) atomicMax(a.span + 1, global_timer_ns());   // last CTA exit
   }
 }
 
-#ifdef LACACHE_DEBUG_CLOCKS
-}  // namespace
-}  // namespace lacache
-extern "C" int lacache_debug_read_clocks(long long* host, int n) {
-  return (int)cudaMemcpyFromSymbol(host, lacache::g_dbg_clocks, sizeof(long long) * n);
-}
-namespace lacache {
-namespace {
-#endif
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -1957,8 +1946,7 @@ cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* map
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  static const bool no_pdl = getenv("LACACHE_NO_PDL") != nullptr;
-  cfg.numAttrs = no_pdl ? 0 : 1;
+  cfg.numAttrs = a.no_pdl ? 0 : 1;
   // six instantiations: build / full recompute; build over key windows; the step of an MHA and of a
   // GQA model, each with either variant of the merge role
   if (a.mode != MODE_STEP) {

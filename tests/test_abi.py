@@ -37,7 +37,8 @@ def test_create_rejects_bad_configs_without_gpu():
     def cfg(**kw):
         base = dict(dtype=0, engine=0, n_q_heads=4, n_kv_heads=2, head_dim=128, rope_theta=1e4,
                     softmax_scale=0.0, batch=1, prompt_lens=pl, gen_len=32, block_len=16,
-                    sc_tiles_per_chunk=0)
+                    sc_tiles_per_chunk=0, out_dtype=binding.OUT_FP32, precision_mode=binding.PRECISION_SPLIT,
+                    cache_granularity=binding.GRANULARITY_TOKEN)
         base.update(kw)
         return binding.LacacheConfig(*[base[f[0]] for f in binding.LacacheConfig._fields_])
 
@@ -49,6 +50,10 @@ def test_create_rejects_bad_configs_without_gpu():
         (cfg(batch=0), binding.ERR_INVALID_ARG),
         (cfg(rope_theta=0.0), binding.ERR_INVALID_ARG),
         (cfg(engine=2, dtype=1), binding.ERR_UNSUPPORTED),
+        (cfg(out_dtype=2), binding.ERR_INVALID_ARG),
+        (cfg(precision_mode=2), binding.ERR_UNSUPPORTED),       # a split of the probabilities is not offered
+        (cfg(cache_granularity=5), binding.ERR_INVALID_ARG),
+        (cfg(cache_granularity=binding.GRANULARITY_TILE, dtype=1), binding.ERR_UNSUPPORTED),   # tcgen05 engine only
     ]
     for c, want in cases:
         st = lib.lacache_create(ctypes.byref(c), ctypes.byref(h))

@@ -120,6 +120,18 @@ def test_block_lengths_that_split_a_warp(block_len):
     _run_points(wl, "tc", seed=8, blocks=[0, wl.n_blocks - 1], sc_tiles_per_chunk=2)
 
 
+@pytest.mark.parametrize("block_len", [48, 64])
+@pytest.mark.parametrize("tiles_per_chunk", [0, 2])
+def test_mha_blocks_of_48_and_64_rows(block_len, tiles_per_chunk):
+    """A model without grouped heads (one KV head per query head) with blocks of 33..64 rows: the step
+    runs unpacked block queries together with the merge variant that takes up to 64 block keys.  Per-head
+    scales up to 2 (the harsh value distribution), a ragged batch, prompts long enough for the block
+    queries' keys to be cut into several chunks."""
+    wl = small_workload(name="mha%d" % block_len, prompt_lens=(700, 333, 61), gen_len=192, block_len=block_len,
+                        steps=2, hq=4, hkv=4, scale_mode="per_head_u(0.5,2)")
+    _run_points(wl, "tc", seed=14, blocks=[0, 1, wl.n_blocks - 1], sc_tiles_per_chunk=tiles_per_chunk)
+
+
 @pytest.mark.parametrize("hq,hkv,block_len", [(6, 2, 64), (10, 2, 32), (7, 1, 64), (14, 2, 16)])
 def test_packed_block_queries_odd_groups(hq, hkv, block_len):
     """GQA steps put the block rows of two (blocks of 33..64 rows) or four (up to 32 rows) heads of a KV
@@ -211,13 +223,19 @@ def test_runs_are_bit_reproducible():
         assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
 
 
-@pytest.mark.parametrize("cfg", [2, 4, 5])
-def test_back_to_back_steps_match_synchronised_steps(cfg):
-    """Consecutive steps overlap on the device (the next step's kernels are scheduled while
-    the previous attention kernel drains).  A stream of steps and builds issued without any
-    host synchronisation must give, bit for bit, what the same calls give when the host
-    waits after each one -- with a separate output buffer per step and with one reused."""
-    wl = WORKLOADS[cfg]
+_MHA64 = small_workload(name="mha64", prompt_lens=(700, 333, 61), gen_len=192, block_len=64, steps=6, hq=4, hkv=4,
+                        scale_mode="per_head_u(0.5,2)")
+
+
+@pytest.mark.parametrize("cfg", [2, 4, 5, "mha64"])
+@pytest.mark.parametrize("overlap", [True, False])
+def test_back_to_back_steps_match_synchronised_steps(cfg, overlap):
+    """With the overlap of consecutive steps switched on (precomputed inputs), the next step's kernels
+    are scheduled while the previous attention kernel drains.  A stream of steps and builds issued
+    without any host synchronisation must give, bit for bit, what the same calls give when the host
+    waits after each one -- with a separate output buffer per step and with one reused; likewise with
+    the default, plain stream order."""
+    wl = _MHA64 if cfg == "mha64" else WORKLOADS[cfg]
     S = min(wl.steps_per_block, 6)
     calls = []   # ("build", blk, q, k, v) / ("step", qb, kb, vb)
     sch = SyntheticSchedule(wl, seed=21)
@@ -231,6 +249,7 @@ def test_back_to_back_steps_match_synchronised_steps(cfg):
 
     def run(sync, one_buffer):
         ctx = make_ctx(wl, engine=ENGINES["tc"])
+        ctx.set_step_overlap(overlap)
         bufs = [new_outputs(wl) for _ in range(1 if one_buffer else n_steps)]
         res, i = [], 0
         for c in calls:
@@ -263,10 +282,10 @@ def test_back_to_back_steps_match_synchronised_steps(cfg):
 
 
 @pytest.mark.parametrize("cfg", [2, 5])
-def test_steps_fed_by_same_stream_writes_with_overlap_off(cfg):
+def test_steps_fed_by_same_stream_writes(cfg):
     """Block inputs that are written on the stream between two steps (here: copied into one reused
-    trio of buffers right before each step) with the cross-step overlap switched off: every kernel
-    of a step is then ordered after the copy.  Bit for bit what synchronised steps give."""
+    trio of buffers right before each step) with the default setting (no cross-step overlap): every
+    kernel of a step is ordered after the copy.  Bit for bit what synchronised steps give."""
     wl = WORKLOADS[cfg]
     S = min(wl.steps_per_block, 5)
     sch = SyntheticSchedule(wl, seed=33)
@@ -280,7 +299,6 @@ def test_steps_fed_by_same_stream_writes_with_overlap_off(cfg):
         ctx.step(qb, kb, vb, out, lse)
         torch.cuda.synchronize()
         ref.append((out, lse))
-    ctx.set_step_overlap(False)
     qs, ks, vs = (torch.empty_like(t) for t in steps[0])
     for rep in range(3):
         got = [new_outputs(wl) for _ in steps]
@@ -314,7 +332,11 @@ def test_step_split_over_several_launches(cfg, monkeypatch):
     torch.cuda.synchronize()
     assert ctx.last_launch_count == 2
     for cap in ("3", "1"):
-        monkeypatch.setenv("LACACHE_DEEP_UNITS", cap)
+        monkeypatch.setenv("LACACHE_DEEP_UNITS", cap)     # (experiment knobs are read when a context is created)
+        ctx.destroy()
+        ctx = make_ctx(wl, engine=ENGINES["tc"])
+        ctx.set_step_overlap(True)
+        ctx.build(b, q, k, v)
         got = []
         for qb, kb, vb in steps:              # back to back: the launches of consecutive steps overlap
             out, lse = new_outputs(wl)

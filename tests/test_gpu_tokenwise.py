@@ -333,10 +333,11 @@ def test_projection_odd_shapes(d_model, hq, hkv, n):
     prod.destroy()
 
 
-def test_back_to_back_token_steps_match_synchronised_ones():
-    """Token-fed steps issued without any host synchronisation (the norm kernel of a step then runs
-    alongside the previous step's attention kernel) give, bit for bit, what the same calls give when
-    the host waits after each."""
+@pytest.mark.parametrize("overlap", [True, False])
+def test_back_to_back_token_steps_match_synchronised_ones(overlap):
+    """Token-fed steps issued without any host synchronisation (with the overlap of consecutive steps
+    switched on, the norm kernel of a step runs alongside the previous step's attention kernel) give,
+    bit for bit, what the same calls give when the host waits after each."""
     wl = W.small_workload(prompt_lens=(300, 170), gen_len=64, block_len=32, steps=6, hq=8, hkv=4)
     tm = TokenModel(wl, 512, 1500)
     T = wl.total_tokens
@@ -347,6 +348,7 @@ def test_back_to_back_token_steps_match_synchronised_ones():
     def run(sync):
         prod = make_producer(tm, T)
         ctx = make_ctx(wl)
+        ctx.set_step_overlap(overlap)
         ctx.build_tokens(prod, 0, token_ids=ids_full)
         res = []
         for ids in ids_steps:

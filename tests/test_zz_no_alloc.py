@@ -34,10 +34,13 @@ def test_static_entry_point_matches_context_entry_point(dtype):
         ref, ref_lse = new_outputs(wl)
         ctx.full_recompute(q, k, v, ref, ref_lse)
         torch.cuda.synchronize()
-        for rep in range(2):             # and the same size twice
+        for rep in range(2):             # and the same size twice (the second finds its tables in place)
             out, lse = new_outputs(wl)
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             binding.full_recompute_static(dt, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.rope_theta, q, k, v, out, lse)
             torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before      # nothing was allocated on the device
             assert torch.isfinite(out).all()
             assert (out - ref).abs().max().item() <= TOL_CACHED_VS_FULL[dtype]
             assert (lse - ref_lse).abs().max().item() <= 1e-5
