@@ -219,7 +219,6 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     if (!tc_ok) return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs bf16, head_dim 128, block_len <= 64");
     c->engine = LACACHE_ENGINE_TCGEN05;
   } else return fail(c, LACACHE_ERR_INVALID_ARG, "engine %d", cfg->engine);
-  if (cfg->out_dtype == LACACHE_OUT_BF16) return fail(c, LACACHE_ERR_UNSUPPORTED, "bf16 out: not built yet");   // TEMP
   if (cfg->precision_mode == LACACHE_PRECISION_PLAIN && c->engine == LACACHE_ENGINE_TCGEN05)
     return fail(c, LACACHE_ERR_UNSUPPORTED, "plain operands: not built yet");   // TEMP
   if (cfg->cache_granularity == LACACHE_GRANULARITY_TILE && c->engine != LACACHE_ENGINE_TCGEN05)
@@ -447,10 +446,14 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
             window(from, cs, cs, ce, W_OUT);
             from = items.size();
           }
+          // (no unit without keys: a sequence with nothing before the overlapping tiles starts its state in
+          // the second launch, one with nothing after them is complete after the first)
+          if (pass == 0 && lo == cs) continue;
+          if (pass == 1 && hi == ce) continue;
           add_row_tiles(items, b, cs, lo, R, cs, ce, s0);
           add_row_tiles(items, b, hi, ce, R, cs, ce, s0);
           if (pass == 0) window(from, cs, cs, lo, 0);
-          else if (pass == 1) window(from, hi, hi, ce, W_INIT);
+          else if (pass == 1) window(from, hi, hi, ce, lo > cs ? W_INIT : 0);
           else window(from, lo, lo, hi, W_INIT | W_OUT);
         }
         (pass == 0 ? c->tile_prefix : pass == 1 ? c->tile_suffix : c->tile_step).push_back({off, (int)items.size() - off});
@@ -560,6 +563,7 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
   a.st = c->st;
   a.out = out;
   a.lse = lse;
+  a.out_bf16 = c->cfg.out_dtype == LACACHE_OUT_BF16 ? 1 : 0;
   a.part_m = c->part_m; a.part_l = c->part_l; a.part_o = c->part_o;
   a.counters = c->counters;
   a.max_chunks = c->max_chunks;
@@ -647,7 +651,7 @@ cudaError_t launch_tc(lacache_ctx* c, AttnArgs a, const TcMaps* maps, cudaStream
 
 lacache_status run_attention(lacache_ctx* c, const AttnArgs& a, bool scratch, cudaStream_t s) {
   if (c->engine == LACACHE_ENGINE_TCGEN05 && a.out) {
-    if (!tc_set_out(scratch ? c->maps_scratch : c->maps, c->g, a.out, c->err, sizeof(c->err))) return LACACHE_ERR_CUDA;
+    if (!tc_set_out(scratch ? c->maps_scratch : c->maps, c->g, a.out, a.out_bf16 != 0, c->err, sizeof(c->err))) return LACACHE_ERR_CUDA;
   }
   if (c->ev_start) CU_TRY(c, cudaEventRecord(c->ev_start, s));
   if (c->engine == LACACHE_ENGINE_TCGEN05 && a.split_merge) {
@@ -723,7 +727,7 @@ lacache_status ensure_staging(lacache_ctx* c) {
   CU_TRY(c, dev_alloc(c, &f, bk * es));
   c->hs_q = a; c->hs_k = b; c->hs_v = cc; c->hs_qb = d; c->hs_kb = e; c->hs_vb = f;
   CU_TRY(c, dev_alloc(c, &c->hs_lse, (size_t)g.T * g.Hq));
-  CU_TRY(c, dev_alloc(c, &c->hs_out, nq));
+  CU_TRY(c, dev_alloc(c, &c->hs_out, nq));   // (sized for fp32; a bf16 out uses half of it)
   return LACACHE_OK;
 }
 
@@ -1152,7 +1156,8 @@ lacache_status lacache_step_host(lacache_ctx* c, const void* q, const void* k, c
   CU_TRY(c, cudaMemcpyAsync(c->hs_vb, v, rows * g.Hkv * g.d * es, cudaMemcpyHostToDevice, s));
   st = lacache_step(c, c->hs_qb, c->hs_kb, c->hs_vb, c->hs_out, lse ? c->hs_lse : nullptr, stream);
   if (st != LACACHE_OK) return st;
-  CU_TRY(c, cudaMemcpyAsync(out, c->hs_out, sizeof(float) * g.T * g.Hq * g.d, cudaMemcpyDeviceToHost, s));
+  const size_t out_es = c->cfg.out_dtype == LACACHE_OUT_BF16 ? 2 : 4;
+  CU_TRY(c, cudaMemcpyAsync(out, c->hs_out, out_es * g.T * g.Hq * g.d, cudaMemcpyDeviceToHost, s));
   if (lse) CU_TRY(c, cudaMemcpyAsync(lse, c->hs_lse, sizeof(float) * g.T * g.Hq, cudaMemcpyDeviceToHost, s));
   return LACACHE_OK;
 }

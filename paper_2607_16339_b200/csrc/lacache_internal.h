@@ -126,6 +126,7 @@ struct AttnArgs {
   StateBuffers snap;         // ... and where units with the snapshot bit store their state after the first key tile
                              // (may alias init: a unit loads its rows before it stores them)
   float* out; float* lse;    // token-major [T,Hq,d], [T,Hq]
+  int out_bf16;              // `out` holds bf16 elements (lse stays fp32)
   // split-key partial states of block queries and their arrival counters
   float* part_m; float* part_l; float* part_o; int* counters; int max_chunks;
   int32_t* status;
@@ -170,7 +171,7 @@ cudaError_t tc_prepare();
 // err on failure
 TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, char* err, int errlen);
 // (re)encodes the descriptor of the caller's output buffer when it changed
-bool tc_set_out(TcMaps* m, const Geometry& g, float* out, char* err, int errlen);
+bool tc_set_out(TcMaps* m, const Geometry& g, float* out, bool out_bf16, char* err, int errlen);
 void tc_free_maps(TcMaps* m);
 
 // token-wise producer (lacache_qkv.cu): the scratch rows the *_tokens entry points project into,

@@ -10,6 +10,8 @@
 // warps owns 4 rows.  Per key tile, lane j holds the score of key j for the
 // warp's 4 rows (dot product over d from shared memory), row max / sum are
 // warp shuffles, and for P.V lane c owns output features c, c+32, ...
+#include <cuda_bf16.h>
+
 #include "lacache_internal.h"
 
 namespace lacache {
@@ -149,8 +151,14 @@ __global__ void __launch_bounds__(WARPS * 32) simt_attn_kernel(Geometry g, AttnA
     } else {
       float inv = 1.f / l[i];
       size_t row = (size_t)tok * g.Hq + h;
+      if (a.out_bf16) {
+        __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(a.out);
 #pragma unroll
-      for (int t = 0; t < DPL; ++t) a.out[row * D + lane + 32 * t] = o[i][t] * inv;
+        for (int t = 0; t < DPL; ++t) ob[row * D + lane + 32 * t] = __float2bfloat16_rn(o[i][t] * inv);
+      } else {
+#pragma unroll
+        for (int t = 0; t < DPL; ++t) a.out[row * D + lane + 32 * t] = o[i][t] * inv;
+      }
       if (a.lse && lane == 0) a.lse[row] = (m[i] + log2f(l[i])) * LN2;
     }
   }

@@ -32,6 +32,7 @@
 // Every mbarrier wait is bounded; a wait that runs out sets the status word
 // and the CTA unwinds (TMEM is always freed).
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <stdio.h>
 
@@ -177,6 +178,20 @@ __device__ __forceinline__ float ex2(float x) {
 __device__ __forceinline__ float round_to_half_bits(float p) {
   float c = __fmul_rn(p, 8193.0f);
   return __fsub_rn(c, __fsub_rn(c, p));
+}
+// four consecutive output elements at element offset `off` of `out` (fp32, or bf16 when the context's
+// out_dtype says so)
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ void store_out4(const AttnArgs& a, size_t off, float4 v) {
+  if (a.out_bf16) {
+    *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.out) + off) =
+        make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+  } else {
+    *reinterpret_cast<float4*>(a.out + off) = v;
+  }
 }
 __device__ __forceinline__ WorkItem load_item(const WorkItem* p) {
   const int4* q = reinterpret_cast<const int4*>(p);
@@ -580,8 +595,10 @@ __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
     const Unit un = decode_stream<PACKED, KIND>(g, a, it, u);
     const int n_tiles = un.t1 - un.t0;
-    // O~ of the previous unit has been read by the row threads (observed once per unit, in order)
-    if (uu >= 1 && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
+    // O~ of the previous unit has been read by the row threads.  (A unit without key tiles issues nothing
+    // and does not wait: the row threads cannot complete this unit's phase of the barrier before the
+    // products of its tiles are done, so when a unit with tiles looks, the barrier is at most one phase on.)
+    if (uu >= 1 && n_tiles > 0 && !wait_bar(c, BAR_O_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;
     for (int j = 0; j < n_tiles; ++j, ++jp) {
       const uint32_t b = jp & 1u, sv = jp & 1u, ph = (jp >> 1) & 1u;
       if (!wait_bar(c, BAR_P_FULL + b, ph, LOC_WAIT_S)) return;
@@ -614,6 +631,18 @@ __device__ __forceinline__ void coop_store_rows(const Cta& c, uint32_t stage_off
     const int rr = i >> 5, ch = i & 31;
     float4 v = *reinterpret_cast<const float4*>(c.gen + stage_off + rr * STAGE_ROW + ((ch ^ (rr & 7)) << 4));
     *reinterpret_cast<float4*>(gbase + (size_t)rr * stride + ch * 4) = v;
+  }
+}
+
+// The same for rows of `out` (element offset `off0` of the first row, `stride` elements between rows), in
+// the output's element type.
+__device__ __forceinline__ void coop_store_out_rows(const Cta& c, const AttnArgs& a, uint32_t stage_off, size_t off0,
+                                                    size_t stride, int nrows) {
+  const int t = threadIdx.x - 64;
+  for (int i = t; i < nrows * 32; i += ROW_THREADS) {
+    const int rr = i >> 5, ch = i & 31;
+    float4 v = *reinterpret_cast<const float4*>(c.gen + stage_off + rr * STAGE_ROW + ((ch ^ (rr & 7)) << 4));
+    store_out4(a, off0 + (size_t)rr * stride + ch * 4, v);
   }
 }
 
@@ -663,8 +692,7 @@ __device__ __forceinline__ void merge_few(const Geometry& g, const AttnArgs& a, 
       }
       const float inv = 1.f / L;
       const size_t orow = (size_t)(row0 + rr) * g.Hq + h;
-      *reinterpret_cast<float4*>(a.out + orow * D + ch * 4) =
-          make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+      store_out4(a, orow * D + ch * 4, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
       if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
     }
   }
@@ -719,7 +747,7 @@ __device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs
     }
     const float inv = 1.f / L;
     const size_t orow = (size_t)(row0 + rr) * g.Hq + h;
-    *reinterpret_cast<float4*>(a.out + orow * D + ch * 4) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+    store_out4(a, orow * D + ch * 4, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
     if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
   }
 }
@@ -739,7 +767,9 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
   volatile float* xch = reinterpret_cast<volatile float*>(c.gen + SM_XCH + r * 16);  // 4 exchange slots per row
   uint32_t epi_phase = 0, epi_unit = 0, pair_phase = 0, xslot = 0;
   int jj = 0;
+  int uu = -1;   // ordinal of the unit in this CTA
   for (int u = first; u < n_units; u += stride) {
+    ++uu;
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
     const Unit un = decode_stream<PACKED, KIND>(g, a, it, u);
@@ -785,7 +815,15 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     float m_ref = -INFINITY, l_part = 0.f;
     bool first_tile = true;
     bool have_o = false;   // O~ in TMEM holds something before the unit's first P~V
+    if (WINDOW && un.t1 <= un.t0) {
+      // A unit without key tiles gives these threads nothing to wait for, and the other roles' parity
+      // waits hold only while nobody runs more than one phase ahead: stay in step with the producer (the
+      // unit's Q load lands only after the previous unit has been released by these threads).
+      if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
+    }
     if (WINDOW && un.init) {
+      // (the state may have been written by the launch just before this one)
+      grid_dependency_wait();
       // The unit continues from a stored state (m, l, O~) of its rows: the reference exponent and the
       // normaliser go to registers (the normaliser to the first thread of the pair), O~ to the
       // accumulator columns this thread owns.  Nobody else reads or writes those cells between units
@@ -1140,8 +1178,8 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_ref + log2f(l_run)) * LN2;
       if (!epi_sync(c, epi_phase)) return;
       for (int j = 0; j < un.nh; ++j)   // one head's rows at a time (a single head unless block queries are packed)
-        coop_store_rows(c, stage_off + (uint32_t)(j * un.rh) * STAGE_ROW, a.out + ((size_t)un.row0 * g.Hq + un.h + j) * D,
-                        (size_t)g.Hq * D, un.nrows);
+        coop_store_out_rows(c, a, stage_off + (uint32_t)(j * un.rh) * STAGE_ROW, ((size_t)un.row0 * g.Hq + un.h + j) * D,
+                            (size_t)g.Hq * D, un.nrows);
     }
     if (!epi_sync(c, epi_phase)) return;  // the staging rows have been read
     if (un.q_rows == BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));  // the Q region may be reloaded
@@ -1153,10 +1191,15 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
 // for a clipped tile boxes of 64, 32, 16 and 8 rows (each starts on a multiple of 8 rows,
 // where the staging tile's swizzle pattern repeats).  Returns the rows covered; the last
 // nrows % 8 rows are left to the row threads.  The caller commits the bulk group.
-__device__ __forceinline__ int store_out_tile(const TcMaps& maps, uint32_t src, int h, int row0, int nrows) {
+// With a bf16 `out` the tile holds two boxes of 64 bf16 features x 128 rows, at the places of the fp32
+// boxes 0 and 2, and the tensor maps describe bf16 boxes.
+__device__ __forceinline__ int store_out_tile(const TcMaps& maps, uint32_t src, int h, int row0, int nrows,
+                                              bool bf16) {
+  const int nb = bf16 ? 2 : 4;                     // boxes per tile
+  const uint32_t bstep = bf16 ? 2 * IO_BOX : IO_BOX;
+  const int fstep = bf16 ? 64 : 32;                // features per box
   if (nrows == BM) {
-#pragma unroll
-    for (int cb = 0; cb < 4; ++cb) tma_store_3d(&maps.out, src + cb * IO_BOX, 32 * cb, h, row0);
+    for (int cb = 0; cb < nb; ++cb) tma_store_3d(&maps.out, src + cb * bstep, fstep * cb, h, row0);
     return BM;
   }
   int done = 0;
@@ -1164,13 +1207,72 @@ __device__ __forceinline__ int store_out_tile(const TcMaps& maps, uint32_t src, 
   for (int i = 0; i < 4; ++i) {
     const int bs = 64 >> i;
     if (nrows - done >= bs) {
-#pragma unroll
-      for (int cb = 0; cb < 4; ++cb)
-        tma_store_3d(&maps.out_sub[i], src + cb * IO_BOX + done * 128, 32 * cb, h, row0 + done);
+      for (int cb = 0; cb < nb; ++cb)
+        tma_store_3d(&maps.out_sub[i], src + cb * bstep + done * 128, fstep * cb, h, row0 + done);
       done += bs;
     }
   }
   return done;
+}
+
+// The merge roles' combine, out = (alpha O~_cache + P~V) / l, for this thread's 64 features of tile row r, in
+// place in the staging tile: `sbox` is the row's place in the thread's first fp32 box (box 2 * half; the
+// second follows IO_BOX further), `o_tmem` the TMEM address of its 64 P~V columns.  With a bf16 `out` the 64
+// results are packed and written over the row of the first box (128 bytes, the layout of a bf16 box).
+__device__ __forceinline__ void combine_row(uint8_t* sbox, int sw, uint32_t o_tmem, float a_inv, float inv, bool bf16) {
+  if (!bf16) {
+#pragma unroll
+    for (int q2 = 0; q2 < 2; ++q2) {
+      uint32_t rr[32];
+      tmem_ld32(o_tmem + 32 * q2, rr);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float4* p4 = reinterpret_cast<float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
+        float4 oc = *p4;
+        oc.x = fmaf(oc.x, a_inv, __uint_as_float(rr[4 * i]) * inv);
+        oc.y = fmaf(oc.y, a_inv, __uint_as_float(rr[4 * i + 1]) * inv);
+        oc.z = fmaf(oc.z, a_inv, __uint_as_float(rr[4 * i + 2]) * inv);
+        oc.w = fmaf(oc.w, a_inv, __uint_as_float(rr[4 * i + 3]) * inv);
+        *p4 = oc;
+      }
+    }
+    return;
+  }
+  uint32_t pk[32];   // 64 bf16 results
+#pragma unroll
+  for (int q2 = 0; q2 < 2; ++q2) {
+    uint32_t rr[32];
+    tmem_ld32(o_tmem + 32 * q2, rr);
+    tmem_ld_wait();
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float4 oc = *reinterpret_cast<const float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
+      pk[16 * q2 + 2 * i] = pack_bf16x2(fmaf(oc.x, a_inv, __uint_as_float(rr[4 * i]) * inv),
+                                        fmaf(oc.y, a_inv, __uint_as_float(rr[4 * i + 1]) * inv));
+      pk[16 * q2 + 2 * i + 1] = pack_bf16x2(fmaf(oc.z, a_inv, __uint_as_float(rr[4 * i + 2]) * inv),
+                                            fmaf(oc.w, a_inv, __uint_as_float(rr[4 * i + 3]) * inv));
+    }
+  }
+  // (every read of the row's two fp32 boxes is done: only this thread touches them)
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+    *reinterpret_cast<uint4*>(sbox + ((j ^ sw) << 4)) = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+}
+// one row of a clipped tile's tail, from the staging tile straight to `out` (this thread's 64 features)
+__device__ __forceinline__ void store_tail_row(const AttnArgs& a, const uint8_t* sbox, int sw, size_t orow, int half) {
+  if (a.out_bf16) {
+    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.out) + orow * D + 64 * half);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) dst[j] = *reinterpret_cast<const uint4*>(sbox + ((j ^ sw) << 4));
+  } else {
+    float4* dst = reinterpret_cast<float4*>(a.out + orow * D + 64 * half);
+#pragma unroll
+    for (int q2 = 0; q2 < 2; ++q2)
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        dst[8 * q2 + i] = *reinterpret_cast<const float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
+  }
 }
 
 // ===========================================================================
@@ -1326,22 +1428,7 @@ __device__ void merge_rows(const Cta& c, const TcMaps& maps, const Geometry& g, 
     if (!wait_bar(c, BAR_IO_FULL, uu & 1, LOC_WAIT_V)) return;
     tc_fence_after();
     // out = (alpha O~_cache + P~V) / l, in place in the staging tile
-#pragma unroll
-    for (int q2 = 0; q2 < 2; ++q2) {
-      uint32_t rr[32];
-      tmem_ld32(tlane + TM_O + 128 * b + 64 * half + 32 * q2, rr);
-      tmem_ld_wait();
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        float4* p4 = reinterpret_cast<float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
-        float4 oc = *p4;
-        oc.x = fmaf(oc.x, a_inv, __uint_as_float(rr[4 * i]) * inv);
-        oc.y = fmaf(oc.y, a_inv, __uint_as_float(rr[4 * i + 1]) * inv);
-        oc.z = fmaf(oc.z, a_inv, __uint_as_float(rr[4 * i + 2]) * inv);
-        oc.w = fmaf(oc.w, a_inv, __uint_as_float(rr[4 * i + 3]) * inv);
-        *p4 = oc;
-      }
-    }
+    combine_row(sbox, sw, tlane + TM_O + 128 * b + 64 * half, a_inv, inv, a.out_bf16 != 0);
     tc_fence_before();
     mbar_arrive(c.bar(BAR_O_FREE + b));
     grid_dependency_wait();  // no global store before the preceding grids are complete
@@ -1349,18 +1436,13 @@ __device__ void merge_rows(const Cta& c, const TcMaps& maps, const Geometry& g, 
     if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_new + log2f(l_new)) * LN2;
     if (row_valid && r >= (it.nrows & ~7)) {
       // the last nrows % 8 rows of a clipped tile go out one by one (the rest by bulk stores)
-      float4* dst = reinterpret_cast<float4*>(a.out + orow * D + 64 * half);
-#pragma unroll
-      for (int q2 = 0; q2 < 2; ++q2)
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-          dst[8 * q2 + i] = *reinterpret_cast<const float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
+      store_tail_row(a, sbox, sw, orow, half);
     }
     fence_async_smem();
     if (!epi_sync(c, epi_phase)) return;  // the whole tile is in the staging buffer
     if (threadIdx.x == 64) {
       grid_dependency_wait();
-      if (store_out_tile(maps, c.base + SM_IO, h, it.row0, it.nrows) > 0) {
+      if (store_out_tile(maps, c.base + SM_IO, h, it.row0, it.nrows, a.out_bf16 != 0) > 0) {
         bulk_commit();
         bulk_wait_read();               // the copies have read the staging tile
       }
@@ -1396,7 +1478,8 @@ __device__ __forceinline__ DUnit deep_unit(const Cta& c, int i) {
   return DUnit{v.x, v.y, v.z, v.w & 0xFFFF, v.w >> 16};
 }
 
-__device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& g, int n_my, bool kv_computed) {
+__device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& g, int n_my, bool kv_computed,
+                              bool out_bf16) {
   if (n_my == 0) return;
   auto load_q = [&](int i) {
     const DUnit un = deep_unit(c, i);
@@ -1458,7 +1541,7 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
     if (mbar_test(c.bar((su & 1) ? BAR_OUT_RDY1 : BAR_OUT_RDY), (su >> 1) & 1)) {
       const DUnit un = deep_unit(c, su);
       if (!dep_done) { grid_dependency_wait(); dep_done = true; }  // no store before the preceding grids are complete
-      if (store_out_tile(maps, c.base + DM_IO + (su & 1) * DM_IO_TILE, un.h, un.row0, un.nrows) > 0) {
+      if (store_out_tile(maps, c.base + DM_IO + (su & 1) * DM_IO_TILE, un.h, un.row0, un.nrows, out_bf16) > 0) {
         bulk_commit();
         pending_read = true;
       }
@@ -1647,22 +1730,7 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
     if (!wait_bar(c, b ? BAR_IO_FULL1 : BAR_IO_FULL, par, LOC_WAIT_V)) return;
     tc_fence_after();
     // out = (alpha O~_cache + P~V) / l, in place in the staging tile
-#pragma unroll
-    for (int q2 = 0; q2 < 2; ++q2) {
-      uint32_t rr[32];
-      tmem_ld32(tlane + TM_O + 128 * b + 64 * half + 32 * q2, rr);
-      tmem_ld_wait();
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        float4* p4 = reinterpret_cast<float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
-        float4 oc = *p4;
-        oc.x = fmaf(oc.x, a_inv, __uint_as_float(rr[4 * i]) * inv);
-        oc.y = fmaf(oc.y, a_inv, __uint_as_float(rr[4 * i + 1]) * inv);
-        oc.z = fmaf(oc.z, a_inv, __uint_as_float(rr[4 * i + 2]) * inv);
-        oc.w = fmaf(oc.w, a_inv, __uint_as_float(rr[4 * i + 3]) * inv);
-        *p4 = oc;
-      }
-    }
+    combine_row(sbox, sw, tlane + TM_O + 128 * b + 64 * half, a_inv, inv, a.out_bf16 != 0);
     tc_fence_before();
     mbar_arrive(c.bar(BAR_O_FREE + b));
     grid_dependency_wait();  // no global store before the preceding grids are complete
@@ -1670,12 +1738,7 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
     if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_new + log2f(l_new)) * LN2;
     if (row_valid && r >= (un.nrows & ~7)) {
       // the last nrows % 8 rows of a clipped tile go out one by one (the rest by bulk stores)
-      float4* dst = reinterpret_cast<float4*>(a.out + orow * D + 64 * half);
-#pragma unroll
-      for (int q2 = 0; q2 < 2; ++q2)
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-          dst[8 * q2 + i] = *reinterpret_cast<const float4*>(sbox + q2 * IO_BOX + ((i ^ sw) << 4));
+      store_tail_row(a, sbox, sw, orow, half);
     }
     fence_async_smem();  // the producer thread's bulk store reads this tile
     mbar_arrive(c.bar(b ? BAR_OUT_RDY1 : BAR_OUT_RDY));
@@ -1780,7 +1843,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
     if (stream) {
       if (tid == 0) stream_producer<PACKED, KIND>(c, maps, g, a, first, stride, n_units, it0);
     } else if (deep) {
-      if (tid == 0) deep_producer(c, maps, g, n_my, a.k_raw != nullptr);
+      if (tid == 0) deep_producer(c, maps, g, n_my, a.k_raw != nullptr, a.out_bf16 != 0);
     } else {
       if (tid == 0) merge_producer(c, maps, g, a, first, stride, n_units, it0);
     }
@@ -1830,15 +1893,18 @@ EncodeTiledFn get_encode() {
   return fn;
 }
 
+// rows of D features, fp32 (boxes of 32 features) or bf16 (boxes of 64): either way a box row is 128 bytes
 bool make_f32_map(CUtensorMap* m, void* base, cuuint64_t d1, cuuint64_t d2, cuuint32_t b1, cuuint32_t b2, char* err,
-                  int errlen) {
+                  int errlen, bool bf16 = false) {
   EncodeTiledFn enc = get_encode();
   if (!enc) { snprintf(err, errlen, "cuTensorMapEncodeTiled entry point not found"); return false; }
+  const cuuint64_t es = bf16 ? 2 : 4;
   cuuint64_t dims[3] = {(cuuint64_t)D, d1, d2};
-  cuuint64_t strides[2] = {(cuuint64_t)D * 4, d1 * D * 4};
-  cuuint32_t box[3] = {32, b1, b2};
+  cuuint64_t strides[2] = {(cuuint64_t)D * es, d1 * D * es};
+  cuuint32_t box[3] = {bf16 ? 64u : 32u, b1, b2};
   cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+  CUresult r = enc(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides,
+                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { snprintf(err, errlen, "cuTensorMapEncodeTiled (fp32) failed with CUresult %d", (int)r); return false; }
   return true;
@@ -1902,11 +1968,11 @@ cudaError_t tc_prepare() {
   return cudaSuccess;
 }
 
-bool tc_set_out(TcMaps* m, const Geometry& g, float* out, char* err, int errlen) {
+bool tc_set_out(TcMaps* m, const Geometry& g, float* out, bool out_bf16, char* err, int errlen) {
   if (m->out_ptr == out) return true;
-  if (!make_f32_map(&m->out, out, (cuuint64_t)g.Hq, (cuuint64_t)g.T, 1, BM, err, errlen)) return false;
+  if (!make_f32_map(&m->out, out, (cuuint64_t)g.Hq, (cuuint64_t)g.T, 1, BM, err, errlen, out_bf16)) return false;
   for (int i = 0; i < 4; ++i)
-    if (!make_f32_map(&m->out_sub[i], out, (cuuint64_t)g.Hq, (cuuint64_t)g.T, 1, 64u >> i, err, errlen)) return false;
+    if (!make_f32_map(&m->out_sub[i], out, (cuuint64_t)g.Hq, (cuuint64_t)g.T, 1, 64u >> i, err, errlen, out_bf16)) return false;
   m->out_ptr = out;
   return true;
 }

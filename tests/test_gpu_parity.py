@@ -394,6 +394,47 @@ def test_large_batch_extension_full_size():
     ctx.destroy()
 
 
+@pytest.mark.parametrize("case", ["ragged3", "gqa", "gqa32", "blk16", "mha64"])
+@pytest.mark.parametrize("engine", ["tc", "simt"])
+def test_bf16_output(case, engine):
+    """out_dtype = bf16: every epilogue (fixed rows through both merge variants, block rows, merged key
+    chunks, the full recompute) rounds the very fp32 value the fp32 context writes, once, to nearest even:
+    the two outputs agree bit for bit after that rounding.  Against the oracle the error is the fp32
+    path's plus at most half a bf16 unit of the value (2^-9 |o|); the figures are printed."""
+    kw = dict(prompt_lens=(700, 333, 61), gen_len=192, block_len=64, steps=2, hq=4, hkv=4) if case == "mha64" else dict(SMALL[case])
+    wl = small_workload(name=case, dtype="bf16", d=128, **kw)
+    sch = SyntheticSchedule(wl, seed=31)
+    b = wl.n_blocks - 1
+    q, k, v = (to_dev(a, wl) for a in advance_to_block(sch, b))
+    qb, kb, vb = (to_dev(a, wl) for a in sch.draw_step(b, 1))
+    T = wl.total_tokens
+    res = {}
+    for od in (binding.OUT_FP32, binding.OUT_BF16):
+        ctx = make_ctx(wl, engine=ENGINES[engine], out_dtype=od, sc_tiles_per_chunk=2)
+        tdt = torch.float32 if od == binding.OUT_FP32 else torch.bfloat16
+        out = torch.full((T, wl.n_q_heads, wl.head_dim), float("nan"), device="cuda", dtype=tdt)
+        fout = torch.full_like(out, float("nan"))
+        lse = torch.full((T, wl.n_q_heads), float("nan"), device="cuda")
+        ctx.build(b, q, k, v)
+        ctx.step(qb, kb, vb, out, lse)
+        ctx.full_recompute(to_dev(sch.q, wl), to_dev(sch.k, wl), to_dev(sch.v, wl), fout, None)
+        torch.cuda.synchronize()
+        assert ctx.poll_status()[0] == 0
+        res[od] = (out, fout, lse)
+        ctx.destroy()
+    o32, f32, l32 = res[binding.OUT_FP32]
+    o16, f16, l16 = res[binding.OUT_BF16]
+    assert torch.equal(o32.to(torch.bfloat16), o16)
+    assert torch.equal(f32.to(torch.bfloat16), f16)
+    assert torch.equal(l32, l16)
+    ref, _ = oracle.attention(sch.q, sch.k, sch.v, wl.cu_seqlens, wl.rope_theta, wl.head_dim ** -0.5)
+    e32 = np.abs(o32.cpu().numpy().astype(np.float64) - ref)
+    e16 = np.abs(o16.float().cpu().numpy().astype(np.float64) - ref)
+    assert (e16 <= e32 + 2.0 ** -9 * (np.abs(ref) + e32) + 1e-12).all()
+    print("bf16 out, %s/%s: max abs err %.4g (fp32 out %.4g), mean %.4g (%.4g), max |o| %.3g"
+          % (case, engine, e16.max(), e32.max(), e16.mean(), e32.mean(), np.abs(ref).max()))
+
+
 def test_error_paths():
     wl = small_workload(prompt_lens=(40,), gen_len=64, block_len=32, steps=1, hq=2, hkv=2, d=128)
     sch = SyntheticSchedule(wl, seed=1)
