@@ -24,7 +24,7 @@
  *   - Q/K/V element type is `dtype` (bf16 or fp32).  `out` is fp32 or bf16
  *     (`out_dtype`; the `float* out` parameters point to bf16 data then), `lse`
  *     fp32 in natural-log units (L = m + log l, Algorithm 1).  A bf16 `out` adds
- *     its own rounding, up to 2^-9 |o| per element (0.016 for 4 <= |o| < 8): the
+ *     its own rounding, up to 2^-8 |o| per element (0.016 for 4 <= |o| < 8): the
  *     stated tolerances are for fp32.
  *   - Query head h reads KV head h / (Hq / Hkv).  Positions are 0-based
  *     inside each sequence.  RoPE pairs feature c with c + d/2 and uses

@@ -54,6 +54,7 @@ struct lacache_ctx {
   ListRef full_list;
   int max_chunks = 1;
   std::vector<WorkItem> items_host;
+  bool split = true;       // tcgen05 engine: rotated Q', K' kept as two bf16 planes (precision_mode SPLIT)
 
   // device memory
   std::vector<void*> allocs;
@@ -158,11 +159,13 @@ lacache_status alloc_rot(lacache_ctx* c, RotBuffers* r) {
   if (c->engine == LACACHE_ENGINE_TCGEN05) {
     // hi and lo planes of a tensor share one allocation (the lo plane starts
     // right after the hi plane): the tensor maps address them as one 5-D tensor
+    // (plain operands: no lo plane at all)
     uint16_t *a, *cc, *e;
-    CU_TRY(c, dev_alloc(c, &a, 2 * nq, true));
-    CU_TRY(c, dev_alloc(c, &cc, 2 * nk, true));
+    const size_t planes = c->split ? 2 : 1;
+    CU_TRY(c, dev_alloc(c, &a, planes * nq, true));
+    CU_TRY(c, dev_alloc(c, &cc, planes * nk, true));
     CU_TRY(c, dev_alloc(c, &e, nk, true));
-    *r = RotBuffers{a, a + nq, cc, cc + nk, e};
+    *r = RotBuffers{a, c->split ? a + nq : nullptr, cc, c->split ? cc + nk : nullptr, e};
   } else {
     float *a, *b, *cc;
     CU_TRY(c, dev_alloc(c, &a, nq, true));
@@ -219,8 +222,6 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     if (!tc_ok) return fail(c, LACACHE_ERR_UNSUPPORTED, "tcgen05 engine needs bf16, head_dim 128, block_len <= 64");
     c->engine = LACACHE_ENGINE_TCGEN05;
   } else return fail(c, LACACHE_ERR_INVALID_ARG, "engine %d", cfg->engine);
-  if (cfg->precision_mode == LACACHE_PRECISION_PLAIN && c->engine == LACACHE_ENGINE_TCGEN05)
-    return fail(c, LACACHE_ERR_UNSUPPORTED, "plain operands: not built yet");   // TEMP
   if (cfg->cache_granularity == LACACHE_GRANULARITY_TILE && c->engine != LACACHE_ENGINE_TCGEN05)
     return fail(c, LACACHE_ERR_UNSUPPORTED, "tile-granular caching needs the tcgen05 engine (bf16, head_dim 128, block_len <= 64)");
 
@@ -263,6 +264,8 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
 
   // ---- work lists ----
   const bool tc = c->engine == LACACHE_ENGINE_TCGEN05;
+  c->split = cfg->precision_mode == LACACHE_PRECISION_SPLIT;
+  const int TC_KEYS = tc_keys(c->split);
   const int R = tc ? TC_ROWS : SIMT_ROWS;
   std::vector<WorkItem> items;
   // Block-query units: the keys of each (sequence, head) are cut into balanced
@@ -530,9 +533,9 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   CU_TRY(c, dev_alloc(c, &c->counters, (size_t)g.B * g.Hq, true));
   CU_TRY(c, dev_alloc(c, &c->d_status, 4, true));
   if (tc) {
-    c->maps = tc_make_maps(g, c->rot, c->st.o, c->err, sizeof(c->err));
+    c->maps = tc_make_maps(g, c->rot, c->st.o, c->split, c->err, sizeof(c->err));
     if (!c->maps) return LACACHE_ERR_CUDA;
-    c->maps_scratch = tc_make_maps(g, c->rot_scratch, c->st.o, c->err, sizeof(c->err));
+    c->maps_scratch = tc_make_maps(g, c->rot_scratch, c->st.o, c->split, c->err, sizeof(c->err));
     if (!c->maps_scratch) return LACACHE_ERR_CUDA;
   }
   CU_TRY(c, cudaDeviceSynchronize());
@@ -569,6 +572,7 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
   a.max_chunks = c->max_chunks;
   a.status = c->d_status;
   a.no_pdl = c->knobs.no_pdl ? 1 : 0;
+  a.split = c->split ? 1 : 0;
   if (c->engine == LACACHE_ENGINE_TCGEN05) {
     // persistent grid: one CTA per SM, split between the two roles by a cost
     // estimate (units x per-unit cost, in arbitrary time units)

@@ -131,6 +131,7 @@ struct AttnArgs {
   float* part_m; float* part_l; float* part_o; int* counters; int max_chunks;
   int32_t* status;
   int no_pdl;                // host only: launch the ordinary way (experiment knob)
+  int split;                 // host only: rotated Q', K' are split bf16 planes (which kernel instantiation runs)
   // optional (lacache_set_span_ring): two device words of this launch; every CTA folds the global
   // nanosecond timer into them at entry (minimum) and at exit (maximum)
   unsigned long long* span;
@@ -169,7 +170,7 @@ cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* map
 cudaError_t tc_prepare();
 // builds TMA descriptors for a rotated buffer set; returns nullptr and fills
 // err on failure
-TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, char* err, int errlen);
+TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, bool split, char* err, int errlen);
 // (re)encodes the descriptor of the caller's output buffer when it changed
 bool tc_set_out(TcMaps* m, const Geometry& g, float* out, bool out_bf16, char* err, int errlen);
 void tc_free_maps(TcMaps* m);
@@ -190,10 +191,11 @@ bool qkv_full_owner_is(const lacache_qkv* p, const void* ctx, int n_tokens);
 
 constexpr int SIMT_ROWS = 32;    // query rows per SIMT work item
 constexpr int TC_ROWS = 128;     // query rows per tcgen05 work item
-#ifndef LACACHE_TC_KEYS
-#define LACACHE_TC_KEYS 96
-#endif
-constexpr int TC_KEYS = LACACHE_TC_KEYS;   // keys per tile of the tcgen05 stream role
+// keys per tile of the tcgen05 stream role: 96 with split operands (two stages of {K hi, K lo} and of V fit
+// beside the Q tile), 128 with plain ones
+constexpr int TC_KEYS_SPLIT = 96;
+constexpr int TC_KEYS_PLAIN = 128;
+inline int tc_keys(bool split) { return split ? TC_KEYS_SPLIT : TC_KEYS_PLAIN; }
 constexpr int TC_MAX_BLOCK = 64;
 constexpr int TC_DEEP_MAX_UNITS = 512;  // units per CTA the pipelined merge role can tabulate // largest block length the tcgen05 merge role handles
 

@@ -28,7 +28,8 @@ __device__ __forceinline__ void store8_split(void* hi_plane, void* lo_plane, siz
   uint4 uh, ul;
   rope_split8(y, uh, ul);
   *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(hi_plane) + off) = uh;
-  *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(lo_plane) + off) = ul;
+  // (plain operands keep the hi plane alone: the rotated value rounded once to bf16)
+  if (lo_plane) *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(lo_plane) + off) = ul;
 }
 
 __device__ __forceinline__ void store8_f16(void* plane, size_t off, const float (&y)[8]) {
@@ -120,7 +121,7 @@ template <bool TC>
 __device__ __forceinline__ float read_rot(const void* hi, const void* lo, size_t off) {
   if (TC) {
     return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(hi)[off]) +
-           __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(lo)[off]);
+           (lo ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(lo)[off]) : 0.f);
   }
   return reinterpret_cast<const float*>(hi)[off];
 }

@@ -68,9 +68,6 @@ namespace {
 
 constexpr int D = 128;
 constexpr int BM = TC_ROWS;   // 128 query rows (TMEM lanes)
-constexpr int BN = TC_KEYS;   // 96 keys per tile (stream role): two stages of keys AND of values fit
-constexpr int HC = BN / 2;    // columns per row thread
-static_assert(BN % 32 == 0 && BN <= 128, "tile width");
 constexpr float RESCALE_SLACK = 3.f;
 constexpr int ROW_WARPS = 8;
 constexpr int ROW_THREADS = ROW_WARPS * 32;
@@ -81,12 +78,27 @@ constexpr int THREADS = 64 + ROW_THREADS + 32;   // warp 0: TMA producer, warp 1
 constexpr uint32_t SM_Q = 0;                      // Q hi plane (two boxes), then the lo plane
 // stream role: two stages of one key tile {K hi (2 boxes), K lo (2 boxes)}, two stages of V
 constexpr uint32_t SM_K = 65536;
-constexpr uint32_t KS_BOX = BN * 128;             // one [BN rows][64 cols] 16-bit box
-constexpr uint32_t K_STAGE = 4 * KS_BOX;          // K hi (2 boxes), K lo (2 boxes)
-constexpr uint32_t SK_LO = 2 * KS_BOX;
-constexpr uint32_t SM_V = SM_K + 2 * K_STAGE;     // two stages of V (2 boxes each)
-constexpr uint32_t V_STAGE = 2 * KS_BOX;
-static_assert(KS_BOX % 1024 == 0, "swizzled boxes need 1024-byte alignment");
+constexpr uint32_t SM_XCH = 229376;   // both roles: 16 bytes per row for exchanges between the two threads of a row
+// What depends on the precision mode.  SPLIT: rotated Q', K' as two bf16 planes (hi, lo), three score
+// products, key tiles of 96 (two stages of keys AND of values fit beside the Q tile).  Plain: one plane,
+// one product, key tiles of 128.
+template <bool SPLIT>
+struct Tile {
+  static constexpr int BN = SPLIT ? TC_KEYS_SPLIT : TC_KEYS_PLAIN;   // keys per tile (stream role)
+  static constexpr int HC = BN / 2;                                  // columns per row thread
+  static constexpr uint32_t PLANES = SPLIT ? 2 : 1;
+  static constexpr uint32_t KS_BOX = BN * 128;                       // one [BN rows][64 cols] 16-bit box
+  static constexpr uint32_t K_STAGE = 2 * PLANES * KS_BOX;           // K hi (2 boxes) [, K lo (2 boxes)]
+  static constexpr uint32_t SK_LO = 2 * KS_BOX;
+  static constexpr uint32_t SM_V = SM_K + 2 * K_STAGE;               // two stages of V (2 boxes each)
+  static constexpr uint32_t V_STAGE = 2 * KS_BOX;
+  static_assert(BN % 32 == 0 && BN <= 128, "tile width");
+  static_assert(KS_BOX % 1024 == 0, "swizzled boxes need 1024-byte alignment");
+  static_assert(SM_V + 2 * V_STAGE <= SM_XCH, "stream-role tiles overrun");
+  // (A key tile is wider than a block, so no tile lies wholly inside the keys a build excludes: every
+  // tile in [t0, t1) is processed, excluded columns are masked by the row threads.)
+  static_assert(BN > TC_MAX_BLOCK, "a key tile could fall wholly inside the excluded block");
+};
 // The stream role stages its epilogue (128 rows x 512 B, 16-byte chunks XOR-swizzled
 // by the row so row-wise writes and row-wise reads are both conflict-free) in the
 // Q region: in all of it for 128-row units (the next unit's Q load waits for the
@@ -101,9 +113,6 @@ constexpr uint32_t KV_V = 32768;
 constexpr uint32_t K_BOX = 64 * 128;              // one [64 rows][64 cols] 16-bit box
 constexpr uint32_t SM_IO = SM_KV + 2 * KV_STAGE;  // four swizzled boxes of 32 fp32 columns x 128 rows
 constexpr uint32_t IO_BOX = 128 * 128;
-// both roles: 16 bytes per row for exchanges between the two threads of a row
-constexpr uint32_t SM_XCH = 229376;
-static_assert(SM_V + 2 * V_STAGE <= SM_XCH, "stream-role tiles overrun");
 static_assert(SM_IO + 4 * IO_BOX <= SM_XCH, "merge-role staging overruns");
 constexpr uint32_t SM_BAR = SM_XCH + BM * 16;
 constexpr uint32_t SM_TOTAL = SM_BAR + 256;
@@ -258,8 +267,9 @@ struct Unit {
   int base1;              // >= 0: key tiles after the first are counted from this token instead of key_base + BN
 };
 // first key (token index) of key tile t of a unit
-template <int KIND>
+template <int KIND, bool SPLIT>
 __device__ __forceinline__ int tile_key_row(const Unit& un, int t) {
+  constexpr int BN = Tile<SPLIT>::BN;
   if (KIND == KIND_WINDOW && un.base1 >= 0 && t > 0) return un.base1 + (t - 1) * BN;
   return un.key_base + t * BN;
 }
@@ -273,8 +283,10 @@ __device__ __forceinline__ bool unit_row_valid(const Unit& un, int r) {
 // PACKED (a.pack > 1): the units are block queries of several heads side by side in one tile.  A template
 // parameter of the whole kernel, so that the kernel a build or an MHA step runs carries none of the per-row
 // head arithmetic: this kernel is sensitive to its code size.
-template <bool PACKED, int KIND>
+template <bool PACKED, int KIND, bool SPLIT>
 __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs& a, const WorkItem& it, int u) {
+  using TL = Tile<SPLIT>;
+  constexpr int BN = TL::BN;
   constexpr bool STEP = KIND == KIND_STEP;
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
@@ -345,15 +357,13 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
   }
   return un;
 }
-// (A key tile is wider than a block -- BN > TC_MAX_BLOCK -- so no tile lies wholly inside the keys a
-// build excludes: every tile in [t0, t1) is processed, excluded columns are masked by the row threads.)
-static_assert(BN > TC_MAX_BLOCK, "a key tile could fall wholly inside the excluded block");
 
 // S (+)= Q' K'^T as hi.hi + hi.lo + lo.hi; Q planes at q_base (lo plane after the hi
 // plane's two boxes) with boxes of q_box bytes, K planes at k_hi / k_lo with boxes of
 // k_box bytes.  The four base descriptors are built once; each MMA adds a small
 // constant to the start-address field (a single thread issues these back to back,
 // so every instruction saved here shortens the critical path).
+template <bool SPLIT>
 __device__ __forceinline__ void issue_s_mma(uint32_t q_base, uint32_t q_box, uint32_t k_hi, uint32_t k_lo,
                                             uint32_t k_box, uint32_t s_tmem, uint32_t idesc) {
   const uint64_t qd[2] = {smem_desc(q_base, 16, 1024), smem_desc(q_base + 2u * q_box, 16, 1024)};
@@ -361,7 +371,7 @@ __device__ __forceinline__ void issue_s_mma(uint32_t q_base, uint32_t q_box, uin
   const uint32_t qb16 = q_box >> 4, kb16 = k_box >> 4;
   uint32_t acc = 0;
 #pragma unroll
-  for (int term = 0; term < 3; ++term) {
+  for (int term = 0; term < (SPLIT ? 3 : 1); ++term) {   // hi.hi [+ hi.lo + lo.hi]
     const uint64_t qa = qd[term == 2 ? 1 : 0];
     const uint64_t ka = kd[term == 1 ? 1 : 0];
 #pragma unroll
@@ -383,17 +393,19 @@ __device__ __forceinline__ void issue_pv_mma(uint32_t v_base, uint32_t v_box, ui
   for (int ks = 0; ks < ksteps; ++ks)
     mma_ts(o_tmem, p_tmem + 8 * ks, vd + (uint64_t)(ks * (2048 >> 4)), idesc, (ks > 0) ? 1u : accumulate);
 }
+template <bool SPLIT>
 __device__ __forceinline__ void load_kv_tile(const TcMaps& maps, uint32_t kv_base, uint32_t bar, int krow, int kh) {
   static_assert(KV_KLO == 2 * K_BOX && KV_V == 4 * K_BOX, "K hi, K lo and V boxes are contiguous");
-  mbar_expect_tx(bar, 6 * K_BOX);
+  mbar_expect_tx(bar, (SPLIT ? 6 : 4) * K_BOX);   // (one plane: the place of the lo boxes stays empty)
   load_qk_box(kv_base, &maps.k64, bar, krow, kh);
   load_v_box(kv_base + KV_V, &maps.v64, bar, krow, kh);
 }
+template <bool SPLIT>
 __device__ __forceinline__ void load_q_tile(const Cta& c, const TcMaps& maps, int q_rows, int row0, int h,
                                             bool packed = false) {
   const uint32_t bar = c.bar(BAR_Q_FULL);
   const uint32_t box = (uint32_t)q_rows * 128u;
-  mbar_expect_tx(bar, 4 * box);
+  mbar_expect_tx(bar, (SPLIT ? 4 : 2) * box);
   if (packed) tma_load_5d(c.base + SM_Q, &maps.q_pack, bar, 0, row0, h, 0, 0);   // heads h, h + 1, ... side by side
   else load_qk_box(c.base + SM_Q, q_rows == 64 ? &maps.q64 : &maps.q, bar, row0, h);
 }
@@ -410,7 +422,7 @@ struct TileCursor {
   Unit un;
   bool valid, q_done, loads_q;
 };
-template <bool PACKED, int KIND>
+template <bool PACKED, int KIND, bool SPLIT>
 __device__ __forceinline__ void cursor_load_unit(const Geometry& g, const AttnArgs& a, TileCursor& cu, int n_units) {
   constexpr bool STEP = KIND == KIND_STEP;
   constexpr bool WINDOW = KIND == KIND_WINDOW;
@@ -418,11 +430,11 @@ __device__ __forceinline__ void cursor_load_unit(const Geometry& g, const AttnAr
   cu.valid = cu.u < n_units;
   if (!cu.valid) return;
   cu.it = load_item(a.items + cu.u / (PACKED ? a.stream_slots : g.Hq));
-  cu.un = decode_stream<PACKED, KIND>(g, a, cu.it, cu.u);
+  cu.un = decode_stream<PACKED, KIND, SPLIT>(g, a, cu.it, cu.u);
   cu.t = cu.un.t0;
   cu.q_done = !cu.loads_q;
 }
-template <bool PACKED, int KIND>
+template <bool PACKED, int KIND, bool SPLIT>
 __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs& a, TileCursor& cu, int stride,
                                                int n_units) {
   constexpr bool STEP = KIND == KIND_STEP;
@@ -436,24 +448,27 @@ __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs
   while (cu.valid && cu.t >= cu.un.t1 && cu.q_done) {
     cu.u += stride;
     ++cu.uu;
-    cursor_load_unit<PACKED, KIND>(g, a, cu, n_units);
+    cursor_load_unit<PACKED, KIND, SPLIT>(g, a, cu, n_units);
   }
 }
 
-template <bool PACKED, int KIND>
+template <bool PACKED, int KIND, bool SPLIT>
 __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a,
                                 int first, int stride, int n_units, WorkItem it) {
+  using TL = Tile<SPLIT>;
+  constexpr int BN = TL::BN;
+  constexpr uint32_t KS_BOX = TL::KS_BOX, K_STAGE = TL::K_STAGE, SM_V = TL::SM_V, V_STAGE = TL::V_STAGE;
   constexpr bool STEP = KIND == KIND_STEP;
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
   // three independent cursors: Q tiles (one per unit), key tiles, value tiles
   TileCursor cq, ck, cv;
   cq.u = first; cq.uu = 0; cq.jj = 0; cq.loads_q = true;
-  cursor_load_unit<PACKED, KIND>(g, a, cq, n_units);
+  cursor_load_unit<PACKED, KIND, SPLIT>(g, a, cq, n_units);
   ck = cq;
   ck.loads_q = false;  // the key and value cursors never load Q
   ck.q_done = true;
-  if (ck.valid && ck.t >= ck.un.t1) cursor_advance<PACKED, KIND>(g, a, ck, stride, n_units);
+  if (ck.valid && ck.t >= ck.un.t1) cursor_advance<PACKED, KIND, SPLIT>(g, a, ck, stride, n_units);
   cv = ck;
   // What the RoPE kernel launched just before this one writes must not be loaded
   // before that grid has completed (this kernel may have started early): in a step
@@ -477,15 +492,15 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         mbar_arrive(c.bar(BAR_Q_FULL));
         cq.q_done = true;
         cq.t = cq.un.t1;
-        cursor_advance<PACKED, KIND>(g, a, cq, stride, n_units);
+        cursor_advance<PACKED, KIND, SPLIT>(g, a, cq, stride, n_units);
         did = true;
       } else if (!dep_done) {
         blocked_on_dep = true;
       } else if (cq.uu == 0 || mbar_test(c.bar(BAR_Q_FREE), (cq.uu - 1) & 1)) {
-        load_q_tile(c, maps, cq.un.q_rows, cq.un.row0, cq.un.h, cq.un.rh != 0);
+        load_q_tile<SPLIT>(c, maps, cq.un.q_rows, cq.un.row0, cq.un.h, cq.un.rh != 0);
         cq.q_done = true;
         cq.t = cq.un.t1;
-        cursor_advance<PACKED, KIND>(g, a, cq, stride, n_units);
+        cursor_advance<PACKED, KIND, SPLIT>(g, a, cq, stride, n_units);
         // a build's Q tiles come from HBM once the batch outgrows L2: the next unit's tile is asked
         // into L2 a whole unit ahead of its load
         if (!STEP && cq.valid) tma_prefetch_5d(&maps.q, 0, cq.un.row0, 0, cq.un.h, 0);
@@ -497,12 +512,12 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
       if (!dep_done && tile_depends(ck)) {
         blocked_on_dep = true;
       } else if (kuse == 0 || mbar_test(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE), (kuse - 1) & 1)) {
-        const int krow = tile_key_row<KIND>(ck.un, ck.t);
+        const int krow = tile_key_row<KIND, SPLIT>(ck.un, ck.t);
         const uint32_t bar = c.bar(sk ? BAR_K_FULL1 : BAR_K_FULL);
         const uint32_t khi = c.base + SM_K + sk * K_STAGE;
-        mbar_expect_tx(bar, 4 * KS_BOX);
-        load_qk_box(khi, &maps.k, bar, krow, ck.un.kh);  // the lo plane lands at khi + SK_LO
-        cursor_advance<PACKED, KIND>(g, a, ck, stride, n_units);
+        mbar_expect_tx(bar, K_STAGE);
+        load_qk_box(khi, &maps.k, bar, krow, ck.un.kh);  // (split: the lo plane lands at khi + SK_LO)
+        cursor_advance<PACKED, KIND, SPLIT>(g, a, ck, stride, n_units);
         did = true;
       }
     }
@@ -511,11 +526,11 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
       if (!dep_done && tile_depends(cv)) {
         blocked_on_dep = true;
       } else if (vuse == 0 || mbar_test(c.bar(sv ? BAR_V_FREE1 : BAR_V_FREE), (vuse - 1) & 1)) {
-        const int krow = tile_key_row<KIND>(cv.un, cv.t);
+        const int krow = tile_key_row<KIND, SPLIT>(cv.un, cv.t);
         const uint32_t bar = c.bar(sv ? BAR_V_FULL1 : BAR_V_FULL), vb = c.base + SM_V + sv * V_STAGE;
         mbar_expect_tx(bar, 2 * KS_BOX);
         load_v_box(vb, &maps.v, bar, krow, cv.un.kh);
-        cursor_advance<PACKED, KIND>(g, a, cv, stride, n_units);
+        cursor_advance<PACKED, KIND, SPLIT>(g, a, cv, stride, n_units);
         did = true;
       }
     }
@@ -548,9 +563,12 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
 // Scores of tile j need its keys and the score buffer of tile j - 2 read (= the probabilities of tile
 // j - 2 written); P~V of tile j needs its probabilities and its values.  Each code block exists once
 // (the unrolled MMA sequences are large, and cold instruction fetches are slow).
-template <bool PACKED, int KIND>
+template <bool PACKED, int KIND, bool SPLIT>
 __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
                                   int n_units, WorkItem it) {
+  using TL = Tile<SPLIT>;
+  constexpr int BN = TL::BN;
+  constexpr uint32_t KS_BOX = TL::KS_BOX, K_STAGE = TL::K_STAGE, SK_LO = TL::SK_LO;
   constexpr bool STEP = KIND == KIND_STEP;
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
@@ -560,7 +578,7 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
-    const Unit un = decode_stream<PACKED, KIND>(g, a, it, u);
+    const Unit un = decode_stream<PACKED, KIND, SPLIT>(g, a, it, u);
     const uint32_t q_box = (uint32_t)un.q_rows * 128u;
     const int n_tiles = un.t1 - un.t0;
     if (!wait_bar(c, BAR_Q_FULL, uu & 1, LOC_WAIT_Q)) return;
@@ -573,7 +591,7 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
       if (!wait_bar(c, sk ? BAR_K_FULL1 : BAR_K_FULL, (js >> 1) & 1u, LOC_WAIT_K)) return;
       const uint32_t khi = c.base + SM_K + sk * K_STAGE, klo = khi + SK_LO;
       tc_fence_after();
-      issue_s_mma(c.base + SM_Q, q_box, khi, klo, KS_BOX, c.tmem + TS_S + 128 * b, IDESC_S);
+      issue_s_mma<SPLIT>(c.base + SM_Q, q_box, khi, klo, KS_BOX, c.tmem + TS_S + 128 * b, IDESC_S);
       tc_commit(c.bar(BAR_S_FULL + b));
       tc_commit(c.bar(sk ? BAR_K_FREE1 : BAR_K_FREE));
     }
@@ -582,9 +600,12 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   }
 }
 
-template <bool PACKED, int KIND>
+template <bool PACKED, int KIND, bool SPLIT>
 __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride,
                               int n_units, WorkItem it) {
+  using TL = Tile<SPLIT>;
+  constexpr int BN = TL::BN;
+  constexpr uint32_t KS_BOX = TL::KS_BOX, SM_V = TL::SM_V, V_STAGE = TL::V_STAGE;
   constexpr bool STEP = KIND == KIND_STEP;
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
@@ -593,7 +614,7 @@ __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
-    const Unit un = decode_stream<PACKED, KIND>(g, a, it, u);
+    const Unit un = decode_stream<PACKED, KIND, SPLIT>(g, a, it, u);
     const int n_tiles = un.t1 - un.t0;
     // O~ of the previous unit has been read by the row threads.  (A unit without key tiles issues nothing
     // and does not wait: the row threads cannot complete this unit's phase of the barrier before the
@@ -752,9 +773,12 @@ __device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs
   }
 }
 
-template <bool PACKED, int KIND>
+template <bool PACKED, int KIND, bool SPLIT>
 __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units,
                             WorkItem it) {
+  using TL = Tile<SPLIT>;
+  constexpr int BN = TL::BN;
+  constexpr int HC = TL::HC;
   constexpr bool STEP = KIND == KIND_STEP;
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
@@ -772,7 +796,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     ++uu;
     WorkItem nxt = it;
     if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
-    const Unit un = decode_stream<PACKED, KIND>(g, a, it, u);
+    const Unit un = decode_stream<PACKED, KIND, SPLIT>(g, a, it, u);
     it = nxt;
     if (u == first && STEP && a.q_raw != nullptr) {
       // The CTA's first unit: rotate the block's queries of this (sequence, head) here,
@@ -802,8 +826,10 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         uint8_t* const q0 = c.gen + SM_Q + qi * 128 + ((ch ^ (qi & 7)) << 4);
         *reinterpret_cast<uint4*>(q0) = h1;                 // hi plane, features [0, 64)
         *reinterpret_cast<uint4*>(q0 + box) = h2;           // hi plane, features [64, 128)
-        *reinterpret_cast<uint4*>(q0 + 2 * box) = l1;       // lo plane
-        *reinterpret_cast<uint4*>(q0 + 3 * box) = l2;
+        if (SPLIT) {
+          *reinterpret_cast<uint4*>(q0 + 2 * box) = l1;     // lo plane
+          *reinterpret_cast<uint4*>(q0 + 3 * box) = l2;
+        }
       }
       fence_async_smem();  // the MMA reads shared memory through the async proxy
       mbar_arrive(c.bar(BAR_QC));
@@ -895,7 +921,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
             if (half == 0) { a.snap.m[srow] = m_ref; a.snap.l[srow] = l_sum; }
           }
         }
-        const int tile_lo = tile_key_row<KIND>(un, t);
+        const int tile_lo = tile_key_row<KIND, SPLIT>(un, t);
         const int v_lo = max(un.k0 - tile_lo, 0), v_hi = min(un.k1 - tile_lo, BN);
         const int e_lo = un.x0 - tile_lo, e_hi = un.x1 - tile_lo;
         const bool all_valid = v_lo == 0 && v_hi == BN && (un.x1 <= un.x0 || e_hi <= 0 || e_lo >= BN);
@@ -1278,6 +1304,7 @@ __device__ __forceinline__ void store_tail_row(const AttnArgs& a, const uint8_t*
 // ===========================================================================
 // merge role: fixed queries x block keys, merged into the cached state
 // ===========================================================================
+template <bool SPLIT>
 __device__ void merge_producer(const Cta& c, const TcMaps& maps, const Geometry& g, const AttnArgs& a, int first,
                                int stride, int n_units, WorkItem it) {
   int uu = 0;
@@ -1287,7 +1314,7 @@ __device__ void merge_producer(const Cta& c, const TcMaps& maps, const Geometry&
     const int h = u % g.Hq;
     const int b = uu & 1, k = uu >> 1;
     if (uu >= 1 && !wait_bar(c, BAR_Q_FREE, (uu - 1) & 1, LOC_WAIT_Q)) return;
-    load_q_tile(c, maps, BM, it.row0, h);
+    load_q_tile<SPLIT>(c, maps, BM, it.row0, h);
     if (uu == 0) {
       // first unit: the cached O~ tile does not depend on the RoPE kernel launched
       // just before this one, the block's keys and values do: wait for that grid
@@ -1297,13 +1324,13 @@ __device__ void merge_producer(const Cta& c, const TcMaps& maps, const Geometry&
       for (int cb = 0; cb < 4; ++cb)
         tma_load_3d(c.base + SM_IO + cb * IO_BOX, &maps.st_o, c.bar(BAR_IO_FULL), 32 * cb, it.row0, h);
       grid_dependency_wait();
-      load_kv_tile(maps, c.base + SM_KV, c.bar(BAR_KV_FULL), it.blk_start, h / g.group);
+      load_kv_tile<SPLIT>(maps, c.base + SM_KV, c.bar(BAR_KV_FULL), it.blk_start, h / g.group);
     } else {
       // later units: keys first (their stage frees early), then the cached O~
       // tile (four boxes of 32 features x 128 rows; rows past nrows are read but
       // never used) once the previous unit's output has left the staging tile
       if (k >= 1 && !wait_bar(c, BAR_KV_FREE + b, (k - 1) & 1, LOC_WAIT_K)) return;
-      load_kv_tile(maps, c.base + SM_KV + b * KV_STAGE, c.bar(BAR_KV_FULL + b), it.blk_start, h / g.group);
+      load_kv_tile<SPLIT>(maps, c.base + SM_KV + b * KV_STAGE, c.bar(BAR_KV_FULL + b), it.blk_start, h / g.group);
       if (!wait_bar(c, BAR_IO_FREE, (uu - 1) & 1, LOC_WAIT_V)) return;
       mbar_expect_tx(c.bar(BAR_IO_FULL), 4 * IO_BOX);
 #pragma unroll
@@ -1314,6 +1341,7 @@ __device__ void merge_producer(const Cta& c, const TcMaps& maps, const Geometry&
   }
 }
 
+template <bool SPLIT>
 __device__ void merge_mma(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units) {
   const int n_s = (g.block_len + 15) & ~15;  // score columns (keys), a multiple of 16
   const uint32_t idesc_s = idesc_f16(1u, 0u, BM, (uint32_t)n_s);
@@ -1322,7 +1350,7 @@ __device__ void merge_mma(const Cta& c, const Geometry& g, const AttnArgs& a, in
     if (!wait_bar(c, BAR_Q_FULL, 0, LOC_WAIT_Q)) return;
     if (!wait_bar(c, BAR_KV_FULL, 0, LOC_WAIT_K)) return;
     tc_fence_after();
-    issue_s_mma(c.base + SM_Q, BM * 128u, c.base + SM_KV, c.base + SM_KV + KV_KLO, K_BOX, c.tmem + TM_S, idesc_s);
+    issue_s_mma<SPLIT>(c.base + SM_Q, BM * 128u, c.base + SM_KV, c.base + SM_KV + KV_KLO, K_BOX, c.tmem + TM_S, idesc_s);
     tc_commit(c.bar(BAR_S_FULL));
     tc_commit(c.bar(BAR_Q_FREE));
   }
@@ -1340,7 +1368,7 @@ __device__ void merge_mma(const Cta& c, const Geometry& g, const AttnArgs& a, in
       if (!wait_bar(c, BAR_Q_FULL, (uu + 1) & 1, LOC_WAIT_Q)) return;
       if (!wait_bar(c, BAR_KV_FULL + bn, ((uu + 1) >> 1) & 1, LOC_WAIT_K)) return;
       tc_fence_after();
-      issue_s_mma(c.base + SM_Q, BM * 128u, c.base + SM_KV + bn * KV_STAGE, c.base + SM_KV + bn * KV_STAGE + KV_KLO, K_BOX,
+      issue_s_mma<SPLIT>(c.base + SM_Q, BM * 128u, c.base + SM_KV + bn * KV_STAGE, c.base + SM_KV + bn * KV_STAGE + KV_KLO, K_BOX,
                   c.tmem + TM_S + 64 * bn, idesc_s);
       tc_commit(c.bar(BAR_S_FULL + bn));
       tc_commit(c.bar(BAR_Q_FREE));
@@ -1478,12 +1506,13 @@ __device__ __forceinline__ DUnit deep_unit(const Cta& c, int i) {
   return DUnit{v.x, v.y, v.z, v.w & 0xFFFF, v.w >> 16};
 }
 
+template <bool SPLIT>
 __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& g, int n_my, bool kv_computed,
                               bool out_bf16) {
   if (n_my == 0) return;
   auto load_q = [&](int i) {
     const DUnit un = deep_unit(c, i);
-    load_q_tile(c, maps, BM, un.row0, un.h);
+    load_q_tile<SPLIT>(c, maps, BM, un.row0, un.h);
   };
   auto load_io = [&](int i) {
     const DUnit un = deep_unit(c, i);
@@ -1497,7 +1526,7 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
     const DUnit un = deep_unit(c, i);
     const uint32_t bar = c.bar(BAR_KV_FULL), kb = c.base + DM_K;
     const int kh = un.h / g.group;
-    mbar_expect_tx(bar, 4 * DM_KBOX);
+    mbar_expect_tx(bar, (SPLIT ? 4 : 2) * DM_KBOX);
     load_qk_box(kb, &maps.k32, bar, un.blk_start, kh);
   };
   auto load_v = [&](int i) {
@@ -1571,6 +1600,7 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
   bulk_wait_read();  // shared memory stays valid until the last store has read it
 }
 
+template <bool SPLIT>
 __device__ void deep_mma(const Cta& c, const Geometry& g, int n_my, bool kv_computed) {
   if (n_my == 0) return;
   const int n_s = (g.block_len + 15) & ~15;
@@ -1580,7 +1610,7 @@ __device__ void deep_mma(const Cta& c, const Geometry& g, int n_my, bool kv_comp
   if (!wait_bar(c, BAR_KV_FULL, 0, LOC_WAIT_K)) return;
   if (kv_computed && !wait_bar(c, BAR_QC, 0, LOC_WAIT_K)) return;  // keys and values written by the row threads
   tc_fence_after();
-  issue_s_mma(c.base + SM_Q, BM * 128u, kb, kb + 2 * DM_KBOX, DM_KBOX, c.tmem + TM_S, idesc_s);
+  issue_s_mma<SPLIT>(c.base + SM_Q, BM * 128u, kb, kb + 2 * DM_KBOX, DM_KBOX, c.tmem + TM_S, idesc_s);
   tc_commit(c.bar(BAR_S_FULL));
   tc_commit(c.bar(BAR_Q_FREE));
   tc_commit(c.bar(BAR_KV_FREE));
@@ -1598,7 +1628,7 @@ __device__ void deep_mma(const Cta& c, const Geometry& g, int n_my, bool kv_comp
       if (!wait_bar(c, BAR_Q_FULL, (uu + 1) & 1, LOC_WAIT_Q)) return;
       if (!wait_bar(c, BAR_KV_FULL, (uu + 1) & 1, LOC_WAIT_K)) return;
       tc_fence_after();
-      issue_s_mma(c.base + SM_Q, BM * 128u, kb, kb + 2 * DM_KBOX, DM_KBOX, c.tmem + TM_S + 64 * bn, idesc_s);
+      issue_s_mma<SPLIT>(c.base + SM_Q, BM * 128u, kb, kb + 2 * DM_KBOX, DM_KBOX, c.tmem + TM_S + 64 * bn, idesc_s);
       tc_commit(c.bar(BAR_S_FULL + bn));
       tc_commit(c.bar(BAR_Q_FREE));
       tc_commit(c.bar(BAR_KV_FREE));
@@ -1606,6 +1636,7 @@ __device__ void deep_mma(const Cta& c, const Geometry& g, int n_my, bool kv_comp
   }
 }
 
+template <bool SPLIT>
 __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, int n_my) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int quad = warp & 3;
@@ -1652,8 +1683,10 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
       uint8_t* const k0 = c.gen + DM_K + ki * 128 + ((ch ^ (ki & 7)) << 4);
       *reinterpret_cast<uint4*>(k0) = h1;
       *reinterpret_cast<uint4*>(k0 + DM_KBOX) = h2;
-      *reinterpret_cast<uint4*>(k0 + 2 * DM_KBOX) = l1;
-      *reinterpret_cast<uint4*>(k0 + 3 * DM_KBOX) = l2;
+      if (SPLIT) {
+        *reinterpret_cast<uint4*>(k0 + 2 * DM_KBOX) = l1;
+        *reinterpret_cast<uint4*>(k0 + 3 * DM_KBOX) = l2;
+      }
       // values: the same two 8-feature chunks of row ki, unrotated
       float v1[8], v2[8];
       rope_load8(a.v_raw, soff + c0, true, v1);
@@ -1669,7 +1702,7 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
       const uint4 z = make_uint4(0u, 0u, 0u, 0u);
       uint8_t* const k0 = c.gen + DM_K + ki * 128 + ((ch ^ (ki & 7)) << 4);
       *reinterpret_cast<uint4*>(k0) = z; *reinterpret_cast<uint4*>(k0 + DM_KBOX) = z;
-      *reinterpret_cast<uint4*>(k0 + 2 * DM_KBOX) = z; *reinterpret_cast<uint4*>(k0 + 3 * DM_KBOX) = z;
+      if (SPLIT) { *reinterpret_cast<uint4*>(k0 + 2 * DM_KBOX) = z; *reinterpret_cast<uint4*>(k0 + 3 * DM_KBOX) = z; }
       uint8_t* const v0 = c.gen + DM_V + ki * 128 + ((ch ^ (ki & 7)) << 4);
       *reinterpret_cast<uint4*>(v0) = z; *reinterpret_cast<uint4*>(v0 + DM_KBOX) = z;
     }
@@ -1745,7 +1778,7 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
   }
 }
 
-template <bool PACKED, int KIND, bool DEEP>
+template <bool PACKED, int KIND, bool DEEP, bool SPLIT>
 __global__ void __launch_bounds__(THREADS, 1)
 tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const AttnArgs a) {
   constexpr bool STEP = KIND == KIND_STEP;
@@ -1841,23 +1874,23 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
 
   if (warp == 0) {
     if (stream) {
-      if (tid == 0) stream_producer<PACKED, KIND>(c, maps, g, a, first, stride, n_units, it0);
+      if (tid == 0) stream_producer<PACKED, KIND, SPLIT>(c, maps, g, a, first, stride, n_units, it0);
     } else if (deep) {
-      if (tid == 0) deep_producer(c, maps, g, n_my, a.k_raw != nullptr, a.out_bf16 != 0);
+      if (tid == 0) deep_producer<SPLIT>(c, maps, g, n_my, a.k_raw != nullptr, a.out_bf16 != 0);
     } else {
-      if (tid == 0) merge_producer(c, maps, g, a, first, stride, n_units, it0);
+      if (tid == 0) merge_producer<SPLIT>(c, maps, g, a, first, stride, n_units, it0);
     }
   } else if (warp == 1) {
     if (tid == 32) {
-      if (stream) stream_mma_scores<PACKED, KIND>(c, g, a, first, stride, n_units, it0);
-      else if (deep) deep_mma(c, g, n_my, a.k_raw != nullptr);
-      else merge_mma(c, g, a, first, stride, n_units);
+      if (stream) stream_mma_scores<PACKED, KIND, SPLIT>(c, g, a, first, stride, n_units, it0);
+      else if (deep) deep_mma<SPLIT>(c, g, n_my, a.k_raw != nullptr);
+      else merge_mma<SPLIT>(c, g, a, first, stride, n_units);
     }
   } else if (warp == 10) {
-    if (tid == 320 && stream) stream_mma_pv<PACKED, KIND>(c, g, a, first, stride, n_units, it0);
+    if (tid == 320 && stream) stream_mma_pv<PACKED, KIND, SPLIT>(c, g, a, first, stride, n_units, it0);
   } else {
-    if (stream) stream_rows<PACKED, KIND>(c, g, a, first, stride, n_units, it0);
-    else if (deep) deep_rows(c, g, a, n_my);
+    if (stream) stream_rows<PACKED, KIND, SPLIT>(c, g, a, first, stride, n_units, it0);
+    else if (deep) deep_rows<SPLIT>(c, g, a, n_my);
     else merge_rows(c, maps, g, a, first, stride, n_units, it0);
     bulk_wait_read();
   }
@@ -1913,12 +1946,13 @@ bool make_f32_map(CUtensorMap* m, void* base, cuuint64_t d1, cuuint64_t d2, cuui
 // Split-bf16 planes [plane][H][2][Tp][64] (hi plane at `base`, lo plane `plane_elems` further) as a 5-D
 // tensor; fp16 values [H][2][Tp][64] as a 4-D tensor.  Box: `box_rows` rows of one head, both feature
 // halves (and both planes).
-bool make_qk_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* err, int errlen) {
+bool make_qk_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, int planes, char* err, int errlen) {
   EncodeTiledFn enc = get_encode();
   if (!enc) { snprintf(err, errlen, "cuTensorMapEncodeTiled entry point not found"); return false; }
-  cuuint64_t dims[5] = {64, (cuuint64_t)Tp, 2, (cuuint64_t)H, 2};
+  // (with one plane the last dimension has extent 1: the same instruction loads half as much)
+  cuuint64_t dims[5] = {64, (cuuint64_t)Tp, 2, (cuuint64_t)H, (cuuint64_t)planes};
   cuuint64_t strides[4] = {128, (cuuint64_t)Tp * 128, (cuuint64_t)Tp * 256, (cuuint64_t)H * Tp * 256};
-  cuuint32_t box[5] = {64, (cuuint32_t)box_rows, 2, 1, 2};
+  cuuint32_t box[5] = {64, (cuuint32_t)box_rows, 2, 1, (cuuint32_t)planes};
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1928,12 +1962,12 @@ bool make_qk_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* 
 }
 // The same planes with the head dimension inside the half dimension, so that a box of `pack` heads x
 // `rows` rows lands as one [plane][half][pack * rows][64] tile.
-bool make_qpack_map(CUtensorMap* m, void* base, int H, int Tp, int rows, int pack, char* err, int errlen) {
+bool make_qpack_map(CUtensorMap* m, void* base, int H, int Tp, int rows, int pack, int planes, char* err, int errlen) {
   EncodeTiledFn enc = get_encode();
   if (!enc) { snprintf(err, errlen, "cuTensorMapEncodeTiled entry point not found"); return false; }
-  cuuint64_t dims[5] = {64, (cuuint64_t)Tp, (cuuint64_t)H, 2, 2};
+  cuuint64_t dims[5] = {64, (cuuint64_t)Tp, (cuuint64_t)H, 2, (cuuint64_t)planes};
   cuuint64_t strides[4] = {128, (cuuint64_t)Tp * 256, (cuuint64_t)Tp * 128, (cuuint64_t)H * Tp * 256};
-  cuuint32_t box[5] = {64, (cuuint32_t)rows, (cuuint32_t)pack, 2, 2};
+  cuuint32_t box[5] = {64, (cuuint32_t)rows, (cuuint32_t)pack, 2, (cuuint32_t)planes};
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, base, dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1957,13 +1991,26 @@ bool make_v_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* e
 
 }  // namespace
 
+namespace {
+// twelve instantiations: {split, plain operands} x {build / full recompute; build over key windows; the
+// step of an MHA and of a GQA model, each with either variant of the merge role}
+template <bool SPLIT>
+const void* const* kernel_table() {
+  static const void* const t[6] = {
+      (const void*)tc_attn_kernel<false, KIND_BUILD, false, SPLIT>, (const void*)tc_attn_kernel<false, KIND_WINDOW, false, SPLIT>,
+      (const void*)tc_attn_kernel<false, KIND_STEP, false, SPLIT>,  (const void*)tc_attn_kernel<false, KIND_STEP, true, SPLIT>,
+      (const void*)tc_attn_kernel<true, KIND_STEP, false, SPLIT>,   (const void*)tc_attn_kernel<true, KIND_STEP, true, SPLIT>};
+  return t;
+}
+}  // namespace
+
 cudaError_t tc_prepare() {
-  const void* kernels[] = {(const void*)tc_attn_kernel<false, KIND_BUILD, false>, (const void*)tc_attn_kernel<false, KIND_WINDOW, false>,
-                           (const void*)tc_attn_kernel<false, KIND_STEP, false>, (const void*)tc_attn_kernel<false, KIND_STEP, true>,
-                           (const void*)tc_attn_kernel<true, KIND_STEP, false>, (const void*)tc_attn_kernel<true, KIND_STEP, true>};
-  for (const void* k : kernels) {
-    cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
-    if (e != cudaSuccess) return e;
+  for (int split = 0; split < 2; ++split) {
+    const void* const* t = split ? kernel_table<true>() : kernel_table<false>();
+    for (int i = 0; i < 6; ++i) {
+      cudaError_t e = cudaFuncSetAttribute(t[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
+      if (e != cudaSuccess) return e;
+    }
   }
   return cudaSuccess;
 }
@@ -1977,19 +2024,21 @@ bool tc_set_out(TcMaps* m, const Geometry& g, float* out, bool out_bf16, char* e
   return true;
 }
 
-TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, char* err, int errlen) {
+TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, bool split, char* err, int errlen) {
   TcMaps* m = new TcMaps();
   m->out_ptr = nullptr;
   m->out = CUtensorMap{};
-  // (the lo planes follow the hi planes at a fixed distance: see alloc_rot)
-  bool ok = make_qk_map(&m->q, rot.q_hi, g.Hq, g.Tp, BM, err, errlen) &&
-            make_qk_map(&m->q64, rot.q_hi, g.Hq, g.Tp, 64, err, errlen) &&
+  // (split: the lo planes follow the hi planes at a fixed distance, see alloc_rot)
+  const int planes = split ? 2 : 1;
+  const int bn = tc_keys(split);
+  bool ok = make_qk_map(&m->q, rot.q_hi, g.Hq, g.Tp, BM, planes, err, errlen) &&
+            make_qk_map(&m->q64, rot.q_hi, g.Hq, g.Tp, 64, planes, err, errlen) &&
             make_qpack_map(&m->q_pack, rot.q_hi, g.Hq, g.Tp, g.block_len <= 32 ? 32 : 64,
-                           std::max(1, std::min(g.block_len <= 32 ? 4 : 2, g.group)), err, errlen) &&
-            make_qk_map(&m->k, rot.k_hi, g.Hkv, g.Tp, BN, err, errlen) &&
-            make_qk_map(&m->k64, rot.k_hi, g.Hkv, g.Tp, 64, err, errlen) &&
-            make_qk_map(&m->k32, rot.k_hi, g.Hkv, g.Tp, 32, err, errlen) &&
-            make_v_map(&m->v, rot.v, g.Hkv, g.Tp, BN, err, errlen) &&
+                           std::max(1, std::min(g.block_len <= 32 ? 4 : 2, g.group)), planes, err, errlen) &&
+            make_qk_map(&m->k, rot.k_hi, g.Hkv, g.Tp, bn, planes, err, errlen) &&
+            make_qk_map(&m->k64, rot.k_hi, g.Hkv, g.Tp, 64, planes, err, errlen) &&
+            make_qk_map(&m->k32, rot.k_hi, g.Hkv, g.Tp, 32, planes, err, errlen) &&
+            make_v_map(&m->v, rot.v, g.Hkv, g.Tp, bn, err, errlen) &&
             make_v_map(&m->v64, rot.v, g.Hkv, g.Tp, 64, err, errlen) &&
             make_v_map(&m->v32, rot.v, g.Hkv, g.Tp, 32, err, errlen) &&
             make_f32_map(&m->st_o, state_o, (cuuint64_t)g.Tp, (cuuint64_t)g.Hq, BM, 1, err, errlen);
@@ -2013,18 +2062,12 @@ cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* map
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = a.no_pdl ? 0 : 1;
-  // six instantiations: build / full recompute; build over key windows; the step of an MHA and of a
-  // GQA model, each with either variant of the merge role
-  if (a.mode != MODE_STEP) {
-    if (a.window) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, KIND_WINDOW, false>, *maps, g, a);
-    return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, KIND_BUILD, false>, *maps, g, a);
-  }
-  if (a.pack > 1) {
-    if (a.merge_deep) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true, KIND_STEP, true>, *maps, g, a);
-    return cudaLaunchKernelEx(&cfg, tc_attn_kernel<true, KIND_STEP, false>, *maps, g, a);
-  }
-  if (a.merge_deep) return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, KIND_STEP, true>, *maps, g, a);
-  return cudaLaunchKernelEx(&cfg, tc_attn_kernel<false, KIND_STEP, false>, *maps, g, a);
+  const void* const* t = a.split ? kernel_table<true>() : kernel_table<false>();
+  int which;
+  if (a.mode != MODE_STEP) which = a.window ? 1 : 0;
+  else which = (a.pack > 1 ? 4 : 2) + (a.merge_deep ? 1 : 0);
+  void* params[3] = {const_cast<TcMaps*>(maps), const_cast<Geometry*>(&g), const_cast<AttnArgs*>(&a)};
+  return cudaLaunchKernelExC(&cfg, t[which], params);
 }
 
 }  // namespace lacache

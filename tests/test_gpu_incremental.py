@@ -42,10 +42,10 @@ def _state(ctx, wl):
     return m.double(), l.double(), o.double()
 
 
-def _run(wl, seed):
+def _run(wl, seed, **ctx_kw):
     sch = SyntheticSchedule(wl, seed=seed)
-    inc = make_ctx(wl, engine=binding.ENGINE_TCGEN05)
-    ref = make_ctx(wl, engine=binding.ENGINE_TCGEN05)
+    inc = make_ctx(wl, engine=binding.ENGINE_TCGEN05, **ctx_kw)
+    ref = make_ctx(wl, engine=binding.ENGINE_TCGEN05, **ctx_kw)
     out, lse = new_outputs(wl)
     rout, rlse = new_outputs(wl)
     fin = None
@@ -90,6 +90,23 @@ def _run(wl, seed):
 @pytest.mark.parametrize("case", sorted(CASES))
 def test_advanced_context_serves_steps_like_a_rebuilt_one(case):
     _run(small_workload(name=case, **CASES[case]), seed=21)
+
+
+@pytest.mark.parametrize("case", ["gqa64", "long", "noprompt", "mha64"])
+def test_advanced_context_with_plain_operands(case):
+    """The same walk with precision_mode = plain (128-key tiles in the key-window units) on the value
+    distribution that mode is meant for."""
+    kw = dict(CASES[case]) if case in CASES else dict(prompt_lens=(700, 333, 61), gen_len=192, block_len=64, steps=1,
+                                                       hq=4, hkv=4)
+    kw["scale_mode"] = "inv_sqrt_d"
+    _run(small_workload(name=case, **kw), seed=22, precision_mode=binding.PRECISION_PLAIN)
+
+
+@pytest.mark.parametrize("block_len", [48, 64])
+def test_advanced_context_mha_blocks_of_48_and_64_rows(block_len):
+    """No grouped heads, blocks of 33..64 rows, per-head scales up to 2, ragged, long prompts."""
+    _run(small_workload(name="mha%d" % block_len, prompt_lens=(700, 333, 61), gen_len=192, block_len=block_len, steps=2,
+                        hq=4, hkv=4, scale_mode="per_head_u(0.5,2)"), seed=23)
 
 
 def test_incremental_build_at_a_later_block_then_advance():

@@ -352,7 +352,8 @@ def test_step_split_over_several_launches(cfg, monkeypatch):
     ctx.destroy()
 
 
-def test_large_batch_extension_full_size():
+@pytest.mark.parametrize("mode", ["split", "plain"])
+def test_large_batch_extension_full_size(mode):
     """The large-batch extension (256 sequences, 28/4 heads, ~287k tokens) at full size, in the
     launch configuration the bench times: the step's fixed rows exceed one launch of the pipelined
     merge variant and go out in several.  Cached path vs full recompute on every row; vs the oracle
@@ -361,7 +362,8 @@ def test_large_batch_extension_full_size():
     wl = WORKLOADS[6]
     S = 3
     sched = DeviceSchedule(wl, 17, torch.device("cuda"), S)
-    ctx = make_ctx(wl, engine=ENGINES["tc"])
+    ctx = make_ctx(wl, engine=ENGINES["tc"],
+                   precision_mode=binding.PRECISION_PLAIN if mode == "plain" else binding.PRECISION_SPLIT)
     q, k, v = sched.full[0]
     ctx.build(0, q, k, v)
     out, lse = new_outputs(wl)
@@ -394,13 +396,27 @@ def test_large_batch_extension_full_size():
     ctx.destroy()
 
 
+@pytest.mark.parametrize("case", sorted(SMALL) + ["mha64", "long48"])
+def test_plain_operands_small_cases(case):
+    """precision_mode = plain (one bf16 plane of the rotated Q', K', one score product, 128-key tiles) on
+    the value distribution it is meant for, N(0,1)/sqrt(d): same tolerances against the oracle and
+    against the GPU full recompute as the split mode."""
+    extra = {"mha64": dict(prompt_lens=(700, 333, 61), gen_len=192, block_len=64, steps=2, hq=4, hkv=4),
+             "long48": dict(prompt_lens=(900, 333), gen_len=96, block_len=48, steps=2, hq=8, hkv=2)}
+    kw = dict(extra[case] if case in extra else SMALL[case])
+    kw["scale_mode"] = "inv_sqrt_d"
+    wl = small_workload(name=case, dtype="bf16", d=128, **kw)
+    for tiles_per_chunk in (0, 2):
+        _run_points(wl, "tc", seed=6, precision_mode=binding.PRECISION_PLAIN, sc_tiles_per_chunk=tiles_per_chunk)
+
+
 @pytest.mark.parametrize("case", ["ragged3", "gqa", "gqa32", "blk16", "mha64"])
 @pytest.mark.parametrize("engine", ["tc", "simt"])
 def test_bf16_output(case, engine):
     """out_dtype = bf16: every epilogue (fixed rows through both merge variants, block rows, merged key
     chunks, the full recompute) rounds the very fp32 value the fp32 context writes, once, to nearest even:
     the two outputs agree bit for bit after that rounding.  Against the oracle the error is the fp32
-    path's plus at most half a bf16 unit of the value (2^-9 |o|); the figures are printed."""
+    path's plus at most half a bf16 unit of the value (at most 2^-8 |o|); the figures are printed."""
     kw = dict(prompt_lens=(700, 333, 61), gen_len=192, block_len=64, steps=2, hq=4, hkv=4) if case == "mha64" else dict(SMALL[case])
     wl = small_workload(name=case, dtype="bf16", d=128, **kw)
     sch = SyntheticSchedule(wl, seed=31)
@@ -430,7 +446,7 @@ def test_bf16_output(case, engine):
     ref, _ = oracle.attention(sch.q, sch.k, sch.v, wl.cu_seqlens, wl.rope_theta, wl.head_dim ** -0.5)
     e32 = np.abs(o32.cpu().numpy().astype(np.float64) - ref)
     e16 = np.abs(o16.float().cpu().numpy().astype(np.float64) - ref)
-    assert (e16 <= e32 + 2.0 ** -9 * (np.abs(ref) + e32) + 1e-12).all()
+    assert (e16 <= e32 + 2.0 ** -8 * (np.abs(ref) + e32) + 1e-12).all()
     print("bf16 out, %s/%s: max abs err %.4g (fp32 out %.4g), mean %.4g (%.4g), max |o| %.3g"
           % (case, engine, e16.max(), e32.max(), e16.mean(), e32.mean(), np.abs(ref).max()))
 
@@ -505,10 +521,12 @@ def test_cfg1_every_step():
     ctx.destroy()
 
 
-@pytest.mark.parametrize("cfg", [2, 3, 4, 5])
-def test_full_size_configs_at_parity_points(cfg):
+@pytest.mark.parametrize("cfg,mode", [(2, "split"), (3, "split"), (4, "split"), (5, "split"), (5, "plain")])
+def test_full_size_configs_at_parity_points(cfg, mode):
     """Full-size workloads in the launch configuration the benchmark times;
-    the oracle is evaluated on all block rows, edge rows and a seeded sample."""
+    the oracle is evaluated on all block rows, edge rows and a seeded sample.  The GQA long-context
+    configuration (values ~ N(0,1)/sqrt(d)) also with plain operands."""
     wl = WORKLOADS[cfg]
     blocks = sorted({b for b, _ in parity_points(wl)})
-    _run_points(wl, "tc", seed=0, blocks=blocks, rows_fn=sample_rows, check_full=True, check_state=(cfg == 2))
+    _run_points(wl, "tc", seed=0, blocks=blocks, rows_fn=sample_rows, check_full=True, check_state=(cfg == 2),
+                precision_mode=binding.PRECISION_PLAIN if mode == "plain" else binding.PRECISION_SPLIT)

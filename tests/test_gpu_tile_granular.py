@@ -50,6 +50,12 @@ def test_long_ragged_batch_tile_granular():
     _run_points(wl, "tc", seed=4, cache_granularity=binding.GRANULARITY_TILE)
 
 
+def test_tile_granular_with_plain_operands():
+    wl = small_workload(name="tile-plain", prompt_lens=(700, 333, 61, 128), gen_len=192, block_len=32, steps=2,
+                        hq=4, hkv=2, scale_mode="inv_sqrt_d")
+    _run_points(wl, "tc", seed=3, cache_granularity=binding.GRANULARITY_TILE, precision_mode=binding.PRECISION_PLAIN)
+
+
 def test_cached_state_is_the_tile_level_state():
     """What the tile-granular build caches: for every row outside the tiles that overlap the block, the
     state of Eq. 2-6 over exactly the keys outside those tiles (compared through O~/l and m + log l: the

@@ -79,3 +79,20 @@ def test_bf16_probabilities_without_integer_reference_would_break_cached_vs_reco
     # with the integer reference exponent the rounding of P is identical on both paths
     _, _, diff = _emulate(0, "split", _bf)
     assert diff < 1e-4
+
+
+def test_plain_operands_hold_where_the_scores_are_small():
+    """Which inputs the plain mode (one bf16 plane of the rotated Q', K', one score product) suits: the
+    rounding of an operand to bf16 moves a score by about 2^-9 |s|, so the error against the fp64
+    definition grows with the magnitude of the scores.  With q, k ~ N(0,1)/sqrt(d) (the GQA long-context
+    configuration; |s| << 1) it is orders of magnitude inside the bar, at per-head scale 1 (|s| ~ 10) still
+    a factor of five inside, at scale 2 (|s| ~ 50; the LLaDA-shaped configurations) outside."""
+    d = 128
+    emax, emean, diff = _emulate(0, "bf16", _f16, scale_h=d ** -0.5)
+    assert emax < 1e-3 and emean < 1e-4 and diff < 1e-3
+    rows = {}
+    for sh in (0.5, 1.0, 2.0):
+        rows[sh] = _emulate(0, "bf16", _f16, scale_h=sh)
+    assert rows[0.5][0] < 2e-2 and rows[0.5][1] < 2e-3     # scores of order 3: still inside
+    assert rows[2.0][0] > 2e-2                             # scores of order 50: outside
+    assert rows[0.5][0] < rows[1.0][0] < rows[2.0][0]
