@@ -367,7 +367,7 @@ def run_cuda(args):
     # the attention kernel stamping the GPU's global timer at its first CTA's entry and last CTA's exit ----
     span = None
     if tc:
-        n_slots = 4 * (rrk.K // R + 2) + 8
+        n_slots = 16 * (rrk.K // R + 2) + 8
         rings = [torch.empty(n_slots, 2, dtype=torch.int64, device=dev) for _ in range(R)]
         for r_ in rings:
             r_[:, 0] = -1       # UINT64_MAX
@@ -377,7 +377,7 @@ def run_cuda(args):
 
         def note(kind, c):
             if kind in ("built", "stepped"):
-                kinds[idx[id(c)]] += [kind] * (c.last_launch_count - 1)     # (one RoPE launch per call)
+                kinds[idx[id(c)]].append((kind, c.last_launch_count - 1))     # (one RoPE launch per call)
 
         rrk.prepare()
         torch.cuda.synchronize()
@@ -390,8 +390,13 @@ def run_cuda(args):
         sp = {"stepped": [], "built": []}
         for r_, ks in zip(rings, kinds):
             h = r_.cpu().numpy()
-            for slot, kind in enumerate(ks[:n_slots]):
-                sp[kind].append(float(h[slot, 1] - h[slot, 0]) * 1e-3)     # ns -> us
+            slot = 0
+            for kind, n in ks:       # a call's launches (several when a step's fixed rows go out in more than one)
+                if slot + n > n_slots:
+                    break
+                if n > 0:
+                    sp[kind].append(float(h[slot:slot + n, 1].max() - h[slot:slot + n, 0].min()) * 1e-3)     # ns -> us
+                slot += n
         if sp["stepped"]:
             span = {"step_us": round(statistics.mean(sp["stepped"]), 2),
                     "step_us_median": round(statistics.median(sp["stepped"]), 2),

@@ -938,36 +938,28 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
                                             : (span_bits(v_lo - mc, v_hi - mc) &
                                                ~((un.x1 > un.x0) ? span_bits(e_lo - mc, e_hi - mc) : 0ull));
         const uint32_t s_addr = tlane + TS_S + 128 * b;
-        // Pass 1: maximum over this thread's columns.  Instruction count on
-        // these threads is what limits the kernel, so a tile with no masked
-        // column (the common case) takes a path with no per-column tests, and
-        // the maximum runs as four independent chains.
-        float mx = -INFINITY;
+        // This thread's HC scores come out of TMEM once, every load in flight before the one wait (the
+        // time of these threads per tile is what bounds a build: a second pass over TMEM and a wait per
+        // sixteen columns cost more than the registers).  Columns that take no part are set to -inf here,
+        // so that the maximum and the exponentials below need no per-column tests (the common tile has none).
+        uint32_t sr[HC];
+#pragma unroll
+        for (int cb = 0; cb < HC / 16; ++cb)
+          tmem_ld16(s_addr + mc + 16 * cb, *reinterpret_cast<uint32_t(*)[16]>(sr + 16 * cb));
+        tmem_ld_wait();
+        if (!all_valid) {
+#pragma unroll
+          for (int j = 0; j < HC; ++j) sr[j] = ((col_bits >> j) & 1ull) ? sr[j] : 0xff800000u;
+        }
+        float mx;
         {
-          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
-#pragma unroll 1
-          for (int cb = 0; cb < HC / 16; ++cb) {
-            uint32_t rr[16];
-            tmem_ld16(s_addr + mc + 16 * cb, rr);
-            tmem_ld_wait();
-            if (all_valid) {
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;   // four independent chains
 #pragma unroll
-              for (int j = 0; j < 16; j += 4) {
-                m0 = fmaxf(m0, __uint_as_float(rr[j]));
-                m1 = fmaxf(m1, __uint_as_float(rr[j + 1]));
-                m2 = fmaxf(m2, __uint_as_float(rr[j + 2]));
-                m3 = fmaxf(m3, __uint_as_float(rr[j + 3]));
-              }
-            } else {
-              const uint32_t bits = (uint32_t)(col_bits >> (16 * cb)) & 0xffffu;
-#pragma unroll
-              for (int j = 0; j < 16; j += 4) {
-                m0 = fmaxf(m0, ((bits >> j) & 1u) ? __uint_as_float(rr[j]) : -INFINITY);
-                m1 = fmaxf(m1, ((bits >> (j + 1)) & 1u) ? __uint_as_float(rr[j + 1]) : -INFINITY);
-                m2 = fmaxf(m2, ((bits >> (j + 2)) & 1u) ? __uint_as_float(rr[j + 2]) : -INFINITY);
-                m3 = fmaxf(m3, ((bits >> (j + 3)) & 1u) ? __uint_as_float(rr[j + 3]) : -INFINITY);
-              }
-            }
+          for (int j = 0; j < HC; j += 4) {
+            m0 = fmaxf(m0, __uint_as_float(sr[j]));
+            m1 = fmaxf(m1, __uint_as_float(sr[j + 1]));
+            m2 = fmaxf(m2, __uint_as_float(sr[j + 2]));
+            m3 = fmaxf(m3, __uint_as_float(sr[j + 3]));
           }
           mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
         }
@@ -1006,39 +998,24 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
             tmem_st16(tlane + TS_O + 64 * half + 16 * cb, rr, 0);
           }
         }
-        // Pass 2: probabilities of this thread's 64 columns.
-        float ps0 = 0.f, ps1 = 0.f;
-#pragma unroll 1
-        for (int cb = 0; cb < HC / 16; ++cb) {
-          uint32_t rr[16], pk[8];
-          tmem_ld16(s_addr + mc + 16 * cb, rr);
-          tmem_ld_wait();
-          if (all_valid) {
+        // Probabilities of this thread's columns, from the registers: P~ = 2^(S c - m) rounded to fp16 (what
+        // the P~V product multiplies); the normaliser sums the rounded values, converted back exactly.
+        float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
+        uint32_t pk[HC / 2];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              float p0 = round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j]), g.scale_log2, -m_use)));
-              float p1 = round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j + 1]), g.scale_log2, -m_use)));
-              ps0 += p0;  // the normaliser sums exactly what the MMA multiplies
-              ps1 += p1;
-              __half2 hp = __floats2half2_rn(p0, p1);
-              pk[j] = *reinterpret_cast<uint32_t*>(&hp);
-            }
-          } else {
-            const uint32_t bits = (uint32_t)(col_bits >> (16 * cb)) & 0xffffu;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              float p0 = round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j]), g.scale_log2, -m_use)));
-              float p1 = round_to_half_bits(ex2(fmaf(__uint_as_float(rr[2 * j + 1]), g.scale_log2, -m_use)));
-              p0 = ((bits >> (2 * j)) & 1u) ? p0 : 0.f;
-              p1 = ((bits >> (2 * j + 1)) & 1u) ? p1 : 0.f;
-              ps0 += p0;
-              ps1 += p1;
-              __half2 hp = __floats2half2_rn(p0, p1);
-              pk[j] = *reinterpret_cast<uint32_t*>(&hp);
-            }
-          }
-          tmem_st8(tlane + TS_P + 64 * b + (HC / 2) * half + 8 * cb, pk);
+        for (int j = 0; j < HC / 2; ++j) {
+          const float p0 = ex2(fmaf(__uint_as_float(sr[2 * j]), g.scale_log2, -m_use));
+          const float p1 = ex2(fmaf(__uint_as_float(sr[2 * j + 1]), g.scale_log2, -m_use));
+          const __half2 hp = __floats2half2_rn(p0, p1);
+          const float2 pf = __half22float2(hp);
+          if (j & 1) { ps2 += pf.x; ps3 += pf.y; } else { ps0 += pf.x; ps1 += pf.y; }
+          pk[j] = *reinterpret_cast<const uint32_t*>(&hp);
         }
+#pragma unroll
+        for (int cb = 0; cb < HC / 16; ++cb)
+          tmem_st8(tlane + TS_P + 64 * b + (HC / 2) * half + 8 * cb, *reinterpret_cast<uint32_t(*)[8]>(pk + 8 * cb));
+        ps0 += ps2;
+        ps1 += ps3;
         const float psum = ps0 + ps1;
         l_part = l_part * alpha + psum;
         m_ref = m_new;
