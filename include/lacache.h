@@ -275,10 +275,18 @@ lacache_status lacache_full_recompute_static(int dtype, int n_tokens, int n_q_he
                                              float* out, float* lse, void* cuda_stream);
 
 /*
- * Same operations with HOST buffers: inputs are copied host->device and
- * results device->host on `cuda_stream` inside the call (asynchronously when
- * the host memory is pinned).  Staging is allocated on first use.  The caller
- * synchronises the stream before reading out_host.  No paper counterpart.
+ * Same operations with HOST buffers: inputs are copied host->device on `cuda_stream` and results
+ * device->host inside the call (asynchronously when the host memory is pinned).  Staging, a copy
+ * stream and four events are allocated on first use.  No paper counterpart.
+ *
+ * lacache_step_host copies its result to the host on a stream of the context, so that the copy of one
+ * step (the larger transfer by far) runs beside the next step's input copy and kernels; two result
+ * buffers alternate on the device.  out_host / lse_host of a call are complete
+ *   - once the device is synchronised, or
+ *   - once `cuda_stream` is synchronised after lacache_join_host(ctx, cuda_stream), which makes that
+ *     stream wait for the latest result copy (a later lacache_step_host call joins the copy of the call
+ *     before it in the same way, behind its own kernels).
+ * The host buffers of a call must stay valid and untouched until then.
  */
 lacache_status lacache_build_host(lacache_ctx* ctx, int block_idx, const void* q_pre_host,
                                   const void* k_pre_host, const void* v_pre_host,
@@ -286,6 +294,7 @@ lacache_status lacache_build_host(lacache_ctx* ctx, int block_idx, const void* q
 lacache_status lacache_step_host(lacache_ctx* ctx, const void* q_blk_host, const void* k_blk_host,
                                  const void* v_blk_host, float* out_host, float* lse_host,
                                  void* cuda_stream);
+lacache_status lacache_join_host(lacache_ctx* ctx, void* cuda_stream);
 
 /*
  * Token-wise producer (Sec. 3.3.2, EmbedCache and RoPECache; Eq. 1): the operators that act on
@@ -395,6 +404,23 @@ lacache_status lacache_build_tokens_update(lacache_ctx* ctx, lacache_qkv* p, int
 lacache_status lacache_step_tokens(lacache_ctx* ctx, lacache_qkv* p, const int32_t* blk_token_ids,
                                    const void* blk_hidden, float* out, float* lse,
                                    void* cuda_stream);
+
+/*
+ * Every device-side wait of the projection kernel is bounded (about 2 s by default): a wait that runs
+ * out sets LACACHE_ERR_TIMEOUT and where it gave up in the producer's status word, the kernel's thread
+ * blocks unwind (loads in flight have landed long before; no tensor-core product was issued; TMEM is
+ * freed) and return, and the handle stays usable.  lacache_qkv_set_wait_limit sets that bound for later
+ * launches (microseconds, approximate; 0 = the default).  No paper counterpart.
+ *
+ * lacache_qkv_project_without_norm is a TEST HOOK for that path: it launches the projection kernel of
+ * lacache_qkv_project on `hidden` rows WITHOUT the norm kernel that would publish them, so the kernel's
+ * wait for its operand rows runs out.  Set a short limit first (a millisecond or so).  It writes
+ * nothing to q / k / v; lacache_qkv_poll_status then returns LACACHE_ERR_TIMEOUT, and later calls on
+ * the handle work as usual.
+ */
+lacache_status lacache_qkv_set_wait_limit(lacache_qkv* p, double microseconds);
+lacache_status lacache_qkv_project_without_norm(lacache_qkv* p, const void* hidden, int n_tokens, void* q,
+                                                void* k, void* v, void* cuda_stream);
 
 /* Profiling hook like lacache_set_timing_events, around the projection (GEMM) kernel. */
 lacache_status lacache_qkv_set_timing_events(lacache_qkv* p, void* ev_start, void* ev_stop);

@@ -30,7 +30,8 @@ EXPORTS = [
     "lacache_qkv_poll_status", "lacache_qkv_last_error", "lacache_set_step_overlap",
     "lacache_build_tokens_update", "lacache_build_incremental", "lacache_build_advance",
     "lacache_build_tokens_incremental", "lacache_build_advance_tokens", "lacache_sample_block",
-    "lacache_set_span_ring",
+    "lacache_set_span_ring", "lacache_join_host", "lacache_qkv_set_wait_limit",
+    "lacache_qkv_project_without_norm",
 ]
 
 
@@ -90,6 +91,7 @@ def load():
     lib.lacache_set_timing_events.argtypes = [vp, vp, vp]
     lib.lacache_set_step_overlap.argtypes = [vp, ip]
     lib.lacache_set_span_ring.argtypes = [vp, vp, ip]
+    lib.lacache_join_host.argtypes = [vp, vp]
     lib.lacache_sample_block.argtypes = [vp, vp, ip, ip, vp, vp, vp, vp]
     lib.lacache_full_recompute_static.argtypes = [ip, ip, ip, ip, ip, ctypes.c_float, ctypes.c_float, vp, vp, vp, vp,
                                                   vp, vp]
@@ -107,6 +109,8 @@ def load():
     lib.lacache_build_advance_tokens.argtypes = [vp, vp, vp, vp, vp]
     lib.lacache_step_tokens.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.lacache_build_tokens_update.argtypes = [vp, vp, ip, vp, vp, vp, ip, vp]
+    lib.lacache_qkv_set_wait_limit.argtypes = [vp, ctypes.c_double]
+    lib.lacache_qkv_project_without_norm.argtypes = [vp, vp, ip, vp, vp, vp, vp]
     lib.lacache_qkv_set_timing_events.argtypes = [vp, vp, vp]
     lib.lacache_qkv_last_launch_count.argtypes = [vp]
     lib.lacache_qkv_poll_status.argtypes = [vp]
@@ -224,6 +228,9 @@ class Context:
         self._check(self._lib.lacache_step_host(self._h, _ptr(q_blk), _ptr(k_blk), _ptr(v_blk),
                                                 _ptr(out), _ptr(lse), _stream(stream)))
 
+    def join_host(self, stream=None):
+        self._check(self._lib.lacache_join_host(self._h, _stream(stream)))
+
     def export_state(self, m, l, o_acc, stream=None):
         self._check(self._lib.lacache_export_state(self._h, _ptr(m), _ptr(l), _ptr(o_acc), _stream(stream)))
 
@@ -326,6 +333,14 @@ class QkvProducer:
     def project(self, n_tokens, q, k, v, token_ids=None, hidden=None, h_out=None, stream=None):
         self._check(self._lib.lacache_qkv_project(self._h, _ptr(token_ids), _ptr(hidden), int(n_tokens),
                                                   _ptr(q), _ptr(k), _ptr(v), _ptr(h_out), _stream(stream)))
+
+    def set_wait_limit(self, microseconds):
+        self._check(self._lib.lacache_qkv_set_wait_limit(self._h, float(microseconds)))
+
+    def project_without_norm(self, n_tokens, q, k, v, hidden, stream=None):
+        """Test hook: the projection kernel alone, whose wait for its operand rows then runs out."""
+        self._check(self._lib.lacache_qkv_project_without_norm(self._h, _ptr(hidden), int(n_tokens), _ptr(q),
+                                                               _ptr(k), _ptr(v), _stream(stream)))
 
     def set_timing_events(self, ev_start, ev_stop):
         h = lambda e: None if e is None else ctypes.c_void_p(e.cuda_event)

@@ -78,7 +78,10 @@ struct lacache_ctx {
   // staging for the *_host entry points
   void *hs_q = nullptr, *hs_k = nullptr, *hs_v = nullptr;       // full arrays
   void *hs_qb = nullptr, *hs_kb = nullptr, *hs_vb = nullptr;    // block arrays
-  float *hs_out = nullptr, *hs_lse = nullptr;
+  float *hs_out[2] = {nullptr, nullptr}, *hs_lse[2] = {nullptr, nullptr};   // results of alternate lacache_step_host calls
+  cudaStream_t copy_stream = nullptr;     // device -> host copies of a step's result run here, beside the next step
+  cudaEvent_t ev_ready[2] = {nullptr, nullptr}, ev_copied[2] = {nullptr, nullptr};
+  unsigned host_steps = 0;                // lacache_step_host calls so far
 
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
   unsigned long long* span_ring = nullptr;   // lacache_set_span_ring: [n_slots][2] device words
@@ -545,6 +548,11 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
 void destroy_impl(lacache_ctx* c) {
   cudaDeviceSynchronize();
   for (void* p : c->allocs) cudaFree(p);
+  for (int b = 0; b < 2; ++b) {
+    if (c->ev_ready[b]) cudaEventDestroy(c->ev_ready[b]);
+    if (c->ev_copied[b]) cudaEventDestroy(c->ev_copied[b]);
+  }
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   if (c->maps) tc_free_maps(c->maps);
   if (c->maps_scratch) tc_free_maps(c->maps_scratch);
   delete c;
@@ -717,7 +725,7 @@ lacache_status rope_all(lacache_ctx* c, const void* q, const void* k, const void
 }
 
 lacache_status ensure_staging(lacache_ctx* c) {
-  if (c->hs_out) return LACACHE_OK;
+  if (c->hs_out[0]) return LACACHE_OK;
   const Geometry& g = c->g;
   size_t es = elem_size(c->cfg.dtype);
   size_t nq = (size_t)g.T * g.Hq * g.d, nk = (size_t)g.T * g.Hkv * g.d;
@@ -730,8 +738,15 @@ lacache_status ensure_staging(lacache_ctx* c) {
   CU_TRY(c, dev_alloc(c, &e, bk * es));
   CU_TRY(c, dev_alloc(c, &f, bk * es));
   c->hs_q = a; c->hs_k = b; c->hs_v = cc; c->hs_qb = d; c->hs_kb = e; c->hs_vb = f;
-  CU_TRY(c, dev_alloc(c, &c->hs_lse, (size_t)g.T * g.Hq));
-  CU_TRY(c, dev_alloc(c, &c->hs_out, nq));   // (sized for fp32; a bf16 out uses half of it)
+  const size_t out_elems = c->cfg.out_dtype == LACACHE_OUT_BF16 ? (nq + 1) / 2 : nq;   // in floats
+  for (int b = 0; b < 2; ++b) {
+    CU_TRY(c, dev_alloc(c, &c->hs_lse[b], (size_t)g.T * g.Hq));
+    CU_TRY(c, cudaEventCreateWithFlags(&c->ev_ready[b], cudaEventDisableTiming));
+    CU_TRY(c, cudaEventCreateWithFlags(&c->ev_copied[b], cudaEventDisableTiming));
+  }
+  CU_TRY(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+  CU_TRY(c, dev_alloc(c, &c->hs_out[1], out_elems));
+  CU_TRY(c, dev_alloc(c, &c->hs_out[0], out_elems));   // (last: its being set marks the staging as complete)
   return LACACHE_OK;
 }
 
@@ -1155,14 +1170,33 @@ lacache_status lacache_step_host(lacache_ctx* c, const void* q, const void* k, c
   const Geometry& g = c->g;
   size_t es = elem_size(c->cfg.dtype);
   size_t rows = (size_t)g.B * g.block_len;
+  const unsigned i = c->host_steps;
+  const int b = (int)(i & 1u);
   CU_TRY(c, cudaMemcpyAsync(c->hs_qb, q, rows * g.Hq * g.d * es, cudaMemcpyHostToDevice, s));
   CU_TRY(c, cudaMemcpyAsync(c->hs_kb, k, rows * g.Hkv * g.d * es, cudaMemcpyHostToDevice, s));
   CU_TRY(c, cudaMemcpyAsync(c->hs_vb, v, rows * g.Hkv * g.d * es, cudaMemcpyHostToDevice, s));
-  st = lacache_step(c, c->hs_qb, c->hs_kb, c->hs_vb, c->hs_out, lse ? c->hs_lse : nullptr, stream);
+  // the step writes the result buffer that the copy of the call before last has left
+  if (i >= 2) CU_TRY(c, cudaStreamWaitEvent(s, c->ev_copied[b], 0));
+  st = lacache_step(c, c->hs_qb, c->hs_kb, c->hs_vb, c->hs_out[b], lse ? c->hs_lse[b] : nullptr, stream);
   if (st != LACACHE_OK) return st;
+  // ... and its copy to the host runs on the context's copy stream, beside whatever the caller's stream does
+  // next (the following step, as a rule)
+  CU_TRY(c, cudaEventRecord(c->ev_ready[b], s));
+  CU_TRY(c, cudaStreamWaitEvent(c->copy_stream, c->ev_ready[b], 0));
   const size_t out_es = c->cfg.out_dtype == LACACHE_OUT_BF16 ? 2 : 4;
-  CU_TRY(c, cudaMemcpyAsync(out, c->hs_out, out_es * g.T * g.Hq * g.d, cudaMemcpyDeviceToHost, s));
-  if (lse) CU_TRY(c, cudaMemcpyAsync(lse, c->hs_lse, sizeof(float) * g.T * g.Hq, cudaMemcpyDeviceToHost, s));
+  CU_TRY(c, cudaMemcpyAsync(out, c->hs_out[b], out_es * g.T * g.Hq * g.d, cudaMemcpyDeviceToHost, c->copy_stream));
+  if (lse) CU_TRY(c, cudaMemcpyAsync(lse, c->hs_lse[b], sizeof(float) * g.T * g.Hq, cudaMemcpyDeviceToHost, c->copy_stream));
+  CU_TRY(c, cudaEventRecord(c->ev_copied[b], c->copy_stream));
+  c->host_steps = i + 1;
+  // the previous call's copy joins the caller's stream behind this call's kernels
+  if (i >= 1) CU_TRY(c, cudaStreamWaitEvent(s, c->ev_copied[b ^ 1], 0));
+  return LACACHE_OK;
+}
+
+lacache_status lacache_join_host(lacache_ctx* c, void* stream) {
+  if (!c) return LACACHE_ERR_INVALID_ARG;
+  if (c->host_steps == 0) return LACACHE_OK;
+  CU_TRY(c, cudaStreamWaitEvent((cudaStream_t)stream, c->ev_copied[(c->host_steps - 1) & 1u], 0));
   return LACACHE_OK;
 }
 

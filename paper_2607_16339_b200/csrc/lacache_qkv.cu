@@ -61,6 +61,7 @@ struct lacache_qkv {
   cudaEvent_t ev_start = nullptr, ev_stop = nullptr;
   int last_launches = 0;
   // experiment knobs, read from the environment once at create
+  long long wait_cycles = 0;  // limit of the projection kernel's waits (lacache_qkv_set_wait_limit); 0 = default
   bool no_pdl = false;        // LACACHE_NO_PDL: plain stream-ordered launches
   bool plain_split = false;   // LACACHE_QKV_PLAIN_SPLIT: no closer / helper roles
   char err[512];
@@ -85,7 +86,7 @@ enum { QB_FULL = 0, QB_FREE = MAX_STAGES, QB_ACC_FULL = 2 * MAX_STAGES, QB_ACC_F
        QB_N = QB_ACC_FREE + 2 };
 constexpr uint32_t SMQ_TOTAL = SMQ_BAR + 8 * QB_N + 32;
 static_assert(SMQ_TOTAL <= 232448, "exceeds the 227 KB per-CTA limit");
-constexpr long long Q_WAIT_CYCLES = 4000000000ll;  // ~2 s
+constexpr long long Q_WAIT_CYCLES = 4000000000ll;  // ~2 s: the default limit of every device-side wait
 enum { QLOC_SMEM_ALIGN = 101, QLOC_WAIT_FULL = 102, QLOC_WAIT_FREE = 103, QLOC_WAIT_ACC_FULL = 104,
        QLOC_WAIT_ACC_FREE = 105, QLOC_TOKEN_ID = 106, QLOC_ROW = 107, QLOC_WAIT_ROWS = 108, QLOC_WAIT_PARTS = 109 };
 
@@ -110,6 +111,7 @@ struct GemmArgs {
   float* ws;
   int* counters;
   int32_t* status;
+  long long wait_cycles;     // limit of every device-side wait, in SM clock cycles
 };
 
 struct QCta {
@@ -117,6 +119,7 @@ struct QCta {
   volatile int* abort_flag;
   volatile int* rows_ready;   // set by the producer once the operand rows of this launch are complete
   int32_t* status;
+  long long wait_cycles;      // limit of every wait of this launch
   __device__ __forceinline__ uint32_t bar(int slot) const { return base + SMQ_BAR + 8u * slot; }
 };
 
@@ -127,7 +130,7 @@ __device__ __noinline__ bool q_wait_slow(const QCta& c, uint32_t bar, uint32_t p
     for (int i = 0; i < 32; ++i)
       if (mbar_try(bar, parity)) return true;
     if (*c.abort_flag) return false;
-    if (clock64() - t0 > Q_WAIT_CYCLES) {
+    if (clock64() - t0 > c.wait_cycles) {
       *c.abort_flag = 1;
       if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
         c.status[1] = loc;
@@ -258,7 +261,7 @@ __device__ __forceinline__ void gemm_producer(const QCta& c, const CUtensorMap* 
       asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(cnt) : "l"(a.ready) : "memory");
       if (cnt - a.ready_target >= 0) break;
       if (*c.abort_flag) return;
-      if (clock64() - t_start > Q_WAIT_CYCLES) {
+      if (clock64() - t_start > c.wait_cycles) {
         *c.abort_flag = 1;
         if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
           c.status[1] = QLOC_WAIT_ROWS; c.status[2] = blockIdx.x; c.status[3] = cnt;
@@ -339,7 +342,7 @@ __device__ __forceinline__ void closer_epilogue(const QCta& c, const GemmArgs& a
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(cnt) : "l"(a.counters + tile) : "memory");
       if (cnt == a.hp) break;
       if (*c.abort_flag) { ok = 0; break; }
-      if (clock64() - t_start > Q_WAIT_CYCLES) {
+      if (clock64() - t_start > c.wait_cycles) {
         *c.abort_flag = 1;
         if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
           c.status[1] = QLOC_WAIT_PARTS; c.status[2] = blockIdx.x; c.status[3] = cnt;
@@ -560,6 +563,7 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
   c.abort_flag = reinterpret_cast<volatile int*>(words + 1);
   c.rows_ready = reinterpret_cast<volatile int*>(words + 3);
   c.status = a.status;
+  c.wait_cycles = a.wait_cycles;
   if ((c.base & 1023u) != 0) {
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = QLOC_SMEM_ALIGN;
     return;
@@ -912,9 +916,20 @@ lacache_status lacache_qkv_project(lacache_qkv* p, const int32_t* token_ids, con
 }  // extern "C"
 
 namespace lacache {
+namespace {
+lacache_status project_impl(lacache_qkv* p, const int32_t* token_ids, const void* hidden, int n_tokens, void* q,
+                            void* k, void* v, void* h_out, const int32_t* dst_rows, int max_rows, bool early_inputs,
+                            void* stream, bool without_norm);
+}
 lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const void* hidden, int n_tokens, void* q,
                                 void* k, void* v, void* h_out, const int32_t* dst_rows, int max_rows, bool early_inputs,
                                 void* stream) {
+  return project_impl(p, token_ids, hidden, n_tokens, q, k, v, h_out, dst_rows, max_rows, early_inputs, stream, false);
+}
+namespace {
+lacache_status project_impl(lacache_qkv* p, const int32_t* token_ids, const void* hidden, int n_tokens, void* q,
+                            void* k, void* v, void* h_out, const int32_t* dst_rows, int max_rows, bool early_inputs,
+                            void* stream, bool without_norm) {
   if (!p) return LACACHE_ERR_INVALID_ARG;
   if ((token_ids == nullptr) == (hidden == nullptr))
     return qfail(p, LACACHE_ERR_INVALID_ARG, "pass exactly one of token_ids and hidden");
@@ -947,7 +962,7 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   const bool no_pdl = p->no_pdl;
-  {
+  if (!without_norm) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_tokens);
     cfg.blockDim = dim3(N_THREADS);
@@ -958,8 +973,10 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   }
   // the norm kernel is enqueued and will publish its n_tokens rows: only now does the count the
   // projection waits for move (a failed launch above leaves counter and target in step)
-  p->ready_target += (unsigned)n_tokens;
-  p->last_launches++;
+  if (!without_norm) {
+    p->ready_target += (unsigned)n_tokens;
+    p->last_launches++;
+  }
 
   GemmArgs ga{};
   int tn_idx = 0;
@@ -979,7 +996,9 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   ga.dst_rows = dst_rows;
   ga.max_rows = max_rows;
   ga.ready = p->ready;
-  ga.ready_target = (int)p->ready_target;
+  // (the time-out test hook: a count that no norm kernel will ever publish; the handle's own target stays)
+  ga.ready_target = (int)(p->ready_target + (without_norm ? (unsigned)n_tokens : 0u));
+  ga.wait_cycles = p->wait_cycles > 0 ? p->wait_cycles : Q_WAIT_CYCLES;
   ga.ws = p->ws;
   ga.counters = p->counters;
   ga.status = p->status;
@@ -1012,9 +1031,22 @@ lacache_status qkv_project_rows(lacache_qkv* p, const int32_t* token_ids, const 
   p->last_launches++;
   return LACACHE_OK;
 }
+}  // namespace
 }  // namespace lacache
 
 extern "C" {
+
+lacache_status lacache_qkv_set_wait_limit(lacache_qkv* p, double microseconds) {
+  if (!p) return LACACHE_ERR_INVALID_ARG;
+  if (!(microseconds >= 0.0) || microseconds > 1.0e7) return qfail(p, LACACHE_ERR_INVALID_ARG, "wait limit %g us", microseconds);
+  p->wait_cycles = (long long)(microseconds * 2000.0);   // SM clock cycles at about 2 GHz
+  return LACACHE_OK;
+}
+
+lacache_status lacache_qkv_project_without_norm(lacache_qkv* p, const void* hidden, int n_tokens, void* q, void* k,
+                                                void* v, void* stream) {
+  return lacache::project_impl(p, nullptr, hidden, n_tokens, q, k, v, nullptr, nullptr, 0, false, stream, true);
+}
 
 lacache_status lacache_qkv_set_timing_events(lacache_qkv* p, void* ev_start, void* ev_stop) {
   if (!p) return LACACHE_ERR_INVALID_ARG;

@@ -101,6 +101,41 @@ def test_projection_small_model(small_model, n):
     prod.destroy()
 
 
+@pytest.mark.parametrize("n", [32, 300])
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_handle_stays_usable(small_model, n):
+    """Every device-side wait is bounded.  Here one is made to run out without any fault: the projection
+    kernel is launched without the norm kernel that publishes its operand rows, with the bound set to
+    about a millisecond.  Its thread blocks give up, unwind and return; the status word says time-out and
+    where; the outputs are untouched; and the next ordinary projection on the same handle is correct."""
+    import time
+    tm = small_model
+    prod = make_producer(tm, 300)
+    ids = np.random.default_rng(3 * n).integers(0, tm.vocab, n).astype(np.int32)
+    st, msg, q, k, v, _ = project(prod, tm, n, ids=ids)          # an ordinary call first
+    assert st == binding.OK, msg
+    prod.set_wait_limit(1000.0)
+    wl = tm.wl
+    qx = torch.full((n, wl.n_q_heads, wl.head_dim), 7.0, device="cuda", dtype=torch.bfloat16)
+    kx = torch.full((n, wl.n_kv_heads, wl.head_dim), 7.0, device="cuda", dtype=torch.bfloat16)
+    vx = torch.full_like(kx, 7.0)
+    hidden = torch.zeros(n, tm.d_model, device="cuda", dtype=torch.bfloat16)
+    t0 = time.perf_counter()
+    prod.project_without_norm(n, qx, kx, vx, hidden)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 1.0                         # gave up after about a millisecond, not two seconds
+    st, msg = prod.poll_status()
+    assert st == binding.ERR_TIMEOUT, (st, msg)
+    assert "location" in msg
+    assert (qx == 7.0).all() and (kx == 7.0).all() and (vx == 7.0).all()    # nothing was written
+    assert prod.poll_status()[0] == binding.OK                    # the status word is cleared by the read
+    prod.set_wait_limit(0.0)
+    st, msg, q2, k2, v2, _ = project(prod, tm, n, ids=ids)        # and the handle works as before
+    assert st == binding.OK, msg
+    assert torch.equal(q, q2) and torch.equal(k, k2) and torch.equal(v, v2)
+    check_qkv(tm, q2, k2, v2, ids=ids, what="after a time-out, n=%d" % n)
+    prod.destroy()
+
+
 @pytest.fixture(scope="module")
 def llada_model():
     return TokenModel(W.WORKLOADS[2], 4096, 4096)
