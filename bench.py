@@ -857,11 +857,12 @@ def token_path_leg(wl, dev, peaks, seed, n_steps):
 
 
 # per-launch DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the
-# step attention kernel from the committed ncu capture
-# (profiles/tc_attn_kernel_cfg2_ncu_full.txt, tc_attn_kernel_cfg{3,4,5}_step_ncu_full.txt),
-# bytes; None where no capture exists for the workload.  The fp32 output (12.6 MB) is still in L2 when the
+# step attention kernel from the committed ncu captures
+# (profiles/tc_attn_kernel_cfg2_ncu_full.txt, tc_attn_kernel_cfg{3,4}_step_ncu_full.txt,
+# tc_attn_kernel_cfg5_{split,plain}_ncu_full.txt), bytes; None where no capture exists for the workload
+# and precision mode.  The fp32 output (12.6 MB) is still in L2 when the
 # kernel ends, so the figure is dominated by reads.
-TRAFFIC_PER_LAUNCH = {(2, 1): 45337856, (3, 1): 93736960, (4, 1): 456532736, (5, 1): 208314880}   # (config, precision mode)
+TRAFFIC_PER_LAUNCH = {(2, 1): 48370432, (3, 1): 93736960, (4, 1): 460605952, (5, 1): 209015552, (5, 0): 161659392}   # (config, precision mode)
 
 
 # ----------------------------------------------------------------------------
