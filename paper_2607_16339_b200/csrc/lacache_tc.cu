@@ -840,6 +840,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     const bool active = unit_row_valid(un, quad * 32);  // this warp holds at least one real row (its first)
     float m_ref = -INFINITY, l_part = 0.f;
     bool first_tile = true;
+    bool calm = false;     // the unit's latest tile moved no reference exponent of this warp
     bool have_o = false;   // O~ in TMEM holds something before the unit's first P~V
     if (WINDOW && un.t1 <= un.t0) {
       // A unit without key tiles gives these threads nothing to wait for, and the other roles' parity
@@ -963,53 +964,70 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
           }
           mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
         }
-        {
-          // the slots alternate between consecutive exchanges
-          volatile float* mxch = xch + 2 * (xslot & 1u);
-          ++xslot;
-          mxch[half] = mx;
-          mbar_arrive(c.bar(BAR_PAIR + quad));
-          if (!wait_bar(c, BAR_PAIR + quad, pair_phase & 1, LOC_WAIT_S)) return;
-          ++pair_phase;
-          mx = fmaxf(mxch[0], mxch[1]);
-        }
+        // The pair's maxima cross through shared memory (the slots alternate between consecutive exchanges).
+        // That round trip sits between the maximum and the exponentials of every tile, so a build does not
+        // wait for it: after a unit's first tile the reference exponent almost never moves (it moves only
+        // when a row's maximum outgrows it by more than RESCALE_SLACK), so the probabilities are formed
+        // with the reference as it stands while the exchange is under way, and formed again, the exact
+        // way, only when the exchange says that some row of the warp has to move its reference.
+        volatile float* mxch = xch + 2 * (xslot & 1u);
+        ++xslot;
+        mxch[half] = mx;
+        mbar_arrive(c.bar(BAR_PAIR + quad));
+        float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
+        uint32_t pk[HC / 2];
+        // Probabilities of this thread's columns, from the registers: P~ = 2^(S c - m) rounded to fp16 (what
+        // the P~V product multiplies); the normaliser sums the rounded values, converted back exactly.
+        auto probabilities = [&](float m_sub) {
+          ps0 = ps1 = ps2 = ps3 = 0.f;
+#pragma unroll
+          for (int j = 0; j < HC / 2; ++j) {
+            const float p0 = ex2(fmaf(__uint_as_float(sr[2 * j]), g.scale_log2, -m_sub));
+            const float p1 = ex2(fmaf(__uint_as_float(sr[2 * j + 1]), g.scale_log2, -m_sub));
+            const __half2 hp = __floats2half2_rn(p0, p1);
+            const float2 pf = __half22float2(hp);
+            if (j & 1) { ps2 += pf.x; ps3 += pf.y; } else { ps0 += pf.x; ps1 += pf.y; }
+            pk[j] = *reinterpret_cast<const uint32_t*>(&hp);
+          }
+        };
+        // (not for the block queries of a step: few tiles per unit, and that kernel is sensitive to its size;
+        // and only after a tile that left every reference of the warp where it was: with large scores the
+        // references of a unit's first tiles move often, and forming the probabilities twice costs more
+        // than the exchange)
+        const bool ahead = !STEP && calm && !__any_sync(0xffffffffu, m_ref == -INFINITY);
+        if (ahead) probabilities(m_ref);
+        if (!wait_bar(c, BAR_PAIR + quad, pair_phase & 1, LOC_WAIT_S)) return;
+        ++pair_phase;
+        mx = fmaxf(mxch[0], mxch[1]);
         // integer reference exponent, moved only when the row maximum outgrows it
         // by more than RESCALE_SLACK (so P~ <= 2^RESCALE_SLACK and rescales are rare)
         const float cand = ceilf(mx * g.scale_log2);
         float m_new = m_ref;
         if (m_ref == -INFINITY || cand > m_ref + RESCALE_SLACK) m_new = fmaxf(m_ref, cand);
-        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
         float alpha = 1.f;
-        if (m_new != m_ref) alpha = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
-        if ((!first_tile || (WINDOW && have_o)) && __any_sync(0xffffffffu, alpha != 1.f)) {
-          // O~ in TMEM is rescaled in place: P~V of the previous tile must be done
-          if (!o_waited) {
-            if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
-            o_waited = true;
-            tc_fence_after();
-          }
+        // (both warps of the pair see the same rows and the same maxima: they take the same branch)
+        calm = !__any_sync(0xffffffffu, m_new != m_ref);
+        if (!(ahead && calm)) {
+          const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+          if (m_new != m_ref) alpha = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
+          if ((!first_tile || (WINDOW && have_o)) && __any_sync(0xffffffffu, alpha != 1.f)) {
+            // O~ in TMEM is rescaled in place: P~V of the previous tile must be done
+            if (!o_waited) {
+              if (!wait_bar(c, BAR_O_FULL, (jj - 1) & 1, LOC_WAIT_O)) return;
+              o_waited = true;
+              tc_fence_after();
+            }
 #pragma unroll 1
-          for (int cb = 0; cb < 4; ++cb) {
-            uint32_t rr[16];
-            tmem_ld16(tlane + TS_O + 64 * half + 16 * cb, rr);
-            tmem_ld_wait();
+            for (int cb = 0; cb < 4; ++cb) {
+              uint32_t rr[16];
+              tmem_ld16(tlane + TS_O + 64 * half + 16 * cb, rr);
+              tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j) rr[j] = __float_as_uint(__uint_as_float(rr[j]) * alpha);
-            tmem_st16(tlane + TS_O + 64 * half + 16 * cb, rr, 0);
+              for (int j = 0; j < 16; ++j) rr[j] = __float_as_uint(__uint_as_float(rr[j]) * alpha);
+              tmem_st16(tlane + TS_O + 64 * half + 16 * cb, rr, 0);
+            }
           }
-        }
-        // Probabilities of this thread's columns, from the registers: P~ = 2^(S c - m) rounded to fp16 (what
-        // the P~V product multiplies); the normaliser sums the rounded values, converted back exactly.
-        float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
-        uint32_t pk[HC / 2];
-#pragma unroll
-        for (int j = 0; j < HC / 2; ++j) {
-          const float p0 = ex2(fmaf(__uint_as_float(sr[2 * j]), g.scale_log2, -m_use));
-          const float p1 = ex2(fmaf(__uint_as_float(sr[2 * j + 1]), g.scale_log2, -m_use));
-          const __half2 hp = __floats2half2_rn(p0, p1);
-          const float2 pf = __half22float2(hp);
-          if (j & 1) { ps2 += pf.x; ps3 += pf.y; } else { ps0 += pf.x; ps1 += pf.y; }
-          pk[j] = *reinterpret_cast<const uint32_t*>(&hp);
+          probabilities(m_use);
         }
 #pragma unroll
         for (int cb = 0; cb < HC / 16; ++cb)
