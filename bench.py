@@ -282,7 +282,7 @@ def timed_region(rr, W, min_ms=50.0, max_repeats=200):
         times.append(e0.elapsed_time(e1))
         if i == 0:   # size the number of repeats from the first one (the same on every rank: max over ranks)
             t1 = reduce_max(times[0], torch.device("cuda", torch.cuda.current_device()))
-            repeats = 1 if t1 >= 4 * min_ms else max(3, min(max_repeats, math.ceil(min_ms / max(t1, 1e-3))))
+            repeats = 1 if t1 >= 4 * min_ms else max(5, min(max_repeats, math.ceil(min_ms / max(t1, 1e-3))))
         i += 1
     return times, launches, builds, wall
 
