@@ -28,7 +28,7 @@ struct lacache_ctx {
   // per block, tcgen05: row tiles x key windows of the incremental build (prefix state from scratch;
   // cached state = prefix state + the keys after the block; the finished block's rows from scratch;
   // every other row advanced by the finished block's keys and completed by the keys after the block)
-  std::vector<ListRef> inc_prefix, inc_comb, inc_fresh, inc_fused;
+  std::vector<ListRef> inc_prefix, inc_comb, inc_fresh, inc_fresh_chunks, inc_fused;
   // per block, tile-granular caching (Algorithm 1's overlap predicates): the build in two launches over
   // the key tiles before / after the tiles that overlap the block, the step in one
   std::vector<ListRef> tile_prefix, tile_suffix, tile_step;
@@ -49,10 +49,12 @@ struct lacache_ctx {
     bool no_deep = false;    // LACACHE_NO_DEEP: earlier merge variant
     bool no_qcomp = false;   // LACACHE_NO_QCOMP: no in-kernel rotation of first units
     bool no_pack = false;    // LACACHE_NO_PACK: no head packing of GQA block queries
+    bool no_chunked_advance = false;  // LACACHE_NO_CHUNKED_ADVANCE: an advance computes the finished block's rows as key-window units
     bool verbose = false;    // LACACHE_VERBOSE: prints the step plan
   } knobs;
   ListRef full_list;
-  int max_chunks = 1;
+  int max_chunks = 1;      // most key chunks of a step's block-row units
+  int part_chunks = 1;     // chunk slots per (sequence, head) of the partial-state buffers (the advance may use more)
   std::vector<WorkItem> items_host;
   bool split = true;       // tcgen05 engine: rotated Q', K' kept as two bf16 planes (precision_mode SPLIT)
 
@@ -195,6 +197,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     k.no_deep = getenv("LACACHE_NO_DEEP") != nullptr;
     k.no_qcomp = getenv("LACACHE_NO_QCOMP") != nullptr;
     k.no_pack = getenv("LACACHE_NO_PACK") != nullptr;
+    k.no_chunked_advance = getenv("LACACHE_NO_CHUNKED_ADVANCE") != nullptr;
     k.verbose = getenv("LACACHE_VERBOSE") != nullptr;
   }
   if (cfg->batch < 1 || !cfg->prompt_lens) return fail(c, LACACHE_ERR_INVALID_ARG, "batch < 1 or prompt_lens NULL");
@@ -359,6 +362,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     }
     c->build_list.push_back({rows_off, (int)items.size() - rows_off});
   }
+  int inc_chunks = 1;
   for (int k = 0; k < g.n_blk && tc; ++k) {
     // Incremental build.  With s the block's first token and e one past its last, of a sequence
     // [cs, ce): the prefix state holds keys [cs, s); the cached state adds keys [e, ce); advancing
@@ -402,6 +406,28 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
       window(from, cs, cs, s0, 0);
     }
     c->inc_fresh.push_back({off, (int)items.size() - off});
+    // the same rows as block-row units of the step kernel, their keys [cs, s0) cut into chunks that
+    // spread over the SMs (a handful of row tiles otherwise walk the whole prefix one after the other)
+    off = (int)items.size();
+    for (int b = 0; b < g.B && k > 0; ++b) {
+      const int cs = c->cu[b], s0 = c->blk_start_all[(size_t)k * g.B + b];
+      const int nkt = (s0 - cs + TC_KEYS - 1) / TC_KEYS;
+      const int slots = std::max(1, g.B * g.Hq / std::max(1, std::min(128 / (g.block_len <= 32 ? 32 : 64), g.group)));
+      int chunks = std::max(1, std::min({16, nkt, c->num_sms / slots}));
+      const int per = (nkt + chunks - 1) / chunks;
+      chunks = (nkt + per - 1) / per;
+      inc_chunks = std::max(inc_chunks, chunks);
+      for (int ch = 0; ch < chunks; ++ch) {
+        WorkItem w{};
+        w.kind = ITEM_BLOCK_CHUNK; w.seq = b; w.row0 = s0 - g.block_len; w.nrows = g.block_len;
+        w.chunk = ch; w.kt0 = ch * per; w.kt1 = std::min(nkt, (ch + 1) * per);
+        w.pad = chunks;
+        w.seq_start = cs; w.seq_end = s0;       // (the end of the key range, not of the sequence)
+        w.blk_start = s0 - g.block_len;
+        items.push_back(w);
+      }
+    }
+    c->inc_fresh_chunks.push_back({off, (int)items.size() - off});
     off = (int)items.size();
     for (int b = 0; b < g.B && k > 0; ++b) {
       const int cs = c->cu[b], ce = c->cu[b + 1], s0 = c->blk_start_all[(size_t)k * g.B + b], e0 = s0 + g.block_len;
@@ -419,6 +445,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     }
     c->inc_fused.push_back({off, (int)items.size() - off});
   }
+  c->part_chunks = std::max(c->max_chunks, inc_chunks);
   if (cfg->cache_granularity == LACACHE_GRANULARITY_TILE) {
     // Algorithm 1 at tile granularity, tiles of TC_ROWS tokens counted from the start of each sequence
     // (B_r = B_c).  With [lo, hi) the tokens of the tiles that overlap the block: state is cached for the
@@ -529,7 +556,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   CU_TRY(c, dev_alloc(c, &c->st.m, (size_t)g.Hq * g.Tp, true));
   CU_TRY(c, dev_alloc(c, &c->st.l, (size_t)g.Hq * g.Tp, true));
   CU_TRY(c, dev_alloc(c, &c->st.o, (size_t)g.Hq * g.Tp * g.d, true));
-  size_t nparts = (size_t)g.B * g.Hq * c->max_chunks * g.block_len;
+  size_t nparts = (size_t)g.B * g.Hq * c->part_chunks * g.block_len;
   CU_TRY(c, dev_alloc(c, &c->part_m, nparts));
   CU_TRY(c, dev_alloc(c, &c->part_l, nparts));
   CU_TRY(c, dev_alloc(c, &c->part_o, nparts * g.d));
@@ -562,6 +589,18 @@ void destroy_impl(lacache_ctx* c) {
 // LACACHE_DEEP_UNITS knob lowers it so that small cases exercise the multi-launch path).
 int deep_unit_cap(const lacache_ctx* c) { return c->knobs.deep_units; }
 
+// block queries of a GQA model: heads of one KV group side by side in the 128 lanes of a tile
+void set_packing(lacache_ctx* c, AttnArgs& a) {
+  if (c->g.group < 2 || c->knobs.no_pack) return;
+  const int rows = c->g.block_len <= 32 ? 32 : 64;
+  const int pack = std::min(128 / rows, c->g.group);
+  if (c->g.Hq < 128 / rows) return;   // the packed tile's load takes 128 / rows heads at a time
+  if (pack >= 2) {
+    a.pack = pack; a.pack_rows = rows;
+    a.stream_slots = c->g.Hkv * ((c->g.group + pack - 1) / pack);
+  }
+}
+
 AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk, const RotBuffers& rot,
                    float* out, float* lse) {
   AttnArgs a{};
@@ -577,7 +616,7 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
   a.out_bf16 = c->cfg.out_dtype == LACACHE_OUT_BF16 ? 1 : 0;
   a.part_m = c->part_m; a.part_l = c->part_l; a.part_o = c->part_o;
   a.counters = c->counters;
-  a.max_chunks = c->max_chunks;
+  a.max_chunks = c->part_chunks;
   a.status = c->d_status;
   a.no_pdl = c->knobs.no_pdl ? 1 : 0;
   a.split = c->split ? 1 : 0;
@@ -586,15 +625,7 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
     // estimate (units x per-unit cost, in arbitrary time units)
     const int Hq = c->g.Hq;
     a.stream_slots = Hq; a.pack = 1; a.pack_rows = 0;
-    if (mode == MODE_STEP && c->g.group >= 2 && !c->knobs.no_pack) {
-      // block queries of a GQA model: heads of one KV group side by side in the 128 lanes of a tile
-      const int rows = c->g.block_len <= 32 ? 32 : 64;
-      const int pack = std::min(128 / rows, c->g.group);
-      if (pack >= 2) {
-        a.pack = pack; a.pack_rows = rows;
-        a.stream_slots = c->g.Hkv * ((c->g.group + pack - 1) / pack);
-      }
-    }
+    if (mode == MODE_STEP) set_packing(c, a);
     long long units_stream = (long long)list.n * a.stream_slots;
     if (mode == MODE_STEP) {
       lacache_ctx::ListRef ml = c->merge_list[blk];
@@ -835,6 +866,21 @@ lacache_status ensure_prefix_state(lacache_ctx* c) {
   return LACACHE_OK;
 }
 // one launch over a list of key-window items: dst = (init +) the window's keys
+// Block-row units of the step kernel (key chunks, heads of a KV group packed) whose merged result is the
+// rows' state, stored to dst, instead of normalised rows; no fixed-row units, nothing rotated on the fly.
+lacache_status run_block_rows_to_state(lacache_ctx* c, lacache_ctx::ListRef list, int blk, const StateBuffers& dst,
+                                       cudaStream_t s) {
+  if (list.n == 0) return LACACHE_OK;
+  AttnArgs a = attn_args(c, MODE_FULL, list, blk, c->rot, nullptr, nullptr);
+  a.mode = MODE_STEP;
+  set_packing(c, a);
+  a.n_ctas_stream = (int)std::min<long long>(c->num_sms, (long long)list.n * a.stream_slots);
+  a.n_ctas = a.n_ctas_stream;
+  a.blk_to_state = 1;
+  a.st = dst;
+  return run_attention(c, a, false, s);
+}
+
 lacache_status run_window(lacache_ctx* c, lacache_ctx::ListRef list, int blk, const StateBuffers& init,
                           const StateBuffers& dst, const StateBuffers& snap, cudaStream_t s, float* out, float* lse) {
   if (list.n == 0) return LACACHE_OK;
@@ -904,8 +950,15 @@ lacache_status lacache_build_advance(lacache_ctx* c, const void* q, const void* 
   r.in_dtype = c->cfg.dtype;
   CU_TRY(c, rope_write(c->g, r, c->engine, s));
   c->last_launches++;
-  lacache_status st = run_window(c, c->inc_fresh[blk], blk, StateBuffers{}, c->pst, StateBuffers{}, s);
+  lacache_status st = c->knobs.no_chunked_advance ? run_window(c, c->inc_fresh[blk], blk, StateBuffers{}, c->pst, StateBuffers{}, s)
+                                                  : run_block_rows_to_state(c, c->inc_fresh_chunks[blk], blk, c->pst, s);
   if (st != LACACHE_OK) return st;
+  if (c->knobs.verbose) {   // which of the two launches a device status belongs to
+    int32_t hs[4] = {0, 0, 0, 0};
+    cudaStreamSynchronize(s);
+    cudaMemcpy(hs, c->d_status, sizeof(hs), cudaMemcpyDeviceToHost);
+    fprintf(stderr, "lacache: advance to block %d, after the finished block's rows: status %d %d %d %d\n", blk, hs[0], hs[1], hs[2], hs[3]);
+  }
   st = run_window(c, c->inc_fused[blk], blk, c->pst, c->st, c->pst, s);
   if (st != LACACHE_OK) return st;
   c->built_block = blk;

@@ -130,6 +130,8 @@ struct AttnArgs {
   // split-key partial states of block queries and their arrival counters
   float* part_m; float* part_l; float* part_o; int* counters; int max_chunks;
   int32_t* status;
+  int blk_to_state;          // block-row units write the merged state (m, l, O~) of their rows to `st` instead
+                             // of normalised rows to `out` (first launch of an incremental advance)
   int no_pdl;                // host only: launch the ordinary way (experiment knob)
   int split;                 // host only: rotated Q', K' are split bf16 planes (which kernel instantiation runs)
   // optional (lacache_set_span_ring): two device words of this launch; every CTA folds the global

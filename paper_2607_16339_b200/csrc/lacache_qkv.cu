@@ -610,6 +610,13 @@ qkv_gemm_kernel(const __grid_constant__ CUtensorMap w_map, const __grid_constant
   // this grid must not complete before the grids ahead of it have: whatever waits for it relies on that
   grid_dependency_wait();
   // teardown: free TMEM once every thread is past its last TMEM access
+  if (*c.abort_flag) {
+    // a bounded wait ran out: copies requested before that may still be on their way into this CTA's shared
+    // memory; give them time to land (a fixed 50 us) before it is given up
+    const long long t0 = clock64();
+    while (clock64() - t0 < 100000ll) {
+    }
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {  // the warp that allocated

@@ -350,7 +350,8 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
     un.t1 = it.kt1;
     un.chunk = it.chunk;
     un.nchunks = it.pad;
-    un.epi = it.pad > 1 ? EPI_PARTIAL : EPI_OUT;
+    // (block rows whose result is a state always go through the chunk merge, which knows where to put it)
+    un.epi = (it.pad > 1 || a.blk_to_state) ? EPI_PARTIAL : EPI_OUT;
     un.q_rows = un.rh ? BM : 64;
   } else {
     un.epi = EPI_OUT;
@@ -667,13 +668,29 @@ __device__ __forceinline__ void coop_store_out_rows(const Cta& c, const AttnArgs
   }
 }
 
+// One 16-byte column of a merged row: the normalised output (and lse), or -- when the launch computes
+// the block rows' state for the incremental build -- the unnormalised triple itself.
+__device__ __forceinline__ void store_merged(const Geometry& g, const AttnArgs& a, int row, int h, int ch, float M,
+                                             float L, float4 acc) {
+  if (a.blk_to_state) {
+    const size_t srow = (size_t)h * g.Tp + row;
+    *reinterpret_cast<float4*>(a.st.o + srow * D + ch * 4) = acc;
+    if (ch == 0) { a.st.m[srow] = M; a.st.l[srow] = L; }
+    return;
+  }
+  const float LN2 = 0.69314718055994530942f;
+  const float inv = 1.f / L;
+  const size_t orow = (size_t)row * g.Hq + h;
+  store_out4(a, orow * D + ch * 4, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
+  if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
+}
+
 // Few chunks (at most NC): each thread takes BATCH (row, 16-byte column) items at a
 // time and issues every load of the batch -- references, normalisers, 16 bytes of
 // each partial O~ -- before any is used: one L2 round trip per batch.
 template <int NC, int BATCH>
 __device__ __forceinline__ void merge_few(const Geometry& g, const AttnArgs& a, size_t pbase, int nchunks,
                                           int block_len, int row0, int h) {
-  const float LN2 = 0.69314718055994530942f;
   const int t = threadIdx.x - 64;
   const int n_items = block_len * 32;
   for (int i0 = t; i0 < n_items; i0 += BATCH * ROW_THREADS) {
@@ -711,10 +728,7 @@ __device__ __forceinline__ void merge_few(const Geometry& g, const AttnArgs& a, 
         acc.z = fmaf(v[bi][k].z, w, acc.z);
         acc.w = fmaf(v[bi][k].w, w, acc.w);
       }
-      const float inv = 1.f / L;
-      const size_t orow = (size_t)(row0 + rr) * g.Hq + h;
-      store_out4(a, orow * D + ch * 4, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
-      if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
+      store_merged(g, a, row0 + rr, h, ch, M, L, acc);
     }
   }
 }
@@ -724,7 +738,6 @@ __device__ __forceinline__ void merge_few(const Geometry& g, const AttnArgs& a, 
 // read with coalesced loads straight from L2 and the normalised rows written out.
 __device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs& a, size_t pbase, int nchunks,
                                                int block_len, int row0, int h) {
-  const float LN2 = 0.69314718055994530942f;
   const int t = threadIdx.x - 64;
   if (nchunks <= 2) {
     merge_few<2, 4>(g, a, pbase, nchunks, block_len, row0, h);
@@ -766,10 +779,7 @@ __device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs
         acc.w = fmaf(v[k].w, w[k], acc.w);
       }
     }
-    const float inv = 1.f / L;
-    const size_t orow = (size_t)(row0 + rr) * g.Hq + h;
-    store_out4(a, orow * D + ch * 4, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
-    if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
+    store_merged(g, a, row0 + rr, h, ch, M, L, acc);
   }
 }
 
@@ -1892,6 +1902,15 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   __syncwarp();
 
   // teardown: free TMEM once every thread is past its last TMEM access
+  if (*c.abort_flag) {
+    // A bounded wait ran out and the roles have returned where they stood.  Bulk copies and tensor-core
+    // products that were issued before that may still be in flight towards this CTA's shared memory and
+    // TMEM: give them time to land (they take microseconds; the limit is a fixed 50 us) before both are
+    // given up.
+    const long long t0 = clock64();
+    while (clock64() - t0 < 100000ll) {
+    }
+  }
   tc_fence_before();
   mbar_arrive(c.bar(BAR_DONE));
   if (warp == 1) {  // the warp that allocated
@@ -2028,8 +2047,11 @@ TcMaps* tc_make_maps(const Geometry& g, const RotBuffers& rot, float* state_o, b
   const int bn = tc_keys(split);
   bool ok = make_qk_map(&m->q, rot.q_hi, g.Hq, g.Tp, BM, planes, err, errlen) &&
             make_qk_map(&m->q64, rot.q_hi, g.Hq, g.Tp, 64, planes, err, errlen) &&
+            // (the box always fills the 128 lanes of the tile, whose layout the MMA descriptors assume: with
+            // fewer heads in a KV group than fit, the lanes past them hold other heads' rows and are ignored;
+            // a model with fewer query heads than that does not pack)
             make_qpack_map(&m->q_pack, rot.q_hi, g.Hq, g.Tp, g.block_len <= 32 ? 32 : 64,
-                           std::max(1, std::min(g.block_len <= 32 ? 4 : 2, g.group)), planes, err, errlen) &&
+                           std::max(1, std::min(g.block_len <= 32 ? 4 : 2, g.Hq)), planes, err, errlen) &&
             make_qk_map(&m->k, rot.k_hi, g.Hkv, g.Tp, bn, planes, err, errlen) &&
             make_qk_map(&m->k64, rot.k_hi, g.Hkv, g.Tp, 64, planes, err, errlen) &&
             make_qk_map(&m->k32, rot.k_hi, g.Hkv, g.Tp, 32, planes, err, errlen) &&

@@ -312,6 +312,22 @@ def test_steps_fed_by_same_stream_writes(cfg):
     ctx.destroy()
 
 
+@pytest.mark.parametrize("hq,hkv,block_len", [(4, 2, 32), (6, 2, 16), (8, 2, 32), (6, 2, 64), (4, 2, 64)])
+def test_packed_block_rows_several_units_per_cta(hq, hkv, block_len, monkeypatch):
+    """Block rows of a GQA model share a tile (heads of a KV group side by side).  A CTA's first unit
+    rotates its queries itself; every later unit's tile comes through the packed tensor map, whose box
+    must fill the tile whatever the group size (2 and 3 heads of 32 rows leave lanes over).  Forced here
+    with two stream CTAs for all units, and once with the first unit loaded the same way."""
+    wl = small_workload(name="packed-%d-%d-%d" % (hq, hkv, block_len), prompt_lens=(150, 61, 230), gen_len=2 * block_len,
+                        block_len=block_len, steps=2, hq=hq, hkv=hkv)
+    monkeypatch.setenv("LACACHE_STREAM_CTAS", "2")       # (experiment knobs are read when a context is created)
+    _run_points(wl, "tc", seed=8)
+    monkeypatch.setenv("LACACHE_NO_QCOMP", "1")
+    _run_points(wl, "tc", seed=9, check_state=False)
+    monkeypatch.delenv("LACACHE_NO_QCOMP")
+    monkeypatch.delenv("LACACHE_STREAM_CTAS")
+
+
 @pytest.mark.parametrize("cfg", [3, 4])
 def test_step_split_over_several_launches(cfg, monkeypatch):
     """A step with more fixed-row tiles per CTA than the pipelined merge variant tabulates goes out in
