@@ -54,6 +54,8 @@ struct lacache_ctx {
   } knobs;
   ListRef full_list;
   int max_chunks = 1;      // most key chunks of a step's block-row units
+  std::vector<int32_t> adv_tab;   // per (block, sequence): first row and key chunks of an advance's block-row units
+  int32_t* d_adv_tab = nullptr;
   int part_chunks = 1;     // chunk slots per (sequence, head) of the partial-state buffers (the advance may use more)
   std::vector<WorkItem> items_host;
   bool split = true;       // tcgen05 engine: rotated Q', K' kept as two bf16 planes (precision_mode SPLIT)
@@ -363,6 +365,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     c->build_list.push_back({rows_off, (int)items.size() - rows_off});
   }
   int inc_chunks = 1;
+  c->adv_tab.assign((size_t)g.n_blk * g.B * 2, 0);
   for (int k = 0; k < g.n_blk && tc; ++k) {
     // Incremental build.  With s the block's first token and e one past its last, of a sequence
     // [cs, ce): the prefix state holds keys [cs, s); the cached state adds keys [e, ce); advancing
@@ -412,11 +415,17 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     for (int b = 0; b < g.B && k > 0; ++b) {
       const int cs = c->cu[b], s0 = c->blk_start_all[(size_t)k * g.B + b];
       const int nkt = (s0 - cs + TC_KEYS - 1) / TC_KEYS;
-      const int slots = std::max(1, g.B * g.Hq / std::max(1, std::min(128 / (g.block_len <= 32 ? 32 : 64), g.group)));
-      int chunks = std::max(1, std::min({16, nkt, c->num_sms / slots}));
+      // (units of all sequences: one per sequence and head, or per packed group of heads; at most eight
+      // chunks, which the last one to arrive merges with every load in flight at once)
+      const int fit = 128 / (g.block_len <= 32 ? 32 : 64);
+      const int pack = (g.group >= 2 && g.Hq >= fit && !c->knobs.no_pack) ? std::min(fit, g.group) : 1;
+      const int slots = g.B * g.Hkv * ((g.group + pack - 1) / pack);
+      int chunks = std::max(1, std::min({8, nkt, c->num_sms / slots}));
       const int per = (nkt + chunks - 1) / chunks;
       chunks = (nkt + per - 1) / per;
       inc_chunks = std::max(inc_chunks, chunks);
+      c->adv_tab[((size_t)k * g.B + b) * 2] = s0 - g.block_len;
+      c->adv_tab[((size_t)k * g.B + b) * 2 + 1] = chunks;
       for (int ch = 0; ch < chunks; ++ch) {
         WorkItem w{};
         w.kind = ITEM_BLOCK_CHUNK; w.seq = b; w.row0 = s0 - g.block_len; w.nrows = g.block_len;
@@ -510,6 +519,8 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   CU_TRY(c, cudaMemcpy(c->d_blk_start_all, c->blk_start_all.data(), sizeof(int32_t) * c->blk_start_all.size(), cudaMemcpyHostToDevice));
   CU_TRY(c, dev_alloc(c, &c->d_pos, g.T));
   CU_TRY(c, cudaMemcpy(c->d_pos, c->pos_of_tok.data(), sizeof(int32_t) * g.T, cudaMemcpyHostToDevice));
+  CU_TRY(c, dev_alloc(c, &c->d_adv_tab, c->adv_tab.size()));
+  CU_TRY(c, cudaMemcpy(c->d_adv_tab, c->adv_tab.data(), sizeof(int32_t) * c->adv_tab.size(), cudaMemcpyHostToDevice));
   CU_TRY(c, dev_alloc(c, &c->d_items, items.size()));
   CU_TRY(c, cudaMemcpy(c->d_items, items.data(), sizeof(WorkItem) * items.size(), cudaMemcpyHostToDevice));
   {
@@ -876,9 +887,19 @@ lacache_status run_block_rows_to_state(lacache_ctx* c, lacache_ctx::ListRef list
   set_packing(c, a);
   a.n_ctas_stream = (int)std::min<long long>(c->num_sms, (long long)list.n * a.stream_slots);
   a.n_ctas = a.n_ctas_stream;
-  a.blk_to_state = 1;
-  a.st = dst;
-  return run_attention(c, a, false, s);
+  a.blk_to_state = 1;   // the units leave partial states ...
+  lacache_status st = run_attention(c, a, false, s);
+  if (st != LACACHE_OK) return st;
+  ChunkMergeArgs m{};    // ... which a launch over all rows and heads merges (the last chunk to arrive, as in a
+                         // step, would merge its heads alone, one L2 round trip after the other)
+  m.part_m = c->part_m; m.part_l = c->part_l; m.part_o = c->part_o;
+  m.max_chunks = c->part_chunks;
+  m.tab = c->d_adv_tab + (size_t)blk * c->g.B * 2;
+  m.st = dst;
+  m.no_pdl = c->knobs.no_pdl ? 1 : 0;
+  CU_TRY(c, merge_chunk_states(c->g, m, s));
+  c->last_launches++;
+  return LACACHE_OK;
 }
 
 lacache_status run_window(lacache_ctx* c, lacache_ctx::ListRef list, int blk, const StateBuffers& init,

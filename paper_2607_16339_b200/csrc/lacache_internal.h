@@ -157,6 +157,16 @@ struct ExportArgs {
   float* q_rot; float* k_rot; float* v;  // token-major outputs (may be null)
 };
 
+// Partial states [B][Hq][max_chunks][block_len] (the layout the step kernel's block-row units write) of
+// `tab[2 b + 1]` key chunks per sequence b, merged into the state of rows tab[2 b] ... of every head.
+struct ChunkMergeArgs {
+  const float* part_m; const float* part_l; const float* part_o; int max_chunks;
+  const int32_t* tab;
+  StateBuffers st;
+  int no_pdl;   // host only: launch the ordinary way
+};
+cudaError_t merge_chunk_states(const Geometry& g, const ChunkMergeArgs& a, cudaStream_t s);
+
 // ---- launchers implemented by the kernel files -----------------------------
 // Each returns the cudaError_t of the launch (cudaGetLastError()).
 // engine: LACACHE_ENGINE_SIMT or LACACHE_ENGINE_TCGEN05 (selects the storage

@@ -155,7 +155,71 @@ __global__ void __launch_bounds__(256) export_kernel(Geometry g, ExportArgs a) {
   }
 }
 
+// Partial states of the key chunks of block rows -> the rows' state (Eq. 2-6 merge): thread = 16 bytes of
+// one row of one head; every load of the (at most eight at a time) chunks is issued before any is used.
+__global__ void __launch_bounds__(256) merge_chunk_states_kernel(Geometry g, ChunkMergeArgs a) {
+  // launched programmatically dependent on the kernel that writes the partial states: the launch itself and
+  // the start of the kernel after this one overlap their neighbours; nothing is read before that kernel is complete
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int i = blockIdx.x * 256 + threadIdx.x;
+  if (i >= g.block_len * 32) return;
+  const int rr = i >> 5, ch = i & 31, h = blockIdx.y, b = blockIdx.z;
+  const int row0 = a.tab[2 * b], n = a.tab[2 * b + 1];
+  const size_t pbase = ((size_t)b * g.Hq + h) * a.max_chunks;
+  float M = -INFINITY, L = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int c0 = 0; c0 < n; c0 += 8) {
+    float mv[8], lv[8];
+    float4 v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if (c0 + k < n) {
+        const size_t pr = (pbase + c0 + k) * g.block_len + rr;
+        mv[k] = __ldcg(a.part_m + pr);
+        lv[k] = __ldcg(a.part_l + pr);
+        v[k] = __ldcg(reinterpret_cast<const float4*>(a.part_o + pr * g.d) + ch);
+      } else {
+        mv[k] = -INFINITY; lv[k] = 0.f; v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    float Mn = M;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) Mn = fmaxf(Mn, mv[k]);
+    const float w0 = (M == -INFINITY) ? 0.f : exp2f(M - Mn);
+    L *= w0; acc.x *= w0; acc.y *= w0; acc.z *= w0; acc.w *= w0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float w = (mv[k] == -INFINITY) ? 0.f : exp2f(mv[k] - Mn);
+      L = fmaf(lv[k], w, L);
+      acc.x = fmaf(v[k].x, w, acc.x);
+      acc.y = fmaf(v[k].y, w, acc.y);
+      acc.z = fmaf(v[k].z, w, acc.z);
+      acc.w = fmaf(v[k].w, w, acc.w);
+    }
+    M = Mn;
+  }
+  const size_t srow = (size_t)h * g.Tp + row0 + rr;
+  *reinterpret_cast<float4*>(a.st.o + srow * g.d + ch * 4) = acc;
+  if (ch == 0) { a.st.m[srow] = M; a.st.l[srow] = L; }
+}
+
 }  // namespace
+
+cudaError_t merge_chunk_states(const Geometry& g, const ChunkMergeArgs& a, cudaStream_t s) {
+  // (head_dim 128: 32 sixteen-byte columns per row, the only shape the tcgen05 engine serves)
+  dim3 grid((unsigned)((g.block_len * 32 + 255) / 256), (unsigned)g.Hq, (unsigned)g.B);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(256);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = a.no_pdl ? 0 : 1;
+  return cudaLaunchKernelEx(&cfg, merge_chunk_states_kernel, g, a);
+}
 
 cudaError_t rope_write(const Geometry& g, const RopeArgs& a, int engine, cudaStream_t s) {
   long long total = (long long)a.n_src_rows * (g.Hq + 2 * g.Hkv) * (g.d / 16);

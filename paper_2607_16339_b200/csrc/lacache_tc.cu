@@ -350,7 +350,8 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
     un.t1 = it.kt1;
     un.chunk = it.chunk;
     un.nchunks = it.pad;
-    // (block rows whose result is a state always go through the chunk merge, which knows where to put it)
+    // (block rows whose result is a state, not normalised rows, always leave partial states: a launch of
+    // its own merges them)
     un.epi = (it.pad > 1 || a.blk_to_state) ? EPI_PARTIAL : EPI_OUT;
     un.q_rows = un.rh ? BM : 64;
   } else {
@@ -668,29 +669,13 @@ __device__ __forceinline__ void coop_store_out_rows(const Cta& c, const AttnArgs
   }
 }
 
-// One 16-byte column of a merged row: the normalised output (and lse), or -- when the launch computes
-// the block rows' state for the incremental build -- the unnormalised triple itself.
-__device__ __forceinline__ void store_merged(const Geometry& g, const AttnArgs& a, int row, int h, int ch, float M,
-                                             float L, float4 acc) {
-  if (a.blk_to_state) {
-    const size_t srow = (size_t)h * g.Tp + row;
-    *reinterpret_cast<float4*>(a.st.o + srow * D + ch * 4) = acc;
-    if (ch == 0) { a.st.m[srow] = M; a.st.l[srow] = L; }
-    return;
-  }
-  const float LN2 = 0.69314718055994530942f;
-  const float inv = 1.f / L;
-  const size_t orow = (size_t)row * g.Hq + h;
-  store_out4(a, orow * D + ch * 4, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
-  if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
-}
-
 // Few chunks (at most NC): each thread takes BATCH (row, 16-byte column) items at a
 // time and issues every load of the batch -- references, normalisers, 16 bytes of
 // each partial O~ -- before any is used: one L2 round trip per batch.
 template <int NC, int BATCH>
 __device__ __forceinline__ void merge_few(const Geometry& g, const AttnArgs& a, size_t pbase, int nchunks,
                                           int block_len, int row0, int h) {
+  const float LN2 = 0.69314718055994530942f;
   const int t = threadIdx.x - 64;
   const int n_items = block_len * 32;
   for (int i0 = t; i0 < n_items; i0 += BATCH * ROW_THREADS) {
@@ -728,7 +713,10 @@ __device__ __forceinline__ void merge_few(const Geometry& g, const AttnArgs& a, 
         acc.z = fmaf(v[bi][k].z, w, acc.z);
         acc.w = fmaf(v[bi][k].w, w, acc.w);
       }
-      store_merged(g, a, row0 + rr, h, ch, M, L, acc);
+      const float inv = 1.f / L;
+      const size_t orow = (size_t)(row0 + rr) * g.Hq + h;
+      store_out4(a, orow * D + ch * 4, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
+      if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
     }
   }
 }
@@ -738,6 +726,7 @@ __device__ __forceinline__ void merge_few(const Geometry& g, const AttnArgs& a, 
 // read with coalesced loads straight from L2 and the normalised rows written out.
 __device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs& a, size_t pbase, int nchunks,
                                                int block_len, int row0, int h) {
+  const float LN2 = 0.69314718055994530942f;
   const int t = threadIdx.x - 64;
   if (nchunks <= 2) {
     merge_few<2, 4>(g, a, pbase, nchunks, block_len, row0, h);
@@ -779,7 +768,10 @@ __device__ __forceinline__ void merge_partials(const Geometry& g, const AttnArgs
         acc.w = fmaf(v[k].w, w[k], acc.w);
       }
     }
-    store_merged(g, a, row0 + rr, h, ch, M, L, acc);
+    const float inv = 1.f / L;
+    const size_t orow = (size_t)(row0 + rr) * g.Hq + h;
+    store_out4(a, orow * D + ch * 4, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
+    if (ch == 0 && a.lse) a.lse[orow] = (M + log2f(L)) * LN2;
   }
 }
 
@@ -1108,6 +1100,10 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       tc_fence_before();
       mbar_arrive(c.bar(BAR_O_FREE));  // the next unit may overwrite O~
       if (!epi_sync(c, epi_phase)) return;  // every partial store of the CTA happens-before thread 64's fence
+      if (a.blk_to_state) {  // merged into the rows' state by the launch that follows: nothing to count
+        if (un.q_rows == BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));
+        continue;
+      }
       if (threadIdx.x == 64) {
         __threadfence();  // cumulative: publishes the whole CTA's partial state before the counts
         uint32_t last_bits = 0;   // bit j: this chunk was the last of head un.h + j to arrive

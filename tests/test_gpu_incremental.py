@@ -92,6 +92,14 @@ def test_advanced_context_serves_steps_like_a_rebuilt_one(case):
     _run(small_workload(name=case, **CASES[case]), seed=21)
 
 
+def test_advance_with_the_finished_rows_as_window_units(monkeypatch):
+    """The finished block's rows over the keys before the next block: by default block-row units of the
+    step kernel over key chunks plus a merge launch; behind a knob, key-window units of the build kernel."""
+    monkeypatch.setenv("LACACHE_NO_CHUNKED_ADVANCE", "1")      # (read when a context is created)
+    _run(small_workload(name="long-window", **CASES["long"]), seed=22)
+    monkeypatch.delenv("LACACHE_NO_CHUNKED_ADVANCE")
+
+
 @pytest.mark.parametrize("case", ["gqa64", "long", "noprompt", "mha64"])
 def test_advanced_context_with_plain_operands(case):
     """The same walk with precision_mode = plain (128-key tiles in the key-window units) on the value
