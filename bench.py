@@ -444,6 +444,43 @@ def run_cuda(args):
     torch.cuda.synchronize()
     flush_step_ms = statistics.mean(a.elapsed_time(b) for a, b in fl_pairs)
     del flush
+    # ---- for context: a plain device-to-device copy that moves the step kernel's algorithmic bytes (half of
+    # them read, half written), under both timing protocols of the step; what a launch of this size can reach ----
+    copy_ref = None
+    try:
+        nb = int(counts["step_attn_bytes"]) // 2
+        rc = max(2, min(R, (4 << 30) // max(2 * nb, 1)))
+        srcs = [torch.empty(nb, dtype=torch.uint8, device=dev) for _ in range(rc)]
+        dsts = [torch.empty(nb, dtype=torch.uint8, device=dev) for _ in range(rc)]
+        n_cp = max(4 * rc, 32)
+        for i in range(rc):
+            dsts[i].copy_(srcs[i])
+        torch.cuda.synchronize()
+        e0, e1 = mk(), mk()
+        e0.record()
+        for i in range(n_cp):
+            dsts[i % rc].copy_(srcs[i % rc])
+        e1.record()
+        torch.cuda.synchronize()
+        cp_b2b = e0.elapsed_time(e1) / n_cp
+        cp_pairs = []
+        for i in range(n_cp):
+            e = (mk(), mk())
+            e[0].record(); dsts[i % rc].copy_(srcs[i % rc]); e[1].record()
+            cp_pairs.append(e)
+            if i % 4 == 3:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        cp_ev = statistics.mean(a.elapsed_time(b) for a, b in cp_pairs)
+        copy_ref = {"bytes": 2 * nb, "back_to_back_us": round(cp_b2b * 1e3, 2), "event_bracketed_us": round(cp_ev * 1e3, 2),
+                    "back_to_back_gbs": round(2 * nb / (cp_b2b * 1e-3) / 1e9, 1),
+                    "event_bracketed_gbs": round(2 * nb / (cp_ev * 1e-3) / 1e9, 1), "buffers": rc,
+                    "how": "torch copy_ between two device buffers of half the step kernel's algorithmic bytes each, "
+                           "buffer pairs visited round-robin: context for the fraction above (the measured peak is a "
+                           "2 GB copy; a launch of this size cannot reach it), not a denominator"}
+        del srcs, dsts
+    except Exception as ex:
+        sys.stderr.write("same-size copy skipped: %r\n" % (ex,))
     clocks.mark()      # window: the headline repeats, the per-kernel passes, the full recompute and the flushed pass
     clock_info = clocks.stop()
 
@@ -529,6 +566,8 @@ def run_cuda(args):
                        "the library (the pair keeps the launch from overlapping its neighbours and contains its "
                        "launch latency)",
                 "algorithmic_bytes_per_launch": counts["step_attn_bytes"]}
+        if copy_ref:
+            roof["copy_of_the_same_bytes"] = copy_ref
         if span:
             a2 = counts["step_attn_bytes"] / (span["step_us"] * 1e-6) / 1e9
             roof["overlapped"] = dict(span, achieved=round(a2, 1), frac=round(a2 / peaks["hbm_gbs"], 4),
