@@ -94,13 +94,18 @@ __global__ void __launch_bounds__(SAMPLE_THREADS, 4) sample_rows_kernel(SampleAr
       // Four independent 16-byte loads in flight per thread, then two batches of two vectors each
       // (batch_add: the lanes of a warp move their running maxima at different elements, so a
       // per-element branch would run both of its sides -- two exponentials, and the exponential
-      // unit is what bounds this kernel -- nearly every time).
+      // unit is what bounds this kernel -- nearly every time).  A slice is often shorter than four
+      // vectors per thread (a block of 32 rows on 148 SMs gets ~18 slices of ~7000 entries a row): the
+      // vectors past its end are filled with -inf, which adds nothing, so that the loads a thread does
+      // have still leave together instead of one round trip after the other.
       constexpr int STEP = SAMPLE_THREADS * VEC;
-      int i = lo + threadIdx.x * VEC;
-      for (; i + 3 * STEP < hi_v; i += 4 * STEP) {
+      const uint32_t ninf = sizeof(T) == 2 ? 0xFF80FF80u : 0xFF800000u;
+      for (int i = lo + threadIdx.x * VEC; i < hi_v; i += 4 * STEP) {
         uint4 raw[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) raw[u] = *reinterpret_cast<const uint4*>(x + i + u * STEP);
+        for (int u = 0; u < 4; ++u)
+          raw[u] = (i + u * STEP < hi_v) ? *reinterpret_cast<const uint4*>(x + i + u * STEP)
+                                         : make_uint4(ninf, ninf, ninf, ninf);
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           float f[2 * VEC];
@@ -112,14 +117,6 @@ __global__ void __launch_bounds__(SAMPLE_THREADS, 4) sample_rows_kernel(SampleAr
           }
           batch_add<2, VEC>(acc, f, i + 2 * h * STEP, STEP);
         }
-      }
-      for (; i < hi_v; i += STEP) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(x + i);
-        const T* e = reinterpret_cast<const T*>(&raw);
-        float f[VEC];
-#pragma unroll
-        for (int j = 0; j < VEC; ++j) f[j] = to_float(e[j]);
-        batch_add<1, VEC>(acc, f, i, STEP);
       }
       for (int i = hi_v + threadIdx.x; i < hi; i += SAMPLE_THREADS) acc_add(acc, to_float(x[i]), i);
     } else {
