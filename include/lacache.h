@@ -77,9 +77,15 @@ enum { LACACHE_OUT_BF16 = 0, LACACHE_OUT_FP32 = 1 };
  *          (16 significant bits): needed for the LLaDA-shaped configurations whose per-head scale
  *          reaches 2 and whose keys carry 4x outliers.  Twice the Q'/K' bytes and twice the
  *          tensor-core work of PLAIN.
+ *   FP16   one fp16 plane per tensor (the rotated value rounded once to fp16, saturated to the finite
+ *          range), one product per score tile, 128-key tiles: PLAIN's cost with three more significant
+ *          bits (~2^-12 * |s| per score).  Holds the tolerance at per-head scales of 2 with a factor of
+ *          about two in hand on the maximum and four on the mean (measured against the fp64 evaluation
+ *          on the LLaDA-shaped configurations, outlier keys included); SPLIT has a factor of twenty.
+ *          Rotated values beyond the fp16 range (|x| > 65504) saturate: inputs of that size need SPLIT.
  * The fp32 CUDA-core engine ignores the mode (its operands are fp32).
  */
-enum { LACACHE_PRECISION_PLAIN = 0, LACACHE_PRECISION_SPLIT = 1 };
+enum { LACACHE_PRECISION_PLAIN = 0, LACACHE_PRECISION_SPLIT = 1, LACACHE_PRECISION_FP16 = 2 };
 /*
  * What a build caches (Sec. 3.3.3 last paragraph; Algorithm 1's Q_overlap / K_overlap predicates):
  *   TOKEN  the index sets U and C of Sec. 3.3.1 at token granularity: every fixed row keeps a state

@@ -219,8 +219,9 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
 
   if (cfg->out_dtype != LACACHE_OUT_BF16 && cfg->out_dtype != LACACHE_OUT_FP32)
     return fail(c, LACACHE_ERR_INVALID_ARG, "out_dtype %d", cfg->out_dtype);
-  if (cfg->precision_mode != LACACHE_PRECISION_PLAIN && cfg->precision_mode != LACACHE_PRECISION_SPLIT)
-    return fail(c, LACACHE_ERR_UNSUPPORTED, "precision_mode %d (0 = plain bf16 operands, 1 = split)", cfg->precision_mode);
+  if (cfg->precision_mode != LACACHE_PRECISION_PLAIN && cfg->precision_mode != LACACHE_PRECISION_SPLIT &&
+      cfg->precision_mode != LACACHE_PRECISION_FP16)
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "precision_mode %d (0 = plain bf16 operands, 1 = split, 2 = plain fp16 operands)", cfg->precision_mode);
   if (cfg->cache_granularity != LACACHE_GRANULARITY_TOKEN && cfg->cache_granularity != LACACHE_GRANULARITY_TILE)
     return fail(c, LACACHE_ERR_INVALID_ARG, "cache_granularity %d", cfg->cache_granularity);
   bool tc_ok = cfg->dtype == LACACHE_DTYPE_BF16 && cfg->head_dim == 128 && cfg->block_len <= TC_MAX_BLOCK;
@@ -273,6 +274,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
   // ---- work lists ----
   const bool tc = c->engine == LACACHE_ENGINE_TCGEN05;
   c->split = cfg->precision_mode == LACACHE_PRECISION_SPLIT;
+  c->g.op_f16 = (c->engine == LACACHE_ENGINE_TCGEN05 && cfg->precision_mode == LACACHE_PRECISION_FP16) ? 1 : 0;
   const int TC_KEYS = tc_keys(c->split);
   const int R = tc ? TC_ROWS : SIMT_ROWS;
   std::vector<WorkItem> items;

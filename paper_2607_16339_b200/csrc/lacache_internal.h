@@ -61,6 +61,7 @@ struct Geometry {
   int Hq, Hkv, d, group;
   int gen_len, block_len, n_blk;
   float scale_log2;  // softmax_scale * log2(e)
+  int op_f16;        // tcgen05 engine, one-plane modes: the rotated Q', K' planes hold fp16 (else bf16)
 };
 
 // Rotated cache / scratch set.  SIMT engine: fp32 planes (q, k, v).

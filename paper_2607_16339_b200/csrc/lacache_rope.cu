@@ -24,7 +24,11 @@ __device__ __forceinline__ void store8_f32(void* plane, size_t off, const float 
 }
 
 __device__ __forceinline__ void store8_split(void* hi_plane, void* lo_plane, size_t off,
-                                             const float (&y)[8]) {
+                                             const float (&y)[8], bool f16) {
+  if (f16) {   // one fp16 plane: the rotated value rounded once to fp16
+    *reinterpret_cast<uint4*>(reinterpret_cast<__half*>(hi_plane) + off) = rope_half8(y);
+    return;
+  }
   uint4 uh, ul;
   rope_split8(y, uh, ul);
   *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(hi_plane) + off) = uh;
@@ -100,11 +104,11 @@ __global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a)
     const size_t o1 = ((size_t)(2 * h) * g.Tp + tok) * 64 + c0;
     const size_t o2 = ((size_t)(2 * h + 1) * g.Tp + tok) * 64 + c0;
     if (which == 0) {
-      store8_split(a.dst.q_hi, a.dst.q_lo, o1, y1);
-      store8_split(a.dst.q_hi, a.dst.q_lo, o2, y2);
+      store8_split(a.dst.q_hi, a.dst.q_lo, o1, y1, g.op_f16 != 0);
+      store8_split(a.dst.q_hi, a.dst.q_lo, o2, y2, g.op_f16 != 0);
     } else if (which == 1) {
-      store8_split(a.dst.k_hi, a.dst.k_lo, o1, y1);
-      store8_split(a.dst.k_hi, a.dst.k_lo, o2, y2);
+      store8_split(a.dst.k_hi, a.dst.k_lo, o1, y1, g.op_f16 != 0);
+      store8_split(a.dst.k_hi, a.dst.k_lo, o2, y2, g.op_f16 != 0);
     } else {
       store8_f16(a.dst.v, o1, y1);
       store8_f16(a.dst.v, o2, y2);
@@ -118,7 +122,8 @@ __global__ void __launch_bounds__(256) rope_write_kernel(Geometry g, RopeArgs a)
 
 // Export kernels: head-major storage -> token-major fp32.
 template <bool TC>
-__device__ __forceinline__ float read_rot(const void* hi, const void* lo, size_t off) {
+__device__ __forceinline__ float read_rot(const void* hi, const void* lo, size_t off, bool f16) {
+  if (TC && f16) return __half2float(reinterpret_cast<const __half*>(hi)[off]);
   if (TC) {
     return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(hi)[off]) +
            (lo ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(lo)[off]) : 0.f);
@@ -144,10 +149,10 @@ __global__ void __launch_bounds__(256) export_kernel(Geometry g, ExportArgs a) {
     if (a.m) a.m[(size_t)tok * g.Hq + h] = a.st.m[(size_t)h * g.Tp + tok] * LN2;
     if (a.l) a.l[(size_t)tok * g.Hq + h] = a.st.l[(size_t)h * g.Tp + tok];
   }
-  if (a.q_rot) a.q_rot[idx] = read_rot<TC>(a.rot.q_hi, a.rot.q_lo, src);
+  if (a.q_rot) a.q_rot[idx] = read_rot<TC>(a.rot.q_hi, a.rot.q_lo, src, g.op_f16 != 0);
   if (h < g.Hkv) {
     size_t dst = ((size_t)tok * g.Hkv + h) * g.d + c;
-    if (a.k_rot) a.k_rot[dst] = read_rot<TC>(a.rot.k_hi, a.rot.k_lo, src);
+    if (a.k_rot) a.k_rot[dst] = read_rot<TC>(a.rot.k_hi, a.rot.k_lo, src, g.op_f16 != 0);
     if (a.v) {
       a.v[dst] = TC ? __half2float(reinterpret_cast<const __half*>(a.rot.v)[src])
                     : reinterpret_cast<const float*>(a.rot.v)[src];

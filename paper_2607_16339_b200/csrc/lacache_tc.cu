@@ -574,7 +574,8 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   constexpr bool STEP = KIND == KIND_STEP;
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
-  constexpr uint32_t IDESC_S = idesc_f16(1u /*bf16*/, 0u, BM, BN);
+  // (operand format of the score product: bf16 planes, or fp16 in the one-plane fp16 mode)
+  const uint32_t IDESC_S = idesc_f16((!SPLIT && g.op_f16) ? 0u : 1u, 0u, BM, BN);
   int uu = 0;
   uint32_t js = 0;  // score tiles issued so far (stage and buffer = js & 1, phase = (js >> 1) & 1)
   for (int u = first; u < n_units; u += stride, ++uu) {
@@ -823,8 +824,13 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
         sn[0] = sa.x; sn[1] = sa.y; sn[2] = sa.z; sn[3] = sa.w; sn[4] = sb.x; sn[5] = sb.y; sn[6] = sb.z; sn[7] = sb.w;
         rope_rotate8(x1, x2, cs, sn, y1, y2);
         uint4 h1, l1, h2, l2;
-        rope_split8(y1, h1, l1);
-        rope_split8(y2, h2, l2);
+        if (!SPLIT && g.op_f16) {
+          h1 = rope_half8(y1);
+          h2 = rope_half8(y2);
+        } else {
+          rope_split8(y1, h1, l1);
+          rope_split8(y2, h2, l2);
+        }
         uint8_t* const q0 = c.gen + SM_Q + qi * 128 + ((ch ^ (qi & 7)) << 4);
         *reinterpret_cast<uint4*>(q0) = h1;                 // hi plane, features [0, 64)
         *reinterpret_cast<uint4*>(q0 + box) = h2;           // hi plane, features [64, 128)
@@ -1345,7 +1351,7 @@ __device__ void merge_producer(const Cta& c, const TcMaps& maps, const Geometry&
 template <bool SPLIT>
 __device__ void merge_mma(const Cta& c, const Geometry& g, const AttnArgs& a, int first, int stride, int n_units) {
   const int n_s = (g.block_len + 15) & ~15;  // score columns (keys), a multiple of 16
-  const uint32_t idesc_s = idesc_f16(1u, 0u, BM, (uint32_t)n_s);
+  const uint32_t idesc_s = idesc_f16((!SPLIT && g.op_f16) ? 0u : 1u, 0u, BM, (uint32_t)n_s);
   int uu = 0;
   if (first < n_units) {
     if (!wait_bar(c, BAR_Q_FULL, 0, LOC_WAIT_Q)) return;
@@ -1605,7 +1611,7 @@ template <bool SPLIT>
 __device__ void deep_mma(const Cta& c, const Geometry& g, int n_my, bool kv_computed) {
   if (n_my == 0) return;
   const int n_s = (g.block_len + 15) & ~15;
-  const uint32_t idesc_s = idesc_f16(1u, 0u, BM, (uint32_t)n_s);
+  const uint32_t idesc_s = idesc_f16((!SPLIT && g.op_f16) ? 0u : 1u, 0u, BM, (uint32_t)n_s);
   const uint32_t kb = c.base + DM_K;
   if (!wait_bar(c, BAR_Q_FULL, 0, LOC_WAIT_Q)) return;
   if (!wait_bar(c, BAR_KV_FULL, 0, LOC_WAIT_K)) return;
@@ -1679,8 +1685,13 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
       sn[0] = sa.x; sn[1] = sa.y; sn[2] = sa.z; sn[3] = sa.w; sn[4] = sb.x; sn[5] = sb.y; sn[6] = sb.z; sn[7] = sb.w;
       rope_rotate8(x1, x2, cs, sn, y1, y2);
       uint4 h1, l1, h2, l2;
-      rope_split8(y1, h1, l1);
-      rope_split8(y2, h2, l2);
+      if (!SPLIT && g.op_f16) {
+        h1 = rope_half8(y1);
+        h2 = rope_half8(y2);
+      } else {
+        rope_split8(y1, h1, l1);
+        rope_split8(y2, h2, l2);
+      }
       uint8_t* const k0 = c.gen + DM_K + ki * 128 + ((ch ^ (ki & 7)) << 4);
       *reinterpret_cast<uint4*>(k0) = h1;
       *reinterpret_cast<uint4*>(k0 + DM_KBOX) = h2;

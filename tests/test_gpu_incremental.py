@@ -110,6 +110,14 @@ def test_advanced_context_with_plain_operands(case):
     _run(small_workload(name=case, **kw), seed=22, precision_mode=binding.PRECISION_PLAIN)
 
 
+@pytest.mark.parametrize("case", ["gqa64", "long", "ragged3", "mha64"])
+def test_advanced_context_with_fp16_operands(case):
+    """The same walk with precision_mode = fp16 (one fp16 plane per operand) at the harsh value scale."""
+    kw = dict(CASES[case]) if case in CASES else dict(prompt_lens=(700, 333, 61), gen_len=192, block_len=64, steps=1,
+                                                       hq=4, hkv=4)
+    _run(small_workload(name=case, **kw), seed=23, precision_mode=binding.PRECISION_FP16)
+
+
 @pytest.mark.parametrize("block_len", [48, 64])
 def test_advanced_context_mha_blocks_of_48_and_64_rows(block_len):
     """No grouped heads, blocks of 33..64 rows, per-head scales up to 2, ragged, long prompts."""

@@ -29,7 +29,8 @@ def draw_case(seed):
     batch = int(rng.integers(1, 5))
     prompts = tuple(int(x) for x in rng.choice([0, 3, 40, 95, 96, 130, 257, 390, 520], size=batch))
     n_blocks = int(rng.integers(2, 5))
-    plain = bool(rng.integers(2))
+    mode = int(rng.integers(3))      # 0: one bf16 plane (small scores), 1: split bf16 planes, 2: one fp16 plane
+    plain = mode == 0
     wl_kw = dict(prompt_lens=prompts, gen_len=n_blocks * block_len, block_len=block_len, steps=int(rng.integers(1, 3)),
                  hq=hq, hkv=hkv, scale_mode="inv_sqrt_d" if plain else "per_head_u(0.5,2)")
     knobs = {}
@@ -43,7 +44,7 @@ def draw_case(seed):
         knobs["LACACHE_NO_QCOMP"] = "1"
     if rng.integers(4) == 0:
         knobs["LACACHE_DEEP_UNITS"] = str(int(rng.choice([1, 2, 5])))
-    ctx_kw = dict(precision_mode=binding.PRECISION_PLAIN if plain else binding.PRECISION_SPLIT,
+    ctx_kw = dict(precision_mode=(binding.PRECISION_PLAIN, binding.PRECISION_SPLIT, binding.PRECISION_FP16)[mode],
                   cache_granularity=binding.GRANULARITY_TILE if rng.integers(3) == 0 else binding.GRANULARITY_TOKEN)
     return wl_kw, knobs, ctx_kw
 

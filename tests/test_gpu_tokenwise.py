@@ -211,12 +211,13 @@ def test_hidden_state_entry_and_bad_token_id(small_model):
     prod.destroy()
 
 
-@pytest.mark.parametrize("shape", ["mha", "gqa-ragged"])
+@pytest.mark.parametrize("shape", ["mha", "gqa-ragged", "mha-fp16"])
 def test_build_and_step_from_token_ids(shape):
     """Algorithm 1 fed by token ids: build_tokens over all T tokens, then step_tokens over the block's
     tokens; checked against the oracle chain (token-wise oracle at model precision -> attention
     oracle) and, bit for bit, against lacache_build / lacache_step fed with the projected rows."""
-    if shape == "mha":
+    ctx_kw = dict(precision_mode=binding.PRECISION_FP16) if shape == "mha-fp16" else {}
+    if shape in ("mha", "mha-fp16"):
         wl = W.small_workload(prompt_lens=(200,), gen_len=96, block_len=32, steps=3, hq=4, hkv=4)
     else:
         wl = W.small_workload(prompt_lens=(150, 61), gen_len=128, block_len=64, steps=2, hq=8, hkv=2,
@@ -224,8 +225,8 @@ def test_build_and_step_from_token_ids(shape):
     tm = TokenModel(wl, 512, 3000)
     T, nb = wl.total_tokens, wl.batch * wl.block_len
     prod = make_producer(tm, T)
-    ctx = make_ctx(wl)
-    ctx2 = make_ctx(wl)
+    ctx = make_ctx(wl, **ctx_kw)
+    ctx2 = make_ctx(wl, **ctx_kw)
     sch = SyntheticSchedule(wl)   # index sets only
     b = 1
     ids_full = tm.full_ids(b)

@@ -30,6 +30,8 @@ def _emulate(seed, qk_mode, p_round, N=768, P=512, Lb=32, scale_h=2.0, tile=128)
     qf, kf = qr.float().double(), kr.float().double()
     if qk_mode == "bf16":
         S = _bf(qf) @ _bf(kf).T
+    elif qk_mode == "fp16":
+        S = _f16(qf) @ _f16(kf).T
     else:
         qh, kh = _bf(qf), _bf(kf)
         ql, kl = _bf(qf - qh), _bf(kf - kh)
@@ -96,3 +98,17 @@ def test_plain_operands_hold_where_the_scores_are_small():
     assert rows[0.5][0] < 2e-2 and rows[0.5][1] < 2e-3     # scores of order 3: still inside
     assert rows[2.0][0] > 2e-2                             # scores of order 50: outside
     assert rows[0.5][0] < rows[1.0][0] < rows[2.0][0]
+
+
+def test_one_fp16_plane_holds_at_the_harsh_scale_with_a_smaller_margin_than_the_split():
+    """fp16 keeps three more significant bits than bf16, so one fp16 plane per operand moves a score by
+    about 2^-12 |s|: at per-head scale 2 (scores of order 50), where one bf16 plane is outside the bar by
+    a factor of three, it is inside by a factor of about two on the maximum and four on the mean; the
+    split planes are inside by a factor of twenty.  Both paths round alike, so cached and recomputed
+    outputs still agree."""
+    for seed in range(3):
+        emax, emean, diff = _emulate(seed, "fp16", _f16)
+        assert emax < 1.2e-2 and emean < 7e-4
+        assert diff < 1e-3
+        smax, smean, _ = _emulate(seed, "split", _f16)
+        assert smax < emax and smean < emean
