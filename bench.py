@@ -934,7 +934,8 @@ def token_path_leg(wl, dev, peaks, seed, n_steps, precision):
 # and precision mode.  The fp32 output (12.6 MB) is still in L2 when the
 # kernel ends, so the figure is dominated by reads.
 DEFAULT_PRECISION = {1: 1, 2: 2, 3: 1, 4: 2, 5: 2, 6: 2}   # binding.PRECISION_*: 1 = split bf16 planes, 2 = one fp16 plane
-TRAFFIC_PER_LAUNCH = {(2, 1): 48370432, (3, 1): 93736960, (4, 1): 460605952, (5, 1): 209015552, (5, 0): 161659392}   # (config, precision mode)
+TRAFFIC_PER_LAUNCH = {(2, 1): 48370432, (3, 1): 93736960, (4, 1): 460605952, (5, 1): 209015552, (5, 0): 161659392,
+                      (2, 2): 34979584, (4, 2): 345821952, (5, 2): 161281536}   # (config, precision mode)
 
 
 # ----------------------------------------------------------------------------
