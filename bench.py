@@ -933,9 +933,9 @@ def token_path_leg(wl, dev, peaks, seed, n_steps, precision):
 # tc_attn_kernel_cfg5_{split,plain}_ncu_full.txt), bytes; None where no capture exists for the workload
 # and precision mode.  The fp32 output (12.6 MB) is still in L2 when the
 # kernel ends, so the figure is dominated by reads.
-DEFAULT_PRECISION = {1: 1, 2: 2, 3: 1, 4: 2, 5: 2, 6: 2}   # binding.PRECISION_*: 1 = split bf16 planes, 2 = one fp16 plane
+DEFAULT_PRECISION = {1: 1, 2: 3, 3: 1, 4: 3, 5: 3, 6: 3}   # binding.PRECISION_*: 1 = split bf16 planes, 3 = one fp16 plane
 TRAFFIC_PER_LAUNCH = {(2, 1): 48370432, (3, 1): 93736960, (4, 1): 460605952, (5, 1): 209015552, (5, 0): 161659392,
-                      (2, 2): 34979584, (4, 2): 345821952, (5, 2): 161281536}   # (config, precision mode)
+                      (2, 3): 34979584, (4, 3): 345821952, (5, 3): 161281536}   # (config, precision mode)
 
 
 # ----------------------------------------------------------------------------
@@ -1038,7 +1038,7 @@ def main():
     ap.add_argument("--no-split-leg", action="store_true", help="skip the extra leg with split bf16 operands")
     ap.add_argument("--no-tile-granular", action="store_true", help="skip the extra leg with tile-granular caching")
     ap.add_argument("--precision-mode", type=int, default=-1,
-                    help="0 = one bf16 plane per operand (suits the small-score configurations 5 and 6), 1 = split bf16 planes (any input), 2 = one fp16 plane (default except for configuration 3, whose outlier keys need the split)")
+                    help="0 = one bf16 plane per operand (suits the small-score configurations 5 and 6), 1 = split bf16 planes (any input), 3 = one fp16 plane (default except for configuration 3, whose outlier keys need the split)")
     ap.add_argument("--out-dtype", default="f32", choices=["f32", "bf16"])
     args = ap.parse_args()
     if args.warmup < 3:

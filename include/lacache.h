@@ -85,7 +85,8 @@ enum { LACACHE_OUT_BF16 = 0, LACACHE_OUT_FP32 = 1 };
  *          Rotated values beyond the fp16 range (|x| > 65504) saturate: inputs of that size need SPLIT.
  * The fp32 CUDA-core engine ignores the mode (its operands are fp32).
  */
-enum { LACACHE_PRECISION_PLAIN = 0, LACACHE_PRECISION_SPLIT = 1, LACACHE_PRECISION_FP16 = 2 };
+enum { LACACHE_PRECISION_PLAIN = 0, LACACHE_PRECISION_SPLIT = 1, LACACHE_PRECISION_FP16 = 3 };
+/* (2 is reserved: split planes plus split probabilities, which this library does not offer) */
 /*
  * What a build caches (Sec. 3.3.3 last paragraph; Algorithm 1's Q_overlap / K_overlap predicates):
  *   TOKEN  the index sets U and C of Sec. 3.3.1 at token granularity: every fixed row keeps a state

@@ -16,7 +16,7 @@ OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_STATE, ERR_UNSUPPORTED, ERR_OOM, ERR_CUDA, E
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 ENGINE_AUTO, ENGINE_SIMT, ENGINE_TCGEN05 = 0, 1, 2
 OUT_BF16, OUT_FP32 = 0, 1
-PRECISION_PLAIN, PRECISION_SPLIT, PRECISION_FP16 = 0, 1, 2
+PRECISION_PLAIN, PRECISION_SPLIT, PRECISION_FP16 = 0, 1, 3
 GRANULARITY_TOKEN, GRANULARITY_TILE = 0, 1
 
 EXPORTS = [

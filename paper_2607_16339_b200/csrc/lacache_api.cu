@@ -221,7 +221,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     return fail(c, LACACHE_ERR_INVALID_ARG, "out_dtype %d", cfg->out_dtype);
   if (cfg->precision_mode != LACACHE_PRECISION_PLAIN && cfg->precision_mode != LACACHE_PRECISION_SPLIT &&
       cfg->precision_mode != LACACHE_PRECISION_FP16)
-    return fail(c, LACACHE_ERR_UNSUPPORTED, "precision_mode %d (0 = plain bf16 operands, 1 = split, 2 = plain fp16 operands)", cfg->precision_mode);
+    return fail(c, LACACHE_ERR_UNSUPPORTED, "precision_mode %d (0 = one bf16 plane per operand, 1 = split bf16 planes, 3 = one fp16 plane)", cfg->precision_mode);
   if (cfg->cache_granularity != LACACHE_GRANULARITY_TOKEN && cfg->cache_granularity != LACACHE_GRANULARITY_TILE)
     return fail(c, LACACHE_ERR_INVALID_ARG, "cache_granularity %d", cfg->cache_granularity);
   bool tc_ok = cfg->dtype == LACACHE_DTYPE_BF16 && cfg->head_dim == 128 && cfg->block_len <= TC_MAX_BLOCK;

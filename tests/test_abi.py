@@ -51,7 +51,8 @@ def test_create_rejects_bad_configs_without_gpu():
         (cfg(rope_theta=0.0), binding.ERR_INVALID_ARG),
         (cfg(engine=2, dtype=1), binding.ERR_UNSUPPORTED),
         (cfg(out_dtype=2), binding.ERR_INVALID_ARG),
-        (cfg(precision_mode=3), binding.ERR_UNSUPPORTED),       # a split of the probabilities is not offered
+        (cfg(precision_mode=2), binding.ERR_UNSUPPORTED),       # a split of the probabilities is not offered
+        (cfg(precision_mode=4), binding.ERR_UNSUPPORTED),       # no such mode
         (cfg(cache_granularity=5), binding.ERR_INVALID_ARG),
         (cfg(cache_granularity=binding.GRANULARITY_TILE, dtype=1), binding.ERR_UNSUPPORTED),   # tcgen05 engine only
     ]
