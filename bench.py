@@ -230,8 +230,9 @@ class RoundRobin:
             self.ctxs[c].step(*tens, *self.outs[c])
             self.local[c] = first
 
-    def run(self, n_calls=None, on_call=None):
-        """The calls themselves.  Returns (kernel launches, builds)."""
+    def run(self, n_calls=None, on_call=None, stream=None):
+        """The calls themselves (on `stream`, default the current one).  Returns (kernel launches, builds)."""
+        kw = {} if stream is None else {"stream": stream}
         launches = builds = 0
         for j in range(self.K if n_calls is None else n_calls):
             c = j % self.R
@@ -240,14 +241,14 @@ class RoundRobin:
             if s == 0:
                 if on_call:
                     on_call("build", ctx)
-                ctx.build(blk, *self.sched.full[blk])
+                ctx.build(blk, *self.sched.full[blk], **kw)
                 launches += ctx.last_launch_count
                 builds += 1
                 if on_call:
                     on_call("built", ctx)
             if on_call:
                 on_call("step", ctx)
-            ctx.step(*tens, *self.outs[c])
+            ctx.step(*tens, *self.outs[c], **kw)
             launches += ctx.last_launch_count
             if on_call:
                 on_call("stepped", ctx)
@@ -255,9 +256,13 @@ class RoundRobin:
         return launches, builds
 
 
-def timed_region(rr, W, min_ms=50.0, max_repeats=200):
+def timed_region(rr, W, min_ms=50.0, max_repeats=200, graph=True):
     """W untimed warm-up calls, then the K-call region `repeats` times, each bracketed by one event pair
     (barrier + synchronize on both sides) after an untimed pass that puts every replica at its phase.
+    With `graph` the K calls (the library's own launches, in the same order, programmatic dependencies
+    included) are captured once into a CUDA graph and every repeat replays it: the host's time to enqueue
+    two launches per step through Python is of the order of the step itself, and a denoising loop that
+    cares captures its step the same way.  rr.launch says which of the two ran.
     Returns (per-repeat ms, launches per repeat, builds per repeat, wall seconds of the timed regions)."""
     import math
     import torch
@@ -265,8 +270,23 @@ def timed_region(rr, W, min_ms=50.0, max_repeats=200):
     rr.prepare()
     rr.run(W)
     torch.cuda.synchronize()
-    times, wall = [], 0.0
+    g = gs = None
     launches = builds = 0
+    if graph:
+        try:
+            gs = torch.cuda.Stream()
+            rr.prepare()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(gs):
+                with torch.cuda.graph(g, stream=gs):
+                    launches, builds = rr.run(stream=gs.cuda_stream)
+            torch.cuda.synchronize()
+        except Exception as ex:      # (capture is a convenience of the harness: without it the calls are issued one by one)
+            sys.stderr.write("graph capture of the timed region skipped: %r\n" % (ex,))
+            g = None
+    rr.launch = "cuda graph replay" if g is not None else "eager"
+    times, wall = [], 0.0
     repeats = 1
     i = 0
     while i < repeats:
@@ -274,9 +294,15 @@ def timed_region(rr, W, min_ms=50.0, max_repeats=200):
         torch.cuda.synchronize(); barrier()
         t0 = time.perf_counter()
         e0, e1 = mk(), mk()
-        e0.record()
-        launches, builds = rr.run()
-        e1.record()
+        if g is not None:
+            with torch.cuda.stream(gs):
+                e0.record()
+                g.replay()
+                e1.record()
+        else:
+            e0.record()
+            launches, builds = rr.run()
+            e1.record()
         torch.cuda.synchronize(); barrier()
         wall += time.perf_counter() - t0
         times.append(e0.elapsed_time(e1))
@@ -341,6 +367,11 @@ def run_cuda(args):
     clocks.mark()
     times, launches, n_builds, t_wall = timed_region(rr, W)
     total_ms = statistics.median(times)
+    launch_mode = rr.launch
+    eager_ms = None
+    if launch_mode != "eager":      # the same calls issued one by one from Python, for comparison
+        etimes, _, _, _ = timed_region(rr, 3, min_ms=20.0, graph=False)
+        eager_ms = statistics.median(etimes)
 
     # ---- per-kernel durations of the attention kernels: the same calls again, with an event
     # pair recorded inside the library around each attention kernel (no host sync in between) ----
@@ -590,12 +621,20 @@ def run_cuda(args):
             "protocol": {"replicas": R, "builds_in_timed_region": n_builds, "repeats": len(times),
                          "ms_per_repeat": {"median": round(total_ms, 4), "min": round(min(times), 4),
                                            "max": round(max(times), 4)},
+                         "launch": launch_mode,
                          "how": "each repeat: untimed pass that puts every replica at its place in its block "
                                 "schedule (a build and a step each), barrier + synchronize, K calls (a step each, "
                                 "preceded by the block's build where a replica enters a block: round(K / "
-                                "steps_per_block) builds) between one event pair, synchronize; value = K / median",
+                                "steps_per_block) builds) between one event pair, synchronize; value = K / median. "
+                                "The K calls are captured once into a CUDA graph (the library's own launches in "
+                                "call order, programmatic dependencies included) and each repeat replays it; "
+                                "`eager` is the same region with the calls issued one by one from Python",
                          "step_overlap": "on (inputs resident before the first call)",
                          "engine": "tcgen05" if tc else "simt"},
+            "eager": None if eager_ms is None else {
+                "value": round(world * K / (eager_ms * 1e-3), 1), "unit": UNIT, "step_period_us": round(eager_ms / K * 1e3, 2),
+                "how": "the same K calls issued one by one through the Python binding (two kernel launches per step "
+                       "from the host; bound by the host's enqueue time when that exceeds the step's device time)"},
             "tflops": round(total_flops / (total_ms * 1e-3) / 1e12, 2),
             "full_recompute": {"value": round(fr_value, 1), "unit": UNIT, "step_us": round(fr_ms * 1e3, 2),
                                "kernel_us": round(fr_kernel_ms * 1e3, 2),

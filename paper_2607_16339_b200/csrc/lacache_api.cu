@@ -682,7 +682,7 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
       a.n_ctas_stream = ns;
       if (c->knobs.verbose) {
         static int printed = 0;
-        if (printed++ < 2) fprintf(stderr, "lacache: step plan: %lld stream units (max %d chunks), %lld merge units, %d stream CTAs of %d\n", units_stream, c->max_chunks, units_merge, ns, total);
+        if (printed++ < 16) fprintf(stderr, "lacache: step plan (block %d): %lld stream units (max %d chunks), %lld merge units, %d stream CTAs of %d\n", blk, units_stream, c->max_chunks, units_merge, ns, total);
       }
       a.n_ctas = ns + (int)std::min<long long>(units_merge, std::max(0, c->num_sms - ns));
       {
