@@ -49,6 +49,7 @@ struct lacache_ctx {
     bool no_deep = false;    // LACACHE_NO_DEEP: earlier merge variant
     bool no_qcomp = false;   // LACACHE_NO_QCOMP: no in-kernel rotation of first units
     bool no_pack = false;    // LACACHE_NO_PACK: no head packing of GQA block queries
+    bool no_pair = false;    // LACACHE_NO_PAIR: no paired CTAs (thread-block clusters) for two-chunk block rows
     bool no_chunked_advance = false;  // LACACHE_NO_CHUNKED_ADVANCE: an advance computes the finished block's rows as key-window units
     bool verbose = false;    // LACACHE_VERBOSE: prints the step plan
   } knobs;
@@ -93,7 +94,7 @@ struct lacache_ctx {
   unsigned span_next = 0;
   // the role split of a step is planned once per (block, table size) and reused: a step is called
   // thousands of times per second and the host must stay ahead of the device
-  struct StepPlan { int deep_cap = -1, ns = 0; };
+  struct StepPlan { int deep_cap = -1, ns = 0, pair = -1; };   // pair: every block-row item of the step has two key chunks (-1: not looked at yet)
   std::vector<StepPlan> step_plan;
   int step_overlap = 0;   // consecutive steps may overlap on the device (the caller opts in: a step then reads its inputs early)
   int steps_since_build = 0;
@@ -199,6 +200,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     k.no_deep = getenv("LACACHE_NO_DEEP") != nullptr;
     k.no_qcomp = getenv("LACACHE_NO_QCOMP") != nullptr;
     k.no_pack = getenv("LACACHE_NO_PACK") != nullptr;
+    k.no_pair = getenv("LACACHE_NO_PAIR") != nullptr;
     k.no_chunked_advance = getenv("LACACHE_NO_CHUNKED_ADVANCE") != nullptr;
     k.verbose = getenv("LACACHE_VERBOSE") != nullptr;
   }
@@ -690,6 +692,21 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
         const long long per_cta = n_merge_ctas > 0 ? (units_merge + n_merge_ctas - 1) / n_merge_ctas : 0;
         a.merge_deep = (deep_ok && per_cta <= deep_cap) ? 1 : 0;
         a.split_merge = (deep_ok && per_cta > deep_cap) ? 1 : 0;
+      }
+      // Two key chunks per (sequence, head), one round of block-row units, unpacked heads, one-plane operands:
+      // the two chunks of a head run as a pair of CTAs that merge through distributed shared memory.
+      if (!c->split && a.pack == 1 && a.merge_deep && !a.split_merge && !c->knobs.no_pair && c->g.block_len <= 32 &&
+          units_stream == ns && (ns % 2) == 0 && (a.n_ctas % 2) == 0) {
+        if (plan.pair < 0) {
+          plan.pair = 1;
+          for (int i = 0; i < list.n; ++i)
+            if (c->items_host[list.off + i].pad != 2) plan.pair = 0;
+        }
+        a.pair_chunks = plan.pair;
+      }
+      if (c->knobs.verbose && a.pair_chunks) {
+        static int printed_pair = 0;
+        if (printed_pair++ < 4) fprintf(stderr, "lacache: step plan (block %d): the two key chunks of a head run as a pair of CTAs\n", blk);
       }
     } else {
       a.n_ctas_stream = (int)std::min<long long>(c->num_sms, units_stream);

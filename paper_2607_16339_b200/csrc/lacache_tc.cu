@@ -104,6 +104,11 @@ struct Tile {
 // Q region: in all of it for 128-row units (the next unit's Q load waits for the
 // epilogue), in its upper half for 64-row units (whose Q tile needs only the lower half).
 constexpr uint32_t STAGE_ROW = 512;
+// paired step, one-plane operands: where the partner CTA puts its partial state -- O~ of up to 32 rows in the
+// staging layout (512 bytes a row, 16-byte chunks XOR-swizzled by the row), then (m, l) per row
+constexpr uint32_t SM_RX = Tile<false>::SM_V + 2 * Tile<false>::V_STAGE;
+constexpr uint32_t SM_RX_ML = SM_RX + 32 * STAGE_ROW;
+static_assert(SM_RX_ML + 32 * 8 <= SM_XCH, "no room for the partner's partial state");
 // merge role: the 96 KB after Q hold 2 stages of the block's keys {K hi, K lo, V} of 64
 // rows, then the staging tile of the cached O~ / the output
 constexpr uint32_t SM_KV = SM_K;
@@ -141,10 +146,11 @@ enum {
   BAR_QC,  // stream role: the row threads have written the rotated Q tile of the CTA's first unit
   BAR_IO_FULL1, BAR_OUT_RDY, BAR_OUT_RDY1,  // pipelined merge role: second staging tile; output tile b is complete
   BAR_PAIR,  // 4 barriers: the two warps that share a TMEM lane quadrant
-  N_BARS = BAR_PAIR + 4
+  N_BARS = BAR_PAIR + 4,
+  BAR_RX = BAR_IO_FULL   // stream role of a paired step (it has no staging-tile barriers): the partner's partial state has arrived
 };
 
-enum { EPI_STATE = 0, EPI_OUT = 1, EPI_PARTIAL = 2 };
+enum { EPI_STATE = 0, EPI_OUT = 1, EPI_PARTIAL = 2, EPI_SEND = 3 };   // SEND: the partial state goes to the partner CTA
 
 constexpr long long WAIT_CYCLES = 4000000000ll;  // ~2 s
 
@@ -253,7 +259,12 @@ __device__ __forceinline__ bool wait_bar(const Cta& c, int slot, uint32_t parity
 // What the stream role's templates are instantiated for: a build or a full recompute; a step; a build
 // over key windows (units may start from a stored state and store a snapshot: the incremental rebuild).
 // Separate kernels, so that the plain build and the step carry none of the window code.
-enum StreamKind : int { KIND_BUILD = 0, KIND_STEP = 1, KIND_WINDOW = 2 };
+// KIND_STEP2: a step whose block-row units all have exactly two key chunks, run by the two CTAs of a
+// thread-block cluster: the CTA with the second chunk hands its partial state to its partner through
+// distributed shared memory, and the partner writes the merged rows (one round of units, unpacked heads,
+// one-plane operands: the receiving buffer needs 32 KB that the split planes' tiles leave no room for).
+enum StreamKind : int { KIND_BUILD = 0, KIND_STEP = 1, KIND_WINDOW = 2, KIND_STEP2 = 3 };
+__host__ __device__ constexpr bool kind_is_step(int k) { return k == KIND_STEP || k == KIND_STEP2; }
 
 struct Unit {
   int row0, nrows, h, kh, seq;
@@ -280,6 +291,14 @@ __device__ __forceinline__ bool unit_row_valid(const Unit& un, int r) {
   return un.rh ? ((r >> (un.rh == 64 ? 6 : 5)) < un.nh && (r & (un.rh - 1)) < un.nrows) : r < un.nrows;
 }
 
+// which work item unit u belongs to (units are head-minor; in a paired step unit pair u / 2 is head
+// (u / 2) % Hq of sequence (u / 2) / Hq, and u % 2 its key chunk: a sequence's two chunk items are adjacent)
+template <bool PACKED, int KIND>
+__device__ __forceinline__ int unit_item(const Geometry& g, const AttnArgs& a, int u) {
+  if (KIND == KIND_STEP2) return ((u >> 1) / g.Hq) * 2 + (u & 1);
+  return u / (PACKED ? a.stream_slots : g.Hq);
+}
+
 // PACKED (a.pack > 1): the units are block queries of several heads side by side in one tile.  A template
 // parameter of the whole kernel, so that the kernel a build or an MHA step runs carries none of the per-row
 // head arithmetic: this kernel is sensitive to its code size.
@@ -287,13 +306,13 @@ template <bool PACKED, int KIND, bool SPLIT>
 __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs& a, const WorkItem& it, int u) {
   using TL = Tile<SPLIT>;
   constexpr int BN = TL::BN;
-  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool STEP = kind_is_step(KIND);
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
   Unit un;
   // units are head-minor: unit u = item u / slots of head (or head group) u % slots (a CTA's units, a
   // fixed stride apart, then cycle through the items instead of drawing one item's heads)
-  const int slot = u % (PACKED ? a.stream_slots : g.Hq);
+  const int slot = (KIND == KIND_STEP2 ? (u >> 1) : u) % (PACKED ? a.stream_slots : g.Hq);
   if (PACKED) {
     const int per_kv = (g.group + a.pack - 1) / a.pack;
     un.kh = slot / per_kv;
@@ -353,6 +372,7 @@ __device__ __forceinline__ Unit decode_stream(const Geometry& g, const AttnArgs&
     // (block rows whose result is a state, not normalised rows, always leave partial states: a launch of
     // its own merges them)
     un.epi = (it.pad > 1 || a.blk_to_state) ? EPI_PARTIAL : EPI_OUT;
+    if (KIND == KIND_STEP2) un.epi = it.chunk == 0 ? EPI_OUT : EPI_SEND;   // (every unit has two chunks)
     un.q_rows = un.rh ? BM : 64;
   } else {
     un.epi = EPI_OUT;
@@ -426,12 +446,12 @@ struct TileCursor {
 };
 template <bool PACKED, int KIND, bool SPLIT>
 __device__ __forceinline__ void cursor_load_unit(const Geometry& g, const AttnArgs& a, TileCursor& cu, int n_units) {
-  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool STEP = kind_is_step(KIND);
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
   cu.valid = cu.u < n_units;
   if (!cu.valid) return;
-  cu.it = load_item(a.items + cu.u / (PACKED ? a.stream_slots : g.Hq));
+  cu.it = load_item(a.items + unit_item<PACKED, KIND>(g, a, cu.u));
   cu.un = decode_stream<PACKED, KIND, SPLIT>(g, a, cu.it, cu.u);
   cu.t = cu.un.t0;
   cu.q_done = !cu.loads_q;
@@ -439,7 +459,7 @@ __device__ __forceinline__ void cursor_load_unit(const Geometry& g, const AttnAr
 template <bool PACKED, int KIND, bool SPLIT>
 __device__ __forceinline__ void cursor_advance(const Geometry& g, const AttnArgs& a, TileCursor& cu, int stride,
                                                int n_units) {
-  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool STEP = kind_is_step(KIND);
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
   // move to the next tile; cross into the next unit(s) when this one is exhausted
@@ -460,7 +480,7 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
   using TL = Tile<SPLIT>;
   constexpr int BN = TL::BN;
   constexpr uint32_t KS_BOX = TL::KS_BOX, K_STAGE = TL::K_STAGE, SM_V = TL::SM_V, V_STAGE = TL::V_STAGE;
-  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool STEP = kind_is_step(KIND);
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
   // three independent cursors: Q tiles (one per unit), key tiles, value tiles
@@ -571,7 +591,7 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   using TL = Tile<SPLIT>;
   constexpr int BN = TL::BN;
   constexpr uint32_t KS_BOX = TL::KS_BOX, K_STAGE = TL::K_STAGE, SK_LO = TL::SK_LO;
-  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool STEP = kind_is_step(KIND);
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
   // (operand format of the score product: bf16 planes, or fp16 in the one-plane fp16 mode)
@@ -580,7 +600,7 @@ __device__ void stream_mma_scores(const Cta& c, const Geometry& g, const AttnArg
   uint32_t js = 0;  // score tiles issued so far (stage and buffer = js & 1, phase = (js >> 1) & 1)
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
+    if (u + stride < n_units) nxt = load_item(a.items + unit_item<PACKED, KIND>(g, a, u + stride));
     const Unit un = decode_stream<PACKED, KIND, SPLIT>(g, a, it, u);
     const uint32_t q_box = (uint32_t)un.q_rows * 128u;
     const int n_tiles = un.t1 - un.t0;
@@ -609,14 +629,14 @@ __device__ void stream_mma_pv(const Cta& c, const Geometry& g, const AttnArgs& a
   using TL = Tile<SPLIT>;
   constexpr int BN = TL::BN;
   constexpr uint32_t KS_BOX = TL::KS_BOX, SM_V = TL::SM_V, V_STAGE = TL::V_STAGE;
-  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool STEP = kind_is_step(KIND);
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
   int uu = 0;
   uint32_t jp = 0;  // P~V tiles issued so far
   for (int u = first; u < n_units; u += stride, ++uu) {
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
+    if (u + stride < n_units) nxt = load_item(a.items + unit_item<PACKED, KIND>(g, a, u + stride));
     const Unit un = decode_stream<PACKED, KIND, SPLIT>(g, a, it, u);
     const int n_tiles = un.t1 - un.t0;
     // O~ of the previous unit has been read by the row threads.  (A unit without key tiles issues nothing
@@ -782,7 +802,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
   using TL = Tile<SPLIT>;
   constexpr int BN = TL::BN;
   constexpr int HC = TL::HC;
-  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool STEP = kind_is_step(KIND);
   constexpr bool WINDOW = KIND == KIND_WINDOW;
   (void)WINDOW;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -798,7 +818,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
   for (int u = first; u < n_units; u += stride) {
     ++uu;
     WorkItem nxt = it;
-    if (u + stride < n_units) nxt = load_item(a.items + (u + stride) / (PACKED ? a.stream_slots : g.Hq));
+    if (u + stride < n_units) nxt = load_item(a.items + unit_item<PACKED, KIND>(g, a, u + stride));
     const Unit un = decode_stream<PACKED, KIND, SPLIT>(g, a, it, u);
     it = nxt;
     if (u == first && STEP && a.q_raw != nullptr) {
@@ -1072,7 +1092,71 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
     lx[half] = l_part;
     if (!epi_sync(c, epi_phase)) return;
     const float l_run = lx[0] + lx[1];
-    const float mul = (un.epi == EPI_OUT) ? 1.f / l_run : 1.f;
+    float mul = (un.epi == EPI_OUT) ? 1.f / l_run : 1.f;
+    float mul_rx = 0.f, lse2 = 0.f;   // paired step: weight of the partner's O~, merged log2 normaliser
+    if (KIND == KIND_STEP2) {
+      const uint32_t rx_row = SM_RX + (uint32_t)r * STAGE_ROW;
+      if (un.epi == EPI_SEND) {
+        // Second key chunk of its (sequence, head): O~ of the block's rows from TMEM into the partner CTA's
+        // receiving buffer (the layout of a staging tile), m and l behind it, then one arrival per thread on
+        // the partner's barrier -- the release that makes the stores visible to its acquiring wait.
+        const uint32_t peer = cluster_ctarank() ^ 1u;
+        const uint32_t dst = mapa_shared(c.base + rx_row, peer);
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t rr[16];
+          if (!first_tile) {
+            tmem_ld16(tlane + TS_O + 64 * half + 16 * cb, rr);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) rr[j] = 0u;
+          }
+          if (row_valid) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int ch = 16 * half + 4 * cb + i;
+              st_cluster_v4(dst + ((ch ^ (r & 7)) << 4), __uint_as_float(rr[4 * i]), __uint_as_float(rr[4 * i + 1]),
+                            __uint_as_float(rr[4 * i + 2]), __uint_as_float(rr[4 * i + 3]));
+            }
+          }
+        }
+        if (row_valid && half == 0) st_cluster_v2(mapa_shared(c.base + SM_RX_ML + (uint32_t)r * 8u, peer), m_ref, l_run);
+        mbar_arrive_cluster(mapa_shared(c.bar(BAR_RX), peer));
+        tc_fence_before();
+        mbar_arrive(c.bar(BAR_O_FREE));  // (a paired step has one unit per CTA; kept for the barrier's phase count)
+        continue;
+      }
+      // First key chunk: wait (bounded) for the partner's partial state, then merge the two states of the row
+      // (Eq. 2-6) into the weights of the two O~ rows; the rows leave through the ordinary output epilogue.
+      {
+        const uint32_t bar = c.bar(BAR_RX);
+        const long long t0 = clock64();
+        while (!mbar_try_acquire_cluster(bar, 0u)) {
+          if (*c.abort_flag) return;
+          if (clock64() - t0 > WAIT_CYCLES) {
+            *c.abort_flag = 1;
+            if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
+              c.status[1] = LOC_WAIT_O; c.status[2] = blockIdx.x; c.status[3] = threadIdx.x;
+            }
+            return;
+          }
+        }
+      }
+      float m2 = -INFINITY, l2 = 0.f;
+      if (row_valid) {
+        const float2 ml = *reinterpret_cast<const float2*>(c.gen + SM_RX_ML + r * 8);
+        m2 = ml.x; l2 = ml.y;
+      }
+      const float M = fmaxf(m_ref, m2);
+      const float w1 = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - M);
+      const float w2 = (m2 == -INFINITY) ? 0.f : ex2(m2 - M);
+      const float L = fmaf(l_run, w1, l2 * w2);
+      const float inv = 1.f / L;
+      mul = w1 * inv;
+      mul_rx = w2 * inv;
+      lse2 = M + log2f(L);
+    }
     if (un.epi == EPI_PARTIAL) {
       // Partial state of this key chunk, straight from TMEM to global memory (each
       // thread 256 contiguous bytes of its row); the last chunk of the (sequence,
@@ -1193,9 +1277,14 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int ch = 16 * half + 4 * cb + i;
-          *reinterpret_cast<float4*>(srow + ((ch ^ (r & 7)) << 4)) =
-              make_float4(__uint_as_float(rr[4 * i]) * mul, __uint_as_float(rr[4 * i + 1]) * mul,
-                          __uint_as_float(rr[4 * i + 2]) * mul, __uint_as_float(rr[4 * i + 3]) * mul);
+          float4 v = make_float4(__uint_as_float(rr[4 * i]) * mul, __uint_as_float(rr[4 * i + 1]) * mul,
+                                 __uint_as_float(rr[4 * i + 2]) * mul, __uint_as_float(rr[4 * i + 3]) * mul);
+          if (KIND == KIND_STEP2 && row_valid) {   // + the partner chunk's O~, weighted
+            const float4 p = *reinterpret_cast<const float4*>(c.gen + SM_RX + r * STAGE_ROW + ((ch ^ (r & 7)) << 4));
+            v.x = fmaf(p.x, mul_rx, v.x); v.y = fmaf(p.y, mul_rx, v.y);
+            v.z = fmaf(p.z, mul_rx, v.z); v.w = fmaf(p.w, mul_rx, v.w);
+          }
+          *reinterpret_cast<float4*>(srow + ((ch ^ (r & 7)) << 4)) = v;
         }
       }
     }
@@ -1208,7 +1297,7 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       coop_store_rows(c, stage_off, a.st.o + ((size_t)un.h * g.Tp + un.row0) * D, D, un.nrows);
     } else if (un.epi == EPI_OUT) {
       const size_t orow = (size_t)row * g.Hq + hrow;
-      if (row_valid && half == 0 && a.lse) a.lse[orow] = (m_ref + log2f(l_run)) * LN2;
+      if (row_valid && half == 0 && a.lse) a.lse[orow] = (KIND == KIND_STEP2 ? lse2 : m_ref + log2f(l_run)) * LN2;
       if (!epi_sync(c, epi_phase)) return;
       for (int j = 0; j < un.nh; ++j)   // one head's rows at a time (a single head unless block queries are packed)
         coop_store_out_rows(c, a, stage_off + (uint32_t)(j * un.rh) * STAGE_ROW, ((size_t)un.row0 * g.Hq + un.h + j) * D,
@@ -1793,7 +1882,7 @@ __device__ void deep_rows(const Cta& c, const Geometry& g, const AttnArgs& a, in
 template <bool PACKED, int KIND, bool DEEP, bool SPLIT>
 __global__ void __launch_bounds__(THREADS, 1)
 tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const AttnArgs a) {
-  constexpr bool STEP = KIND == KIND_STEP;
+  constexpr bool STEP = kind_is_step(KIND);
   // (PACKED: the steps of a GQA model whose block queries share tiles across heads, see decode_stream;
   // KIND: see StreamKind; DEEP: which variant of the merge role a step runs)
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -1836,7 +1925,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   }
   const int n_my = first < n_units ? (n_units - first + stride - 1) / stride : 0;
   WorkItem it0{};
-  if (!deep && first < n_units) it0 = stream ? load_item(a.items + first / (PACKED ? a.stream_slots : g.Hq))
+  if (!deep && first < n_units) it0 = stream ? load_item(a.items + unit_item<PACKED, KIND>(g, a, first))
                                              : load_item(a.items_merge + first / g.Hq);
   if ((c.base & 1023u) != 0) {  // swizzled tiles need a 1024-byte aligned base
     if (tid == 0 && atomicCAS(a.status, 0, (int)LACACHE_ERR_CUDA) == 0) a.status[1] = LOC_SMEM_ALIGN;
@@ -1854,6 +1943,7 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
         count = ROW_THREADS;
       if (i == BAR_DONE) count = THREADS;
       if (i == BAR_Q_FREE && stream) count = 2;  // score MMAs done + epilogue staging read
+      if (KIND == KIND_STEP2 && i == BAR_RX && stream) count = ROW_THREADS;  // the partner's row threads
       if (i >= BAR_PAIR) count = 64;
       mbar_init(c.bar(i), count);
     }
@@ -1883,6 +1973,9 @@ tc_attn_kernel(const __grid_constant__ TcMaps maps, const Geometry g, const Attn
   __syncthreads();
   tc_fence_after();
   c.tmem = words[0];
+  // (paired step: nobody writes into the partner's shared memory or arrives on its barrier before the
+  // partner has initialised them)
+  if (KIND == KIND_STEP2) cluster_sync_all();
 
   if (warp == 0) {
     if (stream) {
@@ -2017,10 +2110,12 @@ namespace {
 // step of an MHA and of a GQA model, each with either variant of the merge role}
 template <bool SPLIT>
 const void* const* kernel_table() {
-  static const void* const t[6] = {
+  // (the paired step exists for one-plane operands only: with split planes the entry repeats the ordinary step)
+  static const void* const t[7] = {
       (const void*)tc_attn_kernel<false, KIND_BUILD, false, SPLIT>, (const void*)tc_attn_kernel<false, KIND_WINDOW, false, SPLIT>,
       (const void*)tc_attn_kernel<false, KIND_STEP, false, SPLIT>,  (const void*)tc_attn_kernel<false, KIND_STEP, true, SPLIT>,
-      (const void*)tc_attn_kernel<true, KIND_STEP, false, SPLIT>,   (const void*)tc_attn_kernel<true, KIND_STEP, true, SPLIT>};
+      (const void*)tc_attn_kernel<true, KIND_STEP, false, SPLIT>,   (const void*)tc_attn_kernel<true, KIND_STEP, true, SPLIT>,
+      (const void*)tc_attn_kernel<false, SPLIT ? KIND_STEP : KIND_STEP2, true, SPLIT>};
   return t;
 }
 }  // namespace
@@ -2028,7 +2123,7 @@ const void* const* kernel_table() {
 cudaError_t tc_prepare() {
   for (int split = 0; split < 2; ++split) {
     const void* const* t = split ? kernel_table<true>() : kernel_table<false>();
-    for (int i = 0; i < 6; ++i) {
+    for (int i = 0; i < 7; ++i) {
       cudaError_t e = cudaFuncSetAttribute(t[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM_TOTAL);
       if (e != cudaSuccess) return e;
     }
@@ -2081,14 +2176,27 @@ cudaError_t tc_attention(const Geometry& g, const AttnArgs& a, const TcMaps* map
   cfg.blockDim = dim3(THREADS);
   cfg.dynamicSmemBytes = SM_TOTAL;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  int n_attr = 0;
+  if (!a.no_pdl) {
+    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+    ++n_attr;
+  }
+  const bool paired = a.mode == MODE_STEP && a.pair_chunks && !a.split;
+  if (paired) {   // CTAs 2k and 2k + 1 form a cluster: the two key chunks of one (sequence, head)
+    attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+    attr[n_attr].val.clusterDim.x = 2;
+    attr[n_attr].val.clusterDim.y = 1;
+    attr[n_attr].val.clusterDim.z = 1;
+    ++n_attr;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = a.no_pdl ? 0 : 1;
+  cfg.numAttrs = n_attr;
   const void* const* t = a.split ? kernel_table<true>() : kernel_table<false>();
   int which;
   if (a.mode != MODE_STEP) which = a.window ? 1 : 0;
+  else if (paired) which = 6;
   else which = (a.pack > 1 ? 4 : 2) + (a.merge_deep ? 1 : 0);
   void* params[3] = {const_cast<TcMaps*>(maps), const_cast<Geometry*>(&g), const_cast<AttnArgs*>(&a)};
   return cudaLaunchKernelExC(&cfg, t[which], params);

@@ -328,6 +328,41 @@ def test_packed_block_rows_several_units_per_cta(hq, hkv, block_len, monkeypatch
     monkeypatch.delenv("LACACHE_STREAM_CTAS")
 
 
+@pytest.mark.parametrize("mode", ["fp16", "plain"])
+@pytest.mark.parametrize("block_len", [16, 32])
+def test_two_key_chunks_as_a_pair_of_ctas(mode, block_len, monkeypatch):
+    """With one-plane operands, unpacked heads, one round of block-row units and exactly two key chunks per
+    (sequence, head), the two chunks run as a thread-block cluster of two CTAs: the second hands its partial
+    state to the first through distributed shared memory, and the first writes the merged rows.  Forced here
+    by the chunk size and the role split; the same cases with the pairing switched off must agree within the
+    tolerance between two orders of the same merge, and both with the oracle."""
+    kw = dict(prompt_lens=(150, 180, 130), gen_len=2 * block_len, block_len=block_len, steps=2, hq=4, hkv=4)
+    if mode == "plain":
+        kw["scale_mode"] = "inv_sqrt_d"
+    wl = small_workload(name="pair-%s-%d" % (mode, block_len), dtype="bf16", d=128, **kw)
+    units = wl.batch * 2 * wl.n_q_heads
+    monkeypatch.setenv("LACACHE_STREAM_CTAS", str(units))      # (experiment knobs are read when a context is created)
+    outs = {}
+    for pair in (True, False):
+        if not pair:
+            monkeypatch.setenv("LACACHE_NO_PAIR", "1")
+        _run_points(wl, "tc", seed=12, precision_mode=_MODES[mode], sc_tiles_per_chunk=1)
+        sch = SyntheticSchedule(wl, seed=12)
+        ctx = make_ctx(wl, engine=ENGINES["tc"], precision_mode=_MODES[mode], sc_tiles_per_chunk=1)
+        q, k, v = (to_dev(a, wl) for a in advance_to_block(sch, 1))
+        ctx.build(1, q, k, v)
+        out, lse = new_outputs(wl)
+        ctx.step(*(to_dev(a, wl) for a in sch.draw_step(1, 1)), out, lse)
+        torch.cuda.synchronize()
+        assert ctx.poll_status()[0] == 0
+        outs[pair] = (out.clone(), lse.clone())
+        ctx.destroy()
+    monkeypatch.delenv("LACACHE_NO_PAIR")
+    monkeypatch.delenv("LACACHE_STREAM_CTAS")
+    assert (outs[True][0] - outs[False][0]).abs().max().item() <= 1e-5
+    assert (outs[True][1] - outs[False][1]).abs().max().item() <= 1e-5
+
+
 @pytest.mark.parametrize("cfg", [3, 4])
 def test_step_split_over_several_launches(cfg, monkeypatch):
     """A step with more fixed-row tiles per CTA than the pipelined merge variant tabulates goes out in
