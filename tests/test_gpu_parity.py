@@ -227,7 +227,7 @@ _MHA64 = small_workload(name="mha64", prompt_lens=(700, 333, 61), gen_len=192, b
                         scale_mode="per_head_u(0.5,2)")
 
 
-@pytest.mark.parametrize("cfg", [2, 4, 5, "mha64"])
+@pytest.mark.parametrize("cfg", [2, 4, 5, "mha64", "2-fp16", "4-fp16"])
 @pytest.mark.parametrize("overlap", [True, False])
 def test_back_to_back_steps_match_synchronised_steps(cfg, overlap):
     """With the overlap of consecutive steps switched on (precomputed inputs), the next step's kernels
@@ -235,6 +235,10 @@ def test_back_to_back_steps_match_synchronised_steps(cfg, overlap):
     without any host synchronisation must give, bit for bit, what the same calls give when the host
     waits after each one -- with a separate output buffer per step and with one reused; likewise with
     the default, plain stream order."""
+    # ("-fp16": one fp16 plane per operand; at config 2 the step then runs its two key chunks as pairs of CTAs)
+    mode = binding.PRECISION_SPLIT
+    if isinstance(cfg, str) and cfg.endswith("-fp16"):
+        cfg, mode = int(cfg[0]), binding.PRECISION_FP16
     wl = _MHA64 if cfg == "mha64" else WORKLOADS[cfg]
     S = min(wl.steps_per_block, 6)
     calls = []   # ("build", blk, q, k, v) / ("step", qb, kb, vb)
@@ -248,7 +252,7 @@ def test_back_to_back_steps_match_synchronised_steps(cfg, overlap):
     n_steps = sum(1 for c in calls if c[0] == "step")
 
     def run(sync, one_buffer):
-        ctx = make_ctx(wl, engine=ENGINES["tc"])
+        ctx = make_ctx(wl, engine=ENGINES["tc"], precision_mode=mode)
         ctx.set_step_overlap(overlap)
         bufs = [new_outputs(wl) for _ in range(1 if one_buffer else n_steps)]
         res, i = [], 0
