@@ -49,6 +49,7 @@ struct lacache_ctx {
     bool no_deep = false;    // LACACHE_NO_DEEP: earlier merge variant
     bool no_qcomp = false;   // LACACHE_NO_QCOMP: no in-kernel rotation of first units
     bool no_pack = false;    // LACACHE_NO_PACK: no head packing of GQA block queries
+    bool no_staged_state = false;   // LACACHE_NO_STAGED_STATE: builds store the cached state from the row threads
     bool no_pair = false;    // LACACHE_NO_PAIR: no paired CTAs (thread-block clusters) for two-chunk block rows
     bool no_chunked_advance = false;  // LACACHE_NO_CHUNKED_ADVANCE: an advance computes the finished block's rows as key-window units
     bool verbose = false;    // LACACHE_VERBOSE: prints the step plan
@@ -201,6 +202,7 @@ lacache_status create_impl(const lacache_config* cfg, lacache_ctx* c) {
     k.no_qcomp = getenv("LACACHE_NO_QCOMP") != nullptr;
     k.no_pack = getenv("LACACHE_NO_PACK") != nullptr;
     k.no_pair = getenv("LACACHE_NO_PAIR") != nullptr;
+    k.no_staged_state = getenv("LACACHE_NO_STAGED_STATE") != nullptr;
     k.no_chunked_advance = getenv("LACACHE_NO_CHUNKED_ADVANCE") != nullptr;
     k.verbose = getenv("LACACHE_VERBOSE") != nullptr;
   }
@@ -711,6 +713,8 @@ AttnArgs attn_args(lacache_ctx* c, int mode, lacache_ctx::ListRef list, int blk,
     } else {
       a.n_ctas_stream = (int)std::min<long long>(c->num_sms, units_stream);
       a.n_ctas = a.n_ctas_stream;
+      // (a plain build writes the cached state itself: the buffer the tensor map of the state describes)
+      a.st_tma = (mode == MODE_BUILD && !c->split && !c->knobs.no_staged_state) ? 1 : 0;
     }
   }
   return a;

@@ -133,6 +133,8 @@ struct AttnArgs {
   int32_t* status;
   int blk_to_state;          // block-row units write the merged state (m, l, O~) of their rows to `st` instead
                              // of normalised rows to `out` (first launch of an incremental advance)
+  int st_tma;                // build: `st.o` is the buffer the cached-state tensor map was encoded for, so full row tiles
+                             // may leave through bulk tensor stores (one-plane operands)
   int pair_chunks;           // host only: a step whose block-row units all have two key chunks, as pairs of CTAs
                              // (thread-block clusters of two) that merge through distributed shared memory
   int no_pdl;                // host only: launch the ordinary way (experiment knob)

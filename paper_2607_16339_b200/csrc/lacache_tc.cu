@@ -109,6 +109,11 @@ constexpr uint32_t STAGE_ROW = 512;
 constexpr uint32_t SM_RX = Tile<false>::SM_V + 2 * Tile<false>::V_STAGE;
 constexpr uint32_t SM_RX_ML = SM_RX + 32 * STAGE_ROW;
 static_assert(SM_RX_ML + 32 * 8 <= SM_XCH, "no room for the partner's partial state");
+// build, one-plane operands: staging of a unit's cached O~ tile for bulk tensor stores, four swizzled boxes of
+// 32 features x 128 rows -- two in the upper half of the Q region (a one-plane Q tile needs the lower half),
+// two in the 32 KB behind the value stages
+__host__ __device__ constexpr uint32_t st_box(int cb) { return cb < 2 ? SM_Q + 32768u + (uint32_t)cb * 16384u : SM_RX + (uint32_t)(cb - 2) * 16384u; }
+static_assert(SM_RX + 2 * 16384u <= SM_XCH, "no room for the state staging tile");
 // merge role: the 96 KB after Q hold 2 stages of the block's keys {K hi, K lo, V} of 64
 // rows, then the staging tile of the cached O~ / the output
 constexpr uint32_t SM_KV = SM_K;
@@ -147,7 +152,9 @@ enum {
   BAR_IO_FULL1, BAR_OUT_RDY, BAR_OUT_RDY1,  // pipelined merge role: second staging tile; output tile b is complete
   BAR_PAIR,  // 4 barriers: the two warps that share a TMEM lane quadrant
   N_BARS = BAR_PAIR + 4,
-  BAR_RX = BAR_IO_FULL   // stream role of a paired step (it has no staging-tile barriers): the partner's partial state has arrived
+  BAR_RX = BAR_IO_FULL,  // stream role of a paired step (it has no staging-tile barriers): the partner's partial state has arrived
+  // stream role of a build with one-plane operands: a unit's state tile is staged / its bulk store has read the staging
+  BAR_ST_RDY = BAR_OUT_RDY, BAR_ST_FREE = BAR_IO_FREE
 };
 
 enum { EPI_STATE = 0, EPI_OUT = 1, EPI_PARTIAL = 2, EPI_SEND = 3 };   // SEND: the partial state goes to the partner CTA
@@ -498,6 +505,12 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
   // that overlap the block -- so tiles of fixed tokens are requested at once and
   // the wait comes only when nothing else can be issued.
   bool dep_done = false;
+  // build with one-plane operands: full row tiles leave as bulk tensor stores from a staging tile the row
+  // threads fill (units in the order of the Q loads; at most two are between their Q load and their store)
+  constexpr bool STAGED = KIND == KIND_BUILD && !SPLIT;
+  int st_slot0 = 0, st_slot1 = 0;   // row0 | head << 24 of the (at most two) units between their Q load and their store
+  int st_head = 0, st_tail = 0;
+  bool st_pending = false;
   const bool q_computed = STEP && a.q_raw != nullptr;
   auto tile_depends = [&](const TileCursor& cu) {
     if (!STEP) return true;
@@ -505,8 +518,22 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
     return krow < cu.it.blk_start + g.block_len && krow + BN > cu.it.blk_start;
   };
   long long t_idle = 0;
-  while (cq.valid || ck.valid || cv.valid) {
+  while (cq.valid || ck.valid || cv.valid || (STAGED && (st_head < st_tail || st_pending))) {
     bool did = false, blocked_on_dep = false;
+    if (STAGED && st_head < st_tail && mbar_test(c.bar(BAR_ST_RDY), st_head & 1)) {
+      // (dep_done: the unit's Q tile was loaded after the wait for the preceding grids, so no store precedes it)
+      const int sv = (st_head & 1) ? st_slot1 : st_slot0;
+      if (sv >= 0) {
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) tma_store_3d(&maps.st_o, c.base + st_box(cb), 32 * cb, sv & 0xFFFFFF, sv >> 24);
+        bulk_commit();
+        st_pending = true;
+      } else {
+        mbar_arrive(c.bar(BAR_ST_FREE));
+      }
+      ++st_head;
+      did = true;
+    }
     if (cq.valid) {  // a unit without key tiles still needs its Q load (the MMA thread waits for it)
       if (cq.uu == 0 && q_computed) {
         // the row threads rotate this tile from the raw queries: nothing to load,
@@ -520,6 +547,11 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
         blocked_on_dep = true;
       } else if (cq.uu == 0 || mbar_test(c.bar(BAR_Q_FREE), (cq.uu - 1) & 1)) {
         load_q_tile<SPLIT>(c, maps, cq.un.q_rows, cq.un.row0, cq.un.h, cq.un.rh != 0);
+        if (STAGED && a.st_tma && cq.un.epi == EPI_STATE) {
+          const int sv = cq.un.row0 | (cq.un.h << 24) | (cq.un.nrows == BM ? 0 : (int)0x80000000u);   // (top bit: a clipped tile, nothing staged)
+          if (st_tail & 1) st_slot1 = sv; else st_slot0 = sv;
+          ++st_tail;
+        }
         cq.q_done = true;
         cq.t = cq.un.t1;
         cursor_advance<PACKED, KIND, SPLIT>(g, a, cq, stride, n_units);
@@ -561,20 +593,27 @@ __device__ void stream_producer(const Cta& c, const TcMaps& maps, const Geometry
       dep_done = true;
       did = true;
     }
+    if (STAGED && !did && st_pending) {   // nothing else to issue: the last store has read its staging tile by now
+      bulk_wait_read();
+      mbar_arrive(c.bar(BAR_ST_FREE));
+      st_pending = false;
+      did = true;
+    }
     if (did) {
       t_idle = 0;
     } else {  // nothing free: bounded idle
       if (t_idle == 0) t_idle = clock64();
-      if (*c.abort_flag) return;
+      if (*c.abort_flag) break;
       if (clock64() - t_idle > WAIT_CYCLES) {
         *c.abort_flag = 1;
         if (atomicCAS(c.status, 0, (int)LACACHE_ERR_TIMEOUT) == 0) {
           c.status[1] = LOC_WAIT_K; c.status[2] = blockIdx.x; c.status[3] = threadIdx.x;
         }
-        return;
+        break;
       }
     }
   }
+  if (STAGED) bulk_wait_read();  // shared memory stays valid until the last store has read it
   // (a CTA without units never touches memory the RoPE kernel writes)
 }
 
@@ -1219,6 +1258,47 @@ __device__ void stream_rows(const Cta& c, const Geometry& g, const AttnArgs& a, 
       if (!epi_sync(c, epi_phase)) return;  // the flag may be rewritten
       if (un.q_rows == BM && threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));
       continue;
+    }
+    if (KIND == KIND_BUILD && !SPLIT && un.epi == EPI_STATE && a.st_tma) {
+      // Build with one-plane operands: the state of a full row tile goes to a staging tile (four swizzled
+      // boxes outside the Q tile and the key / value stages) and leaves as bulk tensor stores issued by the
+      // producer thread, so these threads are back at the next unit's tiles after 16 shared-memory stores
+      // each instead of eight 32-byte global stores that touch 32 different lines per warp instruction.
+      // Every unit takes part in the hand-over (a clipped tile stores the old way and hands over nothing),
+      // so the barriers' phases follow the unit count.
+      if (uu >= 1 && !wait_bar(c, BAR_ST_FREE, (uu - 1) & 1, LOC_WAIT_O)) return;  // the previous store has read the tile
+      if (un.nrows == BM) {
+        if (threadIdx.x == 64) mbar_arrive(c.bar(BAR_Q_FREE));
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {     // sixteen features at a time: half a box row
+          uint32_t rr[16];
+          if (!first_tile) {
+            tmem_ld16(tlane + TS_O + 64 * half + 16 * cb, rr);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) rr[j] = 0u;
+          }
+          uint8_t* const sb = c.gen + st_box(2 * half + (cb >> 1)) + r * 128;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int ch = 4 * (cb & 1) + i;
+            *reinterpret_cast<float4*>(sb + ((ch ^ (r & 7)) << 4)) =
+                make_float4(__uint_as_float(rr[4 * i]), __uint_as_float(rr[4 * i + 1]), __uint_as_float(rr[4 * i + 2]),
+                            __uint_as_float(rr[4 * i + 3]));
+          }
+        }
+        if (half == 0) {
+          const size_t srow = (size_t)un.h * g.Tp + row;
+          a.st.m[srow] = m_ref; a.st.l[srow] = l_run;
+        }
+        fence_async_smem();   // the bulk stores read the tile through the async proxy
+        mbar_arrive(c.bar(BAR_ST_RDY));
+        tc_fence_before();
+        mbar_arrive(c.bar(BAR_O_FREE));  // the next unit may overwrite O~
+        continue;
+      }
+      mbar_arrive(c.bar(BAR_ST_RDY));   // (nothing staged: the producer answers at once)
     }
     if (un.epi == EPI_STATE && un.q_rows == BM) {
       // Cached state of a build unit, straight from TMEM to global memory (each thread 256
