@@ -2186,7 +2186,7 @@ bool make_v_map(CUtensorMap* m, void* base, int H, int Tp, int box_rows, char* e
 }  // namespace
 
 namespace {
-// twelve instantiations: {split, plain operands} x {build / full recompute; build over key windows; the
+// thirteen instantiations: {split planes, one plane per operand} x {build / full recompute; build over key windows; the
 // step of an MHA and of a GQA model, each with either variant of the merge role}
 template <bool SPLIT>
 const void* const* kernel_table() {
