@@ -1714,10 +1714,12 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
   };
   // Q' and cached O~ of fixed rows do not depend on the RoPE kernel launched
   // just before this one; the block's keys and values do
+  // (the second unit's cached-O~ tile is requested once the first Q' tile has landed, not with it: at the start
+  // of a step every CTA's requests queue in front of HBM, and the tile that is needed last gives way)
   load_q(0);
   load_io(0);
-  if (n_my > 1) load_io(1);
   bool dep_done = false;
+  bool q0_landed = false;   // (latched: the barrier's parity comes round again)
   if (kv_computed) {
     // the row threads rotate / convert the block's keys and values of the first unit
     // from the raw inputs (plain arrivals keep the barriers' phase counts in step)
@@ -1729,7 +1731,7 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
     load_k(0);
     load_v(0);
   }
-  int qu = 1, ku = 1, vu = 1, iu = 2, su = 0;
+  int qu = 1, ku = 1, vu = 1, iu = 1, su = 0;
   bool pending_read = false;  // an output store may still be reading its staging tile
   long long t_idle = 0;
   while (su < n_my) {
@@ -1753,7 +1755,8 @@ __device__ void deep_producer(const Cta& c, const TcMaps& maps, const Geometry& 
       ++su;
       did = true;
     }
-    if (!did && iu < n_my && su > iu - 2) {  // the tile of unit iu - 2 has been handed to its store
+    if (!q0_landed && mbar_test(c.bar(BAR_Q_FULL), 0)) q0_landed = true;
+    if (!did && iu < n_my && su > iu - 2 && q0_landed) {  // the tile of unit iu - 2 has been handed to its store
       if (pending_read) { bulk_wait_read(); pending_read = false; }
       load_io(iu);
       ++iu;
