@@ -974,7 +974,7 @@ def token_path_leg(wl, dev, peaks, seed, n_steps, precision):
 # kernel ends, so the figure is dominated by reads.
 DEFAULT_PRECISION = {1: 1, 2: 3, 3: 1, 4: 3, 5: 3, 6: 3}   # binding.PRECISION_*: 1 = split bf16 planes, 3 = one fp16 plane
 TRAFFIC_PER_LAUNCH = {(2, 1): 48370432, (3, 1): 93736960, (4, 1): 460605952, (5, 1): 209015552, (5, 0): 161659392,
-                      (2, 3): 34915328, (4, 3): 345821952, (5, 3): 161281536}   # (config, precision mode)
+                      (2, 3): 34980608, (4, 3): 345821952, (5, 3): 161281536}   # (config, precision mode)
 
 
 # ----------------------------------------------------------------------------
